@@ -1,0 +1,185 @@
+/*
+ * matkv.h -- C ABI of the B200 (sm_100a) attention path that remains on the GPU
+ * in MatKV-style retrieval-augmented inference.
+ *
+ * Method (paper, Section III-A and Section IV): the K,V tensors of every
+ * document chunk are computed once, each chunk alone with its tokens at
+ * positions 0..len-1, stored under a chunk id, and at request time loaded
+ * instead of recomputed and placed BEFORE the query.  Only the query suffix
+ * (the "sub-prefill" after loading) and the generated tokens attend to them.
+ * This library computes that attention directly over the scattered chunk
+ * buffers: no concatenated copy is ever made.
+ *
+ * Conventions
+ *   - every function returns MATKV_OK (0) or a negative MATKV_E_* code and never
+ *     throws; matkv_last_error() gives a thread-local text for the last failure;
+ *   - "device" pointers are CUDA device memory of the context's GPU, "host"
+ *     pointers are ordinary or pinned host memory, as stated per argument;
+ *   - streams are cudaStream_t passed as void* (NULL = the legacy default stream);
+ *   - all attend / stage / table calls are asynchronous on the given stream and
+ *     validate their arguments on the host before anything is launched;
+ *   - the library allocates only small tables; chunk blobs, slots, tails,
+ *     workspace, queries and outputs are owned by the caller and BORROWED;
+ *   - problems only the device can see (a bounds check, a bounded wait that ran
+ *     out) are written to a device status word, read with matkv_status();
+ *   - one context serves one stream of attend calls at a time (they share the
+ *     workspace); calls from several host threads on one context must be
+ *     serialised by the caller.
+ *
+ * Data layouts (bf16 = 2-byte bfloat16, fp32 accumulation everywhere)
+ *   chunk blob   [n_layers][2 (K, then V)][n_kv_heads][n_tokens][head_dim] bf16,
+ *                contiguous, base 256-byte aligned.  K is stored as the model
+ *                produced it (already rotated for positions 0..n_tokens-1) and is
+ *                never modified or re-rotated.
+ *   tail         [batch][n_layers][n_kv_heads][max_tail_tokens][head_dim] bf16, one
+ *                buffer for K and one for V: the K,V of the query suffix and of the
+ *                generated tokens.  Must not hold NaN/Inf bit patterns (zero it once).
+ *   grouped-query attention: query head h reads KV head floor(h / G), G = Hq / Hkv.
+ */
+#ifndef MATKV_H
+#define MATKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MATKV_OK               0
+#define MATKV_E_INVALID_ARG   (-1)
+#define MATKV_E_UNKNOWN_CHUNK (-2)
+#define MATKV_E_NOT_STAGED    (-3)  /* chunk has no device copy (never staged or evicted)   */
+#define MATKV_E_NOT_READY     (-4)  /* an asynchronous copy has not finished yet             */
+#define MATKV_E_CAPACITY      (-5)  /* too many chunks / slots / tail tokens / batch          */
+#define MATKV_E_ALIGNMENT     (-6)
+#define MATKV_E_CUDA          (-7)
+#define MATKV_E_TIMEOUT       (-8)  /* device status: a bounded wait inside a kernel ran out */
+#define MATKV_E_BOUNDS        (-9)  /* device status: a table-derived index was out of range */
+
+typedef struct matkv_ctx matkv_ctx;     /* opaque; owned by the library            */
+typedef struct matkv_table matkv_table; /* opaque; one per in-flight request batch */
+
+typedef struct {
+    int32_t n_layers, n_q_heads, n_kv_heads;
+    int32_t head_dim;            /* 64 or 128                                               */
+    int32_t max_batch;           /* requests per table, 1..1024                             */
+    int32_t max_chunks_per_req;  /* upper bound on a request's chunk list                   */
+    int32_t max_tail_tokens;     /* capacity of each request's tail (suffix + generated)    */
+    float softmax_scale;         /* 0 => 1/sqrt(head_dim)                                   */
+    float rope_theta;            /* 0 => q and k_new arrive already rotated (default)       */
+    int32_t pos_mode;            /* rotary mode only: position of the first tail token.
+                                    0 = sum of the request's chunk lengths (the query continues
+                                    after the documents, each of which starts at position 0);
+                                    1 = longest chunk length.  Inert when rope_theta == 0.     */
+    int32_t device;              /* CUDA device ordinal, -1 = current device                */
+} matkv_config;
+
+/* options for matkv_set_option */
+#define MATKV_OPT_DECODE_CTAS   1  /* number of CTAs the streaming kernel splits the KV over; 0 = auto */
+#define MATKV_OPT_PREFILL_IMPL  2  /* 0 = auto (tensor-core tiles when the suffix is large enough),
+                                      1 = force the streaming kernel, 2 = force the tensor-core kernel */
+#define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
+
+/* ---- context -------------------------------------------------------------------------- */
+/* Creates a context on cfg->device.  Allocates the device status word and nothing large.   */
+int matkv_create(const matkv_config *cfg, matkv_ctx **out);
+/* Destroys the context and every table built from it.  Borrowed buffers are not touched.   */
+int matkv_destroy(matkv_ctx *ctx);
+const char *matkv_last_error(void);
+int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value);
+
+/* Scratch memory for the split-KV partial results (fp32 o and log-sum-exp per part) and the
+ * per-unit arrival counters.  matkv_workspace_bytes() is the size needed for the largest
+ * launch the configuration allows; matkv_set_workspace() borrows `dev` (256-byte aligned
+ * device memory) and clears its counter region with a synchronous memset.                  */
+size_t matkv_workspace_bytes(const matkv_ctx *ctx);
+int matkv_set_workspace(matkv_ctx *ctx, void *dev, size_t bytes);
+
+/* Reads the device status word (synchronises the context's device first): 0 or MATKV_E_*.
+ * `clear` != 0 resets it.                                                                  */
+int matkv_status(matkv_ctx *ctx, int32_t *dev_status_out, int32_t clear);
+
+/* ---- a1: chunk registry (the paper's "file named chunk_id"; Section IV, store_KV) ------- */
+/* Records where the materialised K,V of `chunk_id` live.  host_blob: pinned (or pageable)
+ * host memory or NULL; dev_blob: device memory or NULL; at least one non-NULL.  Both are
+ * borrowed until matkv_unregister_chunk / matkv_destroy.  Re-registering an id is an error. */
+int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const void *host_blob,
+                         void *dev_blob);
+/* The paper's delete(O) (Section IV): forgets the chunk.  Tables built earlier keep the
+ * device address they resolved; the caller keeps that memory alive until they are freed.    */
+int matkv_unregister_chunk(matkv_ctx *ctx, uint64_t chunk_id);
+
+/* ---- a2: staging (the paper's load_KV, CPU bounce buffer -> GPU; Section IV, and the
+ *      overlap of the next batch's load with the current decode, Section III-B) ------------ */
+/* Copies the listed chunks' host blobs into `dev_slots` (n_slots slots of slot_bytes each,
+ * device memory, 256-byte aligned, borrowed) with one asynchronous copy per chunk on
+ * `copy_stream`, and records an event per call.  Duplicates in the list, chunks registered
+ * with a dev_blob, and chunks already sitting in this same slot region are not copied again;
+ * every other previous occupant of the region is evicted.  Before overwriting, copy_stream is
+ * made to wait for the last table that used the region (see matkv_table_free).  *ticket_out
+ * identifies the call for matkv_stage_query / matkv_stage_wait.  Never blocks the host.       */
+int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *chunk_ids, int32_t n, void *dev_slots,
+                             size_t slot_bytes, int32_t n_slots, void *copy_stream, uint64_t *ticket_out);
+/* MATKV_OK when the ticket's copies have finished, MATKV_E_NOT_READY otherwise (no blocking). */
+int matkv_stage_query(matkv_ctx *ctx, uint64_t ticket);
+/* Blocks the calling host thread until the ticket's copies have finished.                     */
+int matkv_stage_wait(matkv_ctx *ctx, uint64_t ticket);
+
+/* ---- a3: chunk table (replaces the concatenation of put_KV, Section IV) ------------------ */
+/* chunk_ids_flat is the concatenation of each request's ORDERED id list (documents before
+ * the query, Section III-A); n_chunks_per_req[r] may be 0 and ids may repeat.  tail_k / tail_v:
+ * device tails (layout above, batch = `batch`), borrowed, written by the attend calls.
+ * Resolves every id to its device copy (MATKV_E_NOT_STAGED if it has none), makes `stream`
+ * wait for the staging copies it depends on (never the host), uploads the table on `stream`
+ * and sets every request's tail length to 0.                                                 */
+int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chunks_per_req,
+                            const uint64_t *chunk_ids_flat, void *tail_k, void *tail_v, void *stream,
+                            matkv_table **out);
+/* Marks, on `stream`, the end of the table's use of staged slot regions (so that a later
+ * matkv_stage_chunks_async into them waits for it) and frees the table stream-ordered.        */
+int matkv_table_free(matkv_table *table, void *stream);
+/* Adds n_tokens to every request's tail length (device-side counter, so a captured decode
+ * loop can replay it).  Attend calls never move it: all layers of one step see one length.    */
+int matkv_table_advance(matkv_table *table, int32_t n_tokens, void *stream);
+int matkv_table_set_tail_len(matkv_table *table, int32_t tail_len, void *stream);
+
+/* ---- a4: query sub-prefill (Section V-A "Prefill time": from the end of loading to the
+ *      first token; the query is prefilled on top of the loaded KVs) ----------------------- */
+/* q [B][S][Hq][D], k_new / v_new [B][S][Hkv][D], out [B][S][Hq][D] bf16 device; lse_out NULL
+ * or [B][S][Hq] fp32 device (natural log).  Writes k_new / v_new to tail[t0 .. t0+S) of
+ * `layer` (t0 = current tail length) and lets suffix token i attend to every chunk token and
+ * to tail[0 .. t0+i].  In rotary mode q and k_new are rotated at position base + t0 + i first. */
+int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *table, int32_t layer, int32_t S, const void *q,
+                         const void *k_new, const void *v_new, void *out, float *lse_out, void *stream);
+
+/* ---- a5 + a6: decode step (Section V-A "Decode time"; memory-bound streaming over the
+ *      loaded KVs) with split-KV partials merged by log-sum-exp ---------------------------- */
+/* One new token per request.  q [B][Hq][D], k_new / v_new [B][Hkv][D], out [B][Hq][D] bf16
+ * device; lse_out NULL or [B][Hq] fp32.  Writes k_new / v_new to tail[t0] of `layer` and
+ * attends to every chunk token and to tail[0 .. t0].                                         */
+int matkv_attend_decode(matkv_ctx *ctx, matkv_table *table, int32_t layer, const void *q, const void *k_new,
+                        const void *v_new, void *out, float *lse_out, void *stream);
+/* The same for every layer in ONE launch: q [L][B][Hq][D], k_new / v_new [L][B][Hkv][D],
+ * out [L][B][Hq][D], lse_out NULL or [L][B][Hq].  Only usable when all layers' queries exist
+ * up front (an attention-only benchmark; a real model produces layer l+1's q from layer l).  */
+int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *table, const void *q, const void *k_new,
+                                   const void *v_new, void *out, float *lse_out, void *stream);
+
+/* a6 alone: merges n_parts partial attentions per row.  o_parts [n_rows][n_parts][D] fp32
+ * (each normalised within its part), lse_parts [n_rows][n_parts] fp32 natural log (-inf =
+ * empty part), out [n_rows][D] bf16, lse_out NULL or [n_rows] fp32; all device.              */
+int matkv_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts,
+                      const float *lse_parts, void *out, float *lse_out, void *stream);
+
+/* ---- debugging aid: the concatenation the table stands for ------------------------------- */
+/* Copies, for (layer, request), the K and V rows the table addresses into contiguous
+ * k_out / v_out [Hkv][n_chunk_tokens + tail_len][D] bf16 device buffers (bit-exact gather).
+ * rows_out (host, may be NULL) receives n_chunk_tokens + tail_len as known to the host.      */
+int matkv_gather_debug(matkv_ctx *ctx, matkv_table *table, int32_t layer, int32_t req, void *k_out,
+                       void *v_out, int64_t capacity_rows, int64_t *rows_out, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MATKV_H */

@@ -173,5 +173,14 @@ class Request:
         vis = [t0 + i + 1 for i in range(n)]
         return attend(self.shape, layer, self.chunks, self.tail_k[layer], self.tail_v[layer], qr, vis, evaluator)
 
+    def append_only(self, layer: int, k_new: np.ndarray, v_new: np.ndarray) -> None:
+        """Write n new tokens at tail[tail_len..) of ``layer`` without attending (bookkeeping only)."""
+        n = k_new.shape[0]
+        t0 = self.tail_len
+        assert t0 + n <= self.cap
+        kr = self._rot(k_new, self.pos_base + t0)
+        self.tail_k[layer, :, t0:t0 + n, :] = np.transpose(kr, (1, 0, 2))
+        self.tail_v[layer, :, t0:t0 + n, :] = np.transpose(_u16(v_new), (1, 0, 2))
+
     def advance(self, n: int) -> None:
         self.tail_len += n

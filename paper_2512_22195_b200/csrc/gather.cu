@@ -1,0 +1,83 @@
+// Debug gather (bit-exact copy of the rows a chunk table addresses) and the tail-length counter kernel.
+#include "matkv_internal.h"
+
+namespace matkv {
+
+// One CTA per (kv head, block of rows).  Each row of D bf16 is moved as 16-byte vectors, so the
+// output is a byte-for-byte concatenation chunk_0 | chunk_1 | ... | tail[0..tail_len).
+__global__ void k_gather(const DevSeg *__restrict__ segs, DevReq rq, const __nv_bfloat16 *__restrict__ tail_k,
+                         const __nv_bfloat16 *__restrict__ tail_v, int32_t tail_rows, int32_t max_tail, int32_t layer,
+                         int32_t Hkv, int32_t D, int64_t rows, uint4 *__restrict__ k_out, uint4 *__restrict__ v_out,
+                         int32_t *status) {
+    const int g = blockIdx.y;
+    const int vec_per_row = D / 8;
+    const int64_t n_vec = rows * vec_per_row;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / vec_per_row;
+        const int v = (int)(i % vec_per_row);
+        const uint4 *ksrc, *vsrc;
+        if (row < rq.n_chunk_tokens) {
+            // binary search the segment that holds this row
+            int lo = 0, hi = rq.n_seg - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (segs[rq.seg_begin + mid].start <= row) lo = mid; else hi = mid - 1;
+            }
+            const DevSeg sg = segs[rq.seg_begin + lo];
+            const int64_t t = row - sg.start;
+            if (t < 0 || t >= sg.len) {
+                atomicCAS(status, 0, MATKV_E_BOUNDS);
+                continue;
+            }
+            const int64_t kslab = ((int64_t)layer * 2 * Hkv + g) * sg.len;
+            const int64_t vslab = (((int64_t)layer * 2 + 1) * Hkv + g) * sg.len;
+            ksrc = (const uint4 *)(sg.base + (kslab + t) * D);
+            vsrc = (const uint4 *)(sg.base + (vslab + t) * D);
+        } else {
+            const int64_t t = row - rq.n_chunk_tokens;
+            if (t >= tail_rows) {
+                atomicCAS(status, 0, MATKV_E_BOUNDS);
+                continue;
+            }
+            ksrc = (const uint4 *)(tail_k + ((int64_t)g * max_tail + t) * D);
+            vsrc = (const uint4 *)(tail_v + ((int64_t)g * max_tail + t) * D);
+        }
+        k_out[((int64_t)g * rows + row) * vec_per_row + v] = ksrc[v];
+        v_out[((int64_t)g * rows + row) * vec_per_row + v] = vsrc[v];
+    }
+}
+
+__global__ void k_tail_len(int32_t *tail_len, int32_t batch, int32_t delta, int32_t value, int32_t set, int32_t max_tail,
+                           int32_t *status) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= batch) return;
+    int32_t v = set ? value : tail_len[i] + delta;
+    if (v > max_tail) {  // a replayed graph ran past the tail's capacity: clamp and report
+        v = max_tail;
+        atomicCAS(status, 0, MATKV_E_CAPACITY);
+    }
+    tail_len[i] = v;
+}
+
+int launch_gather(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out, int64_t rows,
+                  cudaStream_t stream) {
+    const matkv_config &c = ctx->cfg;
+    const int64_t tail_off = ((int64_t)req * c.n_layers + layer) * c.n_kv_heads * (int64_t)c.max_tail_tokens * c.head_dim;
+    const int64_t n_vec = rows * (c.head_dim / 8);
+    int bx = (int)std::min<int64_t>((n_vec + 255) / 256, 4 * (int64_t)ctx->n_sm);
+    dim3 grid(bx < 1 ? 1 : bx, c.n_kv_heads);
+    k_gather<<<grid, 256, 0, stream>>>(t->d_segs, t->h_reqs[req], t->tail_k + tail_off, t->tail_v + tail_off,
+                                       t->tail_len_host, c.max_tail_tokens, layer, c.n_kv_heads, c.head_dim, rows,
+                                       (uint4 *)k_out, (uint4 *)v_out, ctx->d_status);
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
+int launch_add_tail_len(matkv_table *t, int32_t delta, int32_t set_value, bool set, cudaStream_t stream) {
+    k_tail_len<<<(t->batch + 127) / 128, 128, 0, stream>>>(t->d_tail_len, t->batch, delta, set_value, set ? 1 : 0,
+                                                          t->ctx->cfg.max_tail_tokens, t->ctx->d_status);
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
+}  // namespace matkv

@@ -1,0 +1,614 @@
+// Host side of the C ABI: context, chunk registry, staging, chunk table, status.
+// No attention arithmetic lives here; the kernels and their launchers are in the other files.
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <cmath>
+
+#include "matkv_internal.h"
+
+namespace matkv {
+
+static thread_local char g_err[512] = "";
+
+int fail(int code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int cuda_fail(cudaError_t e, const char *what) {
+    return fail(MATKV_E_CUDA, "CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+size_t workspace_bytes_for(const matkv_config &c, WorkspaceView *v, void *base) {
+    const int64_t G = c.n_q_heads / c.n_kv_heads;
+    const int64_t units_decode = (int64_t)c.n_layers * c.max_batch * c.n_kv_heads;
+    const int64_t units_prefill = (int64_t)c.max_batch * c.max_tail_tokens * c.n_kv_heads;
+    const int64_t n_units = std::max(units_decode, units_prefill);
+    const int64_t n_parts = n_units + kMaxGridCtas;
+    size_t off = 0;
+    const size_t counters_off = off;
+    off = align_up(off + sizeof(int32_t) * (size_t)n_units, 256);
+    const size_t lse_off = off;
+    off = align_up(off + sizeof(float) * (size_t)(n_parts * G), 256);
+    const size_t o_off = off;
+    off = align_up(off + sizeof(float) * (size_t)(n_parts * G * c.head_dim), 256);
+    if (v) {
+        char *b = (char *)base;
+        v->counters = (int32_t *)(b + counters_off);
+        v->part_lse = (float *)(b + lse_off);
+        v->part_o = (float *)(b + o_off);
+        v->n_counter_slots = n_units;
+        v->n_part_slots = n_parts;
+    }
+    return off;
+}
+
+static void reap_graveyard(matkv_ctx *ctx, bool force);
+
+}  // namespace matkv
+
+using namespace matkv;
+
+// tables whose stream work may still be running when the caller frees them
+struct Grave {
+    cudaEvent_t ev;
+    void *h_pinned;
+    void *d_image;
+};
+static std::map<matkv_ctx *, std::vector<Grave>> g_graves;
+
+static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
+    auto it = g_graves.find(ctx);
+    if (it == g_graves.end()) return;
+    auto &v = it->second;
+    for (size_t i = 0; i < v.size();) {
+        bool done = force;
+        if (force) cudaEventSynchronize(v[i].ev);
+        else done = (cudaEventQuery(v[i].ev) == cudaSuccess);
+        if (done) {
+            cudaFreeHost(v[i].h_pinned);
+            cudaFree(v[i].d_image);
+            cudaEventDestroy(v[i].ev);
+            v[i] = v.back();
+            v.pop_back();
+        } else {
+            ++i;
+        }
+    }
+    if (force) g_graves.erase(it);
+}
+
+extern "C" {
+
+const char *matkv_last_error(void) { return g_err; }
+
+int matkv_create(const matkv_config *cfg, matkv_ctx **out) {
+    if (!cfg || !out) return fail(MATKV_E_INVALID_ARG, "matkv_create: null argument");
+    *out = nullptr;
+    if (cfg->n_layers < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads % cfg->n_kv_heads)
+        return fail(MATKV_E_INVALID_ARG, "matkv_create: bad layer/head counts");
+    const int G = cfg->n_q_heads / cfg->n_kv_heads;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128)
+        return fail(MATKV_E_INVALID_ARG, "matkv_create: head_dim must be 64 or 128");
+    if (G != 1 && G != 2 && G != 4 && G != 8)
+        return fail(MATKV_E_INVALID_ARG, "matkv_create: query heads per KV head must be 1, 2, 4 or 8");
+    if (cfg->max_batch < 1 || cfg->max_batch > 1024 || cfg->max_chunks_per_req < 0 || cfg->max_tail_tokens < 1)
+        return fail(MATKV_E_INVALID_ARG, "matkv_create: bad capacity");
+    if (cfg->softmax_scale < 0.f || cfg->rope_theta < 0.f || cfg->pos_mode < 0 || cfg->pos_mode > 1)
+        return fail(MATKV_E_INVALID_ARG, "matkv_create: bad scale / rotary settings");
+    int dev = cfg->device;
+    if (dev < 0) MATKV_CUDA(cudaGetDevice(&dev));
+    DeviceGuard guard(dev);
+    cudaDeviceProp prop;
+    MATKV_CUDA(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10)
+        return fail(MATKV_E_CUDA, "matkv_create: device %d is sm_%d%d; this library is built for sm_100a only", dev,
+                    prop.major, prop.minor);
+    matkv_ctx *ctx = new matkv_ctx();
+    ctx->cfg = *cfg;
+    ctx->device = dev;
+    ctx->cfg.device = dev;
+    ctx->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+    ctx->n_sm = prop.multiProcessorCount;
+    cudaError_t e = cudaMalloc(&ctx->d_status, sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int32_t));
+    if (e != cudaSuccess) {
+        delete ctx;
+        return cuda_fail(e, "status word");
+    }
+    *out = ctx;
+    return MATKV_OK;
+}
+
+int matkv_destroy(matkv_ctx *ctx) {
+    if (!ctx) return MATKV_OK;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    for (matkv_table *t : std::vector<matkv_table *>(ctx->tables)) {
+        cudaFreeHost(t->h_pinned);
+        cudaFree(t->d_image);
+        delete t;
+    }
+    ctx->tables.clear();
+    reap_graveyard(ctx, true);
+    for (auto &kv : ctx->tickets) cudaEventDestroy(kv.second.done);
+    for (auto &kv : ctx->regions) {
+        if (kv.second->last_use) cudaEventDestroy(kv.second->last_use);
+        delete kv.second;
+    }
+    cudaFree(ctx->d_status);
+    delete ctx;
+    return MATKV_OK;
+}
+
+int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
+    if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_set_option: null context");
+    switch (option) {
+        case MATKV_OPT_DECODE_CTAS:
+            if (value < 0 || value > kMaxGridCtas) return fail(MATKV_E_INVALID_ARG, "decode CTAs must be 0..%d", kMaxGridCtas);
+            ctx->opt_decode_ctas = value;
+            return MATKV_OK;
+        case MATKV_OPT_PREFILL_IMPL:
+            if (value < 0 || value > 2) return fail(MATKV_E_INVALID_ARG, "prefill impl must be 0, 1 or 2");
+            ctx->opt_prefill_impl = value;
+            return MATKV_OK;
+        case MATKV_OPT_PREFILL_CTAS:
+            if (value < 0 || value > 64) return fail(MATKV_E_INVALID_ARG, "prefill CTAs per head must be 0..64");
+            ctx->opt_prefill_ctas = value;
+            return MATKV_OK;
+    }
+    return fail(MATKV_E_INVALID_ARG, "matkv_set_option: unknown option %d", option);
+}
+
+size_t matkv_workspace_bytes(const matkv_ctx *ctx) {
+    if (!ctx) return 0;
+    return workspace_bytes_for(ctx->cfg, nullptr, nullptr);
+}
+
+int matkv_set_workspace(matkv_ctx *ctx, void *dev, size_t bytes) {
+    if (!ctx || !dev) return fail(MATKV_E_INVALID_ARG, "matkv_set_workspace: null argument");
+    if ((uintptr_t)dev % 256) return fail(MATKV_E_ALIGNMENT, "workspace must be 256-byte aligned");
+    WorkspaceView v;
+    const size_t need = workspace_bytes_for(ctx->cfg, &v, dev);
+    if (bytes < need) return fail(MATKV_E_CAPACITY, "workspace of %zu bytes is smaller than the %zu needed", bytes, need);
+    DeviceGuard guard(ctx->device);
+    MATKV_CUDA(cudaDeviceSynchronize());
+    MATKV_CUDA(cudaMemset(v.counters, 0, sizeof(int32_t) * (size_t)v.n_counter_slots));
+    ctx->workspace = dev;
+    ctx->workspace_bytes = bytes;
+    return MATKV_OK;
+}
+
+int matkv_status(matkv_ctx *ctx, int32_t *dev_status_out, int32_t clear) {
+    if (!ctx || !dev_status_out) return fail(MATKV_E_INVALID_ARG, "matkv_status: null argument");
+    DeviceGuard guard(ctx->device);
+    MATKV_CUDA(cudaDeviceSynchronize());
+    MATKV_CUDA(cudaMemcpy(dev_status_out, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (clear) MATKV_CUDA(cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    return MATKV_OK;
+}
+
+// ---- a1 --------------------------------------------------------------------------------------
+int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const void *host_blob, void *dev_blob) {
+    if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_register_chunk: null context");
+    if (n_tokens < 1) return fail(MATKV_E_INVALID_ARG, "chunk %llu: n_tokens must be >= 1", (unsigned long long)chunk_id);
+    if (!host_blob && !dev_blob) return fail(MATKV_E_INVALID_ARG, "chunk %llu: no blob given", (unsigned long long)chunk_id);
+    if (dev_blob && (uintptr_t)dev_blob % 256)
+        return fail(MATKV_E_ALIGNMENT, "chunk %llu: device blob must be 256-byte aligned", (unsigned long long)chunk_id);
+    if (host_blob && (uintptr_t)host_blob % 16)
+        return fail(MATKV_E_ALIGNMENT, "chunk %llu: host blob must be 16-byte aligned", (unsigned long long)chunk_id);
+    if (ctx->chunks.count(chunk_id))
+        return fail(MATKV_E_INVALID_ARG, "chunk %llu is already registered", (unsigned long long)chunk_id);
+    Chunk c;
+    c.n_tokens = n_tokens;
+    c.host_blob = host_blob;
+    c.dev_blob = dev_blob;
+    ctx->chunks.emplace(chunk_id, c);
+    return MATKV_OK;
+}
+
+int matkv_unregister_chunk(matkv_ctx *ctx, uint64_t chunk_id) {
+    if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_unregister_chunk: null context");
+    auto it = ctx->chunks.find(chunk_id);
+    if (it == ctx->chunks.end()) return fail(MATKV_E_UNKNOWN_CHUNK, "chunk %llu is not registered", (unsigned long long)chunk_id);
+    Chunk &c = it->second;
+    if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;
+    ctx->chunks.erase(it);
+    return MATKV_OK;
+}
+
+static size_t blob_bytes(const matkv_config &c, int32_t n_tokens) {
+    return (size_t)c.n_layers * 2 * c.n_kv_heads * (size_t)n_tokens * c.head_dim * sizeof(__nv_bfloat16);
+}
+
+// ---- a2 --------------------------------------------------------------------------------------
+int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, void *dev_slots, size_t slot_bytes,
+                             int32_t n_slots, void *copy_stream, uint64_t *ticket_out) {
+    if (!ctx || (!ids && n > 0) || !dev_slots || !ticket_out)
+        return fail(MATKV_E_INVALID_ARG, "matkv_stage_chunks_async: null argument");
+    if (n < 0 || n_slots < 1 || slot_bytes == 0) return fail(MATKV_E_INVALID_ARG, "matkv_stage_chunks_async: bad sizes");
+    if ((uintptr_t)dev_slots % 256 || slot_bytes % 256)
+        return fail(MATKV_E_ALIGNMENT, "slot base and slot size must be multiples of 256 bytes");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t cs = (cudaStream_t)copy_stream;
+    reap_graveyard(ctx, false);
+
+    // distinct ids that need a copy into this region
+    std::vector<uint64_t> want;
+    for (int32_t i = 0; i < n; ++i) {
+        auto it = ctx->chunks.find(ids[i]);
+        if (it == ctx->chunks.end())
+            return fail(MATKV_E_UNKNOWN_CHUNK, "chunk %llu is not registered", (unsigned long long)ids[i]);
+        const Chunk &c = it->second;
+        if (c.dev_blob) continue;  // resident: nothing to do
+        if (!c.host_blob) return fail(MATKV_E_INVALID_ARG, "chunk %llu has no host blob to stage", (unsigned long long)ids[i]);
+        if (blob_bytes(ctx->cfg, c.n_tokens) > slot_bytes)
+            return fail(MATKV_E_CAPACITY, "chunk %llu (%zu bytes) does not fit a slot of %zu bytes",
+                        (unsigned long long)ids[i], blob_bytes(ctx->cfg, c.n_tokens), slot_bytes);
+        if (std::find(want.begin(), want.end(), ids[i]) == want.end()) want.push_back(ids[i]);
+    }
+    if ((int64_t)want.size() > n_slots)
+        return fail(MATKV_E_CAPACITY, "%zu distinct chunks do not fit %d slots", want.size(), n_slots);
+
+    Region *&rp = ctx->regions[dev_slots];
+    if (!rp) {
+        rp = new Region();
+        rp->base = dev_slots;
+    }
+    Region *r = rp;
+    if (r->slot_bytes != slot_bytes || r->n_slots != n_slots) {
+        // geometry changed: drop every occupant
+        for (size_t s = 0; s < r->occupant.size(); ++s)
+            if (r->used[s]) {
+                auto it = ctx->chunks.find(r->occupant[s]);
+                if (it != ctx->chunks.end() && it->second.region == r) {
+                    it->second.staged = nullptr;
+                    it->second.region = nullptr;
+                    it->second.slot = -1;
+                }
+            }
+        r->slot_bytes = slot_bytes;
+        r->n_slots = n_slots;
+        r->occupant.assign(n_slots, 0);
+        r->used.assign(n_slots, 0);
+    }
+    // keep occupants that are wanted again, evict the rest
+    for (int32_t s = 0; s < n_slots; ++s) {
+        if (!r->used[s]) continue;
+        const uint64_t id = r->occupant[s];
+        if (std::find(want.begin(), want.end(), id) != want.end()) continue;
+        auto it = ctx->chunks.find(id);
+        if (it != ctx->chunks.end() && it->second.region == r && it->second.slot == s) {
+            it->second.staged = nullptr;
+            it->second.region = nullptr;
+            it->second.slot = -1;
+        }
+        r->used[s] = 0;
+    }
+    // the region's previous readers must be done before anything is overwritten
+    if (r->has_last_use) MATKV_CUDA(cudaStreamWaitEvent(cs, r->last_use, 0));
+
+    Ticket tk;
+    MATKV_CUDA(cudaEventCreateWithFlags(&tk.done, cudaEventDisableTiming));
+    const uint64_t ticket = ctx->next_ticket++;
+    int32_t next_free = 0;
+    for (uint64_t id : want) {
+        Chunk &c = ctx->chunks[id];
+        if (c.region == r && c.slot >= 0 && r->used[c.slot] && r->occupant[c.slot] == id) continue;  // already here
+        while (next_free < n_slots && r->used[next_free]) ++next_free;
+        if (next_free >= n_slots) {
+            cudaEventDestroy(tk.done);
+            return fail(MATKV_E_CAPACITY, "no free slot left in the region");
+        }
+        if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;  // moves from another region
+        void *dst = (char *)dev_slots + (size_t)next_free * slot_bytes;
+        cudaError_t e = cudaMemcpyAsync(dst, c.host_blob, blob_bytes(ctx->cfg, c.n_tokens), cudaMemcpyHostToDevice, cs);
+        if (e != cudaSuccess) {
+            cudaEventDestroy(tk.done);
+            return cuda_fail(e, "staging copy");
+        }
+        r->used[next_free] = 1;
+        r->occupant[next_free] = id;
+        c.staged = dst;
+        c.region = r;
+        c.slot = next_free;
+        c.ready = tk.done;
+        c.ticket = ticket;
+    }
+    MATKV_CUDA(cudaEventRecord(tk.done, cs));
+    ctx->tickets.emplace(ticket, tk);
+    *ticket_out = ticket;
+    return MATKV_OK;
+}
+
+int matkv_stage_query(matkv_ctx *ctx, uint64_t ticket) {
+    if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_stage_query: null context");
+    auto it = ctx->tickets.find(ticket);
+    if (it == ctx->tickets.end()) return fail(MATKV_E_INVALID_ARG, "unknown staging ticket %llu", (unsigned long long)ticket);
+    cudaError_t e = cudaEventQuery(it->second.done);
+    if (e == cudaSuccess) return MATKV_OK;
+    if (e == cudaErrorNotReady) return fail(MATKV_E_NOT_READY, "staging ticket %llu still copying", (unsigned long long)ticket);
+    return cuda_fail(e, "cudaEventQuery");
+}
+
+int matkv_stage_wait(matkv_ctx *ctx, uint64_t ticket) {
+    if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_stage_wait: null context");
+    auto it = ctx->tickets.find(ticket);
+    if (it == ctx->tickets.end()) return fail(MATKV_E_INVALID_ARG, "unknown staging ticket %llu", (unsigned long long)ticket);
+    MATKV_CUDA(cudaEventSynchronize(it->second.done));
+    return MATKV_OK;
+}
+
+// ---- a3 --------------------------------------------------------------------------------------
+int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chunks_per_req, const uint64_t *ids,
+                            void *tail_k, void *tail_v, void *stream, matkv_table **out) {
+    if (!ctx || !n_chunks_per_req || !tail_k || !tail_v || !out)
+        return fail(MATKV_E_INVALID_ARG, "matkv_build_chunk_table: null argument");
+    *out = nullptr;
+    if (batch < 1 || batch > ctx->cfg.max_batch)
+        return fail(MATKV_E_CAPACITY, "batch %d outside 1..%d", batch, ctx->cfg.max_batch);
+    if ((uintptr_t)tail_k % 256 || (uintptr_t)tail_v % 256) return fail(MATKV_E_ALIGNMENT, "tails must be 256-byte aligned");
+    int64_t total = 0;
+    for (int32_t r = 0; r < batch; ++r) {
+        if (n_chunks_per_req[r] < 0 || n_chunks_per_req[r] > ctx->cfg.max_chunks_per_req)
+            return fail(MATKV_E_CAPACITY, "request %d lists %d chunks (max %d)", r, n_chunks_per_req[r],
+                        ctx->cfg.max_chunks_per_req);
+        total += n_chunks_per_req[r];
+    }
+    if (total > 0 && !ids) return fail(MATKV_E_INVALID_ARG, "matkv_build_chunk_table: null id list");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    reap_graveyard(ctx, false);
+
+    matkv_table *t = new matkv_table();
+    t->ctx = ctx;
+    t->batch = batch;
+    t->tail_k = (__nv_bfloat16 *)tail_k;
+    t->tail_v = (__nv_bfloat16 *)tail_v;
+    std::vector<cudaEvent_t> waits;
+    int64_t k = 0;
+    for (int32_t r = 0; r < batch; ++r) {
+        DevReq rq;
+        memset(&rq, 0, sizeof rq);
+        rq.seg_begin = (int32_t)t->h_segs.size();
+        rq.n_seg = n_chunks_per_req[r];
+        int32_t longest = 0;
+        for (int32_t i = 0; i < rq.n_seg; ++i, ++k) {
+            auto it = ctx->chunks.find(ids[k]);
+            if (it == ctx->chunks.end()) {
+                delete t;
+                return fail(MATKV_E_UNKNOWN_CHUNK, "request %d: chunk %llu is not registered", r, (unsigned long long)ids[k]);
+            }
+            const Chunk &c = it->second;
+            const void *dev = c.dev_blob ? c.dev_blob : c.staged;
+            if (!dev) {
+                delete t;
+                return fail(MATKV_E_NOT_STAGED, "request %d: chunk %llu has no device copy (stage it first)", r,
+                            (unsigned long long)ids[k]);
+            }
+            if (!c.dev_blob) {
+                if (std::find(waits.begin(), waits.end(), c.ready) == waits.end()) waits.push_back(c.ready);
+                if (std::find(t->regions.begin(), t->regions.end(), c.region) == t->regions.end())
+                    t->regions.push_back(c.region);
+            }
+            DevSeg sg;
+            sg.base = (const __nv_bfloat16 *)dev;
+            sg.len = c.n_tokens;
+            sg.start = rq.n_chunk_tokens;
+            t->h_segs.push_back(sg);
+            rq.n_chunk_tokens += c.n_tokens;
+            rq.chunk_tiles += (c.n_tokens + kTile - 1) / kTile;
+            longest = std::max(longest, c.n_tokens);
+        }
+        rq.pos_base = ctx->cfg.pos_mode == 0 ? rq.n_chunk_tokens : longest;
+        t->max_chunk_tiles = std::max(t->max_chunk_tiles, rq.chunk_tiles);
+        t->total_chunk_tiles += rq.chunk_tiles;
+        t->h_reqs.push_back(rq);
+    }
+    t->n_seg_total = (int32_t)t->h_segs.size();
+
+    const size_t segs_bytes = align_up(sizeof(DevSeg) * std::max<size_t>(t->h_segs.size(), 1), 256);
+    const size_t reqs_bytes = align_up(sizeof(DevReq) * (size_t)batch, 256);
+    const size_t tl_bytes = align_up(sizeof(int32_t) * (size_t)batch, 256);
+    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes;
+    cudaError_t e = cudaMallocHost(&t->h_pinned, t->image_bytes);
+    if (e == cudaSuccess) e = cudaMalloc(&t->d_image, t->image_bytes);
+    if (e != cudaSuccess) {
+        cudaFreeHost(t->h_pinned);
+        delete t;
+        return cuda_fail(e, "table allocation");
+    }
+    memset(t->h_pinned, 0, t->image_bytes);
+    if (!t->h_segs.empty()) memcpy(t->h_pinned, t->h_segs.data(), sizeof(DevSeg) * t->h_segs.size());
+    memcpy((char *)t->h_pinned + segs_bytes, t->h_reqs.data(), sizeof(DevReq) * (size_t)batch);
+    t->d_segs = (DevSeg *)t->d_image;
+    t->d_reqs = (DevReq *)((char *)t->d_image + segs_bytes);
+    t->d_tail_len = (int32_t *)((char *)t->d_image + segs_bytes + reqs_bytes);
+    for (cudaEvent_t ev : waits) {
+        e = cudaStreamWaitEvent(st, ev, 0);  // the stream waits for the copies; the host does not
+        if (e != cudaSuccess) break;
+    }
+    if (e == cudaSuccess) e = cudaMemcpyAsync(t->d_image, t->h_pinned, t->image_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) {
+        cudaFreeHost(t->h_pinned);
+        cudaFree(t->d_image);
+        delete t;
+        return cuda_fail(e, "table upload");
+    }
+    ctx->tables.push_back(t);
+    *out = t;
+    return MATKV_OK;
+}
+
+int matkv_table_free(matkv_table *t, void *stream) {
+    if (!t) return MATKV_OK;
+    matkv_ctx *ctx = t->ctx;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    for (Region *r : t->regions) {
+        if (!r->last_use) MATKV_CUDA(cudaEventCreateWithFlags(&r->last_use, cudaEventDisableTiming));
+        MATKV_CUDA(cudaEventRecord(r->last_use, st));
+        r->has_last_use = true;
+    }
+    Grave g;
+    MATKV_CUDA(cudaEventCreateWithFlags(&g.ev, cudaEventDisableTiming));
+    MATKV_CUDA(cudaEventRecord(g.ev, st));
+    g.h_pinned = t->h_pinned;
+    g.d_image = t->d_image;
+    g_graves[ctx].push_back(g);
+    ctx->tables.erase(std::remove(ctx->tables.begin(), ctx->tables.end(), t), ctx->tables.end());
+    delete t;
+    reap_graveyard(ctx, false);
+    return MATKV_OK;
+}
+
+int matkv_table_advance(matkv_table *t, int32_t n_tokens, void *stream) {
+    if (!t) return fail(MATKV_E_INVALID_ARG, "matkv_table_advance: null table");
+    if (n_tokens < 0) return fail(MATKV_E_INVALID_ARG, "matkv_table_advance: negative count");
+    if (t->tail_len_host + n_tokens > t->ctx->cfg.max_tail_tokens)
+        return fail(MATKV_E_CAPACITY, "tail would hold %d tokens (max %d)", t->tail_len_host + n_tokens,
+                    t->ctx->cfg.max_tail_tokens);
+    DeviceGuard guard(t->ctx->device);
+    int rc = launch_add_tail_len(t, n_tokens, 0, false, (cudaStream_t)stream);
+    if (rc == MATKV_OK) t->tail_len_host += n_tokens;
+    return rc;
+}
+
+int matkv_table_set_tail_len(matkv_table *t, int32_t tail_len, void *stream) {
+    if (!t) return fail(MATKV_E_INVALID_ARG, "matkv_table_set_tail_len: null table");
+    if (tail_len < 0 || tail_len > t->ctx->cfg.max_tail_tokens)
+        return fail(MATKV_E_CAPACITY, "tail length %d outside 0..%d", tail_len, t->ctx->cfg.max_tail_tokens);
+    DeviceGuard guard(t->ctx->device);
+    int rc = launch_add_tail_len(t, 0, tail_len, true, (cudaStream_t)stream);
+    if (rc == MATKV_OK) t->tail_len_host = tail_len;
+    return rc;
+}
+
+// ---- a4 / a5 / a6 argument checks, then the launchers -----------------------------------------
+static int check_attend(matkv_ctx *ctx, matkv_table *t, const void *q, const void *kn, const void *vn, void *out,
+                        int32_t n_new, const char *who) {
+    if (!ctx || !t || !q || !kn || !vn || !out) return fail(MATKV_E_INVALID_ARG, "%s: null argument", who);
+    if (t->ctx != ctx) return fail(MATKV_E_INVALID_ARG, "%s: table belongs to another context", who);
+    if (((uintptr_t)q | (uintptr_t)kn | (uintptr_t)vn | (uintptr_t)out) % 16)
+        return fail(MATKV_E_ALIGNMENT, "%s: q, k_new, v_new and out must be 16-byte aligned", who);
+    if (!ctx->workspace) return fail(MATKV_E_INVALID_ARG, "%s: no workspace set (matkv_set_workspace)", who);
+    if (t->tail_len_host + n_new > ctx->cfg.max_tail_tokens)
+        return fail(MATKV_E_CAPACITY, "%s: tail holds %d tokens, %d more exceed max_tail_tokens %d", who, t->tail_len_host,
+                    n_new, ctx->cfg.max_tail_tokens);
+    if (ctx->cfg.rope_theta != 0.f)
+        return fail(MATKV_E_INVALID_ARG, "%s: rotary mode is not available in this build; pass rotated q and k_new", who);
+    return MATKV_OK;
+}
+
+int matkv_attend_decode(matkv_ctx *ctx, matkv_table *t, int32_t layer, const void *q, const void *kn, const void *vn,
+                        void *out, float *lse_out, void *stream) {
+    int rc = check_attend(ctx, t, q, kn, vn, out, 1, "matkv_attend_decode");
+    if (rc) return rc;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(MATKV_E_INVALID_ARG, "matkv_attend_decode: layer %d", layer);
+    DeviceGuard guard(ctx->device);
+    const matkv_config &c = ctx->cfg;
+    AttendArgs a;
+    a.layer0 = layer;
+    a.n_layers_launch = 1;
+    a.S = 1;
+    a.q = (const __nv_bfloat16 *)q;
+    a.k_new = (const __nv_bfloat16 *)kn;
+    a.v_new = (const __nv_bfloat16 *)vn;
+    a.out = (__nv_bfloat16 *)out;
+    a.lse_out = lse_out;
+    a.q_sl = 0; a.q_sb = (int64_t)c.n_q_heads * c.head_dim; a.q_ss = 0;
+    a.kn_sl = 0; a.kn_sb = (int64_t)c.n_kv_heads * c.head_dim; a.kn_ss = 0;
+    a.lse_sl = 0; a.lse_sb = c.n_q_heads; a.lse_ss = 0;
+    return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+}
+
+int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *t, const void *q, const void *kn, const void *vn,
+                                   void *out, float *lse_out, void *stream) {
+    int rc = check_attend(ctx, t, q, kn, vn, out, 1, "matkv_attend_decode_all_layers");
+    if (rc) return rc;
+    DeviceGuard guard(ctx->device);
+    const matkv_config &c = ctx->cfg;
+    AttendArgs a;
+    a.layer0 = 0;
+    a.n_layers_launch = c.n_layers;
+    a.S = 1;
+    a.q = (const __nv_bfloat16 *)q;
+    a.k_new = (const __nv_bfloat16 *)kn;
+    a.v_new = (const __nv_bfloat16 *)vn;
+    a.out = (__nv_bfloat16 *)out;
+    a.lse_out = lse_out;
+    a.q_sb = (int64_t)c.n_q_heads * c.head_dim; a.q_sl = a.q_sb * t->batch; a.q_ss = 0;
+    a.kn_sb = (int64_t)c.n_kv_heads * c.head_dim; a.kn_sl = a.kn_sb * t->batch; a.kn_ss = 0;
+    a.lse_sb = c.n_q_heads; a.lse_sl = a.lse_sb * t->batch; a.lse_ss = 0;
+    return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+}
+
+int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t S, const void *q, const void *kn,
+                         const void *vn, void *out, float *lse_out, void *stream) {
+    if (S < 1) return fail(MATKV_E_INVALID_ARG, "matkv_attend_prefill: S must be >= 1");
+    int rc = check_attend(ctx, t, q, kn, vn, out, S, "matkv_attend_prefill");
+    if (rc) return rc;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(MATKV_E_INVALID_ARG, "matkv_attend_prefill: layer %d", layer);
+    DeviceGuard guard(ctx->device);
+    const matkv_config &c = ctx->cfg;
+    AttendArgs a;
+    a.layer0 = layer;
+    a.n_layers_launch = 1;
+    a.S = S;
+    a.q = (const __nv_bfloat16 *)q;
+    a.k_new = (const __nv_bfloat16 *)kn;
+    a.v_new = (const __nv_bfloat16 *)vn;
+    a.out = (__nv_bfloat16 *)out;
+    a.lse_out = lse_out;
+    a.q_ss = (int64_t)c.n_q_heads * c.head_dim; a.q_sb = a.q_ss * S; a.q_sl = 0;
+    a.kn_ss = (int64_t)c.n_kv_heads * c.head_dim; a.kn_sb = a.kn_ss * S; a.kn_sl = 0;
+    a.lse_ss = c.n_q_heads; a.lse_sb = a.lse_ss * S; a.lse_sl = 0;
+    return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+}
+
+int matkv_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts,
+                      const float *lse_parts, void *out, float *lse_out, void *stream) {
+    if (!ctx || !o_parts || !lse_parts || !out) return fail(MATKV_E_INVALID_ARG, "matkv_lse_combine: null argument");
+    if (n_rows < 0 || n_parts < 1 || D < 32 || D > 256 || D % 32)
+        return fail(MATKV_E_INVALID_ARG, "matkv_lse_combine: bad sizes (D must be a multiple of 32, at most 256)");
+    if (n_rows == 0) return MATKV_OK;
+    DeviceGuard guard(ctx->device);
+    return launch_lse_combine(ctx, n_rows, n_parts, D, o_parts, lse_parts, out, lse_out, (cudaStream_t)stream);
+}
+
+int matkv_gather_debug(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out,
+                       int64_t capacity_rows, int64_t *rows_out, void *stream) {
+    if (!ctx || !t || !k_out || !v_out) return fail(MATKV_E_INVALID_ARG, "matkv_gather_debug: null argument");
+    if (t->ctx != ctx) return fail(MATKV_E_INVALID_ARG, "matkv_gather_debug: table belongs to another context");
+    if (layer < 0 || layer >= ctx->cfg.n_layers || req < 0 || req >= t->batch)
+        return fail(MATKV_E_INVALID_ARG, "matkv_gather_debug: layer %d / request %d out of range", layer, req);
+    const int64_t rows = (int64_t)t->h_reqs[req].n_chunk_tokens + t->tail_len_host;
+    if (rows_out) *rows_out = rows;
+    if (rows > capacity_rows) return fail(MATKV_E_CAPACITY, "gather needs %lld rows, buffers hold %lld", (long long)rows,
+                                          (long long)capacity_rows);
+    if (((uintptr_t)k_out | (uintptr_t)v_out) % 16) return fail(MATKV_E_ALIGNMENT, "gather outputs must be 16-byte aligned");
+    if (rows == 0) return MATKV_OK;
+    DeviceGuard guard(ctx->device);
+    return launch_gather(ctx, t, layer, req, k_out, v_out, rows, (cudaStream_t)stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,138 @@
+// Internal declarations shared by the host-side C ABI and the kernels' launchers.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include <map>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/matkv.h"
+
+namespace matkv {
+
+constexpr int kTile = 32;          // KV tokens per streaming tile (one ring slot holds K or V of one tile)
+constexpr int kMaxGridCtas = 1024; // upper bound on the streaming kernel's grid (workspace is sized for it)
+
+// ---- device-side table --------------------------------------------------------------------
+// One segment = one materialised chunk as seen by one request (device address of its blob).
+struct DevSeg {
+    const __nv_bfloat16 *base;  // blob [L][2][Hkv][len][D]
+    int32_t len;                // tokens
+    int32_t start;              // tokens before this segment in the request's logical order
+};
+struct DevReq {
+    int32_t seg_begin;       // index of the request's first segment in the segment array
+    int32_t n_seg;
+    int32_t n_chunk_tokens;  // sum of len
+    int32_t chunk_tiles;     // sum of ceil(len / kTile)
+    int32_t pos_base;        // rotary mode: position of tail token 0
+    int32_t pad[3];
+};
+
+// ---- host-side objects --------------------------------------------------------------------
+struct Region;  // staged slot region
+
+struct Chunk {
+    int32_t n_tokens = 0;
+    const void *host_blob = nullptr;
+    void *dev_blob = nullptr;      // caller-resident device copy
+    void *staged = nullptr;        // device copy inside a slot region (or nullptr)
+    Region *region = nullptr;
+    int32_t slot = -1;
+    cudaEvent_t ready = nullptr;   // event of the staging call that (last) copied it; borrowed from the ticket
+    uint64_t ticket = 0;
+};
+
+struct Region {
+    void *base = nullptr;
+    size_t slot_bytes = 0;
+    int32_t n_slots = 0;
+    std::vector<uint64_t> occupant;  // chunk id per slot
+    std::vector<uint8_t> used;
+    cudaEvent_t last_use = nullptr;  // recorded by matkv_table_free
+    bool has_last_use = false;
+};
+
+struct Ticket {
+    cudaEvent_t done = nullptr;
+};
+
+}  // namespace matkv
+
+struct matkv_ctx {
+    matkv_config cfg;
+    int device = 0;
+    float scale = 0.f;
+    int n_sm = 0;
+    int32_t *d_status = nullptr;
+    void *workspace = nullptr;
+    size_t workspace_bytes = 0;
+    int64_t opt_decode_ctas = 0, opt_prefill_impl = 0, opt_prefill_ctas = 0;
+    std::unordered_map<uint64_t, matkv::Chunk> chunks;
+    std::map<void *, matkv::Region *> regions;
+    std::unordered_map<uint64_t, matkv::Ticket> tickets;
+    uint64_t next_ticket = 1;
+    std::vector<matkv_table *> tables;
+};
+
+struct matkv_table {
+    matkv_ctx *ctx = nullptr;
+    int32_t batch = 0;
+    int32_t n_seg_total = 0;
+    std::vector<matkv::DevSeg> h_segs;
+    std::vector<matkv::DevReq> h_reqs;
+    int32_t tail_len_host = 0;   // host mirror (not moved by graph replays)
+    int32_t max_chunk_tiles = 0;
+    int64_t total_chunk_tiles = 0;
+    void *h_pinned = nullptr;    // pinned upload image
+    void *d_image = nullptr;     // device image: segs | reqs | tail_len[B]
+    size_t image_bytes = 0;
+    matkv::DevSeg *d_segs = nullptr;
+    matkv::DevReq *d_reqs = nullptr;
+    int32_t *d_tail_len = nullptr;
+    __nv_bfloat16 *tail_k = nullptr, *tail_v = nullptr;
+    std::vector<matkv::Region *> regions;  // staged regions this table reads
+};
+
+namespace matkv {
+
+int fail(int code, const char *fmt, ...);   // records the thread-local message, returns code
+int cuda_fail(cudaError_t e, const char *what);
+#define MATKV_CUDA(x)                                              \
+    do {                                                           \
+        cudaError_t e__ = (x);                                     \
+        if (e__ != cudaSuccess) return ::matkv::cuda_fail(e__, #x); \
+    } while (0)
+
+// Workspace layout: [counters: int32 x n_counter_slots][lse parts: fp32][o parts: fp32]
+struct WorkspaceView {
+    int32_t *counters;
+    float *part_lse;   // [n_part_slots][G]
+    float *part_o;     // [n_part_slots][G][D]
+    int64_t n_counter_slots, n_part_slots;
+};
+size_t workspace_bytes_for(const matkv_config &c, WorkspaceView *view_from_base, void *base);
+
+// ---- launchers (defined next to their kernels) ----------------------------------------------
+struct AttendArgs {
+    // which units
+    int32_t layer0, n_layers_launch, S;
+    // inputs / outputs (bf16 device) and their element strides per (layer, request, suffix token)
+    const __nv_bfloat16 *q, *k_new, *v_new;
+    __nv_bfloat16 *out;
+    float *lse_out;
+    int64_t q_sl, q_sb, q_ss;     // q / out strides: layer, request, token (elements)
+    int64_t kn_sl, kn_sb, kn_ss;  // k_new / v_new strides
+    int64_t lse_sl, lse_sb, lse_ss;
+};
+int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
+int launch_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts,
+                       const float *lse_parts, void *out, float *lse_out, cudaStream_t stream);
+int launch_gather(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out,
+                  int64_t rows, cudaStream_t stream);
+int launch_add_tail_len(matkv_table *t, int32_t delta, int32_t set_value, bool set, cudaStream_t stream);
+
+}  // namespace matkv

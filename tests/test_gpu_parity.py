@@ -1,0 +1,261 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import matkv_inputs as mi
+import oracle
+from _util import check, rand_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def _session(L, Hq, Hkv, D, B, max_chunks, max_tail, **kw):
+    from paper_2512_22195_b200.harness import Session
+    return Session(L, Hq, Hkv, D, B, max_chunks, max_tail, **kw)
+
+
+def _dev(a):
+    from paper_2512_22195_b200.harness import bits_to_dev
+    return bits_to_dev(a)
+
+
+def _bits(t):
+    from paper_2512_22195_b200.harness import dev_to_bits
+    return dev_to_bits(t)
+
+
+def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=False, q_shift=0, cap=None,
+                 prefill_impl=0):
+    """Prefill S tokens then T decode steps for a batch; compare every output with the oracle."""
+    import paper_2512_22195_b200 as mk
+    B = len(lens_per_req)
+    cap = cap or (S + T)
+    sess = _session(L, Hq, Hkv, D, B, max(1, max(len(x) for x in lens_per_req)), cap)
+    if ctas:
+        mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, ctas)
+    if prefill_impl:
+        mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_IMPL, prefill_impl)
+    sh = oracle.Shape(L, Hq, Hkv, D)
+    blobs, ids, cid = {}, [], 0
+    for r, lens in enumerate(lens_per_req):
+        row = []
+        for n in lens:
+            blobs[cid] = rand_bits(seed, 1000 + cid, (L, 2, Hkv, n, D))
+            sess.register_device_chunk(cid, blobs[cid])
+            row.append(cid)
+            cid += 1
+        ids.append(row)
+    sess.build_table(ids)
+    reqs = [oracle.Request(sh, [blobs[c] for c in row], cap) for row in ids]
+    worst = [0.0, 0.0, 0.0]
+
+    def upd(m):
+        for i in range(3):
+            worst[i] = max(worst[i], m[i])
+
+    if S > 0:
+        for layer in range(L):
+            q = rand_bits(seed, 10 + layer, (B, S, Hq, D), q_shift)
+            k = rand_bits(seed, 40 + layer, (B, S, Hkv, D))
+            v = rand_bits(seed, 70 + layer, (B, S, Hkv, D))
+            out, lse = sess.prefill(layer, _dev(q), _dev(k), _dev(v))
+            ob, lb = _bits(out), lse.cpu().numpy()
+            for r in range(B):
+                o_ref, l_ref = reqs[r].attend_new(layer, q[r], k[r], v[r])
+                upd(check(ob[r], o_ref, lb[r], l_ref, f"prefill layer {layer} req {r}"))
+        sess.advance(S)
+        for r in reqs:
+            r.advance(S)
+    for t in range(T):
+        q = rand_bits(seed, 2000 + t, (L, B, Hq, D), q_shift)
+        k = rand_bits(seed, 3000 + t, (L, B, Hkv, D))
+        v = rand_bits(seed, 4000 + t, (L, B, Hkv, D))
+        qd, kd, vd = _dev(q), _dev(k), _dev(v)
+        if all_layers:
+            out, lse = sess.decode_all_layers(qd, kd, vd)
+            ob, lb = _bits(out), lse.cpu().numpy()
+        else:
+            outs = [sess.decode(layer, qd[layer], kd[layer], vd[layer]) for layer in range(L)]
+            ob = np.stack([_bits(o) for o, _ in outs])
+            lb = np.stack([l.cpu().numpy() for _, l in outs])
+        for layer in range(L):
+            for r in range(B):
+                o_ref, l_ref = reqs[r].attend_new(layer, q[layer, r][None], k[layer, r][None], v[layer, r][None])
+                upd(check(ob[layer, r], o_ref[0], lb[layer, r], l_ref[0], f"decode step {t} layer {layer} req {r}"))
+        sess.advance(1)
+        for r in reqs:
+            r.advance(1)
+    # the tails the kernels wrote must equal the oracle's bookkeeping bit for bit
+    tk, tv = _bits(sess.tail_k), _bits(sess.tail_v)
+    for r in range(B):
+        n = reqs[r].tail_len
+        assert np.array_equal(tk[r, :, :, :n], reqs[r].tail_k[:, :, :n]) and np.array_equal(tv[r, :, :, :n], reqs[r].tail_v[:, :, :n])
+    assert sess.status() == 0
+    sess.close()
+    return worst
+
+
+def test_cfg1_full():
+    """Config 1: 1 layer, 8 q heads / 2 kv heads, D=64, 2 chunks x 128, 16-token suffix, 8 decode steps."""
+    w = mi.workload("cfg1")
+    run_requests(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, [[128, 128]], w.suffix, w.decode_steps, seed=0)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (4, 4, 128), (8, 4, 128), (32, 8, 128), (64, 8, 128), (8, 1, 64), (2, 2, 64)])
+def test_head_shapes(Hq, Hkv, D):
+    run_requests(2, Hq, Hkv, D, [[40, 7], [129]], 5, 3, seed=21)
+
+
+@pytest.mark.parametrize("lens", [[[1]], [[7, 127, 129, 1000]], [[]], [[33], [], [1, 1, 1]], [[64, 64], [32]]])
+def test_ragged_chunks_and_empty_lists(lens):
+    run_requests(1, 8, 2, 64, lens, 3, 4, seed=22)
+
+
+def test_tail_crosses_tile_boundaries():
+    run_requests(1, 4, 2, 128, [[50]], 30, 40, seed=23)           # tail grows through 32 and 64
+
+
+def test_all_layers_launch_matches_oracle():
+    run_requests(3, 8, 2, 128, [[200, 31], [97]], 4, 3, seed=24, all_layers=True)
+
+
+def test_peaky_queries():
+    run_requests(1, 8, 2, 128, [[300, 300]], 8, 4, seed=25, q_shift=3)   # q scaled by 8: sharp softmax
+
+
+@pytest.mark.parametrize("ctas", [1, 2, 3, 7, 0])
+def test_p7_split_count_invariance(ctas):
+    run_requests(2, 8, 2, 128, [[500, 77, 260]], 2, 3, seed=26, ctas=ctas)
+
+
+def test_p7_combine_kernel_alone():
+    import paper_2512_22195_b200 as mk
+    sess = _session(1, 8, 2, 64, 1, 1, 8)
+    rng = np.random.default_rng(3)
+    for n_rows, P, D in [(5, 1, 64), (9, 7, 128), (3, 40, 128), (2, 33, 32)]:
+        o_parts = rng.normal(size=(n_rows, P, D)).astype(np.float32)
+        lse_parts = (rng.normal(size=(n_rows, P)) * 4).astype(np.float32)
+        lse_parts[0, 0] = -np.inf
+        if P > 1:
+            lse_parts[1, :] = -np.inf
+            lse_parts[1, 1] = 0.5
+        op, lp = torch.from_numpy(o_parts).cuda(), torch.from_numpy(lse_parts).cuda()
+        out = torch.empty((n_rows, D), dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty(n_rows, dtype=torch.float32, device="cuda")
+        mk.matkv_lse_combine(sess.ctx, n_rows, P, D, op.data_ptr(), lp.data_ptr(), out.data_ptr(), lse.data_ptr())
+        ob, lb = _bits(out), lse.cpu().numpy()
+        for r in range(n_rows):
+            o_ref, l_ref = oracle.lse_merge(o_parts[r].astype(np.float64), lse_parts[r].astype(np.float64))
+            if np.isneginf(l_ref):
+                assert np.all(ob[r] == 0) and np.isneginf(lb[r])
+                continue
+            o = mi.bf16_bits_to_f64(ob[r])
+            assert np.max(np.abs(o - o_ref)) <= 2 ** -8 * max(1.0, np.max(np.abs(o_ref))) and abs(lb[r] - l_ref) <= 1e-4
+    sess.close()
+
+
+def test_p4_needle_on_gpu():
+    """A planted dominant key at every segment edge, tile edge and the causal edge of the tail."""
+    L, Hq, Hkv, D = 1, 4, 2, 128
+    lens = [33, 64, 1, 95]
+    sess = _session(L, Hq, Hkv, D, 1, 4, 40)
+    seed, g, h = 31, 1, 3
+    q = rand_bits(seed, 1, (1, Hq, D))
+    qv = mi.bf16_bits_to_f64(q[0, h])
+    needle = mi.f32_to_bf16_bits((qv * 16.0).astype(np.float32))
+    blobs = [rand_bits(seed, 10 + i, (L, 2, Hkv, n, D)) for i, n in enumerate(lens)]
+    spots = [(c, t) for c, n in enumerate(lens) for t in sorted({0, n - 1, min(31, n - 1), min(32, n - 1)})]
+    k_new, v_new = rand_bits(seed, 2, (1, Hkv, D)), rand_bits(seed, 3, (1, Hkv, D))
+    for trial, (c, t) in enumerate(spots):
+        bl = [b.copy() for b in blobs]
+        bl[c][0, 0, g, t] = needle
+        for i, b in enumerate(bl):
+            sess.register_device_chunk(100 * trial + i, b)
+        sess.build_table([[100 * trial + i for i in range(4)]])
+        out, _ = sess.decode(0, _dev(q), _dev(k_new), _dev(v_new))
+        o = mi.bf16_bits_to_f64(_bits(out))[0, h]
+        want = mi.bf16_bits_to_f64(bl[c][0, 1, g, t])
+        assert np.max(np.abs(o - want)) <= 2 ** -7 * np.max(np.abs(want)) + 1e-6, (c, t)
+    # needle as the new token itself (tail[v-1]) is visible
+    kn = k_new.copy()
+    kn[0, g] = needle
+    out, _ = sess.decode(0, _dev(q), _dev(kn), _dev(v_new))
+    o = mi.bf16_bits_to_f64(_bits(out))[0, h]
+    want = mi.bf16_bits_to_f64(v_new[0, g])
+    assert np.max(np.abs(o - want)) <= 2 ** -7 * np.max(np.abs(want)) + 1e-6
+    # a needle sitting in the tail one past the visible range must not be seen
+    sess.tail_k[0, 0, g, 1] = _dev(needle)
+    out2, _ = sess.decode(0, _dev(q), _dev(k_new), _dev(v_new))
+    sess.tail_k[0, 0, g, 1] = 0
+    out3, _ = sess.decode(0, _dev(q), _dev(k_new), _dev(v_new))
+    assert np.array_equal(_bits(out2), _bits(out3))
+    sess.close()
+
+
+def test_p5_p6_order_and_duplicates_on_gpu():
+    L, Hq, Hkv, D = 1, 8, 2, 64
+    sess = _session(L, Hq, Hkv, D, 3, 4, 8)
+    seed = 32
+    blobs = [rand_bits(seed, 10 + i, (L, 2, Hkv, n, D)) for i, n in enumerate([70, 33, 128])]
+    for i, b in enumerate(blobs):
+        sess.register_device_chunk(i, b)
+    q = rand_bits(seed, 1, (3, Hq, D))
+    q[1], q[2] = q[0], q[0]
+    kn = np.repeat(rand_bits(seed, 2, (1, Hkv, D)), 3, axis=0)
+    vn = np.repeat(rand_bits(seed, 3, (1, Hkv, D)), 3, axis=0)
+    sess.build_table([[0, 1, 2], [2, 0, 1], [1, 2, 0]])
+    out, lse = sess.decode(0, _dev(q), _dev(kn), _dev(vn))
+    o, l = mi.bf16_bits_to_f64(_bits(out)), lse.cpu().numpy()
+    assert np.max(np.abs(o[0] - o[1])) <= 2 ** -7 and np.max(np.abs(o[0] - o[2])) <= 2 ** -7
+    assert np.max(np.abs(l[0] - l[1])) <= 1e-4 and np.max(np.abs(l[0] - l[2])) <= 1e-4
+    # [A, A] against [A]: same o, lse larger by ln 2 -- compare through the oracle (the new token is also seen)
+    sh = oracle.Shape(L, Hq, Hkv, D)
+    sess.build_table([[0, 0], [0], []])
+    out, lse = sess.decode(0, _dev(q), _dev(kn), _dev(vn))
+    ob, lb = _bits(out), lse.cpu().numpy()
+    for r, ch in enumerate([[blobs[0], blobs[0]], [blobs[0]], []]):
+        o_ref, l_ref = oracle.Request(sh, ch, 8).attend_new(0, q[r][None], kn[r][None], vn[r][None])
+        check(ob[r], o_ref[0], lb[r], l_ref[0], f"dup case {r}")
+    sess.close()
+
+
+def test_cfg2_shape_two_layers_sampled_steps():
+    """Llama-3-8B head shape, 5 x 1,024-token chunks, 64-token suffix, 128 decode steps, 2 layers;
+    all steps run on the GPU, the oracle checks the prefill of layer 1 rows {0, 31, 63} and decode
+    steps {0, 1, 63, 127} (every layer, every head)."""
+    L, Hq, Hkv, D, S, T = 2, 32, 8, 128, 64, 128
+    seed = 1
+    sess = _session(L, Hq, Hkv, D, 1, 5, S + T)
+    sh = oracle.Shape(L, Hq, Hkv, D)
+    blobs = [rand_bits(seed, 1000 + i, (L, 2, Hkv, 1024, D)) for i in range(5)]
+    for i, b in enumerate(blobs):
+        sess.register_device_chunk(i, b)
+    sess.build_table([list(range(5))])
+    req = oracle.Request(sh, blobs, S + T)
+    for layer in range(L):
+        q, k, v = rand_bits(seed, 10 + layer, (1, S, Hq, D)), rand_bits(seed, 40 + layer, (1, S, Hkv, D)), rand_bits(seed, 70 + layer, (1, S, Hkv, D))
+        out, lse = sess.prefill(layer, _dev(q), _dev(k), _dev(v))
+        req.append_only(layer, k[0], v[0])
+        if layer == 1:
+            rows = [0, 31, 63]
+            o_ref, l_ref = oracle.attend(sh, layer, blobs, req.tail_k[layer], req.tail_v[layer], q[0][rows], [r + 1 for r in rows])
+            check(_bits(out)[0][rows], o_ref, lse.cpu().numpy()[0][rows], l_ref, "cfg2 prefill")
+    sess.advance(S)
+    req.advance(S)
+    for t in range(T):
+        q, k, v = rand_bits(seed, 2000 + t, (L, 1, Hq, D)), rand_bits(seed, 3000 + t, (L, 1, Hkv, D)), rand_bits(seed, 4000 + t, (L, 1, Hkv, D))
+        out, lse = sess.decode_all_layers(_dev(q), _dev(k), _dev(v))
+        for layer in range(L):
+            req.append_only(layer, k[layer], v[layer])
+        if t in (0, 1, 63, 127):
+            ob, lb = _bits(out), lse.cpu().numpy()
+            for layer in range(L):
+                o_ref, l_ref = oracle.attend(sh, layer, blobs, req.tail_k[layer], req.tail_v[layer], q[layer], [req.tail_len + 1])
+                check(ob[layer], o_ref, lb[layer], l_ref, f"cfg2 decode step {t} layer {layer}")
+        sess.advance(1)
+        req.advance(1)
+    assert sess.status() == 0
+    sess.close()

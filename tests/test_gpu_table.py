@@ -1,0 +1,137 @@
+"""GPU tests of the chunk table, the bit-exact gather, staging and the host-side error paths."""
+import numpy as np
+import pytest
+import torch
+
+from _util import rand_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def _mk():
+    import paper_2512_22195_b200 as mk
+    from paper_2512_22195_b200.harness import Session, bits_to_dev, dev_to_bits
+    return mk, Session, bits_to_dev, dev_to_bits
+
+
+def test_p8_gather_is_bit_exact_with_shared_and_ragged_chunks():
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D = 2, 4, 2, 64
+    sess = Session(L, Hq, Hkv, D, 3, 5, 16)
+    lens = [1, 7, 127, 129, 300]
+    blobs = [rand_bits(41, i, (L, 2, Hkv, n, D)) for i, n in enumerate(lens)]
+    for i, b in enumerate(blobs):
+        sess.register_device_chunk(i, b)
+    ids = [[4, 0, 2], [2, 2, 1, 3], []]
+    sess.build_table(ids)
+    # put something in the tails too
+    tk, tv = rand_bits(41, 90, (3, L, Hkv, 16, D)), rand_bits(41, 91, (3, L, Hkv, 16, D))
+    sess.tail_k.copy_(to_dev(tk)); sess.tail_v.copy_(to_dev(tv))
+    mk.matkv_table_set_tail_len(sess.table, 5)
+    for r, row in enumerate(ids):
+        for layer in range(L):
+            rows = sum(lens[c] for c in row) + 5
+            k, v = sess.gather(layer, r, rows)
+            want_k = np.concatenate([blobs[c][layer, 0] for c in row] + [tk[r, layer, :, :5]], axis=1)
+            want_v = np.concatenate([blobs[c][layer, 1] for c in row] + [tv[r, layer, :, :5]], axis=1)
+            assert np.array_equal(to_bits(k), want_k) and np.array_equal(to_bits(v), want_v)
+    assert sess.status() == 0
+    sess.close()
+
+
+def test_staging_then_gather_bit_exact_and_overlap_bookkeeping():
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D, n = 2, 4, 2, 64, 96
+    sess = Session(L, Hq, Hkv, D, 2, 3, 8)
+    blobs = [rand_bits(42, i, (L, 2, Hkv, n, D)) for i in range(5)]
+    for i, b in enumerate(blobs):
+        sess.register_host_chunk(i, b)
+    slot_bytes = blobs[0].nbytes
+    assert slot_bytes % 256 == 0
+    slots_a = torch.empty(3 * slot_bytes, dtype=torch.uint8, device="cuda")
+    slots_b = torch.empty(3 * slot_bytes, dtype=torch.uint8, device="cuda")
+    copy = torch.cuda.Stream()
+    # not staged yet -> the table cannot be built
+    with pytest.raises(mk.MatkvError) as e:
+        sess.build_table([[0, 1], [1]])
+    assert e.value.code == mk.E_NOT_STAGED
+    t1 = sess.stage([0, 1, 1, 0], slots_a, slot_bytes, copy)           # duplicates are copied once
+    sess.build_table([[0, 1], [1]])                                    # stream waits for the copies, host does not
+    k, v = sess.gather(1, 0, 2 * n)
+    assert np.array_equal(to_bits(k), np.concatenate([blobs[0][1, 0], blobs[1][1, 0]], axis=1))
+    # next batch goes to the other region while the first table is alive
+    t2 = sess.stage([2, 3, 4], slots_b, slot_bytes, copy)
+    mk.matkv_stage_wait(sess.ctx, t2)
+    assert mk.matkv_stage_query(sess.ctx, t1) and mk.matkv_stage_query(sess.ctx, t2)
+    sess.build_table([[4, 2], [3]])
+    k, v = sess.gather(0, 0, 2 * n)
+    assert np.array_equal(to_bits(v), np.concatenate([blobs[4][0, 1], blobs[2][0, 1]], axis=1))
+    # re-staging into region A evicts chunk 0 but keeps chunk 1 in place (no new copy needed)
+    sess.stage([1, 2], slots_a, slot_bytes, copy)
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_build_chunk_table(sess.ctx, [[0]], sess.tail_k.data_ptr(), sess.tail_v.data_ptr())
+    assert e.value.code == mk.E_NOT_STAGED
+    sess.build_table([[1, 2], [2]])
+    k, v = sess.gather(1, 1, n)
+    assert np.array_equal(to_bits(k), blobs[2][1, 0])
+    # too many distinct chunks for the region
+    with pytest.raises(mk.MatkvError) as e:
+        sess.stage([0, 1, 2, 3], slots_a, slot_bytes, copy)
+    assert e.value.code == mk.E_CAPACITY
+    sess.close()
+
+
+def test_host_side_error_paths():
+    mk, Session, to_dev, to_bits = _mk()
+    with pytest.raises(mk.MatkvError):
+        mk.matkv_create(1, 8, 3, 64, 1, 1, 8)             # heads do not divide
+    with pytest.raises(mk.MatkvError):
+        mk.matkv_create(1, 8, 2, 96, 1, 1, 8)             # unsupported head_dim
+    sess = Session(1, 8, 2, 64, 2, 2, 4)
+    blob = rand_bits(43, 0, (1, 2, 2, 8, 64))
+    sess.register_device_chunk(7, blob)
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_register_chunk(sess.ctx, 7, 8, None, sess.chunks[7].data_ptr())     # duplicate id
+    assert e.value.code == mk.E_INVALID_ARG
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_register_chunk(sess.ctx, 8, 8, None, sess.chunks[7].data_ptr() + 2)  # misaligned
+    assert e.value.code == mk.E_ALIGNMENT
+    with pytest.raises(mk.MatkvError) as e:
+        sess.build_table([[99]])
+    assert e.value.code == mk.E_UNKNOWN_CHUNK
+    with pytest.raises(mk.MatkvError) as e:
+        sess.build_table([[7, 7, 7]])                                             # more than max_chunks_per_req
+    assert e.value.code == mk.E_CAPACITY
+    with pytest.raises(mk.MatkvError) as e:
+        sess.build_table([[7], [7], [7]])                                         # batch > max_batch
+    assert e.value.code == mk.E_CAPACITY
+    sess.build_table([[7], []])
+    q = to_dev(rand_bits(43, 1, (2, 5, 8, 64)))
+    kv = to_dev(rand_bits(43, 2, (2, 5, 2, 64)))
+    with pytest.raises(mk.MatkvError) as e:
+        sess.prefill(0, q, kv, kv)                                               # 5 tokens > tail capacity 4
+    assert e.value.code == mk.E_CAPACITY
+    with pytest.raises(mk.MatkvError) as e:
+        sess.decode(3, q[:, 0], kv[:, 0], kv[:, 0])                              # layer out of range
+    assert e.value.code == mk.E_INVALID_ARG
+    mk.matkv_table_set_tail_len(sess.table, 4)
+    with pytest.raises(mk.MatkvError) as e:
+        sess.decode(0, q[:, 0], kv[:, 0], kv[:, 0])                              # tail full
+    assert e.value.code == mk.E_CAPACITY
+    mk.matkv_unregister_chunk(sess.ctx, 7)
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_unregister_chunk(sess.ctx, 7)
+    assert e.value.code == mk.E_UNKNOWN_CHUNK
+    assert sess.status() == 0
+    sess.close()
+
+
+def test_device_generator_matches_host_generator():
+    import matkv_inputs as mi
+    import matkv_inputs.device as gen
+    _, _, _, to_bits = _mk()
+    t = torch.empty(100003, dtype=torch.bfloat16, device="cuda")
+    gen.fill_bf16(t, seed=5, stream=77, shift=0, start=12345)
+    assert np.array_equal(to_bits(t), mi.normal_bf16(5, 77, 100003, 0, start=12345))
+    gen.fill_bf16(t, seed=5, stream=78, shift=3, start=0)
+    assert np.array_equal(to_bits(t), mi.normal_bf16(5, 78, 100003, 3))
