@@ -5,8 +5,8 @@
 // [c*W/n, (c+1)*W/n) of that list, so every SM streams the same number of bytes whatever the shape.
 // Inside a CTA one producer thread walks its range and moves each tile's K rows and V rows from the
 // scattered chunk blobs (or the tail, or the new tokens) into a shared-memory ring with bulk
-// asynchronous copies (cp.async.bulk + mbarrier complete_tx); eight consumer warps each take every
-// eighth tile and run an independent online softmax for the G query heads that share the KV head
+// asynchronous copies (cp.async.bulk + mbarrier complete_tx); seven consumer warps each take every
+// seventh tile and run an independent online softmax for the G query heads that share the KV head
 // (fp32, exp2-based).  At the end of a unit the warps' states are merged through shared memory; a
 // unit that spans several CTAs leaves one partial (normalised o, lse) per CTA in the workspace and
 // the last CTA to arrive (atomic ticket, no waiting) merges them by log-sum-exp.
@@ -20,7 +20,7 @@
 
 namespace matkv {
 
-constexpr int kConsumerWarps = 8;
+constexpr int kConsumerWarps = 7;  // registers are allocated to warps in fours: 8 warps x 255 registers fill the file
 constexpr int kThreads = (kConsumerWarps + 1) * 32;
 constexpr int kMaxDynSmem = 232448;            // 227 KB opt-in limit per CTA on sm_100
 constexpr long long kWaitCycles = 2000000000LL;  // bounded waits give up after about a second
@@ -298,8 +298,9 @@ struct StreamCfg {
     static constexpr int NF = NP / LPR;                        // scores per lane after the reduce-scatter
     static constexpr int LPH = LPR / G;                        // lanes of a group that end up with the same head
     static constexpr int SLOT_BYTES = kTile * D * 2;
-    static constexpr int MERGE_BYTES = kConsumerWarps * G * (D + 2) * 4;
-    static constexpr int PS_BYTES = kConsumerWarps * (kTile * G + G) * 4;
+    static constexpr int MERGE_BYTES = (kConsumerWarps * G * (D + 2) * 4 + 15) / 16 * 16;
+    static constexpr int PS_STRIDE = (kTile * G + G + 3) / 4 * 4;  // floats per warp, 16-byte multiple
+    static constexpr int PS_BYTES = kConsumerWarps * PS_STRIDE * 4;
     static constexpr int FIXED_BYTES = MERGE_BYTES + PS_BYTES + 1024;
     static constexpr int NSLOT_MAX = ((kMaxDynSmem - FIXED_BYTES) / SLOT_BYTES) & ~1;
     static constexpr int NSLOT = NSLOT_MAX > 24 ? 24 : NSLOT_MAX;
@@ -308,15 +309,15 @@ struct StreamCfg {
 };
 
 template <int D, int G>
-__global__ void __maxnreg__(224) k_attend_stream(const StreamParams p) {
+__global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParams p) {
     using C = StreamCfg<D, G>;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char *ring = smem;
     float *merge_o = (float *)(smem + C::NSLOT * C::SLOT_BYTES);         // [warp][G][D]
     float *merge_m = merge_o + kConsumerWarps * G * D;                   // [warp][G]
     float *merge_l = merge_m + kConsumerWarps * G;                       // [warp][G]
-    float *ps_all = merge_l + kConsumerWarps * G;                        // [warp][kTile*G + G]
-    unsigned char *misc = (unsigned char *)(ps_all + kConsumerWarps * (kTile * G + G));
+    float *ps_all = (float *)(smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES);  // [warp][PS_STRIDE]
+    unsigned char *misc = smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES + C::PS_BYTES;
     uint64_t *bars = (uint64_t *)misc;                                   // full[NSLOT], empty[NSLOT]
     CtaRange *range = (CtaRange *)(misc + 2 * 24 * 8);
     volatile int *flags = (volatile int *)(misc + 2 * 24 * 8 + sizeof(CtaRange) + 8);  // [0] abort, [1] last arriver
@@ -388,7 +389,7 @@ __global__ void __maxnreg__(224) k_attend_stream(const StreamParams p) {
     // ================= consumers =================
     const int grp = lane / C::LPR, jl = lane % C::LPR;
     const int my_h = jl / C::LPH;  // head whose scores this lane holds after the reduce-scatter
-    float *ps = ps_all + warp * (kTile * G + G);  // this warp's p[row][head], then alpha[head]
+    float *ps = ps_all + warp * C::PS_STRIDE;  // this warp's p[row][head], then alpha[head]
     float *alpha_s = ps + kTile * G;
 
     float qf[G][C::DPL];

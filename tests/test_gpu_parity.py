@@ -179,7 +179,10 @@ def test_p4_needle_on_gpu():
         o = mi.bf16_bits_to_f64(_bits(out))[0, h]
         want = mi.bf16_bits_to_f64(bl[c][0, 1, g, t])
         assert np.max(np.abs(o - want)) <= 2 ** -7 * np.max(np.abs(want)) + 1e-6, (c, t)
-    # needle as the new token itself (tail[v-1]) is visible
+    # needle as the new token itself (tail[v-1]) is visible (clean chunks: no other needle around)
+    for i, b in enumerate(blobs):
+        sess.register_device_chunk(9000 + i, b)
+    sess.build_table([[9000 + i for i in range(4)]])
     kn = k_new.copy()
     kn[0, g] = needle
     out, _ = sess.decode(0, _dev(q), _dev(kn), _dev(v_new))
