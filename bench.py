@@ -1,0 +1,425 @@
+#!/usr/bin/env python
+"""Benchmark of the attention path over materialised KV chunks (one JSON line on stdout).
+
+A "step" is one pass of the whole hot path for one request batch: build the chunk table, run the
+query sub-prefill for every layer, then T decode steps over every layer (split-KV partials merged
+by log-sum-exp inside the same launches).  `value` is decode tokens per second of that whole step
+with every input already resident in HBM; `e2e` repeats it through the same C-ABI calls starting
+from HOST buffers (chunk blobs staged from pinned host memory, q/k/v copied in per step, outputs
+copied back).  The numbers are attention-path only (no model weights, no MLP).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--decode-launch all_layers|per_layer]
+  python bench.py --impl reference ...      # the CPU oracle as it stands, on the host cores
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import matkv_inputs as mi  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per decode launch from the committed ncu capture (profiles/), by workload and launch mode.
+NCU_TRAFFIC_BYTES = {}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+# ---- clocks ------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], None, set()
+        for ts, line in self.rows:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7 or not (t0 - 0.05 <= ts <= t1 + 0.15):
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx = float(f[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---- the CPU oracle legs -------------------------------------------------------------------------
+class OracleState:
+    """Host copies of one batch and the oracle's requests (used by cpu_baseline and --impl reference)."""
+
+    def __init__(self, w: mi.Workload, host_chunks, ids):
+        import oracle
+        self.oracle, self.w = oracle, w
+        self.sh = oracle.Shape(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim)
+        cap = w.suffix + w.decode_steps
+        self.reqs = [oracle.Request(self.sh, [host_chunks[c] for c in row], cap) for row in ids]
+        self.cores = os.cpu_count() or 1
+        # the tail as it stands after the sub-prefill: appended without attending (bookkeeping only)
+        for layer in range(w.n_layers):
+            _, k, v = mi.prefill_inputs(w, layer)
+            for r, rq in enumerate(self.reqs):
+                rq.append_only(layer, k[r], v[r])
+        for rq in self.reqs:
+            rq.advance(w.suffix)
+
+    def decode_steps(self, first_step: int, n_steps: int):
+        """Time n_steps decode steps (all layers, all requests) on all host cores; returns seconds."""
+        w = self.w
+        t0 = time.perf_counter()
+        with ThreadPoolExecutor(max_workers=self.cores) as ex:
+            for s in range(first_step, first_step + n_steps):
+                q, k, v = mi.decode_inputs(w, s)
+                jobs = [(layer, r) for layer in range(w.n_layers) for r in range(w.batch)]
+                list(ex.map(lambda lr: self.reqs[lr[1]].attend_new(lr[0], q[lr[0], lr[1]][None], k[lr[0], lr[1]][None],
+                                                                   v[lr[0], lr[1]][None]), jobs))
+                for rq in self.reqs:
+                    rq.advance(1)
+        return time.perf_counter() - t0
+
+    def rewind(self, n_steps: int):
+        for rq in self.reqs:
+            rq.tail_len -= n_steps
+
+
+def host_chunks_numpy(w: mi.Workload, needed):
+    return {c: mi.chunk_blob(w, c) for c in needed}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on this machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    w = mi.workload(args.workload)
+    ids = w.chunk_ids(0)
+    needed = sorted({c for row in ids for c in row})
+    log(f"[reference] generating {len(needed)} chunks on the host ...")
+    st = OracleState(w, host_chunks_numpy(w, needed), ids)
+    per_step = 1  # each bench step = one decode step of the workload over all layers and requests
+    for _ in range(args.warmup):
+        st.decode_steps(0, per_step)
+        st.rewind(per_step)
+    t = 0.0
+    for _ in range(args.steps):
+        t += st.decode_steps(0, per_step)
+        st.rewind(per_step)
+    tok_s = args.steps * per_step * w.batch / t
+    sample = f"decode step 0 of {w.name} (all {w.n_layers} layers, batch {w.batch}), repeated per bench step"
+    print(json.dumps({
+        "impl": "reference", "metric": "decode_tokens_per_s", "value": tok_s, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": st.cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+# ---- the CUDA arm ----------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="matkv", choices=["matkv", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--decode-launch", default="all_layers", choices=["all_layers", "per_layer"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--decode-ctas", type=int, default=0)
+    ap.add_argument("--no-other-mode", action="store_true", help="skip the second pass in the other decode launch mode")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2512_22195_b200 as mk
+    import matkv_inputs.device as gen
+    from paper_2512_22195_b200.harness import Session
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    w = mi.workload(args.workload)
+    L, B, S, T, Hq, Hkv, D = w.n_layers, w.batch, w.suffix, w.decode_steps, w.n_q_heads, w.n_kv_heads, w.head_dim
+    ids = w.chunk_ids(0)
+    needed = sorted({c for row in ids for c in row})
+    sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
+    if args.decode_ctas:
+        mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, args.decode_ctas)
+    # every rank works on its own replica of the batch (independent requests: no data-path collective)
+    chunks = {}
+    for c in needed:
+        t_ = torch.empty((L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
+        gen.fill_bf16(t_, w.seed, mi.STREAM_CHUNK + c)
+        chunks[c] = t_
+        sess.register_device_chunk(c, t_)
+    q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device=dev)
+    k_pf = torch.empty((L, B, S, Hkv, D), dtype=torch.bfloat16, device=dev)
+    v_pf = torch.empty_like(k_pf)
+    gen.fill_bf16(q_pf, w.seed, mi.STREAM_Q_PREFILL)
+    gen.fill_bf16(k_pf, w.seed, mi.STREAM_K_PREFILL)
+    gen.fill_bf16(v_pf, w.seed, mi.STREAM_V_PREFILL)
+    q_dc = torch.empty((T, L, B, Hq, D), dtype=torch.bfloat16, device=dev)
+    k_dc = torch.empty((T, L, B, Hkv, D), dtype=torch.bfloat16, device=dev)
+    v_dc = torch.empty_like(k_dc)
+    gen.fill_bf16(q_dc, w.seed, mi.STREAM_Q_DECODE)
+    gen.fill_bf16(k_dc, w.seed, mi.STREAM_K_DECODE)
+    gen.fill_bf16(v_dc, w.seed, mi.STREAM_V_DECODE)
+    o_pf = torch.empty_like(q_pf)
+    o_dc = torch.empty_like(q_dc)
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.Stream(device=dev)
+    sp = stream.cuda_stream
+    ctx = sess.ctx
+    qs_l, ks_l = q_pf[0].numel() * 2, k_pf[0].numel() * 2
+    qd_t, kd_t = q_dc[0].numel() * 2, k_dc[0].numel() * 2
+    qd_l, kd_l = q_dc[0, 0].numel() * 2, k_dc[0, 0].numel() * 2
+    launches = {"n": 0}
+    ev_d0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev_d1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ev_p0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+
+    def one_step(q_pf_p, k_pf_p, v_pf_p, q_dc_p, k_dc_p, v_dc_p, timed_index=None, mode=args.decode_launch):
+        """All pointers are device addresses; nothing here but C-ABI calls."""
+        table = sess.build_table(ids, sp)
+        if timed_index is not None:
+            ev_p0[timed_index].record(stream)
+        for layer in range(L):
+            mk.matkv_attend_prefill(ctx, table, layer, S, q_pf_p + layer * qs_l, k_pf_p + layer * ks_l, v_pf_p + layer * ks_l,
+                                    o_pf.data_ptr() + layer * qs_l, None, sp)
+        mk.matkv_table_advance(table, S, sp)
+        if timed_index is not None:
+            ev_d0[timed_index].record(stream)
+        n = L + 1
+        for t in range(T):
+            if mode == "all_layers":
+                mk.matkv_attend_decode_all_layers(ctx, table, q_dc_p + t * qd_t, k_dc_p + t * kd_t, v_dc_p + t * kd_t,
+                                                  o_dc.data_ptr() + t * qd_t, None, sp)
+                n += 2
+            else:
+                for layer in range(L):
+                    mk.matkv_attend_decode(ctx, table, layer, q_dc_p + t * qd_t + layer * qd_l, k_dc_p + t * kd_t + layer * kd_l,
+                                           v_dc_p + t * kd_t + layer * kd_l, o_dc.data_ptr() + t * qd_t + layer * qd_l, None, sp)
+                n += L + 1
+            mk.matkv_table_advance(table, 1, sp)
+        if timed_index is not None:
+            ev_d1[timed_index].record(stream)
+        return n
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_region(fn, steps):
+        """K steps bracketed by barrier + synchronize; returns device milliseconds (max over ranks)."""
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0 = time.time()
+        e0.record(stream)
+        n = 0
+        for i in range(steps):
+            n += fn(i)
+        e1.record(stream)
+        barrier()
+        t1 = time.time()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            tt = torch.tensor([ms], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms = float(tt.item())
+        return ms, n, t0, t1
+
+    dev_ptrs = (q_pf.data_ptr(), k_pf.data_ptr(), v_pf.data_ptr(), q_dc.data_ptr(), k_dc.data_ptr(), v_dc.data_ptr())
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            one_step(*dev_ptrs)
+        sampler = ClockSampler(local) if rank == 0 else None
+        ms, n_launch, t0, t1 = timed_region(lambda i: one_step(*dev_ptrs, timed_index=i), args.steps)
+        clocks = sampler.stop(t0, t1) if sampler else None
+        st = sess.status()
+        if st != 0:
+            raise RuntimeError(f"device status {st} after the timed region")
+        dec_ms = sum(a.elapsed_time(b) for a, b in zip(ev_d0, ev_d1))
+        pre_ms = sum(a.elapsed_time(b) for a, b in zip(ev_p0, ev_d0))
+        # the other launch mode, for the record (same work, different launch granularity)
+        other = "per_layer" if args.decode_launch == "all_layers" else "all_layers"
+        dec_ms_o = None
+        if not args.no_other_mode:
+            one_step(*dev_ptrs, mode=other)
+            timed_region(lambda i: one_step(*dev_ptrs, timed_index=i, mode=other), min(args.steps, 5))
+            dec_ms_o = sum(a.elapsed_time(b) for a, b in zip(ev_d0[:min(args.steps, 5)], ev_d1[:min(args.steps, 5)]))
+
+    # algorithmic KV bytes of the decode loop of one step: every visible K and V element once
+    n_req = [sum(chunks[c].shape[3] for c in row) for row in ids]
+    kv_bytes_decode = sum((n + S + t + 1) * w.beta for n in n_req for t in range(T)) * L
+    kv_bytes_prefill = sum((n + S) * w.beta for n in n_req) * L
+    tokens = B * T * world
+    value = tokens * args.steps / (ms * 1e-3)
+    decode_launches = T * (1 if args.decode_launch == "all_layers" else L)
+    avg_launch_ms = dec_ms / (args.steps * decode_launches)
+    achieved = kv_bytes_decode / decode_launches / (avg_launch_ms * 1e-3) / 1e9
+    peaks, peak_kind = measured_peaks()
+    peak = float(peaks["hbm_gbs"])
+    result = {
+        "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 in, fp32 softmax/accumulate", "data": "synthetic",
+        "config": {"workload": w.name, "layers": L, "q_heads": Hq, "kv_heads": Hkv, "head_dim": D, "batch": B,
+                   "chunks_per_request": w.chunks_per_req, "chunk_tokens": w.chunk_tokens, "suffix": S, "decode_steps": T,
+                   "decode_launch": args.decode_launch, "l2": "inputs larger than L2 (KV per decode step = "
+                   f"{kv_bytes_decode / T / 1e6:.0f} MB vs 126 MB L2)", "multi_gpu": "independent replicas per rank"},
+        "gpu_launches": n_launch,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "k_attend_stream (decode)", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                     "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.decode_launch)),
+                     "algorithmic_bytes_per_launch": kv_bytes_decode / decode_launches,
+                     "avg_launch_us": avg_launch_ms * 1e3},
+        "phases": {"prefill_ms_per_step": pre_ms / args.steps, "decode_ms_per_step": dec_ms / args.steps,
+                   "decode_only_tokens_per_s": B * T * args.steps / (dec_ms * 1e-3),
+                   "decode_kv_gbs": kv_bytes_decode * args.steps / (dec_ms * 1e-3) / 1e9,
+                   "prefill_kv_gbs": kv_bytes_prefill * args.steps / (pre_ms * 1e-3) / 1e9,
+                   f"decode_only_tokens_per_s_{other}": (B * T * min(args.steps, 5) / (dec_ms_o * 1e-3)) if dec_ms_o else None},
+    }
+
+    # ---- end to end: the same step through the same calls, from host buffers --------------------
+    if not args.no_e2e:
+        copy = torch.cuda.Stream(device=dev)
+        host = {c: torch.empty(chunks[c].shape, dtype=torch.bfloat16, pin_memory=True) for c in needed}
+        for c in needed:
+            host[c].copy_(chunks[c])
+        hq_pf, hk_pf, hv_pf = (x.cpu().pin_memory() for x in (q_pf, k_pf, v_pf))
+        hq_dc, hk_dc, hv_dc = (x.cpu().pin_memory() for x in (q_dc, k_dc, v_dc))
+        ho_pf = torch.empty(o_pf.shape, dtype=torch.bfloat16, pin_memory=True)
+        ho_dc = torch.empty(o_dc.shape, dtype=torch.bfloat16, pin_memory=True)
+        torch.cuda.synchronize()
+        sess2 = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
+        for c in needed:
+            mk.matkv_register_chunk(sess2.ctx, c, w.chunk_tokens, host[c].data_ptr(), None)
+        slot_bytes = w.chunk_bytes
+        slots = [torch.empty(len(needed) * slot_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+        dq_pf, dk_pf, dv_pf = torch.empty_like(q_pf), torch.empty_like(k_pf), torch.empty_like(v_pf)
+        dq_dc, dk_dc, dv_dc = torch.empty_like(q_dc), torch.empty_like(k_dc), torch.empty_like(v_dc)
+        h2d = len(needed) * slot_bytes + sum(x.numel() * 2 for x in (hq_pf, hk_pf, hv_pf, hq_dc, hk_dc, hv_dc))
+        d2h = (ho_pf.numel() + ho_dc.numel()) * 2
+        ctx2 = sess2.ctx
+
+        def e2e_step(i):
+            # load: pinned host -> device slots on the copy stream; the compute stream waits through the table
+            sess2.stage(needed, slots[i % 2], slot_bytes, copy)
+            table = sess2.build_table(ids, sp)
+            dq_pf.copy_(hq_pf, non_blocking=True); dk_pf.copy_(hk_pf, non_blocking=True); dv_pf.copy_(hv_pf, non_blocking=True)
+            for layer in range(L):
+                mk.matkv_attend_prefill(ctx2, table, layer, S, dq_pf.data_ptr() + layer * qs_l, dk_pf.data_ptr() + layer * ks_l,
+                                        dv_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
+            mk.matkv_table_advance(table, S, sp)
+            ho_pf.copy_(o_pf, non_blocking=True)
+            for t in range(T):
+                dq_dc[t].copy_(hq_dc[t], non_blocking=True); dk_dc[t].copy_(hk_dc[t], non_blocking=True)
+                dv_dc[t].copy_(hv_dc[t], non_blocking=True)
+                mk.matkv_attend_decode_all_layers(ctx2, table, dq_dc.data_ptr() + t * qd_t, dk_dc.data_ptr() + t * kd_t,
+                                                  dv_dc.data_ptr() + t * kd_t, o_dc.data_ptr() + t * qd_t, None, sp) \
+                    if args.decode_launch == "all_layers" else [
+                        mk.matkv_attend_decode(ctx2, table, layer, dq_dc.data_ptr() + t * qd_t + layer * qd_l,
+                                               dk_dc.data_ptr() + t * kd_t + layer * kd_l, dv_dc.data_ptr() + t * kd_t + layer * kd_l,
+                                               o_dc.data_ptr() + t * qd_t + layer * qd_l, None, sp) for layer in range(L)]
+                mk.matkv_table_advance(table, 1, sp)
+                ho_dc[t].copy_(o_dc[t], non_blocking=True)      # the step's result goes back to the host
+            return 0
+
+        with torch.cuda.stream(stream):
+            for i in range(2):
+                e2e_step(i)
+            k_e2e = min(args.steps, 5)
+            ms_e, _, _, _ = timed_region(e2e_step, k_e2e)
+        if sess2.status() != 0:
+            raise RuntimeError("device status non-zero after the end-to-end region")
+        result["e2e"] = {"value": tokens * k_e2e / (ms_e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
+                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e,
+                         "h2d_gbs_if_copy_bound": h2d * k_e2e / (ms_e * 1e-3) / 1e9}
+        sess2.close()
+        del host, slots
+
+    # ---- the oracle on this machine's host cores, bounded sample (rank 0, N = 1 only) ------------------
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        from paper_2512_22195_b200.harness import dev_to_bits
+        host_np = {c: dev_to_bits(chunks[c]) for c in needed}
+        st_o = OracleState(w, host_np, ids)
+        t_one = st_o.decode_steps(0, 1)
+        n_s = int(max(1, min(T - 1, round(12.0 / max(t_one, 1e-3)))))
+        t_s = st_o.decode_steps(1, n_s)
+        result["cpu_baseline"] = {"value": n_s * B / t_s, "unit": "tokens/s", "cores": st_o.cores, "kind": "oracle",
+                                  "sample": f"decode steps 1..{n_s} of {T} of {w.name} (all {L} layers, batch {B}), "
+                                            f"{t_s:.1f} s on {st_o.cores} threads",
+                                  "kv_gbs": sum((n + S + t + 1) * w.beta for n in n_req for t in range(1, 1 + n_s)) * L / t_s / 1e9}
+    if rank == 0:
+        print(json.dumps(result), flush=True)
+    sess.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
