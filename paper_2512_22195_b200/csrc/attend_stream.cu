@@ -104,7 +104,7 @@ struct UnitPos {
     int32_t l_rel, b, i, g;  // layer (relative to layer0), request, suffix token, KV head
     int32_t tile;            // first tile of this CTA's share inside the unit
     int32_t rt;              // tiles in the unit
-    int32_t chunk_tiles, tail_tiles, t0;
+    int32_t chunk_tiles, tail_tiles, t0, seg_begin;
     int64_t flat_begin;      // flat index of the unit's first tile
 };
 
@@ -126,6 +126,7 @@ __device__ __forceinline__ void load_req(const StreamParams &p, UnitPos &u) {
     const DevReq rq = p.reqs[u.b];
     u.t0 = clamp_t0(p, u.b);
     u.chunk_tiles = rq.chunk_tiles;
+    u.seg_begin = rq.seg_begin;
     u.tail_tiles = ceil_div(u.t0, kTile);
 }
 __device__ __forceinline__ void set_rt(UnitPos &u) { u.rt = u.chunk_tiles + u.tail_tiles + ceil_div(u.i + 1, kTile); }
@@ -198,10 +199,12 @@ struct TileSrc {
     int32_t new_first;           // >= 0: tile holds new tokens new_first .. new_first+rows-1; else -1
 };
 
-// Sequential cursor over a request's segments (tile indices only ever grow inside a unit).
+// The producer's cursor over a request's segments.  Tile indices only grow inside a unit, so the
+// current segment stays in registers and global memory is touched once per segment, not per tile.
 struct SegCursor {
-    int32_t seg, tiles_before;
-    __device__ __forceinline__ void reset() { seg = 0; tiles_before = 0; }
+    int32_t seg, tiles_before, seg_tiles;
+    DevSeg sg;
+    __device__ __forceinline__ void reset() { seg = -1; tiles_before = 0; seg_tiles = 0; }
 };
 
 template <int D>
@@ -209,22 +212,19 @@ __device__ __forceinline__ TileSrc tile_source(const StreamParams &p, const Unit
     TileSrc s;
     const int layer = p.layer0 + u.l_rel;
     if (tile < u.chunk_tiles) {
-        const DevReq rq = p.reqs[u.b];
-        const DevSeg *segs = p.segs + rq.seg_begin;
-        int len = segs[cur.seg].len;
-        while (tile >= cur.tiles_before + ceil_div(len, kTile)) {
-            cur.tiles_before += ceil_div(len, kTile);
+        while (cur.seg < 0 || tile >= cur.tiles_before + cur.seg_tiles) {
+            cur.tiles_before += cur.seg_tiles;
             ++cur.seg;
-            len = segs[cur.seg].len;
+            cur.sg = p.segs[u.seg_begin + cur.seg];
+            cur.seg_tiles = ceil_div(cur.sg.len, kTile);
         }
-        const DevSeg sg = segs[cur.seg];
         const int r0 = (tile - cur.tiles_before) * kTile;
-        const int64_t kslab = ((int64_t)layer * 2 * p.Hkv + u.g) * sg.len;
-        const int64_t vslab = (((int64_t)layer * 2 + 1) * p.Hkv + u.g) * sg.len;
-        s.k = sg.base + (kslab + r0) * D;
-        s.v = sg.base + (vslab + r0) * D;
+        const int64_t kslab = ((int64_t)layer * 2 * p.Hkv + u.g) * cur.sg.len;
+        const int64_t vslab = (((int64_t)layer * 2 + 1) * p.Hkv + u.g) * cur.sg.len;
+        s.k = cur.sg.base + (kslab + r0) * D;
+        s.v = cur.sg.base + (vslab + r0) * D;
         s.row_stride = D;
-        s.rows = min(kTile, sg.len - r0);
+        s.rows = min(kTile, cur.sg.len - r0);
         s.new_first = -1;
     } else if (tile < u.chunk_tiles + u.tail_tiles) {
         const int r0 = (tile - u.chunk_tiles) * kTile;
@@ -285,11 +285,30 @@ __global__ void k_lse_combine(int n_rows, int P, int D, const float *__restrict_
 }
 
 // ---- K1 -------------------------------------------------------------------------------------------
+// packed fp32 pairs: sm_100 issues two FMAs per instruction on a 64-bit register pair
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;"
+        : "=l"(d)
+        : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)),
+          "l"(*reinterpret_cast<unsigned long long *>(&c)));
+    return *reinterpret_cast<float2 *>(&d);
+}
+__device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;"
+        : "=l"(d)
+        : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)));
+    return *reinterpret_cast<float2 *>(&d);
+}
+__device__ __forceinline__ float2 bf2(uint32_t w) { return make_float2(bf_lo(w), bf_hi(w)); }
+
 template <int D, int G>
 struct StreamCfg {
     static constexpr int LPR = (D == 128 && G == 8) ? 16 : 8;  // lanes that share one K/V row
     static constexpr int DPL = D / LPR;                        // dims per lane
     static constexpr int NV = DPL / 8;                         // 16-byte vectors per lane per row
+    static constexpr int NPAIR = DPL / 2;                      // fp32 pairs per lane per row
     static constexpr int RG = 32 / LPR;                        // row groups per warp
     static constexpr int RPG = kTile / RG;                     // rows per group per tile
     static constexpr int SUBR = (RPG < 32 / G) ? RPG : 32 / G; // rows per group per reduce batch
@@ -299,7 +318,7 @@ struct StreamCfg {
     static constexpr int LPH = LPR / G;                        // lanes of a group that end up with the same head
     static constexpr int SLOT_BYTES = kTile * D * 2;
     static constexpr int MERGE_BYTES = (kConsumerWarps * G * (D + 2) * 4 + 15) / 16 * 16;
-    static constexpr int PS_STRIDE = (kTile * G + G + 3) / 4 * 4;  // floats per warp, 16-byte multiple
+    static constexpr int PS_STRIDE = (kTile * G * 2 + G + 3) / 4 * 4;  // floats per warp: p pairs [row][head], alpha[head]
     static constexpr int PS_BYTES = kConsumerWarps * PS_STRIDE * 4;
     static constexpr int FIXED_BYTES = MERGE_BYTES + PS_BYTES + 1024;
     static constexpr int NSLOT_MAX = ((kMaxDynSmem - FIXED_BYTES) / SLOT_BYTES) & ~1;
@@ -319,8 +338,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
     float *ps_all = (float *)(smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES);  // [warp][PS_STRIDE]
     unsigned char *misc = smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES + C::PS_BYTES;
     uint64_t *bars = (uint64_t *)misc;                                   // full[NSLOT], empty[NSLOT]
-    CtaRange *range = (CtaRange *)(misc + 2 * 24 * 8);
-    volatile int *flags = (volatile int *)(misc + 2 * 24 * 8 + sizeof(CtaRange) + 8);  // [0] abort, [1] last arriver
+    int32_t *meta = (int32_t *)(misc + 2 * 24 * 8);                      // per slot: rows | (own new row + 1) << 8
+    CtaRange *range = (CtaRange *)(misc + 2 * 24 * 8 + 24 * 4);
+    volatile int *flags = (volatile int *)(misc + 2 * 24 * 8 + 24 * 4 + sizeof(CtaRange) + 8);  // [0] abort, [1] last arriver
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -340,7 +360,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
     const uint32_t ring_u32 = smem_u32(ring), full_u32 = smem_u32(bars), empty_u32 = smem_u32(bars + C::NSLOT);
 
     if (warp == kConsumerWarps) {
-        // ================= producer: one thread feeds the ring =================
+        // ================= producer: one thread walks the table and feeds the ring =================
         if (lane != 0) return;
         UnitPos u = range->first;
         SegCursor cur;
@@ -352,6 +372,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
             const int t_end = (int)min((int64_t)u.rt, f_end - u.flat_begin);
             for (int t = u.tile; t < t_end && ok; ++t, ++f) {
                 const TileSrc s = tile_source<D>(p, u, t, cur);
+                int32_t m = s.rows;
+                if (s.new_first >= 0 && u.i >= s.new_first && u.i < s.new_first + s.rows) m |= (u.i - s.new_first + 1) << 8;
 #pragma unroll
                 for (int kv = 0; kv < 2; ++kv, ++seq) {
                     const uint32_t slot = seq % C::NSLOT, use = seq / C::NSLOT;
@@ -361,6 +383,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
                     }
                     const __nv_bfloat16 *src = kv ? s.v : s.k;
                     const uint32_t dst = ring_u32 + slot * C::SLOT_BYTES, bar = full_u32 + slot * 8;
+                    meta[slot] = m;  // ordered before the consumers' wait by the barrier's release/acquire
                     mbar_expect_tx(bar, (uint32_t)s.rows * D * 2);
                     if (s.row_stride == D) {
                         bulk_g2s(dst, src, (uint32_t)s.rows * D * 2, bar);
@@ -389,15 +412,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
     // ================= consumers =================
     const int grp = lane / C::LPR, jl = lane % C::LPR;
     const int my_h = jl / C::LPH;  // head whose scores this lane holds after the reduce-scatter
-    float *ps = ps_all + warp * C::PS_STRIDE;  // this warp's p[row][head], then alpha[head]
-    float *alpha_s = ps + kTile * G;
+    float *ps = ps_all + warp * C::PS_STRIDE;     // this warp's (p, p)[row][head], then alpha[head]
+    float *alpha_s = ps + kTile * G * 2;
 
-    float qf[G][C::DPL];
-    float of[G][C::DPL];
+    float2 qf[G][C::NPAIR];
+    float2 of[G][C::NPAIR];
     float m_run = -CUDART_INF_F, l_run = 0.f;
 
     UnitPos u = range->first;
-    SegCursor cur;
     int64_t f_unit = f_begin;   // flat index of this CTA's first tile inside the current unit
     int64_t j_base = 0;         // CTA-local index of that tile
     while (f_unit < f_end) {
@@ -408,32 +430,29 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
         {
             const __nv_bfloat16 *qb = p.q + (int64_t)u.l_rel * p.q_sl + (int64_t)u.b * p.q_sb + (int64_t)u.i * p.q_ss +
                                       (int64_t)u.g * G * D;
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
 #pragma unroll
             for (int h = 0; h < G; ++h)
 #pragma unroll
                 for (int v = 0; v < C::NV; ++v) {
                     const uint4 w = *(const uint4 *)(qb + h * D + (v * C::LPR + jl) * 8);
-                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        qf[h][v * 8 + 2 * e] = bf_lo(ww[e]) * p.scale_log2;
-                        qf[h][v * 8 + 2 * e + 1] = bf_hi(ww[e]) * p.scale_log2;
-                    }
+                    qf[h][v * 4 + 0] = fmul2(bf2(w.x), sc2);
+                    qf[h][v * 4 + 1] = fmul2(bf2(w.y), sc2);
+                    qf[h][v * 4 + 2] = fmul2(bf2(w.z), sc2);
+                    qf[h][v * 4 + 3] = fmul2(bf2(w.w), sc2);
                 }
 #pragma unroll
             for (int h = 0; h < G; ++h)
 #pragma unroll
-                for (int d = 0; d < C::DPL; ++d) of[h][d] = 0.f;
+                for (int d = 0; d < C::NPAIR; ++d) of[h][d] = make_float2(0.f, 0.f);
             m_run = -CUDART_INF_F;
             l_run = 0.f;
-            cur.reset();
         }
         // ---- this warp's tiles of the unit ----
         // CTA-local tile index j = j_base + (t - t_begin); warp w takes j == w (mod kConsumerWarps)
         int t = t_begin + (int)((warp - j_base % kConsumerWarps + kConsumerWarps) % kConsumerWarps);
         for (; t < t_end; t += kConsumerWarps) {
             const int64_t j = j_base + (t - t_begin);
-            const TileSrc s = tile_source<D>(p, u, t, cur);
             const uint32_t seq_k = (uint32_t)(2 * j), seq_v = seq_k + 1;
             const uint32_t slot_k = seq_k % C::NSLOT, slot_v = seq_v % C::NSLOT;
             const unsigned char *ks = ring + slot_k * C::SLOT_BYTES;
@@ -441,6 +460,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
 
             // ---------- scores ----------
             mbar_wait(full_u32 + slot_k * 8, (seq_k / C::NSLOT) & 1, flags);
+            const int32_t mt = meta[slot_k];
+            const int rows = mt & 0xff, own_row = (mt >> 8) - 1;
             float sc[C::NSUB][C::NF];
 #pragma unroll
             for (int sub = 0; sub < C::NSUB; ++sub) {
@@ -448,21 +469,19 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
 #pragma unroll
                 for (int r = 0; r < C::SUBR; ++r) {
                     const int row = (sub * C::SUBR + r) * C::RG + grp;
-                    float kf[C::DPL];
+                    float2 kf[C::NPAIR];
 #pragma unroll
                     for (int v = 0; v < C::NV; ++v) {
                         const uint4 w = *(const uint4 *)(ks + row * (D * 2) + (v * C::LPR + jl) * 16);
-                        kf[v * 8 + 0] = bf_lo(w.x); kf[v * 8 + 1] = bf_hi(w.x);
-                        kf[v * 8 + 2] = bf_lo(w.y); kf[v * 8 + 3] = bf_hi(w.y);
-                        kf[v * 8 + 4] = bf_lo(w.z); kf[v * 8 + 5] = bf_hi(w.z);
-                        kf[v * 8 + 6] = bf_lo(w.w); kf[v * 8 + 7] = bf_hi(w.w);
+                        kf[v * 4 + 0] = bf2(w.x); kf[v * 4 + 1] = bf2(w.y);
+                        kf[v * 4 + 2] = bf2(w.z); kf[v * 4 + 3] = bf2(w.w);
                     }
 #pragma unroll
                     for (int h = 0; h < G; ++h) {
-                        float a = 0.f;
+                        float2 a = make_float2(0.f, 0.f);
 #pragma unroll
-                        for (int d = 0; d < C::DPL; ++d) a = fmaf(qf[h][d], kf[d], a);
-                        part[h * C::SUBR + r] = a;
+                        for (int d = 0; d < C::NPAIR; ++d) a = ffma2(qf[h][d], kf[d], a);
+                        part[h * C::SUBR + r] = a.x + a.y;
                     }
                 }
                 // reduce-scatter over the LPR lanes of the row group: afterwards this lane holds the
@@ -483,16 +502,13 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
                 for (int k = 0; k < C::NF; ++k) {
                     const int r = (jl % C::LPH) * C::NF + k;  // row of the batch (head index = my_h)
                     const int row = (sub * C::SUBR + r) * C::RG + grp;
-                    sc[sub][k] = row < s.rows ? part[k] : -CUDART_INF_F;
+                    sc[sub][k] = row < rows ? part[k] : -CUDART_INF_F;
                 }
             }
             // the new token's K row goes to the tail for later steps (this unit's own token only)
-            if (s.new_first >= 0 && u.i >= s.new_first && u.i < s.new_first + s.rows && u.t0 + u.i < p.max_tail) {
-                const int row = u.i - s.new_first;
+            if (own_row >= 0 && u.t0 + u.i < p.max_tail) {
                 const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + u.t0 + u.i) * D;
-                if (lane < D / 8) {
-                    *(uint4 *)(p.tail_k + off + lane * 8) = *(const uint4 *)(ks + row * (D * 2) + lane * 16);
-                }
+                if (lane < D / 8) *(uint4 *)(p.tail_k + off + lane * 8) = *(const uint4 *)(ks + own_row * (D * 2) + lane * 16);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_u32 + slot_k * 8);
@@ -518,7 +534,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
                     psum += pv;
                     const int r = (jl % C::LPH) * C::NF + k;
                     const int row = (sub * C::SUBR + r) * C::RG + grp;
-                    ps[row * G + my_h] = pv;
+                    *(float2 *)(ps + (row * G + my_h) * 2) = make_float2(pv, pv);
                 }
             l_run = l_run * alpha + psum;
             m_run = m_new;
@@ -531,47 +547,43 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
 #pragma unroll
                 for (int h = 0; h < G; ++h) {
                     const float a = alpha_s[h];
+                    const float2 a2 = make_float2(a, a);
 #pragma unroll
-                    for (int d = 0; d < C::DPL; ++d) of[h][d] *= a;
+                    for (int d = 0; d < C::NPAIR; ++d) of[h][d] = fmul2(of[h][d], a2);
                 }
             }
             mbar_wait(full_u32 + slot_v * 8, (seq_v / C::NSLOT) & 1, flags);
 #pragma unroll
             for (int r = 0; r < C::RPG; ++r) {
                 const int row = r * C::RG + grp;
-                if (row < s.rows) {
-                    float vf[C::DPL];
+                if (row < rows) {
+                    float2 vf[C::NPAIR];
 #pragma unroll
                     for (int v = 0; v < C::NV; ++v) {
                         const uint4 w = *(const uint4 *)(vs + row * (D * 2) + (v * C::LPR + jl) * 16);
-                        vf[v * 8 + 0] = bf_lo(w.x); vf[v * 8 + 1] = bf_hi(w.x);
-                        vf[v * 8 + 2] = bf_lo(w.y); vf[v * 8 + 3] = bf_hi(w.y);
-                        vf[v * 8 + 4] = bf_lo(w.z); vf[v * 8 + 5] = bf_hi(w.z);
-                        vf[v * 8 + 6] = bf_lo(w.w); vf[v * 8 + 7] = bf_hi(w.w);
+                        vf[v * 4 + 0] = bf2(w.x); vf[v * 4 + 1] = bf2(w.y);
+                        vf[v * 4 + 2] = bf2(w.z); vf[v * 4 + 3] = bf2(w.w);
                     }
-                    float pr[G];
-                    if constexpr (G % 4 == 0) {
+                    float2 pr[G];
+                    if constexpr (G % 2 == 0) {
 #pragma unroll
-                        for (int h4 = 0; h4 < G / 4; ++h4) {
-                            const float4 t4 = *(const float4 *)(ps + row * G + h4 * 4);
-                            pr[h4 * 4 + 0] = t4.x; pr[h4 * 4 + 1] = t4.y; pr[h4 * 4 + 2] = t4.z; pr[h4 * 4 + 3] = t4.w;
+                        for (int h2 = 0; h2 < G / 2; ++h2) {
+                            const float4 t4 = *(const float4 *)(ps + (row * G + h2 * 2) * 2);
+                            pr[h2 * 2 + 0] = make_float2(t4.x, t4.y);
+                            pr[h2 * 2 + 1] = make_float2(t4.z, t4.w);
                         }
                     } else {
-#pragma unroll
-                        for (int h = 0; h < G; ++h) pr[h] = ps[row * G + h];
+                        pr[0] = *(const float2 *)(ps + row * 2);
                     }
 #pragma unroll
                     for (int h = 0; h < G; ++h)
 #pragma unroll
-                        for (int d = 0; d < C::DPL; ++d) of[h][d] = fmaf(pr[h], vf[d], of[h][d]);
+                        for (int d = 0; d < C::NPAIR; ++d) of[h][d] = ffma2(pr[h], vf[d], of[h][d]);
                 }
             }
-            if (s.new_first >= 0 && u.i >= s.new_first && u.i < s.new_first + s.rows && u.t0 + u.i < p.max_tail) {
-                const int row = u.i - s.new_first;
+            if (own_row >= 0 && u.t0 + u.i < p.max_tail) {
                 const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + u.t0 + u.i) * D;
-                if (lane < D / 8) {
-                    *(uint4 *)(p.tail_v + off + lane * 8) = *(const uint4 *)(vs + row * (D * 2) + lane * 16);
-                }
+                if (lane < D / 8) *(uint4 *)(p.tail_v + off + lane * 8) = *(const uint4 *)(vs + own_row * (D * 2) + lane * 16);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_u32 + slot_v * 8);
@@ -587,10 +599,13 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
 #pragma unroll
             for (int h = 0; h < G; ++h)
 #pragma unroll
-                for (int d = 0; d < C::DPL; ++d) {
-                    float x = of[h][d];
+                for (int d = 0; d < C::NPAIR; ++d) {
+                    float2 x = of[h][d];
 #pragma unroll
-                    for (int off = C::LPR; off < 32; off <<= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+                    for (int off = C::LPR; off < 32; off <<= 1) {
+                        x.x += __shfl_xor_sync(0xffffffffu, x.x, off);
+                        x.y += __shfl_xor_sync(0xffffffffu, x.y, off);
+                    }
                     of[h][d] = x;
                 }
             if (grp == 0) {
@@ -599,8 +614,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
 #pragma unroll
                     for (int v = 0; v < C::NV; ++v)
 #pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            merge_o[(warp * G + h) * D + (v * C::LPR + jl) * 8 + e] = of[h][v * 8 + e];
+                        for (int e = 0; e < 4; ++e)
+                            *(float2 *)(merge_o + (warp * G + h) * D + (v * C::LPR + jl) * 8 + 2 * e) = of[h][v * 4 + e];
                 if (jl % C::LPH == 0) {
                     merge_m[warp * G + my_h] = m_run;
                     merge_l[warp * G + my_h] = l_tot;
