@@ -5,8 +5,7 @@
 // [c*W/n, (c+1)*W/n) of that list, so every SM streams the same number of bytes whatever the shape.
 // Inside a CTA one producer thread walks its range and moves each tile's K rows and V rows from the
 // scattered chunk blobs (or the tail, or the new tokens) into a shared-memory ring with bulk
-// asynchronous copies (cp.async.bulk + mbarrier complete_tx); seven consumer warps each take every
-// seventh tile and run an independent online softmax for the G query heads that share the KV head
+// asynchronous copies (cp.async.bulk + mbarrier complete_tx); the consumer warps take the tiles round-robin and run an independent online softmax for the G query heads that share the KV head
 // (fp32, exp2-based).  At the end of a unit the warps' states are merged through shared memory; a
 // unit that spans several CTAs leaves one partial (normalised o, lse) per CTA in the workspace and
 // the last CTA to arrive (atomic ticket, no waiting) merges them by log-sum-exp.
@@ -20,8 +19,13 @@
 
 namespace matkv {
 
-constexpr int kConsumerWarps = 7;  // registers are allocated to warps in fours: 8 warps x 255 registers fill the file
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
+// Consumer warps per CTA (+1 producer warp).  Registers are allocated to warps in fours, so a CTA is
+// 8 warps x 255 registers or 16 warps x 128 registers; the thin variant hides more latency and is used
+// whenever q and o of the G heads fit its register budget.
+// A thin warp takes half a tile, so that 15 of them hold fewer ring slots than the ring has: a warp
+// may only wait on a slot whose previous fill has already completed (mbarrier phases are one bit).
+template <int G> constexpr bool thin_variant() { return G == 2 || G == 4; }
+template <int G> constexpr int consumer_warps() { return thin_variant<G>() ? 15 : 7; }
 constexpr int kMaxDynSmem = 232448;            // 227 KB opt-in limit per CTA on sm_100
 constexpr long long kWaitCycles = 2000000000LL;  // bounded waits give up after about a second
 constexpr float kLog2e = 1.4426950408889634f;
@@ -83,7 +87,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
+template <int CW> __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(CW * 32) : "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -305,36 +309,41 @@ __device__ __forceinline__ float2 bf2(uint32_t w) { return make_float2(bf_lo(w),
 
 template <int D, int G>
 struct StreamCfg {
-    static constexpr int LPR = (D == 128 && G == 8) ? 16 : 8;  // lanes that share one K/V row
+    static constexpr int CW = consumer_warps<G>();             // consumer warps
+    static constexpr int THREADS = (CW + 1) * 32;
+    static constexpr int SPLIT = thin_variant<G>() ? 2 : 1;    // warps that share one tile
+    static constexpr int HROWS = kTile / SPLIT;                // rows of a tile one warp handles
+    static constexpr int LPR = (D == 128 && (SPLIT == 2 || G == 8)) ? 16 : 8;  // lanes that share one K/V row
     static constexpr int DPL = D / LPR;                        // dims per lane
     static constexpr int NV = DPL / 8;                         // 16-byte vectors per lane per row
     static constexpr int NPAIR = DPL / 2;                      // fp32 pairs per lane per row
     static constexpr int RG = 32 / LPR;                        // row groups per warp
-    static constexpr int RPG = kTile / RG;                     // rows per group per tile
+    static constexpr int RPG = HROWS / RG;                     // rows per group per work item
     static constexpr int SUBR = (RPG < 32 / G) ? RPG : 32 / G; // rows per group per reduce batch
     static constexpr int NSUB = RPG / SUBR;
     static constexpr int NP = G * SUBR;                        // partial dot products per lane per batch
     static constexpr int NF = NP / LPR;                        // scores per lane after the reduce-scatter
     static constexpr int LPH = LPR / G;                        // lanes of a group that end up with the same head
     static constexpr int SLOT_BYTES = kTile * D * 2;
-    static constexpr int MERGE_BYTES = (kConsumerWarps * G * (D + 2) * 4 + 15) / 16 * 16;
-    static constexpr int PS_STRIDE = (kTile * G * 2 + G + 3) / 4 * 4;  // floats per warp: p pairs [row][head], alpha[head]
-    static constexpr int PS_BYTES = kConsumerWarps * PS_STRIDE * 4;
+    static constexpr int MERGE_BYTES = (CW * G * (D + 2) * 4 + 15) / 16 * 16;
+    static constexpr int PS_STRIDE = (HROWS * G * 2 + G + 3) / 4 * 4;  // floats per warp: p pairs [row][head], alpha[head]
+    static constexpr int PS_BYTES = CW * PS_STRIDE * 4;
     static constexpr int FIXED_BYTES = MERGE_BYTES + PS_BYTES + 1024;
     static constexpr int NSLOT_MAX = ((kMaxDynSmem - FIXED_BYTES) / SLOT_BYTES) & ~1;
     static constexpr int NSLOT = NSLOT_MAX > 24 ? 24 : NSLOT_MAX;
     static constexpr int SMEM_BYTES = NSLOT * SLOT_BYTES + FIXED_BYTES;
     static_assert(DPL % 8 == 0 && NF >= 1 && SUBR % NF == 0 && LPH >= 1, "unsupported head_dim / group size");
+    static_assert(2 * CW < NSLOT * SPLIT, "a warp would wait on a ring slot more than one phase ahead");
 };
 
 template <int D, int G>
-__global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParams p) {
+__global__ void __launch_bounds__((consumer_warps<G>() + 1) * 32, 1) k_attend_stream(const StreamParams p) {
     using C = StreamCfg<D, G>;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char *ring = smem;
     float *merge_o = (float *)(smem + C::NSLOT * C::SLOT_BYTES);         // [warp][G][D]
-    float *merge_m = merge_o + kConsumerWarps * G * D;                   // [warp][G]
-    float *merge_l = merge_m + kConsumerWarps * G;                       // [warp][G]
+    float *merge_m = merge_o + C::CW * G * D;                   // [warp][G]
+    float *merge_l = merge_m + C::CW * G;                       // [warp][G]
     float *ps_all = (float *)(smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES);  // [warp][PS_STRIDE]
     unsigned char *misc = smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES + C::PS_BYTES;
     uint64_t *bars = (uint64_t *)misc;                                   // full[NSLOT], empty[NSLOT]
@@ -346,7 +355,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
     if (tid == 0) {
         for (int s = 0; s < C::NSLOT; ++s) {
             mbar_init(smem_u32(bars + s), 1);
-            mbar_init(smem_u32(bars + C::NSLOT + s), 1);
+            mbar_init(smem_u32(bars + C::NSLOT + s), C::SPLIT);
         }
         flags[0] = 0;
         flags[1] = 0;
@@ -359,7 +368,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
     if (f_begin >= f_end) return;
     const uint32_t ring_u32 = smem_u32(ring), full_u32 = smem_u32(bars), empty_u32 = smem_u32(bars + C::NSLOT);
 
-    if (warp == kConsumerWarps) {
+    if (warp == C::CW) {
         // ================= producer: one thread walks the table and feeds the ring =================
         if (lane != 0) return;
         UnitPos u = range->first;
@@ -413,7 +422,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
     const int grp = lane / C::LPR, jl = lane % C::LPR;
     const int my_h = jl / C::LPH;  // head whose scores this lane holds after the reduce-scatter
     float *ps = ps_all + warp * C::PS_STRIDE;     // this warp's (p, p)[row][head], then alpha[head]
-    float *alpha_s = ps + kTile * G * 2;
+    float *alpha_s = ps + C::HROWS * G * 2;
 
     float2 qf[G][C::NPAIR];
     float2 of[G][C::NPAIR];
@@ -448,20 +457,34 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
             m_run = -CUDART_INF_F;
             l_run = 0.f;
         }
-        // ---- this warp's tiles of the unit ----
-        // CTA-local tile index j = j_base + (t - t_begin); warp w takes j == w (mod kConsumerWarps)
-        int t = t_begin + (int)((warp - j_base % kConsumerWarps + kConsumerWarps) % kConsumerWarps);
-        for (; t < t_end; t += kConsumerWarps) {
-            const int64_t j = j_base + (t - t_begin);
+        // ---- this warp's work items of the unit ----
+        // CTA-local tile j = j_base + (t - t_begin) splits into SPLIT work items hj = j*SPLIT + half;
+        // warp w takes hj == w (mod CW)
+        const int64_t hj_begin = j_base * C::SPLIT, hj_end = (j_base + (t_end - t_begin)) * C::SPLIT;
+        int64_t hj = hj_begin + (int)((warp - hj_begin % C::CW + C::CW) % C::CW);
+        for (; hj < hj_end; hj += C::CW) {
+            const int64_t j = hj / C::SPLIT;
+            const int row0 = (int)(hj % C::SPLIT) * C::HROWS;
             const uint32_t seq_k = (uint32_t)(2 * j), seq_v = seq_k + 1;
             const uint32_t slot_k = seq_k % C::NSLOT, slot_v = seq_v % C::NSLOT;
-            const unsigned char *ks = ring + slot_k * C::SLOT_BYTES;
-            const unsigned char *vs = ring + slot_v * C::SLOT_BYTES;
+            const unsigned char *ks = ring + slot_k * C::SLOT_BYTES + row0 * (D * 2);
+            const unsigned char *vs = ring + slot_v * C::SLOT_BYTES + row0 * (D * 2);
 
             // ---------- scores ----------
             mbar_wait(full_u32 + slot_k * 8, (seq_k / C::NSLOT) & 1, flags);
             const int32_t mt = meta[slot_k];
-            const int rows = mt & 0xff, own_row = (mt >> 8) - 1;
+            const int rows = (mt & 0xff) - row0;        // valid rows of this work item (may be <= 0)
+            int own_row = (mt >> 8) - 1 - row0;         // the unit's own new token, if it sits in this work item
+            if (own_row >= C::HROWS) own_row = -1;
+            if (rows <= 0) {                            // the tile ends before this half: just release the slots
+                mbar_wait(full_u32 + slot_v * 8, (seq_v / C::NSLOT) & 1, flags);
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(empty_u32 + slot_k * 8);
+                    mbar_arrive(empty_u32 + slot_v * 8);
+                }
+                continue;
+            }
             float sc[C::NSUB][C::NF];
 #pragma unroll
             for (int sub = 0; sub < C::NSUB; ++sub) {
@@ -523,7 +546,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
             for (int off = 1; off < C::LPH; off <<= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, off));
 #pragma unroll
             for (int off = C::LPR; off < 32; off <<= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, off));
-            const float m_new = fmaxf(m_run, tmax);  // finite: every tile has at least one valid row
+            const float m_new = fmaxf(m_run, tmax);  // finite: the work item has at least one valid row
             const float alpha = fast_exp2(m_run - m_new);
             float psum = 0.f;
 #pragma unroll
@@ -622,7 +645,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
                 }
             }
         }
-        consumer_bar();
+        consumer_bar<C::CW>();
         const int64_t unit_index = (((int64_t)u.l_rel * p.B + u.b) * p.S + u.i) * p.Hkv + u.g;
         const int c_first = cta_of(u.flat_begin, W, gridDim.x);
         const int c_last = cta_of(u.flat_begin + u.rt - 1, W, gridDim.x);
@@ -632,14 +655,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
         const int64_t slot = unit_index + blockIdx.x;
         const bool slot_ok = slot < p.n_part_slots && unit_index < p.n_counter_slots;
         if (n_parts > 1 && !slot_ok && tid == 0) atomicCAS(p.status, 0, MATKV_E_BOUNDS);
-        for (int idx = tid; idx < G * D; idx += kConsumerWarps * 32) {
+        for (int idx = tid; idx < G * D; idx += C::CW * 32) {
             const int h = idx / D, d = idx % D;
             float M = -CUDART_INF_F;
 #pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, merge_m[w * G + h]);
+            for (int w = 0; w < C::CW; ++w) M = fmaxf(M, merge_m[w * G + h]);
             float acc = 0.f, L = 0.f;
 #pragma unroll
-            for (int w = 0; w < kConsumerWarps; ++w) {
+            for (int w = 0; w < C::CW; ++w) {
                 const float sw = fast_exp2(merge_m[w * G + h] - M);
                 acc = fmaf(sw, merge_o[(w * G + h) * D + d], acc);
                 L = fmaf(sw, merge_l[w * G + h], L);
@@ -656,23 +679,23 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
         }
         if (n_parts > 1 && slot_ok) {
             __threadfence();
-            consumer_bar();
+            consumer_bar<C::CW>();
             if (tid == 0) {
                 const int old = atomicAdd(p.counters + unit_index, 1);
                 const int last = (old == n_parts - 1);
                 if (last) p.counters[unit_index] = 0;  // ready for the next launch
                 flags[1] = last;
             }
-            consumer_bar();
+            consumer_bar<C::CW>();
             if (flags[1]) {
                 __threadfence();
                 const int64_t first_slot = unit_index + c_first;
-                for (int h = warp; h < G; h += kConsumerWarps)
+                for (int h = warp; h < G; h += C::CW)
                     combine_warp(p.part_o + (first_slot * G + h) * D, (int64_t)G * D, p.part_lse + first_slot * G + h, G,
                                  n_parts, D, p.out + io_off + h * D, p.lse_out ? p.lse_out + lse_off + h : nullptr);
             }
         }
-        consumer_bar();  // merge area and flags are free again
+        consumer_bar<C::CW>();  // merge area and flags are free again
 
         j_base += t_end - t_begin;
         f_unit = u.flat_begin + t_end;
@@ -690,7 +713,7 @@ static int launch_stream_t(const StreamParams &p, int grid, cudaStream_t stream)
         MATKV_CUDA(cudaFuncSetAttribute(k_attend_stream<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
         configured = true;
     }
-    k_attend_stream<D, G><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p);
+    k_attend_stream<D, G><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(p);
     MATKV_CUDA(cudaGetLastError());
     return MATKV_OK;
 }
