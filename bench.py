@@ -308,6 +308,22 @@ def main():
             timed_region(lambda i: one_step(*dev_ptrs, timed_index=i, mode=other), min(args.steps, 5))
             dec_ms_o = sum(a.elapsed_time(b) for a, b in zip(ev_d0[:min(args.steps, 5)], ev_d1[:min(args.steps, 5)]))
 
+    # read-only streaming probe over the same chunk memory (plain 16-byte loads), same run
+    probe_gbs = None
+    with torch.cuda.stream(stream):
+        big = max(chunks.values(), key=lambda x: x.numel())
+        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(2):
+            for c in needed:
+                mk.matkv_probe_read(ctx, chunks[c].data_ptr(), chunks[c].numel() * 2, sp)
+        pe0.record(stream)
+        for _ in range(3):
+            for c in needed:
+                mk.matkv_probe_read(ctx, chunks[c].data_ptr(), chunks[c].numel() * 2, sp)
+        pe1.record(stream)
+        torch.cuda.synchronize()
+        probe_gbs = 3 * sum(chunks[c].numel() * 2 for c in needed) / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
+
     # algorithmic KV bytes of the decode loop of one step: every visible K and V element once
     n_req = [sum(chunks[c].shape[3] for c in row) for row in ids]
     kv_bytes_decode = sum((n + S + t + 1) * w.beta for n in n_req for t in range(T)) * L
@@ -332,6 +348,7 @@ def main():
         "roofline": {"bound": "hbm", "kernel": "k_attend_stream (decode)", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                     "read_probe_gbs_same_run": probe_gbs,
                      "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.decode_launch)),
                      "algorithmic_bytes_per_launch": kv_bytes_decode / decode_launches,
                      "avg_launch_us": avg_launch_ms * 1e3},

@@ -179,6 +179,11 @@ int matkv_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D
 int matkv_gather_debug(matkv_ctx *ctx, matkv_table *table, int32_t layer, int32_t req, void *k_out,
                        void *v_out, int64_t capacity_rows, int64_t *rows_out, void *stream);
 
+/* ---- measurement aid: read-only streaming probe ------------------------------------------- */
+/* Reads `bytes` of device memory once with plain 16-byte loads (nothing is written): the HBM read
+ * ceiling a decode launch is compared with.  No counterpart in the paper.  Asynchronous on `stream`. */
+int matkv_probe_read(matkv_ctx *ctx, const void *dev, size_t bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,6 +24,7 @@ EXPORTS = [
     "matkv_stage_chunks_async", "matkv_stage_query", "matkv_stage_wait", "matkv_build_chunk_table",
     "matkv_table_free", "matkv_table_advance", "matkv_table_set_tail_len", "matkv_attend_prefill",
     "matkv_attend_decode", "matkv_attend_decode_all_layers", "matkv_lse_combine", "matkv_gather_debug",
+    "matkv_probe_read",
 ]
 
 
@@ -74,6 +75,7 @@ def lib() -> C.CDLL:
             "matkv_attend_decode_all_layers": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, vp]),
             "matkv_lse_combine": (C.c_int, [vp, i32, i32, i32, vp, vp, vp, vp, vp]),
             "matkv_gather_debug": (C.c_int, [vp, vp, i32, i32, vp, vp, i64, C.POINTER(i64), vp]),
+            "matkv_probe_read": (C.c_int, [vp, vp, C.c_size_t, vp]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -201,3 +203,7 @@ def matkv_gather_debug(ctx: int, table: int, layer: int, req: int, k_out: int, v
     rows = C.c_int64(0)
     _check(lib().matkv_gather_debug(ctx, table, layer, req, k_out, v_out, capacity_rows, C.byref(rows), stream or None))
     return rows.value
+
+
+def matkv_probe_read(ctx: int, dev_ptr: int, nbytes: int, stream: int = 0) -> None:
+    _check(lib().matkv_probe_read(ctx, dev_ptr, nbytes, stream or None))

@@ -22,8 +22,9 @@ namespace matkv {
 // Consumer warps per CTA (+1 producer warp).  Registers are allocated to warps in fours, so a CTA is
 // 8 warps x 255 registers or 16 warps x 128 registers; the thin variant hides more latency and is used
 // whenever q and o of the G heads fit its register budget.
-// A thin warp takes half a tile, so that 15 of them hold fewer ring slots than the ring has: a warp
-// may only wait on a slot whose previous fill has already completed (mbarrier phases are one bit).
+// Copies are issued per 64-token tile (large copies keep the copy engine's per-copy cost low); a warp
+// works on a quarter (thin variant) or half (fat variant) of a tile so that the slots being consumed
+// leave room in the ring for tiles in flight.
 template <int G> constexpr bool thin_variant() { return G == 2 || G == 4; }
 template <int G> constexpr int consumer_warps() { return thin_variant<G>() ? 15 : 7; }
 constexpr int kMaxDynSmem = 232448;            // 227 KB opt-in limit per CTA on sm_100
@@ -79,6 +80,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (clock64() - t0 > kWaitCycles) {
             *abort_flag = 1;
             return false;
+        }
+    }
+}
+// A consumer's wait for fill number `want` of a ring slot.  Warps take work items round-robin, so a
+// warp can reach a slot whose PREVIOUS fill is still in flight, and the one-bit phase of an mbarrier
+// cannot tell "fill n-1 incomplete" from "fill n complete".  The producer therefore publishes the fill
+// number of a slot (upper half of the slot's tag word) before it issues the copy, which it does only
+// after the slot's previous fill was consumed and released; once the consumer sees its number there,
+// the parity test is unambiguous.  Returns the tag word, or 0 after the bounded wait ran out.
+__device__ __forceinline__ uint32_t slot_wait(const volatile uint32_t *tag, uint32_t want, uint32_t bar, uint32_t parity,
+                                              volatile int *abort_flag) {
+    uint32_t w = *tag;
+    if ((w >> 16) == (want & 0xffffu) && mbar_try_wait(bar, parity)) return w;
+    const long long t0 = clock64();
+    while (true) {
+        w = *tag;
+        if ((w >> 16) == (want & 0xffffu) && mbar_try_wait(bar, parity)) return w;
+        if (*abort_flag) return 0;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            return 0;
         }
     }
 }
@@ -311,7 +333,7 @@ template <int D, int G>
 struct StreamCfg {
     static constexpr int CW = consumer_warps<G>();             // consumer warps
     static constexpr int THREADS = (CW + 1) * 32;
-    static constexpr int SPLIT = thin_variant<G>() ? 2 : 1;    // warps that share one tile
+    static constexpr int SPLIT = thin_variant<G>() ? 4 : 2;    // warps that share one tile
     static constexpr int HROWS = kTile / SPLIT;                // rows of a tile one warp handles
     static constexpr int LPR = (D == 128 && (SPLIT == 2 || G == 8)) ? 16 : 8;  // lanes that share one K/V row
     static constexpr int DPL = D / LPR;                        // dims per lane
@@ -329,11 +351,11 @@ struct StreamCfg {
     static constexpr int PS_STRIDE = (HROWS * G * 2 + G + 3) / 4 * 4;  // floats per warp: p pairs [row][head], alpha[head]
     static constexpr int PS_BYTES = CW * PS_STRIDE * 4;
     static constexpr int FIXED_BYTES = MERGE_BYTES + PS_BYTES + 1024;
-    static constexpr int NSLOT_MAX = ((kMaxDynSmem - FIXED_BYTES) / SLOT_BYTES) & ~1;
+    static constexpr int NSLOT_MAX = (kMaxDynSmem - FIXED_BYTES) / SLOT_BYTES;
     static constexpr int NSLOT = NSLOT_MAX > 24 ? 24 : NSLOT_MAX;
     static constexpr int SMEM_BYTES = NSLOT * SLOT_BYTES + FIXED_BYTES;
     static_assert(DPL % 8 == 0 && NF >= 1 && SUBR % NF == 0 && LPH >= 1, "unsupported head_dim / group size");
-    static_assert(2 * CW < NSLOT * SPLIT, "a warp would wait on a ring slot more than one phase ahead");
+    static_assert(NSLOT >= 4, "ring too small");
 };
 
 template <int D, int G>
@@ -347,15 +369,17 @@ __global__ void __launch_bounds__((consumer_warps<G>() + 1) * 32, 1) k_attend_st
     float *ps_all = (float *)(smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES);  // [warp][PS_STRIDE]
     unsigned char *misc = smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES + C::PS_BYTES;
     uint64_t *bars = (uint64_t *)misc;                                   // full[NSLOT], empty[NSLOT]
-    int32_t *meta = (int32_t *)(misc + 2 * 24 * 8);                      // per slot: rows | (own new row + 1) << 8
-    CtaRange *range = (CtaRange *)(misc + 2 * 24 * 8 + 24 * 4);
-    volatile int *flags = (volatile int *)(misc + 2 * 24 * 8 + 24 * 4 + sizeof(CtaRange) + 8);  // [0] abort, [1] last arriver
+    // per slot tag: rows | (the unit's own new row + 1) << 8 | (number of the slot's current fill) << 16
+    volatile uint32_t *tags = (volatile uint32_t *)(misc + 2 * 24 * 8);
+    CtaRange *range = (CtaRange *)(misc + 2 * 24 * 8 + 2 * 24 * 4);
+    volatile int *flags = (volatile int *)(misc + 2 * 24 * 8 + 2 * 24 * 4 + sizeof(CtaRange) + 8);  // [0] abort, [1] last arriver
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         for (int s = 0; s < C::NSLOT; ++s) {
             mbar_init(smem_u32(bars + s), 1);
             mbar_init(smem_u32(bars + C::NSLOT + s), C::SPLIT);
+            tags[s] = 0xffff0000u;
         }
         flags[0] = 0;
         flags[1] = 0;
@@ -381,8 +405,8 @@ __global__ void __launch_bounds__((consumer_warps<G>() + 1) * 32, 1) k_attend_st
             const int t_end = (int)min((int64_t)u.rt, f_end - u.flat_begin);
             for (int t = u.tile; t < t_end && ok; ++t, ++f) {
                 const TileSrc s = tile_source<D>(p, u, t, cur);
-                int32_t m = s.rows;
-                if (s.new_first >= 0 && u.i >= s.new_first && u.i < s.new_first + s.rows) m |= (u.i - s.new_first + 1) << 8;
+                uint32_t m = (uint32_t)s.rows;
+                if (s.new_first >= 0 && u.i >= s.new_first && u.i < s.new_first + s.rows) m |= (uint32_t)(u.i - s.new_first + 1) << 8;
 #pragma unroll
                 for (int kv = 0; kv < 2; ++kv, ++seq) {
                     const uint32_t slot = seq % C::NSLOT, use = seq / C::NSLOT;
@@ -392,7 +416,7 @@ __global__ void __launch_bounds__((consumer_warps<G>() + 1) * 32, 1) k_attend_st
                     }
                     const __nv_bfloat16 *src = kv ? s.v : s.k;
                     const uint32_t dst = ring_u32 + slot * C::SLOT_BYTES, bar = full_u32 + slot * 8;
-                    meta[slot] = m;  // ordered before the consumers' wait by the barrier's release/acquire
+                    tags[slot] = m | (use << 16);  // published only after the slot's previous fill was consumed and released
                     mbar_expect_tx(bar, (uint32_t)s.rows * D * 2);
                     if (s.row_stride == D) {
                         bulk_g2s(dst, src, (uint32_t)s.rows * D * 2, bar);
@@ -471,13 +495,12 @@ __global__ void __launch_bounds__((consumer_warps<G>() + 1) * 32, 1) k_attend_st
             const unsigned char *vs = ring + slot_v * C::SLOT_BYTES + row0 * (D * 2);
 
             // ---------- scores ----------
-            mbar_wait(full_u32 + slot_k * 8, (seq_k / C::NSLOT) & 1, flags);
-            const int32_t mt = meta[slot_k];
-            const int rows = (mt & 0xff) - row0;        // valid rows of this work item (may be <= 0)
-            int own_row = (mt >> 8) - 1 - row0;         // the unit's own new token, if it sits in this work item
+            const uint32_t mt = slot_wait(tags + slot_k, seq_k / C::NSLOT, full_u32 + slot_k * 8, (seq_k / C::NSLOT) & 1, flags);
+            const int rows = (int)(mt & 0xff) - row0;   // valid rows of this work item (may be <= 0)
+            int own_row = (int)((mt >> 8) & 0xff) - 1 - row0;  // the unit's own new token, if it sits in this work item
             if (own_row >= C::HROWS) own_row = -1;
             if (rows <= 0) {                            // the tile ends before this half: just release the slots
-                mbar_wait(full_u32 + slot_v * 8, (seq_v / C::NSLOT) & 1, flags);
+                slot_wait(tags + slot_v, seq_v / C::NSLOT, full_u32 + slot_v * 8, (seq_v / C::NSLOT) & 1, flags);
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(empty_u32 + slot_k * 8);
@@ -575,7 +598,7 @@ __global__ void __launch_bounds__((consumer_warps<G>() + 1) * 32, 1) k_attend_st
                     for (int d = 0; d < C::NPAIR; ++d) of[h][d] = fmul2(of[h][d], a2);
                 }
             }
-            mbar_wait(full_u32 + slot_v * 8, (seq_v / C::NSLOT) & 1, flags);
+            slot_wait(tags + slot_v, seq_v / C::NSLOT, full_u32 + slot_v * 8, (seq_v / C::NSLOT) & 1, flags);
 #pragma unroll
             for (int r = 0; r < C::RPG; ++r) {
                 const int row = r * C::RG + grp;

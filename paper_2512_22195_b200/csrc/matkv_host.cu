@@ -129,8 +129,8 @@ int matkv_create(const matkv_config *cfg, matkv_ctx **out) {
     ctx->cfg.device = dev;
     ctx->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
     ctx->n_sm = prop.multiProcessorCount;
-    cudaError_t e = cudaMalloc(&ctx->d_status, sizeof(int32_t));
-    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(int32_t));
+    cudaError_t e = cudaMalloc(&ctx->d_status, 4 * sizeof(int32_t));  // [0] status, [1] probe sink
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 4 * sizeof(int32_t));
     if (e != cudaSuccess) {
         delete ctx;
         return cuda_fail(e, "status word");
@@ -593,6 +593,13 @@ int matkv_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D
     if (n_rows == 0) return MATKV_OK;
     DeviceGuard guard(ctx->device);
     return launch_lse_combine(ctx, n_rows, n_parts, D, o_parts, lse_parts, out, lse_out, (cudaStream_t)stream);
+}
+
+int matkv_probe_read(matkv_ctx *ctx, const void *dev, size_t bytes, void *stream) {
+    if (!ctx || !dev) return fail(MATKV_E_INVALID_ARG, "matkv_probe_read: null argument");
+    if ((uintptr_t)dev % 16 || bytes < 16) return fail(MATKV_E_ALIGNMENT, "matkv_probe_read: buffer must be 16-byte aligned and non-empty");
+    DeviceGuard guard(ctx->device);
+    return launch_read_probe(ctx, dev, bytes, (cudaStream_t)stream);
 }
 
 int matkv_gather_debug(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out,
