@@ -1,13 +1,20 @@
 // K1: chunk-table streaming attention (decode, and small query suffixes) + K2: log-sum-exp combine.
 //
 // One persistent CTA per SM.  The work of a launch is the flat list of KV tiles (kTile tokens of one
-// (layer, request, suffix token, KV head) "unit"); CTA c owns the contiguous range
+// "unit" = (layer, request, block of suffix tokens, KV head)); CTA c owns the contiguous range
 // [c*W/n, (c+1)*W/n) of that list, so every SM streams the same number of bytes whatever the shape.
 // Inside a CTA one producer thread walks its range and moves each tile's K rows and V rows from the
-// scattered chunk blobs (or the tail, or the new tokens) into a shared-memory ring with bulk
-// asynchronous copies (cp.async.bulk + mbarrier complete_tx); the consumer warps take the tiles round-robin and run an independent online softmax for the G query heads that share the KV head
-// (fp32, exp2-based).  At the end of a unit the warps' states are merged through shared memory; a
-// unit that spans several CTAs leaves one partial (normalised o, lse) per CTA in the workspace and
+// scattered chunk blobs (or the tail) into a shared-memory ring with TMA tensor copies (128-byte
+// swizzle, mbarrier complete_tx).  Seven consumer warps take 16-token pieces of the tiles round-robin;
+// each keeps the unit's query rows (up to 8: the G heads of the KV group for up to 8/G suffix tokens)
+// as mma A fragments and runs an independent online softmax: S = Q K^T and O += P V are warp-level
+// m16n8k16 bf16 MMAs fed by ldmatrix from the swizzled tiles, so the instruction stream per KV byte is
+// short enough for the kernel to stay HBM-bound at any G (a plain-FMA inner product measured
+// issue-bound: 42% issue utilisation with 8 resident warps and 48% of DRAM peak).  fp32 scores,
+// exp2-based softmax, fp32 accumulators; P is rounded to bf16 for the second MMA.
+// The new tokens of the call (not yet in the tail) are attended by a short scalar path and appended to
+// the tail by the same warp.  At the end of a unit the warps' states are merged through shared memory;
+// a unit that spans several CTAs leaves one partial (normalised o, lse) per CTA in the workspace and
 // the last CTA to arrive (atomic ticket, no waiting) merges them by log-sum-exp.
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
@@ -19,22 +26,21 @@
 
 namespace matkv {
 
-// Consumer warps per CTA (+1 producer warp).  Registers are allocated to warps in fours, so a CTA is
-// 8 warps x 255 registers or 16 warps x 128 registers; the thin variant hides more latency and is used
-// whenever q and o of the G heads fit its register budget.
-// Copies are issued per 64-token tile (large copies keep the copy engine's per-copy cost low); a warp
-// works on a quarter (thin variant) or half (fat variant) of a tile so that the slots being consumed
-// leave room in the ring for tiles in flight.
-template <int G> constexpr bool thin_variant() { return G == 2 || G == 4; }
-template <int G> constexpr int consumer_warps() { return thin_variant<G>() ? 15 : 7; }
-constexpr int kMaxDynSmem = 232448;            // 227 KB opt-in limit per CTA on sm_100
-constexpr long long kWaitCycles = 2000000000LL;  // bounded waits give up after about a second
+constexpr int kCW = 7;                          // consumer warps (+1 producer warp)
+constexpr int kThreads = (kCW + 1) * 32;
+constexpr int kItemRows = 16;                   // tokens per consumer work item
+constexpr int kItems = kTile / kItemRows;       // work items per tile
+constexpr int kMaxDynSmem = 232448;             // 227 KB opt-in limit per CTA on sm_100
+constexpr long long kWaitCycles = 2000000000LL; // bounded waits give up after about a second
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr uint32_t kTagNew = 0x8000u;           // tile tag: the unit's new-token pseudo tile (no copy)
 
 struct StreamParams {
-    const DevSeg *segs;
     const DevReq *reqs;
+    const CUtensorMap *tmaps;   // [n_seg_total] chunk maps, then tail K, tail V
+    const DevSeg *segs;         // [n_seg_total]
+    int32_t n_seg_total;
     const int32_t *tail_len;
     __nv_bfloat16 *tail_k, *tail_v;
     const __nv_bfloat16 *q, *k_new, *v_new;
@@ -83,14 +89,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
-// A consumer's wait for fill number `want` of a ring slot.  Warps take work items round-robin, so a
-// warp can reach a slot whose PREVIOUS fill is still in flight, and the one-bit phase of an mbarrier
+// A consumer's wait for fill number `want` of a ring stage.  Warps take work items round-robin, so a
+// warp can reach a stage whose PREVIOUS fill is still in flight, and the one-bit phase of an mbarrier
 // cannot tell "fill n-1 incomplete" from "fill n complete".  The producer therefore publishes the fill
-// number of a slot (upper half of the slot's tag word) before it issues the copy, which it does only
-// after the slot's previous fill was consumed and released; once the consumer sees its number there,
-// the parity test is unambiguous.  Returns the tag word, or 0 after the bounded wait ran out.
-__device__ __forceinline__ uint32_t slot_wait(const volatile uint32_t *tag, uint32_t want, uint32_t bar, uint32_t parity,
-                                              volatile int *abort_flag) {
+// number of a stage (upper half of the stage's tag word) before it issues the copies, which it does
+// only after the stage's previous fill was consumed and released; once the consumer sees its number
+// there, the parity test is unambiguous.  Returns the tag word, or 0 after the bounded wait ran out.
+__device__ __forceinline__ uint32_t stage_wait(const volatile uint32_t *tag, uint32_t want, uint32_t bar, uint32_t parity,
+                                               volatile int *abort_flag) {
     uint32_t w = *tag;
     if ((w >> 16) == (want & 0xffffu) && mbar_try_wait(bar, parity)) return w;
     const long long t0 = clock64();
@@ -104,34 +110,53 @@ __device__ __forceinline__ uint32_t slot_wait(const volatile uint32_t *tag, uint
         }
     }
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
+// TMA: one 64-column x kTile-row box of a [rows][D] bf16 tensor, starting at column x (a multiple of
+// 64: 128 bytes, so the 16-byte rule on the innermost coordinate holds) and row y.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
 }
-template <int CW> __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(CW * 32) : "memory"); }
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kCW * 32) : "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
 }
 __device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 // ---- the flat work list ----------------------------------------------------------------------------
 __host__ __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
-// sum over i in [0, S) of ceil((i + 1) / kTile)
-__host__ __device__ __forceinline__ int64_t new_tiles_sum(int S) {
-    const int64_t full = S / kTile, rem = S % kTile;
-    return (int64_t)kTile * full * (full + 1) / 2 + rem * (full + 1);
-}
 
 struct UnitPos {
-    int32_t l_rel, b, i, g;  // layer (relative to layer0), request, suffix token, KV head
-    int32_t tile;            // first tile of this CTA's share inside the unit
-    int32_t rt;              // tiles in the unit
+    int32_t l_rel, b, blk, g;  // layer (relative to layer0), request, block of suffix tokens, KV head
+    int32_t tile;              // first tile of this CTA's share inside the unit
+    int32_t rt;                // tiles in the unit: chunk tiles, tail tiles, one pseudo tile for the new tokens
     int32_t chunk_tiles, tail_tiles, t0, seg_begin;
-    int64_t flat_begin;      // flat index of the unit's first tile
+    int64_t flat_begin;        // flat index of the unit's first tile
 };
 
 struct CtaRange {
@@ -154,33 +179,29 @@ __device__ __forceinline__ void load_req(const StreamParams &p, UnitPos &u) {
     u.chunk_tiles = rq.chunk_tiles;
     u.seg_begin = rq.seg_begin;
     u.tail_tiles = ceil_div(u.t0, kTile);
+    u.rt = u.chunk_tiles + u.tail_tiles + 1;
 }
-__device__ __forceinline__ void set_rt(UnitPos &u) { u.rt = u.chunk_tiles + u.tail_tiles + ceil_div(u.i + 1, kTile); }
 
-// advance to the next unit in (layer, request, token, head) order
-__device__ __forceinline__ void next_unit(const StreamParams &p, UnitPos &u) {
+// advance to the next unit in (layer, request, token block, head) order
+__device__ __forceinline__ void next_unit(const StreamParams &p, UnitPos &u, int n_blk) {
     u.flat_begin += u.rt;
     u.tile = 0;
     if (++u.g < p.Hkv) return;
     u.g = 0;
-    if (++u.i < p.S) {
-        set_rt(u);
-        return;
-    }
-    u.i = 0;
+    if (++u.blk < n_blk) return;
+    u.blk = 0;
     if (++u.b >= p.B) {
         u.b = 0;
         ++u.l_rel;
     }
     if (u.l_rel < p.n_layers_launch) load_req(p, u);
-    set_rt(u);
 }
 
-__device__ void locate_range(const StreamParams &p, CtaRange &r) {
+__device__ void locate_range(const StreamParams &p, CtaRange &r, int n_blk) {
     int64_t w_layer = 0;
     for (int b = 0; b < p.B; ++b) {
-        const int base = p.reqs[b].chunk_tiles + ceil_div(clamp_t0(p, b), kTile);
-        w_layer += (int64_t)p.Hkv * ((int64_t)p.S * base + new_tiles_sum(p.S));
+        const int rt = p.reqs[b].chunk_tiles + ceil_div(clamp_t0(p, b), kTile) + 1;
+        w_layer += (int64_t)p.Hkv * n_blk * rt;
     }
     r.W = w_layer * p.n_layers_launch;
     const int64_t n = gridDim.x, c = blockIdx.x;
@@ -189,26 +210,20 @@ __device__ void locate_range(const StreamParams &p, CtaRange &r) {
     UnitPos &u = r.first;
     u = UnitPos{};
     if (r.begin >= r.end) return;
-    int64_t f = r.begin;
+    const int64_t f = r.begin;
     u.l_rel = (int32_t)(f / w_layer);
     int64_t rem = f % w_layer;
     int b = 0;
     for (; b < p.B; ++b) {
-        const int base = p.reqs[b].chunk_tiles + ceil_div(clamp_t0(p, b), kTile);
-        const int64_t blk = (int64_t)p.Hkv * ((int64_t)p.S * base + new_tiles_sum(p.S));
+        const int rt = p.reqs[b].chunk_tiles + ceil_div(clamp_t0(p, b), kTile) + 1;
+        const int64_t blk = (int64_t)p.Hkv * n_blk * rt;
         if (rem < blk) break;
         rem -= blk;
     }
     u.b = b;
     load_req(p, u);
-    int i = 0;
-    for (; i < p.S; ++i) {
-        const int64_t blk = (int64_t)p.Hkv * (u.chunk_tiles + u.tail_tiles + ceil_div(i + 1, kTile));
-        if (rem < blk) break;
-        rem -= blk;
-    }
-    u.i = i;
-    set_rt(u);
+    u.blk = (int32_t)(rem / ((int64_t)p.Hkv * u.rt));
+    rem -= (int64_t)u.blk * p.Hkv * u.rt;
     u.g = (int32_t)(rem / u.rt);
     u.tile = (int32_t)(rem % u.rt);
     u.flat_begin = f - u.tile;
@@ -216,61 +231,6 @@ __device__ void locate_range(const StreamParams &p, CtaRange &r) {
 
 // CTA that owns flat tile f when W tiles are split over n CTAs as [c*W/n, (c+1)*W/n)
 __device__ __forceinline__ int cta_of(int64_t f, int64_t W, int64_t n) { return (int)(((f + 1) * n - 1) / W); }
-
-// Where a unit's tile lives.
-struct TileSrc {
-    const __nv_bfloat16 *k, *v;  // first row
-    int64_t row_stride;          // elements between rows
-    int32_t rows;
-    int32_t new_first;           // >= 0: tile holds new tokens new_first .. new_first+rows-1; else -1
-};
-
-// The producer's cursor over a request's segments.  Tile indices only grow inside a unit, so the
-// current segment stays in registers and global memory is touched once per segment, not per tile.
-struct SegCursor {
-    int32_t seg, tiles_before, seg_tiles;
-    DevSeg sg;
-    __device__ __forceinline__ void reset() { seg = -1; tiles_before = 0; seg_tiles = 0; }
-};
-
-template <int D>
-__device__ __forceinline__ TileSrc tile_source(const StreamParams &p, const UnitPos &u, int tile, SegCursor &cur) {
-    TileSrc s;
-    const int layer = p.layer0 + u.l_rel;
-    if (tile < u.chunk_tiles) {
-        while (cur.seg < 0 || tile >= cur.tiles_before + cur.seg_tiles) {
-            cur.tiles_before += cur.seg_tiles;
-            ++cur.seg;
-            cur.sg = p.segs[u.seg_begin + cur.seg];
-            cur.seg_tiles = ceil_div(cur.sg.len, kTile);
-        }
-        const int r0 = (tile - cur.tiles_before) * kTile;
-        const int64_t kslab = ((int64_t)layer * 2 * p.Hkv + u.g) * cur.sg.len;
-        const int64_t vslab = (((int64_t)layer * 2 + 1) * p.Hkv + u.g) * cur.sg.len;
-        s.k = cur.sg.base + (kslab + r0) * D;
-        s.v = cur.sg.base + (vslab + r0) * D;
-        s.row_stride = D;
-        s.rows = min(kTile, cur.sg.len - r0);
-        s.new_first = -1;
-    } else if (tile < u.chunk_tiles + u.tail_tiles) {
-        const int r0 = (tile - u.chunk_tiles) * kTile;
-        const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + r0) * D;
-        s.k = p.tail_k + off;
-        s.v = p.tail_v + off;
-        s.row_stride = D;
-        s.rows = min(kTile, u.t0 - r0);
-        s.new_first = -1;
-    } else {
-        const int r0 = (tile - u.chunk_tiles - u.tail_tiles) * kTile;
-        const int64_t off = (int64_t)u.l_rel * p.kn_sl + (int64_t)u.b * p.kn_sb + (int64_t)r0 * p.kn_ss + (int64_t)u.g * D;
-        s.k = p.k_new + off;
-        s.v = p.v_new + off;
-        s.row_stride = p.kn_ss;
-        s.rows = min(kTile, u.i + 1 - r0);
-        s.new_first = r0;
-    }
-    return s;
-}
 
 // ---- K2 core: merge P partial attentions of one row with one warp -----------------------------------
 // o_parts: part p at o_parts + p*o_stride (D floats, normalised inside the part); lse natural log.
@@ -311,146 +271,140 @@ __global__ void k_lse_combine(int n_rows, int P, int D, const float *__restrict_
 }
 
 // ---- K1 -------------------------------------------------------------------------------------------
-// packed fp32 pairs: sm_100 issues two FMAs per instruction on a 64-bit register pair
-__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
-    unsigned long long d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;"
-        : "=l"(d)
-        : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)),
-          "l"(*reinterpret_cast<unsigned long long *>(&c)));
-    return *reinterpret_cast<float2 *>(&d);
-}
-__device__ __forceinline__ float2 fmul2(float2 a, float2 b) {
-    unsigned long long d;
-    asm("mul.rn.f32x2 %0, %1, %2;"
-        : "=l"(d)
-        : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)));
-    return *reinterpret_cast<float2 *>(&d);
-}
-__device__ __forceinline__ float2 bf2(uint32_t w) { return make_float2(bf_lo(w), bf_hi(w)); }
-
 template <int D, int G>
 struct StreamCfg {
-    static constexpr int CW = consumer_warps<G>();             // consumer warps
-    static constexpr int THREADS = (CW + 1) * 32;
-    static constexpr int SPLIT = thin_variant<G>() ? 4 : 2;    // warps that share one tile
-    static constexpr int HROWS = kTile / SPLIT;                // rows of a tile one warp handles
-    static constexpr int LPR = (D == 128 && (SPLIT == 2 || G == 8)) ? 16 : 8;  // lanes that share one K/V row
-    static constexpr int DPL = D / LPR;                        // dims per lane
-    static constexpr int NV = DPL / 8;                         // 16-byte vectors per lane per row
-    static constexpr int NPAIR = DPL / 2;                      // fp32 pairs per lane per row
-    static constexpr int RG = 32 / LPR;                        // row groups per warp
-    static constexpr int RPG = HROWS / RG;                     // rows per group per work item
-    static constexpr int SUBR = (RPG < 32 / G) ? RPG : 32 / G; // rows per group per reduce batch
-    static constexpr int NSUB = RPG / SUBR;
-    static constexpr int NP = G * SUBR;                        // partial dot products per lane per batch
-    static constexpr int NF = NP / LPR;                        // scores per lane after the reduce-scatter
-    static constexpr int LPH = LPR / G;                        // lanes of a group that end up with the same head
-    static constexpr int SLOT_BYTES = kTile * D * 2;
-    static constexpr int MERGE_BYTES = (CW * G * (D + 2) * 4 + 15) / 16 * 16;
-    static constexpr int PS_STRIDE = (HROWS * G * 2 + G + 3) / 4 * 4;  // floats per warp: p pairs [row][head], alpha[head]
-    static constexpr int PS_BYTES = CW * PS_STRIDE * 4;
-    static constexpr int FIXED_BYTES = MERGE_BYTES + PS_BYTES + 1024;
-    static constexpr int NSLOT_MAX = (kMaxDynSmem - FIXED_BYTES) / SLOT_BYTES;
-    static constexpr int NSLOT = NSLOT_MAX > 24 ? 24 : NSLOT_MAX;
-    static constexpr int SMEM_BYTES = NSLOT * SLOT_BYTES + FIXED_BYTES;
-    static_assert(DPL % 8 == 0 && NF >= 1 && SUBR % NF == 0 && LPH >= 1, "unsupported head_dim / group size");
-    static_assert(NSLOT >= 4, "ring too small");
+    static constexpr int TPU = kUnitRows / G;              // suffix tokens per unit
+    static constexpr int NBOX = D / 64;                    // 64-column TMA boxes per row
+    static constexpr int BOX_BYTES = kTile * 128;          // one box: kTile rows x 128 bytes (swizzled)
+    static constexpr int STAGE_BYTES = 2 * NBOX * BOX_BYTES;  // K boxes then V boxes
+    static constexpr int KS = D / 16;                      // k-steps of S = Q K^T; also n-block pairs of O += P V
+    static constexpr int MERGE_BYTES = (kCW * kUnitRows * (D + 2) * 4 + 15) / 16 * 16;
+    static constexpr int FIXED_BYTES = MERGE_BYTES + 1024 + 1024;  // + misc + slack for 1024-byte alignment of the ring
+    static constexpr int NSTAGE_MAX = (kMaxDynSmem - FIXED_BYTES) / STAGE_BYTES;
+    static constexpr int NSTAGE = NSTAGE_MAX > 12 ? 12 : NSTAGE_MAX;
+    static constexpr int SMEM_BYTES = NSTAGE * STAGE_BYTES + FIXED_BYTES;
+    static_assert(G >= 1 && G <= kUnitRows && kUnitRows % G == 0, "unsupported group size");
+    static_assert(D % 64 == 0 && NSTAGE >= 3, "unsupported head_dim");
 };
 
+// byte offset of 16-byte chunk c of row r inside one 128-byte-swizzled box
+__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
+
 template <int D, int G>
-__global__ void __launch_bounds__((consumer_warps<G>() + 1) * 32, 1) k_attend_stream(const StreamParams p) {
+__global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParams p) {
     using C = StreamCfg<D, G>;
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ unsigned char smem_raw[];
+    // the swizzle pattern repeats every 1024 bytes: align the ring to it
+    unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char *ring = smem;
-    float *merge_o = (float *)(smem + C::NSLOT * C::SLOT_BYTES);         // [warp][G][D]
-    float *merge_m = merge_o + C::CW * G * D;                   // [warp][G]
-    float *merge_l = merge_m + C::CW * G;                       // [warp][G]
-    float *ps_all = (float *)(smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES);  // [warp][PS_STRIDE]
-    unsigned char *misc = smem + C::NSLOT * C::SLOT_BYTES + C::MERGE_BYTES + C::PS_BYTES;
-    uint64_t *bars = (uint64_t *)misc;                                   // full[NSLOT], empty[NSLOT]
-    // per slot tag: rows | (the unit's own new row + 1) << 8 | (number of the slot's current fill) << 16
-    volatile uint32_t *tags = (volatile uint32_t *)(misc + 2 * 24 * 8);
-    CtaRange *range = (CtaRange *)(misc + 2 * 24 * 8 + 2 * 24 * 4);
-    volatile int *flags = (volatile int *)(misc + 2 * 24 * 8 + 2 * 24 * 4 + sizeof(CtaRange) + 8);  // [0] abort, [1] last arriver
+    float *merge_o = (float *)(smem + C::NSTAGE * C::STAGE_BYTES);  // [warp][row][D]
+    float *merge_m = merge_o + kCW * kUnitRows * D;                 // [warp][row]  (log2 units, scaled)
+    float *merge_l = merge_m + kCW * kUnitRows;                     // [warp][row]
+    unsigned char *misc = smem + C::NSTAGE * C::STAGE_BYTES + C::MERGE_BYTES;
+    uint64_t *bars = (uint64_t *)misc;                              // full[NSTAGE], empty[NSTAGE]
+    // per stage tag: valid rows | kTagNew | (number of the stage's current fill) << 16
+    volatile uint32_t *tags = (volatile uint32_t *)(misc + 2 * 12 * 8);
+    CtaRange *range = (CtaRange *)(misc + 2 * 12 * 8 + 12 * 4 + 8);
+    volatile int *flags = (volatile int *)(misc + 2 * 12 * 8 + 12 * 4 + 8 + sizeof(CtaRange) + 8);  // [0] abort, [1] last arriver
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_blk = ceil_div(p.S, C::TPU);
     if (tid == 0) {
-        for (int s = 0; s < C::NSLOT; ++s) {
+        for (int s = 0; s < C::NSTAGE; ++s) {
             mbar_init(smem_u32(bars + s), 1);
-            mbar_init(smem_u32(bars + C::NSLOT + s), C::SPLIT);
+            mbar_init(smem_u32(bars + C::NSTAGE + s), kItems);
             tags[s] = 0xffff0000u;
         }
         flags[0] = 0;
         flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        locate_range(p, *range);
+        locate_range(p, *range, n_blk);
     }
     __syncthreads();
     const int64_t f_begin = range->begin, f_end = range->end, W = range->W;
     if (f_begin >= f_end) return;
-    const uint32_t ring_u32 = smem_u32(ring), full_u32 = smem_u32(bars), empty_u32 = smem_u32(bars + C::NSLOT);
+    const uint32_t ring_u32 = smem_u32(ring), full_u32 = smem_u32(bars), empty_u32 = smem_u32(bars + C::NSTAGE);
 
-    if (warp == C::CW) {
+    if (warp == kCW) {
         // ================= producer: one thread walks the table and feeds the ring =================
         if (lane != 0) return;
         UnitPos u = range->first;
-        SegCursor cur;
-        cur.reset();
+        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;  // cursor over the request's segments
         int64_t f = f_begin;
         uint32_t seq = 0;
         bool ok = true;
         while (f < f_end && ok) {
             const int t_end = (int)min((int64_t)u.rt, f_end - u.flat_begin);
-            for (int t = u.tile; t < t_end && ok; ++t, ++f) {
-                const TileSrc s = tile_source<D>(p, u, t, cur);
-                uint32_t m = (uint32_t)s.rows;
-                if (s.new_first >= 0 && u.i >= s.new_first && u.i < s.new_first + s.rows) m |= (uint32_t)(u.i - s.new_first + 1) << 8;
+            const int layer = p.layer0 + u.l_rel;
+            for (int t = u.tile; t < t_end; ++t, ++f, ++seq) {
+                const uint32_t stage = seq % C::NSTAGE, use = seq / C::NSTAGE;
+                if (use > 0 && !mbar_wait(empty_u32 + stage * 8, (use - 1) & 1, flags)) {
+                    ok = false;
+                    break;
+                }
+                const uint32_t bar = full_u32 + stage * 8, dst = ring_u32 + stage * C::STAGE_BYTES;
+                if (t >= u.chunk_tiles + u.tail_tiles) {  // the new tokens: nothing to copy
+                    tags[stage] = kTagNew | (use << 16);
+                    mbar_arrive(bar);
+                    continue;
+                }
+                const CUtensorMap *mk, *mv;
+                int32_t yk, yv, rows;
+                if (t < u.chunk_tiles) {
+                    while (seg < 0 || t >= tiles_before + seg_tiles) {
+                        tiles_before += seg_tiles;
+                        ++seg;
+                        seg_len = p.segs[u.seg_begin + seg].len;
+                        seg_tiles = ceil_div(seg_len, kTile);
+                    }
+                    const int r0 = (t - tiles_before) * kTile;
+                    mk = mv = p.tmaps + u.seg_begin + seg;
+                    yk = ((layer * 2) * p.Hkv + u.g) * seg_len + r0;
+                    yv = ((layer * 2 + 1) * p.Hkv + u.g) * seg_len + r0;
+                    rows = min(kTile, seg_len - r0);
+                } else {
+                    const int r0 = (t - u.chunk_tiles) * kTile;
+                    mk = p.tmaps + p.n_seg_total;
+                    mv = mk + 1;
+                    yk = yv = ((u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + r0;
+                    rows = min(kTile, u.t0 - r0);
+                }
+                tags[stage] = (uint32_t)rows | (use << 16);  // published only after the stage's previous fill was released
+                mbar_expect_tx(bar, C::STAGE_BYTES);
 #pragma unroll
-                for (int kv = 0; kv < 2; ++kv, ++seq) {
-                    const uint32_t slot = seq % C::NSLOT, use = seq / C::NSLOT;
-                    if (use > 0 && !mbar_wait(empty_u32 + slot * 8, (use - 1) & 1, flags)) {
-                        ok = false;
-                        break;
-                    }
-                    const __nv_bfloat16 *src = kv ? s.v : s.k;
-                    const uint32_t dst = ring_u32 + slot * C::SLOT_BYTES, bar = full_u32 + slot * 8;
-                    tags[slot] = m | (use << 16);  // published only after the slot's previous fill was consumed and released
-                    mbar_expect_tx(bar, (uint32_t)s.rows * D * 2);
-                    if (s.row_stride == D) {
-                        bulk_g2s(dst, src, (uint32_t)s.rows * D * 2, bar);
-                    } else {
-                        for (int r = 0; r < s.rows; ++r) bulk_g2s(dst + r * D * 2, src + (int64_t)r * s.row_stride, D * 2, bar);
-                    }
+                for (int bx = 0; bx < C::NBOX; ++bx) {
+                    tma_load_2d(dst + bx * C::BOX_BYTES, mk, bx * 64, yk, bar);
+                    tma_load_2d(dst + (C::NBOX + bx) * C::BOX_BYTES, mv, bx * 64, yv, bar);
                 }
             }
             if (f < f_end && ok) {
-                next_unit(p, u);
-                cur.reset();
+                next_unit(p, u, n_blk);
+                seg = -1; tiles_before = 0; seg_tiles = 0;
             }
         }
         if (!ok) {
             // gave up: wait (bounded) for the copies already issued so none lands after the CTA has gone
             atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
-            const uint32_t lo = seq > (uint32_t)C::NSLOT ? seq - C::NSLOT : 0;
+            const uint32_t lo = seq > (uint32_t)C::NSTAGE ? seq - C::NSTAGE : 0;
             for (uint32_t s2 = lo; s2 < seq; ++s2) {
                 const long long t0 = clock64();
-                while (!mbar_try_wait(full_u32 + (s2 % C::NSLOT) * 8, (s2 / C::NSLOT) & 1) && clock64() - t0 < kWaitCycles) {}
+                while (!mbar_try_wait(full_u32 + (s2 % C::NSTAGE) * 8, (s2 / C::NSTAGE) & 1) && clock64() - t0 < kWaitCycles) {}
             }
         }
         return;
     }
 
     // ================= consumers =================
-    const int grp = lane / C::LPR, jl = lane % C::LPR;
-    const int my_h = jl / C::LPH;  // head whose scores this lane holds after the reduce-scatter
-    float *ps = ps_all + warp * C::PS_STRIDE;     // this warp's (p, p)[row][head], then alpha[head]
-    float *alpha_s = ps + C::HROWS * G * 2;
+    // mma fragment coordinates of this thread: query row `qr` (rows 8..15 of the 16-row tile are padding),
+    // column pair `qc` (two adjacent columns 2*qc, 2*qc+1 of every 8-column block)
+    const int qr = lane >> 2, qc = lane & 3;
+    // ldmatrix row addressing: matrix mi = lane / 8 of the x4 group, row ri = lane % 8 inside it
+    const int mi = lane >> 3, ri = lane & 7;
 
-    float2 qf[G][C::NPAIR];
-    float2 of[G][C::NPAIR];
-    float m_run = -CUDART_INF_F, l_run = 0.f;
+    uint32_t qa[C::KS][2];   // A fragments of Q for the real rows: [k-step][cols 0-7 | cols 8-15]
+    float o[2 * C::KS][4];   // O accumulators: [8-column block of d][c0, c1 real row; c2, c3 padding rows]
+    float m_run = -CUDART_INF_F, l_run = 0.f;  // running max (scaled, log2 units) and this thread's share of the sum
 
     UnitPos u = range->first;
     int64_t f_unit = f_begin;   // flat index of this CTA's first tile inside the current unit
@@ -459,270 +413,216 @@ __global__ void __launch_bounds__((consumer_warps<G>() + 1) * 32, 1) k_attend_st
         const int t_begin = u.tile;
         const int t_end = (int)min((int64_t)u.rt, f_end - u.flat_begin);
         const int layer = p.layer0 + u.l_rel;
-        // ---- per-unit setup: query (pre-scaled by scale*log2 e), cleared state ----
+        const int tok0 = u.blk * C::TPU;                    // first suffix token of the unit
+        const int n_tok = min(C::TPU, p.S - tok0);
+        const int n_rows = n_tok * G;                       // real query rows: row = token * G + head
+        const int64_t q_base = (int64_t)u.l_rel * p.q_sl + (int64_t)u.b * p.q_sb + (int64_t)tok0 * p.q_ss + (int64_t)u.g * G * D;
+        // ---- per-unit setup ----
         {
-            const __nv_bfloat16 *qb = p.q + (int64_t)u.l_rel * p.q_sl + (int64_t)u.b * p.q_sb + (int64_t)u.i * p.q_ss +
-                                      (int64_t)u.g * G * D;
-            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2);
+            const bool real = qr < n_rows;
+            const __nv_bfloat16 *qrow = p.q + q_base + (int64_t)(qr / G) * p.q_ss + (qr % G) * D;
 #pragma unroll
-            for (int h = 0; h < G; ++h)
+            for (int ks = 0; ks < C::KS; ++ks) {
+                qa[ks][0] = real ? *(const uint32_t *)(qrow + ks * 16 + 2 * qc) : 0u;
+                qa[ks][1] = real ? *(const uint32_t *)(qrow + ks * 16 + 8 + 2 * qc) : 0u;
+            }
 #pragma unroll
-                for (int v = 0; v < C::NV; ++v) {
-                    const uint4 w = *(const uint4 *)(qb + h * D + (v * C::LPR + jl) * 8);
-                    qf[h][v * 4 + 0] = fmul2(bf2(w.x), sc2);
-                    qf[h][v * 4 + 1] = fmul2(bf2(w.y), sc2);
-                    qf[h][v * 4 + 2] = fmul2(bf2(w.z), sc2);
-                    qf[h][v * 4 + 3] = fmul2(bf2(w.w), sc2);
-                }
-#pragma unroll
-            for (int h = 0; h < G; ++h)
-#pragma unroll
-                for (int d = 0; d < C::NPAIR; ++d) of[h][d] = make_float2(0.f, 0.f);
+            for (int nb = 0; nb < 2 * C::KS; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
             m_run = -CUDART_INF_F;
             l_run = 0.f;
         }
         // ---- this warp's work items of the unit ----
-        // CTA-local tile j = j_base + (t - t_begin) splits into SPLIT work items hj = j*SPLIT + half;
-        // warp w takes hj == w (mod CW)
-        const int64_t hj_begin = j_base * C::SPLIT, hj_end = (j_base + (t_end - t_begin)) * C::SPLIT;
-        int64_t hj = hj_begin + (int)((warp - hj_begin % C::CW + C::CW) % C::CW);
-        for (; hj < hj_end; hj += C::CW) {
-            const int64_t j = hj / C::SPLIT;
-            const int row0 = (int)(hj % C::SPLIT) * C::HROWS;
-            const uint32_t seq_k = (uint32_t)(2 * j), seq_v = seq_k + 1;
-            const uint32_t slot_k = seq_k % C::NSLOT, slot_v = seq_v % C::NSLOT;
-            const unsigned char *ks = ring + slot_k * C::SLOT_BYTES + row0 * (D * 2);
-            const unsigned char *vs = ring + slot_v * C::SLOT_BYTES + row0 * (D * 2);
+        // CTA-local tile j = j_base + (t - t_begin) splits into kItems work items hj = j*kItems + piece;
+        // warp w takes hj == w (mod kCW)
+        const int64_t hj_begin = j_base * kItems, hj_end = (j_base + (t_end - t_begin)) * kItems;
+        int64_t hj = hj_begin + (int)((warp - hj_begin % kCW + kCW) % kCW);
+        for (; hj < hj_end; hj += kCW) {
+            const uint32_t j = (uint32_t)(hj / kItems);
+            const int piece = (int)(hj % kItems);
+            const int r0 = piece * kItemRows;
+            const uint32_t stage = j % C::NSTAGE, use = j / C::NSTAGE;
+            const uint32_t tag = stage_wait(tags + stage, use, full_u32 + stage * 8, use & 1, flags);
+            const uint32_t stage_u32 = ring_u32 + stage * C::STAGE_BYTES;
 
-            // ---------- scores ----------
-            const uint32_t mt = slot_wait(tags + slot_k, seq_k / C::NSLOT, full_u32 + slot_k * 8, (seq_k / C::NSLOT) & 1, flags);
-            const int rows = (int)(mt & 0xff) - row0;   // valid rows of this work item (may be <= 0)
-            int own_row = (int)((mt >> 8) & 0xff) - 1 - row0;  // the unit's own new token, if it sits in this work item
-            if (own_row >= C::HROWS) own_row = -1;
-            if (rows <= 0) {                            // the tile ends before this half: just release the slots
-                slot_wait(tags + slot_v, seq_v / C::NSLOT, full_u32 + slot_v * 8, (seq_v / C::NSLOT) & 1, flags);
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(empty_u32 + slot_k * 8);
-                    mbar_arrive(empty_u32 + slot_v * 8);
+            if (tag & kTagNew) {
+                // ---------- the call's new tokens (scalar path, one warp per unit) ----------
+                if (piece == 0) {
+                    const int n_new = tok0 + n_tok;  // new rows 0 .. tok0+n_tok-1 exist; row `qr` sees 0 .. tok0 + qr/G
+                    const int my_last = tok0 + qr / G;
+                    constexpr int DL = D / 32;       // dims per lane in the dot product
+                    float qs[kUnitRows][DL];
+#pragma unroll
+                    for (int r = 0; r < kUnitRows; ++r) {
+                        const __nv_bfloat16 *qrow = p.q + q_base + (int64_t)(r / G) * p.q_ss + (r % G) * D + lane * DL;
+#pragma unroll
+                        for (int d = 0; d < DL; ++d) qs[r][d] = r < n_rows ? __bfloat162float(qrow[d]) : 0.f;
+                    }
+                    const int64_t kn_base = (int64_t)u.l_rel * p.kn_sl + (int64_t)u.b * p.kn_sb + (int64_t)u.g * D;
+                    for (int jn = 0; jn < n_new; ++jn) {
+                        const __nv_bfloat16 *krow = p.k_new + kn_base + (int64_t)jn * p.kn_ss;
+                        const __nv_bfloat16 *vrow = p.v_new + kn_base + (int64_t)jn * p.kn_ss;
+                        float kd[DL];
+#pragma unroll
+                        for (int d = 0; d < DL; ++d) kd[d] = __bfloat162float(krow[lane * DL + d]);
+                        float mine = 0.f;
+#pragma unroll
+                        for (int r = 0; r < kUnitRows; ++r) {
+                            float a = 0.f;
+#pragma unroll
+                            for (int d = 0; d < DL; ++d) a = fmaf(qs[r][d], kd[d], a);
+#pragma unroll
+                            for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+                            if (r == qr) mine = a;
+                        }
+                        const bool vis = qr < n_rows && jn <= my_last;
+                        const float s = vis ? mine * p.scale_log2 : -CUDART_INF_F;
+                        const float m_new = fmaxf(m_run, s);
+                        const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);
+                        const float pv = vis ? fast_exp2(s - m_new) : 0.f;
+                        l_run = l_run * alpha + (qc == 0 ? pv : 0.f);
+                        m_run = m_new;
+#pragma unroll
+                        for (int nb = 0; nb < 2 * C::KS; ++nb) {
+                            const uint32_t vv = *(const uint32_t *)(vrow + nb * 8 + 2 * qc);
+                            o[nb][0] = fmaf(pv, bf_lo(vv), o[nb][0] * alpha);
+                            o[nb][1] = fmaf(pv, bf_hi(vv), o[nb][1] * alpha);
+                        }
+                        // the unit's own tokens go to the tail for later calls
+                        if (jn >= tok0 && u.t0 + jn < p.max_tail) {
+                            const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + u.t0 + jn) * D;
+                            if (lane < D / 8) {
+                                *(uint4 *)(p.tail_k + off + lane * 8) = *(const uint4 *)(krow + lane * 8);
+                                *(uint4 *)(p.tail_v + off + lane * 8) = *(const uint4 *)(vrow + lane * 8);
+                            }
+                        }
+                    }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_u32 + stage * 8);
                 continue;
             }
-            float sc[C::NSUB][C::NF];
-#pragma unroll
-            for (int sub = 0; sub < C::NSUB; ++sub) {
-                float part[C::NP];
-#pragma unroll
-                for (int r = 0; r < C::SUBR; ++r) {
-                    const int row = (sub * C::SUBR + r) * C::RG + grp;
-                    float2 kf[C::NPAIR];
-#pragma unroll
-                    for (int v = 0; v < C::NV; ++v) {
-                        const uint4 w = *(const uint4 *)(ks + row * (D * 2) + (v * C::LPR + jl) * 16);
-                        kf[v * 4 + 0] = bf2(w.x); kf[v * 4 + 1] = bf2(w.y);
-                        kf[v * 4 + 2] = bf2(w.z); kf[v * 4 + 3] = bf2(w.w);
-                    }
-#pragma unroll
-                    for (int h = 0; h < G; ++h) {
-                        float2 a = make_float2(0.f, 0.f);
-#pragma unroll
-                        for (int d = 0; d < C::NPAIR; ++d) a = ffma2(qf[h][d], kf[d], a);
-                        part[h * C::SUBR + r] = a.x + a.y;
-                    }
-                }
-                // reduce-scatter over the LPR lanes of the row group: afterwards this lane holds the
-                // complete dot products number base + 0..NF-1, base = its lane bits read as an index
-                int n = C::NP;
-#pragma unroll
-                for (int off = C::LPR / 2; off >= 1; off >>= 1) {
-                    n >>= 1;
-                    const bool upper = (jl & off) != 0;
-#pragma unroll
-                    for (int k = 0; k < n; ++k) {
-                        const float send = upper ? part[k] : part[k + n];
-                        const float keep = upper ? part[k + n] : part[k];
-                        part[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-                    }
-                }
-#pragma unroll
-                for (int k = 0; k < C::NF; ++k) {
-                    const int r = (jl % C::LPH) * C::NF + k;  // row of the batch (head index = my_h)
-                    const int row = (sub * C::SUBR + r) * C::RG + grp;
-                    sc[sub][k] = row < rows ? part[k] : -CUDART_INF_F;
-                }
-            }
-            // the new token's K row goes to the tail for later steps (this unit's own token only)
-            if (own_row >= 0 && u.t0 + u.i < p.max_tail) {
-                const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + u.t0 + u.i) * D;
-                if (lane < D / 8) *(uint4 *)(p.tail_k + off + lane * 8) = *(const uint4 *)(ks + own_row * (D * 2) + lane * 16);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_u32 + slot_k * 8);
 
-            // ---------- online softmax over the tile ----------
-            float tmax = -CUDART_INF_F;
+            const int rows = (int)(tag & 0xff) - r0;  // valid rows of this work item (may be <= 0)
+            if (rows > 0) {
+                // ---------- S = Q K^T for 16 tokens (two 8-token blocks) ----------
+                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int sub = 0; sub < C::NSUB; ++sub)
-#pragma unroll
-                for (int k = 0; k < C::NF; ++k) tmax = fmaxf(tmax, sc[sub][k]);
-#pragma unroll
-            for (int off = 1; off < C::LPH; off <<= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, off));
-#pragma unroll
-            for (int off = C::LPR; off < 32; off <<= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, off));
-            const float m_new = fmaxf(m_run, tmax);  // finite: the work item has at least one valid row
-            const float alpha = fast_exp2(m_run - m_new);
-            float psum = 0.f;
-#pragma unroll
-            for (int sub = 0; sub < C::NSUB; ++sub)
-#pragma unroll
-                for (int k = 0; k < C::NF; ++k) {
-                    const float pv = fast_exp2(sc[sub][k] - m_new);
-                    psum += pv;
-                    const int r = (jl % C::LPH) * C::NF + k;
-                    const int row = (sub * C::SUBR + r) * C::RG + grp;
-                    *(float2 *)(ps + (row * G + my_h) * 2) = make_float2(pv, pv);
+                for (int ks = 0; ks < C::KS; ++ks) {
+                    // matrices: (tokens 0-7, d-chunk 2ks), (tokens 0-7, 2ks+1), (tokens 8-15, 2ks), (tokens 8-15, 2ks+1)
+                    const int c = (ks * 2 + (mi & 1)) & 7;
+                    uint32_t kb[4];
+                    ldsm_x4(stage_u32 + (ks / 4) * C::BOX_BYTES + swz(r0 + (mi >> 1) * 8 + ri, c), kb);
+                    mma_bf16(s0, qa[ks][0], 0u, qa[ks][1], 0u, kb[0], kb[1]);
+                    mma_bf16(s1, qa[ks][0], 0u, qa[ks][1], 0u, kb[2], kb[3]);
                 }
-            l_run = l_run * alpha + psum;
-            m_run = m_new;
-            alpha_s[my_h] = alpha;
-            const bool rescale = __any_sync(0xffffffffu, alpha != 1.0f);
-            __syncwarp();
-
-            // ---------- weighted sum of V ----------
-            if (rescale) {
+                // ---------- online softmax (this thread: row qr, tokens 2qc, 2qc+1, 8+2qc, 9+2qc) ----------
+                const float x0 = 2 * qc < rows ? s0[0] * p.scale_log2 : -CUDART_INF_F;
+                const float x1 = 2 * qc + 1 < rows ? s0[1] * p.scale_log2 : -CUDART_INF_F;
+                const float x2 = 8 + 2 * qc < rows ? s1[0] * p.scale_log2 : -CUDART_INF_F;
+                const float x3 = 9 + 2 * qc < rows ? s1[1] * p.scale_log2 : -CUDART_INF_F;
+                float tmax = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+                const float m_new = fmaxf(m_run, tmax);  // finite: token 0 of the item is valid
+                const float alpha = fast_exp2(m_run - m_new);
+                const float p0 = fast_exp2(x0 - m_new), p1 = fast_exp2(x1 - m_new);
+                const float p2 = fast_exp2(x2 - m_new), p3 = fast_exp2(x3 - m_new);
+                l_run = l_run * alpha + ((p0 + p1) + (p2 + p3));
+                m_run = m_new;
+                if (__any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll
-                for (int h = 0; h < G; ++h) {
-                    const float a = alpha_s[h];
-                    const float2 a2 = make_float2(a, a);
-#pragma unroll
-                    for (int d = 0; d < C::NPAIR; ++d) of[h][d] = fmul2(of[h][d], a2);
-                }
-            }
-            slot_wait(tags + slot_v, seq_v / C::NSLOT, full_u32 + slot_v * 8, (seq_v / C::NSLOT) & 1, flags);
-#pragma unroll
-            for (int r = 0; r < C::RPG; ++r) {
-                const int row = r * C::RG + grp;
-                if (row < rows) {
-                    float2 vf[C::NPAIR];
-#pragma unroll
-                    for (int v = 0; v < C::NV; ++v) {
-                        const uint4 w = *(const uint4 *)(vs + row * (D * 2) + (v * C::LPR + jl) * 16);
-                        vf[v * 4 + 0] = bf2(w.x); vf[v * 4 + 1] = bf2(w.y);
-                        vf[v * 4 + 2] = bf2(w.z); vf[v * 4 + 3] = bf2(w.w);
+                    for (int nb = 0; nb < 2 * C::KS; ++nb) {
+                        o[nb][0] *= alpha;
+                        o[nb][1] *= alpha;
                     }
-                    float2 pr[G];
-                    if constexpr (G % 2 == 0) {
-#pragma unroll
-                        for (int h2 = 0; h2 < G / 2; ++h2) {
-                            const float4 t4 = *(const float4 *)(ps + (row * G + h2 * 2) * 2);
-                            pr[h2 * 2 + 0] = make_float2(t4.x, t4.y);
-                            pr[h2 * 2 + 1] = make_float2(t4.z, t4.w);
-                        }
-                    } else {
-                        pr[0] = *(const float2 *)(ps + row * 2);
-                    }
-#pragma unroll
-                    for (int h = 0; h < G; ++h)
-#pragma unroll
-                        for (int d = 0; d < C::NPAIR; ++d) of[h][d] = ffma2(pr[h], vf[d], of[h][d]);
                 }
-            }
-            if (own_row >= 0 && u.t0 + u.i < p.max_tail) {
-                const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + u.t0 + u.i) * D;
-                if (lane < D / 8) *(uint4 *)(p.tail_v + off + lane * 8) = *(const uint4 *)(vs + own_row * (D * 2) + lane * 16);
+                const uint32_t pa0 = pack_bf16(p0, p1), pa2 = pack_bf16(p2, p3);
+                // ---------- O += P V ----------
+                const uint32_t v_u32 = stage_u32 + C::NBOX * C::BOX_BYTES;
+#pragma unroll
+                for (int dp = 0; dp < C::KS; ++dp) {
+                    // matrices: (tokens 0-7, d-chunk 2dp), (tokens 8-15, 2dp), (tokens 0-7, 2dp+1), (tokens 8-15, 2dp+1)
+                    const int c = (dp * 2 + (mi >> 1)) & 7;
+                    uint32_t vb[4];
+                    ldsm_x4_trans(v_u32 + (dp / 4) * C::BOX_BYTES + swz(r0 + (mi & 1) * 8 + ri, c), vb);
+                    mma_bf16(o[2 * dp], pa0, 0u, pa2, 0u, vb[0], vb[1]);
+                    mma_bf16(o[2 * dp + 1], pa0, 0u, pa2, 0u, vb[2], vb[3]);
+                }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty_u32 + slot_v * 8);
+            if (lane == 0) mbar_arrive(empty_u32 + stage * 8);
         }
 
         // ---- end of this CTA's share of the unit: merge the warps' states ----
         {
             float l_tot = l_run;
+            l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
+            l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
 #pragma unroll
-            for (int off = 1; off < C::LPH; off <<= 1) l_tot += __shfl_xor_sync(0xffffffffu, l_tot, off);
-#pragma unroll
-            for (int off = C::LPR; off < 32; off <<= 1) l_tot += __shfl_xor_sync(0xffffffffu, l_tot, off);
-#pragma unroll
-            for (int h = 0; h < G; ++h)
-#pragma unroll
-                for (int d = 0; d < C::NPAIR; ++d) {
-                    float2 x = of[h][d];
-#pragma unroll
-                    for (int off = C::LPR; off < 32; off <<= 1) {
-                        x.x += __shfl_xor_sync(0xffffffffu, x.x, off);
-                        x.y += __shfl_xor_sync(0xffffffffu, x.y, off);
-                    }
-                    of[h][d] = x;
-                }
-            if (grp == 0) {
-#pragma unroll
-                for (int h = 0; h < G; ++h)
-#pragma unroll
-                    for (int v = 0; v < C::NV; ++v)
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            *(float2 *)(merge_o + (warp * G + h) * D + (v * C::LPR + jl) * 8 + 2 * e) = of[h][v * 4 + e];
-                if (jl % C::LPH == 0) {
-                    merge_m[warp * G + my_h] = m_run;
-                    merge_l[warp * G + my_h] = l_tot;
-                }
+            for (int nb = 0; nb < 2 * C::KS; ++nb)
+                *(float2 *)(merge_o + (warp * kUnitRows + qr) * D + nb * 8 + 2 * qc) = make_float2(o[nb][0], o[nb][1]);
+            if (qc == 0) {
+                merge_m[warp * kUnitRows + qr] = m_run;
+                merge_l[warp * kUnitRows + qr] = l_tot;
             }
         }
-        consumer_bar<C::CW>();
-        const int64_t unit_index = (((int64_t)u.l_rel * p.B + u.b) * p.S + u.i) * p.Hkv + u.g;
+        consumer_bar();
+        const int64_t unit_index = (((int64_t)u.l_rel * p.B + u.b) * n_blk + u.blk) * p.Hkv + u.g;
         const int c_first = cta_of(u.flat_begin, W, gridDim.x);
         const int c_last = cta_of(u.flat_begin + u.rt - 1, W, gridDim.x);
         const int n_parts = c_last - c_first + 1;
-        const int64_t io_off = (int64_t)u.l_rel * p.q_sl + (int64_t)u.b * p.q_sb + (int64_t)u.i * p.q_ss + (int64_t)u.g * G * D;
-        const int64_t lse_off = (int64_t)u.l_rel * p.lse_sl + (int64_t)u.b * p.lse_sb + (int64_t)u.i * p.lse_ss + (int64_t)u.g * G;
+        const int64_t lse_base = (int64_t)u.l_rel * p.lse_sl + (int64_t)u.b * p.lse_sb + (int64_t)tok0 * p.lse_ss + (int64_t)u.g * G;
         const int64_t slot = unit_index + blockIdx.x;
         const bool slot_ok = slot < p.n_part_slots && unit_index < p.n_counter_slots;
         if (n_parts > 1 && !slot_ok && tid == 0) atomicCAS(p.status, 0, MATKV_E_BOUNDS);
-        for (int idx = tid; idx < G * D; idx += C::CW * 32) {
-            const int h = idx / D, d = idx % D;
+        for (int idx = tid; idx < n_rows * D; idx += kCW * 32) {
+            const int r = idx / D, d = idx % D;
             float M = -CUDART_INF_F;
 #pragma unroll
-            for (int w = 0; w < C::CW; ++w) M = fmaxf(M, merge_m[w * G + h]);
+            for (int w = 0; w < kCW; ++w) M = fmaxf(M, merge_m[w * kUnitRows + r]);
             float acc = 0.f, L = 0.f;
 #pragma unroll
-            for (int w = 0; w < C::CW; ++w) {
-                const float sw = fast_exp2(merge_m[w * G + h] - M);
-                acc = fmaf(sw, merge_o[(w * G + h) * D + d], acc);
-                L = fmaf(sw, merge_l[w * G + h], L);
+            for (int w = 0; w < kCW; ++w) {
+                const float mw = merge_m[w * kUnitRows + r];
+                const float sw = mw == -CUDART_INF_F ? 0.f : fast_exp2(mw - M);
+                acc = fmaf(sw, merge_o[(w * kUnitRows + r) * D + d], acc);
+                L = fmaf(sw, merge_l[w * kUnitRows + r], L);
             }
-            const float o = acc / L;
+            const float ov = acc / L;
             const float lse = (M + log2f(L)) * kLn2;
             if (n_parts == 1) {
-                p.out[io_off + h * D + d] = __float2bfloat16(o);
-                if (p.lse_out && d == 0) p.lse_out[lse_off + h] = lse;
+                p.out[q_base + (int64_t)(r / G) * p.q_ss + (r % G) * D + d] = __float2bfloat16(ov);
+                if (p.lse_out && d == 0) p.lse_out[lse_base + (int64_t)(r / G) * p.lse_ss + (r % G)] = lse;
             } else if (slot_ok) {
-                p.part_o[(slot * G + h) * D + d] = o;
-                if (d == 0) p.part_lse[slot * G + h] = lse;
+                p.part_o[(slot * kUnitRows + r) * D + d] = ov;
+                if (d == 0) p.part_lse[slot * kUnitRows + r] = lse;
             }
         }
         if (n_parts > 1 && slot_ok) {
             __threadfence();
-            consumer_bar<C::CW>();
+            consumer_bar();
             if (tid == 0) {
                 const int old = atomicAdd(p.counters + unit_index, 1);
                 const int last = (old == n_parts - 1);
                 if (last) p.counters[unit_index] = 0;  // ready for the next launch
                 flags[1] = last;
             }
-            consumer_bar<C::CW>();
+            consumer_bar();
             if (flags[1]) {
                 __threadfence();
                 const int64_t first_slot = unit_index + c_first;
-                for (int h = warp; h < G; h += C::CW)
-                    combine_warp(p.part_o + (first_slot * G + h) * D, (int64_t)G * D, p.part_lse + first_slot * G + h, G,
-                                 n_parts, D, p.out + io_off + h * D, p.lse_out ? p.lse_out + lse_off + h : nullptr);
+                for (int r = warp; r < n_rows; r += kCW)
+                    combine_warp(p.part_o + (first_slot * kUnitRows + r) * D, (int64_t)kUnitRows * D,
+                                 p.part_lse + first_slot * kUnitRows + r, kUnitRows, n_parts, D,
+                                 p.out + q_base + (int64_t)(r / G) * p.q_ss + (r % G) * D,
+                                 p.lse_out ? p.lse_out + lse_base + (int64_t)(r / G) * p.lse_ss + (r % G) : nullptr);
             }
         }
-        consumer_bar<C::CW>();  // merge area and flags are free again
+        consumer_bar();  // merge area and flags are free again
 
         j_base += t_end - t_begin;
         f_unit = u.flat_begin + t_end;
-        if (f_unit < f_end) next_unit(p, u);
+        if (f_unit < f_end) next_unit(p, u, n_blk);
     }
     if (flags[0] && tid == 0) atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
 }
@@ -736,7 +636,7 @@ static int launch_stream_t(const StreamParams &p, int grid, cudaStream_t stream)
         MATKV_CUDA(cudaFuncSetAttribute(k_attend_stream<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
         configured = true;
     }
-    k_attend_stream<D, G><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(p);
+    k_attend_stream<D, G><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p);
     MATKV_CUDA(cudaGetLastError());
     return MATKV_OK;
 }
@@ -745,9 +645,13 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     const matkv_config &c = ctx->cfg;
     WorkspaceView ws;
     workspace_bytes_for(c, &ws, ctx->workspace);
+    const int G = c.n_q_heads / c.n_kv_heads;
+    const int n_blk = ceil_div(a.S, kUnitRows / G);
     StreamParams p;
-    p.segs = t->d_segs;
     p.reqs = t->d_reqs;
+    p.tmaps = t->d_tmaps;
+    p.segs = t->d_segs;
+    p.n_seg_total = t->n_seg_total;
     p.tail_len = t->d_tail_len;
     p.tail_k = t->tail_k;
     p.tail_v = t->tail_v;
@@ -761,20 +665,17 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     p.counters = ws.counters; p.part_lse = ws.part_lse; p.part_o = ws.part_o;
     p.n_part_slots = ws.n_part_slots; p.n_counter_slots = ws.n_counter_slots;
     p.status = ctx->d_status;
-    const int64_t n_units = (int64_t)a.n_layers_launch * t->batch * a.S * c.n_kv_heads;
+    const int64_t n_units = (int64_t)a.n_layers_launch * t->batch * n_blk * c.n_kv_heads;
     if (n_units > ws.n_counter_slots)
         return fail(MATKV_E_CAPACITY, "launch of %lld units exceeds the workspace's %lld", (long long)n_units,
                     (long long)ws.n_counter_slots);
     // tiles in the launch as far as the host knows (the device recomputes it from its own tail length)
     int64_t W = 0;
-    for (int b = 0; b < t->batch; ++b) {
-        const int base = t->h_reqs[b].chunk_tiles + ceil_div(t->tail_len_host, kTile);
-        W += (int64_t)c.n_kv_heads * ((int64_t)a.S * base + new_tiles_sum(a.S));
-    }
+    for (int b = 0; b < t->batch; ++b)
+        W += (int64_t)c.n_kv_heads * n_blk * (t->h_reqs[b].chunk_tiles + ceil_div(t->tail_len_host, kTile) + 1);
     W *= a.n_layers_launch;
     int64_t grid = ctx->opt_decode_ctas > 0 ? ctx->opt_decode_ctas : ctx->n_sm;
     grid = std::max<int64_t>(1, std::min<int64_t>(grid, W));
-    const int G = c.n_q_heads / c.n_kv_heads;
 #define MATKV_CASE(DD, GG) \
     if (c.head_dim == DD && G == GG) return launch_stream_t<DD, GG>(p, (int)grid, stream);
     MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)

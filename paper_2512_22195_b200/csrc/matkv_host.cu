@@ -38,8 +38,32 @@ struct DeviceGuard {
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+int encode_rows_map(CUtensorMap *out, const void *base, int D, uint64_t rows) {
+    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+        if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p)
+            return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+        fn = (EncodeFn)p;
+    }
+    const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)D * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    const cuuint32_t estride[2] = {1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estride,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
+    return MATKV_OK;
+}
+
 size_t workspace_bytes_for(const matkv_config &c, WorkspaceView *v, void *base) {
-    const int64_t G = c.n_q_heads / c.n_kv_heads;
+    const int64_t G = kUnitRows;
     const int64_t units_decode = (int64_t)c.n_layers * c.max_batch * c.n_kv_heads;
     const int64_t units_prefill = (int64_t)c.max_batch * c.max_tail_tokens * c.n_kv_heads;
     const int64_t n_units = std::max(units_decode, units_prefill);
@@ -222,6 +246,10 @@ int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, co
     c.n_tokens = n_tokens;
     c.host_blob = host_blob;
     c.dev_blob = dev_blob;
+    if (dev_blob) {
+        int rc = encode_rows_map(&c.tmap, dev_blob, ctx->cfg.head_dim, (uint64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * n_tokens);
+        if (rc) return rc;
+    }
     ctx->chunks.emplace(chunk_id, c);
     return MATKV_OK;
 }
@@ -326,6 +354,13 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
             cudaEventDestroy(tk.done);
             return cuda_fail(e, "staging copy");
         }
+        {
+            int rc = encode_rows_map(&c.tmap, dst, ctx->cfg.head_dim, (uint64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * c.n_tokens);
+            if (rc) {
+                cudaEventDestroy(tk.done);
+                return rc;
+            }
+        }
         r->used[next_free] = 1;
         r->occupant[next_free] = id;
         c.staged = dst;
@@ -385,6 +420,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     t->tail_k = (__nv_bfloat16 *)tail_k;
     t->tail_v = (__nv_bfloat16 *)tail_v;
     std::vector<cudaEvent_t> waits;
+    std::vector<const CUtensorMap *> seg_maps;
     int64_t k = 0;
     for (int32_t r = 0; r < batch; ++r) {
         DevReq rq;
@@ -415,6 +451,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
             sg.len = c.n_tokens;
             sg.start = rq.n_chunk_tokens;
             t->h_segs.push_back(sg);
+            seg_maps.push_back(&c.tmap);
             rq.n_chunk_tokens += c.n_tokens;
             rq.chunk_tiles += (c.n_tokens + kTile - 1) / kTile;
             longest = std::max(longest, c.n_tokens);
@@ -429,7 +466,18 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     const size_t segs_bytes = align_up(sizeof(DevSeg) * std::max<size_t>(t->h_segs.size(), 1), 256);
     const size_t reqs_bytes = align_up(sizeof(DevReq) * (size_t)batch, 256);
     const size_t tl_bytes = align_up(sizeof(int32_t) * (size_t)batch, 256);
-    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes;
+    const size_t maps_bytes = sizeof(CUtensorMap) * (seg_maps.size() + 2);
+    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes + maps_bytes;
+    CUtensorMap tail_maps[2];
+    {
+        const uint64_t tail_rows = (uint64_t)batch * ctx->cfg.n_layers * ctx->cfg.n_kv_heads * ctx->cfg.max_tail_tokens;
+        int rc = encode_rows_map(&tail_maps[0], tail_k, ctx->cfg.head_dim, tail_rows);
+        if (!rc) rc = encode_rows_map(&tail_maps[1], tail_v, ctx->cfg.head_dim, tail_rows);
+        if (rc) {
+            delete t;
+            return rc;
+        }
+    }
     cudaError_t e = cudaMallocHost(&t->h_pinned, t->image_bytes);
     if (e == cudaSuccess) e = cudaMalloc(&t->d_image, t->image_bytes);
     if (e != cudaSuccess) {
@@ -443,6 +491,12 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     t->d_segs = (DevSeg *)t->d_image;
     t->d_reqs = (DevReq *)((char *)t->d_image + segs_bytes);
     t->d_tail_len = (int32_t *)((char *)t->d_image + segs_bytes + reqs_bytes);
+    t->d_tmaps = (CUtensorMap *)((char *)t->d_image + segs_bytes + reqs_bytes + tl_bytes);
+    {
+        CUtensorMap *hm = (CUtensorMap *)((char *)t->h_pinned + segs_bytes + reqs_bytes + tl_bytes);
+        for (size_t i = 0; i < seg_maps.size(); ++i) memcpy(hm + i, seg_maps[i], sizeof(CUtensorMap));
+        memcpy(hm + seg_maps.size(), tail_maps, sizeof(tail_maps));
+    }
     for (cudaEvent_t ev : waits) {
         e = cudaStreamWaitEvent(st, ev, 0);  // the stream waits for the copies; the host does not
         if (e != cudaSuccess) break;

@@ -1,5 +1,6 @@
 // Internal declarations shared by the host-side C ABI and the kernels' launchers.
 #pragma once
+#include <cuda.h>  // CUtensorMap (types only; the encoder is fetched through the runtime, libcuda is not linked)
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -44,6 +45,7 @@ struct Chunk {
     int32_t slot = -1;
     cudaEvent_t ready = nullptr;   // event of the staging call that (last) copied it; borrowed from the ticket
     uint64_t ticket = 0;
+    alignas(64) CUtensorMap tmap;  // 2-D view [rows][D] of the current device copy, 64 x kTile boxes, 128-byte swizzle
 };
 
 struct Region {
@@ -93,6 +95,7 @@ struct matkv_table {
     matkv::DevSeg *d_segs = nullptr;
     matkv::DevReq *d_reqs = nullptr;
     int32_t *d_tail_len = nullptr;
+    CUtensorMap *d_tmaps = nullptr;  // one per segment, then the K tail and the V tail
     __nv_bfloat16 *tail_k = nullptr, *tail_v = nullptr;
     std::vector<matkv::Region *> regions;  // staged regions this table reads
 };
@@ -107,11 +110,16 @@ int cuda_fail(cudaError_t e, const char *what);
         if (e__ != cudaSuccess) return ::matkv::cuda_fail(e__, #x); \
     } while (0)
 
+constexpr int kUnitRows = 8;  // query rows (suffix tokens x heads of one KV group) one streaming unit carries
+
+// 2-D tensor map over `rows` rows of D bf16 starting at `base` (box 64 x kTile, 128-byte swizzle, zero fill)
+int encode_rows_map(CUtensorMap *out, const void *base, int D, uint64_t rows);
+
 // Workspace layout: [counters: int32 x n_counter_slots][lse parts: fp32][o parts: fp32]
 struct WorkspaceView {
     int32_t *counters;
-    float *part_lse;   // [n_part_slots][G]
-    float *part_o;     // [n_part_slots][G][D]
+    float *part_lse;   // [n_part_slots][kUnitRows]
+    float *part_o;     // [n_part_slots][kUnitRows][D]
     int64_t n_counter_slots, n_part_slots;
 };
 size_t workspace_bytes_for(const matkv_config &c, WorkspaceView *view_from_base, void *base);
