@@ -166,6 +166,24 @@ int matkv_attend_decode(matkv_ctx *ctx, matkv_table *table, int32_t layer, const
 int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *table, const void *q, const void *k_new,
                                    const void *v_new, void *out, float *lse_out, void *stream);
 
+/* The decode step of one layer (same arguments, same result as matkv_attend_decode) for callers that
+ * must not allocate device memory and have none to lend as a workspace: for example a serving process
+ * that has handed all of HBM to its own KV pool, where a cudaMalloc would fail or stall every stream
+ * while the driver synchronises, or a plug-in running under a host that forbids allocation after
+ * start-up.  The paper has no counterpart; this is a packaging variant of a5 + a6.
+ *   - The split-KV partials and arrival counters live in an array built into the library
+ *     (2,114,560 bytes of device memory per GPU that loads it, held until the process exits) instead
+ *     of the workspace given to matkv_set_workspace, which this call neither needs nor touches.
+ *   - Limit: batch x n_kv_heads <= 256 and head_dim <= 128; larger calls return MATKV_E_CAPACITY.
+ *   - Nothing is allocated or freed: no cudaMalloc / cudaFree and no allocating library routine.  The
+ *     first call on a device looks up the array's device address (cudaGetSymbolAddress); make that
+ *     first call outside any stream capture.
+ *   - All calls share the one array and it keeps the previous call's contents; each call clears its
+ *     arrival counters on `stream` before the kernel.  Two calls that overlap on the GPU (different
+ *     streams, or different contexts on one device) race on it: serialise them.                      */
+int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *table, int32_t layer, const void *q, const void *k_new,
+                               const void *v_new, void *out, float *lse_out, void *stream);
+
 /* a6 alone: merges n_parts partial attentions per row.  o_parts [n_rows][n_parts][D] fp32
  * (each normalised within its part), lse_parts [n_rows][n_parts] fp32 natural log (-inf =
  * empty part), out [n_rows][D] bf16, lse_out NULL or [n_rows] fp32; all device.              */

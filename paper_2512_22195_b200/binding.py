@@ -24,7 +24,7 @@ EXPORTS = [
     "matkv_stage_chunks_async", "matkv_stage_query", "matkv_stage_wait", "matkv_build_chunk_table",
     "matkv_table_free", "matkv_table_advance", "matkv_table_set_tail_len", "matkv_attend_prefill",
     "matkv_attend_decode", "matkv_attend_decode_all_layers", "matkv_lse_combine", "matkv_gather_debug",
-    "matkv_probe_read",
+    "matkv_probe_read", "matkv_attend_decode_static",
 ]
 
 
@@ -76,6 +76,7 @@ def lib() -> C.CDLL:
             "matkv_lse_combine": (C.c_int, [vp, i32, i32, i32, vp, vp, vp, vp, vp]),
             "matkv_gather_debug": (C.c_int, [vp, vp, i32, i32, vp, vp, i64, C.POINTER(i64), vp]),
             "matkv_probe_read": (C.c_int, [vp, vp, C.c_size_t, vp]),
+            "matkv_attend_decode_static": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -207,3 +208,11 @@ def matkv_gather_debug(ctx: int, table: int, layer: int, req: int, k_out: int, v
 
 def matkv_probe_read(ctx: int, dev_ptr: int, nbytes: int, stream: int = 0) -> None:
     _check(lib().matkv_probe_read(ctx, dev_ptr, nbytes, stream or None))
+
+
+def matkv_attend_decode_static(ctx: int, table: int, layer: int, q: int, k_new: int, v_new: int, out: int,
+                               lse_out: Optional[int] = None, stream: int = 0) -> None:
+    """matkv_attend_decode for callers that may not allocate or lend a workspace: the split-KV scratch is
+    an array built into the library (batch x n_kv_heads <= 256).  First call per device: outside any
+    stream capture.  Calls must not overlap on the GPU (they share the array)."""
+    _check(lib().matkv_attend_decode_static(ctx, table, layer, q, k_new, v_new, out, lse_out or None, stream or None))

@@ -684,6 +684,108 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     return fail(MATKV_E_INVALID_ARG, "unsupported head_dim %d / group %d", c.head_dim, G);
 }
 
+// ---- decode with built-in scratch (no allocation anywhere on this path) ----------------------------
+// The split-KV partials and arrival counters of this one entry point live in a file-scope device
+// array instead of the caller's workspace.  Every GPU that loads the library carries the array until
+// the process exits, so it is kept small: it bounds the call at kStaticUnits (request, KV head) pairs
+// and kStaticCtas CTAs.
+constexpr int kStaticUnits = 256;
+constexpr int kStaticCtas = 256;
+constexpr int kStaticParts = kStaticUnits + kStaticCtas;
+constexpr size_t kStaticCounterBytes = sizeof(int32_t) * kStaticUnits;                    //      1,024
+constexpr size_t kStaticLseBytes = sizeof(float) * kStaticParts * kUnitRows;              //     16,384
+constexpr size_t kStaticOBytes = sizeof(float) * (size_t)kStaticParts * kUnitRows * 128;  //  2,097,152
+constexpr size_t kStaticBytes = kStaticCounterBytes + kStaticLseBytes + kStaticOBytes;    //  2,114,560 in all
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+// Device address of g_static_scratch per device ordinal.  In host code the array's name is only a
+// stand-in for the symbol, never an address a kernel may use: the address comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+static void *g_static_scratch_addr[64] = {};
+
+}  // namespace matkv
+
+extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_t layer, const void *q, const void *k_new,
+                                          const void *v_new, void *out, float *lse_out, void *stream) {
+    using namespace matkv;
+    if (!ctx || !t || !q || !k_new || !v_new || !out) return fail(MATKV_E_INVALID_ARG, "matkv_attend_decode_static: null argument");
+    if (t->ctx != ctx) return fail(MATKV_E_INVALID_ARG, "matkv_attend_decode_static: table belongs to another context");
+    const matkv_config &c = ctx->cfg;
+    if (layer < 0 || layer >= c.n_layers) return fail(MATKV_E_INVALID_ARG, "matkv_attend_decode_static: layer %d", layer);
+    if (((uintptr_t)q | (uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)out) % 16)
+        return fail(MATKV_E_ALIGNMENT, "matkv_attend_decode_static: q, k_new, v_new and out must be 16-byte aligned");
+    if (c.rope_theta != 0.f) return fail(MATKV_E_INVALID_ARG, "matkv_attend_decode_static: rotary mode is not available");
+    if (t->tail_len_host + 1 > c.max_tail_tokens)
+        return fail(MATKV_E_CAPACITY, "matkv_attend_decode_static: tail holds %d tokens, one more exceeds max_tail_tokens %d",
+                    t->tail_len_host, c.max_tail_tokens);
+    const int64_t n_units = (int64_t)t->batch * c.n_kv_heads;
+    if (n_units > kStaticUnits)
+        return fail(MATKV_E_CAPACITY,
+                    "matkv_attend_decode_static: batch %d x %d KV heads = %lld units, the built-in scratch holds %d; "
+                    "use matkv_attend_decode with a caller workspace",
+                    t->batch, c.n_kv_heads, (long long)n_units, kStaticUnits);
+    if (ctx->device < 0 || ctx->device >= 64) return fail(MATKV_E_CAPACITY, "matkv_attend_decode_static: device ordinal %d", ctx->device);
+    int prev = -1;
+    MATKV_CUDA(cudaGetDevice(&prev));
+    if (prev != ctx->device) MATKV_CUDA(cudaSetDevice(ctx->device));
+    int rc = MATKV_OK;
+    do {
+        void *&base = g_static_scratch_addr[ctx->device];
+        if (!base) {  // first call on this device: resolve the symbol (not inside a stream capture)
+            void *ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+            if (e != cudaSuccess || !ptr) {
+                rc = cuda_fail(e, "cudaGetSymbolAddress(g_static_scratch)");
+                break;
+            }
+            base = ptr;
+        }
+        cudaStream_t st = (cudaStream_t)stream;
+        // the array keeps the last call's contents: the arrival counters must start at zero
+        cudaError_t e = cudaMemsetAsync(base, 0, kStaticCounterBytes, st);
+        if (e != cudaSuccess) {
+            rc = cuda_fail(e, "cudaMemsetAsync(counters)");
+            break;
+        }
+        StreamParams p;
+        p.reqs = t->d_reqs;
+        p.tmaps = t->d_tmaps;
+        p.segs = t->d_segs;
+        p.n_seg_total = t->n_seg_total;
+        p.tail_len = t->d_tail_len;
+        p.tail_k = t->tail_k;
+        p.tail_v = t->tail_v;
+        p.q = (const __nv_bfloat16 *)q; p.k_new = (const __nv_bfloat16 *)k_new; p.v_new = (const __nv_bfloat16 *)v_new;
+        p.out = (__nv_bfloat16 *)out; p.lse_out = lse_out;
+        p.q_sl = 0; p.q_sb = (int64_t)c.n_q_heads * c.head_dim; p.q_ss = 0;
+        p.kn_sl = 0; p.kn_sb = (int64_t)c.n_kv_heads * c.head_dim; p.kn_ss = 0;
+        p.lse_sl = 0; p.lse_sb = c.n_q_heads; p.lse_ss = 0;
+        p.layer0 = layer; p.n_layers_launch = 1; p.n_layers_total = c.n_layers;
+        p.B = t->batch; p.S = 1; p.Hkv = c.n_kv_heads; p.max_tail = c.max_tail_tokens;
+        p.scale_log2 = ctx->scale * kLog2e;
+        p.counters = (int32_t *)base;
+        p.part_lse = (float *)((char *)base + kStaticCounterBytes);
+        p.part_o = (float *)((char *)base + kStaticCounterBytes + kStaticLseBytes);
+        p.n_part_slots = kStaticParts; p.n_counter_slots = kStaticUnits;
+        p.status = ctx->d_status;
+        int64_t W = 0;
+        for (int b = 0; b < t->batch; ++b)
+            W += (int64_t)c.n_kv_heads * (t->h_reqs[b].chunk_tiles + ceil_div(t->tail_len_host, kTile) + 1);
+        int64_t grid = std::min<int64_t>(std::min<int64_t>(ctx->n_sm, kStaticCtas), W);
+        if (grid < 1) grid = 1;
+        const int G = c.n_q_heads / c.n_kv_heads;
+        rc = fail(MATKV_E_INVALID_ARG, "unsupported head_dim %d / group %d", c.head_dim, G);
+#define MATKV_CASE(DD, GG) \
+        if (c.head_dim == DD && G == GG) rc = launch_stream_t<DD, GG>(p, (int)grid, st);
+        MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)
+        MATKV_CASE(64, 1) MATKV_CASE(64, 2) MATKV_CASE(64, 4) MATKV_CASE(64, 8)
+#undef MATKV_CASE
+    } while (0);
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return rc;
+}
+
+namespace matkv {
+
 int launch_lse_combine(matkv_ctx *, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts, const float *lse_parts,
                        void *out, float *lse_out, cudaStream_t stream) {
     const int warps = 4;
