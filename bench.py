@@ -32,7 +32,7 @@ import matkv_inputs as mi  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per decode launch from the committed ncu capture (profiles/), by workload and launch mode.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {("cfg2", "all_layers"): 697.2e6 + 4.4e6}  # profiles/k_attend_stream_decode_cfg2_all_layers.md
 
 
 def log(*a):
@@ -204,11 +204,11 @@ def main():
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, args.decode_ctas)
     # every rank works on its own replica of the batch (independent requests: no data-path collective)
     chunks = {}
-    for c in needed:
-        t_ = torch.empty((L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
-        gen.fill_bf16(t_, w.seed, mi.STREAM_CHUNK + c)
-        chunks[c] = t_
-        sess.register_device_chunk(c, t_)
+    pool = torch.empty((len(needed), L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
+    for i, c in enumerate(needed):
+        gen.fill_bf16(pool[i], w.seed, mi.STREAM_CHUNK + c)
+        chunks[c] = pool[i]
+        sess.register_device_chunk(c, pool[i])
     q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device=dev)
     k_pf = torch.empty((L, B, S, Hkv, D), dtype=torch.bfloat16, device=dev)
     v_pf = torch.empty_like(k_pf)
@@ -311,18 +311,15 @@ def main():
     # read-only streaming probe over the same chunk memory (plain 16-byte loads), same run
     probe_gbs = None
     with torch.cuda.stream(stream):
-        big = max(chunks.values(), key=lambda x: x.numel())
         pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         for _ in range(2):
-            for c in needed:
-                mk.matkv_probe_read(ctx, chunks[c].data_ptr(), chunks[c].numel() * 2, sp)
+            mk.matkv_probe_read(ctx, pool.data_ptr(), pool.numel() * 2, sp)
         pe0.record(stream)
-        for _ in range(3):
-            for c in needed:
-                mk.matkv_probe_read(ctx, chunks[c].data_ptr(), chunks[c].numel() * 2, sp)
+        for _ in range(5):
+            mk.matkv_probe_read(ctx, pool.data_ptr(), pool.numel() * 2, sp)
         pe1.record(stream)
         torch.cuda.synchronize()
-        probe_gbs = 3 * sum(chunks[c].numel() * 2 for c in needed) / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
+        probe_gbs = 5 * pool.numel() * 2 / (pe0.elapsed_time(pe1) * 1e-3) / 1e9
 
     # algorithmic KV bytes of the decode loop of one step: every visible K and V element once
     n_req = [sum(chunks[c].shape[3] for c in row) for row in ids]
