@@ -636,6 +636,10 @@ int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t 
     a.q_ss = (int64_t)c.n_q_heads * c.head_dim; a.q_sb = a.q_ss * S; a.q_sl = 0;
     a.kn_ss = (int64_t)c.n_kv_heads * c.head_dim; a.kn_sb = a.kn_ss * S; a.kn_sl = 0;
     a.lse_ss = c.n_q_heads; a.lse_sb = a.lse_ss * S; a.lse_sl = 0;
+    // long suffixes go to the tcgen05 tile kernel, short ones stay on the streaming kernel
+    const int G = c.n_q_heads / c.n_kv_heads;
+    const bool tensor_core = ctx->opt_prefill_impl == 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
+    if (tensor_core) return launch_prefill_tc(ctx, t, a, (cudaStream_t)stream);
     return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
 }
 

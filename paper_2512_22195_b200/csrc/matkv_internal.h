@@ -137,6 +137,7 @@ struct AttendArgs {
     int64_t lse_sl, lse_sb, lse_ss;
 };
 int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
+int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
 int launch_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts,
                        const float *lse_parts, void *out, float *lse_out, cudaStream_t stream);
 int launch_gather(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out,

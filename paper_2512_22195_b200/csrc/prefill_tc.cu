@@ -1,0 +1,533 @@
+// K3: query sub-prefill over the chunk table on the 5th-generation tensor cores (tcgen05 + TMEM).
+//
+// One CTA = (request, KV head, block of 128 query rows, KV split).  A query row is (suffix token,
+// head of the KV group), row = token * G + head, so the G heads that share a KV head and up to 128/G
+// suffix tokens share every K/V tile that is fetched.  Per 64-token KV tile:
+//     S  = Q K^T      tcgen05.mma  M=128, N=64,  K=D   (both operands K-major, 128-byte swizzle)  -> TMEM
+//     P  = online softmax of S (one thread per row: tcgen05.ld, fp32, exp2-based) -> bf16 in smem
+//     Ot = P V        tcgen05.mma  M=128, N=D,   K=64  (V is MN-major straight from its [token][d] tile) -> TMEM
+//     O  = O * alpha + Ot   in registers of the row's thread (tcgen05.ld), so TMEM is never read-modified
+// Warp roles: warp 0 producer (TMA tensor copies of chunk / tail tiles through the table's descriptors;
+// the call's new tokens are copied by hand into the same swizzled layout and appended to the tail),
+// warp 1 issues the MMAs and owns the TMEM allocation, warps 2-5 are the 128 softmax threads.
+// S and Ot are double-buffered in TMEM (2 x 64 + 2 x D columns) so that the tensor core works on tile
+// j+1 while the softmax threads work on tile j.  Every wait is bounded and reports through the status
+// word; TMEM is always released.
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <math_constants.h>
+
+#include <algorithm>
+
+#include "matkv_internal.h"
+
+namespace matkv {
+
+namespace k3 {
+
+constexpr int kRowsPerCta = 128;
+constexpr int kThreads = 192;  // producer warp, MMA warp, four softmax warps
+constexpr int kStages = 4;
+constexpr long long kWaitCycles = 2000000000LL;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct Params {
+    const DevReq *reqs;
+    const DevSeg *segs;
+    const CUtensorMap *tmaps;
+    int32_t n_seg_total;
+    const int32_t *tail_len;
+    __nv_bfloat16 *tail_k, *tail_v;
+    const __nv_bfloat16 *q, *k_new, *v_new;
+    __nv_bfloat16 *out;
+    float *lse_out;
+    int64_t q_sb, q_ss, kn_sb, kn_ss;  // element strides: request, suffix token
+    int32_t layer, n_layers_total, B, S, Hq, Hkv, max_tail, n_rb, n_split;
+    float scale_log2;
+    float *part_o, *part_lse;  // [row][split][D], [row][split]; row = (b*S + i)*Hq + head
+    int32_t *status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; false once the CTA's abort flag is up or after about a second (which raises it).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor of a 128-byte-swizzled tile whose rows are 128 bytes (64 bf16).
+//   K-major operand  (rows = M or N index, the 128 bytes run along K): SBO = 1024 (next group of 8 rows),
+//                     LBO unused; a 16-element K slice is a 32-byte step of the start address.
+//   MN-major operand (rows = K index, the 128 bytes run along M or N): SBO = 1024 (next 8 K rows),
+//                     LBO = distance to the next 64-wide block along N.
+// bits: [0,14) address >> 4, [16,30) LBO >> 4, [32,46) SBO >> 4, [46,48) version 1, [61,64) layout 2 = SWIZZLE_128B.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 x bf16, A K-major, B K- or MN-major, M x N.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
+           ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__host__ __device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+// tile t of a unit: kind 0 = chunk, 1 = tail, 2 = new tokens
+struct Tile {
+    int kind, seg, r0, rows, seg_len;
+};
+
+template <int D>
+struct Cfg {
+    static constexpr int NBOX = D / 64;
+    static constexpr int BOX_BYTES = kTile * 128;        // 64 rows x 128 bytes
+    static constexpr int KV_BYTES = NBOX * BOX_BYTES;    // K (or V) of one tile
+    static constexpr int STAGE_BYTES = 2 * KV_BYTES;
+    static constexpr int Q_BYTES = NBOX * kRowsPerCta * 128;
+    static constexpr int P_BYTES = kRowsPerCta * 128;    // 128 rows x 64 tokens bf16
+    static constexpr int SMEM_BYTES = 1024 + Q_BYTES + 2 * P_BYTES + kStages * STAGE_BYTES + 512;
+    static constexpr int COL_S = 0, COL_O = 128;         // TMEM columns: S[2] at 0, 64; Ot[2] at 128, 128 + D
+    static constexpr int TMEM_COLS = 512;
+};
+
+template <int D, int G>
+__global__ void __launch_bounds__(kThreads, 1) k_prefill_tc(const Params p) {
+    using C = Cfg<D>;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *q_s = smem;                                   // NBOX boxes [128 rows][128 B]
+    unsigned char *p_s = q_s + C::Q_BYTES;                       // 2 x [128 rows][128 B]
+    unsigned char *kv_s = p_s + 2 * C::P_BYTES;                  // kStages x (K boxes, V boxes)
+    uint64_t *bars = (uint64_t *)(kv_s + kStages * C::STAGE_BYTES);
+    // barriers: full_kv[4], empty_kv[4], s_full[2], p_ready[2], o_full[2], o_free[2], q_ready
+    uint32_t *tmem_slot = (uint32_t *)(bars + 20);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 2);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // which unit
+    int c = blockIdx.x;
+    const int sp = c % p.n_split; c /= p.n_split;
+    const int rb = c % p.n_rb; c /= p.n_rb;
+    const int g = c % p.Hkv;
+    const int b = c / p.Hkv;
+    const DevReq rq = p.reqs[b];
+    int t0 = p.tail_len[b];
+    if (t0 < 0 || t0 + p.S > p.max_tail) {
+        if (tid == 0) atomicCAS(p.status, 0, MATKV_E_CAPACITY);
+        t0 = max(0, min(t0, p.max_tail - p.S));
+    }
+    const int tail_tiles = cdiv(t0, kTile), new_tiles = cdiv(p.S, kTile);
+    const int T = rq.chunk_tiles + tail_tiles + new_tiles;
+    const int t_begin = (int)((int64_t)sp * T / p.n_split), t_end = (int)((int64_t)(sp + 1) * T / p.n_split);
+    const int n_tiles = t_end - t_begin;
+    const int R = p.S * G;                       // query rows of the (request, KV head)
+    const int row0 = rb * kRowsPerCta;
+
+    const uint32_t bar0 = smem_u32(bars);
+    const uint32_t full_kv = bar0, empty_kv = bar0 + 4 * 8, s_full = bar0 + 8 * 8, p_ready = bar0 + 10 * 8,
+                   o_full = bar0 + 12 * 8, o_free = bar0 + 14 * 8, q_ready = bar0 + 16 * 8;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_kv + s * 8, 1);
+            mbar_init(empty_kv + s * 8, 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(s_full + s * 8, 1);
+            mbar_init(p_ready + s * 8, 128);
+            mbar_init(o_full + s * 8, 1);
+            mbar_init(o_free + s * 8, 128);
+        }
+        mbar_init(q_ready, 128);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    if (warp == 1) {  // TMEM: all 512 columns (one CTA per SM)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"((uint32_t)C::TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    // tile lookup shared by the producer and the softmax threads
+    auto tile_at = [&](int t, int &seg, int &tiles_before, int &seg_tiles, int &seg_len) {
+        Tile ti;
+        if (t < rq.chunk_tiles) {
+            while (seg < 0 || t >= tiles_before + seg_tiles) {
+                tiles_before += seg_tiles;
+                ++seg;
+                seg_len = p.segs[rq.seg_begin + seg].len;
+                seg_tiles = cdiv(seg_len, kTile);
+            }
+            ti.kind = 0; ti.seg = seg; ti.seg_len = seg_len;
+            ti.r0 = (t - tiles_before) * kTile;
+            ti.rows = min(kTile, seg_len - ti.r0);
+        } else if (t < rq.chunk_tiles + tail_tiles) {
+            ti.kind = 1; ti.seg = 0; ti.seg_len = 0;
+            ti.r0 = (t - rq.chunk_tiles) * kTile;
+            ti.rows = min(kTile, t0 - ti.r0);
+        } else {
+            ti.kind = 2; ti.seg = 0; ti.seg_len = 0;
+            ti.r0 = (t - rq.chunk_tiles - tail_tiles) * kTile;
+            ti.rows = min(kTile, p.S - ti.r0);
+        }
+        return ti;
+    };
+
+    if (warp == 0) {
+        // ===================== producer =====================
+        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int st = j % kStages, use = j / kStages;
+            if (use > 0) ok = mbar_wait(empty_kv + st * 8, (use - 1) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len);
+            const uint32_t dst = smem_u32(kv_s + st * C::STAGE_BYTES), bar = full_kv + st * 8;
+            if (ti.kind < 2) {
+                if (lane == 0) {
+                    const CUtensorMap *mk, *mv;
+                    int32_t yk, yv;
+                    if (ti.kind == 0) {
+                        mk = mv = p.tmaps + rq.seg_begin + ti.seg;
+                        yk = ((p.layer * 2) * p.Hkv + g) * ti.seg_len + ti.r0;
+                        yv = ((p.layer * 2 + 1) * p.Hkv + g) * ti.seg_len + ti.r0;
+                    } else {
+                        mk = p.tmaps + p.n_seg_total;
+                        mv = mk + 1;
+                        yk = yv = ((b * p.n_layers_total + p.layer) * p.Hkv + g) * p.max_tail + ti.r0;
+                    }
+                    mbar_expect_tx(bar, C::STAGE_BYTES);
+#pragma unroll
+                    for (int bx = 0; bx < C::NBOX; ++bx) {
+                        tma_load_2d(dst + bx * C::BOX_BYTES, mk, bx * 64, yk, bar);
+                        tma_load_2d(dst + C::KV_BYTES + bx * C::BOX_BYTES, mv, bx * 64, yv, bar);
+                    }
+                }
+            } else {
+                // the call's new tokens: copy rows by hand into the swizzled layout (zero rows past S)
+                constexpr int CPR = D / 8;  // 16-byte chunks per row
+                unsigned char *kd = kv_s + st * C::STAGE_BYTES, *vd = kd + C::KV_BYTES;
+                for (int idx = lane; idx < kTile * CPR; idx += 32) {
+                    const int row = idx / CPR, ch = idx % CPR;
+                    const int tok = ti.r0 + row;
+                    uint4 kvv = make_uint4(0, 0, 0, 0), vvv = make_uint4(0, 0, 0, 0);
+                    if (tok < p.S) {
+                        const int64_t off = (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
+                        kvv = *(const uint4 *)(p.k_new + off);
+                        vvv = *(const uint4 *)(p.v_new + off);
+                    }
+                    const int o = (ch / 8) * C::BOX_BYTES + row * 128 + (((ch % 8) ^ (row & 7)) << 4);
+                    *(uint4 *)(kd + o) = kvv;
+                    *(uint4 *)(vd + o) = vvv;
+                }
+                fence_async_smem();  // generic-proxy writes -> visible to the tensor core's async proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar);
+            }
+        }
+        // append the new tokens to the tail for later calls (one CTA per (request, KV head))
+        if (rb == 0 && sp == p.n_split - 1) {
+            constexpr int CPR = D / 8;
+            for (int idx = lane; idx < p.S * CPR; idx += 32) {
+                const int tok = idx / CPR, ch = idx % CPR;
+                if (t0 + tok >= p.max_tail) continue;
+                const int64_t src = (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
+                const int64_t dst = ((((int64_t)b * p.n_layers_total + p.layer) * p.Hkv + g) * p.max_tail + t0 + tok) * D + ch * 8;
+                *(uint4 *)(p.tail_k + dst) = *(const uint4 *)(p.k_new + src);
+                *(uint4 *)(p.tail_v + dst) = *(const uint4 *)(p.v_new + src);
+            }
+        }
+    } else if (warp == 1) {
+        // ===================== MMA issuer (one thread) =====================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = instr_desc(kRowsPerCta, kTile, false);
+            constexpr uint32_t idesc_pv = instr_desc(kRowsPerCta, D, true);
+            const uint32_t q_u32 = smem_u32(q_s), p_u32 = smem_u32(p_s), kv_u32 = smem_u32(kv_s);
+            bool ok = mbar_wait(q_ready, 0, abort_flag);
+            auto do_pv = [&](int t) {
+                const int bf = t & 1, use = t >> 1, st = t % kStages;
+                if (!mbar_wait(p_ready + bf * 8, use & 1, abort_flag)) return false;
+                if (use > 0 && !mbar_wait(o_free + bf * 8, (use - 1) & 1, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t v_u32 = kv_u32 + st * C::STAGE_BYTES + C::KV_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA
+                    umma(tmem + C::COL_O + bf * D, smem_desc(p_u32 + bf * C::P_BYTES + ks * 32, 0, 1024),
+                         smem_desc(v_u32 + ks * 2048, C::BOX_BYTES, 1024), idesc_pv, ks > 0);
+                umma_commit(o_full + bf * 8);
+                umma_commit(empty_kv + st * 8);  // K and V of the tile are free once these MMAs have run
+                return true;
+            };
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int st = j % kStages;
+                ok = mbar_wait(full_kv + st * 8, (j / kStages) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t k_u32 = kv_u32 + st * C::STAGE_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
+                    umma(tmem + C::COL_S + (j & 1) * kTile,
+                         smem_desc(q_u32 + (ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32, 0, 1024),
+                         smem_desc(k_u32 + (ks / 4) * C::BOX_BYTES + (ks % 4) * 32, 0, 1024), idesc_qk, ks > 0);
+                umma_commit(s_full + (j & 1) * 8);
+                if (j >= 1) ok = do_pv(j - 1);
+            }
+            if (ok && n_tiles > 0) do_pv(n_tiles - 1);
+        }
+    } else {
+        // ===================== softmax threads: one query row each =====================
+        const int r = (warp & 3) * 32 + lane;        // TMEM lane = row inside the CTA's block
+        const int grow = row0 + r;                   // row inside the (request, KV head)
+        const bool real = grow < R;
+        const int tok = grow / G, hd = grow % G;     // suffix token and head of the group
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        // Q row -> swizzled smem (zeros for rows past R)
+        {
+            const __nv_bfloat16 *qrow = p.q + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D;
+#pragma unroll
+            for (int ch = 0; ch < D / 8; ++ch) {
+                const uint4 v = real ? *(const uint4 *)(qrow + ch * 8) : make_uint4(0, 0, 0, 0);
+                *(uint4 *)(q_s + (ch / 8) * (kRowsPerCta * 128) + r * 128 + (((ch % 8) ^ (r & 7)) << 4)) = v;
+            }
+            fence_async_smem();
+            mbar_arrive(q_ready);
+        }
+        float o[D];
+#pragma unroll
+        for (int d = 0; d < D; ++d) o[d] = 0.f;
+        float m_run = -CUDART_INF_F, l_run = 0.f, alpha_prev = 1.f;
+        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
+        bool ok = true;
+        auto take_o = [&](int t) {  // O = O * alpha(t) + Ot(t)
+            const int bf = t & 1;
+            if (!mbar_wait(o_full + bf * 8, (t >> 1) & 1, abort_flag)) return false;
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                float v[32];
+                tmem_ld32(lane_base + C::COL_O + bf * D + c0, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) o[c0 + i] = fmaf(o[c0 + i], alpha_prev, v[i]);
+            }
+            tc_fence_before();
+            mbar_arrive(o_free + bf * 8);
+            return true;
+        };
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len);
+            const int bf = j & 1;
+            ok = mbar_wait(s_full + bf * 8, (j >> 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            float s[kTile];
+            {
+                float v[32];
+                tmem_ld32(lane_base + C::COL_S + bf * kTile, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) s[i] = v[i];
+                tmem_ld32(lane_base + C::COL_S + bf * kTile + 32, v);
+#pragma unroll
+                for (int i = 0; i < 32; ++i) s[32 + i] = v[i];
+            }
+            // visible columns: all valid rows of a chunk / tail tile; causal inside the new tokens
+            int n_vis = ti.rows;
+            if (ti.kind == 2) n_vis = min(ti.rows, tok - ti.r0 + 1);
+            if (!real) n_vis = min(n_vis, 1);
+            float tmax = -CUDART_INF_F;
+#pragma unroll
+            for (int i = 0; i < kTile; ++i) {
+                s[i] = i < n_vis ? s[i] * p.scale_log2 : -CUDART_INF_F;
+                tmax = fmaxf(tmax, s[i]);
+            }
+            const float m_new = fmaxf(m_run, tmax);
+            const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);
+            const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
+            float psum = 0.f;
+            unsigned char *prow = p_s + bf * C::P_BYTES + r * 128;
+#pragma unroll
+            for (int ch = 0; ch < kTile / 8; ++ch) {
+                float e[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    e[i] = fast_exp2(s[ch * 8 + i] - m_use);
+                    psum += e[i];
+                }
+                *(uint4 *)(prow + ((ch ^ (r & 7)) << 4)) =
+                    make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7]));
+            }
+            l_run = l_run * alpha + psum;
+            m_run = m_new;
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(p_ready + bf * 8);
+            if (j >= 1) ok = take_o(j - 1);
+            alpha_prev = alpha;
+        }
+        if (ok && n_tiles > 0) ok = take_o(n_tiles - 1);
+        // epilogue
+        if (ok && real) {
+            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+            const float lse = l_run > 0.f ? (m_run + log2f(l_run)) * kLn2 : -CUDART_INF_F;
+            const int64_t orow = ((int64_t)b * p.S + tok) * p.Hq + g * G + hd;
+            if (p.n_split == 1) {
+                __nv_bfloat16 *dst = p.out + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D;
+#pragma unroll
+                for (int ch = 0; ch < D / 8; ++ch)
+                    *(uint4 *)(dst + ch * 8) =
+                        make_uint4(pack_bf16(o[ch * 8] * inv, o[ch * 8 + 1] * inv), pack_bf16(o[ch * 8 + 2] * inv, o[ch * 8 + 3] * inv),
+                                   pack_bf16(o[ch * 8 + 4] * inv, o[ch * 8 + 5] * inv), pack_bf16(o[ch * 8 + 6] * inv, o[ch * 8 + 7] * inv));
+                if (p.lse_out) p.lse_out[orow] = lse;
+            } else {
+                float *dst = p.part_o + (orow * p.n_split + sp) * D;
+#pragma unroll
+                for (int ch = 0; ch < D / 4; ++ch)
+                    *(float4 *)(dst + ch * 4) = make_float4(o[ch * 4] * inv, o[ch * 4 + 1] * inv, o[ch * 4 + 2] * inv, o[ch * 4 + 3] * inv);
+                p.part_lse[orow * p.n_split + sp] = lse;
+            }
+        }
+    }
+    // ---- teardown: every thread gets here, TMEM is always given back ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)C::TMEM_COLS) : "memory");
+    }
+    if (tid == 0 && *abort_flag) atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
+}
+
+}  // namespace k3
+
+template <int D, int G>
+static int launch_k3(const k3::Params &p, int grid, cudaStream_t stream) {
+    using C = k3::Cfg<D>;
+    static bool configured = false;
+    if (!configured) {
+        MATKV_CUDA(cudaFuncSetAttribute(k3::k_prefill_tc<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        configured = true;
+    }
+    k3::k_prefill_tc<D, G><<<grid, k3::kThreads, C::SMEM_BYTES, stream>>>(p);
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
+int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream) {
+    const matkv_config &c = ctx->cfg;
+    const int G = c.n_q_heads / c.n_kv_heads, D = c.head_dim;
+    k3::Params p;
+    p.reqs = t->d_reqs; p.segs = t->d_segs; p.tmaps = t->d_tmaps; p.n_seg_total = t->n_seg_total;
+    p.tail_len = t->d_tail_len; p.tail_k = t->tail_k; p.tail_v = t->tail_v;
+    p.q = a.q; p.k_new = a.k_new; p.v_new = a.v_new; p.out = a.out; p.lse_out = a.lse_out;
+    p.q_sb = a.q_sb; p.q_ss = a.q_ss; p.kn_sb = a.kn_sb; p.kn_ss = a.kn_ss;
+    p.layer = a.layer0; p.n_layers_total = c.n_layers; p.B = t->batch; p.S = a.S; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads;
+    p.max_tail = c.max_tail_tokens;
+    p.n_rb = (a.S * G + k3::kRowsPerCta - 1) / k3::kRowsPerCta;
+    p.scale_log2 = ctx->scale * k3::kLog2e;
+    p.status = ctx->d_status;
+    // KV splits: fill the SMs, never more splits than the shortest request has tiles, and only as many
+    // as the workspace can hold partials for
+    const int64_t combos = (int64_t)t->batch * c.n_kv_heads * p.n_rb;
+    int min_tiles = 1 << 30;
+    for (int b = 0; b < t->batch; ++b)
+        min_tiles = std::min(min_tiles, t->h_reqs[b].chunk_tiles + k3::cdiv(t->tail_len_host, kTile) + k3::cdiv(a.S, kTile));
+    int64_t ns = ctx->opt_prefill_ctas > 0 ? ctx->opt_prefill_ctas : std::max<int64_t>(1, ctx->n_sm / combos);
+    ns = std::min<int64_t>(ns, std::max(1, min_tiles));
+    // the partials live in the workspace's partial regions (its head holds the streaming kernel's counters)
+    WorkspaceView ws;
+    workspace_bytes_for(c, &ws, ctx->workspace);
+    const int64_t rows = (int64_t)t->batch * a.S * c.n_q_heads;
+    ns = std::min<int64_t>(ns, std::max<int64_t>(1, ws.n_part_slots * kUnitRows / rows));
+    ns = std::min<int64_t>(ns, 64);
+    p.n_split = (int)ns;
+    p.part_lse = ws.part_lse;
+    p.part_o = ws.part_o;
+    const int64_t grid = combos * p.n_split;
+    int rc = fail(MATKV_E_INVALID_ARG, "tensor-core prefill: unsupported head_dim %d / group %d", D, G);
+#define MATKV_CASE(DD, GG) \
+    if (D == DD && G == GG) rc = launch_k3<DD, GG>(p, (int)grid, stream);
+    MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)
+    MATKV_CASE(64, 1) MATKV_CASE(64, 2) MATKV_CASE(64, 4) MATKV_CASE(64, 8)
+#undef MATKV_CASE
+    if (rc) return rc;
+    if (p.n_split > 1)
+        return launch_lse_combine(ctx, (int32_t)rows, p.n_split, D, p.part_o, p.part_lse, a.out, a.lse_out, stream);
+    return MATKV_OK;
+}
+
+}  // namespace matkv

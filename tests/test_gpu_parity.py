@@ -28,7 +28,7 @@ def _bits(t):
 
 
 def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=False, q_shift=0, cap=None,
-                 prefill_impl=0):
+                 prefill_impl=0, prefill_ctas=0):
     """Prefill S tokens then T decode steps for a batch; compare every output with the oracle."""
     import paper_2512_22195_b200 as mk
     B = len(lens_per_req)
@@ -38,6 +38,8 @@ def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=Fal
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, ctas)
     if prefill_impl:
         mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_IMPL, prefill_impl)
+    if prefill_ctas:
+        mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_CTAS, prefill_ctas)
     sh = oracle.Shape(L, Hq, Hkv, D)
     blobs, ids, cid = {}, [], 0
     for r, lens in enumerate(lens_per_req):
@@ -223,6 +225,51 @@ def test_p5_p6_order_and_duplicates_on_gpu():
         o_ref, l_ref = oracle.Request(sh, ch, 8).attend_new(0, q[r][None], kn[r][None], vn[r][None])
         check(ob[r], o_ref[0], lb[r], l_ref[0], f"dup case {r}")
     sess.close()
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,lens,S", [
+    (8, 2, 64, [[128, 128]], 16),                 # config 1 shape: 64 query rows per KV head
+    (32, 8, 128, [[300, 77], [129]], 40),         # ragged chunks, two requests, 160 rows -> two row blocks
+    (64, 8, 128, [[200]], 20),                    # G = 8
+    (4, 4, 128, [[65, 1, 64]], 70),               # G = 1, suffix longer than one tile (causal across two new tiles)
+    (8, 2, 128, [[]], 33),                        # no chunks at all: plain causal attention over the suffix
+    (8, 4, 64, [[31], [], [500, 3]], 130),        # D = 64, three new tiles, an empty request in the batch
+    (8, 2, 128, [[64]], 1),                       # a single suffix token through the tile kernel
+])
+def test_prefill_tensor_core_kernel(Hq, Hkv, D, lens, S):
+    run_requests(2, Hq, Hkv, D, lens, S, 3, seed=41, prefill_impl=2)
+
+
+@pytest.mark.parametrize("splits", [1, 2, 5])
+def test_prefill_tensor_core_split_invariance(splits):
+    run_requests(1, 32, 8, 128, [[700, 260, 64]], 24, 2, seed=42, prefill_impl=2, prefill_ctas=splits)
+
+
+def test_prefill_streaming_kernel_long_suffix():
+    run_requests(1, 8, 2, 128, [[100, 30]], 37, 2, seed=43, prefill_impl=1)   # forced onto the streaming kernel
+
+
+def test_prefill_appends_after_existing_tail():
+    """Two prefill calls in a row (chunked sub-prefill): the second sees the first's tokens in the tail."""
+    import paper_2512_22195_b200 as mk
+    L, Hq, Hkv, D = 1, 8, 2, 128
+    for impl in (1, 2):
+        sess = _session(L, Hq, Hkv, D, 1, 2, 80)
+        mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_IMPL, impl)
+        blobs = [rand_bits(44, i, (L, 2, Hkv, n, D)) for i, n in enumerate([90, 70])]
+        for i, b in enumerate(blobs):
+            sess.register_device_chunk(i, b)
+        sess.build_table([[0, 1]])
+        req = oracle.Request(oracle.Shape(L, Hq, Hkv, D), blobs, 80)
+        for part, S in enumerate([40, 24]):
+            q, k, v = rand_bits(44, 10 + part, (1, S, Hq, D)), rand_bits(44, 20 + part, (1, S, Hkv, D)), rand_bits(44, 30 + part, (1, S, Hkv, D))
+            out, lse = sess.prefill(0, _dev(q), _dev(k), _dev(v))
+            o_ref, l_ref = req.attend_new(0, q[0], k[0], v[0])
+            check(_bits(out)[0], o_ref, lse.cpu().numpy()[0], l_ref, f"impl {impl} part {part}")
+            sess.advance(S)
+            req.advance(S)
+        assert sess.status() == 0
+        sess.close()
 
 
 def test_cfg2_shape_two_layers_sampled_steps():
