@@ -378,38 +378,51 @@ def main():
         d2h = (ho_pf.numel() + ho_dc.numel()) * 2
         ctx2 = sess2.ctx
 
-        def e2e_step(i):
-            # load: pinned host -> device slots on the copy stream; the compute stream waits through the table
+        state = {"staged": -1}
+
+        def stage(i):
             sess2.stage(needed, slots[i % 2], slot_bytes, copy)
-            table = sess2.build_table(ids, sp)
+            state["staged"] = i
+
+        def e2e_step(i):
+            # load: pinned host -> device slots on the copy stream; the compute stream waits through the table.
+            # The NEXT step's chunks are staged into the other slot region right after this step's table is
+            # built, so that their copies run under this step's prefill and decode (the paper's overlap).
+            if state["staged"] < i:
+                stage(i)
+            # this step's query-side inputs, before the next step's chunk copies are queued on the copy engine
             dq_pf.copy_(hq_pf, non_blocking=True); dk_pf.copy_(hk_pf, non_blocking=True); dv_pf.copy_(hv_pf, non_blocking=True)
+            dq_dc.copy_(hq_dc, non_blocking=True); dk_dc.copy_(hk_dc, non_blocking=True); dv_dc.copy_(hv_dc, non_blocking=True)
+            table = sess2.build_table(ids, sp)
+            stage(i + 1)
             for layer in range(L):
                 mk.matkv_attend_prefill(ctx2, table, layer, S, dq_pf.data_ptr() + layer * qs_l, dk_pf.data_ptr() + layer * ks_l,
                                         dv_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
             mk.matkv_table_advance(table, S, sp)
-            ho_pf.copy_(o_pf, non_blocking=True)
             for t in range(T):
-                dq_dc[t].copy_(hq_dc[t], non_blocking=True); dk_dc[t].copy_(hk_dc[t], non_blocking=True)
-                dv_dc[t].copy_(hv_dc[t], non_blocking=True)
-                mk.matkv_attend_decode_all_layers(ctx2, table, dq_dc.data_ptr() + t * qd_t, dk_dc.data_ptr() + t * kd_t,
-                                                  dv_dc.data_ptr() + t * kd_t, o_dc.data_ptr() + t * qd_t, None, sp) \
-                    if args.decode_launch == "all_layers" else [
+                if args.decode_launch == "all_layers":
+                    mk.matkv_attend_decode_all_layers(ctx2, table, dq_dc.data_ptr() + t * qd_t, dk_dc.data_ptr() + t * kd_t,
+                                                      dv_dc.data_ptr() + t * kd_t, o_dc.data_ptr() + t * qd_t, None, sp)
+                else:
+                    for layer in range(L):
                         mk.matkv_attend_decode(ctx2, table, layer, dq_dc.data_ptr() + t * qd_t + layer * qd_l,
                                                dk_dc.data_ptr() + t * kd_t + layer * kd_l, dv_dc.data_ptr() + t * kd_t + layer * kd_l,
-                                               o_dc.data_ptr() + t * qd_t + layer * qd_l, None, sp) for layer in range(L)]
+                                               o_dc.data_ptr() + t * qd_t + layer * qd_l, None, sp)
                 mk.matkv_table_advance(table, 1, sp)
-                ho_dc[t].copy_(o_dc[t], non_blocking=True)      # the step's result goes back to the host
+            ho_pf.copy_(o_pf, non_blocking=True)                # the step's results go back to the host
+            ho_dc.copy_(o_dc, non_blocking=True)
             return 0
 
         with torch.cuda.stream(stream):
             for i in range(2):
                 e2e_step(i)
             k_e2e = min(args.steps, 5)
-            ms_e, _, _, _ = timed_region(e2e_step, k_e2e)
+            ms_e, _, _, _ = timed_region(lambda i: e2e_step(i + 2), k_e2e)
         if sess2.status() != 0:
             raise RuntimeError("device status non-zero after the end-to-end region")
         result["e2e"] = {"value": tokens * k_e2e / (ms_e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                          "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e,
+                         "overlap": "next step's chunks staged on a side stream under this step's prefill and decode",
                          "h2d_gbs_if_copy_bound": h2d * k_e2e / (ms_e * 1e-3) / 1e9}
         sess2.close()
         del host, slots

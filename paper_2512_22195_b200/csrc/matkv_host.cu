@@ -92,12 +92,21 @@ static void reap_graveyard(matkv_ctx *ctx, bool force);
 
 using namespace matkv;
 
-// tables whose stream work may still be running when the caller frees them
+// table images (pinned upload buffer + device copy) are recycled: allocating them per batch costs
+// milliseconds (cudaMallocHost and cudaMalloc synchronise).  A freed table's image waits in the
+// graveyard until the stream work that may still read it has finished, then moves to the pool.
 struct Grave {
     cudaEvent_t ev;
     void *h_pinned;
     void *d_image;
+    size_t bytes;
 };
+struct PooledImage {
+    void *h_pinned;
+    void *d_image;
+    size_t bytes;
+};
+static std::map<matkv_ctx *, std::vector<PooledImage>> g_pool;
 static std::map<matkv_ctx *, std::vector<Grave>> g_graves;
 
 static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
@@ -109,8 +118,12 @@ static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
         if (force) cudaEventSynchronize(v[i].ev);
         else done = (cudaEventQuery(v[i].ev) == cudaSuccess);
         if (done) {
-            cudaFreeHost(v[i].h_pinned);
-            cudaFree(v[i].d_image);
+            if (force) {
+                cudaFreeHost(v[i].h_pinned);
+                cudaFree(v[i].d_image);
+            } else {
+                g_pool[ctx].push_back(PooledImage{v[i].h_pinned, v[i].d_image, v[i].bytes});
+            }
             cudaEventDestroy(v[i].ev);
             v[i] = v.back();
             v.pop_back();
@@ -118,7 +131,17 @@ static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
             ++i;
         }
     }
-    if (force) g_graves.erase(it);
+    if (force) {
+        g_graves.erase(it);
+        auto pit = g_pool.find(ctx);
+        if (pit != g_pool.end()) {
+            for (auto &im : pit->second) {
+                cudaFreeHost(im.h_pinned);
+                cudaFree(im.d_image);
+            }
+            g_pool.erase(pit);
+        }
+    }
 }
 
 extern "C" {
@@ -478,8 +501,24 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
             return rc;
         }
     }
-    cudaError_t e = cudaMallocHost(&t->h_pinned, t->image_bytes);
-    if (e == cudaSuccess) e = cudaMalloc(&t->d_image, t->image_bytes);
+    cudaError_t e = cudaSuccess;
+    {
+        auto &pool = g_pool[ctx];
+        for (size_t i = 0; i < pool.size(); ++i)
+            if (pool[i].bytes >= t->image_bytes) {
+                t->h_pinned = pool[i].h_pinned;
+                t->d_image = pool[i].d_image;
+                t->image_alloc = pool[i].bytes;
+                pool[i] = pool.back();
+                pool.pop_back();
+                break;
+            }
+    }
+    if (!t->h_pinned) {
+        t->image_alloc = std::max<size_t>(t->image_bytes, 64 * 1024);
+        e = cudaMallocHost(&t->h_pinned, t->image_alloc);
+        if (e == cudaSuccess) e = cudaMalloc(&t->d_image, t->image_alloc);
+    }
     if (e != cudaSuccess) {
         cudaFreeHost(t->h_pinned);
         delete t;
@@ -528,6 +567,7 @@ int matkv_table_free(matkv_table *t, void *stream) {
     MATKV_CUDA(cudaEventRecord(g.ev, st));
     g.h_pinned = t->h_pinned;
     g.d_image = t->d_image;
+    g.bytes = t->image_alloc;
     g_graves[ctx].push_back(g);
     ctx->tables.erase(std::remove(ctx->tables.begin(), ctx->tables.end(), t), ctx->tables.end());
     delete t;

@@ -91,7 +91,7 @@ struct matkv_table {
     int64_t total_chunk_tiles = 0;
     void *h_pinned = nullptr;    // pinned upload image
     void *d_image = nullptr;     // device image: segs | reqs | tail_len[B]
-    size_t image_bytes = 0;
+    size_t image_bytes = 0, image_alloc = 0;
     matkv::DevSeg *d_segs = nullptr;
     matkv::DevReq *d_reqs = nullptr;
     int32_t *d_tail_len = nullptr;
