@@ -38,19 +38,23 @@ struct DeviceGuard {
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-int encode_rows_map(CUtensorMap *out, const void *base, int D, uint64_t rows) {
-    typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                                 const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                             const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeFn tensor_map_encoder() {
     static EncodeFn fn = nullptr;
     if (!fn) {
         void *p = nullptr;
         cudaDriverEntryPointQueryResult q;
         cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
-        if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !p)
-            return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
-        fn = (EncodeFn)p;
+        if (e == cudaSuccess && q == cudaDriverEntryPointSuccess) fn = (EncodeFn)p;
     }
+    return fn;
+}
+
+int encode_rows_map(CUtensorMap *out, const void *base, int D, uint64_t rows) {
+    EncodeFn fn = tensor_map_encoder();
+    if (!fn) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
     const cuuint64_t gdim[2] = {(cuuint64_t)D, (cuuint64_t)rows};
     const cuuint64_t gstride[1] = {(cuuint64_t)D * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
@@ -59,6 +63,20 @@ int encode_rows_map(CUtensorMap *out, const void *base, int D, uint64_t rows) {
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
+    return MATKV_OK;
+}
+
+int encode_new_rows_map(CUtensorMap *out, const void *base, int D, int Hkv, uint64_t n_tok) {
+    EncodeFn fn = tensor_map_encoder();
+    if (!fn) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    const cuuint64_t gdim[3] = {(cuuint64_t)D, (cuuint64_t)Hkv, (cuuint64_t)n_tok};
+    const cuuint64_t gstride[2] = {(cuuint64_t)D * 2, (cuuint64_t)Hkv * D * 2};
+    const cuuint32_t box[3] = {64, 1, (cuuint32_t)kTile};
+    const cuuint32_t estride[3] = {1, 1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), gdim, gstride, box, estride,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled (new rows) failed with %d", (int)r);
     return MATKV_OK;
 }
 

@@ -114,6 +114,8 @@ constexpr int kUnitRows = 8;  // query rows (suffix tokens x heads of one KV gro
 
 // 2-D tensor map over `rows` rows of D bf16 starting at `base` (box 64 x kTile, 128-byte swizzle, zero fill)
 int encode_rows_map(CUtensorMap *out, const void *base, int D, uint64_t rows);
+// 3-D tensor map over new-token rows [n_tok][Hkv][D]: box 64 columns x 1 head x kTile tokens, 128-byte swizzle
+int encode_new_rows_map(CUtensorMap *out, const void *base, int D, int Hkv, uint64_t n_tok);
 
 // Workspace layout: [counters: int32 x n_counter_slots][lse parts: fp32][o parts: fp32]
 struct WorkspaceView {

@@ -88,6 +88,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, int32_t z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -161,7 +167,8 @@ struct Cfg {
 };
 
 template <int D, int G>
-__global__ void __launch_bounds__(kThreads, 1) k_prefill_tc(const Params p) {
+__global__ void __launch_bounds__(kThreads, 1)
+k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap kn_map, const __grid_constant__ CUtensorMap vn_map) {
     using C = Cfg<D>;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -259,8 +266,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_prefill_tc(const Params p) {
             if (!ok) break;
             const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len);
             const uint32_t dst = smem_u32(kv_s + st * C::STAGE_BYTES), bar = full_kv + st * 8;
-            if (ti.kind < 2) {
-                if (lane == 0) {
+            if (lane == 0) {
+                mbar_expect_tx(bar, C::STAGE_BYTES);
+                if (ti.kind < 2) {
                     const CUtensorMap *mk, *mv;
                     int32_t yk, yv;
                     if (ti.kind == 0) {
@@ -272,45 +280,35 @@ __global__ void __launch_bounds__(kThreads, 1) k_prefill_tc(const Params p) {
                         mv = mk + 1;
                         yk = yv = ((b * p.n_layers_total + p.layer) * p.Hkv + g) * p.max_tail + ti.r0;
                     }
-                    mbar_expect_tx(bar, C::STAGE_BYTES);
 #pragma unroll
                     for (int bx = 0; bx < C::NBOX; ++bx) {
                         tma_load_2d(dst + bx * C::BOX_BYTES, mk, bx * 64, yk, bar);
                         tma_load_2d(dst + C::KV_BYTES + bx * C::BOX_BYTES, mv, bx * 64, yv, bar);
                     }
-                }
-            } else {
-                // the call's new tokens: copy rows by hand into the swizzled layout (zero rows past S)
-                constexpr int CPR = D / 8;  // 16-byte chunks per row
-                unsigned char *kd = kv_s + st * C::STAGE_BYTES, *vd = kd + C::KV_BYTES;
-                for (int idx = lane; idx < kTile * CPR; idx += 32) {
-                    const int row = idx / CPR, ch = idx % CPR;
-                    const int tok = ti.r0 + row;
-                    uint4 kvv = make_uint4(0, 0, 0, 0), vvv = make_uint4(0, 0, 0, 0);
-                    if (tok < p.S) {
-                        const int64_t off = (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
-                        kvv = *(const uint4 *)(p.k_new + off);
-                        vvv = *(const uint4 *)(p.v_new + off);
+                } else {
+                    // the call's new tokens, straight from k_new / v_new [B*S][Hkv][D] (rows past S are masked)
+#pragma unroll
+                    for (int bx = 0; bx < C::NBOX; ++bx) {
+                        tma_load_3d(dst + bx * C::BOX_BYTES, &kn_map, bx * 64, g, b * p.S + ti.r0, bar);
+                        tma_load_3d(dst + C::KV_BYTES + bx * C::BOX_BYTES, &vn_map, bx * 64, g, b * p.S + ti.r0, bar);
                     }
-                    const int o = (ch / 8) * C::BOX_BYTES + row * 128 + (((ch % 8) ^ (row & 7)) << 4);
-                    *(uint4 *)(kd + o) = kvv;
-                    *(uint4 *)(vd + o) = vvv;
                 }
-                fence_async_smem();  // generic-proxy writes -> visible to the tensor core's async proxy
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar);
             }
-        }
-        // append the new tokens to the tail for later calls (one CTA per (request, KV head))
-        if (rb == 0 && sp == p.n_split - 1) {
-            constexpr int CPR = D / 8;
-            for (int idx = lane; idx < p.S * CPR; idx += 32) {
-                const int tok = idx / CPR, ch = idx % CPR;
-                if (t0 + tok >= p.max_tail) continue;
-                const int64_t src = (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
-                const int64_t dst = ((((int64_t)b * p.n_layers_total + p.layer) * p.Hkv + g) * p.max_tail + t0 + tok) * D + ch * 8;
-                *(uint4 *)(p.tail_k + dst) = *(const uint4 *)(p.k_new + src);
-                *(uint4 *)(p.tail_v + dst) = *(const uint4 *)(p.v_new + src);
+            // append this split's share of the new tokens to the tail for later calls (the splits of row
+            // block 0 divide the S tokens among themselves), once the CTA's first loads are in flight
+            if (j == 0 && rb == 0) {
+                constexpr int CPR = D / 8;
+                const int a0 = (int)((int64_t)sp * p.S / p.n_split), a1 = (int)((int64_t)(sp + 1) * p.S / p.n_split);
+#pragma unroll 4
+                for (int idx = a0 * CPR + lane; idx < a1 * CPR; idx += 32) {
+                    const int tok = idx / CPR, ch = idx % CPR;
+                    if (t0 + tok < p.max_tail) {
+                        const int64_t src = (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
+                        const int64_t dsto = ((((int64_t)b * p.n_layers_total + p.layer) * p.Hkv + g) * p.max_tail + t0 + tok) * D + ch * 8;
+                        *(uint4 *)(p.tail_k + dsto) = *(const uint4 *)(p.k_new + src);
+                        *(uint4 *)(p.tail_v + dsto) = *(const uint4 *)(p.v_new + src);
+                    }
+                }
             }
         }
     } else if (warp == 1) {
@@ -475,14 +473,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_prefill_tc(const Params p) {
 }  // namespace k3
 
 template <int D, int G>
-static int launch_k3(const k3::Params &p, int grid, cudaStream_t stream) {
+static int launch_k3(const k3::Params &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
     using C = k3::Cfg<D>;
     static bool configured = false;
     if (!configured) {
         MATKV_CUDA(cudaFuncSetAttribute(k3::k_prefill_tc<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
         configured = true;
     }
-    k3::k_prefill_tc<D, G><<<grid, k3::kThreads, C::SMEM_BYTES, stream>>>(p);
+    k3::k_prefill_tc<D, G><<<grid, k3::kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());
     return MATKV_OK;
 }
@@ -518,9 +516,15 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     p.part_lse = ws.part_lse;
     p.part_o = ws.part_o;
     const int64_t grid = combos * p.n_split;
+    CUtensorMap kn_map, vn_map;
+    {
+        int rc2 = encode_new_rows_map(&kn_map, a.k_new, D, c.n_kv_heads, (uint64_t)t->batch * a.S);
+        if (!rc2) rc2 = encode_new_rows_map(&vn_map, a.v_new, D, c.n_kv_heads, (uint64_t)t->batch * a.S);
+        if (rc2) return rc2;
+    }
     int rc = fail(MATKV_E_INVALID_ARG, "tensor-core prefill: unsupported head_dim %d / group %d", D, G);
 #define MATKV_CASE(DD, GG) \
-    if (D == DD && G == GG) rc = launch_k3<DD, GG>(p, (int)grid, stream);
+    if (D == DD && G == GG) rc = launch_k3<DD, GG>(p, kn_map, vn_map, (int)grid, stream);
     MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)
     MATKV_CASE(64, 1) MATKV_CASE(64, 2) MATKV_CASE(64, 4) MATKV_CASE(64, 8)
 #undef MATKV_CASE
