@@ -263,10 +263,11 @@ def main():
             ev_d1[timed_index].record(stream)
         return n
 
+    from paper_2512_22195_b200 import replicas
+
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     def timed_region(fn, steps):
@@ -281,11 +282,7 @@ def main():
         e1.record(stream)
         barrier()
         t1 = time.time()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            tt = torch.tensor([ms], device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms = float(tt.item())
+        ms = replicas.max_over_ranks(e0.elapsed_time(e1), dev)
         return ms, n, t0, t1
 
     dev_ptrs = (q_pf.data_ptr(), k_pf.data_ptr(), v_pf.data_ptr(), q_dc.data_ptr(), k_dc.data_ptr(), v_dc.data_ptr())

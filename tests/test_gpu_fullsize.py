@@ -1,0 +1,76 @@
+"""Parity at the benchmark's full size and launch configuration (config 2: 32 layers, Llama-3-8B head
+shape, 5 x 1,024-token chunks, 64-token suffix through the tile kernel, 128 decode steps with all layers
+in one launch), on sampled outputs the oracle computes one by one."""
+import numpy as np
+import pytest
+import torch
+
+import matkv_inputs as mi
+import oracle
+from _util import check
+
+pytestmark = pytest.mark.gpu
+
+
+def test_cfg2_full_size_sampled_units():
+    import matkv_inputs.device as gen
+    from paper_2512_22195_b200.harness import Session, dev_to_bits
+    w = mi.workload("cfg2")
+    L, B, S, T, Hq, Hkv, D = w.n_layers, w.batch, w.suffix, w.decode_steps, w.n_q_heads, w.n_kv_heads, w.head_dim
+    ids = w.chunk_ids(0)
+    needed = sorted({c for row in ids for c in row})
+    sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T)
+    pool = torch.empty((len(needed), L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device="cuda")
+    for i, c in enumerate(needed):
+        gen.fill_bf16(pool[i], w.seed, mi.STREAM_CHUNK + c)
+        sess.register_device_chunk(c, pool[i])
+    q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device="cuda")
+    k_pf = torch.empty((L, B, S, Hkv, D), dtype=torch.bfloat16, device="cuda")
+    v_pf = torch.empty_like(k_pf)
+    q_dc = torch.empty((T, L, B, Hq, D), dtype=torch.bfloat16, device="cuda")
+    k_dc = torch.empty((T, L, B, Hkv, D), dtype=torch.bfloat16, device="cuda")
+    v_dc = torch.empty_like(k_dc)
+    for t_, st in ((q_pf, mi.STREAM_Q_PREFILL), (k_pf, mi.STREAM_K_PREFILL), (v_pf, mi.STREAM_V_PREFILL),
+                   (q_dc, mi.STREAM_Q_DECODE), (k_dc, mi.STREAM_K_DECODE), (v_dc, mi.STREAM_V_DECODE)):
+        gen.fill_bf16(t_, w.seed, st)
+    sess.build_table(ids)
+    pf = [sess.prefill(layer, q_pf[layer], k_pf[layer], v_pf[layer]) for layer in range(L)]
+    sess.advance(S)
+    dc = []
+    for t in range(T):
+        dc.append(sess.decode_all_layers(q_dc[t], k_dc[t], v_dc[t]))
+        sess.advance(1)
+    assert sess.status() == 0
+
+    sh1 = oracle.Shape(1, Hq, Hkv, D)                     # the oracle sees one layer's slabs at a time
+
+    def layer_request(layer, n_decode):
+        blobs = [dev_to_bits(pool[needed.index(c)][layer:layer + 1]) for c in ids[0]]
+        rq = oracle.Request(sh1, blobs, S + T)
+        _, k, v = mi.prefill_inputs(w, layer)
+        rq.append_only(0, k[0], v[0])
+        rq.advance(S)
+        for s_ in range(n_decode):
+            _, k, v = mi.decode_inputs(w, s_)
+            rq.append_only(0, k[layer, 0][None], v[layer, 0][None])
+            rq.advance(1)
+        return rq
+
+    # sub-prefill: layers 0 and 31, suffix rows 0, 31, 63
+    for layer in (0, L - 1):
+        rq = layer_request(layer, 0)
+        q, _, _ = mi.prefill_inputs(w, layer)
+        rows = [0, S // 2 - 1, S - 1]
+        o_ref, l_ref = oracle.attend(sh1, 0, rq.chunks, rq.tail_k[0], rq.tail_v[0], q[0][rows], [r + 1 for r in rows])
+        out, lse = pf[layer]
+        check(dev_to_bits(out)[0][rows], o_ref, lse.cpu().numpy()[0][rows], l_ref, f"full-size prefill layer {layer}")
+    # decode: sampled (step, layer) pairs, every head
+    for step, layer in ((0, 0), (0, L - 1), (63, 17), (T - 1, 0), (T - 1, L - 1)):
+        rq = layer_request(layer, step)
+        q, k, v = mi.decode_inputs(w, step)
+        o_ref, l_ref = rq.attend_new(0, q[layer, 0][None], k[layer, 0][None], v[layer, 0][None])
+        out, lse = dc[step]
+        check(dev_to_bits(out)[layer, 0], o_ref[0], lse.cpu().numpy()[layer, 0], l_ref[0], f"full-size decode step {step} layer {layer}")
+    # the inputs the GPU consumed are the generator's bytes (the oracle regenerated them on the host)
+    assert np.array_equal(dev_to_bits(q_dc[5]), mi.decode_inputs(w, 5)[0])
+    sess.close()
