@@ -91,33 +91,36 @@ class ClockSampler:
 
 # ---- the CPU oracle legs -------------------------------------------------------------------------
 class OracleState:
-    """Host copies of one batch and the oracle's requests (used by cpu_baseline and --impl reference)."""
+    """Host copies of one batch and the oracle's requests (used by cpu_baseline and --impl reference).
+    `layers` selects a subset of the model's layers (the work is exactly linear in layers); the chunk
+    blobs handed in hold only those layers, in that order."""
 
-    def __init__(self, w: mi.Workload, host_chunks, ids):
+    def __init__(self, w: mi.Workload, host_chunks, ids, layers=None):
         import oracle
         self.oracle, self.w = oracle, w
-        self.sh = oracle.Shape(w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim)
+        self.layers = list(range(w.n_layers)) if layers is None else list(layers)
+        self.sh = oracle.Shape(len(self.layers), w.n_q_heads, w.n_kv_heads, w.head_dim)
         cap = w.suffix + w.decode_steps
         self.reqs = [oracle.Request(self.sh, [host_chunks[c] for c in row], cap) for row in ids]
         self.cores = os.cpu_count() or 1
         # the tail as it stands after the sub-prefill: appended without attending (bookkeeping only)
-        for layer in range(w.n_layers):
+        for li, layer in enumerate(self.layers):
             _, k, v = mi.prefill_inputs(w, layer)
             for r, rq in enumerate(self.reqs):
-                rq.append_only(layer, k[r], v[r])
+                rq.append_only(li, k[r], v[r])
         for rq in self.reqs:
             rq.advance(w.suffix)
 
     def decode_steps(self, first_step: int, n_steps: int):
-        """Time n_steps decode steps (all layers, all requests) on all host cores; returns seconds."""
+        """Time n_steps decode steps (the selected layers, all requests) on all host cores; returns seconds."""
         w = self.w
         t0 = time.perf_counter()
         with ThreadPoolExecutor(max_workers=self.cores) as ex:
             for s in range(first_step, first_step + n_steps):
                 q, k, v = mi.decode_inputs(w, s)
-                jobs = [(layer, r) for layer in range(w.n_layers) for r in range(w.batch)]
-                list(ex.map(lambda lr: self.reqs[lr[1]].attend_new(lr[0], q[lr[0], lr[1]][None], k[lr[0], lr[1]][None],
-                                                                   v[lr[0], lr[1]][None]), jobs))
+                jobs = [(li, layer, r) for li, layer in enumerate(self.layers) for r in range(w.batch)]
+                list(ex.map(lambda j: self.reqs[j[2]].attend_new(j[0], q[j[1], j[2]][None], k[j[1], j[2]][None],
+                                                                 v[j[1], j[2]][None]), jobs))
                 for rq in self.reqs:
                     rq.advance(1)
         return time.perf_counter() - t0
@@ -142,8 +145,10 @@ def run_reference(args):
     ids = w.chunk_ids(0)
     needed = sorted({c for row in ids for c in row})
     log(f"[reference] generating {len(needed)} chunks on the host ...")
-    st = OracleState(w, host_chunks_numpy(w, needed), ids)
-    per_step = 1  # each bench step = one decode step of the workload over all layers and requests
+    n_l = w.n_layers if w.name in ("cfg1", "cfg2") else 1   # larger workloads: one layer per step (stated in `sample`)
+    blobs = {c: mi.chunk_blob_layers(w, c, n_l) for c in needed}
+    st = OracleState(w, blobs, ids, layers=list(range(n_l)))
+    per_step = 1  # each bench step = one decode step of the workload over the sampled layers and all requests
     for _ in range(args.warmup):
         st.decode_steps(0, per_step)
         st.rewind(per_step)
@@ -151,8 +156,9 @@ def run_reference(args):
     for _ in range(args.steps):
         t += st.decode_steps(0, per_step)
         st.rewind(per_step)
-    tok_s = args.steps * per_step * w.batch / t
-    sample = f"decode step 0 of {w.name} (all {w.n_layers} layers, batch {w.batch}), repeated per bench step"
+    tok_s = args.steps * per_step * w.batch / (t * w.n_layers / n_l)
+    sample = (f"decode step 0 of {w.name} ({n_l} of {w.n_layers} layers, batch {w.batch}), repeated per bench step"
+              + ("" if n_l == w.n_layers else ", extrapolated linearly to all layers"))
     print(json.dumps({
         "impl": "reference", "metric": "decode_tokens_per_s", "value": tok_s, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
@@ -176,6 +182,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--decode-ctas", type=int, default=0)
     ap.add_argument("--no-other-mode", action="store_true", help="skip the second pass in the other decode launch mode")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (small profiling cases)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -196,6 +204,12 @@ def main():
     dev = torch.device("cuda", local)
 
     w = mi.workload(args.workload)
+    if args.layers:
+        w.n_layers = args.layers
+        w.name += f"-L{args.layers}"
+    if args.decode_steps:
+        w.decode_steps = args.decode_steps
+        w.name += f"-T{args.decode_steps}"
     L, B, S, T, Hq, Hkv, D = w.n_layers, w.batch, w.suffix, w.decode_steps, w.n_q_heads, w.n_kv_heads, w.head_dim
     ids = w.chunk_ids(0)
     needed = sorted({c for row in ids for c in row})
@@ -354,7 +368,10 @@ def main():
     }
 
     # ---- end to end: the same step through the same calls, from host buffers --------------------
-    if not args.no_e2e:
+    e2e_bytes = len(needed) * w.chunk_bytes
+    if not args.no_e2e and e2e_bytes > 16e9:
+        result["e2e"] = {"value": None, "unit": "tokens/s", "skipped": f"{e2e_bytes / 1e9:.0f} GB of pinned host chunks: run with a smaller workload"}
+    elif not args.no_e2e:
         copy = torch.cuda.Stream(device=dev)
         host = {c: torch.empty(chunks[c].shape, dtype=torch.bfloat16, pin_memory=True) for c in needed}
         for c in needed:
@@ -429,15 +446,19 @@ def main():
         import oracle
         oracle.build()
         from paper_2512_22195_b200.harness import dev_to_bits
-        host_np = {c: dev_to_bits(chunks[c]) for c in needed}
-        st_o = OracleState(w, host_np, ids)
-        t_one = st_o.decode_steps(0, 1)
-        n_s = int(max(1, min(T - 1, round(12.0 / max(t_one, 1e-3)))))
-        t_s = st_o.decode_steps(1, n_s)
-        result["cpu_baseline"] = {"value": n_s * B / t_s, "unit": "tokens/s", "cores": st_o.cores, "kind": "oracle",
-                                  "sample": f"decode steps 1..{n_s} of {T} of {w.name} (all {L} layers, batch {B}), "
-                                            f"{t_s:.1f} s on {st_o.cores} threads",
-                                  "kv_gbs": sum((n + S + t + 1) * w.beta for n in n_req for t in range(1, 1 + n_s)) * L / t_s / 1e9}
+        # calibrate on one layer, then take as many layers and steps as fit ~12 s (work is linear in both)
+        probe = OracleState(w, {c: dev_to_bits(chunks[c][0:1]) for c in needed}, ids, layers=[0])
+        t_one = max(probe.decode_steps(0, 1), 1e-3)
+        n_l = int(max(1, min(L, 12.0 / t_one)))
+        n_s = int(max(1, min(T - 1, round(12.0 / (t_one * n_l)))))
+        st_o = OracleState(w, {c: dev_to_bits(chunks[c][0:n_l]) for c in needed}, ids, layers=list(range(n_l)))
+        t_s = st_o.decode_steps(0, n_s)
+        per_step_full = t_s / n_s * (L / n_l)
+        how = "" if n_l == L else f", extrapolated linearly from layers 0..{n_l - 1} to all {L}"
+        result["cpu_baseline"] = {"value": B / per_step_full, "unit": "tokens/s", "cores": st_o.cores, "kind": "oracle",
+                                  "sample": f"decode steps 0..{n_s - 1} of {T} of {w.name} ({n_l} of {L} layers, batch {B}), "
+                                            f"{t_s:.1f} s on {st_o.cores} threads{how}",
+                                  "kv_gbs": sum((n + S + t + 1) * w.beta for n in n_req for t in range(n_s)) * n_l / t_s / 1e9}
     if rank == 0:
         print(json.dumps(result), flush=True)
     sess.close()

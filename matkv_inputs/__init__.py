@@ -189,6 +189,13 @@ def chunk_blob(w: Workload, chunk_index: int, n_tokens: int | None = None, shift
         w.n_layers, 2, w.n_kv_heads, t, w.head_dim)
 
 
+def chunk_blob_layers(w: Workload, chunk_index: int, n_layers: int) -> np.ndarray:
+    """The first `n_layers` layers of one materialised chunk, [n_layers][2][Hkv][chunk_tokens][D] (a prefix of
+    the chunk's counter stream, so it equals chunk_blob(...)[:n_layers] without generating the rest)."""
+    n = n_layers * 2 * w.n_kv_heads * w.chunk_tokens * w.head_dim
+    return normal_bf16(w.seed, STREAM_CHUNK + chunk_index, n).reshape(n_layers, 2, w.n_kv_heads, w.chunk_tokens, w.head_dim)
+
+
 def prefill_inputs(w: Workload, layer: int, q_shift: int = 0):
     """(q [B,S,Hq,D], k_new [B,S,Hkv,D], v_new [B,S,Hkv,D]) bf16 bits for one layer."""
     B, S, Hq, Hkv, D = w.batch, w.suffix, w.n_q_heads, w.n_kv_heads, w.head_dim
