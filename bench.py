@@ -169,6 +169,154 @@ def run_reference(args):
     }), flush=True)
 
 
+# ---- pipelined serving (config 5): staging of batch n+1 under the compute of batch n ------------------
+def run_pipeline(args):
+    """Sequential request batches whose chunks live in a pinned host pool.  Three passes over the same
+    batches: staging alone, serial (stage, wait, compute), pipelined (batch n+1 staged on a side stream
+    while batch n is prefilled and decoded).  Overlap efficiency = (t_serial - t_pipelined) / t_stage."""
+    import torch
+    import paper_2512_22195_b200 as mk
+    import matkv_inputs.device as gen
+    from paper_2512_22195_b200.harness import Session
+
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    w = mi.workload(args.workload)
+    if args.layers:
+        w.n_layers = args.layers
+    if args.decode_steps:
+        w.decode_steps = args.decode_steps
+    if args.pool_chunks:
+        w.pool_chunks = args.pool_chunks
+    n_batches = args.batches or w.n_batches
+    L, B, S, T, Hq, Hkv, D = w.n_layers, w.batch, w.suffix, w.decode_steps, w.n_q_heads, w.n_kv_heads, w.head_dim
+    batches = [w.chunk_ids(i) for i in range(n_batches)]
+    needed = [sorted({c for row in ids for c in row}) for ids in batches]
+    n_slots = max(len(x) for x in needed)
+    slot_bytes = w.chunk_bytes
+    log(f"[pipeline] pinned pool: {w.pool_chunks} chunks x {slot_bytes / 1e6:.0f} MB = {w.pool_chunks * slot_bytes / 1e9:.1f} GB; "
+        f"{n_batches} batches of {B} x {w.chunks_per_req} chunks; 2 x {n_slots} device slots")
+    sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=dev.index)
+    host_pool = torch.empty((w.pool_chunks, L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, pin_memory=True)
+    tmp = torch.empty((L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
+    for c in range(w.pool_chunks):
+        gen.fill_bf16(tmp, w.seed, mi.STREAM_CHUNK + c)
+        host_pool[c].copy_(tmp)
+        mk.matkv_register_chunk(sess.ctx, c, w.chunk_tokens, host_pool[c].data_ptr(), None)
+    del tmp
+    slots = [torch.empty(n_slots * slot_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+    q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device=dev)
+    k_pf = torch.empty((L, B, S, Hkv, D), dtype=torch.bfloat16, device=dev)
+    v_pf = torch.empty_like(k_pf)
+    q_dc = torch.empty((T, L, B, Hq, D), dtype=torch.bfloat16, device=dev)
+    k_dc = torch.empty((T, L, B, Hkv, D), dtype=torch.bfloat16, device=dev)
+    v_dc = torch.empty_like(k_dc)
+    for t_, st in ((q_pf, mi.STREAM_Q_PREFILL), (k_pf, mi.STREAM_K_PREFILL), (v_pf, mi.STREAM_V_PREFILL),
+                   (q_dc, mi.STREAM_Q_DECODE), (k_dc, mi.STREAM_K_DECODE), (v_dc, mi.STREAM_V_DECODE)):
+        gen.fill_bf16(t_, w.seed, st)
+    o_pf, o_dc = torch.empty_like(q_pf), torch.empty_like(q_dc)
+    ho_dc = torch.empty(o_dc.shape, dtype=torch.bfloat16, pin_memory=True)
+    stream, copy = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    sp, ctx = stream.cuda_stream, sess.ctx
+    qs_l, ks_l, qd_t, kd_t = q_pf[0].numel() * 2, k_pf[0].numel() * 2, q_dc[0].numel() * 2, k_dc[0].numel() * 2
+    torch.cuda.synchronize()
+
+    def stage(n):
+        return sess.stage(needed[n], slots[n % 2], slot_bytes, copy)
+
+    def compute(n):
+        table = sess.build_table(batches[n], sp)
+        for layer in range(L):
+            mk.matkv_attend_prefill(ctx, table, layer, S, q_pf.data_ptr() + layer * qs_l, k_pf.data_ptr() + layer * ks_l,
+                                    v_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
+        mk.matkv_table_advance(table, S, sp)
+        for t in range(T):
+            mk.matkv_attend_decode_all_layers(ctx, table, q_dc.data_ptr() + t * qd_t, k_dc.data_ptr() + t * kd_t,
+                                              v_dc.data_ptr() + t * kd_t, o_dc.data_ptr() + t * qd_t, None, sp)
+            mk.matkv_table_advance(table, 1, sp)
+        with torch.cuda.stream(stream):
+            ho_dc.copy_(o_dc, non_blocking=True)
+
+    def wall(fn):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        fn()
+        torch.cuda.synchronize()
+        return time.perf_counter() - t0
+
+    def only_stage():
+        for n in range(n_batches):
+            stage(n)
+
+    def serial():
+        for n in range(n_batches):
+            tk = stage(n)
+            mk.matkv_stage_wait(ctx, tk)
+            compute(n)
+            torch.cuda.synchronize()
+
+    def pipelined():
+        stage(0)
+        for n in range(n_batches):
+            compute_with_stage(n)   # builds table n (resolves its slots), then sends batch n+1 to the other region
+
+    def compute_with_stage(n):
+        table = sess.build_table(batches[n], sp)
+        if n + 1 < n_batches:
+            stage(n + 1)
+        for layer in range(L):
+            mk.matkv_attend_prefill(ctx, table, layer, S, q_pf.data_ptr() + layer * qs_l, k_pf.data_ptr() + layer * ks_l,
+                                    v_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
+        mk.matkv_table_advance(table, S, sp)
+        for t in range(T):
+            mk.matkv_attend_decode_all_layers(ctx, table, q_dc.data_ptr() + t * qd_t, k_dc.data_ptr() + t * kd_t,
+                                              v_dc.data_ptr() + t * kd_t, o_dc.data_ptr() + t * qd_t, None, sp)
+            mk.matkv_table_advance(table, 1, sp)
+        with torch.cuda.stream(stream):
+            ho_dc.copy_(o_dc, non_blocking=True)
+
+    # warm-up: two batches through the whole path
+    stage(0); compute(0); stage(1); compute(1)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index)
+    t_stage = wall(only_stage)
+    t_serial = wall(serial)
+    t0 = time.time()
+    t_pipe = wall(pipelined)
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    if sess.status() != 0:
+        raise RuntimeError("device status non-zero after the pipeline")
+    # bytes one pass really copies: a chunk that already sits in the target slot region is not copied again
+    occ, n_copied = [set(), set()], 0
+    for n in range(n_batches):
+        new = set(needed[n]) - occ[n % 2]
+        n_copied += len(new)
+        occ[n % 2] = set(needed[n])
+        occ[(n + 1) % 2] -= new
+    staged_bytes = n_copied * slot_bytes
+    tokens = n_batches * B * T
+    kv_bytes = sum((len(row) * w.chunk_tokens + S + t + 1) * w.beta for ids in batches for row in ids for t in range(T)) * L
+    t_compute = t_serial - t_stage
+    print(json.dumps({
+        "metric": "decode_tokens_per_s", "value": tokens / t_pipe, "unit": "tokens/s", "n_gpus": 1, "steps": n_batches,
+        "warmup": 2, "ms_per_step": 1e3 * t_pipe / n_batches, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 in, fp32 softmax/accumulate", "data": "synthetic",
+        "config": {"workload": w.name, "layers": L, "batch": B, "chunks_per_request": w.chunks_per_req, "suffix": S,
+                   "decode_steps": T, "pool_chunks": w.pool_chunks, "pinned_pool_gb": w.pool_chunks * slot_bytes / 1e9,
+                   "batches": n_batches, "timing": "host wall clock around synchronised passes (copy and compute streams)"},
+        "clocks": clocks,
+        "pipeline": {"t_stage_s": t_stage, "t_serial_s": t_serial, "t_pipelined_s": t_pipe,
+                     "h2d_gbs_staging_alone": staged_bytes / t_stage / 1e9, "staged_bytes": staged_bytes,
+                     "overlap_efficiency": (t_serial - t_pipe) / t_stage if t_stage > 0 else None,
+                     "requests_per_s": n_batches * B / t_pipe, "compute_s_estimate": t_compute,
+                     "decode_kv_gbs_pipelined_lower_bound": kv_bytes / t_pipe / 1e9},
+        "e2e": {"value": tokens / t_pipe, "unit": "tokens/s", "h2d_bytes_per_step": staged_bytes / n_batches,
+                "d2h_bytes_per_step": ho_dc.numel() * 2},
+    }), flush=True)
+    sess.close()
+
+
 # ---- the CUDA arm ----------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -182,11 +330,15 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--decode-ctas", type=int, default=0)
     ap.add_argument("--no-other-mode", action="store_true", help="skip the second pass in the other decode launch mode")
+    ap.add_argument("--batches", type=int, default=0, help="pipelined serving: number of sequential batches")
+    ap.add_argument("--pool-chunks", type=int, default=0, help="pipelined serving: chunks in the pinned host pool")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (small profiling cases)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload == "cfg5":
+        return run_pipeline(args)
     args.warmup = max(args.warmup, 3)
 
     import torch
