@@ -80,6 +80,14 @@ int encode_new_rows_map(CUtensorMap *out, const void *base, int D, int Hkv, uint
     return MATKV_OK;
 }
 
+size_t rope_scratch_bytes(const matkv_config &c) {
+    if (c.rope_theta == 0.f) return 0;
+    const size_t per_tok = (size_t)(c.n_q_heads + c.n_kv_heads) * c.head_dim * sizeof(__nv_bfloat16);
+    const size_t prefill = (size_t)c.max_batch * c.max_tail_tokens * per_tok;  // one layer, up to max_tail tokens
+    const size_t decode = (size_t)c.n_layers * c.max_batch * per_tok;          // all layers, one token
+    return align_up(std::max(prefill, decode), 256);
+}
+
 size_t workspace_bytes_for(const matkv_config &c, WorkspaceView *v, void *base) {
     const int64_t G = kUnitRows;
     const int64_t units_decode = (int64_t)c.n_layers * c.max_batch * c.n_kv_heads;
@@ -101,6 +109,7 @@ size_t workspace_bytes_for(const matkv_config &c, WorkspaceView *v, void *base) 
         v->n_counter_slots = n_units;
         v->n_part_slots = n_parts;
     }
+    off += rope_scratch_bytes(c);  // rotary mode: the rotated q / k_new of one call sit behind the partials
     return off;
 }
 
@@ -626,8 +635,6 @@ static int check_attend(matkv_ctx *ctx, matkv_table *t, const void *q, const voi
     if (t->tail_len_host + n_new > ctx->cfg.max_tail_tokens)
         return fail(MATKV_E_CAPACITY, "%s: tail holds %d tokens, %d more exceed max_tail_tokens %d", who, t->tail_len_host,
                     n_new, ctx->cfg.max_tail_tokens);
-    if (ctx->cfg.rope_theta != 0.f)
-        return fail(MATKV_E_INVALID_ARG, "%s: rotary mode is not available in this build; pass rotated q and k_new", who);
     return MATKV_OK;
 }
 
@@ -650,6 +657,10 @@ int matkv_attend_decode(matkv_ctx *ctx, matkv_table *t, int32_t layer, const voi
     a.q_sl = 0; a.q_sb = (int64_t)c.n_q_heads * c.head_dim; a.q_ss = 0;
     a.kn_sl = 0; a.kn_sb = (int64_t)c.n_kv_heads * c.head_dim; a.kn_ss = 0;
     a.lse_sl = 0; a.lse_sb = c.n_q_heads; a.lse_ss = 0;
+    if (c.rope_theta != 0.f) {
+        rc = launch_rope(ctx, t, a, (cudaStream_t)stream);
+        if (rc) return rc;
+    }
     return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
 }
 
@@ -671,6 +682,10 @@ int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *t, const void *q
     a.q_sb = (int64_t)c.n_q_heads * c.head_dim; a.q_sl = a.q_sb * t->batch; a.q_ss = 0;
     a.kn_sb = (int64_t)c.n_kv_heads * c.head_dim; a.kn_sl = a.kn_sb * t->batch; a.kn_ss = 0;
     a.lse_sb = c.n_q_heads; a.lse_sl = a.lse_sb * t->batch; a.lse_ss = 0;
+    if (c.rope_theta != 0.f) {
+        rc = launch_rope(ctx, t, a, (cudaStream_t)stream);
+        if (rc) return rc;
+    }
     return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
 }
 
@@ -694,6 +709,10 @@ int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t 
     a.q_ss = (int64_t)c.n_q_heads * c.head_dim; a.q_sb = a.q_ss * S; a.q_sl = 0;
     a.kn_ss = (int64_t)c.n_kv_heads * c.head_dim; a.kn_sb = a.kn_ss * S; a.kn_sl = 0;
     a.lse_ss = c.n_q_heads; a.lse_sb = a.lse_ss * S; a.lse_sl = 0;
+    if (c.rope_theta != 0.f) {
+        rc = launch_rope(ctx, t, a, (cudaStream_t)stream);
+        if (rc) return rc;
+    }
     // long suffixes go to the tcgen05 tile kernel, short ones stay on the streaming kernel
     const int G = c.n_q_heads / c.n_kv_heads;
     const bool tensor_core = ctx->opt_prefill_impl == 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);

@@ -125,6 +125,7 @@ struct WorkspaceView {
     int64_t n_counter_slots, n_part_slots;
 };
 size_t workspace_bytes_for(const matkv_config &c, WorkspaceView *view_from_base, void *base);
+size_t rope_scratch_bytes(const matkv_config &c);  // rotated q / k_new of one call (0 unless rotary mode)
 
 // ---- launchers (defined next to their kernels) ----------------------------------------------
 struct AttendArgs {
@@ -139,6 +140,7 @@ struct AttendArgs {
     int64_t lse_sl, lse_sb, lse_ss;
 };
 int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
+int launch_rope(matkv_ctx *ctx, matkv_table *t, AttendArgs &a, cudaStream_t stream);
 int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
 int launch_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts,
                        const float *lse_parts, void *out, float *lse_out, cudaStream_t stream);

@@ -28,12 +28,12 @@ def _bits(t):
 
 
 def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=False, q_shift=0, cap=None,
-                 prefill_impl=0, prefill_ctas=0):
+                 prefill_impl=0, prefill_ctas=0, rope_theta=0.0, pos_mode=0):
     """Prefill S tokens then T decode steps for a batch; compare every output with the oracle."""
     import paper_2512_22195_b200 as mk
     B = len(lens_per_req)
     cap = cap or (S + T)
-    sess = _session(L, Hq, Hkv, D, B, max(1, max(len(x) for x in lens_per_req)), cap)
+    sess = _session(L, Hq, Hkv, D, B, max(1, max(len(x) for x in lens_per_req)), cap, rope_theta=rope_theta, pos_mode=pos_mode)
     if ctas:
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, ctas)
     if prefill_impl:
@@ -51,7 +51,10 @@ def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=Fal
             cid += 1
         ids.append(row)
     sess.build_table(ids)
-    reqs = [oracle.Request(sh, [blobs[c] for c in row], cap) for row in ids]
+    def pos_base(row):
+        lens = [blobs[c].shape[3] for c in row]
+        return None if pos_mode == 0 else max(lens, default=0)
+    reqs = [oracle.Request(sh, [blobs[c] for c in row], cap, rope_theta=rope_theta, pos_base=pos_base(row)) for row in ids]
     worst = [0.0, 0.0, 0.0]
 
     def upd(m):
@@ -270,6 +273,18 @@ def test_prefill_appends_after_existing_tail():
             req.advance(S)
         assert sess.status() == 0
         sess.close()
+
+
+@pytest.mark.parametrize("S,impl", [(5, 0), (40, 2)])
+def test_p9_rotary_mode_positions(S, impl):
+    """q and k_new are rotated at position (sum of chunk lengths) + tail index; stored chunk K is used as it is.
+    The tails must match the oracle's bit for bit (rotation in fp64, rounded once to bf16, on both sides)."""
+    run_requests(2, 8, 2, 128, [[300, 77], [129]], S, 3, seed=51, rope_theta=500000.0, prefill_impl=impl)
+    run_requests(1, 8, 2, 64, [[64, 200]], S, 2, seed=52, rope_theta=10000.0, prefill_impl=impl, all_layers=True)
+
+
+def test_p9_rotary_position_base_is_a_parameter():
+    run_requests(1, 4, 2, 128, [[100, 30]], 6, 2, seed=53, rope_theta=500000.0, pos_mode=1)   # base = longest chunk
 
 
 def test_cfg2_shape_two_layers_sampled_steps():
