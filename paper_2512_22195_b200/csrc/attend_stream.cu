@@ -12,8 +12,8 @@
 // short enough for the kernel to stay HBM-bound at any G (a plain-FMA inner product measured
 // issue-bound: 42% issue utilisation with 8 resident warps and 48% of DRAM peak).  fp32 scores,
 // exp2-based softmax, fp32 accumulators; P is rounded to bf16 for the second MMA.
-// The new tokens of the call (not yet in the tail) are attended by a short scalar path and appended to
-// the tail by the same warp.  At the end of a unit the warps' states are merged through shared memory;
+// The new tokens of the call (not yet in the tail) come through the same ring from k_new / v_new (a
+// per-call TMA descriptor) with a causal mask, and the warp that handles them appends them to the tail.  At the end of a unit the warps' states are merged through shared memory;
 // a unit that spans several CTAs leaves one partial (normalised o, lse) per CTA in the workspace and
 // the last CTA to arrive (atomic ticket, no waiting) merges them by log-sum-exp.
 #include <cuda_runtime.h>
@@ -34,7 +34,7 @@ constexpr int kMaxDynSmem = 232448;             // 227 KB opt-in limit per CTA o
 constexpr long long kWaitCycles = 2000000000LL; // bounded waits give up after about a second
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr uint32_t kTagNew = 0x8000u;           // tile tag: the unit's new-token pseudo tile (no copy)
+constexpr uint32_t kTagNew = 0x8000u;           // tile tag: a tile of the call's new tokens (bits 8..14: its index)
 
 struct StreamParams {
     const DevReq *reqs;
@@ -118,6 +118,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int32_t x, int32_t y, int32_t z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kCW * 32) : "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
@@ -154,7 +160,7 @@ __host__ __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b -
 struct UnitPos {
     int32_t l_rel, b, blk, g;  // layer (relative to layer0), request, block of suffix tokens, KV head
     int32_t tile;              // first tile of this CTA's share inside the unit
-    int32_t rt;                // tiles in the unit: chunk tiles, tail tiles, one pseudo tile for the new tokens
+    int32_t rt;                // tiles in the unit: chunk tiles, tail tiles, ceil(S / kTile) tiles of new tokens
     int32_t chunk_tiles, tail_tiles, t0, seg_begin;
     int64_t flat_begin;        // flat index of the unit's first tile
 };
@@ -179,7 +185,7 @@ __device__ __forceinline__ void load_req(const StreamParams &p, UnitPos &u) {
     u.chunk_tiles = rq.chunk_tiles;
     u.seg_begin = rq.seg_begin;
     u.tail_tiles = ceil_div(u.t0, kTile);
-    u.rt = u.chunk_tiles + u.tail_tiles + 1;
+    u.rt = u.chunk_tiles + u.tail_tiles + ceil_div(p.S, kTile);
 }
 
 // advance to the next unit in (layer, request, token block, head) order
@@ -200,7 +206,7 @@ __device__ __forceinline__ void next_unit(const StreamParams &p, UnitPos &u, int
 __device__ void locate_range(const StreamParams &p, CtaRange &r, int n_blk) {
     int64_t w_layer = 0;
     for (int b = 0; b < p.B; ++b) {
-        const int rt = p.reqs[b].chunk_tiles + ceil_div(clamp_t0(p, b), kTile) + 1;
+        const int rt = p.reqs[b].chunk_tiles + ceil_div(clamp_t0(p, b), kTile) + ceil_div(p.S, kTile);
         w_layer += (int64_t)p.Hkv * n_blk * rt;
     }
     r.W = w_layer * p.n_layers_launch;
@@ -215,7 +221,7 @@ __device__ void locate_range(const StreamParams &p, CtaRange &r, int n_blk) {
     int64_t rem = f % w_layer;
     int b = 0;
     for (; b < p.B; ++b) {
-        const int rt = p.reqs[b].chunk_tiles + ceil_div(clamp_t0(p, b), kTile) + 1;
+        const int rt = p.reqs[b].chunk_tiles + ceil_div(clamp_t0(p, b), kTile) + ceil_div(p.S, kTile);
         const int64_t blk = (int64_t)p.Hkv * n_blk * rt;
         if (rem < blk) break;
         rem -= blk;
@@ -251,14 +257,30 @@ __device__ void combine_warp(const float *o_parts, int64_t o_stride, const float
 #pragma unroll
     for (int off = 16; off; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
     const float lse = m + logf(z);
-    for (int d = lane; d < D; d += 32) {
-        float acc = 0.f;
-        for (int p = 0; p < P; ++p) {
-            const float w = exp2f((__ldcg(lse_parts + p * lse_stride) - lse) * kLog2e);
-            acc = fmaf(w, __ldcg(o_parts + p * o_stride + d), acc);
+    // every lane owns D/32 consecutive dims; the weights of 32 parts at a time sit one per lane and are
+    // broadcast by shuffle, so the loads of the parts' rows are independent and stay in flight together
+    const int dpl = D >> 5;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int p0 = 0; p0 < P; p0 += 32) {
+        const float w_mine = p0 + lane < P ? exp2f((__ldcg(lse_parts + (p0 + lane) * lse_stride) - lse) * kLog2e) : 0.f;
+        const int np = min(32, P - p0);
+#pragma unroll 4
+        for (int pp = 0; pp < np; ++pp) {
+            const float w = __shfl_sync(0xffffffffu, w_mine, pp);
+            const float *row = o_parts + (p0 + pp) * o_stride + lane * dpl;
+            if (dpl == 4) {
+                const float4 v = __ldcg((const float4 *)row);
+                acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+                acc[2] = fmaf(w, v.z, acc[2]); acc[3] = fmaf(w, v.w, acc[3]);
+            } else if (dpl == 2) {
+                const float2 v = __ldcg((const float2 *)row);
+                acc[0] = fmaf(w, v.x, acc[0]); acc[1] = fmaf(w, v.y, acc[1]);
+            } else {
+                for (int i = 0; i < dpl; ++i) acc[i] = fmaf(w, __ldcg(row + i), acc[i]);
+            }
         }
-        out[d] = __float2bfloat16(acc);
     }
+    for (int i = 0; i < dpl; ++i) out[lane * dpl + i] = __float2bfloat16(acc[i]);
     if (lse_out && lane == 0) *lse_out = lse;
 }
 
@@ -291,7 +313,8 @@ struct StreamCfg {
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
 template <int D, int G>
-__global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParams p) {
+__global__ void __launch_bounds__(kThreads, 1)
+k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ CUtensorMap kn_map, const __grid_constant__ CUtensorMap vn_map) {
     using C = StreamCfg<D, G>;
     extern __shared__ unsigned char smem_raw[];
     // the swizzle pattern repeats every 1024 bytes: align the ring to it
@@ -344,9 +367,16 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
                     break;
                 }
                 const uint32_t bar = full_u32 + stage * 8, dst = ring_u32 + stage * C::STAGE_BYTES;
-                if (t >= u.chunk_tiles + u.tail_tiles) {  // the new tokens: nothing to copy
-                    tags[stage] = kTagNew | (use << 16);
-                    mbar_arrive(bar);
+                if (t >= u.chunk_tiles + u.tail_tiles) {  // the call's new tokens, from k_new / v_new [layer][request][token][head][D]
+                    const int nt = t - u.chunk_tiles - u.tail_tiles;
+                    const int32_t z = (u.l_rel * p.B + u.b) * p.S + nt * kTile;
+                    tags[stage] = (uint32_t)min(kTile, p.S - nt * kTile) | ((uint32_t)nt << 8) | kTagNew | (use << 16);
+                    mbar_expect_tx(bar, C::STAGE_BYTES);
+#pragma unroll
+                    for (int bx = 0; bx < C::NBOX; ++bx) {
+                        tma_load_3d(dst + bx * C::BOX_BYTES, &kn_map, bx * 64, u.g, z, bar);
+                        tma_load_3d(dst + (C::NBOX + bx) * C::BOX_BYTES, &vn_map, bx * 64, u.g, z, bar);
+                    }
                     continue;
                 }
                 const CUtensorMap *mk, *mv;
@@ -444,65 +474,16 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
             const uint32_t tag = stage_wait(tags + stage, use, full_u32 + stage * 8, use & 1, flags);
             const uint32_t stage_u32 = ring_u32 + stage * C::STAGE_BYTES;
 
-            if (tag & kTagNew) {
-                // ---------- the call's new tokens (scalar path, one warp per unit) ----------
-                if (piece == 0) {
-                    const int n_new = tok0 + n_tok;  // new rows 0 .. tok0+n_tok-1 exist; row `qr` sees 0 .. tok0 + qr/G
-                    const int my_last = tok0 + qr / G;
-                    constexpr int DL = D / 32;       // dims per lane in the dot product
-                    float qs[kUnitRows][DL];
-#pragma unroll
-                    for (int r = 0; r < kUnitRows; ++r) {
-                        const __nv_bfloat16 *qrow = p.q + q_base + (int64_t)(r / G) * p.q_ss + (r % G) * D + lane * DL;
-#pragma unroll
-                        for (int d = 0; d < DL; ++d) qs[r][d] = r < n_rows ? __bfloat162float(qrow[d]) : 0.f;
-                    }
-                    const int64_t kn_base = (int64_t)u.l_rel * p.kn_sl + (int64_t)u.b * p.kn_sb + (int64_t)u.g * D;
-                    for (int jn = 0; jn < n_new; ++jn) {
-                        const __nv_bfloat16 *krow = p.k_new + kn_base + (int64_t)jn * p.kn_ss;
-                        const __nv_bfloat16 *vrow = p.v_new + kn_base + (int64_t)jn * p.kn_ss;
-                        float kd[DL];
-#pragma unroll
-                        for (int d = 0; d < DL; ++d) kd[d] = __bfloat162float(krow[lane * DL + d]);
-                        float mine = 0.f;
-#pragma unroll
-                        for (int r = 0; r < kUnitRows; ++r) {
-                            float a = 0.f;
-#pragma unroll
-                            for (int d = 0; d < DL; ++d) a = fmaf(qs[r][d], kd[d], a);
-#pragma unroll
-                            for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
-                            if (r == qr) mine = a;
-                        }
-                        const bool vis = qr < n_rows && jn <= my_last;
-                        const float s = vis ? mine * p.scale_log2 : -CUDART_INF_F;
-                        const float m_new = fmaxf(m_run, s);
-                        const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);
-                        const float pv = vis ? fast_exp2(s - m_new) : 0.f;
-                        l_run = l_run * alpha + (qc == 0 ? pv : 0.f);
-                        m_run = m_new;
-#pragma unroll
-                        for (int nb = 0; nb < 2 * C::KS; ++nb) {
-                            const uint32_t vv = *(const uint32_t *)(vrow + nb * 8 + 2 * qc);
-                            o[nb][0] = fmaf(pv, bf_lo(vv), o[nb][0] * alpha);
-                            o[nb][1] = fmaf(pv, bf_hi(vv), o[nb][1] * alpha);
-                        }
-                        // the unit's own tokens go to the tail for later calls
-                        if (jn >= tok0 && u.t0 + jn < p.max_tail) {
-                            const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + u.t0 + jn) * D;
-                            if (lane < D / 8) {
-                                *(uint4 *)(p.tail_k + off + lane * 8) = *(const uint4 *)(krow + lane * 8);
-                                *(uint4 *)(p.tail_v + off + lane * 8) = *(const uint4 *)(vrow + lane * 8);
-                            }
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_u32 + stage * 8);
-                continue;
+            int rows = (int)(tag & 0x7f) - r0;        // valid rows of this work item (may be <= 0)
+            // new tokens: column c of the item is token new0 + c of the call; this thread's query row
+            // (suffix token tok0 + qr / G) sees the tokens up to and including itself
+            const bool is_new = (tag & kTagNew) != 0;
+            const int new0 = (int)((tag >> 8) & 0x7f) * kTile + r0;
+            int vis = rows;                           // columns this thread's row may see
+            if (is_new) {
+                vis = min(rows, tok0 + qr / G - new0 + 1);
+                rows = min(rows, tok0 + n_tok - new0);  // nothing past the unit's last token is visible to any row
             }
-
-            const int rows = (int)(tag & 0xff) - r0;  // valid rows of this work item (may be <= 0)
             if (rows > 0) {
                 // ---------- S = Q K^T for 16 tokens (two 8-token blocks) ----------
                 float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -516,17 +497,19 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
                     mma_bf16(s1, qa[ks][0], 0u, qa[ks][1], 0u, kb[2], kb[3]);
                 }
                 // ---------- online softmax (this thread: row qr, tokens 2qc, 2qc+1, 8+2qc, 9+2qc) ----------
-                const float x0 = 2 * qc < rows ? s0[0] * p.scale_log2 : -CUDART_INF_F;
-                const float x1 = 2 * qc + 1 < rows ? s0[1] * p.scale_log2 : -CUDART_INF_F;
-                const float x2 = 8 + 2 * qc < rows ? s1[0] * p.scale_log2 : -CUDART_INF_F;
-                const float x3 = 9 + 2 * qc < rows ? s1[1] * p.scale_log2 : -CUDART_INF_F;
+                const float x0 = 2 * qc < vis ? s0[0] * p.scale_log2 : -CUDART_INF_F;
+                const float x1 = 2 * qc + 1 < vis ? s0[1] * p.scale_log2 : -CUDART_INF_F;
+                const float x2 = 8 + 2 * qc < vis ? s1[0] * p.scale_log2 : -CUDART_INF_F;
+                const float x3 = 9 + 2 * qc < vis ? s1[1] * p.scale_log2 : -CUDART_INF_F;
                 float tmax = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
                 tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
                 tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-                const float m_new = fmaxf(m_run, tmax);  // finite: token 0 of the item is valid
-                const float alpha = fast_exp2(m_run - m_new);
-                const float p0 = fast_exp2(x0 - m_new), p1 = fast_exp2(x1 - m_new);
-                const float p2 = fast_exp2(x2 - m_new), p3 = fast_exp2(x3 - m_new);
+                const float m_new = fmaxf(m_run, tmax);
+                // a row that has seen nothing yet (causal edge of the new tokens) keeps an empty state
+                const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
+                const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);
+                const float p0 = fast_exp2(x0 - m_use), p1 = fast_exp2(x1 - m_use);
+                const float p2 = fast_exp2(x2 - m_use), p3 = fast_exp2(x3 - m_use);
                 l_run = l_run * alpha + ((p0 + p1) + (p2 + p3));
                 m_run = m_new;
                 if (__any_sync(0xffffffffu, alpha != 1.0f)) {
@@ -547,6 +530,22 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
                     ldsm_x4_trans(v_u32 + (dp / 4) * C::BOX_BYTES + swz(r0 + (mi & 1) * 8 + ri, c), vb);
                     mma_bf16(o[2 * dp], pa0, 0u, pa2, 0u, vb[0], vb[1]);
                     mma_bf16(o[2 * dp + 1], pa0, 0u, pa2, 0u, vb[2], vb[3]);
+                }
+                // ---------- the unit's own new tokens go to the tail for later calls ----------
+                if (is_new) {
+                    constexpr int CPR = D / 8;  // 16-byte chunks per row; lanes 0..CPR-1 move K, the next CPR lanes move V
+                    const unsigned char *ring_stage = ring + stage * C::STAGE_BYTES;
+                    for (int r = max(0, tok0 - new0); r < rows; ++r) {
+                        const int tok = new0 + r;  // token of the call, tok0 <= tok < tok0 + n_tok
+                        if (u.t0 + tok >= p.max_tail) break;
+                        const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + u.t0 + tok) * D;
+                        const int ch = lane % CPR, kv = lane / CPR;
+                        if (kv < 2) {
+                            const uint4 val = *(const uint4 *)(ring_stage + kv * C::NBOX * C::BOX_BYTES + (ch / 8) * C::BOX_BYTES +
+                                                               swz(r0 + r, ch % 8));
+                            *(uint4 *)((kv ? p.tail_v : p.tail_k) + off + ch * 8) = val;
+                        }
+                    }
                 }
             }
             __syncwarp();
@@ -629,14 +628,14 @@ __global__ void __launch_bounds__(kThreads, 1) k_attend_stream(const StreamParam
 
 // ---- launchers --------------------------------------------------------------------------------------
 template <int D, int G>
-static int launch_stream_t(const StreamParams &p, int grid, cudaStream_t stream) {
+static int launch_stream_t(const StreamParams &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
     using C = StreamCfg<D, G>;
     static bool configured = false;
     if (!configured) {
         MATKV_CUDA(cudaFuncSetAttribute(k_attend_stream<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
         configured = true;
     }
-    k_attend_stream<D, G><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p);
+    k_attend_stream<D, G><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());
     return MATKV_OK;
 }
@@ -672,12 +671,20 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     // tiles in the launch as far as the host knows (the device recomputes it from its own tail length)
     int64_t W = 0;
     for (int b = 0; b < t->batch; ++b)
-        W += (int64_t)c.n_kv_heads * n_blk * (t->h_reqs[b].chunk_tiles + ceil_div(t->tail_len_host, kTile) + 1);
+        W += (int64_t)c.n_kv_heads * n_blk * (t->h_reqs[b].chunk_tiles + ceil_div(t->tail_len_host, kTile) + ceil_div(a.S, kTile));
     W *= a.n_layers_launch;
+    // the call's new tokens are fetched through their own descriptor: k_new / v_new [layers][B][S][Hkv][D]
+    CUtensorMap kn_map, vn_map;
+    {
+        const uint64_t n_tok = (uint64_t)a.n_layers_launch * t->batch * a.S;
+        int rc = encode_new_rows_map(&kn_map, a.k_new, c.head_dim, c.n_kv_heads, n_tok);
+        if (!rc) rc = encode_new_rows_map(&vn_map, a.v_new, c.head_dim, c.n_kv_heads, n_tok);
+        if (rc) return rc;
+    }
     int64_t grid = ctx->opt_decode_ctas > 0 ? ctx->opt_decode_ctas : ctx->n_sm;
     grid = std::max<int64_t>(1, std::min<int64_t>(grid, W));
 #define MATKV_CASE(DD, GG) \
-    if (c.head_dim == DD && G == GG) return launch_stream_t<DD, GG>(p, (int)grid, stream);
+    if (c.head_dim == DD && G == GG) return launch_stream_t<DD, GG>(p, kn_map, vn_map, (int)grid, stream);
     MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)
     MATKV_CASE(64, 1) MATKV_CASE(64, 2) MATKV_CASE(64, 4) MATKV_CASE(64, 8)
 #undef MATKV_CASE
@@ -767,6 +774,10 @@ extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_
         p.part_o = (float *)((char *)base + kStaticCounterBytes + kStaticLseBytes);
         p.n_part_slots = kStaticParts; p.n_counter_slots = kStaticUnits;
         p.status = ctx->d_status;
+        CUtensorMap kn_map, vn_map;
+        rc = encode_new_rows_map(&kn_map, k_new, c.head_dim, c.n_kv_heads, (uint64_t)t->batch);
+        if (!rc) rc = encode_new_rows_map(&vn_map, v_new, c.head_dim, c.n_kv_heads, (uint64_t)t->batch);
+        if (rc) break;
         int64_t W = 0;
         for (int b = 0; b < t->batch; ++b)
             W += (int64_t)c.n_kv_heads * (t->h_reqs[b].chunk_tiles + ceil_div(t->tail_len_host, kTile) + 1);
@@ -775,7 +786,7 @@ extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_
         const int G = c.n_q_heads / c.n_kv_heads;
         rc = fail(MATKV_E_INVALID_ARG, "unsupported head_dim %d / group %d", c.head_dim, G);
 #define MATKV_CASE(DD, GG) \
-        if (c.head_dim == DD && G == GG) rc = launch_stream_t<DD, GG>(p, (int)grid, st);
+        if (c.head_dim == DD && G == GG) rc = launch_stream_t<DD, GG>(p, kn_map, vn_map, (int)grid, st);
         MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)
         MATKV_CASE(64, 1) MATKV_CASE(64, 2) MATKV_CASE(64, 4) MATKV_CASE(64, 8)
 #undef MATKV_CASE
