@@ -202,6 +202,13 @@ int matkv_gather_debug(matkv_ctx *ctx, matkv_table *table, int32_t layer, int32_
  * ceiling a decode launch is compared with.  No counterpart in the paper.  Asynchronous on `stream`. */
 int matkv_probe_read(matkv_ctx *ctx, const void *dev, size_t bytes, void *stream);
 
+/* ---- failure-detection self-test ------------------------------------------------------------ */
+/* Launches one thread that waits, with the kernels' bounded-wait logic, on a barrier nothing ever
+ * signals.  After `seconds` (0 < seconds <= 2) of SM clock the wait gives up, the kernel returns
+ * normally and the device status word reads MATKV_E_TIMEOUT (see matkv_status): the context stays
+ * usable.  No counterpart in the paper; it shows how a lost copy or a lost peer would surface.       */
+int matkv_selftest_wait_timeout(matkv_ctx *ctx, double seconds, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,7 @@ EXPORTS = [
     "matkv_stage_chunks_async", "matkv_stage_query", "matkv_stage_wait", "matkv_build_chunk_table",
     "matkv_table_free", "matkv_table_advance", "matkv_table_set_tail_len", "matkv_attend_prefill",
     "matkv_attend_decode", "matkv_attend_decode_all_layers", "matkv_lse_combine", "matkv_gather_debug",
-    "matkv_probe_read", "matkv_attend_decode_static",
+    "matkv_probe_read", "matkv_attend_decode_static", "matkv_selftest_wait_timeout",
 ]
 
 
@@ -77,6 +77,7 @@ def lib() -> C.CDLL:
             "matkv_gather_debug": (C.c_int, [vp, vp, i32, i32, vp, vp, i64, C.POINTER(i64), vp]),
             "matkv_probe_read": (C.c_int, [vp, vp, C.c_size_t, vp]),
             "matkv_attend_decode_static": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp]),
+            "matkv_selftest_wait_timeout": (C.c_int, [vp, C.c_double, vp]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -216,3 +217,7 @@ def matkv_attend_decode_static(ctx: int, table: int, layer: int, q: int, k_new: 
     an array built into the library (batch x n_kv_heads <= 256).  First call per device: outside any
     stream capture.  Calls must not overlap on the GPU (they share the array)."""
     _check(lib().matkv_attend_decode_static(ctx, table, layer, q, k_new, v_new, out, lse_out or None, stream or None))
+
+
+def matkv_selftest_wait_timeout(ctx: int, seconds: float = 0.2, stream: int = 0) -> None:
+    _check(lib().matkv_selftest_wait_timeout(ctx, seconds, stream or None))

@@ -797,6 +797,30 @@ extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_
 
 namespace matkv {
 
+// Self-test of the bounded wait: one thread waits on a barrier that nothing ever signals.  The wait must
+// give up after its limit, report MATKV_E_TIMEOUT through the status word and return normally.
+__global__ void k_wait_selftest(int32_t *status, long long limit_cycles) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const long long t0 = clock64();
+        bool done = false;
+        while (!done && clock64() - t0 <= limit_cycles) done = mbar_try_wait(smem_u32(&bar), 0);
+        if (!done) atomicCAS(status, 0, MATKV_E_TIMEOUT);
+    }
+}
+
+int launch_wait_selftest(matkv_ctx *ctx, double seconds, cudaStream_t stream) {
+    int khz = 0;
+    MATKV_CUDA(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, ctx->device));
+    k_wait_selftest<<<1, 32, 0, stream>>>(ctx->d_status, (long long)(seconds * 1e3 * khz));
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
 int launch_lse_combine(matkv_ctx *, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts, const float *lse_parts,
                        void *out, float *lse_out, cudaStream_t stream) {
     const int warps = 4;

@@ -730,6 +730,13 @@ int matkv_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D
     return launch_lse_combine(ctx, n_rows, n_parts, D, o_parts, lse_parts, out, lse_out, (cudaStream_t)stream);
 }
 
+int matkv_selftest_wait_timeout(matkv_ctx *ctx, double seconds, void *stream) {
+    if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_selftest_wait_timeout: null context");
+    if (!(seconds > 0.0) || seconds > 2.0) return fail(MATKV_E_INVALID_ARG, "matkv_selftest_wait_timeout: limit must be in (0, 2] seconds");
+    DeviceGuard guard(ctx->device);
+    return launch_wait_selftest(ctx, seconds, (cudaStream_t)stream);
+}
+
 int matkv_probe_read(matkv_ctx *ctx, const void *dev, size_t bytes, void *stream) {
     if (!ctx || !dev) return fail(MATKV_E_INVALID_ARG, "matkv_probe_read: null argument");
     if ((uintptr_t)dev % 16 || bytes < 16) return fail(MATKV_E_ALIGNMENT, "matkv_probe_read: buffer must be 16-byte aligned and non-empty");

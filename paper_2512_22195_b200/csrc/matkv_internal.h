@@ -146,6 +146,7 @@ int launch_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t 
                        const float *lse_parts, void *out, float *lse_out, cudaStream_t stream);
 int launch_gather(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out,
                   int64_t rows, cudaStream_t stream);
+int launch_wait_selftest(matkv_ctx *ctx, double seconds, cudaStream_t stream);
 int launch_read_probe(matkv_ctx *ctx, const void *dev, size_t bytes, cudaStream_t stream);
 int launch_add_tail_len(matkv_table *t, int32_t delta, int32_t set_value, bool set, cudaStream_t stream);
 

@@ -135,3 +135,28 @@ def test_device_generator_matches_host_generator():
     assert np.array_equal(to_bits(t), mi.normal_bf16(5, 77, 100003, 0, start=12345))
     gen.fill_bf16(t, seed=5, stream=78, shift=3, start=0)
     assert np.array_equal(to_bits(t), mi.normal_bf16(5, 78, 100003, 3))
+
+
+def test_bounded_wait_runs_out_and_reports_without_losing_the_context():
+    """Failure detection without a fault: a wait that nothing satisfies gives up after its limit and the
+    status word says so; the context keeps working afterwards."""
+    import time
+    mk, Session, to_dev, to_bits = _mk()
+    sess = Session(1, 8, 2, 64, 1, 1, 4)
+    assert sess.status() == 0
+    t0 = time.perf_counter()
+    mk.matkv_selftest_wait_timeout(sess.ctx, 0.25)
+    st = sess.status(clear=True)                      # synchronises
+    dt = time.perf_counter() - t0
+    assert st == mk.E_TIMEOUT
+    assert 0.1 < dt < 3.0, dt
+    assert sess.status() == 0
+    # the same context still computes
+    sess.register_device_chunk(0, rand_bits(44, 0, (1, 2, 2, 40, 64)))
+    sess.build_table([[0]])
+    q, kv = to_dev(rand_bits(44, 1, (1, 8, 64))), to_dev(rand_bits(44, 2, (1, 2, 64)))
+    out, _ = sess.decode(0, q, kv, kv)
+    assert torch.isfinite(out.float()).all() and sess.status() == 0
+    with pytest.raises(mk.MatkvError):
+        mk.matkv_selftest_wait_timeout(sess.ctx, 30.0)
+    sess.close()
