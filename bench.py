@@ -337,6 +337,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    import __graft_entry__ as ge
+    ge.build()                      # no-op when the in-tree libraries are up to date
     if args.workload == "cfg5":
         return run_pipeline(args)
     args.warmup = max(args.warmup, 3)
@@ -621,8 +623,8 @@ def main():
         # calibrate on one layer, then take as many layers and steps as fit ~12 s (work is linear in both)
         probe = OracleState(w, {c: dev_to_bits(chunks[c][0:1]) for c in needed}, ids, layers=[0])
         t_one = max(probe.decode_steps(0, 1), 1e-3)
-        n_l = int(max(1, min(L, 12.0 / t_one)))
-        n_s = int(max(1, min(T - 1, round(12.0 / (t_one * n_l)))))
+        n_l = int(max(1, min(L, 40.0 / t_one)))     # about 40 core-seconds of oracle work in all
+        n_s = int(max(1, min(T - 1, round(40.0 / (t_one * n_l)))))
         st_o = OracleState(w, {c: dev_to_bits(chunks[c][0:n_l]) for c in needed}, ids, layers=list(range(n_l)))
         t_s = st_o.decode_steps(0, n_s)
         per_step_full = t_s / n_s * (L / n_l)

@@ -24,3 +24,11 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Build the CUDA library, the generator twin and the oracle if they are missing or stale (nvcc
+    cross-compiles without a GPU; on a GPU machine this is a no-op when the libraries travelled with the tree)."""
+    import __graft_entry__ as ge
+    ge.build()
