@@ -78,7 +78,9 @@ typedef struct {
 /* options for matkv_set_option */
 #define MATKV_OPT_DECODE_CTAS   1  /* number of CTAs the streaming kernel splits the KV over; 0 = auto */
 #define MATKV_OPT_PREFILL_IMPL  2  /* 0 = auto (tensor-core tiles when the suffix is large enough),
-                                      1 = force the streaming kernel, 2 = force the tensor-core kernel */
+                                      1 = force the streaming kernel, 2 = force the tensor-core kernel,
+                                      3 = tensor-core kernel with two 128-row blocks per CTA whenever a
+                                          (request, KV head) has more than 128 query rows */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
 
 /* ---- context -------------------------------------------------------------------------- */

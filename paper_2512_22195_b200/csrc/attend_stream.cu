@@ -300,7 +300,7 @@ struct StreamCfg {
     static constexpr int BOX_BYTES = kTile * 128;          // one box: kTile rows x 128 bytes (swizzled)
     static constexpr int STAGE_BYTES = 2 * NBOX * BOX_BYTES;  // K boxes then V boxes
     static constexpr int KS = D / 16;                      // k-steps of S = Q K^T; also n-block pairs of O += P V
-    static constexpr int MERGE_BYTES = (kCW * kUnitRows * (D + 2) * 4 + 15) / 16 * 16;
+    static constexpr int MERGE_BYTES = (kCW * kUnitRows * (D + 3) * 4 + 15) / 16 * 16;
     static constexpr int FIXED_BYTES = MERGE_BYTES + 1024 + 1024;  // + misc + slack for 1024-byte alignment of the ring
     static constexpr int NSTAGE_MAX = (kMaxDynSmem - FIXED_BYTES) / STAGE_BYTES;
     static constexpr int NSTAGE = NSTAGE_MAX > 12 ? 12 : NSTAGE_MAX;
@@ -323,6 +323,7 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
     float *merge_o = (float *)(smem + C::NSTAGE * C::STAGE_BYTES);  // [warp][row][D]
     float *merge_m = merge_o + kCW * kUnitRows * D;                 // [warp][row]  (log2 units, scaled)
     float *merge_l = merge_m + kCW * kUnitRows;                     // [warp][row]
+    float *merge_r = merge_l + kCW * kUnitRows;                     // [warp][row]  sum of the rounded numerators
     unsigned char *misc = smem + C::NSTAGE * C::STAGE_BYTES + C::MERGE_BYTES;
     uint64_t *bars = (uint64_t *)misc;                              // full[NSTAGE], empty[NSTAGE]
     // per stage tag: valid rows | kTagNew | (number of the stage's current fill) << 16
@@ -434,7 +435,10 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
 
     uint32_t qa[C::KS][2];   // A fragments of Q for the real rows: [k-step][cols 0-7 | cols 8-15]
     float o[2 * C::KS][4];   // O accumulators: [8-column block of d][c0, c1 real row; c2, c3 padding rows]
-    float m_run = -CUDART_INF_F, l_run = 0.f;  // running max (scaled, log2 units) and this thread's share of the sum
+    // running max (scaled, log2 units), this thread's share of the sum of the numerators (for the log-sum-exp)
+    // and of the sum of their bf16 roundings (what the tensor core multiplies with V: O is normalised by it,
+    // so that a dominant token's rounding error cancels)
+    float m_run = -CUDART_INF_F, l_run = 0.f, l_rnd = 0.f;
 
     UnitPos u = range->first;
     int64_t f_unit = f_begin;   // flat index of this CTA's first tile inside the current unit
@@ -460,6 +464,7 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
             for (int nb = 0; nb < 2 * C::KS; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
             m_run = -CUDART_INF_F;
             l_run = 0.f;
+            l_rnd = 0.f;
         }
         // ---- this warp's work items of the unit ----
         // CTA-local tile j = j_base + (t - t_begin) splits into kItems work items hj = j*kItems + piece;
@@ -510,7 +515,9 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                 const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);
                 const float p0 = fast_exp2(x0 - m_use), p1 = fast_exp2(x1 - m_use);
                 const float p2 = fast_exp2(x2 - m_use), p3 = fast_exp2(x3 - m_use);
+                const uint32_t pa0 = pack_bf16(p0, p1), pa2 = pack_bf16(p2, p3);
                 l_run = l_run * alpha + ((p0 + p1) + (p2 + p3));
+                l_rnd = l_rnd * alpha + ((bf_lo(pa0) + bf_hi(pa0)) + (bf_lo(pa2) + bf_hi(pa2)));
                 m_run = m_new;
                 if (__any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll
@@ -519,7 +526,6 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                         o[nb][1] *= alpha;
                     }
                 }
-                const uint32_t pa0 = pack_bf16(p0, p1), pa2 = pack_bf16(p2, p3);
                 // ---------- O += P V ----------
                 const uint32_t v_u32 = stage_u32 + C::NBOX * C::BOX_BYTES;
 #pragma unroll
@@ -554,15 +560,18 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
 
         // ---- end of this CTA's share of the unit: merge the warps' states ----
         {
-            float l_tot = l_run;
+            float l_tot = l_run, r_tot = l_rnd;
             l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
             l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
+            r_tot += __shfl_xor_sync(0xffffffffu, r_tot, 1);
+            r_tot += __shfl_xor_sync(0xffffffffu, r_tot, 2);
 #pragma unroll
             for (int nb = 0; nb < 2 * C::KS; ++nb)
                 *(float2 *)(merge_o + (warp * kUnitRows + qr) * D + nb * 8 + 2 * qc) = make_float2(o[nb][0], o[nb][1]);
             if (qc == 0) {
                 merge_m[warp * kUnitRows + qr] = m_run;
                 merge_l[warp * kUnitRows + qr] = l_tot;
+                merge_r[warp * kUnitRows + qr] = r_tot;
             }
         }
         consumer_bar();
@@ -579,15 +588,16 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
             float M = -CUDART_INF_F;
 #pragma unroll
             for (int w = 0; w < kCW; ++w) M = fmaxf(M, merge_m[w * kUnitRows + r]);
-            float acc = 0.f, L = 0.f;
+            float acc = 0.f, L = 0.f, Lr = 0.f;
 #pragma unroll
             for (int w = 0; w < kCW; ++w) {
                 const float mw = merge_m[w * kUnitRows + r];
                 const float sw = mw == -CUDART_INF_F ? 0.f : fast_exp2(mw - M);
                 acc = fmaf(sw, merge_o[(w * kUnitRows + r) * D + d], acc);
                 L = fmaf(sw, merge_l[w * kUnitRows + r], L);
+                Lr = fmaf(sw, merge_r[w * kUnitRows + r], Lr);
             }
-            const float ov = acc / L;
+            const float ov = acc / Lr;
             const float lse = (M + log2f(L)) * kLn2;
             if (n_parts == 1) {
                 p.out[q_base + (int64_t)(r / G) * p.q_ss + (r % G) * D + d] = __float2bfloat16(ov);

@@ -242,7 +242,7 @@ int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
             ctx->opt_decode_ctas = value;
             return MATKV_OK;
         case MATKV_OPT_PREFILL_IMPL:
-            if (value < 0 || value > 2) return fail(MATKV_E_INVALID_ARG, "prefill impl must be 0, 1 or 2");
+            if (value < 0 || value > 3) return fail(MATKV_E_INVALID_ARG, "prefill impl must be 0..3");
             ctx->opt_prefill_impl = value;
             return MATKV_OK;
         case MATKV_OPT_PREFILL_CTAS:
@@ -715,7 +715,7 @@ int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t 
     }
     // long suffixes go to the tcgen05 tile kernel, short ones stay on the streaming kernel
     const int G = c.n_q_heads / c.n_kv_heads;
-    const bool tensor_core = ctx->opt_prefill_impl == 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
+    const bool tensor_core = ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
     if (tensor_core) return launch_prefill_tc(ctx, t, a, (cudaStream_t)stream);
     return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
 }

@@ -1,18 +1,21 @@
 // K3: query sub-prefill over the chunk table on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
-// One CTA = (request, KV head, block of 128 query rows, KV split).  A query row is (suffix token,
-// head of the KV group), row = token * G + head, so the G heads that share a KV head and up to 128/G
-// suffix tokens share every K/V tile that is fetched.  Per 64-token KV tile:
+// One CTA = (request, KV head, NBLK blocks of 128 query rows, KV split).  A query row is (suffix token,
+// head of the KV group), row = token * G + head, so the G heads that share a KV head and up to
+// NBLK*128/G suffix tokens share every K/V tile that is fetched.  Per 64-token KV tile and row block:
 //     S  = Q K^T      tcgen05.mma  M=128, N=64,  K=D   (both operands K-major, 128-byte swizzle)  -> TMEM
-//     P  = online softmax of S (one thread per row: tcgen05.ld, fp32, exp2-based) -> bf16 in smem
-//     Ot = P V        tcgen05.mma  M=128, N=D,   K=64  (V is MN-major straight from its [token][d] tile) -> TMEM
-//     O  = O * alpha + Ot   in registers of the row's thread (tcgen05.ld), so TMEM is never read-modified
-// Warp roles: warp 0 producer (TMA tensor copies of chunk / tail tiles through the table's descriptors;
-// the call's new tokens are copied by hand into the same swizzled layout and appended to the tail),
-// warp 1 issues the MMAs and owns the TMEM allocation, warps 2-5 are the 128 softmax threads.
-// S and Ot are double-buffered in TMEM (2 x 64 + 2 x D columns) so that the tensor core works on tile
-// j+1 while the softmax threads work on tile j.  Every wait is bounded and reports through the status
-// word; TMEM is always released.
+//     P  = softmax numerators of S (one thread per row: tcgen05.ld, fp32, exp2-based) -> bf16 in smem
+//     O += P V        tcgen05.mma  M=128, N=D,   K=64  (V is MN-major straight from its [token][d] tile),
+//                     accumulated in TMEM across the tiles
+// The exponent's reference maximum of a row only moves when the running maximum has grown by more than
+// 2^8 (lazy rescale): then the row's thread multiplies its O row in TMEM (tcgen05.ld / tcgen05.st) and
+// its running sum by the same factor, so numerators stay below 2^8 and O, l stay consistent.
+// Warp roles: warp 0 producer (TMA tensor copies of chunk / tail tiles through the table's descriptors,
+// of the call's new tokens through a per-call descriptor; appends the new tokens to the tail), warp 1
+// issues the MMAs and owns the TMEM allocation, then four softmax warps per row block.  S is
+// double-buffered in TMEM so that the tensor core works on tile j+1 while the softmax threads work on
+// tile j; with two row blocks two softmax warps share each SM sub-partition.  Every wait is bounded and
+// reports through the status word; TMEM is always released.
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <math_constants.h>
@@ -142,6 +145,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// multiply 32 consecutive fp32 columns of this thread's TMEM lane by `f` (load, scale, store back)
+__device__ __forceinline__ void tmem_scale32(uint32_t taddr, float f) {
+    float v[32];
+    tmem_ld32(taddr, v);
+    uint32_t r[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i] * f);
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+        "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
+        "r"(r[31])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -153,38 +173,46 @@ struct Tile {
     int kind, seg, r0, rows, seg_len;
 };
 
-template <int D>
+template <int D, int NBLK>
 struct Cfg {
     static constexpr int NBOX = D / 64;
     static constexpr int BOX_BYTES = kTile * 128;        // 64 rows x 128 bytes
     static constexpr int KV_BYTES = NBOX * BOX_BYTES;    // K (or V) of one tile
     static constexpr int STAGE_BYTES = 2 * KV_BYTES;
-    static constexpr int Q_BYTES = NBOX * kRowsPerCta * 128;
-    static constexpr int P_BYTES = kRowsPerCta * 128;    // 128 rows x 64 tokens bf16
-    static constexpr int SMEM_BYTES = 1024 + Q_BYTES + 2 * P_BYTES + kStages * STAGE_BYTES + 512;
-    static constexpr int COL_S = 0, COL_O = 128;         // TMEM columns: S[2] at 0, 64; Ot[2] at 128, 128 + D
-    static constexpr int TMEM_COLS = 512;
+    static constexpr int QBLK_BYTES = NBOX * kRowsPerCta * 128;   // Q of one row block
+    static constexpr int P_BYTES = kRowsPerCta * 128;             // 128 rows x 64 tokens bf16
+    static constexpr int STAGES = NBLK == 2 ? 3 : 4;
+    static constexpr int THREADS = (2 + 4 * NBLK) * 32;           // producer warp, MMA warp, 4 softmax warps per block
+    static constexpr int SMEM_BYTES = 1024 + NBLK * QBLK_BYTES + NBLK * 2 * P_BYTES + STAGES * STAGE_BYTES + 512;
+    // TMEM columns of row block b: S[2] at b*256 + {0, 64}; O at b*256 + 128 (D columns)
+    static constexpr int COL_BLK = 256, COL_O = 128;
+    static constexpr int TMEM_COLS = NBLK == 2 ? 512 : 256;
+    static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 };
 
-template <int D, int G>
-__global__ void __launch_bounds__(kThreads, 1)
+// barrier slots (8 bytes each)
+constexpr int kBarFull = 0, kBarEmpty = 4, kBarSFull = 8 /* [blk][2] */, kBarPReady = 12 /* [blk][2] */,
+              kBarODone = 16 /* [blk] */, kBarQReady = 18, kBarCount = 20;
+
+template <int D, int G, int NBLK>
+__global__ void __launch_bounds__((2 + 4 * NBLK) * 32, 1)
 k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap kn_map, const __grid_constant__ CUtensorMap vn_map) {
-    using C = Cfg<D>;
+    using C = Cfg<D, NBLK>;
+    constexpr int kStages = C::STAGES;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    unsigned char *q_s = smem;                                   // NBOX boxes [128 rows][128 B]
-    unsigned char *p_s = q_s + C::Q_BYTES;                       // 2 x [128 rows][128 B]
-    unsigned char *kv_s = p_s + 2 * C::P_BYTES;                  // kStages x (K boxes, V boxes)
+    unsigned char *q_s = smem;                                   // [NBLK][NBOX boxes][128 rows][128 B]
+    unsigned char *p_s = q_s + NBLK * C::QBLK_BYTES;             // [NBLK][2][128 rows][128 B]
+    unsigned char *kv_s = p_s + NBLK * 2 * C::P_BYTES;           // kStages x (K boxes, V boxes)
     uint64_t *bars = (uint64_t *)(kv_s + kStages * C::STAGE_BYTES);
-    // barriers: full_kv[4], empty_kv[4], s_full[2], p_ready[2], o_full[2], o_free[2], q_ready
-    uint32_t *tmem_slot = (uint32_t *)(bars + 20);
+    uint32_t *tmem_slot = (uint32_t *)(bars + kBarCount);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 2);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // which unit
     int c = blockIdx.x;
     const int sp = c % p.n_split; c /= p.n_split;
-    const int rb = c % p.n_rb; c /= p.n_rb;
+    const int rb = c % p.n_rb; c /= p.n_rb;                      // index of this CTA's group of NBLK row blocks
     const int g = c % p.Hkv;
     const int b = c / p.Hkv;
     const DevReq rq = p.reqs[b];
@@ -198,28 +226,26 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
     const int t_begin = (int)((int64_t)sp * T / p.n_split), t_end = (int)((int64_t)(sp + 1) * T / p.n_split);
     const int n_tiles = t_end - t_begin;
     const int R = p.S * G;                       // query rows of the (request, KV head)
-    const int row0 = rb * kRowsPerCta;
+    const int row0 = rb * NBLK * kRowsPerCta;
 
     const uint32_t bar0 = smem_u32(bars);
-    const uint32_t full_kv = bar0, empty_kv = bar0 + 4 * 8, s_full = bar0 + 8 * 8, p_ready = bar0 + 10 * 8,
-                   o_full = bar0 + 12 * 8, o_free = bar0 + 14 * 8, q_ready = bar0 + 16 * 8;
+    const uint32_t full_kv = bar0 + kBarFull * 8, empty_kv = bar0 + kBarEmpty * 8, s_full = bar0 + kBarSFull * 8,
+                   p_ready = bar0 + kBarPReady * 8, o_done = bar0 + kBarODone * 8, q_ready = bar0 + kBarQReady * 8;
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < 4; ++s) {
             mbar_init(full_kv + s * 8, 1);
             mbar_init(empty_kv + s * 8, 1);
-        }
-        for (int s = 0; s < 2; ++s) {
             mbar_init(s_full + s * 8, 1);
             mbar_init(p_ready + s * 8, 128);
-            mbar_init(o_full + s * 8, 1);
-            mbar_init(o_free + s * 8, 128);
         }
-        mbar_init(q_ready, 128);
+        mbar_init(o_done, 1);
+        mbar_init(o_done + 8, 1);
+        mbar_init(q_ready, 128 * NBLK);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
-    if (warp == 1) {  // TMEM: all 512 columns (one CTA per SM)
+    if (warp == 1) {  // TMEM (one CTA per SM)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"((uint32_t)C::TMEM_COLS)
                      : "memory");
@@ -295,7 +321,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 }
             }
             // append this split's share of the new tokens to the tail for later calls (the splits of row
-            // block 0 divide the S tokens among themselves), once the CTA's first loads are in flight
+            // group 0 divide the S tokens among themselves), once the CTA's first loads are in flight
             if (j == 0 && rb == 0) {
                 constexpr int CPR = D / 8;
                 const int a0 = (int)((int64_t)sp * p.S / p.n_split), a1 = (int)((int64_t)(sp + 1) * p.S / p.n_split);
@@ -318,17 +344,19 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             constexpr uint32_t idesc_pv = instr_desc(kRowsPerCta, D, true);
             const uint32_t q_u32 = smem_u32(q_s), p_u32 = smem_u32(p_s), kv_u32 = smem_u32(kv_s);
             bool ok = mbar_wait(q_ready, 0, abort_flag);
-            auto do_pv = [&](int t) {
-                const int bf = t & 1, use = t >> 1, st = t % kStages;
-                if (!mbar_wait(p_ready + bf * 8, use & 1, abort_flag)) return false;
-                if (use > 0 && !mbar_wait(o_free + bf * 8, (use - 1) & 1, abort_flag)) return false;
-                tc_fence_after();
+            auto do_pv = [&](int t) {  // O[blk] += P(t, blk) V(t) for every row block, then free the K/V stage
+                const int bf = t & 1, st = t % kStages;
                 const uint32_t v_u32 = kv_u32 + st * C::STAGE_BYTES + C::KV_BYTES;
 #pragma unroll
-                for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA
-                    umma(tmem + C::COL_O + bf * D, smem_desc(p_u32 + bf * C::P_BYTES + ks * 32, 0, 1024),
-                         smem_desc(v_u32 + ks * 2048, C::BOX_BYTES, 1024), idesc_pv, ks > 0);
-                umma_commit(o_full + bf * 8);
+                for (int blk = 0; blk < NBLK; ++blk) {
+                    if (!mbar_wait(p_ready + (blk * 2 + bf) * 8, (t >> 1) & 1, abort_flag)) return false;
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA
+                        umma(tmem + blk * C::COL_BLK + C::COL_O, smem_desc(p_u32 + (blk * 2 + bf) * C::P_BYTES + ks * 32, 0, 1024),
+                             smem_desc(v_u32 + ks * 2048, C::BOX_BYTES, 1024), idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+                    umma_commit(o_done + blk * 8);
+                }
                 umma_commit(empty_kv + st * 8);  // K and V of the tile are free once these MMAs have run
                 return true;
             };
@@ -339,85 +367,98 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 tc_fence_after();
                 const uint32_t k_u32 = kv_u32 + st * C::STAGE_BYTES;
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
-                    umma(tmem + C::COL_S + (j & 1) * kTile,
-                         smem_desc(q_u32 + (ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32, 0, 1024),
-                         smem_desc(k_u32 + (ks / 4) * C::BOX_BYTES + (ks % 4) * 32, 0, 1024), idesc_qk, ks > 0);
-                umma_commit(s_full + (j & 1) * 8);
+                for (int blk = 0; blk < NBLK; ++blk) {
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
+                        umma(tmem + blk * C::COL_BLK + (j & 1) * kTile,
+                             smem_desc(q_u32 + blk * C::QBLK_BYTES + (ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32, 0, 1024),
+                             smem_desc(k_u32 + (ks / 4) * C::BOX_BYTES + (ks % 4) * 32, 0, 1024), idesc_qk, ks > 0);
+                    umma_commit(s_full + (blk * 2 + (j & 1)) * 8);
+                }
                 if (j >= 1) ok = do_pv(j - 1);
             }
             if (ok && n_tiles > 0) do_pv(n_tiles - 1);
         }
     } else {
         // ===================== softmax threads: one query row each =====================
-        const int r = (warp & 3) * 32 + lane;        // TMEM lane = row inside the CTA's block
-        const int grow = row0 + r;                   // row inside the (request, KV head)
+        const int blk = (warp - 2) >> 2;                      // row block of this warp
+        const int r = (warp & 3) * 32 + lane;                 // TMEM lane = row inside the block
+        const int grow = row0 + blk * kRowsPerCta + r;        // row inside the (request, KV head)
         const bool real = grow < R;
-        const int tok = grow / G, hd = grow % G;     // suffix token and head of the group
-        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const int tok = grow / G, hd = grow % G;              // suffix token and head of the group
+        const uint32_t lane_base = tmem + blk * C::COL_BLK + ((uint32_t)((warp & 3) * 32) << 16);
         // Q row -> swizzled smem (zeros for rows past R)
         {
             const __nv_bfloat16 *qrow = p.q + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D;
+            unsigned char *qb = q_s + blk * C::QBLK_BYTES;
 #pragma unroll
             for (int ch = 0; ch < D / 8; ++ch) {
                 const uint4 v = real ? *(const uint4 *)(qrow + ch * 8) : make_uint4(0, 0, 0, 0);
-                *(uint4 *)(q_s + (ch / 8) * (kRowsPerCta * 128) + r * 128 + (((ch % 8) ^ (r & 7)) << 4)) = v;
+                *(uint4 *)(qb + (ch / 8) * (kRowsPerCta * 128) + r * 128 + (((ch % 8) ^ (r & 7)) << 4)) = v;
             }
             fence_async_smem();
             mbar_arrive(q_ready);
         }
-        float o[D];
-#pragma unroll
-        for (int d = 0; d < D; ++d) o[d] = 0.f;
-        float m_run = -CUDART_INF_F, l_run = 0.f, alpha_prev = 1.f;
+        // m_ref: the maximum the exponents refer to (log2 units, scaled); it trails the true running maximum by
+        // at most 8, so numerators stay below 2^8.  l_run: sum of the numerators relative to m_ref.
+        // l_rnd: the same sum over the bf16-rounded numerators the tensor core really multiplies with V; O is
+        // normalised by it (a dominant token's rounding error then cancels), the log-sum-exp uses l_run.
+        float m_ref = -CUDART_INF_F, l_run = 0.f, l_rnd = 0.f;
         int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
         bool ok = true;
-        auto take_o = [&](int t) {  // O = O * alpha(t) + Ot(t)
-            const int bf = t & 1;
-            if (!mbar_wait(o_full + bf * 8, (t >> 1) & 1, abort_flag)) return false;
-            tc_fence_after();
-#pragma unroll
-            for (int c0 = 0; c0 < D; c0 += 32) {
-                float v[32];
-                tmem_ld32(lane_base + C::COL_O + bf * D + c0, v);
-#pragma unroll
-                for (int i = 0; i < 32; ++i) o[c0 + i] = fmaf(o[c0 + i], alpha_prev, v[i]);
-            }
-            tc_fence_before();
-            mbar_arrive(o_free + bf * 8);
-            return true;
-        };
         for (int j = 0; j < n_tiles && ok; ++j) {
             const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len);
             const int bf = j & 1;
-            ok = mbar_wait(s_full + bf * 8, (j >> 1) & 1, abort_flag);
+            ok = mbar_wait(s_full + (blk * 2 + bf) * 8, (j >> 1) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);   // the TMEM loads below are warp-collective
             if (!ok) break;
             tc_fence_after();
             float s[kTile];
             {
                 float v[32];
-                tmem_ld32(lane_base + C::COL_S + bf * kTile, v);
+                tmem_ld32(lane_base + bf * kTile, v);
 #pragma unroll
                 for (int i = 0; i < 32; ++i) s[i] = v[i];
-                tmem_ld32(lane_base + C::COL_S + bf * kTile + 32, v);
+                tmem_ld32(lane_base + bf * kTile + 32, v);
 #pragma unroll
                 for (int i = 0; i < 32; ++i) s[32 + i] = v[i];
             }
             // visible columns: all valid rows of a chunk / tail tile; causal inside the new tokens
             int n_vis = ti.rows;
             if (ti.kind == 2) n_vis = min(ti.rows, tok - ti.r0 + 1);
-            if (!real) n_vis = min(n_vis, 1);
             float tmax = -CUDART_INF_F;
 #pragma unroll
             for (int i = 0; i < kTile; ++i) {
                 s[i] = i < n_vis ? s[i] * p.scale_log2 : -CUDART_INF_F;
                 tmax = fmaxf(tmax, s[i]);
             }
-            const float m_new = fmaxf(m_run, tmax);
-            const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);
-            const float m_use = m_new == -CUDART_INF_F ? 0.f : m_new;
-            float psum = 0.f;
-            unsigned char *prow = p_s + bf * C::P_BYTES + r * 128;
+            // lazy rescale: move the reference only when the maximum has grown by more than 2^8
+            const bool grow_ref = tmax > m_ref + 8.0f;   // also true for the first visible column (m_ref = -inf)
+            // Every thread consumes every phase of o_done in order (P V of tile j-1 during tile j): a one-bit
+            // phase can only be told apart from its neighbours, never from a phase two steps away.
+            bool pv_prev_done = j == 0;
+            if (__any_sync(0xffffffffu, grow_ref)) {     // tcgen05.ld / st are warp-collective: decide per warp
+                const float alpha = grow_ref ? (m_ref == -CUDART_INF_F ? 0.f : fast_exp2(m_ref - tmax)) : 1.f;
+                if (j > 0) {
+                    // O of tiles 0..j-1 must be complete before it is scaled
+                    ok = mbar_wait(o_done + blk * 8, (j - 1) & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    pv_prev_done = true;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c0 = 0; c0 < D; c0 += 32) tmem_scale32(lane_base + C::COL_O + c0, alpha);
+                    tc_fence_before();
+                }
+                if (grow_ref) {
+                    l_run *= alpha;
+                    l_rnd *= alpha;
+                    m_ref = tmax;
+                }
+            }
+            const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
+            float psum = 0.f, prnd = 0.f;
+            unsigned char *prow = p_s + (blk * 2 + bf) * C::P_BYTES + r * 128;
 #pragma unroll
             for (int ch = 0; ch < kTile / 8; ++ch) {
                 float e[8];
@@ -426,37 +467,60 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     e[i] = fast_exp2(s[ch * 8 + i] - m_use);
                     psum += e[i];
                 }
-                *(uint4 *)(prow + ((ch ^ (r & 7)) << 4)) =
-                    make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7]));
+                const uint4 pk = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7]));
+                prnd += (__uint_as_float(pk.x << 16) + __uint_as_float(pk.x & 0xffff0000u)) +
+                        (__uint_as_float(pk.y << 16) + __uint_as_float(pk.y & 0xffff0000u)) +
+                        (__uint_as_float(pk.z << 16) + __uint_as_float(pk.z & 0xffff0000u)) +
+                        (__uint_as_float(pk.w << 16) + __uint_as_float(pk.w & 0xffff0000u));
+                *(uint4 *)(prow + ((ch ^ (r & 7)) << 4)) = pk;
             }
-            l_run = l_run * alpha + psum;
-            m_run = m_new;
+            l_run += psum;
+            l_rnd += prnd;
+            if (!pv_prev_done) {  // normally long since complete: the wait only keeps the phase count in step
+                ok = mbar_wait(o_done + blk * 8, (j - 1) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+            }
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(p_ready + bf * 8);
-            if (j >= 1) ok = take_o(j - 1);
-            alpha_prev = alpha;
+            mbar_arrive(p_ready + (blk * 2 + bf) * 8);
         }
-        if (ok && n_tiles > 0) ok = take_o(n_tiles - 1);
-        // epilogue
-        if (ok && real) {
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            const float lse = l_run > 0.f ? (m_run + log2f(l_run)) * kLn2 : -CUDART_INF_F;
+        // epilogue: O is complete once the last P V has run
+        if (ok && n_tiles > 0) {
+            ok = mbar_wait(o_done + blk * 8, (n_tiles - 1) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv = l_rnd > 0.f ? 1.f / l_rnd : 0.f;
+            const float lse = l_run > 0.f ? (m_ref + log2f(l_run)) * kLn2 : -CUDART_INF_F;
             const int64_t orow = ((int64_t)b * p.S + tok) * p.Hq + g * G + hd;
-            if (p.n_split == 1) {
-                __nv_bfloat16 *dst = p.out + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D;
 #pragma unroll
-                for (int ch = 0; ch < D / 8; ++ch)
-                    *(uint4 *)(dst + ch * 8) =
-                        make_uint4(pack_bf16(o[ch * 8] * inv, o[ch * 8 + 1] * inv), pack_bf16(o[ch * 8 + 2] * inv, o[ch * 8 + 3] * inv),
-                                   pack_bf16(o[ch * 8 + 4] * inv, o[ch * 8 + 5] * inv), pack_bf16(o[ch * 8 + 6] * inv, o[ch * 8 + 7] * inv));
-                if (p.lse_out) p.lse_out[orow] = lse;
-            } else {
-                float *dst = p.part_o + (orow * p.n_split + sp) * D;
+            for (int c0 = 0; c0 < D; c0 += 32) {
+                float v[32];
+                tmem_ld32(lane_base + C::COL_O + c0, v);   // warp-collective: every lane loads, real rows store
+                if (real) {
+                    if (p.n_split == 1) {
+                        __nv_bfloat16 *dst = p.out + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D + c0;
 #pragma unroll
-                for (int ch = 0; ch < D / 4; ++ch)
-                    *(float4 *)(dst + ch * 4) = make_float4(o[ch * 4] * inv, o[ch * 4 + 1] * inv, o[ch * 4 + 2] * inv, o[ch * 4 + 3] * inv);
-                p.part_lse[orow * p.n_split + sp] = lse;
+                        for (int ch = 0; ch < 4; ++ch)
+                            *(uint4 *)(dst + ch * 8) = make_uint4(
+                                pack_bf16(v[ch * 8] * inv, v[ch * 8 + 1] * inv), pack_bf16(v[ch * 8 + 2] * inv, v[ch * 8 + 3] * inv),
+                                pack_bf16(v[ch * 8 + 4] * inv, v[ch * 8 + 5] * inv), pack_bf16(v[ch * 8 + 6] * inv, v[ch * 8 + 7] * inv));
+                    } else {
+                        float *dst = p.part_o + (orow * p.n_split + sp) * D + c0;
+#pragma unroll
+                        for (int ch = 0; ch < 8; ++ch)
+                            *(float4 *)(dst + ch * 4) = make_float4(v[ch * 4] * inv, v[ch * 4 + 1] * inv, v[ch * 4 + 2] * inv, v[ch * 4 + 3] * inv);
+                    }
+                }
+            }
+            if (real) {
+                if (p.n_split == 1) {
+                    if (p.lse_out) p.lse_out[orow] = lse;
+                } else {
+                    p.part_lse[orow * p.n_split + sp] = lse;
+                }
             }
         }
     }
@@ -472,15 +536,15 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
 
 }  // namespace k3
 
-template <int D, int G>
+template <int D, int G, int NBLK>
 static int launch_k3(const k3::Params &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
-    using C = k3::Cfg<D>;
+    using C = k3::Cfg<D, NBLK>;
     static bool configured = false;
     if (!configured) {
-        MATKV_CUDA(cudaFuncSetAttribute(k3::k_prefill_tc<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        MATKV_CUDA(cudaFuncSetAttribute(k3::k_prefill_tc<D, G, NBLK>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
         configured = true;
     }
-    k3::k_prefill_tc<D, G><<<grid, k3::kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
+    k3::k_prefill_tc<D, G, NBLK><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());
     return MATKV_OK;
 }
@@ -495,7 +559,12 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     p.q_sb = a.q_sb; p.q_ss = a.q_ss; p.kn_sb = a.kn_sb; p.kn_ss = a.kn_ss;
     p.layer = a.layer0; p.n_layers_total = c.n_layers; p.B = t->batch; p.S = a.S; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads;
     p.max_tail = c.max_tail_tokens;
-    p.n_rb = (a.S * G + k3::kRowsPerCta - 1) / k3::kRowsPerCta;
+    // two row blocks per CTA when the (request, KV head) has more than 128 query rows and there are still
+    // enough CTAs to fill most of the SMs (otherwise one block per CTA and more KV splits)
+    const int R = a.S * G;
+    const bool fill = (int64_t)t->batch * c.n_kv_heads * ((R + 255) / 256) * 10 >= 6 * (int64_t)ctx->n_sm;
+    const int nblk = (R > k3::kRowsPerCta && (fill || ctx->opt_prefill_impl == 3)) ? 2 : 1;
+    p.n_rb = (a.S * G + nblk * k3::kRowsPerCta - 1) / (nblk * k3::kRowsPerCta);
     p.scale_log2 = ctx->scale * k3::kLog2e;
     p.status = ctx->d_status;
     // KV splits: fill the SMs, never more splits than the shortest request has tiles, and only as many
@@ -524,7 +593,7 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     }
     int rc = fail(MATKV_E_INVALID_ARG, "tensor-core prefill: unsupported head_dim %d / group %d", D, G);
 #define MATKV_CASE(DD, GG) \
-    if (D == DD && G == GG) rc = launch_k3<DD, GG>(p, kn_map, vn_map, (int)grid, stream);
+    if (D == DD && G == GG) rc = nblk == 2 ? launch_k3<DD, GG, 2>(p, kn_map, vn_map, (int)grid, stream) : launch_k3<DD, GG, 1>(p, kn_map, vn_map, (int)grid, stream);
     MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)
     MATKV_CASE(64, 1) MATKV_CASE(64, 2) MATKV_CASE(64, 4) MATKV_CASE(64, 8)
 #undef MATKV_CASE

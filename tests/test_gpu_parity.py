@@ -243,6 +243,26 @@ def test_prefill_tensor_core_kernel(Hq, Hkv, D, lens, S):
     run_requests(2, Hq, Hkv, D, lens, S, 3, seed=41, prefill_impl=2)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,lens,S,splits", [
+    (32, 8, 128, [[300, 77], [129]], 40, 0),      # 160 rows: second block partly empty
+    (64, 8, 128, [[200, 64]], 70, 3),             # G = 8, 560 rows: three CTAs of two blocks, KV splits
+    (8, 2, 64, [[100]], 130, 2),                  # D = 64, 520 rows, three new-token tiles
+    (16, 1, 128, [[64], []], 17, 1),              # G = 16 is not supported -> use G = 8 below
+])
+def test_prefill_tensor_core_two_row_blocks(Hq, Hkv, D, lens, S, splits):
+    if Hq // Hkv > 8:
+        Hq = 8 * Hkv
+    run_requests(1, Hq, Hkv, D, lens, S, 2, seed=45, prefill_impl=3, prefill_ctas=splits)
+
+
+@pytest.mark.parametrize("impl", [2, 3])
+def test_prefill_tensor_core_peaky_queries_rescale_in_tmem(impl):
+    """q scaled by 8: the running maximum jumps by far more than 2^8 between tiles, so the O rows are
+    rescaled in tensor memory several times per row."""
+    run_requests(1, 32, 8, 128, [[500, 300, 64]], 40, 2, seed=46, prefill_impl=impl, q_shift=3)
+    run_requests(1, 8, 2, 64, [[129, 64]], 70, 1, seed=47, prefill_impl=impl, q_shift=3, prefill_ctas=1)
+
+
 @pytest.mark.parametrize("splits", [1, 2, 5])
 def test_prefill_tensor_core_split_invariance(splits):
     run_requests(1, 32, 8, 128, [[700, 260, 64]], 24, 2, seed=42, prefill_impl=2, prefill_ctas=splits)
