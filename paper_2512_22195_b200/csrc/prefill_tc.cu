@@ -145,6 +145,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {  // two fp32 adds in one instruction (sm_100)
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;"
+        : "=l"(d)
+        : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)));
+    return *reinterpret_cast<float2 *>(&d);
+}
 // multiply 32 consecutive fp32 columns of this thread's TMEM lane by `f` (load, scale, store back)
 __device__ __forceinline__ void tmem_scale32(uint32_t taddr, float f) {
     float v[32];
@@ -423,15 +430,18 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
 #pragma unroll
                 for (int i = 0; i < 32; ++i) s[32 + i] = v[i];
             }
-            // visible columns: all valid rows of a chunk / tail tile; causal inside the new tokens
+            // visible columns: all valid rows of a chunk / tail tile; causal inside the new tokens.
+            // Scores stay raw (unscaled) here: the scale is folded into the exponent's FMA below.
             int n_vis = ti.rows;
             if (ti.kind == 2) n_vis = min(ti.rows, tok - ti.r0 + 1);
+            if (n_vis < kTile) {  // ragged or causal tile: mask (a full tile skips this)
+#pragma unroll
+                for (int i = 0; i < kTile; ++i) s[i] = i < n_vis ? s[i] : -CUDART_INF_F;
+            }
             float tmax = -CUDART_INF_F;
 #pragma unroll
-            for (int i = 0; i < kTile; ++i) {
-                s[i] = i < n_vis ? s[i] * p.scale_log2 : -CUDART_INF_F;
-                tmax = fmaxf(tmax, s[i]);
-            }
+            for (int i = 0; i < kTile; ++i) tmax = fmaxf(tmax, s[i]);
+            tmax *= p.scale_log2;   // the scale is positive: the maximum commutes with it
             // lazy rescale: move the reference only when the maximum has grown by more than 2^8
             const bool grow_ref = tmax > m_ref + 8.0f;   // also true for the first visible column (m_ref = -inf)
             // Every thread consumes every phase of o_done in order (P V of tile j-1 during tile j): a one-bit
@@ -456,24 +466,23 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     m_ref = tmax;
                 }
             }
-            const float m_use = m_ref == -CUDART_INF_F ? 0.f : m_ref;
-            float psum = 0.f, prnd = 0.f;
+            const float m_neg = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
+            float2 psum2 = make_float2(0.f, 0.f), prnd2 = make_float2(0.f, 0.f);  // packed fp32 pairs: half the adds
             unsigned char *prow = p_s + (blk * 2 + bf) * C::P_BYTES + r * 128;
 #pragma unroll
             for (int ch = 0; ch < kTile / 8; ++ch) {
                 float e[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    e[i] = fast_exp2(s[ch * 8 + i] - m_use);
-                    psum += e[i];
+                for (int i = 0; i < 8; ++i) e[i] = fast_exp2(fmaf(s[ch * 8 + i], p.scale_log2, m_neg));
+                const uint32_t pk[4] = {pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7])};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    psum2 = fadd2(psum2, make_float2(e[2 * i], e[2 * i + 1]));
+                    prnd2 = fadd2(prnd2, make_float2(__uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u)));
                 }
-                const uint4 pk = make_uint4(pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7]));
-                prnd += (__uint_as_float(pk.x << 16) + __uint_as_float(pk.x & 0xffff0000u)) +
-                        (__uint_as_float(pk.y << 16) + __uint_as_float(pk.y & 0xffff0000u)) +
-                        (__uint_as_float(pk.z << 16) + __uint_as_float(pk.z & 0xffff0000u)) +
-                        (__uint_as_float(pk.w << 16) + __uint_as_float(pk.w & 0xffff0000u));
-                *(uint4 *)(prow + ((ch ^ (r & 7)) << 4)) = pk;
+                *(uint4 *)(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
+            const float psum = psum2.x + psum2.y, prnd = prnd2.x + prnd2.y;
             l_run += psum;
             l_rnd += prnd;
             if (!pv_prev_done) {  // normally long since complete: the wait only keeps the phase count in step
