@@ -197,12 +197,34 @@ def run_pipeline(args):
     log(f"[pipeline] pinned pool: {w.pool_chunks} chunks x {slot_bytes / 1e6:.0f} MB = {w.pool_chunks * slot_bytes / 1e9:.1f} GB; "
         f"{n_batches} batches of {B} x {w.chunks_per_req} chunks; 2 x {n_slots} device slots")
     sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=dev.index)
-    host_pool = torch.empty((w.pool_chunks, L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, pin_memory=True)
     tmp = torch.empty((L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
-    for c in range(w.pool_chunks):
-        gen.fill_bf16(tmp, w.seed, mi.STREAM_CHUNK + c)
-        host_pool[c].copy_(tmp)
-        mk.matkv_register_chunk(sess.ctx, c, w.chunk_tokens, host_pool[c].data_ptr(), None)
+    host_pool = ring = None
+    if args.store_dir:
+        # the materialised-KV store: one raw-bytes file per chunk id
+        os.makedirs(args.store_dir, exist_ok=True)
+        bounce = torch.empty(tmp.shape, dtype=torch.bfloat16, pin_memory=True)
+        t_w = time.perf_counter()
+        for c in range(w.pool_chunks):
+            path = os.path.join(args.store_dir, f"{c}.kv")
+            if not (os.path.exists(path) and os.path.getsize(path) == slot_bytes):
+                gen.fill_bf16(tmp, w.seed, mi.STREAM_CHUNK + c)
+                bounce.copy_(tmp)
+                torch.cuda.synchronize()
+                with open(path, "wb") as f:
+                    f.write(memoryview(bounce.view(torch.uint8).numpy()))
+            mk.matkv_register_chunk_file(sess.ctx, c, w.chunk_tokens, path, 0)
+        os.sync()
+        log(f"[pipeline] store written/checked in {time.perf_counter() - t_w:.1f} s")
+        n_slabs = 8
+        ring = torch.empty(n_slabs * slot_bytes + 4096, dtype=torch.uint8, pin_memory=True)
+        ring_base = (ring.data_ptr() + 4095) // 4096 * 4096
+        mk.matkv_set_bounce_buffer(sess.ctx, ring_base, n_slabs * slot_bytes, slot_bytes, args.io_threads)
+    else:
+        host_pool = torch.empty((w.pool_chunks, L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, pin_memory=True)
+        for c in range(w.pool_chunks):
+            gen.fill_bf16(tmp, w.seed, mi.STREAM_CHUNK + c)
+            host_pool[c].copy_(tmp)
+            mk.matkv_register_chunk(sess.ctx, c, w.chunk_tokens, host_pool[c].data_ptr(), None)
     del tmp
     slots = [torch.empty(n_slots * slot_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
     q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device=dev)
@@ -304,10 +326,13 @@ def run_pipeline(args):
         "dtype": "bf16 in, fp32 softmax/accumulate", "data": "synthetic",
         "config": {"workload": w.name, "layers": L, "batch": B, "chunks_per_request": w.chunks_per_req, "suffix": S,
                    "decode_steps": T, "pool_chunks": w.pool_chunks, "pinned_pool_gb": w.pool_chunks * slot_bytes / 1e9,
-                   "batches": n_batches, "timing": "host wall clock around synchronised passes (copy and compute streams)"},
+                   "batches": n_batches, "timing": "host wall clock around synchronised passes (copy and compute streams)",
+                   "chunk_pool": (f"files in {args.store_dir} read with O_DIRECT by {args.io_threads} threads through a pinned ring of 8 slabs"
+                                  if args.store_dir else "pinned host memory")},
         "clocks": clocks,
         "pipeline": {"t_stage_s": t_stage, "t_serial_s": t_serial, "t_pipelined_s": t_pipe,
-                     "h2d_gbs_staging_alone": staged_bytes / t_stage / 1e9, "staged_bytes": staged_bytes,
+                     ("storage_to_hbm_gbs_staging_alone" if args.store_dir else "h2d_gbs_staging_alone"): staged_bytes / t_stage / 1e9,
+                     "staged_bytes": staged_bytes, "load_s_per_request_staging_alone": t_stage / (n_batches * B),
                      "overlap_efficiency": (t_serial - t_pipe) / t_stage if t_stage > 0 else None,
                      "requests_per_s": n_batches * B / t_pipe, "compute_s_estimate": t_compute,
                      "decode_kv_gbs_pipelined_lower_bound": kv_bytes / t_pipe / 1e9},
@@ -332,6 +357,9 @@ def main():
     ap.add_argument("--no-other-mode", action="store_true", help="skip the second pass in the other decode launch mode")
     ap.add_argument("--batches", type=int, default=0, help="pipelined serving: number of sequential batches")
     ap.add_argument("--pool-chunks", type=int, default=0, help="pipelined serving: chunks in the pinned host pool")
+    ap.add_argument("--store-dir", default="", help="pipelined serving: keep the chunk pool as files in this directory "
+                    "(storage tier: reader threads -> pinned bounce ring -> device) instead of in pinned host memory")
+    ap.add_argument("--io-threads", type=int, default=8)
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (small profiling cases)")
     args = ap.parse_args()

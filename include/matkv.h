@@ -56,6 +56,7 @@ extern "C" {
 #define MATKV_E_CUDA          (-7)
 #define MATKV_E_TIMEOUT       (-8)  /* device status: a bounded wait inside a kernel ran out */
 #define MATKV_E_BOUNDS        (-9)  /* device status: a table-derived index was out of range */
+#define MATKV_E_IO            (-10) /* a chunk file could not be opened or read                */
 
 typedef struct matkv_ctx matkv_ctx;     /* opaque; owned by the library            */
 typedef struct matkv_table matkv_table; /* opaque; one per in-flight request batch */
@@ -108,6 +109,17 @@ int matkv_status(matkv_ctx *ctx, int32_t *dev_status_out, int32_t clear);
  * borrowed until matkv_unregister_chunk / matkv_destroy.  Re-registering an id is an error. */
 int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const void *host_blob,
                          void *dev_blob);
+/* The same for a chunk whose blob is stored in a file, `blob bytes` long at file_offset: the paper's
+ * materialised-KV store keeps one raw-bytes file per chunk id on flash (Section IV, store_KV /
+ * load_KV).  The file is opened now (O_DIRECT when offset and size are multiples of 4096 and the file
+ * system allows it) and stays open until unregister / destroy.  Such a chunk is staged through the
+ * bounce buffer set with matkv_set_bounce_buffer.                                                    */
+int matkv_register_chunk_file(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const char *path, uint64_t file_offset);
+/* Lends the library a pinned host ring for file-backed chunks (the paper's CPU bounce buffer between
+ * SSD and GPU, Section IV): `bytes` of page-locked host memory, 4096-byte aligned, cut into slabs of
+ * slab_bytes (>= the largest file-backed chunk, a multiple of 4096, at least two slabs), and starts
+ * n_io_threads reader threads.  Storage reads, host-to-device copies and GPU work then overlap.      */
+int matkv_set_bounce_buffer(matkv_ctx *ctx, void *pinned_host, size_t bytes, size_t slab_bytes, int32_t n_io_threads);
 /* The paper's delete(O) (Section IV): forgets the chunk.  Tables built earlier keep the
  * device address they resolved; the caller keeps that memory alive until they are freed.    */
 int matkv_unregister_chunk(matkv_ctx *ctx, uint64_t chunk_id);

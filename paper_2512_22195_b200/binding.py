@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libmatkv.so")
 
 OK, E_INVALID_ARG, E_UNKNOWN_CHUNK, E_NOT_STAGED, E_NOT_READY = 0, -1, -2, -3, -4
-E_CAPACITY, E_ALIGNMENT, E_CUDA, E_TIMEOUT, E_BOUNDS = -5, -6, -7, -8, -9
+E_CAPACITY, E_ALIGNMENT, E_CUDA, E_TIMEOUT, E_BOUNDS, E_IO = -5, -6, -7, -8, -9, -10
 OPT_DECODE_CTAS, OPT_PREFILL_IMPL, OPT_PREFILL_CTAS = 1, 2, 3
 
 EXPORTS = [
@@ -25,6 +25,7 @@ EXPORTS = [
     "matkv_table_free", "matkv_table_advance", "matkv_table_set_tail_len", "matkv_attend_prefill",
     "matkv_attend_decode", "matkv_attend_decode_all_layers", "matkv_lse_combine", "matkv_gather_debug",
     "matkv_probe_read", "matkv_attend_decode_static", "matkv_selftest_wait_timeout",
+    "matkv_register_chunk_file", "matkv_set_bounce_buffer",
 ]
 
 
@@ -78,6 +79,8 @@ def lib() -> C.CDLL:
             "matkv_probe_read": (C.c_int, [vp, vp, C.c_size_t, vp]),
             "matkv_attend_decode_static": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp]),
             "matkv_selftest_wait_timeout": (C.c_int, [vp, C.c_double, vp]),
+            "matkv_register_chunk_file": (C.c_int, [vp, u64, i32, C.c_char_p, u64]),
+            "matkv_set_bounce_buffer": (C.c_int, [vp, vp, C.c_size_t, C.c_size_t, i32]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -221,3 +224,11 @@ def matkv_attend_decode_static(ctx: int, table: int, layer: int, q: int, k_new: 
 
 def matkv_selftest_wait_timeout(ctx: int, seconds: float = 0.2, stream: int = 0) -> None:
     _check(lib().matkv_selftest_wait_timeout(ctx, seconds, stream or None))
+
+
+def matkv_register_chunk_file(ctx: int, chunk_id: int, n_tokens: int, path: str, file_offset: int = 0) -> None:
+    _check(lib().matkv_register_chunk_file(ctx, chunk_id, n_tokens, path.encode(), file_offset))
+
+
+def matkv_set_bounce_buffer(ctx: int, pinned_host_ptr: int, nbytes: int, slab_bytes: int, n_io_threads: int = 4) -> None:
+    _check(lib().matkv_set_bounce_buffer(ctx, pinned_host_ptr, nbytes, slab_bytes, n_io_threads))

@@ -171,6 +171,10 @@ static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
     }
 }
 
+static size_t blob_bytes(const matkv_config &c, int32_t n_tokens) {
+    return (size_t)c.n_layers * 2 * c.n_kv_heads * (size_t)n_tokens * c.head_dim * sizeof(__nv_bfloat16);
+}
+
 extern "C" {
 
 const char *matkv_last_error(void) { return g_err; }
@@ -216,7 +220,9 @@ int matkv_create(const matkv_config *cfg, matkv_ctx **out) {
 int matkv_destroy(matkv_ctx *ctx) {
     if (!ctx) return MATKV_OK;
     DeviceGuard guard(ctx->device);
-    cudaDeviceSynchronize();
+    cudaDeviceSynchronize();          // pending copies and their host callbacks finish first
+    io_engine_destroy(ctx);
+    for (auto &kv : ctx->chunks) close_chunk_file(kv.second.file_fd);
     for (matkv_table *t : std::vector<matkv_table *>(ctx->tables)) {
         cudaFreeHost(t->h_pinned);
         cudaFree(t->d_image);
@@ -304,19 +310,45 @@ int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, co
     return MATKV_OK;
 }
 
+int matkv_register_chunk_file(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const char *path, uint64_t file_offset) {
+    if (!ctx || !path) return fail(MATKV_E_INVALID_ARG, "matkv_register_chunk_file: null argument");
+    if (n_tokens < 1) return fail(MATKV_E_INVALID_ARG, "chunk %llu: n_tokens must be >= 1", (unsigned long long)chunk_id);
+    if (ctx->chunks.count(chunk_id))
+        return fail(MATKV_E_INVALID_ARG, "chunk %llu is already registered", (unsigned long long)chunk_id);
+    Chunk c;
+    c.n_tokens = n_tokens;
+    c.file_offset = file_offset;
+    int rc = open_chunk_file(path, file_offset, blob_bytes(ctx->cfg, n_tokens), &c.file_fd);
+    if (rc) return rc;
+    ctx->chunks.emplace(chunk_id, c);
+    return MATKV_OK;
+}
+
+int matkv_set_bounce_buffer(matkv_ctx *ctx, void *pinned_host, size_t bytes, size_t slab_bytes, int32_t n_io_threads) {
+    if (!ctx || !pinned_host) return fail(MATKV_E_INVALID_ARG, "matkv_set_bounce_buffer: null argument");
+    if ((uintptr_t)pinned_host % 4096 || slab_bytes == 0 || slab_bytes % 4096)
+        return fail(MATKV_E_ALIGNMENT, "bounce buffer and slab size must be multiples of 4096 bytes");
+    if (bytes / slab_bytes < 2) return fail(MATKV_E_CAPACITY, "bounce buffer must hold at least two slabs");
+    if (n_io_threads < 1 || n_io_threads > 64) return fail(MATKV_E_INVALID_ARG, "reader threads must be 1..64");
+    if (ctx->io) {
+        DeviceGuard guard(ctx->device);
+        MATKV_CUDA(cudaDeviceSynchronize());
+        io_engine_destroy(ctx);
+    }
+    return io_engine_create(ctx, pinned_host, bytes, slab_bytes, n_io_threads);
+}
+
 int matkv_unregister_chunk(matkv_ctx *ctx, uint64_t chunk_id) {
     if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_unregister_chunk: null context");
     auto it = ctx->chunks.find(chunk_id);
     if (it == ctx->chunks.end()) return fail(MATKV_E_UNKNOWN_CHUNK, "chunk %llu is not registered", (unsigned long long)chunk_id);
     Chunk &c = it->second;
     if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;
+    close_chunk_file(c.file_fd);
     ctx->chunks.erase(it);
     return MATKV_OK;
 }
 
-static size_t blob_bytes(const matkv_config &c, int32_t n_tokens) {
-    return (size_t)c.n_layers * 2 * c.n_kv_heads * (size_t)n_tokens * c.head_dim * sizeof(__nv_bfloat16);
-}
 
 // ---- a2 --------------------------------------------------------------------------------------
 int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, void *dev_slots, size_t slot_bytes,
@@ -338,7 +370,12 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
             return fail(MATKV_E_UNKNOWN_CHUNK, "chunk %llu is not registered", (unsigned long long)ids[i]);
         const Chunk &c = it->second;
         if (c.dev_blob) continue;  // resident: nothing to do
-        if (!c.host_blob) return fail(MATKV_E_INVALID_ARG, "chunk %llu has no host blob to stage", (unsigned long long)ids[i]);
+        if (!c.host_blob && c.file_fd < 0)
+            return fail(MATKV_E_INVALID_ARG, "chunk %llu has no host blob or file to stage", (unsigned long long)ids[i]);
+        if (c.file_fd >= 0 && !c.host_blob && blob_bytes(ctx->cfg, c.n_tokens) > io_engine_slab_bytes(ctx))
+            return fail(ctx->io ? MATKV_E_CAPACITY : MATKV_E_INVALID_ARG,
+                        "chunk %llu lives in a file: set a bounce buffer with slabs of at least %zu bytes first",
+                        (unsigned long long)ids[i], blob_bytes(ctx->cfg, c.n_tokens));
         if (blob_bytes(ctx->cfg, c.n_tokens) > slot_bytes)
             return fail(MATKV_E_CAPACITY, "chunk %llu (%zu bytes) does not fit a slot of %zu bytes",
                         (unsigned long long)ids[i], blob_bytes(ctx->cfg, c.n_tokens), slot_bytes);
@@ -399,10 +436,18 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
         }
         if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;  // moves from another region
         void *dst = (char *)dev_slots + (size_t)next_free * slot_bytes;
-        cudaError_t e = cudaMemcpyAsync(dst, c.host_blob, blob_bytes(ctx->cfg, c.n_tokens), cudaMemcpyHostToDevice, cs);
-        if (e != cudaSuccess) {
-            cudaEventDestroy(tk.done);
-            return cuda_fail(e, "staging copy");
+        if (c.host_blob) {
+            cudaError_t e = cudaMemcpyAsync(dst, c.host_blob, blob_bytes(ctx->cfg, c.n_tokens), cudaMemcpyHostToDevice, cs);
+            if (e != cudaSuccess) {
+                cudaEventDestroy(tk.done);
+                return cuda_fail(e, "staging copy");
+            }
+        } else {  // storage tier: read into the bounce ring, then copy, all in the copy stream's order
+            int rc = io_engine_stage(ctx, c.file_fd, c.file_offset, blob_bytes(ctx->cfg, c.n_tokens), dst, cs);
+            if (rc) {
+                cudaEventDestroy(tk.done);
+                return rc;
+            }
         }
         {
             int rc = encode_rows_map(&c.tmap, dst, ctx->cfg.head_dim, (uint64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * c.n_tokens);
@@ -440,6 +485,8 @@ int matkv_stage_wait(matkv_ctx *ctx, uint64_t ticket) {
     auto it = ctx->tickets.find(ticket);
     if (it == ctx->tickets.end()) return fail(MATKV_E_INVALID_ARG, "unknown staging ticket %llu", (unsigned long long)ticket);
     MATKV_CUDA(cudaEventSynchronize(it->second.done));
+    const char *msg = "";
+    if (io_engine_errors(ctx, &msg) > 0) return fail(MATKV_E_IO, "staging from storage failed: %s", msg);
     return MATKV_OK;
 }
 

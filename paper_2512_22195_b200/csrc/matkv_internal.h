@@ -34,11 +34,14 @@ struct DevReq {
 };
 
 // ---- host-side objects --------------------------------------------------------------------
-struct Region;  // staged slot region
+struct Region;    // staged slot region
+struct IoEngine;  // reader threads + pinned bounce ring for file-backed chunks
 
 struct Chunk {
     int32_t n_tokens = 0;
     const void *host_blob = nullptr;
+    int file_fd = -1;              // >= 0: the blob lives in a file, at file_offset
+    uint64_t file_offset = 0;
     void *dev_blob = nullptr;      // caller-resident device copy
     void *staged = nullptr;        // device copy inside a slot region (or nullptr)
     Region *region = nullptr;
@@ -78,6 +81,7 @@ struct matkv_ctx {
     std::unordered_map<uint64_t, matkv::Ticket> tickets;
     uint64_t next_ticket = 1;
     std::vector<matkv_table *> tables;
+    matkv::IoEngine *io = nullptr;
 };
 
 struct matkv_table {
@@ -146,6 +150,13 @@ int launch_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t 
                        const float *lse_parts, void *out, float *lse_out, cudaStream_t stream);
 int launch_gather(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out,
                   int64_t rows, cudaStream_t stream);
+int io_engine_create(matkv_ctx *ctx, void *pinned, size_t bytes, size_t slab_bytes, int n_threads);
+void io_engine_destroy(matkv_ctx *ctx);
+size_t io_engine_slab_bytes(const matkv_ctx *ctx);
+int io_engine_errors(matkv_ctx *ctx, const char **msg);
+int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream);
+int open_chunk_file(const char *path, uint64_t offset, size_t bytes, int *fd_out);
+void close_chunk_file(int fd);
 int launch_wait_selftest(matkv_ctx *ctx, double seconds, cudaStream_t stream);
 int launch_read_probe(matkv_ctx *ctx, const void *dev, size_t bytes, cudaStream_t stream);
 int launch_add_tail_len(matkv_table *t, int32_t delta, int32_t set_value, bool set, cudaStream_t stream);

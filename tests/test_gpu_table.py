@@ -160,3 +160,55 @@ def test_bounded_wait_runs_out_and_reports_without_losing_the_context():
     with pytest.raises(mk.MatkvError):
         mk.matkv_selftest_wait_timeout(sess.ctx, 30.0)
     sess.close()
+
+
+def test_storage_tier_files_through_the_bounce_ring(tmp_path):
+    """Chunks stored as raw-bytes files (one per chunk id): reader threads -> pinned ring -> device slots.
+    More chunks than ring slabs, an odd-sized chunk (buffered read path), then gather bit-exact and decode."""
+    import oracle
+    from _util import check
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D = 2, 8, 2, 64
+    lens = [64, 7, 128, 33, 64, 96, 1]
+    sess = Session(L, Hq, Hkv, D, 2, 4, 8)
+    blobs = [rand_bits(61, i, (L, 2, Hkv, n, D)) for i, n in enumerate(lens)]
+    for i, b in enumerate(blobs):
+        path = tmp_path / f"{i}.kv"
+        with open(path, "wb") as f:
+            f.write(b"\0" * (4096 if i == 2 else 0))          # chunk 2 sits at an offset inside its file
+            f.write(b.tobytes())
+        mk.matkv_register_chunk_file(sess.ctx, i, lens[i], str(path), 4096 if i == 2 else 0)
+    slot_bytes = max(b.nbytes for b in blobs)
+    slot_bytes = (slot_bytes + 4095) // 4096 * 4096
+    slots = torch.empty(len(lens) * slot_bytes, dtype=torch.uint8, device="cuda")
+    copy = torch.cuda.Stream()
+    with pytest.raises(mk.MatkvError):                         # no bounce buffer yet
+        sess.stage([0], slots, slot_bytes, copy)
+    ring = torch.empty(3 * slot_bytes + 4096, dtype=torch.uint8, pin_memory=True)
+    base = (ring.data_ptr() + 4095) // 4096 * 4096
+    mk.matkv_set_bounce_buffer(sess.ctx, base, 3 * slot_bytes, slot_bytes, 2)     # 3 slabs, 7 chunks: the ring wraps
+    tk = sess.stage(list(range(len(lens))), slots, slot_bytes, copy)
+    ids = [[0, 1, 2, 3], [6, 5, 4, 2]]
+    sess.build_table(ids)                                       # the compute stream waits for the copies
+    for r, row in enumerate(ids):
+        rows = sum(lens[c] for c in row)
+        k, v = sess.gather(1, r, rows)
+        assert np.array_equal(to_bits(k), np.concatenate([blobs[c][1, 0] for c in row], axis=1))
+        assert np.array_equal(to_bits(v), np.concatenate([blobs[c][1, 1] for c in row], axis=1))
+    mk.matkv_stage_wait(sess.ctx, tk)
+    assert mk.matkv_stage_query(sess.ctx, tk)
+    sh = oracle.Shape(L, Hq, Hkv, D)
+    q, k, v = rand_bits(61, 100, (2, Hq, D)), rand_bits(61, 101, (2, Hkv, D)), rand_bits(61, 102, (2, Hkv, D))
+    out, lse = sess.decode(0, to_dev(q), to_dev(k), to_dev(v))
+    for r, row in enumerate(ids):
+        o_ref, l_ref = oracle.Request(sh, [blobs[c] for c in row], 8).attend_new(0, q[r][None], k[r][None], v[r][None])
+        check(to_bits(out)[r], o_ref[0], lse.cpu().numpy()[r], l_ref[0], f"file-backed decode req {r}")
+    # error paths: missing file, file shorter than the chunk
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_register_chunk_file(sess.ctx, 100, 8, str(tmp_path / "nope.kv"))
+    assert e.value.code == mk.E_IO
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_register_chunk_file(sess.ctx, 101, 4096, str(tmp_path / "1.kv"))
+    assert e.value.code == mk.E_IO
+    assert sess.status() == 0
+    sess.close()
