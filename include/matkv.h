@@ -204,6 +204,17 @@ int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *table, int32_t layer
 int matkv_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts,
                       const float *lse_parts, void *out, float *lse_out, void *stream);
 
+/* ---- materialisation side (the paper's store_KV, Section IV: a chunk is prefilled alone, starting at
+ *      the first input position, and its K,V are moved GPU -> CPU bounce buffer -> storage) ------------- */
+/* After a causal sub-prefill of a chunk's own tokens over an EMPTY chunk list (matkv_attend_prefill for
+ * every layer, then matkv_table_advance), the request's tail holds exactly the chunk's K,V.  This call
+ * lays the first n_tokens of the tail of request `req` out as a chunk blob [L][2][Hkv][n_tokens][D] in
+ * dev_blob (device, 256-byte aligned, bit-exact copy) and, when host_blob is not NULL, copies the blob
+ * on to host memory (pinned for a truly asynchronous copy) on the same stream.  The blob can then be
+ * written to a file and registered like any other chunk.                                               */
+int matkv_export_tail_as_chunk(matkv_ctx *ctx, matkv_table *table, int32_t req, int32_t n_tokens, void *dev_blob,
+                               void *host_blob, void *stream);
+
 /* ---- debugging aid: the concatenation the table stands for ------------------------------- */
 /* Copies, for (layer, request), the K and V rows the table addresses into contiguous
  * k_out / v_out [Hkv][n_chunk_tokens + tail_len][D] bf16 device buffers (bit-exact gather).

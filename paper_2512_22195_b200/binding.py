@@ -25,7 +25,7 @@ EXPORTS = [
     "matkv_table_free", "matkv_table_advance", "matkv_table_set_tail_len", "matkv_attend_prefill",
     "matkv_attend_decode", "matkv_attend_decode_all_layers", "matkv_lse_combine", "matkv_gather_debug",
     "matkv_probe_read", "matkv_attend_decode_static", "matkv_selftest_wait_timeout",
-    "matkv_register_chunk_file", "matkv_set_bounce_buffer",
+    "matkv_register_chunk_file", "matkv_set_bounce_buffer", "matkv_export_tail_as_chunk",
 ]
 
 
@@ -81,6 +81,7 @@ def lib() -> C.CDLL:
             "matkv_selftest_wait_timeout": (C.c_int, [vp, C.c_double, vp]),
             "matkv_register_chunk_file": (C.c_int, [vp, u64, i32, C.c_char_p, u64]),
             "matkv_set_bounce_buffer": (C.c_int, [vp, vp, C.c_size_t, C.c_size_t, i32]),
+            "matkv_export_tail_as_chunk": (C.c_int, [vp, vp, i32, i32, vp, vp, vp]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -232,3 +233,8 @@ def matkv_register_chunk_file(ctx: int, chunk_id: int, n_tokens: int, path: str,
 
 def matkv_set_bounce_buffer(ctx: int, pinned_host_ptr: int, nbytes: int, slab_bytes: int, n_io_threads: int = 4) -> None:
     _check(lib().matkv_set_bounce_buffer(ctx, pinned_host_ptr, nbytes, slab_bytes, n_io_threads))
+
+
+def matkv_export_tail_as_chunk(ctx: int, table: int, req: int, n_tokens: int, dev_blob: int, host_blob: Optional[int] = None,
+                               stream: int = 0) -> None:
+    _check(lib().matkv_export_tail_as_chunk(ctx, table, req, n_tokens, dev_blob, host_blob or None, stream or None))

@@ -82,6 +82,36 @@ int launch_read_probe(matkv_ctx *ctx, const void *dev, size_t bytes, cudaStream_
     return MATKV_OK;
 }
 
+// Materialisation side: the tail of one request after a causal sub-prefill with an empty chunk list IS
+// the K,V of a chunk computed alone from position 0.  This kernel lays it out as a chunk blob
+// [L][2][Hkv][n][D] (16-byte vectors, bit-exact).
+__global__ void k_export_tail(const uint4 *__restrict__ tail_k, const uint4 *__restrict__ tail_v, uint4 *__restrict__ blob,
+                              int32_t L, int32_t Hkv, int32_t n, int32_t max_tail, int32_t vec_per_row) {
+    const int64_t per_slab = (int64_t)n * vec_per_row;
+    const int64_t total = (int64_t)L * 2 * Hkv * per_slab;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t within = i % per_slab;
+        int64_t r = i / per_slab;
+        const int g = (int)(r % Hkv); r /= Hkv;
+        const int kv = (int)(r % 2);
+        const int l = (int)(r / 2);
+        const int64_t src = ((int64_t)l * Hkv + g) * max_tail * vec_per_row + within;  // tail [L][Hkv][max_tail][D] of the request
+        blob[i] = kv ? tail_v[src] : tail_k[src];
+    }
+}
+
+int launch_export_tail(matkv_ctx *ctx, matkv_table *t, int32_t req, int32_t n_tokens, void *dev_blob, cudaStream_t stream) {
+    const matkv_config &c = ctx->cfg;
+    const int64_t req_off = (int64_t)req * c.n_layers * c.n_kv_heads * (int64_t)c.max_tail_tokens * c.head_dim;
+    const int64_t total = (int64_t)c.n_layers * 2 * c.n_kv_heads * n_tokens * (c.head_dim / 8);
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, 8 * (int64_t)ctx->n_sm);
+    k_export_tail<<<blocks, 256, 0, stream>>>((const uint4 *)(t->tail_k + req_off), (const uint4 *)(t->tail_v + req_off),
+                                             (uint4 *)dev_blob, c.n_layers, c.n_kv_heads, n_tokens, c.max_tail_tokens,
+                                             c.head_dim / 8);
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
 int launch_gather(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out, int64_t rows,
                   cudaStream_t stream) {
     const matkv_config &c = ctx->cfg;

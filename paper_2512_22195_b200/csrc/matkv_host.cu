@@ -777,6 +777,22 @@ int matkv_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D
     return launch_lse_combine(ctx, n_rows, n_parts, D, o_parts, lse_parts, out, lse_out, (cudaStream_t)stream);
 }
 
+int matkv_export_tail_as_chunk(matkv_ctx *ctx, matkv_table *t, int32_t req, int32_t n_tokens, void *dev_blob, void *host_blob,
+                               void *stream) {
+    if (!ctx || !t || !dev_blob) return fail(MATKV_E_INVALID_ARG, "matkv_export_tail_as_chunk: null argument");
+    if (t->ctx != ctx) return fail(MATKV_E_INVALID_ARG, "matkv_export_tail_as_chunk: table belongs to another context");
+    if (req < 0 || req >= t->batch) return fail(MATKV_E_INVALID_ARG, "matkv_export_tail_as_chunk: request %d out of range", req);
+    if (n_tokens < 1 || n_tokens > t->tail_len_host)
+        return fail(MATKV_E_CAPACITY, "matkv_export_tail_as_chunk: %d tokens asked, the tail holds %d", n_tokens, t->tail_len_host);
+    if ((uintptr_t)dev_blob % 256) return fail(MATKV_E_ALIGNMENT, "matkv_export_tail_as_chunk: device blob must be 256-byte aligned");
+    DeviceGuard guard(ctx->device);
+    int rc = launch_export_tail(ctx, t, req, n_tokens, dev_blob, (cudaStream_t)stream);
+    if (rc) return rc;
+    if (host_blob)  // the paper's GPU -> CPU bounce buffer hop of store_KV, asynchronous on the stream
+        MATKV_CUDA(cudaMemcpyAsync(host_blob, dev_blob, blob_bytes(ctx->cfg, n_tokens), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    return MATKV_OK;
+}
+
 int matkv_selftest_wait_timeout(matkv_ctx *ctx, double seconds, void *stream) {
     if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_selftest_wait_timeout: null context");
     if (!(seconds > 0.0) || seconds > 2.0) return fail(MATKV_E_INVALID_ARG, "matkv_selftest_wait_timeout: limit must be in (0, 2] seconds");

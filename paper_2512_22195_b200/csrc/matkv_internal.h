@@ -158,6 +158,7 @@ int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void 
 int open_chunk_file(const char *path, uint64_t offset, size_t bytes, int *fd_out);
 void close_chunk_file(int fd);
 int launch_wait_selftest(matkv_ctx *ctx, double seconds, cudaStream_t stream);
+int launch_export_tail(matkv_ctx *ctx, matkv_table *t, int32_t req, int32_t n_tokens, void *dev_blob, cudaStream_t stream);
 int launch_read_probe(matkv_ctx *ctx, const void *dev, size_t bytes, cudaStream_t stream);
 int launch_add_tail_len(matkv_table *t, int32_t delta, int32_t set_value, bool set, cudaStream_t stream);
 

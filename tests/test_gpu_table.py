@@ -212,3 +212,45 @@ def test_storage_tier_files_through_the_bounce_ring(tmp_path):
     assert e.value.code == mk.E_IO
     assert sess.status() == 0
     sess.close()
+
+
+def test_materialise_then_reuse_round_trip():
+    """store_KV in kernel terms: a chunk's tokens are sub-prefilled alone (empty chunk list, causal, from
+    position 0), the tail is exported as a chunk blob, and that blob serves later requests.  The exported
+    bytes equal the K,V that went in, the causal outputs match the oracle, and a request that reuses the
+    blob gets the same answer as one that was given the original K,V as a chunk."""
+    import oracle
+    from _util import check
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D, n = 2, 8, 2, 128, 150
+    sess = Session(L, Hq, Hkv, D, 1, 2, n)
+    sh = oracle.Shape(L, Hq, Hkv, D)
+    q = rand_bits(71, 1, (L, 1, n, Hq, D))
+    k = rand_bits(71, 2, (L, 1, n, Hkv, D))
+    v = rand_bits(71, 3, (L, 1, n, Hkv, D))
+    sess.build_table([[]])
+    ref = oracle.Request(sh, [], n)
+    for layer in range(L):
+        out, lse = sess.prefill(layer, to_dev(q[layer]), to_dev(k[layer]), to_dev(v[layer]))
+        o_ref, l_ref = ref.attend_new(layer, q[layer, 0], k[layer, 0], v[layer, 0])     # plain causal attention from position 0
+        check(to_bits(out)[0], o_ref, lse.cpu().numpy()[0], l_ref, f"materialisation layer {layer}")
+    sess.advance(n)
+    blob_dev = torch.empty((L, 2, Hkv, n, D), dtype=torch.bfloat16, device="cuda")
+    blob_host = torch.empty((L, 2, Hkv, n, D), dtype=torch.bfloat16, pin_memory=True)
+    mk.matkv_export_tail_as_chunk(sess.ctx, sess.table, 0, n, blob_dev.data_ptr(), blob_host.data_ptr())
+    torch.cuda.synchronize()
+    want = np.stack([np.stack([k[layer, 0].transpose(1, 0, 2), v[layer, 0].transpose(1, 0, 2)]) for layer in range(L)])
+    assert np.array_equal(to_bits(blob_dev), want) and np.array_equal(to_bits(blob_host), want)
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_export_tail_as_chunk(sess.ctx, sess.table, 0, n + 1, blob_dev.data_ptr())
+    assert e.value.code == mk.E_CAPACITY
+    # reuse: the exported blob as a materialised chunk of a new request
+    sess2 = Session(L, Hq, Hkv, D, 1, 2, 8)
+    sess2.register_device_chunk(5, blob_dev)
+    sess2.build_table([[5]])
+    q1, k1, v1 = rand_bits(71, 4, (1, Hq, D)), rand_bits(71, 5, (1, Hkv, D)), rand_bits(71, 6, (1, Hkv, D))
+    out, lse = sess2.decode(1, to_dev(q1), to_dev(k1), to_dev(v1))
+    o_ref, l_ref = oracle.Request(sh, [want], 8).attend_new(1, q1, k1, v1)
+    check(to_bits(out)[0], o_ref[0], lse.cpu().numpy()[0], l_ref[0], "decode over the re-used chunk")
+    assert sess.status() == 0 and sess2.status() == 0
+    sess.close(); sess2.close()
