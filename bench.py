@@ -197,6 +197,10 @@ def run_pipeline(args):
     log(f"[pipeline] pinned pool: {w.pool_chunks} chunks x {slot_bytes / 1e6:.0f} MB = {w.pool_chunks * slot_bytes / 1e9:.1f} GB; "
         f"{n_batches} batches of {B} x {w.chunks_per_req} chunks; 2 x {n_slots} device slots")
     sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=dev.index)
+    if args.stage_ctas < 0:
+        args.stage_ctas = 16
+    if args.stage_ctas:
+        mk.matkv_set_option(sess.ctx, mk.OPT_STAGE_CTAS, args.stage_ctas)
     tmp = torch.empty((L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
     host_pool = ring = None
     if args.store_dir:
@@ -328,7 +332,8 @@ def run_pipeline(args):
                    "decode_steps": T, "pool_chunks": w.pool_chunks, "pinned_pool_gb": w.pool_chunks * slot_bytes / 1e9,
                    "batches": n_batches, "timing": "host wall clock around synchronised passes (copy and compute streams)",
                    "chunk_pool": (f"files in {args.store_dir} read with O_DIRECT by {args.io_threads} threads through a pinned ring of 8 slabs"
-                                  if args.store_dir else "pinned host memory")},
+                                  if args.store_dir else "pinned host memory"),
+                   "staging": f"copy kernel, {args.stage_ctas} CTAs" if args.stage_ctas else "copy engine"},
         "clocks": clocks,
         "pipeline": {"t_stage_s": t_stage, "t_serial_s": t_serial, "t_pipelined_s": t_pipe,
                      ("storage_to_hbm_gbs_staging_alone" if args.store_dir else "h2d_gbs_staging_alone"): staged_bytes / t_stage / 1e9,
@@ -360,6 +365,10 @@ def main():
     ap.add_argument("--store-dir", default="", help="pipelined serving: keep the chunk pool as files in this directory "
                     "(storage tier: reader threads -> pinned bounce ring -> device) instead of in pinned host memory")
     ap.add_argument("--io-threads", type=int, default=8)
+    ap.add_argument("--stage-ctas", type=int, default=-1, help="stage host chunks with a copy kernel of this many CTAs; 0 = copy "
+                    "engine; -1 = auto: 16 CTAs in the pipelined-serving mode (long decode launches that saturate HBM starve "
+                    "the copy engine), copy engine in the single-batch end-to-end leg (short launches: a co-resident copy "
+                    "CTA makes its SM the straggler of every launch)")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (small profiling cases)")
     args = ap.parse_args()
@@ -584,6 +593,8 @@ def main():
         ho_dc = torch.empty(o_dc.shape, dtype=torch.bfloat16, pin_memory=True)
         torch.cuda.synchronize()
         sess2 = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
+        if args.stage_ctas > 0:
+            mk.matkv_set_option(sess2.ctx, mk.OPT_STAGE_CTAS, args.stage_ctas)
         for c in needed:
             mk.matkv_register_chunk(sess2.ctx, c, w.chunk_tokens, host[c].data_ptr(), None)
         slot_bytes = w.chunk_bytes
@@ -639,6 +650,7 @@ def main():
         result["e2e"] = {"value": tokens * k_e2e / (ms_e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                          "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e,
                          "overlap": "next step's chunks staged on a side stream under this step's prefill and decode",
+                         "staging": f"copy kernel, {args.stage_ctas} CTAs" if args.stage_ctas > 0 else "copy engine",
                          "h2d_gbs_if_copy_bound": h2d * k_e2e / (ms_e * 1e-3) / 1e9}
         sess2.close()
         del host, slots

@@ -82,6 +82,9 @@ typedef struct {
                                       1 = force the streaming kernel, 2 = force the tensor-core kernel,
                                       3 = tensor-core kernel with two 128-row blocks per CTA whenever a
                                           (request, KV head) has more than 128 query rows */
+#define MATKV_OPT_STAGE_CTAS    4  /* 0 = stage host blobs with the copy engine (cudaMemcpyAsync); n > 0 = with a copy
+                                      kernel of n small CTAs that runs beside the decode CTAs (the host blobs must
+                                      then be pinned, device-accessible memory) */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
 
 /* ---- context -------------------------------------------------------------------------- */

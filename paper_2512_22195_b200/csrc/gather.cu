@@ -112,6 +112,30 @@ int launch_export_tail(matkv_ctx *ctx, matkv_table *t, int32_t req, int32_t n_to
     return MATKV_OK;
 }
 
+// Staging copy on the SMs: a few small CTAs pull a pinned host blob over PCIe with 16-byte loads and
+// write it to the device slot.  Unlike the copy engine, whose host-to-device rate halves while a decode
+// launch saturates HBM, these CTAs sit next to the persistent decode CTAs (they need no shared memory
+// and few registers) and keep their loads in flight through the SM's own memory pipeline.
+__global__ void __launch_bounds__(128) k_stage_copy(const uint4 *__restrict__ src, uint4 *__restrict__ dst, int64_t n_vec) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 7 * stride < n_vec; i += 8 * stride) {
+        uint4 v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = __ldcs(src + i + k * stride);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) dst[i + k * stride] = v[k];
+    }
+    for (; i < n_vec; i += stride) dst[i] = __ldcs(src + i);
+}
+
+int launch_stage_copy(matkv_ctx *ctx, const void *host_src, void *dev_dst, size_t bytes, int n_ctas, cudaStream_t stream) {
+    (void)ctx;
+    k_stage_copy<<<n_ctas, 128, 0, stream>>>((const uint4 *)host_src, (uint4 *)dev_dst, (int64_t)(bytes / 16));
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
 int launch_gather(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, void *k_out, void *v_out, int64_t rows,
                   cudaStream_t stream) {
     const matkv_config &c = ctx->cfg;

@@ -251,6 +251,10 @@ int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
             if (value < 0 || value > 3) return fail(MATKV_E_INVALID_ARG, "prefill impl must be 0..3");
             ctx->opt_prefill_impl = value;
             return MATKV_OK;
+        case MATKV_OPT_STAGE_CTAS:
+            if (value < 0 || value > 148) return fail(MATKV_E_INVALID_ARG, "staging CTAs must be 0..148");
+            ctx->opt_stage_ctas = value;
+            return MATKV_OK;
         case MATKV_OPT_PREFILL_CTAS:
             if (value < 0 || value > 64) return fail(MATKV_E_INVALID_ARG, "prefill CTAs per head must be 0..64");
             ctx->opt_prefill_ctas = value;
@@ -436,7 +440,14 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
         }
         if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;  // moves from another region
         void *dst = (char *)dev_slots + (size_t)next_free * slot_bytes;
-        if (c.host_blob) {
+        if (c.host_blob && ctx->opt_stage_ctas > 0) {
+            // SM-driven copy (the host blob must be device-accessible: pinned memory under unified addressing)
+            int rc = launch_stage_copy(ctx, c.host_blob, dst, blob_bytes(ctx->cfg, c.n_tokens), (int)ctx->opt_stage_ctas, cs);
+            if (rc) {
+                cudaEventDestroy(tk.done);
+                return rc;
+            }
+        } else if (c.host_blob) {
             cudaError_t e = cudaMemcpyAsync(dst, c.host_blob, blob_bytes(ctx->cfg, c.n_tokens), cudaMemcpyHostToDevice, cs);
             if (e != cudaSuccess) {
                 cudaEventDestroy(tk.done);

@@ -75,7 +75,7 @@ struct matkv_ctx {
     int32_t *d_status = nullptr;
     void *workspace = nullptr;
     size_t workspace_bytes = 0;
-    int64_t opt_decode_ctas = 0, opt_prefill_impl = 0, opt_prefill_ctas = 0;
+    int64_t opt_decode_ctas = 0, opt_prefill_impl = 0, opt_prefill_ctas = 0, opt_stage_ctas = 0;
     std::unordered_map<uint64_t, matkv::Chunk> chunks;
     std::map<void *, matkv::Region *> regions;
     std::unordered_map<uint64_t, matkv::Ticket> tickets;
@@ -158,6 +158,7 @@ int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void 
 int open_chunk_file(const char *path, uint64_t offset, size_t bytes, int *fd_out);
 void close_chunk_file(int fd);
 int launch_wait_selftest(matkv_ctx *ctx, double seconds, cudaStream_t stream);
+int launch_stage_copy(matkv_ctx *ctx, const void *host_src, void *dev_dst, size_t bytes, int n_ctas, cudaStream_t stream);
 int launch_export_tail(matkv_ctx *ctx, matkv_table *t, int32_t req, int32_t n_tokens, void *dev_blob, cudaStream_t stream);
 int launch_read_probe(matkv_ctx *ctx, const void *dev, size_t bytes, cudaStream_t stream);
 int launch_add_tail_len(matkv_table *t, int32_t delta, int32_t set_value, bool set, cudaStream_t stream);

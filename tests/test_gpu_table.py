@@ -81,6 +81,29 @@ def test_staging_then_gather_bit_exact_and_overlap_bookkeeping():
     sess.close()
 
 
+def test_staging_with_the_copy_kernel_is_bit_exact():
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D = 2, 4, 2, 128
+    sess = Session(L, Hq, Hkv, D, 1, 3, 8)
+    mk.matkv_set_option(sess.ctx, mk.OPT_STAGE_CTAS, 4)
+    lens = [1000, 33, 257]
+    blobs = [rand_bits(45, i, (L, 2, Hkv, n, D)) for i, n in enumerate(lens)]
+    for i, b in enumerate(blobs):
+        sess.register_host_chunk(i, b)
+    slot_bytes = (max(b.nbytes for b in blobs) + 255) // 256 * 256
+    slots = torch.empty(3 * slot_bytes, dtype=torch.uint8, device="cuda")
+    copy = torch.cuda.Stream()
+    tk = sess.stage([2, 0, 1], slots, slot_bytes, copy)
+    sess.build_table([[0, 1, 2]])
+    k, v = sess.gather(1, 0, sum(lens))
+    assert np.array_equal(to_bits(k), np.concatenate([b[1, 0] for b in blobs], axis=1))
+    assert np.array_equal(to_bits(v), np.concatenate([b[1, 1] for b in blobs], axis=1))
+    mk.matkv_stage_wait(sess.ctx, tk)
+    with pytest.raises(mk.MatkvError):
+        mk.matkv_set_option(sess.ctx, mk.OPT_STAGE_CTAS, 1000)
+    sess.close()
+
+
 def test_host_side_error_paths():
     mk, Session, to_dev, to_bits = _mk()
     with pytest.raises(mk.MatkvError):
