@@ -32,7 +32,7 @@ import matkv_inputs as mi  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per decode launch from the committed ncu capture (profiles/), by workload and launch mode.
-NCU_TRAFFIC_BYTES = {("cfg2", "all_layers"): 697.2e6 + 4.4e6}  # profiles/k_attend_stream_decode_cfg2_all_layers.md
+NCU_TRAFFIC_BYTES = {("cfg2", "all_layers"): 697.5e6 + 5.0e6}  # profiles/k_attend_stream_decode_cfg2_all_layers.md
 
 
 def log(*a):
