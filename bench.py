@@ -252,9 +252,7 @@ def run_pipeline(args):
 
     def compute(n):
         table = sess.build_table(batches[n], sp)
-        for layer in range(L):
-            mk.matkv_attend_prefill(ctx, table, layer, S, q_pf.data_ptr() + layer * qs_l, k_pf.data_ptr() + layer * ks_l,
-                                    v_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
+        mk.matkv_attend_prefill_all_layers(ctx, table, S, q_pf.data_ptr(), k_pf.data_ptr(), v_pf.data_ptr(), o_pf.data_ptr(), None, sp)
         mk.matkv_table_advance(table, S, sp)
         for t in range(T):
             mk.matkv_attend_decode_all_layers(ctx, table, q_dc.data_ptr() + t * qd_t, k_dc.data_ptr() + t * kd_t,
@@ -290,9 +288,7 @@ def run_pipeline(args):
         table = sess.build_table(batches[n], sp)
         if n + 1 < n_batches:
             stage(n + 1)
-        for layer in range(L):
-            mk.matkv_attend_prefill(ctx, table, layer, S, q_pf.data_ptr() + layer * qs_l, k_pf.data_ptr() + layer * ks_l,
-                                    v_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
+        mk.matkv_attend_prefill_all_layers(ctx, table, S, q_pf.data_ptr(), k_pf.data_ptr(), v_pf.data_ptr(), o_pf.data_ptr(), None, sp)
         mk.matkv_table_advance(table, S, sp)
         for t in range(T):
             mk.matkv_attend_decode_all_layers(ctx, table, q_dc.data_ptr() + t * qd_t, k_dc.data_ptr() + t * kd_t,
@@ -447,13 +443,16 @@ def main():
         table = sess.build_table(ids, sp)
         if timed_index is not None:
             ev_p0[timed_index].record(stream)
-        for layer in range(L):
-            mk.matkv_attend_prefill(ctx, table, layer, S, q_pf_p + layer * qs_l, k_pf_p + layer * ks_l, v_pf_p + layer * ks_l,
-                                    o_pf.data_ptr() + layer * qs_l, None, sp)
+        if mode == "all_layers":
+            mk.matkv_attend_prefill_all_layers(ctx, table, S, q_pf_p, k_pf_p, v_pf_p, o_pf.data_ptr(), None, sp)
+        else:
+            for layer in range(L):
+                mk.matkv_attend_prefill(ctx, table, layer, S, q_pf_p + layer * qs_l, k_pf_p + layer * ks_l, v_pf_p + layer * ks_l,
+                                        o_pf.data_ptr() + layer * qs_l, None, sp)
         mk.matkv_table_advance(table, S, sp)
         if timed_index is not None:
             ev_d0[timed_index].record(stream)
-        n = L + 1
+        n = (1 if mode == "all_layers" else L) + 1
         if mode == "per_layer_graph":
             # one decode step (L per-layer launches + the tail counter) captured once per table and replayed
             # T times; each step's q/k/v are copied into fixed buffers first (a graph replays fixed addresses)
@@ -560,7 +559,7 @@ def main():
         "vs_baseline": None, "dtype": "bf16 in, fp32 softmax/accumulate", "data": "synthetic",
         "config": {"workload": w.name, "layers": L, "q_heads": Hq, "kv_heads": Hkv, "head_dim": D, "batch": B,
                    "chunks_per_request": w.chunks_per_req, "chunk_tokens": w.chunk_tokens, "suffix": S, "decode_steps": T,
-                   "decode_launch": args.decode_launch, "l2": "inputs larger than L2 (KV per decode step = "
+                   "decode_launch": args.decode_launch, "prefill_launch": "all_layers" if args.decode_launch == "all_layers" else "per_layer", "l2": "inputs larger than L2 (KV per decode step = "
                    f"{kv_bytes_decode / T / 1e6:.0f} MB vs 126 MB L2)", "multi_gpu": "independent replicas per rank"},
         "gpu_launches": n_launch,
         "clocks": clocks,
@@ -622,9 +621,12 @@ def main():
             dq_dc.copy_(hq_dc, non_blocking=True); dk_dc.copy_(hk_dc, non_blocking=True); dv_dc.copy_(hv_dc, non_blocking=True)
             table = sess2.build_table(ids, sp)
             stage(i + 1)
-            for layer in range(L):
-                mk.matkv_attend_prefill(ctx2, table, layer, S, dq_pf.data_ptr() + layer * qs_l, dk_pf.data_ptr() + layer * ks_l,
-                                        dv_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
+            if args.decode_launch == "all_layers":
+                mk.matkv_attend_prefill_all_layers(ctx2, table, S, dq_pf.data_ptr(), dk_pf.data_ptr(), dv_pf.data_ptr(), o_pf.data_ptr(), None, sp)
+            else:
+                for layer in range(L):
+                    mk.matkv_attend_prefill(ctx2, table, layer, S, dq_pf.data_ptr() + layer * qs_l, dk_pf.data_ptr() + layer * ks_l,
+                                            dv_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
             mk.matkv_table_advance(table, S, sp)
             for t in range(T):
                 if args.decode_launch == "all_layers":

@@ -170,6 +170,12 @@ int matkv_table_set_tail_len(matkv_table *table, int32_t tail_len, void *stream)
 int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *table, int32_t layer, int32_t S, const void *q,
                          const void *k_new, const void *v_new, void *out, float *lse_out, void *stream);
 
+/* The same for every layer in ONE launch: q [L][B][S][Hq][D], k_new / v_new [L][B][S][Hkv][D], out
+ * [L][B][S][Hq][D], lse_out NULL or [L][B][S][Hq].  Like matkv_attend_decode_all_layers, only usable
+ * when all layers' inputs exist up front (an attention-only benchmark).                              */
+int matkv_attend_prefill_all_layers(matkv_ctx *ctx, matkv_table *table, int32_t S, const void *q, const void *k_new,
+                                    const void *v_new, void *out, float *lse_out, void *stream);
+
 /* ---- a5 + a6: decode step (Section V-A "Decode time"; memory-bound streaming over the
  *      loaded KVs) with split-KV partials merged by log-sum-exp ---------------------------- */
 /* One new token per request.  q [B][Hq][D], k_new / v_new [B][Hkv][D], out [B][Hq][D] bf16

@@ -26,6 +26,7 @@ EXPORTS = [
     "matkv_attend_decode", "matkv_attend_decode_all_layers", "matkv_lse_combine", "matkv_gather_debug",
     "matkv_probe_read", "matkv_attend_decode_static", "matkv_selftest_wait_timeout",
     "matkv_register_chunk_file", "matkv_set_bounce_buffer", "matkv_export_tail_as_chunk",
+    "matkv_attend_prefill_all_layers",
 ]
 
 
@@ -82,6 +83,7 @@ def lib() -> C.CDLL:
             "matkv_register_chunk_file": (C.c_int, [vp, u64, i32, C.c_char_p, u64]),
             "matkv_set_bounce_buffer": (C.c_int, [vp, vp, C.c_size_t, C.c_size_t, i32]),
             "matkv_export_tail_as_chunk": (C.c_int, [vp, vp, i32, i32, vp, vp, vp]),
+            "matkv_attend_prefill_all_layers": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -238,3 +240,8 @@ def matkv_set_bounce_buffer(ctx: int, pinned_host_ptr: int, nbytes: int, slab_by
 def matkv_export_tail_as_chunk(ctx: int, table: int, req: int, n_tokens: int, dev_blob: int, host_blob: Optional[int] = None,
                                stream: int = 0) -> None:
     _check(lib().matkv_export_tail_as_chunk(ctx, table, req, n_tokens, dev_blob, host_blob or None, stream or None))
+
+
+def matkv_attend_prefill_all_layers(ctx: int, table: int, S: int, q: int, k_new: int, v_new: int, out: int,
+                                    lse_out: Optional[int] = None, stream: int = 0) -> None:
+    _check(lib().matkv_attend_prefill_all_layers(ctx, table, S, q, k_new, v_new, out, lse_out or None, stream or None))

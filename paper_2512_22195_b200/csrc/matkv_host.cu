@@ -83,9 +83,8 @@ int encode_new_rows_map(CUtensorMap *out, const void *base, int D, int Hkv, uint
 size_t rope_scratch_bytes(const matkv_config &c) {
     if (c.rope_theta == 0.f) return 0;
     const size_t per_tok = (size_t)(c.n_q_heads + c.n_kv_heads) * c.head_dim * sizeof(__nv_bfloat16);
-    const size_t prefill = (size_t)c.max_batch * c.max_tail_tokens * per_tok;  // one layer, up to max_tail tokens
-    const size_t decode = (size_t)c.n_layers * c.max_batch * per_tok;          // all layers, one token
-    return align_up(std::max(prefill, decode), 256);
+    // the largest call: every layer, up to max_tail tokens per request
+    return align_up((size_t)c.n_layers * c.max_batch * c.max_tail_tokens * per_tok, 256);
 }
 
 size_t workspace_bytes_for(const matkv_config &c, WorkspaceView *v, void *base) {
@@ -776,6 +775,52 @@ int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t 
     const bool tensor_core = ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
     if (tensor_core) return launch_prefill_tc(ctx, t, a, (cudaStream_t)stream);
     return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+}
+
+int matkv_attend_prefill_all_layers(matkv_ctx *ctx, matkv_table *t, int32_t S, const void *q, const void *kn, const void *vn,
+                                    void *out, float *lse_out, void *stream) {
+    if (S < 1) return fail(MATKV_E_INVALID_ARG, "matkv_attend_prefill_all_layers: S must be >= 1");
+    int rc = check_attend(ctx, t, q, kn, vn, out, S, "matkv_attend_prefill_all_layers");
+    if (rc) return rc;
+    DeviceGuard guard(ctx->device);
+    const matkv_config &c = ctx->cfg;
+    AttendArgs a;
+    a.layer0 = 0;
+    a.n_layers_launch = c.n_layers;
+    a.S = S;
+    a.q = (const __nv_bfloat16 *)q;
+    a.k_new = (const __nv_bfloat16 *)kn;
+    a.v_new = (const __nv_bfloat16 *)vn;
+    a.out = (__nv_bfloat16 *)out;
+    a.lse_out = lse_out;
+    a.q_ss = (int64_t)c.n_q_heads * c.head_dim; a.q_sb = a.q_ss * S; a.q_sl = a.q_sb * t->batch;
+    a.kn_ss = (int64_t)c.n_kv_heads * c.head_dim; a.kn_sb = a.kn_ss * S; a.kn_sl = a.kn_sb * t->batch;
+    a.lse_ss = c.n_q_heads; a.lse_sb = a.lse_ss * S; a.lse_sl = a.lse_sb * t->batch;
+    if (c.rope_theta != 0.f) {
+        rc = launch_rope(ctx, t, a, (cudaStream_t)stream);
+        if (rc) return rc;
+    }
+    const int G = c.n_q_heads / c.n_kv_heads;
+    const bool tensor_core = ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
+    if (tensor_core) return launch_prefill_tc(ctx, t, a, (cudaStream_t)stream);
+    // short suffixes run on the streaming kernel; when its units do not fit the workspace's counters in one
+    // launch, the layers are launched one by one (same result)
+    WorkspaceView ws;
+    workspace_bytes_for(c, &ws, ctx->workspace);
+    const int64_t n_blk = (S + kUnitRows / G - 1) / (kUnitRows / G);
+    if ((int64_t)c.n_layers * t->batch * n_blk * c.n_kv_heads <= ws.n_counter_slots)
+        return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+    for (int32_t layer = 0; layer < c.n_layers; ++layer) {
+        AttendArgs one = a;
+        one.layer0 = layer;
+        one.n_layers_launch = 1;
+        one.q = a.q + layer * a.q_sl; one.k_new = a.k_new + layer * a.kn_sl; one.v_new = a.v_new + layer * a.kn_sl;
+        one.out = a.out + layer * a.q_sl;
+        one.lse_out = a.lse_out ? a.lse_out + layer * a.lse_sl : nullptr;
+        rc = launch_attend_stream(ctx, t, one, (cudaStream_t)stream);
+        if (rc) return rc;
+    }
+    return MATKV_OK;
 }
 
 int matkv_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts,

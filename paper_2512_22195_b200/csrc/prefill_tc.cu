@@ -45,10 +45,10 @@ struct Params {
     const __nv_bfloat16 *q, *k_new, *v_new;
     __nv_bfloat16 *out;
     float *lse_out;
-    int64_t q_sb, q_ss, kn_sb, kn_ss;  // element strides: request, suffix token
-    int32_t layer, n_layers_total, B, S, Hq, Hkv, max_tail, n_rb, n_split;
+    int64_t q_sl, q_sb, q_ss, kn_sl, kn_sb, kn_ss;  // element strides: layer, request, suffix token
+    int32_t layer0, n_layers_launch, n_layers_total, B, S, Hq, Hkv, max_tail, n_rb, n_split;
     float scale_log2;
-    float *part_o, *part_lse;  // [row][split][D], [row][split]; row = (b*S + i)*Hq + head
+    float *part_o, *part_lse;  // [row][split][D], [row][split]; row = ((layer*B + b)*S + i)*Hq + head
     int32_t *status;
 };
 
@@ -220,8 +220,10 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
     int c = blockIdx.x;
     const int sp = c % p.n_split; c /= p.n_split;
     const int rb = c % p.n_rb; c /= p.n_rb;                      // index of this CTA's group of NBLK row blocks
-    const int g = c % p.Hkv;
-    const int b = c / p.Hkv;
+    const int g = c % p.Hkv; c /= p.Hkv;
+    const int b = c % p.B;
+    const int l_rel = c / p.B;                                   // layer of the launch
+    const int layer = p.layer0 + l_rel;
     const DevReq rq = p.reqs[b];
     int t0 = p.tail_len[b];
     if (t0 < 0 || t0 + p.S > p.max_tail) {
@@ -306,12 +308,12 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     int32_t yk, yv;
                     if (ti.kind == 0) {
                         mk = mv = p.tmaps + rq.seg_begin + ti.seg;
-                        yk = ((p.layer * 2) * p.Hkv + g) * ti.seg_len + ti.r0;
-                        yv = ((p.layer * 2 + 1) * p.Hkv + g) * ti.seg_len + ti.r0;
+                        yk = ((layer * 2) * p.Hkv + g) * ti.seg_len + ti.r0;
+                        yv = ((layer * 2 + 1) * p.Hkv + g) * ti.seg_len + ti.r0;
                     } else {
                         mk = p.tmaps + p.n_seg_total;
                         mv = mk + 1;
-                        yk = yv = ((b * p.n_layers_total + p.layer) * p.Hkv + g) * p.max_tail + ti.r0;
+                        yk = yv = ((b * p.n_layers_total + layer) * p.Hkv + g) * p.max_tail + ti.r0;
                     }
 #pragma unroll
                     for (int bx = 0; bx < C::NBOX; ++bx) {
@@ -322,8 +324,8 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     // the call's new tokens, straight from k_new / v_new [B*S][Hkv][D] (rows past S are masked)
 #pragma unroll
                     for (int bx = 0; bx < C::NBOX; ++bx) {
-                        tma_load_3d(dst + bx * C::BOX_BYTES, &kn_map, bx * 64, g, b * p.S + ti.r0, bar);
-                        tma_load_3d(dst + C::KV_BYTES + bx * C::BOX_BYTES, &vn_map, bx * 64, g, b * p.S + ti.r0, bar);
+                        tma_load_3d(dst + bx * C::BOX_BYTES, &kn_map, bx * 64, g, (l_rel * p.B + b) * p.S + ti.r0, bar);
+                        tma_load_3d(dst + C::KV_BYTES + bx * C::BOX_BYTES, &vn_map, bx * 64, g, (l_rel * p.B + b) * p.S + ti.r0, bar);
                     }
                 }
             }
@@ -336,8 +338,8 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 for (int idx = a0 * CPR + lane; idx < a1 * CPR; idx += 32) {
                     const int tok = idx / CPR, ch = idx % CPR;
                     if (t0 + tok < p.max_tail) {
-                        const int64_t src = (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
-                        const int64_t dsto = ((((int64_t)b * p.n_layers_total + p.layer) * p.Hkv + g) * p.max_tail + t0 + tok) * D + ch * 8;
+                        const int64_t src = (int64_t)l_rel * p.kn_sl + (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
+                        const int64_t dsto = ((((int64_t)b * p.n_layers_total + layer) * p.Hkv + g) * p.max_tail + t0 + tok) * D + ch * 8;
                         *(uint4 *)(p.tail_k + dsto) = *(const uint4 *)(p.k_new + src);
                         *(uint4 *)(p.tail_v + dsto) = *(const uint4 *)(p.v_new + src);
                     }
@@ -396,7 +398,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
         const uint32_t lane_base = tmem + blk * C::COL_BLK + ((uint32_t)((warp & 3) * 32) << 16);
         // Q row -> swizzled smem (zeros for rows past R)
         {
-            const __nv_bfloat16 *qrow = p.q + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D;
+            const __nv_bfloat16 *qrow = p.q + (int64_t)l_rel * p.q_sl + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D;
             unsigned char *qb = q_s + blk * C::QBLK_BYTES;
 #pragma unroll
             for (int ch = 0; ch < D / 8; ++ch) {
@@ -503,14 +505,14 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             tc_fence_after();
             const float inv = l_rnd > 0.f ? 1.f / l_rnd : 0.f;
             const float lse = l_run > 0.f ? (m_ref + log2f(l_run)) * kLn2 : -CUDART_INF_F;
-            const int64_t orow = ((int64_t)b * p.S + tok) * p.Hq + g * G + hd;
+            const int64_t orow = (((int64_t)l_rel * p.B + b) * p.S + tok) * p.Hq + g * G + hd;
 #pragma unroll
             for (int c0 = 0; c0 < D; c0 += 32) {
                 float v[32];
                 tmem_ld32(lane_base + C::COL_O + c0, v);   // warp-collective: every lane loads, real rows store
                 if (real) {
                     if (p.n_split == 1) {
-                        __nv_bfloat16 *dst = p.out + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D + c0;
+                        __nv_bfloat16 *dst = p.out + (int64_t)l_rel * p.q_sl + (int64_t)b * p.q_sb + (int64_t)tok * p.q_ss + (int64_t)(g * G + hd) * D + c0;
 #pragma unroll
                         for (int ch = 0; ch < 4; ++ch)
                             *(uint4 *)(dst + ch * 8) = make_uint4(
@@ -565,20 +567,20 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     p.reqs = t->d_reqs; p.segs = t->d_segs; p.tmaps = t->d_tmaps; p.n_seg_total = t->n_seg_total;
     p.tail_len = t->d_tail_len; p.tail_k = t->tail_k; p.tail_v = t->tail_v;
     p.q = a.q; p.k_new = a.k_new; p.v_new = a.v_new; p.out = a.out; p.lse_out = a.lse_out;
-    p.q_sb = a.q_sb; p.q_ss = a.q_ss; p.kn_sb = a.kn_sb; p.kn_ss = a.kn_ss;
-    p.layer = a.layer0; p.n_layers_total = c.n_layers; p.B = t->batch; p.S = a.S; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads;
+    p.q_sl = a.q_sl; p.q_sb = a.q_sb; p.q_ss = a.q_ss; p.kn_sl = a.kn_sl; p.kn_sb = a.kn_sb; p.kn_ss = a.kn_ss;
+    p.layer0 = a.layer0; p.n_layers_launch = a.n_layers_launch; p.n_layers_total = c.n_layers; p.B = t->batch; p.S = a.S; p.Hq = c.n_q_heads; p.Hkv = c.n_kv_heads;
     p.max_tail = c.max_tail_tokens;
     // two row blocks per CTA when the (request, KV head) has more than 128 query rows and there are still
     // enough CTAs to fill most of the SMs (otherwise one block per CTA and more KV splits)
     const int R = a.S * G;
-    const bool fill = (int64_t)t->batch * c.n_kv_heads * ((R + 255) / 256) * 10 >= 6 * (int64_t)ctx->n_sm;
+    const bool fill = (int64_t)a.n_layers_launch * t->batch * c.n_kv_heads * ((R + 255) / 256) * 10 >= 6 * (int64_t)ctx->n_sm;
     const int nblk = (R > k3::kRowsPerCta && (fill || ctx->opt_prefill_impl == 3)) ? 2 : 1;
     p.n_rb = (a.S * G + nblk * k3::kRowsPerCta - 1) / (nblk * k3::kRowsPerCta);
     p.scale_log2 = ctx->scale * k3::kLog2e;
     p.status = ctx->d_status;
     // KV splits: fill the SMs, never more splits than the shortest request has tiles, and only as many
     // as the workspace can hold partials for
-    const int64_t combos = (int64_t)t->batch * c.n_kv_heads * p.n_rb;
+    const int64_t combos = (int64_t)a.n_layers_launch * t->batch * c.n_kv_heads * p.n_rb;
     int min_tiles = 1 << 30;
     for (int b = 0; b < t->batch; ++b)
         min_tiles = std::min(min_tiles, t->h_reqs[b].chunk_tiles + k3::cdiv(t->tail_len_host, kTile) + k3::cdiv(a.S, kTile));
@@ -587,7 +589,7 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     // the partials live in the workspace's partial regions (its head holds the streaming kernel's counters)
     WorkspaceView ws;
     workspace_bytes_for(c, &ws, ctx->workspace);
-    const int64_t rows = (int64_t)t->batch * a.S * c.n_q_heads;
+    const int64_t rows = (int64_t)a.n_layers_launch * t->batch * a.S * c.n_q_heads;
     ns = std::min<int64_t>(ns, std::max<int64_t>(1, ws.n_part_slots * kUnitRows / rows));
     ns = std::min<int64_t>(ns, 64);
     p.n_split = (int)ns;
@@ -596,8 +598,9 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     const int64_t grid = combos * p.n_split;
     CUtensorMap kn_map, vn_map;
     {
-        int rc2 = encode_new_rows_map(&kn_map, a.k_new, D, c.n_kv_heads, (uint64_t)t->batch * a.S);
-        if (!rc2) rc2 = encode_new_rows_map(&vn_map, a.v_new, D, c.n_kv_heads, (uint64_t)t->batch * a.S);
+        const uint64_t n_tok = (uint64_t)a.n_layers_launch * t->batch * a.S;
+        int rc2 = encode_new_rows_map(&kn_map, a.k_new, D, c.n_kv_heads, n_tok);
+        if (!rc2) rc2 = encode_new_rows_map(&vn_map, a.v_new, D, c.n_kv_heads, n_tok);
         if (rc2) return rc2;
     }
     int rc = fail(MATKV_E_INVALID_ARG, "tensor-core prefill: unsupported head_dim %d / group %d", D, G);

@@ -91,6 +91,14 @@ class Session:
                                 out.data_ptr(), lse.data_ptr() if want_lse else None, stream)
         return out, lse
 
+    def prefill_all_layers(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, want_lse=True, stream: int = 0):
+        L, B, S = q.shape[0], q.shape[1], q.shape[2]
+        out = torch.empty_like(q)
+        lse = torch.empty((L, B, S, self.Hq), dtype=torch.float32, device=self.dev) if want_lse else None
+        mk.matkv_attend_prefill_all_layers(self.ctx, self.table, S, q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
+                                           out.data_ptr(), lse.data_ptr() if want_lse else None, stream)
+        return out, lse
+
     def decode(self, layer: int, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, want_lse=True, stream: int = 0):
         out = torch.empty_like(q)
         lse = torch.empty((q.shape[0], self.Hq), dtype=torch.float32, device=self.dev) if want_lse else None

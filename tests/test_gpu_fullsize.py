@@ -34,7 +34,8 @@ def test_cfg2_full_size_sampled_units():
                    (q_dc, mi.STREAM_Q_DECODE), (k_dc, mi.STREAM_K_DECODE), (v_dc, mi.STREAM_V_DECODE)):
         gen.fill_bf16(t_, w.seed, st)
     sess.build_table(ids)
-    pf = [sess.prefill(layer, q_pf[layer], k_pf[layer], v_pf[layer]) for layer in range(L)]
+    pf_out, pf_lse = sess.prefill_all_layers(q_pf, k_pf, v_pf)       # one launch for all layers, as the bench does
+    pf = [(pf_out[layer], pf_lse[layer]) for layer in range(L)]
     sess.advance(S)
     dc = []
     for t in range(T):

@@ -62,12 +62,19 @@ def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=Fal
             worst[i] = max(worst[i], m[i])
 
     if S > 0:
+        qs = [rand_bits(seed, 10 + layer, (B, S, Hq, D), q_shift) for layer in range(L)]
+        ks = [rand_bits(seed, 40 + layer, (B, S, Hkv, D)) for layer in range(L)]
+        vs = [rand_bits(seed, 70 + layer, (B, S, Hkv, D)) for layer in range(L)]
+        if all_layers:      # one launch for the sub-prefill of every layer
+            out_all, lse_all = sess.prefill_all_layers(_dev(np.stack(qs)), _dev(np.stack(ks)), _dev(np.stack(vs)))
+            ob_all, lb_all = _bits(out_all), lse_all.cpu().numpy()
         for layer in range(L):
-            q = rand_bits(seed, 10 + layer, (B, S, Hq, D), q_shift)
-            k = rand_bits(seed, 40 + layer, (B, S, Hkv, D))
-            v = rand_bits(seed, 70 + layer, (B, S, Hkv, D))
-            out, lse = sess.prefill(layer, _dev(q), _dev(k), _dev(v))
-            ob, lb = _bits(out), lse.cpu().numpy()
+            q, k, v = qs[layer], ks[layer], vs[layer]
+            if all_layers:
+                ob, lb = ob_all[layer], lb_all[layer]
+            else:
+                out, lse = sess.prefill(layer, _dev(q), _dev(k), _dev(v))
+                ob, lb = _bits(out), lse.cpu().numpy()
             for r in range(B):
                 o_ref, l_ref = reqs[r].attend_new(layer, q[r], k[r], v[r])
                 upd(check(ob[r], o_ref, lb[r], l_ref, f"prefill layer {layer} req {r}"))
@@ -125,6 +132,11 @@ def test_tail_crosses_tile_boundaries():
 
 def test_all_layers_launch_matches_oracle():
     run_requests(3, 8, 2, 128, [[200, 31], [97]], 4, 3, seed=24, all_layers=True)
+
+
+@pytest.mark.parametrize("S,impl", [(40, 2), (70, 3), (5, 1)])
+def test_all_layers_prefill_launch(S, impl):
+    run_requests(3, 32, 8, 128, [[200, 31], [97]], S, 2, seed=27, all_layers=True, prefill_impl=impl)
 
 
 def test_peaky_queries():
