@@ -403,6 +403,9 @@ def main():
     sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
     if args.decode_ctas:
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, args.decode_ctas)
+    fused_advance = args.decode_launch == "all_layers"
+    if fused_advance:   # the all-layers decode launch moves the tail itself: no separate counter kernel per step
+        mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_ADVANCES_TAIL, 1)
     # every rank works on its own replica of the batch (independent requests: no data-path collective)
     chunks = {}
     pool = torch.empty((len(needed), L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
@@ -476,7 +479,10 @@ def main():
             if mode == "all_layers":
                 mk.matkv_attend_decode_all_layers(ctx, table, q_dc_p + t * qd_t, k_dc_p + t * kd_t, v_dc_p + t * kd_t,
                                                   o_dc.data_ptr() + t * qd_t, None, sp)
-                n += 2
+                n += 1
+                if fused_advance:
+                    continue
+                n += 1
             else:
                 for layer in range(L):
                     mk.matkv_attend_decode(ctx, table, layer, q_dc_p + t * qd_t + layer * qd_l, k_dc_p + t * kd_t + layer * kd_l,

@@ -85,6 +85,9 @@ typedef struct {
 #define MATKV_OPT_STAGE_CTAS    4  /* 0 = stage host blobs with the copy engine (cudaMemcpyAsync); n > 0 = with a copy
                                       kernel of n small CTAs that runs beside the decode CTAs (the host blobs must
                                       then be pinned, device-accessible memory) */
+#define MATKV_OPT_DECODE_ADVANCES_TAIL 5  /* 1 = matkv_attend_decode_all_layers adds one token to every request's tail
+                                             length itself when the launch is done (its last CTA does it), so the caller
+                                             omits matkv_table_advance between decode steps; 0 (default) = it does not */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
 
 /* ---- context -------------------------------------------------------------------------- */

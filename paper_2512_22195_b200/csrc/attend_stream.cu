@@ -53,6 +53,8 @@ struct StreamParams {
     float *part_lse, *part_o;
     int64_t n_part_slots, n_counter_slots;
     int32_t *status;
+    int32_t advance;      // > 0: the last CTA to finish adds this to every request's tail length
+    int32_t *done_count;  // CTAs of the launch that have finished (reset by the last one)
 };
 
 // ---- PTX helpers ---------------------------------------------------------------------------------
@@ -347,7 +349,26 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
     }
     __syncthreads();
     const int64_t f_begin = range->begin, f_end = range->end, W = range->W;
-    if (f_begin >= f_end) return;
+    // the fused tail advance: the last CTA of the launch to get here moves every request's tail length
+    auto finish_cta = [&]() {
+        if (p.advance <= 0) return;
+        __threadfence();
+        if (atomicAdd(p.done_count, 1) == (int)gridDim.x - 1) {
+            for (int b = 0; b < p.B; ++b) {
+                int32_t v = p.tail_len[b] + p.advance;
+                if (v > p.max_tail) {
+                    v = p.max_tail;
+                    atomicCAS(p.status, 0, MATKV_E_CAPACITY);
+                }
+                const_cast<int32_t *>(p.tail_len)[b] = v;
+            }
+            *p.done_count = 0;
+        }
+    };
+    if (f_begin >= f_end) {
+        if (tid == 0) finish_cta();
+        return;
+    }
     const uint32_t ring_u32 = smem_u32(ring), full_u32 = smem_u32(bars), empty_u32 = smem_u32(bars + C::NSTAGE);
 
     if (warp == kCW) {
@@ -634,6 +655,7 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
         if (f_unit < f_end) next_unit(p, u, n_blk);
     }
     if (flags[0] && tid == 0) atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
+    if (tid == 0) finish_cta();   // after the last consumer barrier: every tile of this CTA has been consumed
 }
 
 // ---- launchers --------------------------------------------------------------------------------------
@@ -674,6 +696,8 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     p.counters = ws.counters; p.part_lse = ws.part_lse; p.part_o = ws.part_o;
     p.n_part_slots = ws.n_part_slots; p.n_counter_slots = ws.n_counter_slots;
     p.status = ctx->d_status;
+    p.advance = a.advance;
+    p.done_count = ctx->d_status + 2;
     const int64_t n_units = (int64_t)a.n_layers_launch * t->batch * n_blk * c.n_kv_heads;
     if (n_units > ws.n_counter_slots)
         return fail(MATKV_E_CAPACITY, "launch of %lld units exceeds the workspace's %lld", (long long)n_units,
@@ -784,6 +808,8 @@ extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_
         p.part_o = (float *)((char *)base + kStaticCounterBytes + kStaticLseBytes);
         p.n_part_slots = kStaticParts; p.n_counter_slots = kStaticUnits;
         p.status = ctx->d_status;
+        p.advance = 0;
+        p.done_count = ctx->d_status + 2;
         CUtensorMap kn_map, vn_map;
         rc = encode_new_rows_map(&kn_map, k_new, c.head_dim, c.n_kv_heads, (uint64_t)t->batch);
         if (!rc) rc = encode_new_rows_map(&vn_map, v_new, c.head_dim, c.n_kv_heads, (uint64_t)t->batch);

@@ -250,6 +250,10 @@ int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
             if (value < 0 || value > 3) return fail(MATKV_E_INVALID_ARG, "prefill impl must be 0..3");
             ctx->opt_prefill_impl = value;
             return MATKV_OK;
+        case MATKV_OPT_DECODE_ADVANCES_TAIL:
+            if (value < 0 || value > 1) return fail(MATKV_E_INVALID_ARG, "decode-advances-tail must be 0 or 1");
+            ctx->opt_fused_advance = value;
+            return MATKV_OK;
         case MATKV_OPT_STAGE_CTAS:
             if (value < 0 || value > 148) return fail(MATKV_E_INVALID_ARG, "staging CTAs must be 0..148");
             ctx->opt_stage_ctas = value;
@@ -743,7 +747,10 @@ int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *t, const void *q
         rc = launch_rope(ctx, t, a, (cudaStream_t)stream);
         if (rc) return rc;
     }
-    return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+    a.advance = ctx->opt_fused_advance ? 1 : 0;   // the launch itself moves the tail by one token when it is done
+    rc = launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+    if (rc == MATKV_OK && a.advance) t->tail_len_host += 1;
+    return rc;
 }
 
 int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t S, const void *q, const void *kn,

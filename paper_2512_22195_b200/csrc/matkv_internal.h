@@ -75,7 +75,7 @@ struct matkv_ctx {
     int32_t *d_status = nullptr;
     void *workspace = nullptr;
     size_t workspace_bytes = 0;
-    int64_t opt_decode_ctas = 0, opt_prefill_impl = 0, opt_prefill_ctas = 0, opt_stage_ctas = 0;
+    int64_t opt_decode_ctas = 0, opt_prefill_impl = 0, opt_prefill_ctas = 0, opt_stage_ctas = 0, opt_fused_advance = 0;
     std::unordered_map<uint64_t, matkv::Chunk> chunks;
     std::map<void *, matkv::Region *> regions;
     std::unordered_map<uint64_t, matkv::Ticket> tickets;
@@ -142,6 +142,7 @@ struct AttendArgs {
     int64_t q_sl, q_sb, q_ss;     // q / out strides: layer, request, token (elements)
     int64_t kn_sl, kn_sb, kn_ss;  // k_new / v_new strides
     int64_t lse_sl, lse_sb, lse_ss;
+    int32_t advance = 0;          // streaming kernel only: tokens the launch adds to the tail lengths when it is done
 };
 int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
 int launch_rope(matkv_ctx *ctx, matkv_table *t, AttendArgs &a, cudaStream_t stream);

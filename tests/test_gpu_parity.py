@@ -28,7 +28,7 @@ def _bits(t):
 
 
 def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=False, q_shift=0, cap=None,
-                 prefill_impl=0, prefill_ctas=0, rope_theta=0.0, pos_mode=0):
+                 prefill_impl=0, prefill_ctas=0, rope_theta=0.0, pos_mode=0, fused_advance=False):
     """Prefill S tokens then T decode steps for a batch; compare every output with the oracle."""
     import paper_2512_22195_b200 as mk
     B = len(lens_per_req)
@@ -40,6 +40,8 @@ def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=Fal
         mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_IMPL, prefill_impl)
     if prefill_ctas:
         mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_CTAS, prefill_ctas)
+    if fused_advance:
+        mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_ADVANCES_TAIL, 1)
     sh = oracle.Shape(L, Hq, Hkv, D)
     blobs, ids, cid = {}, [], 0
     for r, lens in enumerate(lens_per_req):
@@ -97,7 +99,8 @@ def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=Fal
             for r in range(B):
                 o_ref, l_ref = reqs[r].attend_new(layer, q[layer, r][None], k[layer, r][None], v[layer, r][None])
                 upd(check(ob[layer, r], o_ref[0], lb[layer, r], l_ref[0], f"decode step {t} layer {layer} req {r}"))
-        sess.advance(1)
+        if not (fused_advance and all_layers):
+            sess.advance(1)
         for r in reqs:
             r.advance(1)
     # the tails the kernels wrote must equal the oracle's bookkeeping bit for bit
@@ -137,6 +140,11 @@ def test_all_layers_launch_matches_oracle():
 @pytest.mark.parametrize("S,impl", [(40, 2), (70, 3), (5, 1)])
 def test_all_layers_prefill_launch(S, impl):
     run_requests(3, 32, 8, 128, [[200, 31], [97]], S, 2, seed=27, all_layers=True, prefill_impl=impl)
+
+
+@pytest.mark.parametrize("ctas", [0, 3, 1000])
+def test_decode_launch_that_advances_the_tail_itself(ctas):
+    run_requests(2, 8, 2, 128, [[200, 31], [97], []], 3, 5, seed=28, all_layers=True, fused_advance=True, ctas=ctas)
 
 
 def test_peaky_queries():
