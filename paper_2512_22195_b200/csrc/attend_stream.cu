@@ -245,6 +245,42 @@ __device__ __forceinline__ int cta_of(int64_t f, int64_t W, int64_t n) { return 
 __device__ void combine_warp(const float *o_parts, int64_t o_stride, const float *lse_parts, int64_t lse_stride, int P,
                              int D, __nv_bfloat16 *out, float *lse_out) {
     const int lane = threadIdx.x & 31;
+    const int dpl = D >> 5;  // every lane owns D/32 consecutive dims
+    if (P <= 32 && dpl == 4) {
+        // common case (at most 32 parts, D = 128): one part's lse per lane, a single round trip for them,
+        // then the parts' rows 16 loads at a time; weights travel by shuffle
+        const float lse_l = lane < P ? __ldcg(lse_parts + lane * lse_stride) : -CUDART_INF_F;
+        float m = lse_l;
+#pragma unroll
+        for (int off = 16; off; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+        if (m == -CUDART_INF_F) {  // no part saw any key
+            *(uint2 *)(out + lane * 4) = make_uint2(0u, 0u);
+            if (lse_out && lane == 0) *lse_out = -CUDART_INF_F;
+            return;
+        }
+        float w_l = lse_l == -CUDART_INF_F ? 0.f : exp2f((lse_l - m) * kLog2e);
+        float z = w_l;
+#pragma unroll
+        for (int off = 16; off; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
+        w_l /= z;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p0 = 0; p0 < P; p0 += 16) {
+            float4 v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                v[i] = p0 + i < P ? __ldcg((const float4 *)(o_parts + (p0 + i) * o_stride + lane * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float w = __shfl_sync(0xffffffffu, w_l, (p0 + i) & 31);
+                acc.x = fmaf(w, v[i].x, acc.x); acc.y = fmaf(w, v[i].y, acc.y);
+                acc.z = fmaf(w, v[i].z, acc.z); acc.w = fmaf(w, v[i].w, acc.w);
+            }
+        }
+        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        *(uint2 *)(out + lane * 4) = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+        if (lse_out && lane == 0) *lse_out = m + logf(z);
+        return;
+    }
     float m = -CUDART_INF_F;
     for (int p = lane; p < P; p += 32) m = fmaxf(m, __ldcg(lse_parts + p * lse_stride));
 #pragma unroll
@@ -259,9 +295,8 @@ __device__ void combine_warp(const float *o_parts, int64_t o_stride, const float
 #pragma unroll
     for (int off = 16; off; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
     const float lse = m + logf(z);
-    // every lane owns D/32 consecutive dims; the weights of 32 parts at a time sit one per lane and are
-    // broadcast by shuffle, so the loads of the parts' rows are independent and stay in flight together
-    const int dpl = D >> 5;
+    // the weights of 32 parts at a time sit one per lane and are broadcast by shuffle, so the loads of the
+    // parts' rows are independent and stay in flight together
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     for (int p0 = 0; p0 < P; p0 += 32) {
         const float w_mine = p0 + lane < P ? exp2f((__ldcg(lse_parts + (p0 + lane) * lse_stride) - lse) * kLog2e) : 0.f;

@@ -190,6 +190,8 @@ int matkv_create(const matkv_config *cfg, matkv_ctx **out) {
         return fail(MATKV_E_INVALID_ARG, "matkv_create: query heads per KV head must be 1, 2, 4 or 8");
     if (cfg->max_batch < 1 || cfg->max_batch > 1024 || cfg->max_chunks_per_req < 0 || cfg->max_tail_tokens < 1)
         return fail(MATKV_E_INVALID_ARG, "matkv_create: bad capacity");
+    if ((int64_t)cfg->max_batch * cfg->n_layers * cfg->n_kv_heads * cfg->max_tail_tokens >= (int64_t)1 << 31)
+        return fail(MATKV_E_CAPACITY, "matkv_create: max_batch x layers x KV heads x max_tail_tokens must stay below 2^31 rows");
     if (cfg->softmax_scale < 0.f || cfg->rope_theta < 0.f || cfg->pos_mode < 0 || cfg->pos_mode > 1)
         return fail(MATKV_E_INVALID_ARG, "matkv_create: bad scale / rotary settings");
     int dev = cfg->device;
@@ -298,6 +300,8 @@ int matkv_status(matkv_ctx *ctx, int32_t *dev_status_out, int32_t clear) {
 int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const void *host_blob, void *dev_blob) {
     if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_register_chunk: null context");
     if (n_tokens < 1) return fail(MATKV_E_INVALID_ARG, "chunk %llu: n_tokens must be >= 1", (unsigned long long)chunk_id);
+    if ((int64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * n_tokens >= (int64_t)1 << 31)
+        return fail(MATKV_E_CAPACITY, "chunk %llu: layers x 2 x KV heads x tokens must stay below 2^31 rows", (unsigned long long)chunk_id);
     if (!host_blob && !dev_blob) return fail(MATKV_E_INVALID_ARG, "chunk %llu: no blob given", (unsigned long long)chunk_id);
     if (dev_blob && (uintptr_t)dev_blob % 256)
         return fail(MATKV_E_ALIGNMENT, "chunk %llu: device blob must be 256-byte aligned", (unsigned long long)chunk_id);
@@ -320,6 +324,8 @@ int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, co
 int matkv_register_chunk_file(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const char *path, uint64_t file_offset) {
     if (!ctx || !path) return fail(MATKV_E_INVALID_ARG, "matkv_register_chunk_file: null argument");
     if (n_tokens < 1) return fail(MATKV_E_INVALID_ARG, "chunk %llu: n_tokens must be >= 1", (unsigned long long)chunk_id);
+    if ((int64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * n_tokens >= (int64_t)1 << 31)
+        return fail(MATKV_E_CAPACITY, "chunk %llu: layers x 2 x KV heads x tokens must stay below 2^31 rows", (unsigned long long)chunk_id);
     if (ctx->chunks.count(chunk_id))
         return fail(MATKV_E_INVALID_ARG, "chunk %llu is already registered", (unsigned long long)chunk_id);
     Chunk c;
