@@ -365,6 +365,8 @@ def main():
                     "engine; -1 = auto: 16 CTAs in the pipelined-serving mode (long decode launches that saturate HBM starve "
                     "the copy engine), copy engine in the single-batch end-to-end leg (short launches: a co-resident copy "
                     "CTA makes its SM the straggler of every launch)")
+    ap.add_argument("--decode-impl", type=int, default=0, choices=[0, 1, 2],
+                    help="decode kernel: 0 auto (chunk-major when the batch's requests share chunks), 1 request-major, 2 chunk-major")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (small profiling cases)")
     args = ap.parse_args()
@@ -403,6 +405,8 @@ def main():
     sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
     if args.decode_ctas:
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, args.decode_ctas)
+    if args.decode_impl:
+        mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, args.decode_impl)
     fused_advance = args.decode_launch == "all_layers"
     if fused_advance:   # the all-layers decode launch moves the tail itself: no separate counter kernel per step
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_ADVANCES_TAIL, 1)
@@ -559,6 +563,9 @@ def main():
     achieved = kv_bytes_decode / decode_launches / (avg_launch_ms * 1e-3) / 1e9
     peaks, peak_kind = measured_peaks()
     peak = float(peaks["hbm_gbs"])
+    # chunk tiles the batch lists against the tiles the decode kernel in use reads (chunk-major stacking)
+    tiles_logical, tiles_read = mk.matkv_table_sharing(sess.table)
+    chunk_major = args.decode_impl == 2 or (args.decode_impl == 0 and tiles_logical * 4 >= tiles_read * 5)
     result = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -569,7 +576,9 @@ def main():
                    f"{kv_bytes_decode / T / 1e6:.0f} MB vs 126 MB L2)", "multi_gpu": "independent replicas per rank"},
         "gpu_launches": n_launch,
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "kernel": "k_attend_stream (decode)", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "k_attend_shared (chunk-major decode)" if chunk_major else "k_attend_stream (decode)",
+                     "chunk_tiles_listed_vs_read": [tiles_logical, tiles_read if chunk_major else tiles_logical],
+                     "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                      "read_probe_gbs_same_run": probe_gbs,

@@ -88,6 +88,10 @@ typedef struct {
 #define MATKV_OPT_DECODE_ADVANCES_TAIL 5  /* 1 = matkv_attend_decode_all_layers adds one token to every request's tail
                                              length itself when the launch is done (its last CTA does it), so the caller
                                              omits matkv_table_advance between decode steps; 0 (default) = it does not */
+#define MATKV_OPT_DECODE_IMPL   6  /* decode kernel: 0 = auto (chunk-major when the batch's requests share chunks and the
+                                      workspace has room for its partials), 1 = request-major always, 2 = chunk-major
+                                      always (MATKV_E_CAPACITY when the workspace is too small) */
+#define MATKV_OPT_SHARE_TILES   7  /* chunk-major decode: 64-token tiles per work item (default 16); read when a table is built */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
 
 /* ---- context -------------------------------------------------------------------------- */
@@ -209,6 +213,22 @@ int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *table, const voi
  *     streams, or different contexts on one device) race on it: serialise them.                      */
 int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *table, int32_t layer, const void *q, const void *k_new,
                                const void *v_new, void *out, float *lse_out, void *stream);
+
+/* Chunk-major decode for batches whose requests share chunks (the paper's skewed retrieval: a few
+ * materialised chunks take most of the hits, Section V).  matkv_attend_decode and
+ * matkv_attend_decode_all_layers then read a chunk listed by several requests of the table ONCE per
+ * layer and KV head: the requests' query heads are stacked into one tensor-core tile (16 / G requests;
+ * more requests repeat the read right away, where it hits L2), every (chunk, request) pair leaves a
+ * partial result and the last one merges the request's partials by log-sum-exp.  Same results as the
+ * request-major kernel up to summation order.  Two chunks are "the same" when they resolve to the same
+ * device copy and length.
+ *   matkv_table_sharing: chunk tiles (64 tokens) the table's requests list per layer and KV head, and
+ *     the tiles the chunk-major kernel reads for them (either pointer may be NULL).
+ *   matkv_table_workspace_bytes: size the workspace given to matkv_set_workspace must have for
+ *     chunk-major launches of n_layers_launch layers on this table (never less than
+ *     matkv_workspace_bytes); with a smaller workspace the automatic choice stays request-major.      */
+int matkv_table_sharing(const matkv_table *table, int64_t *logical_tiles_out, int64_t *read_tiles_out);
+size_t matkv_table_workspace_bytes(const matkv_table *table, int32_t n_layers_launch);
 
 /* a6 alone: merges n_parts partial attentions per row.  o_parts [n_rows][n_parts][D] fp32
  * (each normalised within its part), lse_parts [n_rows][n_parts] fp32 natural log (-inf =

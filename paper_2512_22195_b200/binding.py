@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(HERE, "libmatkv.so")
 OK, E_INVALID_ARG, E_UNKNOWN_CHUNK, E_NOT_STAGED, E_NOT_READY = 0, -1, -2, -3, -4
 E_CAPACITY, E_ALIGNMENT, E_CUDA, E_TIMEOUT, E_BOUNDS, E_IO = -5, -6, -7, -8, -9, -10
 OPT_DECODE_CTAS, OPT_PREFILL_IMPL, OPT_PREFILL_CTAS, OPT_STAGE_CTAS, OPT_DECODE_ADVANCES_TAIL = 1, 2, 3, 4, 5
+OPT_DECODE_IMPL, OPT_SHARE_TILES = 6, 7
 
 EXPORTS = [
     "matkv_create", "matkv_destroy", "matkv_last_error", "matkv_set_option", "matkv_workspace_bytes",
@@ -26,7 +27,7 @@ EXPORTS = [
     "matkv_attend_decode", "matkv_attend_decode_all_layers", "matkv_lse_combine", "matkv_gather_debug",
     "matkv_probe_read", "matkv_attend_decode_static", "matkv_selftest_wait_timeout",
     "matkv_register_chunk_file", "matkv_set_bounce_buffer", "matkv_export_tail_as_chunk",
-    "matkv_attend_prefill_all_layers",
+    "matkv_attend_prefill_all_layers", "matkv_table_sharing", "matkv_table_workspace_bytes",
 ]
 
 
@@ -84,6 +85,8 @@ def lib() -> C.CDLL:
             "matkv_set_bounce_buffer": (C.c_int, [vp, vp, C.c_size_t, C.c_size_t, i32]),
             "matkv_export_tail_as_chunk": (C.c_int, [vp, vp, i32, i32, vp, vp, vp]),
             "matkv_attend_prefill_all_layers": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp]),
+            "matkv_table_sharing": (C.c_int, [vp, C.POINTER(i64), C.POINTER(i64)]),
+            "matkv_table_workspace_bytes": (C.c_size_t, [vp, i32]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -245,3 +248,14 @@ def matkv_export_tail_as_chunk(ctx: int, table: int, req: int, n_tokens: int, de
 def matkv_attend_prefill_all_layers(ctx: int, table: int, S: int, q: int, k_new: int, v_new: int, out: int,
                                     lse_out: Optional[int] = None, stream: int = 0) -> None:
     _check(lib().matkv_attend_prefill_all_layers(ctx, table, S, q, k_new, v_new, out, lse_out or None, stream or None))
+
+
+def matkv_table_sharing(table: int):
+    """(chunk tiles the table's requests list, chunk tiles the chunk-major decode reads) per layer and KV head."""
+    a, b = C.c_int64(0), C.c_int64(0)
+    _check(lib().matkv_table_sharing(table, C.byref(a), C.byref(b)))
+    return a.value, b.value
+
+
+def matkv_table_workspace_bytes(table: int, n_layers_launch: int) -> int:
+    return int(lib().matkv_table_workspace_bytes(table, n_layers_launch))

@@ -260,6 +260,14 @@ int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
             if (value < 0 || value > 148) return fail(MATKV_E_INVALID_ARG, "staging CTAs must be 0..148");
             ctx->opt_stage_ctas = value;
             return MATKV_OK;
+        case MATKV_OPT_DECODE_IMPL:
+            if (value < 0 || value > 2) return fail(MATKV_E_INVALID_ARG, "decode impl must be 0..2");
+            ctx->opt_decode_impl = value;
+            return MATKV_OK;
+        case MATKV_OPT_SHARE_TILES:
+            if (value < 1 || value > 1024) return fail(MATKV_E_INVALID_ARG, "tiles per chunk-major item must be 1..1024");
+            ctx->opt_share_tiles = value;
+            return MATKV_OK;
         case MATKV_OPT_PREFILL_CTAS:
             if (value < 0 || value > 64) return fail(MATKV_E_INVALID_ARG, "prefill CTAs per head must be 0..64");
             ctx->opt_prefill_ctas = value;
@@ -580,11 +588,64 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     }
     t->n_seg_total = (int32_t)t->h_segs.size();
 
+    // chunk-major decode: requests that list the same device copy of a chunk are stacked, 16 / G per item,
+    // so that the chunk's rows are read once for all of them; a long chunk is cut into items of at most
+    // opt_share_tiles tiles.  Every (item, request) pair produces one partial, the request's tail one more.
+    std::vector<DevItem> items;
+    {
+        const int G = ctx->cfg.n_q_heads / ctx->cfg.n_kv_heads;
+        const int R = (G >= 1 && G <= kShareRows && kShareRows % G == 0) ? kShareRows / G : 0;
+        const int T = (int)ctx->opt_share_tiles;
+        std::map<std::pair<const void *, int32_t>, std::vector<std::pair<int32_t, int32_t>>> members;  // -> (request, segment)
+        std::vector<int32_t> part_off(t->h_segs.size(), 0);
+        int32_t part_base = 0;
+        for (int32_t r = 0; r < batch; ++r) {
+            DevReq &rq = t->h_reqs[r];
+            int32_t n = 0;
+            for (int32_t i = 0; i < rq.n_seg; ++i) {
+                const int32_t si = rq.seg_begin + i;
+                const DevSeg &sg = t->h_segs[si];
+                members[{(const void *)sg.base, sg.len}].push_back({r, si});
+                part_off[si] = n;
+                n += ((sg.len + kTile - 1) / kTile + T - 1) / T;
+            }
+            rq.n_parts = n + 1;
+            rq.part_base = part_base;
+            part_base += rq.n_parts;
+        }
+        t->parts_total = part_base;
+        if (R > 0) {
+            for (auto &kv : members) {
+                const int32_t len = kv.first.second, tiles = (len + kTile - 1) / kTile;
+                const auto &m = kv.second;
+                for (int32_t tile0 = 0, sub = 0; tile0 < tiles; tile0 += T, ++sub)
+                    for (size_t j0 = 0; j0 < m.size(); j0 += R) {
+                        DevItem it;
+                        memset(&it, 0, sizeof it);
+                        it.tmap = m[j0].second;
+                        it.len = len;
+                        it.tile0 = tile0;
+                        it.n_tiles = std::min(T, tiles - tile0);
+                        it.n_req = (int32_t)std::min<size_t>(R, m.size() - j0);
+                        for (int32_t j = 0; j < it.n_req; ++j) {
+                            it.req[j] = m[j0 + j].first;
+                            it.part[j] = part_off[m[j0 + j].second] + sub;
+                        }
+                        t->item_tiles += it.n_tiles;
+                        items.push_back(it);
+                    }
+            }
+            t->n_items = (int32_t)items.size();
+            t->share_ok = true;
+        }
+    }
+
     const size_t segs_bytes = align_up(sizeof(DevSeg) * std::max<size_t>(t->h_segs.size(), 1), 256);
     const size_t reqs_bytes = align_up(sizeof(DevReq) * (size_t)batch, 256);
     const size_t tl_bytes = align_up(sizeof(int32_t) * (size_t)batch, 256);
-    const size_t maps_bytes = sizeof(CUtensorMap) * (seg_maps.size() + 2);
-    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes + maps_bytes;
+    const size_t maps_bytes = align_up(sizeof(CUtensorMap) * (seg_maps.size() + 2), 256);
+    const size_t items_bytes = sizeof(DevItem) * std::max<size_t>(items.size(), 1);
+    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes + maps_bytes + items_bytes;
     CUtensorMap tail_maps[2];
     {
         const uint64_t tail_rows = (uint64_t)batch * ctx->cfg.n_layers * ctx->cfg.n_kv_heads * ctx->cfg.max_tail_tokens;
@@ -625,6 +686,9 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     t->d_reqs = (DevReq *)((char *)t->d_image + segs_bytes);
     t->d_tail_len = (int32_t *)((char *)t->d_image + segs_bytes + reqs_bytes);
     t->d_tmaps = (CUtensorMap *)((char *)t->d_image + segs_bytes + reqs_bytes + tl_bytes);
+    t->d_items = (DevItem *)((char *)t->d_image + segs_bytes + reqs_bytes + tl_bytes + maps_bytes);
+    if (!items.empty())
+        memcpy((char *)t->h_pinned + segs_bytes + reqs_bytes + tl_bytes + maps_bytes, items.data(), sizeof(DevItem) * items.size());
     {
         CUtensorMap *hm = (CUtensorMap *)((char *)t->h_pinned + segs_bytes + reqs_bytes + tl_bytes);
         for (size_t i = 0; i < seg_maps.size(); ++i) memcpy(hm + i, seg_maps[i], sizeof(CUtensorMap));
@@ -705,6 +769,67 @@ static int check_attend(matkv_ctx *ctx, matkv_table *t, const void *q, const voi
     return MATKV_OK;
 }
 
+// Where the chunk-major decode may keep its partials: the part of the configured workspace behind the
+// arrival counters (in front of the rotary scratch) if that is large enough, else whatever the caller's
+// workspace holds beyond the configured size.
+static bool shared_region(matkv_ctx *ctx, const matkv_table *t, int n_layers_launch, void **region, size_t *bytes) {
+    WorkspaceView v;
+    const size_t cfg_bytes = workspace_bytes_for(ctx->cfg, &v, ctx->workspace);
+    const size_t need = shared_region_bytes(ctx->cfg, t, n_layers_launch);
+    const size_t a_off = (size_t)((char *)v.part_lse - (char *)ctx->workspace);
+    const size_t a_bytes = cfg_bytes - rope_scratch_bytes(ctx->cfg) - a_off;
+    if (need <= a_bytes) {
+        *region = (char *)ctx->workspace + a_off;
+        *bytes = a_bytes;
+        return true;
+    }
+    const size_t b_off = align_up(cfg_bytes, 256);
+    if (ctx->workspace_bytes >= b_off + need) {
+        *region = (char *)ctx->workspace + b_off;
+        *bytes = ctx->workspace_bytes - b_off;
+        return true;
+    }
+    return false;
+}
+
+// a5: picks the request-major or the chunk-major kernel for a decode launch
+static int launch_decode(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream) {
+    const int64_t impl = ctx->opt_decode_impl;
+    // automatic choice: chunk-major when stacking saves at least a fifth of the chunk reads
+    bool shared = impl == 2 || (impl == 0 && t->share_ok && t->n_items > 0 && t->total_chunk_tiles * 4 >= t->item_tiles * 5);
+    void *region = nullptr;
+    size_t region_bytes = 0;
+    if (shared) {
+        if (!t->share_ok) return fail(MATKV_E_INVALID_ARG, "chunk-major decode does not support this head grouping");
+        if (!shared_region(ctx, t, a.n_layers_launch, &region, &region_bytes)) {
+            if (impl == 2)
+                return fail(MATKV_E_CAPACITY, "chunk-major decode needs a workspace of %zu bytes (matkv_table_workspace_bytes), %zu given",
+                            matkv_table_workspace_bytes(t, a.n_layers_launch), ctx->workspace_bytes);
+            shared = false;
+        }
+    }
+    if (shared) return launch_attend_shared(ctx, t, a, region, region_bytes, stream);
+    return launch_attend_stream(ctx, t, a, stream);
+}
+
+size_t matkv_table_workspace_bytes(const matkv_table *t, int32_t n_layers_launch) {
+    if (!t || n_layers_launch < 1) return 0;
+    const matkv_config &c = t->ctx->cfg;
+    WorkspaceView v;
+    const size_t cfg_bytes = workspace_bytes_for(c, &v, nullptr);
+    const size_t need = shared_region_bytes(c, t, n_layers_launch);
+    const size_t a_off = (size_t)((char *)v.part_lse - (char *)nullptr);
+    if (need <= cfg_bytes - rope_scratch_bytes(c) - a_off) return cfg_bytes;
+    return align_up(cfg_bytes, 256) + need;
+}
+
+int matkv_table_sharing(const matkv_table *t, int64_t *logical_tiles_out, int64_t *read_tiles_out) {
+    if (!t) return fail(MATKV_E_INVALID_ARG, "matkv_table_sharing: null table");
+    if (logical_tiles_out) *logical_tiles_out = t->total_chunk_tiles;
+    if (read_tiles_out) *read_tiles_out = t->share_ok ? t->item_tiles : t->total_chunk_tiles;
+    return MATKV_OK;
+}
+
 int matkv_attend_decode(matkv_ctx *ctx, matkv_table *t, int32_t layer, const void *q, const void *kn, const void *vn,
                         void *out, float *lse_out, void *stream) {
     int rc = check_attend(ctx, t, q, kn, vn, out, 1, "matkv_attend_decode");
@@ -728,7 +853,7 @@ int matkv_attend_decode(matkv_ctx *ctx, matkv_table *t, int32_t layer, const voi
         rc = launch_rope(ctx, t, a, (cudaStream_t)stream);
         if (rc) return rc;
     }
-    return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+    return launch_decode(ctx, t, a, (cudaStream_t)stream);
 }
 
 int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *t, const void *q, const void *kn, const void *vn,
@@ -754,7 +879,7 @@ int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *t, const void *q
         if (rc) return rc;
     }
     a.advance = ctx->opt_fused_advance ? 1 : 0;   // the launch itself moves the tail by one token when it is done
-    rc = launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
+    rc = launch_decode(ctx, t, a, (cudaStream_t)stream);
     if (rc == MATKV_OK && a.advance) t->tail_len_host += 1;
     return rc;
 }

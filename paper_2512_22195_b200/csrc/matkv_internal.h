@@ -30,7 +30,22 @@ struct DevReq {
     int32_t n_chunk_tokens;  // sum of len
     int32_t chunk_tiles;     // sum of ceil(len / kTile)
     int32_t pos_base;        // rotary mode: position of tail token 0
+    int32_t n_parts;         // chunk-major decode: partial results the request collects (its items, then its tail)
+    int32_t part_base;       // chunk-major decode: first partial slot of the request inside one (layer, KV head)
+    int32_t pad;
+};
+// One work item of the chunk-major decode: up to `n_tiles` tiles of one chunk, read once for every
+// request stacked in the item (16 / G of them at most: their G query heads fill the 16 MMA rows).
+constexpr int kShareRows = 16;
+struct DevItem {
+    int32_t tmap;      // index of the chunk's descriptor
+    int32_t len;       // chunk tokens
+    int32_t tile0;     // first tile of the item inside the chunk
+    int32_t n_tiles;
+    int32_t n_req;     // requests stacked in the item
     int32_t pad[3];
+    int32_t req[kShareRows];   // request per stacked slot
+    int32_t part[kShareRows];  // index of this item's partial among that request's parts
 };
 
 // ---- host-side objects --------------------------------------------------------------------
@@ -76,6 +91,7 @@ struct matkv_ctx {
     void *workspace = nullptr;
     size_t workspace_bytes = 0;
     int64_t opt_decode_ctas = 0, opt_prefill_impl = 0, opt_prefill_ctas = 0, opt_stage_ctas = 0, opt_fused_advance = 0;
+    int64_t opt_decode_impl = 0, opt_share_tiles = 16;
     std::unordered_map<uint64_t, matkv::Chunk> chunks;
     std::map<void *, matkv::Region *> regions;
     std::unordered_map<uint64_t, matkv::Ticket> tickets;
@@ -100,6 +116,11 @@ struct matkv_table {
     matkv::DevReq *d_reqs = nullptr;
     int32_t *d_tail_len = nullptr;
     CUtensorMap *d_tmaps = nullptr;  // one per segment, then the K tail and the V tail
+    matkv::DevItem *d_items = nullptr;  // chunk-major decode: the chunk items of one (layer, KV head)
+    bool share_ok = false;              // the head grouping fits the chunk-major kernel
+    int32_t n_items = 0;                // chunk items (the requests' tail items follow implicitly)
+    int32_t parts_total = 0;            // partial slots of one (layer, KV head): sum of the requests' n_parts
+    int64_t item_tiles = 0;             // tiles the chunk items read per (layer, KV head); total_chunk_tiles is the logical count
     __nv_bfloat16 *tail_k = nullptr, *tail_v = nullptr;
     std::vector<matkv::Region *> regions;  // staged regions this table reads
 };
@@ -145,6 +166,9 @@ struct AttendArgs {
     int32_t advance = 0;          // streaming kernel only: tokens the launch adds to the tail lengths when it is done
 };
 int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
+// chunk-major decode (S = 1): region = scratch for the partials, region_bytes its size
+int launch_attend_shared(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, void *region, size_t region_bytes, cudaStream_t stream);
+size_t shared_region_bytes(const matkv_config &c, const matkv_table *t, int n_layers_launch);
 int launch_rope(matkv_ctx *ctx, matkv_table *t, AttendArgs &a, cudaStream_t stream);
 int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
 int launch_lse_combine(matkv_ctx *ctx, int32_t n_rows, int32_t n_parts, int32_t D, const float *o_parts,

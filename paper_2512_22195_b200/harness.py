@@ -77,6 +77,11 @@ class Session:
         self.batch = len(ids_per_req)
         self.table = mk.matkv_build_chunk_table(self.ctx, ids_per_req, self.tail_k.data_ptr(), self.tail_v.data_ptr(),
                                                 stream)
+        # room for the chunk-major decode's partials (all layers in one launch) when this table needs more
+        need = mk.matkv_table_workspace_bytes(self.table, self.L)
+        if need > self.workspace.numel():
+            self.workspace = torch.empty(need, dtype=torch.uint8, device=self.dev)
+            mk.matkv_set_workspace(self.ctx, self.workspace.data_ptr(), need)
         return self.table
 
     def advance(self, n: int, stream: int = 0) -> None:

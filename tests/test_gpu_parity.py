@@ -28,12 +28,19 @@ def _bits(t):
 
 
 def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=False, q_shift=0, cap=None,
-                 prefill_impl=0, prefill_ctas=0, rope_theta=0.0, pos_mode=0, fused_advance=False):
-    """Prefill S tokens then T decode steps for a batch; compare every output with the oracle."""
+                 prefill_impl=0, prefill_ctas=0, rope_theta=0.0, pos_mode=0, fused_advance=False, pool=None,
+                 decode_impl=0, share_tiles=0):
+    """Prefill S tokens then T decode steps for a batch; compare every output with the oracle.
+    lens_per_req: chunk lengths per request (every chunk its own), or, with `pool` (a list of chunk lengths),
+    indices into the pool per request, so that requests can list the same chunk."""
     import paper_2512_22195_b200 as mk
     B = len(lens_per_req)
     cap = cap or (S + T)
     sess = _session(L, Hq, Hkv, D, B, max(1, max(len(x) for x in lens_per_req)), cap, rope_theta=rope_theta, pos_mode=pos_mode)
+    if decode_impl:
+        mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, decode_impl)
+    if share_tiles:
+        mk.matkv_set_option(sess.ctx, mk.OPT_SHARE_TILES, share_tiles)
     if ctas:
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, ctas)
     if prefill_impl:
@@ -44,14 +51,20 @@ def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=Fal
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_ADVANCES_TAIL, 1)
     sh = oracle.Shape(L, Hq, Hkv, D)
     blobs, ids, cid = {}, [], 0
-    for r, lens in enumerate(lens_per_req):
-        row = []
-        for n in lens:
+    if pool is not None:
+        for cid, n in enumerate(pool):
             blobs[cid] = rand_bits(seed, 1000 + cid, (L, 2, Hkv, n, D))
             sess.register_device_chunk(cid, blobs[cid])
-            row.append(cid)
-            cid += 1
-        ids.append(row)
+        ids = [list(row) for row in lens_per_req]
+    else:
+        for r, lens in enumerate(lens_per_req):
+            row = []
+            for n in lens:
+                blobs[cid] = rand_bits(seed, 1000 + cid, (L, 2, Hkv, n, D))
+                sess.register_device_chunk(cid, blobs[cid])
+                row.append(cid)
+                cid += 1
+            ids.append(row)
     sess.build_table(ids)
     def pos_base(row):
         lens = [blobs[c].shape[3] for c in row]
@@ -363,4 +376,44 @@ def test_cfg2_shape_two_layers_sampled_steps():
         sess.advance(1)
         req.advance(1)
     assert sess.status() == 0
+    sess.close()
+
+
+# ---- chunk-major decode (requests that list the same chunks) ----------------------------------------
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 128), (32, 8, 128), (16, 2, 128), (4, 4, 64), (4, 2, 64), (8, 2, 64)])
+def test_chunk_major_decode_shared_chunks(Hq, Hkv, D):
+    """Seven requests over a pool of five chunks (ragged lengths, one listed by six requests, one request
+    listing a chunk twice, one without chunks): the chunk-major kernel against the oracle."""
+    pool = [200, 64, 33, 129, 1]
+    ids = [[0, 1], [0, 2, 3], [1, 0], [0], [3, 0, 3], [], [4, 0, 2]]
+    run_requests(2, Hq, Hkv, D, ids, 3, 4, seed=61, pool=pool, decode_impl=2)
+
+
+def test_chunk_major_decode_all_layers_fused_advance_and_small_items():
+    """One launch for all layers with the tail advanced by the launch itself; items of two tiles, so long
+    chunks are cut into several items (several partials per chunk and request); few CTAs and many."""
+    pool = [300, 130, 70]
+    ids = [[0, 1, 2], [2, 0], [0], [1, 0], [0, 2]]
+    for ctas in (3, 0):
+        run_requests(3, 8, 2, 128, ids, 2, 5, seed=62, pool=pool, decode_impl=2, share_tiles=2, all_layers=True,
+                     fused_advance=True, ctas=ctas)
+
+
+def test_chunk_major_decode_tail_grows_over_tiles():
+    """A tail that grows through 64 tokens under the chunk-major kernel (the tail item spans tiles)."""
+    run_requests(1, 4, 2, 128, [[0], [0]], 60, 10, seed=63, pool=[50], decode_impl=2)
+
+
+def test_auto_choice_matches_sharing():
+    """The automatic choice takes the chunk-major kernel only when stacking saves chunk reads."""
+    import paper_2512_22195_b200 as mk
+    sess = _session(1, 8, 2, 128, 4, 2, 8)
+    for cid, n in enumerate([128, 128, 64]):
+        sess.register_device_chunk(cid, rand_bits(5, cid, (1, 2, 2, n, 128)))
+    t = sess.build_table([[0, 1], [0, 1], [0, 2], [0]])
+    logical, read = mk.matkv_table_sharing(t)
+    assert (logical, read) == (4 + 4 + 3 + 2, 2 + 2 + 1)   # 13 tiles listed; chunks 0, 1, 2 read once each
+    t = sess.build_table([[0], [1], [2]])
+    assert mk.matkv_table_sharing(t) == (5, 5)
+    assert mk.matkv_table_workspace_bytes(t, 1) >= mk.matkv_workspace_bytes(sess.ctx)
     sess.close()
