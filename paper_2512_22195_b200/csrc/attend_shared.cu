@@ -12,14 +12,15 @@
 //
 // Scheduling: one persistent CTA per SM; the producer thread of a CTA draws the next item from a
 // global counter (items are ordered layer, KV head, chunk, so neighbours in time read neighbouring
-// data), feeds the same TMA ring as the request-major kernel and tells the consumer warps which item
-// the tiles belong to through a small queue in shared memory.  All waits are bounded.
+// data), looks it up, feeds the same TMA ring as the request-major kernel and hands the consumer warps the
+// item's description through a small queue in shared memory.  All waits are bounded.
 #include <algorithm>
 
 #include "stream_common.cuh"
 
 namespace matkv {
 
+constexpr int kPend = 96;   // (item, stacked request) pairs whose arrival tickets are drawn together
 constexpr int kItemQ = 16;  // depth of the producer -> consumers item queue (the ring holds fewer tiles than that)
 
 struct SharedParams {
@@ -52,27 +53,33 @@ struct SharedCfg {
     static constexpr int KS = D / 16;
     // merge area: one 64-column half of O per warp and row, then m, l, rounded l per warp and row
     static constexpr int MERGE_BYTES = (kCW * kShareRows * (64 + 3) * 4 + 15) / 16 * 16;
-    static constexpr int FIXED_BYTES = MERGE_BYTES + 1024 + 1024;
+    static constexpr int MISC_BYTES = 3840;                // barriers, tags, flags, the item queue
+    static constexpr int FIXED_BYTES = MERGE_BYTES + MISC_BYTES + 1024;  // + slack for the 1024-byte alignment of the ring
     static constexpr int NSTAGE_MAX = (kMaxDynSmem - FIXED_BYTES) / STAGE_BYTES;
     static constexpr int NSTAGE = NSTAGE_MAX > 12 ? 12 : NSTAGE_MAX;
     static constexpr int SMEM_BYTES = NSTAGE * STAGE_BYTES + FIXED_BYTES;
     static_assert(kShareRows % G == 0, "unsupported group size");
-    static_assert(D % 64 == 0 && NSTAGE >= 3 && NSTAGE < kItemQ, "unsupported head_dim");
+    // the producer runs at most NSTAGE + 1 items ahead of the consumers: the queue must be deeper than that
+    static_assert(D % 64 == 0 && NSTAGE >= 3 && NSTAGE + 3 <= kItemQ, "unsupported head_dim");
 };
 
-// What an item id stands for.  Ids run over (layer of the launch, KV head, item of the table), the table's
-// chunk items first and then one tail item per request.
-struct ItemPos {
-    int32_t l_rel, g, k;
+// One entry of the producer -> consumers item queue: everything the consumers need to know about an item,
+// looked up by the producer while it is ahead.  Item ids run over (layer of the launch, KV head, item of the
+// table); the table's chunk items come first, then one tail item per request.
+struct QEntry {
+    uint32_t seq1;              // number of the item in this CTA's sequence, plus one; written last
+    int32_t id;                 // < 0: no more items
+    int32_t l_rel, g;
     int32_t n_tiles;            // tiles of the item (a tail item: the tail's tiles and one tile for the new token)
-    int32_t tail_tiles, t0, b;  // tail items only (b < 0 for a chunk item)
-    int32_t tmap, len, tile0;   // chunk items only
+    int32_t n_req;              // requests stacked in the item
+    int32_t b, t0;              // tail items: request and tail length (b < 0 for a chunk item)
+    int32_t tmap, len, tile0;   // chunk items: descriptor, chunk tokens, first tile
+    int32_t pad;
+    int32_t part[kShareRows];   // partial slot of (item, stacked request) inside one (layer, KV head)
+    int16_t req[kShareRows];    // stacked requests
+    int16_t np[kShareRows];     // partials each of them collects
 };
-
-struct CurItem {
-    ItemPos u;
-    int32_t n_req, id;
-};
+static_assert(sizeof(QEntry) == 48 + 64 + 64, "queue entry layout");
 
 __device__ __forceinline__ int32_t shared_t0(const SharedParams &p, int b) {
     int32_t t0 = p.tail_len[b];
@@ -83,22 +90,45 @@ __device__ __forceinline__ int32_t shared_t0(const SharedParams &p, int b) {
     return t0;
 }
 
-__device__ __forceinline__ void locate_item(const SharedParams &p, int32_t id, ItemPos &u) {
+// Producer side: looks item `id` up and fills a queue entry (everything but seq1).
+__device__ __forceinline__ void locate_item(const SharedParams &p, int32_t id, volatile QEntry *e) {
     const int32_t per_head = p.n_items + p.B;
-    const int32_t lg = id / per_head;
-    u.k = id % per_head;
-    u.l_rel = lg / p.Hkv;
-    u.g = lg % p.Hkv;
-    if (u.k < p.n_items) {
-        const int4 h = *(const int4 *)(p.items + u.k);  // tmap, len, tile0, n_tiles
-        u.tmap = h.x; u.len = h.y; u.tile0 = h.z; u.n_tiles = h.w;
-        u.b = -1; u.t0 = 0; u.tail_tiles = 0;
+    const int32_t lg = id / per_head, k = id % per_head;
+    e->id = id;
+    e->l_rel = lg / p.Hkv;
+    e->g = lg % p.Hkv;
+    if (k < p.n_items) {
+        const int4 *it = (const int4 *)(p.items + k);
+        const int4 h0 = it[0], h1 = it[1];  // tmap, len, tile0, n_tiles; n_req
+        e->tmap = h0.x; e->len = h0.y; e->tile0 = h0.z; e->n_tiles = h0.w;
+        e->n_req = h1.x;
+        e->b = -1; e->t0 = 0;
+        int4 rq[4], pt[4], np[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            rq[i] = it[2 + i];
+            pt[i] = it[6 + i];
+            np[i] = it[10 + i];
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            e->req[4 * i] = (int16_t)rq[i].x; e->req[4 * i + 1] = (int16_t)rq[i].y;
+            e->req[4 * i + 2] = (int16_t)rq[i].z; e->req[4 * i + 3] = (int16_t)rq[i].w;
+            e->part[4 * i] = pt[i].x; e->part[4 * i + 1] = pt[i].y; e->part[4 * i + 2] = pt[i].z; e->part[4 * i + 3] = pt[i].w;
+            e->np[4 * i] = (int16_t)np[i].x; e->np[4 * i + 1] = (int16_t)np[i].y;
+            e->np[4 * i + 2] = (int16_t)np[i].z; e->np[4 * i + 3] = (int16_t)np[i].w;
+        }
     } else {
-        u.b = u.k - p.n_items;
-        u.t0 = shared_t0(p, u.b);
-        u.tail_tiles = ceil_div(u.t0, kTile);
-        u.n_tiles = u.tail_tiles + 1;
-        u.tmap = 0; u.len = 0; u.tile0 = 0;
+        const int b = k - p.n_items;
+        const DevReq rq = p.reqs[b];
+        const int32_t t0 = shared_t0(p, b);
+        e->b = b; e->t0 = t0;
+        e->n_tiles = ceil_div(t0, kTile) + 1;
+        e->n_req = 1;
+        e->tmap = 0; e->len = 0; e->tile0 = 0;
+        e->req[0] = (int16_t)b;
+        e->part[0] = rq.part_base + rq.n_parts - 1;
+        e->np[0] = (int16_t)rq.n_parts;
     }
 }
 
@@ -114,15 +144,14 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
     float *merge_l = merge_m + kCW * kShareRows;
     float *merge_r = merge_l + kCW * kShareRows;
     unsigned char *misc = smem + C::NSTAGE * C::STAGE_BYTES + C::MERGE_BYTES;
-    uint64_t *bars = (uint64_t *)misc;                                            // full[NSTAGE], empty[NSTAGE]
-    volatile uint32_t *tags = (volatile uint32_t *)(misc + 2 * 12 * 8);           // per stage: rows | kTagNew | fill << 16
-    volatile unsigned long long *item_q = (volatile unsigned long long *)(misc + 2 * 12 * 8 + 12 * 4 + 8);  // (k + 1) << 32 | id
-    volatile int *flags = (volatile int *)(misc + 2 * 12 * 8 + 12 * 4 + 8 + kItemQ * 8);  // [0] abort, [1..] last-arriver per stacked request
-    int64_t *row_slot = (int64_t *)(misc + 2 * 12 * 8 + 12 * 4 + 8 + kItemQ * 8 + (2 + kShareRows) * 4);  // [R] partial slot per stacked request
-    int32_t *row_req = (int32_t *)(row_slot + kShareRows);   // [R] request
-    int32_t *row_np = row_req + kShareRows;                  // [R] parts of that request
-    volatile CurItem *curv = (volatile CurItem *)(row_np + kShareRows);
-    CurItem *cur = const_cast<CurItem *>(curv);
+    uint64_t *bars = (uint64_t *)misc;                                   // full[NSTAGE], empty[NSTAGE]
+    volatile uint32_t *tags = (volatile uint32_t *)(misc + 2 * 12 * 8);  // per stage: rows | kTagNew | fill << 16
+    volatile QEntry *item_q = (volatile QEntry *)(misc + 256);           // [kItemQ]
+    volatile int *flags = (volatile int *)(misc + 256 + kItemQ * sizeof(QEntry));  // [0] abort, [1] end of items
+    int32_t *pend_idx = (int32_t *)(misc + 256 + kItemQ * sizeof(QEntry) + 8);   // [kPend] arrival counter of a pending pair
+    int16_t *pend_np = (int16_t *)(pend_idx + kPend);                             // [kPend] partials its row collects
+    uint8_t *pend_last = (uint8_t *)(pend_np + kPend);                            // [kPend] this CTA delivered the last one
+    static_assert(256 + kItemQ * sizeof(QEntry) + 8 + kPend * 7 <= C::MISC_BYTES, "misc area");
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -131,8 +160,8 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
             mbar_init(smem_u32(bars + C::NSTAGE + s), kItems);
             tags[s] = 0xffff0000u;
         }
-        for (int s = 0; s < kItemQ; ++s) item_q[s] = 0ull;
-        for (int s = 0; s < 2 + kShareRows; ++s) flags[s] = 0;
+        for (int s = 0; s < kItemQ; ++s) item_q[s].seq1 = 0u;
+        flags[0] = flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -141,55 +170,68 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
     const uint32_t ring_u32 = smem_u32(ring), full_u32 = smem_u32(bars), empty_u32 = smem_u32(bars + C::NSTAGE);
 
     if (warp == kCW) {
-        // ================= producer: draws items and feeds the ring =================
+        // ================= producer: draws items, looks them up and feeds the ring =================
         if (lane != 0) return;
+        // entry kq of the queue is filled and published while the tiles of item kq - 1 are being issued: a pause
+        // of the producer (an atomic round trip, then dependent loads) would drain the ring, which is no deeper
+        // than the memory latency
+        auto publish = [&](uint32_t kq, int32_t id) {
+            volatile QEntry *e = item_q + kq % kItemQ;
+            if (id < n_ids) locate_item(p, id, e);
+            else e->id = -1;
+            __threadfence_block();
+            e->seq1 = kq + 1;
+        };
         uint32_t seq = 0, kq = 0;
         bool ok = true;
-        while (ok) {
-            const int32_t id = atomicAdd(p.work, 1);
-            if (id >= n_ids) {
-                item_q[kq % kItemQ] = ((unsigned long long)(kq + 1) << 32) | 0xffffffffull;
-                break;
-            }
-            item_q[kq % kItemQ] = ((unsigned long long)(kq + 1) << 32) | (uint32_t)id;
-            ++kq;
-            ItemPos u;
-            locate_item(p, id, u);
-            const int layer = p.layer0 + u.l_rel;
-            for (int t = 0; t < u.n_tiles; ++t, ++seq) {
+        int32_t id = atomicAdd(p.work, 1);
+        publish(0, id);
+        while (ok && id < n_ids) {
+            volatile QEntry *e = item_q + kq % kItemQ;
+            const int32_t l_rel = e->l_rel, g = e->g, n_tiles = e->n_tiles, b = e->b, t0 = e->t0;
+            const int32_t tmap = e->tmap, len = e->len, tile0 = e->tile0;
+            const int32_t tail_tiles = n_tiles - 1;  // tail items only
+            const int32_t id_next = atomicAdd(p.work, 1);
+            bool next_published = false;
+            const int layer = p.layer0 + l_rel;
+            for (int t = 0; t < n_tiles; ++t, ++seq) {
+                if (t == n_tiles / 2) {
+                    publish(kq + 1, id_next);
+                    next_published = true;
+                }
                 const uint32_t stage = seq % C::NSTAGE, use = seq / C::NSTAGE;
                 if (use > 0 && !mbar_wait(empty_u32 + stage * 8, (use - 1) & 1, flags)) {
                     ok = false;
                     break;
                 }
                 const uint32_t bar = full_u32 + stage * 8, dst = ring_u32 + stage * C::STAGE_BYTES;
-                if (u.b >= 0 && t == u.tail_tiles) {  // the step's new token, from k_new / v_new [layer][request][head][D]
-                    const int32_t z = u.l_rel * p.B + u.b;
+                if (b >= 0 && t == tail_tiles) {  // the step's new token, from k_new / v_new [layer][request][head][D]
+                    const int32_t z = l_rel * p.B + b;
                     tags[stage] = 1u | kTagNew | (use << 16);
                     mbar_expect_tx(bar, C::STAGE_BYTES);
 #pragma unroll
                     for (int bx = 0; bx < C::NBOX; ++bx) {
-                        tma_load_3d(dst + bx * C::BOX_BYTES, &kn_map, bx * 64, u.g, z, bar);
-                        tma_load_3d(dst + (C::NBOX + bx) * C::BOX_BYTES, &vn_map, bx * 64, u.g, z, bar);
+                        tma_load_3d(dst + bx * C::BOX_BYTES, &kn_map, bx * 64, g, z, bar);
+                        tma_load_3d(dst + (C::NBOX + bx) * C::BOX_BYTES, &vn_map, bx * 64, g, z, bar);
                     }
                     continue;
                 }
                 const CUtensorMap *mk, *mv;
                 int32_t yk, yv, rows;
-                if (u.b < 0) {
-                    const int r0 = (u.tile0 + t) * kTile;
-                    mk = mv = p.tmaps + u.tmap;
-                    yk = ((layer * 2) * p.Hkv + u.g) * u.len + r0;
-                    yv = ((layer * 2 + 1) * p.Hkv + u.g) * u.len + r0;
-                    rows = min(kTile, u.len - r0);
+                if (b < 0) {
+                    const int r0 = (tile0 + t) * kTile;
+                    mk = mv = p.tmaps + tmap;
+                    yk = ((layer * 2) * p.Hkv + g) * len + r0;
+                    yv = ((layer * 2 + 1) * p.Hkv + g) * len + r0;
+                    rows = min(kTile, len - r0);
                 } else {
                     const int r0 = t * kTile;
                     mk = p.tmaps + p.n_seg_total;
                     mv = mk + 1;
-                    yk = yv = ((u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + r0;
-                    rows = min(kTile, u.t0 - r0);
+                    yk = yv = ((b * p.n_layers_total + layer) * p.Hkv + g) * p.max_tail + r0;
+                    rows = min(kTile, t0 - r0);
                 }
-                tags[stage] = (uint32_t)rows | (use << 16);
+                tags[stage] = (uint32_t)rows | (use << 16);  // published only after the stage's previous fill was released
                 mbar_expect_tx(bar, C::STAGE_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < C::NBOX; ++bx) {
@@ -197,11 +239,13 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
                     tma_load_2d(dst + (C::NBOX + bx) * C::BOX_BYTES, mv, bx * 64, yv, bar);
                 }
             }
+            if (!ok && !next_published) publish(kq + 1, n_ids);  // gave up: the consumers must not wait for another item
+            ++kq;
+            id = id_next;
         }
         if (!ok) {
-            // gave up: tell the consumers there is nothing more, then wait (bounded) for the copies in flight
+            // wait (bounded) for the copies in flight so that none lands after the CTA has gone
             atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
-            item_q[kq % kItemQ] = ((unsigned long long)(kq + 1) << 32) | 0xffffffffull;
             const uint32_t lo = seq > (uint32_t)C::NSTAGE ? seq - C::NSTAGE : 0;
             for (uint32_t s2 = lo; s2 < seq; ++s2) {
                 const long long t0 = clock64();
@@ -217,84 +261,99 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
 
     uint32_t qa[C::KS][4];   // A fragments of Q: rows qr / qr+8, k columns 0-7 / 8-15 of every k-step
     float o[2 * C::KS][4];   // O accumulators: [8-column block of d][row qr: c0, c1; row qr+8: c2, c3]
-    float m_run[2], l_run[2], l_rnd[2];
+    float m_run[2], l_run[2];
+    float lr[4];             // row sums of the bf16-rounded numerators (an MMA against ones): O is normalised by them
 
-    int64_t j_base = 0;      // CTA-local index of the item's first tile
-    for (uint32_t kq = 0;; ++kq) {
-        // ---- which item: warp 0 reads the queue (bounded wait) and lays the item out for everybody ----
-        if (warp == 0) {
-            int32_t id = -1;
-            if (lane == 0) {
-                unsigned long long v = item_q[kq % kItemQ];
-                if ((uint32_t)(v >> 32) != kq + 1) {
-                    const long long t0 = clock64();
-                    while (true) {
-                        v = item_q[kq % kItemQ];
-                        if ((uint32_t)(v >> 32) == kq + 1 || *flags) break;
-                        if (clock64() - t0 > kWaitCycles) {
-                            *flags = 1;
-                            break;
-                        }
-                    }
-                }
-                if ((uint32_t)(v >> 32) == kq + 1) id = (int32_t)(uint32_t)v;
-            }
-            id = __shfl_sync(0xffffffffu, id, 0);
-            if (id >= 0) {
-                ItemPos w;
-                locate_item(p, id, w);
-                const int lgw = w.l_rel * p.Hkv + w.g;
-                int nr = 1;
-                if (w.b < 0) {
-                    nr = p.items[w.k].n_req;
-                    if (lane < nr) {
-                        const int b = p.items[w.k].req[lane];
-                        const DevReq rq = p.reqs[b];
-                        row_req[lane] = b;
-                        row_np[lane] = rq.n_parts;
-                        row_slot[lane] = (int64_t)lgw * p.parts_total + rq.part_base + p.items[w.k].part[lane];
-                    }
-                } else if (lane == 0) {
-                    const DevReq rq = p.reqs[w.b];
-                    row_req[0] = w.b;
-                    row_np[0] = rq.n_parts;
-                    row_slot[0] = (int64_t)lgw * p.parts_total + rq.part_base + rq.n_parts - 1;
-                }
-                if (lane == 0) {
-                    cur->u = w;
-                    cur->n_req = nr;
+    // thread 0 waits (bounded) for entry k of the queue; flags[1] tells everybody whether it holds an item
+    auto await_entry = [&](uint32_t k) {
+        volatile QEntry *e = item_q + k % kItemQ;
+        bool got = e->seq1 == k + 1;
+        if (!got) {
+            const long long t0 = clock64();
+            while (true) {
+                got = e->seq1 == k + 1;
+                if (got || flags[0]) break;
+                if (clock64() - t0 > kWaitCycles) {
+                    flags[0] = 1;
+                    break;
                 }
             }
-            if (lane == 0) cur->id = id;
         }
-        consumer_bar();
-        if (cur->id < 0) break;
-        const ItemPos u = cur->u;
-        const int n_req = cur->n_req;
-        const int layer = p.layer0 + u.l_rel;
-        const int lg = u.l_rel * p.Hkv + u.g;
-        const int n_rows = n_req * G;
-        // ---- per-item setup: the stacked requests' query rows ----
+        flags[1] = (got && e->id >= 0) ? 0 : 1;
+    };
+    // the query rows of the requests stacked in an item, as A fragments
+    auto load_q = [&](const volatile QEntry *e) {
+        const int n_rows = e->n_req * G;
+        const int64_t base = (int64_t)e->l_rel * p.q_sl + (int64_t)e->g * G * D;
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             const int r = qr + 8 * hh;
             const bool real = r < n_rows;
-            const __nv_bfloat16 *qrow =
-                p.q + (int64_t)u.l_rel * p.q_sl + (int64_t)(real ? row_req[r / G] : 0) * p.q_sb + (int64_t)(u.g * G + r % G) * D;
+            const __nv_bfloat16 *qrow = p.q + base + (int64_t)(real ? e->req[r / G] : 0) * p.q_sb + (r % G) * D;
 #pragma unroll
             for (int ks = 0; ks < C::KS; ++ks) {
                 qa[ks][hh] = real ? *(const uint32_t *)(qrow + ks * 16 + 2 * qc) : 0u;
                 qa[ks][2 + hh] = real ? *(const uint32_t *)(qrow + ks * 16 + 8 + 2 * qc) : 0u;
             }
+        }
+    };
+    // Arrival tickets are settled in batches.  A ticket must follow a device-wide fence, and a fence costs
+    // microseconds while the SM has a ring full of copies in flight: one per item would stall the consumers
+    // as long as a fifth of the item's stream time.  So every (item, stacked request) pair that has left a
+    // partial is only noted in shared memory, and once the list is nearly full (and after the last item) all
+    // its tickets are drawn behind one fence per thread; the last partial of a (layer, request, KV head) to be
+    // ticketed merges that row's partials.
+    int n_pend = 0;  // the same in every consumer thread
+    auto flush = [&]() {
+        consumer_bar();  // the partials of every listed pair have been written
+        for (int i = tid; i < n_pend; i += kCW * 32) {
+            int last = 0;
+            if (pend_np[i] > 1) {
+                __threadfence();
+                int32_t *cnt = p.counters + pend_idx[i];
+                last = atomicAdd(cnt, 1) == pend_np[i] - 1;
+                if (last) *cnt = 0;  // ready for the next launch
+            }
+            pend_last[i] = (uint8_t)last;
+        }
+        consumer_bar();
+        for (int pr = warp; pr < n_pend * G; pr += kCW) {
+            const int i = pr / G, h = pr % G;
+            if (!pend_last[i]) continue;
+            __threadfence();
+            const int lg = pend_idx[i] / p.B, b = pend_idx[i] % p.B;
+            const int l_rel = lg / p.Hkv, g = lg % p.Hkv;
+            const int64_t first = (int64_t)lg * p.parts_total + p.reqs[b].part_base;
+            combine_warp(p.part_o + (first * G + h) * D, (int64_t)G * D, p.part_lse + first * G + h, G, pend_np[i], D,
+                         p.out + (int64_t)l_rel * p.q_sl + (int64_t)b * p.q_sb + (int64_t)(g * G + h) * D,
+                         p.lse_out ? p.lse_out + (int64_t)l_rel * p.lse_sl + (int64_t)b * p.lse_sb + g * G + h : nullptr);
+        }
+        n_pend = 0;  // the list is rewritten only after the next item's first barrier, which every warp reaches after this
+    };
+
+    if (tid == 0) await_entry(0);
+    consumer_bar();
+    bool have = flags[1] == 0;
+    if (have) load_q(item_q);
+    int64_t j_base = 0;      // CTA-local index of the item's first tile
+    uint32_t k = 0;
+    for (; have; ++k) {
+        const volatile QEntry *e = item_q + k % kItemQ;
+        const int l_rel = e->l_rel, g = e->g, n_tiles = e->n_tiles, n_req = e->n_req, b_tail = e->b, t0 = e->t0;
+        const int layer = p.layer0 + l_rel;
+        const int lg = l_rel * p.Hkv + g;
+        const int n_rows = n_req * G;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
             m_run[hh] = -CUDART_INF_F;
             l_run[hh] = 0.f;
-            l_rnd[hh] = 0.f;
         }
+        lr[0] = lr[1] = lr[2] = lr[3] = 0.f;
 #pragma unroll
         for (int nb = 0; nb < 2 * C::KS; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
 
         // ---- this warp's 16-token pieces of the item ----
-        const int64_t hj_begin = j_base * kItems, hj_end = (j_base + u.n_tiles) * kItems;
+        const int64_t hj_begin = j_base * kItems, hj_end = (j_base + n_tiles) * kItems;
         int64_t hj = hj_begin + (int)((warp - hj_begin % kCW + kCW) % kCW);
         for (; hj < hj_end; hj += kCW) {
             const uint32_t j = (uint32_t)(hj / kItems);
@@ -333,7 +392,6 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
                     pa[hh] = pack_bf16(p0, p1);
                     pa[2 + hh] = pack_bf16(p2, p3);
                     l_run[hh] = l_run[hh] * alpha[hh] + ((p0 + p1) + (p2 + p3));
-                    l_rnd[hh] = l_rnd[hh] * alpha[hh] + ((bf_lo(pa[hh]) + bf_hi(pa[hh])) + (bf_lo(pa[2 + hh]) + bf_hi(pa[2 + hh])));
                     m_run[hh] = m_new;
                 }
                 if (__any_sync(0xffffffffu, alpha[0] != 1.0f || alpha[1] != 1.0f)) {
@@ -344,7 +402,10 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
                         o[nb][2] *= alpha[1];
                         o[nb][3] *= alpha[1];
                     }
+                    lr[0] *= alpha[0];
+                    lr[2] *= alpha[1];
                 }
+                mma_bf16(lr, pa[0], pa[1], pa[2], pa[3], 0x3f803f80u, 0x3f803f80u);  // P times a column of ones
                 // ---------- O += P V ----------
                 const uint32_t v_u32 = stage_u32 + C::NBOX * C::BOX_BYTES;
 #pragma unroll
@@ -356,10 +417,10 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
                     mma_bf16(o[2 * dp + 1], pa[0], pa[1], pa[2], pa[3], vb[2], vb[3]);
                 }
                 // ---------- the new token goes to the request's tail for later steps ----------
-                if ((tag & kTagNew) && r0 == 0 && u.t0 < p.max_tail) {
+                if ((tag & kTagNew) && r0 == 0 && t0 < p.max_tail) {
                     constexpr int CPR = D / 8;  // 16-byte chunks per row; lanes 0..CPR-1 move K, the next CPR lanes move V
                     const unsigned char *ring_stage = ring + stage * C::STAGE_BYTES;
-                    const int64_t off = ((((int64_t)u.b * p.n_layers_total + layer) * p.Hkv + u.g) * p.max_tail + u.t0) * D;
+                    const int64_t off = ((((int64_t)b_tail * p.n_layers_total + layer) * p.Hkv + g) * p.max_tail + t0) * D;
                     const int ch = lane % CPR, kv = lane / CPR;
                     if (kv < 2) {
                         const uint4 val = *(const uint4 *)(ring_stage + kv * C::NBOX * C::BOX_BYTES + (ch / 8) * C::BOX_BYTES + swz(0, ch % 8));
@@ -371,22 +432,23 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
             if (lane == 0) mbar_arrive(empty_u32 + stage * 8);
         }
 
-        // ---- end of the item: merge the warps' states, one 64-column half of O at a time ----
-        {
+        // ---- end of the item ----
+        // The global round trips of an item boundary are off the critical path: the next item's description was
+        // prepared by the producer, its query rows are fetched while this item's partials are being reduced, and
+        // the arrival tickets wait for the next batched flush.
+        if (tid == 0) await_entry(k + 1);
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                float l_tot = l_run[hh], r_tot = l_rnd[hh];
-                l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
-                l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
-                r_tot += __shfl_xor_sync(0xffffffffu, r_tot, 1);
-                r_tot += __shfl_xor_sync(0xffffffffu, r_tot, 2);
-                if (qc == 0) {
-                    merge_m[warp * kShareRows + qr + 8 * hh] = m_run[hh];
-                    merge_l[warp * kShareRows + qr + 8 * hh] = l_tot;
-                    merge_r[warp * kShareRows + qr + 8 * hh] = r_tot;
-                }
+        for (int hh = 0; hh < 2; ++hh) {
+            float l_tot = l_run[hh];
+            l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
+            l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
+            if (qc == 0) {
+                merge_m[warp * kShareRows + qr + 8 * hh] = m_run[hh];
+                merge_l[warp * kShareRows + qr + 8 * hh] = l_tot;
+                merge_r[warp * kShareRows + qr + 8 * hh] = lr[2 * hh];
             }
         }
+        bool have_next = false;
 #pragma unroll
         for (int half = 0; half < D / 64; ++half) {
             if (half) consumer_bar();  // the previous half has been read
@@ -396,57 +458,52 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
                 *(float2 *)(merge_o + (warp * kShareRows + qr + 8) * 64 + nb * 8 + 2 * qc) = make_float2(o[half * 8 + nb][2], o[half * 8 + nb][3]);
             }
             consumer_bar();
-            for (int idx = tid; idx < n_rows * 64; idx += kCW * 32) {
-                const int r = idx >> 6, d = half * 64 + (idx & 63);
+            if (half == 0) {
+                if (tid < n_req) {  // note the item's (request, KV head, layer) rows for the next ticket flush
+                    pend_idx[n_pend + tid] = lg * p.B + e->req[tid];
+                    pend_np[n_pend + tid] = e->np[tid];
+                }
+                have_next = flags[1] == 0;
+                if (have_next) load_q(item_q + (k + 1) % kItemQ);
+            }
+            // one (row, four columns) unit per thread and pass
+            for (int idx = tid; idx < n_rows * 16; idx += kCW * 32) {
+                const int r = idx >> 4, c4 = idx & 15;
                 float M = -CUDART_INF_F;
 #pragma unroll
                 for (int w = 0; w < kCW; ++w) M = fmaxf(M, merge_m[w * kShareRows + r]);
-                float acc = 0.f, L = 0.f, Lr = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float L = 0.f, Lr = 0.f;
 #pragma unroll
                 for (int w = 0; w < kCW; ++w) {
                     const float mw = merge_m[w * kShareRows + r];
                     const float sw = mw == -CUDART_INF_F ? 0.f : fast_exp2(mw - M);
-                    acc = fmaf(sw, merge_o[(w * kShareRows + r) * 64 + (idx & 63)], acc);
+                    const float4 v = *(const float4 *)(merge_o + (w * kShareRows + r) * 64 + 4 * c4);
+                    acc.x = fmaf(sw, v.x, acc.x); acc.y = fmaf(sw, v.y, acc.y);
+                    acc.z = fmaf(sw, v.z, acc.z); acc.w = fmaf(sw, v.w, acc.w);
                     L = fmaf(sw, merge_l[w * kShareRows + r], L);
                     Lr = fmaf(sw, merge_r[w * kShareRows + r], Lr);
                 }
-                const float ov = acc / Lr;
-                const int j = r / G, h = r % G;
-                if (row_np[j] == 1) {  // a request without chunks: its tail item is the whole answer
-                    p.out[(int64_t)u.l_rel * p.q_sl + (int64_t)row_req[j] * p.q_sb + (int64_t)(u.g * G + h) * D + d] = __float2bfloat16(ov);
-                    if (p.lse_out && d == 0)
-                        p.lse_out[(int64_t)u.l_rel * p.lse_sl + (int64_t)row_req[j] * p.lse_sb + u.g * G + h] = (M + log2f(L)) * kLn2;
+                const float inv = 1.f / Lr;
+                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+                const int j = r / G, h = r % G, d = half * 64 + 4 * c4;
+                const int b = e->req[j];
+                if (e->np[j] == 1) {  // a request without chunks: its tail item is the whole answer
+                    *(uint2 *)(p.out + (int64_t)l_rel * p.q_sl + (int64_t)b * p.q_sb + (int64_t)(g * G + h) * D + d) =
+                        make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+                    if (p.lse_out && d == 0) p.lse_out[(int64_t)l_rel * p.lse_sl + (int64_t)b * p.lse_sb + g * G + h] = (M + log2f(L)) * kLn2;
                 } else {
-                    p.part_o[(row_slot[j] * G + h) * D + d] = ov;
-                    if (d == 0) p.part_lse[row_slot[j] * G + h] = (M + log2f(L)) * kLn2;
+                    const int64_t row = ((int64_t)lg * p.parts_total + e->part[j]) * G + h;
+                    *(float4 *)(p.part_o + row * D + d) = acc;
+                    if (d == 0) p.part_lse[row] = (M + log2f(L)) * kLn2;
                 }
             }
         }
-        // ---- arrival tickets: the last partial of a (layer, request, KV head) merges them all ----
-        __threadfence();
-        consumer_bar();
-        if (tid < n_req) {
-            int last = 0;
-            if (row_np[tid] > 1) {
-                int32_t *cnt = p.counters + (int64_t)lg * p.B + row_req[tid];
-                last = atomicAdd(cnt, 1) == row_np[tid] - 1;
-                if (last) *cnt = 0;  // ready for the next launch
-            }
-            flags[2 + tid] = last;
-        }
-        consumer_bar();
-        for (int pr = warp; pr < n_rows; pr += kCW) {
-            const int j = pr / G, h = pr % G;
-            if (!flags[2 + j]) continue;
-            __threadfence();
-            const DevReq rq = p.reqs[row_req[j]];
-            const int64_t first = (int64_t)lg * p.parts_total + rq.part_base;
-            combine_warp(p.part_o + (first * G + h) * D, (int64_t)G * D, p.part_lse + first * G + h, G, rq.n_parts, D,
-                         p.out + (int64_t)u.l_rel * p.q_sl + (int64_t)row_req[j] * p.q_sb + (int64_t)(u.g * G + h) * D,
-                         p.lse_out ? p.lse_out + (int64_t)u.l_rel * p.lse_sl + (int64_t)row_req[j] * p.lse_sb + u.g * G + h : nullptr);
-        }
-        consumer_bar();  // merge area, row tables and flags are free again
-        j_base += u.n_tiles;
+        n_pend += n_req;
+        j_base += n_tiles;
+        have = have_next;
+        if (n_pend + kShareRows > kPend || !have) flush();
+        else consumer_bar();  // the merge area is free again
     }
     if (flags[0] && tid == 0) atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
     // the last CTA of the launch to get here re-arms the work counter and, if asked, moves every tail length
@@ -467,6 +524,7 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
         }
     }
 }
+
 
 template <int D, int G>
 static int launch_shared_t(const SharedParams &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {

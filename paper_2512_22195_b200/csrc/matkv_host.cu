@@ -614,7 +614,9 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
             part_base += rq.n_parts;
         }
         t->parts_total = part_base;
-        if (R > 0) {
+        bool fits = true;  // the kernel's item queue keeps request indices and part counts in 16 bits
+        for (int32_t r = 0; r < batch; ++r) fits = fits && t->h_reqs[r].n_parts <= 32767;
+        if (R > 0 && fits) {
             for (auto &kv : members) {
                 const int32_t len = kv.first.second, tiles = (len + kTile - 1) / kTile;
                 const auto &m = kv.second;
@@ -628,8 +630,10 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
                         it.n_tiles = std::min(T, tiles - tile0);
                         it.n_req = (int32_t)std::min<size_t>(R, m.size() - j0);
                         for (int32_t j = 0; j < it.n_req; ++j) {
+                            const DevReq &rq = t->h_reqs[m[j0 + j].first];
                             it.req[j] = m[j0 + j].first;
-                            it.part[j] = part_off[m[j0 + j].second] + sub;
+                            it.part[j] = rq.part_base + part_off[m[j0 + j].second] + sub;
+                            it.np[j] = rq.n_parts;
                         }
                         t->item_tiles += it.n_tiles;
                         items.push_back(it);

@@ -45,7 +45,8 @@ struct DevItem {
     int32_t n_req;     // requests stacked in the item
     int32_t pad[3];
     int32_t req[kShareRows];   // request per stacked slot
-    int32_t part[kShareRows];  // index of this item's partial among that request's parts
+    int32_t part[kShareRows];  // partial slot of (this item, that request) inside one (layer, KV head)
+    int32_t np[kShareRows];    // partials that request collects in all (its n_parts)
 };
 
 // ---- host-side objects --------------------------------------------------------------------
