@@ -399,6 +399,9 @@ def main():
     if args.decode_steps:
         w.decode_steps = args.decode_steps
         w.name += f"-T{args.decode_steps}"
+    if args.pool_chunks:
+        w.pool_chunks = args.pool_chunks
+        w.name += f"-P{args.pool_chunks}"
     L, B, S, T, Hq, Hkv, D = w.n_layers, w.batch, w.suffix, w.decode_steps, w.n_q_heads, w.n_kv_heads, w.head_dim
     ids = w.chunk_ids(0)
     needed = sorted({c for row in ids for c in row})

@@ -1,6 +1,7 @@
 """Parity at the benchmark's full size and launch configuration (config 2: 32 layers, Llama-3-8B head
 shape, 5 x 1,024-token chunks, 64-token suffix through the tile kernel, 128 decode steps with all layers
-in one launch), on sampled outputs the oracle computes one by one."""
+in one launch; config 3: batch 16, 10 of 256 chunks per request by Zipf rank, chunk-major decode), on
+sampled outputs the oracle computes one by one."""
 import numpy as np
 import pytest
 import torch
@@ -74,4 +75,62 @@ def test_cfg2_full_size_sampled_units():
         check(dev_to_bits(out)[layer, 0], o_ref[0], lse.cpu().numpy()[layer, 0], l_ref[0], f"full-size decode step {step} layer {layer}")
     # the inputs the GPU consumed are the generator's bytes (the oracle regenerated them on the host)
     assert np.array_equal(dev_to_bits(q_dc[5]), mi.decode_inputs(w, 5)[0])
+    sess.close()
+
+
+def test_cfg3_full_size_chunk_major_sampled_units():
+    """Config 3 at full size: 16 requests x 10 chunks drawn by Zipf rank from 256 (73 distinct), 32 layers,
+    32-token suffix, 256 decode steps, every step one all-layers launch of the chunk-major kernel that also
+    advances the tail; sampled (step, layer, request) outputs against the oracle."""
+    import matkv_inputs.device as gen
+    import paper_2512_22195_b200 as mk
+    from paper_2512_22195_b200.harness import Session, dev_to_bits
+    w = mi.workload("cfg3")
+    L, B, S, T, Hq, Hkv, D = w.n_layers, w.batch, w.suffix, w.decode_steps, w.n_q_heads, w.n_kv_heads, w.head_dim
+    ids = w.chunk_ids(0)
+    needed = sorted({c for row in ids for c in row})
+    sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T)
+    mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, 2)
+    mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_ADVANCES_TAIL, 1)
+    pool = torch.empty((len(needed), L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device="cuda")
+    for i, c in enumerate(needed):
+        gen.fill_bf16(pool[i], w.seed, mi.STREAM_CHUNK + c)
+        sess.register_device_chunk(c, pool[i])
+    q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device="cuda")
+    k_pf = torch.empty((L, B, S, Hkv, D), dtype=torch.bfloat16, device="cuda")
+    v_pf = torch.empty_like(k_pf)
+    q_dc = torch.empty((T, L, B, Hq, D), dtype=torch.bfloat16, device="cuda")
+    k_dc = torch.empty((T, L, B, Hkv, D), dtype=torch.bfloat16, device="cuda")
+    v_dc = torch.empty_like(k_dc)
+    for t_, st in ((q_pf, mi.STREAM_Q_PREFILL), (k_pf, mi.STREAM_K_PREFILL), (v_pf, mi.STREAM_V_PREFILL),
+                   (q_dc, mi.STREAM_Q_DECODE), (k_dc, mi.STREAM_K_DECODE), (v_dc, mi.STREAM_V_DECODE)):
+        gen.fill_bf16(t_, w.seed, st)
+    table = sess.build_table(ids)
+    listed, read = mk.matkv_table_sharing(table)
+    assert listed == B * w.chunks_per_req * (w.chunk_tokens // 64) and read < listed * 0.6   # stacking nearly halves the reads
+    sess.prefill_all_layers(q_pf, k_pf, v_pf)
+    sess.advance(S)
+    samples = {0: [(0, 0), (L - 1, 3)], 100: [(17, 9)], T - 1: [(0, B - 1), (L - 1, 0)]}   # step -> (layer, request)
+    got = {}
+    for t in range(T):
+        out, lse = sess.decode_all_layers(q_dc[t], k_dc[t], v_dc[t])
+        if t in samples:
+            got[t] = (dev_to_bits(out), lse.cpu().numpy())
+    assert sess.status() == 0
+    sh1 = oracle.Shape(1, Hq, Hkv, D)
+    for step, pairs in samples.items():
+        q, k, v = mi.decode_inputs(w, step)
+        for layer, r in pairs:
+            blobs = [dev_to_bits(pool[needed.index(c)][layer:layer + 1]) for c in ids[r]]
+            rq = oracle.Request(sh1, blobs, S + T)
+            _, kp, vp = mi.prefill_inputs(w, layer)
+            rq.append_only(0, kp[r], vp[r])
+            rq.advance(S)
+            for s_ in range(step):
+                _, kk, vv = mi.decode_inputs(w, s_)
+                rq.append_only(0, kk[layer, r][None], vv[layer, r][None])
+                rq.advance(1)
+            o_ref, l_ref = rq.attend_new(0, q[layer, r][None], k[layer, r][None], v[layer, r][None])
+            check(got[step][0][layer, r], o_ref[0], got[step][1][layer, r], l_ref[0],
+                  f"full-size chunk-major decode step {step} layer {layer} request {r}")
     sess.close()
