@@ -32,7 +32,8 @@ import matkv_inputs as mi  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per decode launch from the committed ncu capture (profiles/), by workload and launch mode.
-NCU_TRAFFIC_BYTES = {("cfg2", "all_layers"): 697.5e6 + 5.0e6}  # profiles/k_attend_stream_decode_cfg2_all_layers.md
+NCU_TRAFFIC_BYTES = {("cfg2", "all_layers"): 697.5e6 + 5.0e6,   # profiles/k_attend_stream_decode_cfg2_all_layers.md
+                     ("cfg3", "all_layers"): 10.02e9 + 0.10e9}   # profiles/k_attend_shared_decode_cfg3.md (chunk-major kernel)
 
 
 def log(*a):
@@ -538,7 +539,8 @@ def main():
         other = "per_layer_graph" if args.decode_launch == "all_layers" else "all_layers"
         dec_ms_o = None
         if not args.no_other_mode:
-            one_step(*dev_ptrs, mode=other)
+            for _ in range(2):   # the first graph capture of a process pays one-off costs
+                one_step(*dev_ptrs, mode=other)
             timed_region(lambda i: one_step(*dev_ptrs, timed_index=i, mode=other), min(args.steps, 5))
             dec_ms_o = sum(a.elapsed_time(b) for a, b in zip(ev_d0[:min(args.steps, 5)], ev_d1[:min(args.steps, 5)]))
 
@@ -569,6 +571,13 @@ def main():
     # chunk tiles the batch lists against the tiles the decode kernel in use reads (chunk-major stacking)
     tiles_logical, tiles_read = mk.matkv_table_sharing(sess.table)
     chunk_major = args.decode_impl == 2 or (args.decode_impl == 0 and tiles_logical * 4 >= tiles_read * 5)
+    logical_gbs = achieved
+    if chunk_major:
+        # the chunk-major kernel reads a chunk once per 16 / G requests that list it: its algorithmic bytes are the
+        # tiles it reads (64 tokens x K and V x all KV heads) plus every request's tail
+        tile_bytes = 64 * w.beta
+        read_bytes_decode = sum(tiles_read * tile_bytes + sum(S + t + 1 for _ in range(B)) * w.beta for t in range(T)) * L
+        achieved = read_bytes_decode / decode_launches / (avg_launch_ms * 1e-3) / 1e9
     result = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -585,8 +594,9 @@ def main():
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                      "read_probe_gbs_same_run": probe_gbs,
-                     "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.decode_launch)),
-                     "algorithmic_bytes_per_launch": kv_bytes_decode / decode_launches,
+                     "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.decode_launch)) if (chunk_major or w.name != "cfg3") else None,
+                     "algorithmic_bytes_per_launch": (read_bytes_decode if chunk_major else kv_bytes_decode) / decode_launches,
+                     "logical_kv_gbs": logical_gbs,
                      "avg_launch_us": avg_launch_ms * 1e3},
         "phases": {"prefill_ms_per_step": pre_ms / args.steps, "decode_ms_per_step": dec_ms / args.steps,
                    "decode_only_tokens_per_s": B * T * args.steps / (dec_ms * 1e-3),
