@@ -56,7 +56,8 @@ struct SharedCfg {
     static constexpr int MISC_BYTES = 3840;                // barriers, tags, flags, the item queue
     static constexpr int FIXED_BYTES = MERGE_BYTES + MISC_BYTES + 1024;  // + slack for the 1024-byte alignment of the ring
     static constexpr int NSTAGE_MAX = (kMaxDynSmem - FIXED_BYTES) / STAGE_BYTES;
-    static constexpr int NSTAGE = NSTAGE_MAX > 12 ? 12 : NSTAGE_MAX;
+    static constexpr int NSTAGE_CAP = 192 * 1024 / STAGE_BYTES;
+    static constexpr int NSTAGE = NSTAGE_MAX > NSTAGE_CAP ? NSTAGE_CAP : NSTAGE_MAX;
     static constexpr int SMEM_BYTES = NSTAGE * STAGE_BYTES + FIXED_BYTES;
     static_assert(kShareRows % G == 0, "unsupported group size");
     // the producer runs at most NSTAGE + 1 items ahead of the consumers: the queue must be deeper than that
@@ -74,7 +75,7 @@ struct QEntry {
     int32_t n_req;              // requests stacked in the item
     int32_t b, t0;              // tail items: request and tail length (b < 0 for a chunk item)
     int32_t tmap, len, tile0;   // chunk items: descriptor, chunk tokens, first tile
-    int32_t pad;
+    int32_t last_read;          // nothing reads these tiles again in this launch: load them with the evict-first L2 policy
     int32_t part[kShareRows];   // partial slot of (item, stacked request) inside one (layer, KV head)
     int16_t req[kShareRows];    // stacked requests
     int16_t np[kShareRows];     // partials each of them collects
@@ -102,6 +103,7 @@ __device__ __forceinline__ void locate_item(const SharedParams &p, int32_t id, v
         const int4 h0 = it[0], h1 = it[1];  // tmap, len, tile0, n_tiles; n_req
         e->tmap = h0.x; e->len = h0.y; e->tile0 = h0.z; e->n_tiles = h0.w;
         e->n_req = h1.x;
+        e->last_read = h1.y;
         e->b = -1; e->t0 = 0;
         int4 rq[4], pt[4], np[4];
 #pragma unroll
@@ -125,6 +127,7 @@ __device__ __forceinline__ void locate_item(const SharedParams &p, int32_t id, v
         e->b = b; e->t0 = t0;
         e->n_tiles = ceil_div(t0, kTile) + 1;
         e->n_req = 1;
+        e->last_read = 1;
         e->tmap = 0; e->len = 0; e->tile0 = 0;
         e->req[0] = (int16_t)b;
         e->part[0] = rq.part_base + rq.n_parts - 1;
@@ -182,6 +185,7 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
             __threadfence_block();
             e->seq1 = kq + 1;
         };
+        const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_normal();
         uint32_t seq = 0, kq = 0;
         bool ok = true;
         int32_t id = atomicAdd(p.work, 1);
@@ -190,6 +194,7 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
             volatile QEntry *e = item_q + kq % kItemQ;
             const int32_t l_rel = e->l_rel, g = e->g, n_tiles = e->n_tiles, b = e->b, t0 = e->t0;
             const int32_t tmap = e->tmap, len = e->len, tile0 = e->tile0;
+            const uint64_t pol = e->last_read ? pol_stream : pol_keep;
             const int32_t tail_tiles = n_tiles - 1;  // tail items only
             const int32_t id_next = atomicAdd(p.work, 1);
             bool next_published = false;
@@ -235,8 +240,8 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
                 mbar_expect_tx(bar, C::STAGE_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < C::NBOX; ++bx) {
-                    tma_load_2d(dst + bx * C::BOX_BYTES, mk, bx * 64, yk, bar);
-                    tma_load_2d(dst + (C::NBOX + bx) * C::BOX_BYTES, mv, bx * 64, yv, bar);
+                    tma_load_2d_hint(dst + bx * C::BOX_BYTES, mk, bx * 64, yk, bar, pol);
+                    tma_load_2d_hint(dst + (C::NBOX + bx) * C::BOX_BYTES, mv, bx * 64, yv, bar, pol);
                 }
             }
             if (!ok && !next_published) publish(kq + 1, n_ids);  // gave up: the consumers must not wait for another item

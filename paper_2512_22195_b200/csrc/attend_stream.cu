@@ -41,6 +41,7 @@ struct StreamParams {
     int32_t *status;
     int32_t advance;      // > 0: the last CTA to finish adds this to every request's tail length
     int32_t *done_count;  // CTAs of the launch that have finished (reset by the last one)
+    int32_t stream_hint;  // 1: no chunk of the table is listed twice, load chunk tiles with the evict-first L2 policy
 };
 
 // ---- the flat work list ----------------------------------------------------------------------------
@@ -145,10 +146,11 @@ struct StreamCfg {
     static constexpr int MERGE_BYTES = (kCW * kUnitRows * (D + 3) * 4 + 15) / 16 * 16;
     static constexpr int FIXED_BYTES = MERGE_BYTES + 1024 + 1024;  // + misc + slack for 1024-byte alignment of the ring
     static constexpr int NSTAGE_MAX = (kMaxDynSmem - FIXED_BYTES) / STAGE_BYTES;
-    // Measured on B200: a ring of 160 KB is faster than one that fills shared memory (config 2: 111.0 us per
-    // all-layers launch with 5 stages of 32 KB, 111.2 with 4, 114.2 with 6, 114.9 with 3; configs 3 and 4 gain
-    // 5-8 % from 6 -> 5): more copies in flight than the memory latency needs only lengthen the DRAM queues.
-    static constexpr int NSTAGE_CAP = 160 * 1024 / STAGE_BYTES;
+    // Measured on B200 (chunk tiles loaded with the evict-first L2 policy): a ring of 128 KB is faster than one
+    // that fills shared memory.  Config 2, all-layers launch: 107.7 us with 4 stages of 32 KB, 107.9 with 5,
+    // 111.1 with 6; config 4: 11.63 / 11.84 / 12.50 ms.  More copies in flight than the memory latency needs
+    // only lengthen the queues in front of DRAM.
+    static constexpr int NSTAGE_CAP = 128 * 1024 / STAGE_BYTES;
     static constexpr int NSTAGE = NSTAGE_MAX > NSTAGE_CAP ? NSTAGE_CAP : NSTAGE_MAX;
     static constexpr int SMEM_BYTES = NSTAGE * STAGE_BYTES + FIXED_BYTES;
     static_assert(G >= 1 && G <= kUnitRows && kUnitRows % G == 0, "unsupported group size");
@@ -216,6 +218,8 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
     if (warp == kCW) {
         // ================= producer: one thread walks the table and feeds the ring =================
         if (lane != 0) return;
+        // chunk rows are read once per launch unless requests share chunks: keep them out of L2's way then
+        const uint64_t pol = p.stream_hint ? l2_policy_evict_first() : l2_policy_evict_normal();
         UnitPos u = range->first;
         int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;  // cursor over the request's segments
         int64_t f = f_begin;
@@ -268,8 +272,8 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                 mbar_expect_tx(bar, C::STAGE_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < C::NBOX; ++bx) {
-                    tma_load_2d(dst + bx * C::BOX_BYTES, mk, bx * 64, yk, bar);
-                    tma_load_2d(dst + (C::NBOX + bx) * C::BOX_BYTES, mv, bx * 64, yv, bar);
+                    tma_load_2d_hint(dst + bx * C::BOX_BYTES, mk, bx * 64, yk, bar, pol);
+                    tma_load_2d_hint(dst + (C::NBOX + bx) * C::BOX_BYTES, mv, bx * 64, yv, bar, pol);
                 }
             }
             if (f < f_end && ok) {
@@ -540,6 +544,7 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     p.status = ctx->d_status;
     p.advance = a.advance;
     p.done_count = ctx->d_status + 2;
+    p.stream_hint = t->distinct_chunk_tiles == t->total_chunk_tiles && n_blk == 1;  // several token blocks re-read the tiles
     const int64_t n_units = (int64_t)a.n_layers_launch * t->batch * n_blk * c.n_kv_heads;
     if (n_units > ws.n_counter_slots)
         return fail(MATKV_E_CAPACITY, "launch of %lld units exceeds the workspace's %lld", (long long)n_units,
@@ -652,6 +657,7 @@ extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_
         p.status = ctx->d_status;
         p.advance = 0;
         p.done_count = ctx->d_status + 2;
+        p.stream_hint = t->distinct_chunk_tiles == t->total_chunk_tiles;
         CUtensorMap kn_map, vn_map;
         rc = encode_new_rows_map(&kn_map, k_new, c.head_dim, c.n_kv_heads, (uint64_t)t->batch);
         if (!rc) rc = encode_new_rows_map(&vn_map, v_new, c.head_dim, c.n_kv_heads, (uint64_t)t->batch);

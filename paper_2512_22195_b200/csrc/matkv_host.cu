@@ -614,6 +614,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
             part_base += rq.n_parts;
         }
         t->parts_total = part_base;
+        for (auto &kv : members) t->distinct_chunk_tiles += (kv.first.second + kTile - 1) / kTile;
         bool fits = true;  // the kernel's item queue keeps request indices and part counts in 16 bits
         for (int32_t r = 0; r < batch; ++r) fits = fits && t->h_reqs[r].n_parts <= 32767;
         if (R > 0 && fits) {
@@ -629,6 +630,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
                         it.tile0 = tile0;
                         it.n_tiles = std::min(T, tiles - tile0);
                         it.n_req = (int32_t)std::min<size_t>(R, m.size() - j0);
+                        it.last_read = j0 + R >= m.size();
                         for (int32_t j = 0; j < it.n_req; ++j) {
                             const DevReq &rq = t->h_reqs[m[j0 + j].first];
                             it.req[j] = m[j0 + j].first;

@@ -43,7 +43,8 @@ struct DevItem {
     int32_t tile0;     // first tile of the item inside the chunk
     int32_t n_tiles;
     int32_t n_req;     // requests stacked in the item
-    int32_t pad[3];
+    int32_t last_read; // 1: no later item reads these tiles again (the chunk's last group of requests)
+    int32_t pad[2];
     int32_t req[kShareRows];   // request per stacked slot
     int32_t part[kShareRows];  // partial slot of (this item, that request) inside one (layer, KV head)
     int32_t np[kShareRows];    // partials that request collects in all (its n_parts)
@@ -110,6 +111,7 @@ struct matkv_table {
     int32_t tail_len_host = 0;   // host mirror (not moved by graph replays)
     int32_t max_chunk_tiles = 0;
     int64_t total_chunk_tiles = 0;
+    int64_t distinct_chunk_tiles = 0;  // tiles of the distinct device copies the requests list
     void *h_pinned = nullptr;    // pinned upload image
     void *d_image = nullptr;     // device image: segs | reqs | tail_len[B]
     size_t image_bytes = 0, image_alloc = 0;
