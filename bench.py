@@ -202,6 +202,8 @@ def run_pipeline(args):
         args.stage_ctas = 16
     if args.stage_ctas:
         mk.matkv_set_option(sess.ctx, mk.OPT_STAGE_CTAS, args.stage_ctas)
+    if args.decode_ctas:
+        mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, args.decode_ctas)
     tmp = torch.empty((L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
     host_pool = ring = None
     if args.store_dir:

@@ -77,7 +77,8 @@ typedef struct {
 } matkv_config;
 
 /* options for matkv_set_option */
-#define MATKV_OPT_DECODE_CTAS   1  /* number of CTAs the streaming kernel splits the KV over; 0 = auto */
+#define MATKV_OPT_DECODE_CTAS   1  /* number of CTAs the streaming kernel splits the KV over; 0 = auto: one per SM,
+                                      less MATKV_OPT_STAGE_CTAS when the staging copy kernel is in use */
 #define MATKV_OPT_PREFILL_IMPL  2  /* 0 = auto (tensor-core tiles when the suffix is large enough),
                                       1 = force the streaming kernel, 2 = force the tensor-core kernel,
                                       3 = tensor-core kernel with two 128-row blocks per CTA whenever a

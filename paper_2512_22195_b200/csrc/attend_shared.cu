@@ -595,7 +595,9 @@ int launch_attend_shared(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, vo
     }
     const int64_t n_ids = (int64_t)a.n_layers_launch * c.n_kv_heads * (t->n_items + t->batch);
     if (n_ids > 0x7fff0000ll) return fail(MATKV_E_CAPACITY, "launch of %lld items", (long long)n_ids);
-    int64_t grid = ctx->opt_decode_ctas > 0 ? ctx->opt_decode_ctas : ctx->n_sm;
+    // by default one CTA per SM, less the SMs left to the staging copy kernel when that is in use (the launch is
+    // bound by HBM with ~130 CTAs already; a copy CTA sharing an SM with a decode CTA makes that SM the straggler)
+    int64_t grid = ctx->opt_decode_ctas > 0 ? ctx->opt_decode_ctas : std::max<int64_t>(ctx->n_sm - ctx->opt_stage_ctas, ctx->n_sm / 2);
     grid = std::max<int64_t>(1, std::min<int64_t>(grid, n_ids));
 #define MATKV_CASE(DD, GG) \
     if (c.head_dim == DD && G == GG) return launch_shared_t<DD, GG>(p, kn_map, vn_map, (int)grid, stream);

@@ -562,7 +562,9 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
         if (!rc) rc = encode_new_rows_map(&vn_map, a.v_new, c.head_dim, c.n_kv_heads, n_tok);
         if (rc) return rc;
     }
-    int64_t grid = ctx->opt_decode_ctas > 0 ? ctx->opt_decode_ctas : ctx->n_sm;
+    // by default one CTA per SM, less the SMs left to the staging copy kernel when that is in use (the launch is
+    // bound by HBM with ~130 CTAs already; a copy CTA sharing an SM with a decode CTA makes that SM the straggler)
+    int64_t grid = ctx->opt_decode_ctas > 0 ? ctx->opt_decode_ctas : std::max<int64_t>(ctx->n_sm - ctx->opt_stage_ctas, ctx->n_sm / 2);
     grid = std::max<int64_t>(1, std::min<int64_t>(grid, W));
 #define MATKV_CASE(DD, GG) \
     if (c.head_dim == DD && G == GG) return launch_stream_t<DD, GG>(p, kn_map, vn_map, (int)grid, stream);
