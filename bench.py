@@ -628,60 +628,84 @@ def main():
             mk.matkv_register_chunk(sess2.ctx, c, w.chunk_tokens, host[c].data_ptr(), None)
         slot_bytes = w.chunk_bytes
         slots = [torch.empty(len(needed) * slot_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
-        dq_pf, dk_pf, dv_pf = torch.empty_like(q_pf), torch.empty_like(k_pf), torch.empty_like(v_pf)
-        dq_dc, dk_dc, dv_dc = torch.empty_like(q_dc), torch.empty_like(k_dc), torch.empty_like(v_dc)
-        h2d = len(needed) * slot_bytes + sum(x.numel() * 2 for x in (hq_pf, hk_pf, hv_pf, hq_dc, hk_dc, hv_dc))
+        # query-side inputs and outputs are double-buffered on the device: step i+1's inputs arrive (copy stream)
+        # and step i-1's outputs leave (output stream) while step i computes
+        d_in = [tuple(torch.empty_like(x) for x in (q_pf, k_pf, v_pf, q_dc, k_dc, v_dc)) for _ in range(2)]
+        d_out = [(torch.empty_like(o_pf), torch.empty_like(o_dc)) for _ in range(2)]
+        h_in = (hq_pf, hk_pf, hv_pf, hq_dc, hk_dc, hv_dc)
+        h2d = len(needed) * slot_bytes + sum(x.numel() * 2 for x in h_in)
         d2h = (ho_pf.numel() + ho_dc.numel()) * 2
         ctx2 = sess2.ctx
+        out_stream = torch.cuda.Stream(device=dev)
+        in_ready = [torch.cuda.Event() for _ in range(2)]
+        comp_done = [torch.cuda.Event() for _ in range(2)]
+        out_done = [torch.cuda.Event() for _ in range(2)]
+        state = {"loaded": -1}
 
-        state = {"staged": -1}
-
-        def stage(i):
+        def load(i):
+            """Everything step i needs from the host, on the copy stream: its query-side inputs (small, first),
+            then its chunks into slot region i % 2."""
+            if i >= 2:
+                copy.wait_event(comp_done[i % 2])          # step i-2 has finished with these input buffers
+            with torch.cuda.stream(copy):
+                for dst, src in zip(d_in[i % 2], h_in):
+                    dst.copy_(src, non_blocking=True)
+                in_ready[i % 2].record(copy)
             sess2.stage(needed, slots[i % 2], slot_bytes, copy)
-            state["staged"] = i
+            state["loaded"] = i
 
-        def e2e_step(i):
-            # load: pinned host -> device slots on the copy stream; the compute stream waits through the table.
-            # The NEXT step's chunks are staged into the other slot region right after this step's table is
-            # built, so that their copies run under this step's prefill and decode (the paper's overlap).
-            if state["staged"] < i:
-                stage(i)
-            # this step's query-side inputs, before the next step's chunk copies are queued on the copy engine
-            dq_pf.copy_(hq_pf, non_blocking=True); dk_pf.copy_(hk_pf, non_blocking=True); dv_pf.copy_(hv_pf, non_blocking=True)
-            dq_dc.copy_(hq_dc, non_blocking=True); dk_dc.copy_(hk_dc, non_blocking=True); dv_dc.copy_(hv_dc, non_blocking=True)
-            table = sess2.build_table(ids, sp)
-            stage(i + 1)
+        def e2e_step(i, last=False):
+            if state["loaded"] < i:
+                load(i)
+            dq_pf, dk_pf, dv_pf, dq_dc, dk_dc, dv_dc = d_in[i % 2]
+            eo_pf, eo_dc = d_out[i % 2]
+            table = sess2.build_table(ids, sp)             # makes the compute stream wait for this step's chunk copies
+            stream.wait_event(in_ready[i % 2])
+            if i >= 2:
+                stream.wait_event(out_done[i % 2])         # step i-2's outputs have left these buffers
+            load(i + 1)                                    # the next step's copies run under this step's compute
             if args.decode_launch == "all_layers":
-                mk.matkv_attend_prefill_all_layers(ctx2, table, S, dq_pf.data_ptr(), dk_pf.data_ptr(), dv_pf.data_ptr(), o_pf.data_ptr(), None, sp)
+                mk.matkv_attend_prefill_all_layers(ctx2, table, S, dq_pf.data_ptr(), dk_pf.data_ptr(), dv_pf.data_ptr(), eo_pf.data_ptr(), None, sp)
             else:
                 for layer in range(L):
                     mk.matkv_attend_prefill(ctx2, table, layer, S, dq_pf.data_ptr() + layer * qs_l, dk_pf.data_ptr() + layer * ks_l,
-                                            dv_pf.data_ptr() + layer * ks_l, o_pf.data_ptr() + layer * qs_l, None, sp)
+                                            dv_pf.data_ptr() + layer * ks_l, eo_pf.data_ptr() + layer * qs_l, None, sp)
             mk.matkv_table_advance(table, S, sp)
             for t in range(T):
                 if args.decode_launch == "all_layers":
                     mk.matkv_attend_decode_all_layers(ctx2, table, dq_dc.data_ptr() + t * qd_t, dk_dc.data_ptr() + t * kd_t,
-                                                      dv_dc.data_ptr() + t * kd_t, o_dc.data_ptr() + t * qd_t, None, sp)
+                                                      dv_dc.data_ptr() + t * kd_t, eo_dc.data_ptr() + t * qd_t, None, sp)
+                    if fused_advance:
+                        continue
                 else:
                     for layer in range(L):
                         mk.matkv_attend_decode(ctx2, table, layer, dq_dc.data_ptr() + t * qd_t + layer * qd_l,
                                                dk_dc.data_ptr() + t * kd_t + layer * kd_l, dv_dc.data_ptr() + t * kd_t + layer * kd_l,
-                                               o_dc.data_ptr() + t * qd_t + layer * qd_l, None, sp)
+                                               eo_dc.data_ptr() + t * qd_t + layer * qd_l, None, sp)
                 mk.matkv_table_advance(table, 1, sp)
-            ho_pf.copy_(o_pf, non_blocking=True)                # the step's results go back to the host
-            ho_dc.copy_(o_dc, non_blocking=True)
+            comp_done[i % 2].record(stream)
+            out_stream.wait_event(comp_done[i % 2])
+            with torch.cuda.stream(out_stream):            # the step's results go back to the host
+                ho_pf.copy_(eo_pf, non_blocking=True)
+                ho_dc.copy_(eo_dc, non_blocking=True)
+                out_done[i % 2].record(out_stream)
+            if last:
+                stream.wait_event(out_done[i % 2])         # the timed region ends when the last result is on the host
             return 0
 
+        if fused_advance:
+            mk.matkv_set_option(ctx2, mk.OPT_DECODE_ADVANCES_TAIL, 1)
         with torch.cuda.stream(stream):
             for i in range(2):
                 e2e_step(i)
             k_e2e = min(args.steps, 5)
-            ms_e, _, _, _ = timed_region(lambda i: e2e_step(i + 2), k_e2e)
+            ms_e, _, _, _ = timed_region(lambda i: e2e_step(i + 2, last=(i == k_e2e - 1)), k_e2e)
         if sess2.status() != 0:
             raise RuntimeError("device status non-zero after the end-to-end region")
         result["e2e"] = {"value": tokens * k_e2e / (ms_e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                          "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e,
-                         "overlap": "next step's chunks staged on a side stream under this step's prefill and decode",
+                         "overlap": "next step's chunks and query-side inputs copied in, and the previous step's outputs copied out, "
+                                    "on side streams under this step's prefill and decode",
                          "staging": f"copy kernel, {args.stage_ctas} CTAs" if args.stage_ctas > 0 else "copy engine",
                          "h2d_gbs_if_copy_bound": h2d * k_e2e / (ms_e * 1e-3) / 1e9}
         sess2.close()
