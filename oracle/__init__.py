@@ -59,6 +59,16 @@ def _load():
         lib.matkv_oracle_lse_merge.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.matkv_oracle_rope.restype = None
         lib.matkv_oracle_rope.argtypes = [C.c_int32, C.c_int32, C.c_double, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.matkv_oracle_e4m3_value.restype = C.c_double
+        lib.matkv_oracle_e4m3_value.argtypes = [C.c_uint8]
+        lib.matkv_oracle_e4m3_encode.restype = C.c_uint8
+        lib.matkv_oracle_e4m3_encode.argtypes = [C.c_double]
+        lib.matkv_oracle_fp8_block_exponent.restype = C.c_int32
+        lib.matkv_oracle_fp8_block_exponent.argtypes = [C.c_double]
+        for name in ("matkv_oracle_fp8_quantize_blob", "matkv_oracle_fp8_dequantize_blob"):
+            f = getattr(lib, name)
+            f.restype = None
+            f.argtypes = [C.POINTER(_Shape), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = lib
     return _lib
 
@@ -133,6 +143,40 @@ def rope(x: np.ndarray, pos: Sequence[int], theta: float) -> np.ndarray:
     assert p.shape == (n,)
     out = np.empty_like(x)
     lib.matkv_oracle_rope(n, D, float(theta), p.ctypes.data, x.ctypes.data, out.ctypes.data)
+    return out
+
+
+def e4m3_value(code: int) -> float:
+    return float(_load().matkv_oracle_e4m3_value(int(code)))
+
+
+def e4m3_encode(x: float) -> int:
+    return int(_load().matkv_oracle_e4m3_encode(float(x)))
+
+
+def fp8_block_exponent(amax: float) -> int:
+    return int(_load().matkv_oracle_fp8_block_exponent(float(amax)))
+
+
+def fp8_quantize_blob(shape: "Shape", blob: np.ndarray):
+    """bf16 chunk blob [L, 2, Hkv, len, D] -> (e4m3 codes, same shape, uint8; exponents [L, 2, Hkv, ceil(len/64)] int8)."""
+    blob = _u16(blob)
+    L, two, Hkv, n, D = blob.shape
+    assert (L, two, Hkv, D) == (shape.n_layers, 2, shape.n_kv_heads, shape.head_dim)
+    codes = np.empty(blob.shape, dtype=np.uint8)
+    exps = np.empty((L, 2, Hkv, (n + 63) // 64), dtype=np.int8)
+    sh = shape.c()
+    _load().matkv_oracle_fp8_quantize_blob(C.byref(sh), n, blob.ctypes.data, codes.ctypes.data, exps.ctypes.data)
+    return codes, exps
+
+
+def fp8_dequantize_blob(shape: "Shape", codes: np.ndarray, exps: np.ndarray) -> np.ndarray:
+    """The bf16 blob a compressed chunk stands for (exact: every value(code) * 2^e is a bf16 number)."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    exps = np.ascontiguousarray(exps, dtype=np.int8)
+    out = np.empty(codes.shape, dtype=np.uint16)
+    sh = shape.c()
+    _load().matkv_oracle_fp8_dequantize_blob(C.byref(sh), codes.shape[3], codes.ctypes.data, exps.ctypes.data, out.ctypes.data)
     return out
 
 

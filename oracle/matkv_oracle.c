@@ -284,3 +284,80 @@ void matkv_oracle_rope(int32_t n_vec, int32_t D, double theta, const int64_t *po
             out[(size_t)i * D + d + half] = narrow_rne(b * c + a * s);
         }
 }
+
+/* ---- fp8 chunk codec (compressed store; the paper names KV compression as the lever on storage cost,
+ *      "Total Cost of Ownership" discussion, without fixing a format) -------------------------------------
+ * Format taken here: every block of up to 64 consecutive tokens of one (layer, K or V, KV head) slab, i.e.
+ * up to 64 x D values, shares one power-of-two scale 2^e (e an int8); each value is stored as an e4m3 code
+ * (1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest finite 448; the two NaN codes
+ * 0x7f / 0xff are never produced).  A stored value stands for  value(code) * 2^e,  which is always exactly
+ * representable in bf16, so attention over a compressed chunk is attention over ordinary bf16 numbers.
+ *   e      = the smallest integer with  amax * 2^-e <= 448  (amax = largest magnitude in the block),
+ *            0 for an all-zero block, clamped to [-127, 127];
+ *   code   = the e4m3 number nearest to  x * 2^-e,  ties to the code with an even mantissa.
+ * Inputs must be finite. */
+double matkv_oracle_e4m3_value(uint8_t code) {
+    const int s = code >> 7, E = (code >> 3) & 15, M = code & 7;
+    const double mag = E == 0 ? ldexp((double)M, -9) : ldexp(1.0 + (double)M / 8.0, E - 7);
+    return s ? -mag : mag;
+}
+
+/* nearest e4m3 code by exhaustive search over the 127 finite magnitudes (0x00 .. 0x7e) */
+uint8_t matkv_oracle_e4m3_encode(double x) {
+    const double a = fabs(x);
+    int best = 0;
+    double best_d = a; /* distance to code 0 */
+    for (int c = 1; c <= 0x7e; ++c) {
+        const double d = fabs(a - matkv_oracle_e4m3_value((uint8_t)c));
+        if (d < best_d || (d == best_d && (c & 1) == 0)) { /* a tie is between neighbours: keep the even one */
+            best_d = d;
+            best = c;
+        }
+    }
+    if (best == 0) return 0; /* zero carries no sign */
+    return (uint8_t)(best | (x < 0 ? 0x80 : 0));
+}
+
+int32_t matkv_oracle_fp8_block_exponent(double amax) {
+    if (amax == 0.0) return 0;
+    int32_t e = -200;
+    while (ldexp(amax, -e) > 448.0) ++e;
+    if (e < -127) e = -127;
+    if (e > 127) e = 127;
+    return e;
+}
+
+/* One block: n_el bf16 values -> n_el codes and the block's exponent. */
+void matkv_oracle_fp8_quantize_block(int64_t n_el, const uint16_t *x, uint8_t *codes, int8_t *e_out) {
+    double amax = 0.0;
+    for (int64_t i = 0; i < n_el; ++i) amax = fmax(amax, fabs(widen(x[i])));
+    const int32_t e = matkv_oracle_fp8_block_exponent(amax);
+    for (int64_t i = 0; i < n_el; ++i) codes[i] = matkv_oracle_e4m3_encode(ldexp(widen(x[i]), -e));
+    *e_out = (int8_t)e;
+}
+
+/* A whole chunk blob [L][2][Hkv][len][D] bf16 -> codes of the same shape and exponents [L][2][Hkv][ceil(len/64)]. */
+void matkv_oracle_fp8_quantize_blob(const matkv_oracle_shape *sh, int32_t len, const uint16_t *blob, uint8_t *codes,
+                                    int8_t *exps) {
+    const int32_t D = sh->head_dim, nb = (len + 63) / 64;
+    const int64_t n_slab = (int64_t)sh->n_layers * 2 * sh->n_kv_heads;
+    for (int64_t s = 0; s < n_slab; ++s)
+        for (int32_t b = 0; b < nb; ++b) {
+            const int32_t t0 = b * 64, nt = len - t0 < 64 ? len - t0 : 64;
+            const int64_t off = (s * len + t0) * D;
+            matkv_oracle_fp8_quantize_block((int64_t)nt * D, blob + off, codes + off, exps + s * nb + b);
+        }
+}
+
+/* ... and back: bf16 bit patterns of value(code) * 2^e (exact). */
+void matkv_oracle_fp8_dequantize_blob(const matkv_oracle_shape *sh, int32_t len, const uint8_t *codes, const int8_t *exps,
+                                      uint16_t *blob) {
+    const int32_t D = sh->head_dim, nb = (len + 63) / 64;
+    const int64_t n_slab = (int64_t)sh->n_layers * 2 * sh->n_kv_heads;
+    for (int64_t s = 0; s < n_slab; ++s)
+        for (int32_t t = 0; t < len; ++t)
+            for (int32_t d = 0; d < D; ++d) {
+                const int64_t i = (s * len + t) * D + d;
+                blob[i] = narrow_rne(ldexp(matkv_oracle_e4m3_value(codes[i]), exps[s * nb + t / 64]));
+            }
+}
