@@ -131,6 +131,29 @@ int matkv_register_chunk_file(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_token
  * slab_bytes (>= the largest file-backed chunk, a multiple of 4096, at least two slabs), and starts
  * n_io_threads reader threads.  Storage reads, host-to-device copies and GPU work then overlap.      */
 int matkv_set_bounce_buffer(matkv_ctx *ctx, void *pinned_host, size_t bytes, size_t slab_bytes, int32_t n_io_threads);
+/* ---- compressed chunk store (the paper names KV compression as the lever on the storage cost of
+ *      materialised KVs, in its discussion of total cost of ownership, without fixing a format) ----------
+ * Format taken here: e4m3 codes (1-4-3 bits, bias 7, largest finite 448) with one power-of-two scale 2^e per
+ * block of 64 consecutive tokens of a (layer, K or V, KV head) slab; a code stands for value(code) * 2^e,
+ * always a bf16 number.  e = the smallest integer with amax * 2^-e <= 448 (0 for an all-zero block, clamped
+ * to [-127, 127]); code = nearest e4m3 to x * 2^-e, ties to even, zero unsigned.  Inputs must be finite.
+ * Compressed blob: codes [n_layers][2][n_kv_heads][n_tokens][head_dim] (bytes), then, at the next multiple
+ * of 256 bytes, exponents [n_layers][2][n_kv_heads][ceil(n_tokens / 64)] (int8).  It halves the bytes on
+ * storage and on the host-to-device link; staging expands it to the ordinary bf16 chunk blob in HBM (exactly),
+ * so tables and attention calls do not change.
+ *   matkv_fp8_blob_bytes     size of the compressed blob of an n_tokens chunk (a multiple of 256).
+ *   matkv_quantize_chunk_fp8 bf16 chunk blob (device) -> compressed blob (device, 256-byte aligned), on `stream`;
+ *                            the materialisation side: copy the result to the host or a file afterwards.
+ *   matkv_register_chunk_fp8 like matkv_register_chunk for a compressed blob in PINNED host memory (256-byte
+ *                            aligned; the expanding copy kernel reads it over the link, MATKV_OPT_STAGE_CTAS
+ *                            CTAs, 16 when that option is 0).  Slots are sized for the bf16 blob.
+ *   matkv_register_chunk_file_fp8  the same for a compressed blob stored in a file (see
+ *                            matkv_register_chunk_file); it passes through the pinned bounce ring.             */
+size_t matkv_fp8_blob_bytes(const matkv_ctx *ctx, int32_t n_tokens);
+int matkv_quantize_chunk_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_blob_fp8, void *stream);
+int matkv_register_chunk_fp8(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const void *host_blob_fp8);
+int matkv_register_chunk_file_fp8(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const char *path, uint64_t file_offset);
+
 /* The paper's delete(O) (Section IV): forgets the chunk.  Tables built earlier keep the
  * device address they resolved; the caller keeps that memory alive until they are freed.    */
 int matkv_unregister_chunk(matkv_ctx *ctx, uint64_t chunk_id);

@@ -28,6 +28,7 @@ EXPORTS = [
     "matkv_probe_read", "matkv_attend_decode_static", "matkv_selftest_wait_timeout",
     "matkv_register_chunk_file", "matkv_set_bounce_buffer", "matkv_export_tail_as_chunk",
     "matkv_attend_prefill_all_layers", "matkv_table_sharing", "matkv_table_workspace_bytes",
+    "matkv_fp8_blob_bytes", "matkv_quantize_chunk_fp8", "matkv_register_chunk_fp8", "matkv_register_chunk_file_fp8",
 ]
 
 
@@ -87,6 +88,10 @@ def lib() -> C.CDLL:
             "matkv_attend_prefill_all_layers": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp]),
             "matkv_table_sharing": (C.c_int, [vp, C.POINTER(i64), C.POINTER(i64)]),
             "matkv_table_workspace_bytes": (C.c_size_t, [vp, i32]),
+            "matkv_fp8_blob_bytes": (C.c_size_t, [vp, i32]),
+            "matkv_quantize_chunk_fp8": (C.c_int, [vp, vp, i32, vp, vp]),
+            "matkv_register_chunk_fp8": (C.c_int, [vp, u64, i32, vp]),
+            "matkv_register_chunk_file_fp8": (C.c_int, [vp, u64, i32, C.c_char_p, u64]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -259,3 +264,19 @@ def matkv_table_sharing(table: int):
 
 def matkv_table_workspace_bytes(table: int, n_layers_launch: int) -> int:
     return int(lib().matkv_table_workspace_bytes(table, n_layers_launch))
+
+
+def matkv_fp8_blob_bytes(ctx: int, n_tokens: int) -> int:
+    return int(lib().matkv_fp8_blob_bytes(ctx, n_tokens))
+
+
+def matkv_quantize_chunk_fp8(ctx: int, dev_blob: int, n_tokens: int, dev_blob_fp8: int, stream: int = 0) -> None:
+    _check(lib().matkv_quantize_chunk_fp8(ctx, dev_blob, n_tokens, dev_blob_fp8, stream or None))
+
+
+def matkv_register_chunk_fp8(ctx: int, chunk_id: int, n_tokens: int, host_blob_fp8: int) -> None:
+    _check(lib().matkv_register_chunk_fp8(ctx, chunk_id, n_tokens, host_blob_fp8))
+
+
+def matkv_register_chunk_file_fp8(ctx: int, chunk_id: int, n_tokens: int, path: str, file_offset: int = 0) -> None:
+    _check(lib().matkv_register_chunk_file_fp8(ctx, chunk_id, n_tokens, path.encode(), file_offset))

@@ -1,0 +1,149 @@
+// Compressed chunk store: a materialised chunk kept on the host (or in a file) as e4m3 codes with one
+// power-of-two scale per block of 64 tokens of a (layer, K or V, KV head) slab, expanded to the ordinary
+// bf16 chunk blob while it is staged into HBM.  The paper names KV compression as the lever on the storage
+// cost of materialised KVs (its discussion of total cost of ownership) and loading as the cost that
+// replaces prefill; this halves the bytes on storage and on the host-to-device link.  Attention itself
+// still reads bf16 from HBM: every value a code stands for, value(code) * 2^e, is a bf16 number, so the
+// expansion is exact and the attention kernels are unchanged.
+//
+// Blob layout: codes [L][2][Hkv][n_tokens][D] (one byte each), then, at the next multiple of 256 bytes,
+// exponents [L][2][Hkv][ceil(n_tokens / 64)] (int8).
+#include <cuda_fp8.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+
+#include "matkv_internal.h"
+
+namespace matkv {
+
+static size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+
+size_t fp8_codes_bytes(const matkv_config &c, int32_t n_tokens) {
+    return (size_t)c.n_layers * 2 * c.n_kv_heads * (size_t)n_tokens * c.head_dim;
+}
+size_t fp8_blob_bytes(const matkv_config &c, int32_t n_tokens) {
+    return up256(fp8_codes_bytes(c, n_tokens)) + up256((size_t)c.n_layers * 2 * c.n_kv_heads * ((n_tokens + 63) / 64));
+}
+
+// ---- quantiser: one CTA per (slab, 64-token block) -------------------------------------------------------
+// e = the smallest integer with amax * 2^-e <= 448 = 1.75 * 2^8 (0 for an all-zero block, clamped to
+// [-127, 127]), read off the bf16 bits of amax; code = e4m3 nearest to x * 2^-e, ties to even, and a zero
+// carries no sign.  Inputs must be finite.
+__global__ void __launch_bounds__(256) k_quantize_fp8(const uint16_t *__restrict__ blob, uint8_t *__restrict__ codes,
+                                                      int8_t *__restrict__ exps, int32_t n_tokens, int32_t D, int32_t nb) {
+    __shared__ uint32_t s_max[8];
+    __shared__ int s_e;
+    const int64_t slab = blockIdx.y;
+    const int b = blockIdx.x;
+    const int t0 = b * 64, nt = min(64, n_tokens - t0);
+    const int64_t off = (slab * n_tokens + t0) * D;
+    const int n_el = nt * D;
+    uint32_t m = 0;
+    for (int i = threadIdx.x; i < n_el; i += blockDim.x) m = max(m, (uint32_t)(blob[off + i] & 0x7fffu));  // |x| orders like its bits
+#pragma unroll
+    for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t a = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) a = max(a, s_max[w]);
+        int e = 0;
+        if (a != 0) {
+            const int E = (int)(a >> 7), frac = (int)(a & 0x7f);
+            e = E == 0 ? -127 : (E - 127) - 8 + (frac > 0x60 ? 1 : 0);  // amax = (1 + frac/128) * 2^(E-127); 1.75 = 1 + 0x60/128
+            e = max(-127, min(127, e));
+        }
+        s_e = e;
+        exps[slab * nb + b] = (int8_t)e;
+    }
+    __syncthreads();
+    const int e = s_e;
+    for (int i = threadIdx.x; i < n_el; i += blockDim.x) {
+        const float x = __uint_as_float((uint32_t)blob[off + i] << 16);
+        uint8_t c = (uint8_t)__nv_cvt_float_to_fp8(ldexpf(x, -e), __NV_SATFINITE, __NV_E4M3);  // exact scaling, then round to nearest even
+        if ((c & 0x7f) == 0) c = 0;
+        codes[off + i] = c;
+    }
+}
+
+// ---- expanding copy: compressed blob (pinned host memory or device memory) -> bf16 blob in HBM -----------
+// A few small CTAs, like the plain staging copy kernel: they sit beside the decode CTAs and keep the loads
+// over the link in flight.  The exponents (a few KB) are first brought into shared memory by every CTA.
+__global__ void __launch_bounds__(128) k_stage_expand_fp8(const uint4 *__restrict__ codes, const int8_t *__restrict__ exps,
+                                                          uint4 *__restrict__ out, int64_t n_vec, int32_t vec_per_slab,
+                                                          int32_t vec_per_block, int32_t nb, int32_t n_exps) {
+    extern __shared__ __align__(16) int8_t s_exps[];
+    // 16 bytes per load: the exponent area is padded to a multiple of 256 bytes, and every load crosses the link
+    for (int i = threadIdx.x; i < (n_exps + 15) / 16; i += blockDim.x) ((uint4 *)s_exps)[i] = __ldcs((const uint4 *)exps + i);
+    __syncthreads();
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n_vec; i0 += 4 * stride) {
+        uint4 v[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            if (i0 + k * stride < n_vec) v[k] = __ldcs(codes + i0 + k * stride);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int64_t i = i0 + k * stride;   // 16 codes: never across a block, a block is a multiple of 16 codes
+            if (i >= n_vec) break;
+            const int64_t slab = i / vec_per_slab;
+            const int blk = (int)((i % vec_per_slab) / vec_per_block);
+            const int e = s_exps[slab * nb + blk];
+            const float scale = __uint_as_float(e > -127 ? (uint32_t)(e + 127) << 23 : 0x00400000u);  // 2^e (2^-127 is a subnormal float)
+            const uint32_t w[4] = {v[k].x, v[k].y, v[k].z, v[k].w};
+            uint32_t o[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t c0 = (w[j] >> (16 * h)) & 0xffu, c1 = (w[j] >> (16 * h + 8)) & 0xffu;
+                    // the code's 7 magnitude bits sit where a float keeps its low exponent bits and top mantissa bits:
+                    // that float is value(code) * 2^-120, subnormal codes included
+                    const float f0 = __uint_as_float(((c0 & 0x80u) << 24) | ((c0 & 0x7fu) << 20)) * 0x1p120f * scale;
+                    const float f1 = __uint_as_float(((c1 & 0x80u) << 24) | ((c1 & 0x7fu) << 20)) * 0x1p120f * scale;
+                    __nv_bfloat162 p = __floats2bfloat162_rn(f0, f1);
+                    o[2 * j + h] = *reinterpret_cast<uint32_t *>(&p);
+                }
+            }
+            out[2 * i] = make_uint4(o[0], o[1], o[2], o[3]);
+            out[2 * i + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+    }
+}
+
+int launch_quantize_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_fp8, cudaStream_t stream) {
+    const matkv_config &c = ctx->cfg;
+    const int nb = (n_tokens + 63) / 64;
+    const int64_t n_slab = (int64_t)c.n_layers * 2 * c.n_kv_heads;
+    if (n_slab > 65535) return fail(MATKV_E_CAPACITY, "too many (layer, head) slabs for one quantiser launch");
+    uint8_t *codes = (uint8_t *)dev_fp8;
+    int8_t *exps = (int8_t *)(codes + up256(fp8_codes_bytes(c, n_tokens)));
+    k_quantize_fp8<<<dim3(nb, (unsigned)n_slab), 256, 0, stream>>>((const uint16_t *)dev_blob, codes, exps, n_tokens, c.head_dim, nb);
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
+int launch_stage_expand_fp8(matkv_ctx *ctx, const void *src_fp8, void *dev_dst, int32_t n_tokens, int n_ctas, cudaStream_t stream) {
+    const matkv_config &c = ctx->cfg;
+    const int nb = (n_tokens + 63) / 64;
+    const int64_t n_slab = (int64_t)c.n_layers * 2 * c.n_kv_heads;
+    const int64_t n_exps = n_slab * nb;
+    if (n_exps > 200 * 1024) return fail(MATKV_E_CAPACITY, "%lld block exponents do not fit the expanding copy's shared memory", (long long)n_exps);
+    const uint8_t *codes = (const uint8_t *)src_fp8;
+    const int8_t *exps = (const int8_t *)(codes + up256(fp8_codes_bytes(c, n_tokens)));
+    const int64_t n_vec = (int64_t)(fp8_codes_bytes(c, n_tokens) / 16);
+    const int32_t vec_per_slab = (int32_t)((int64_t)n_tokens * c.head_dim / 16);
+    const int32_t vec_per_block = 64 * c.head_dim / 16;
+    static bool configured = false;
+    if (!configured) {
+        MATKV_CUDA(cudaFuncSetAttribute(k_stage_expand_fp8, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        configured = true;
+    }
+    k_stage_expand_fp8<<<n_ctas, 128, (size_t)((n_exps + 15) / 16 * 16), stream>>>((const uint4 *)codes, exps, (uint4 *)dev_dst, n_vec, vec_per_slab,
+                                                                                 vec_per_block, nb, (int32_t)n_exps);
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
+}  // namespace matkv

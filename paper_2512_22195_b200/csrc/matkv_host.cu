@@ -345,6 +345,64 @@ int matkv_register_chunk_file(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_token
     return MATKV_OK;
 }
 
+// ---- compressed chunk store -------------------------------------------------------------------
+size_t matkv_fp8_blob_bytes(const matkv_ctx *ctx, int32_t n_tokens) {
+    if (!ctx || n_tokens < 1) return 0;
+    return fp8_blob_bytes(ctx->cfg, n_tokens);
+}
+
+int matkv_quantize_chunk_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_blob_fp8, void *stream) {
+    if (!ctx || !dev_blob || !dev_blob_fp8) return fail(MATKV_E_INVALID_ARG, "matkv_quantize_chunk_fp8: null argument");
+    if (n_tokens < 1) return fail(MATKV_E_INVALID_ARG, "matkv_quantize_chunk_fp8: n_tokens must be >= 1");
+    if ((uintptr_t)dev_blob % 16 || (uintptr_t)dev_blob_fp8 % 256)
+        return fail(MATKV_E_ALIGNMENT, "matkv_quantize_chunk_fp8: the bf16 blob must be 16-byte, the fp8 blob 256-byte aligned");
+    DeviceGuard guard(ctx->device);
+    return launch_quantize_fp8(ctx, dev_blob, n_tokens, dev_blob_fp8, (cudaStream_t)stream);
+}
+
+int matkv_register_chunk_fp8(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const void *host_blob_fp8) {
+    if (!ctx || !host_blob_fp8) return fail(MATKV_E_INVALID_ARG, "matkv_register_chunk_fp8: null argument");
+    if (n_tokens < 1) return fail(MATKV_E_INVALID_ARG, "chunk %llu: n_tokens must be >= 1", (unsigned long long)chunk_id);
+    if ((int64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * n_tokens >= (int64_t)1 << 31)
+        return fail(MATKV_E_CAPACITY, "chunk %llu: layers x 2 x KV heads x tokens must stay below 2^31 rows", (unsigned long long)chunk_id);
+    if ((uintptr_t)host_blob_fp8 % 256)
+        return fail(MATKV_E_ALIGNMENT, "chunk %llu: the compressed blob must be 256-byte aligned", (unsigned long long)chunk_id);
+    if (ctx->chunks.count(chunk_id))
+        return fail(MATKV_E_INVALID_ARG, "chunk %llu is already registered", (unsigned long long)chunk_id);
+    {   // the expanding copy kernel reads the blob over the link: it must be page-locked, device-accessible memory
+        DeviceGuard guard(ctx->device);
+        cudaPointerAttributes at;
+        cudaError_t e = cudaPointerGetAttributes(&at, host_blob_fp8);
+        if (e != cudaSuccess || (at.type != cudaMemoryTypeHost && at.type != cudaMemoryTypeManaged && at.type != cudaMemoryTypeDevice)) {
+            cudaGetLastError();
+            return fail(MATKV_E_INVALID_ARG, "chunk %llu: the compressed blob must be pinned (page-locked) host memory", (unsigned long long)chunk_id);
+        }
+    }
+    Chunk c;
+    c.n_tokens = n_tokens;
+    c.host_blob = host_blob_fp8;
+    c.fp8 = true;
+    ctx->chunks.emplace(chunk_id, c);
+    return MATKV_OK;
+}
+
+int matkv_register_chunk_file_fp8(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const char *path, uint64_t file_offset) {
+    if (!ctx || !path) return fail(MATKV_E_INVALID_ARG, "matkv_register_chunk_file_fp8: null argument");
+    if (n_tokens < 1) return fail(MATKV_E_INVALID_ARG, "chunk %llu: n_tokens must be >= 1", (unsigned long long)chunk_id);
+    if ((int64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * n_tokens >= (int64_t)1 << 31)
+        return fail(MATKV_E_CAPACITY, "chunk %llu: layers x 2 x KV heads x tokens must stay below 2^31 rows", (unsigned long long)chunk_id);
+    if (ctx->chunks.count(chunk_id))
+        return fail(MATKV_E_INVALID_ARG, "chunk %llu is already registered", (unsigned long long)chunk_id);
+    Chunk c;
+    c.n_tokens = n_tokens;
+    c.file_offset = file_offset;
+    c.fp8 = true;
+    int rc = open_chunk_file(path, file_offset, fp8_blob_bytes(ctx->cfg, n_tokens), &c.file_fd);
+    if (rc) return rc;
+    ctx->chunks.emplace(chunk_id, c);
+    return MATKV_OK;
+}
+
 int matkv_set_bounce_buffer(matkv_ctx *ctx, void *pinned_host, size_t bytes, size_t slab_bytes, int32_t n_io_threads) {
     if (!ctx || !pinned_host) return fail(MATKV_E_INVALID_ARG, "matkv_set_bounce_buffer: null argument");
     if ((uintptr_t)pinned_host % 4096 || slab_bytes == 0 || slab_bytes % 4096)
@@ -393,10 +451,11 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
         if (c.dev_blob) continue;  // resident: nothing to do
         if (!c.host_blob && c.file_fd < 0)
             return fail(MATKV_E_INVALID_ARG, "chunk %llu has no host blob or file to stage", (unsigned long long)ids[i]);
-        if (c.file_fd >= 0 && !c.host_blob && blob_bytes(ctx->cfg, c.n_tokens) > io_engine_slab_bytes(ctx))
+        const size_t stored = c.fp8 ? fp8_blob_bytes(ctx->cfg, c.n_tokens) : blob_bytes(ctx->cfg, c.n_tokens);
+        if (c.file_fd >= 0 && !c.host_blob && stored > io_engine_slab_bytes(ctx))
             return fail(ctx->io ? MATKV_E_CAPACITY : MATKV_E_INVALID_ARG,
                         "chunk %llu lives in a file: set a bounce buffer with slabs of at least %zu bytes first",
-                        (unsigned long long)ids[i], blob_bytes(ctx->cfg, c.n_tokens));
+                        (unsigned long long)ids[i], stored);
         if (blob_bytes(ctx->cfg, c.n_tokens) > slot_bytes)
             return fail(MATKV_E_CAPACITY, "chunk %llu (%zu bytes) does not fit a slot of %zu bytes",
                         (unsigned long long)ids[i], blob_bytes(ctx->cfg, c.n_tokens), slot_bytes);
@@ -457,7 +516,15 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
         }
         if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;  // moves from another region
         void *dst = (char *)dev_slots + (size_t)next_free * slot_bytes;
-        if (c.host_blob && ctx->opt_stage_ctas > 0) {
+        if (c.host_blob && c.fp8) {
+            // compressed chunk: expanded to bf16 on its way in (always by the SM copy kernel; the host blob must be
+            // device-accessible pinned memory)
+            int rc = launch_stage_expand_fp8(ctx, c.host_blob, dst, c.n_tokens, ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, cs);
+            if (rc) {
+                cudaEventDestroy(tk.done);
+                return rc;
+            }
+        } else if (c.host_blob && ctx->opt_stage_ctas > 0) {
             // SM-driven copy (the host blob must be device-accessible: pinned memory under unified addressing)
             int rc = launch_stage_copy(ctx, c.host_blob, dst, blob_bytes(ctx->cfg, c.n_tokens), (int)ctx->opt_stage_ctas, cs);
             if (rc) {
@@ -471,7 +538,8 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
                 return cuda_fail(e, "staging copy");
             }
         } else {  // storage tier: read into the bounce ring, then copy, all in the copy stream's order
-            int rc = io_engine_stage(ctx, c.file_fd, c.file_offset, blob_bytes(ctx->cfg, c.n_tokens), dst, cs);
+            int rc = io_engine_stage(ctx, c.file_fd, c.file_offset, c.fp8 ? fp8_blob_bytes(ctx->cfg, c.n_tokens) : blob_bytes(ctx->cfg, c.n_tokens),
+                                     dst, cs, c.fp8 ? c.n_tokens : 0);
             if (rc) {
                 cudaEventDestroy(tk.done);
                 return rc;

@@ -60,6 +60,7 @@ struct Chunk {
     int file_fd = -1;              // >= 0: the blob lives in a file, at file_offset
     uint64_t file_offset = 0;
     void *dev_blob = nullptr;      // caller-resident device copy
+    bool fp8 = false;              // host_blob / the file holds the compressed form (e4m3 codes + block exponents)
     void *staged = nullptr;        // device copy inside a slot region (or nullptr)
     Region *region = nullptr;
     int32_t slot = -1;
@@ -182,7 +183,12 @@ int io_engine_create(matkv_ctx *ctx, void *pinned, size_t bytes, size_t slab_byt
 void io_engine_destroy(matkv_ctx *ctx);
 size_t io_engine_slab_bytes(const matkv_ctx *ctx);
 int io_engine_errors(matkv_ctx *ctx, const char **msg);
-int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream);
+// fp8_tokens > 0: the file holds a compressed chunk of that many tokens, expanded on its way from the slab to dst
+int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream, int32_t fp8_tokens = 0);
+size_t fp8_codes_bytes(const matkv_config &c, int32_t n_tokens);
+size_t fp8_blob_bytes(const matkv_config &c, int32_t n_tokens);
+int launch_quantize_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_fp8, cudaStream_t stream);
+int launch_stage_expand_fp8(matkv_ctx *ctx, const void *src_fp8, void *dev_dst, int32_t n_tokens, int n_ctas, cudaStream_t stream);
 int open_chunk_file(const char *path, uint64_t offset, size_t bytes, int *fd_out);
 void close_chunk_file(int fd);
 int launch_wait_selftest(matkv_ctx *ctx, double seconds, cudaStream_t stream);
