@@ -206,32 +206,52 @@ def run_pipeline(args):
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, args.decode_ctas)
     tmp = torch.empty((L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
     host_pool = ring = None
+    fp8 = args.kv_store == "fp8"
+    stored_bytes = mk.matkv_fp8_blob_bytes(sess.ctx, w.chunk_tokens) if fp8 else slot_bytes   # bytes of a chunk where it is kept
+    tmp8 = torch.empty(stored_bytes, dtype=torch.uint8, device=dev) if fp8 else None
+
+    def chunk_to(dst_u8, c):
+        """Chunk c's stored form (generated on the device, compressed there if asked) into a pinned uint8 buffer."""
+        gen.fill_bf16(tmp, w.seed, mi.STREAM_CHUNK + c)
+        if fp8:
+            mk.matkv_quantize_chunk_fp8(sess.ctx, tmp.data_ptr(), w.chunk_tokens, tmp8.data_ptr())
+            dst_u8.copy_(tmp8)
+        else:
+            dst_u8.copy_(tmp.view(torch.uint8).reshape(-1))
+
     if args.store_dir:
         # the materialised-KV store: one raw-bytes file per chunk id
         os.makedirs(args.store_dir, exist_ok=True)
-        bounce = torch.empty(tmp.shape, dtype=torch.bfloat16, pin_memory=True)
+        bounce = torch.empty(stored_bytes, dtype=torch.uint8, pin_memory=True)
         t_w = time.perf_counter()
         for c in range(w.pool_chunks):
-            path = os.path.join(args.store_dir, f"{c}.kv")
-            if not (os.path.exists(path) and os.path.getsize(path) == slot_bytes):
-                gen.fill_bf16(tmp, w.seed, mi.STREAM_CHUNK + c)
-                bounce.copy_(tmp)
+            path = os.path.join(args.store_dir, f"{c}.kv8" if fp8 else f"{c}.kv")
+            if not (os.path.exists(path) and os.path.getsize(path) == stored_bytes):
+                chunk_to(bounce, c)
                 torch.cuda.synchronize()
                 with open(path, "wb") as f:
-                    f.write(memoryview(bounce.view(torch.uint8).numpy()))
-            mk.matkv_register_chunk_file(sess.ctx, c, w.chunk_tokens, path, 0)
+                    f.write(memoryview(bounce.numpy()))
+            if fp8:
+                mk.matkv_register_chunk_file_fp8(sess.ctx, c, w.chunk_tokens, path, 0)
+            else:
+                mk.matkv_register_chunk_file(sess.ctx, c, w.chunk_tokens, path, 0)
         os.sync()
         log(f"[pipeline] store written/checked in {time.perf_counter() - t_w:.1f} s")
         n_slabs = 8
-        ring = torch.empty(n_slabs * slot_bytes + 4096, dtype=torch.uint8, pin_memory=True)
+        slab = (stored_bytes + 4095) // 4096 * 4096
+        ring = torch.empty(n_slabs * slab + 4096, dtype=torch.uint8, pin_memory=True)
         ring_base = (ring.data_ptr() + 4095) // 4096 * 4096
-        mk.matkv_set_bounce_buffer(sess.ctx, ring_base, n_slabs * slot_bytes, slot_bytes, args.io_threads)
+        mk.matkv_set_bounce_buffer(sess.ctx, ring_base, n_slabs * slab, slab, args.io_threads)
     else:
-        host_pool = torch.empty((w.pool_chunks, L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, pin_memory=True)
+        host_pool = torch.empty((w.pool_chunks, stored_bytes), dtype=torch.uint8, pin_memory=True)
         for c in range(w.pool_chunks):
-            gen.fill_bf16(tmp, w.seed, mi.STREAM_CHUNK + c)
-            host_pool[c].copy_(tmp)
-            mk.matkv_register_chunk(sess.ctx, c, w.chunk_tokens, host_pool[c].data_ptr(), None)
+            chunk_to(host_pool[c], c)
+            if fp8:
+                mk.matkv_register_chunk_fp8(sess.ctx, c, w.chunk_tokens, host_pool[c].data_ptr())
+            else:
+                mk.matkv_register_chunk(sess.ctx, c, w.chunk_tokens, host_pool[c].data_ptr(), None)
+    torch.cuda.synchronize()
+    del tmp8
     del tmp
     slots = [torch.empty(n_slots * slot_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
     q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device=dev)
@@ -319,7 +339,7 @@ def run_pipeline(args):
         n_copied += len(new)
         occ[n % 2] = set(needed[n])
         occ[(n + 1) % 2] -= new
-    staged_bytes = n_copied * slot_bytes
+    staged_bytes = n_copied * stored_bytes          # bytes that crossed the link (or left storage)
     tokens = n_batches * B * T
     kv_bytes = sum((len(row) * w.chunk_tokens + S + t + 1) * w.beta for ids in batches for row in ids for t in range(T)) * L
     t_compute = t_serial - t_stage
@@ -328,7 +348,9 @@ def run_pipeline(args):
         "warmup": 2, "ms_per_step": 1e3 * t_pipe / n_batches, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 in, fp32 softmax/accumulate", "data": "synthetic",
         "config": {"workload": w.name, "layers": L, "batch": B, "chunks_per_request": w.chunks_per_req, "suffix": S,
-                   "decode_steps": T, "pool_chunks": w.pool_chunks, "pinned_pool_gb": w.pool_chunks * slot_bytes / 1e9,
+                   "decode_steps": T, "pool_chunks": w.pool_chunks, "pinned_pool_gb": w.pool_chunks * stored_bytes / 1e9,
+                   "kv_store": ("e4m3 codes + power-of-two scale per 64-token block, expanded to bf16 while staged (lossy store: "
+                                "a workload of its own)" if fp8 else "bf16"),
                    "batches": n_batches, "timing": "host wall clock around synchronised passes (copy and compute streams)",
                    "chunk_pool": (f"files in {args.store_dir} read with O_DIRECT by {args.io_threads} threads through a pinned ring of 8 slabs"
                                   if args.store_dir else "pinned host memory"),
@@ -336,7 +358,8 @@ def run_pipeline(args):
         "clocks": clocks,
         "pipeline": {"t_stage_s": t_stage, "t_serial_s": t_serial, "t_pipelined_s": t_pipe,
                      ("storage_to_hbm_gbs_staging_alone" if args.store_dir else "h2d_gbs_staging_alone"): staged_bytes / t_stage / 1e9,
-                     "staged_bytes": staged_bytes, "load_s_per_request_staging_alone": t_stage / (n_batches * B),
+                     "staged_bytes": staged_bytes, "bf16_bytes_delivered_to_hbm": n_copied * slot_bytes,
+                     "load_s_per_request_staging_alone": t_stage / (n_batches * B),
                      "overlap_efficiency": (t_serial - t_pipe) / t_stage if t_stage > 0 else None,
                      "requests_per_s": n_batches * B / t_pipe, "compute_s_estimate": t_compute,
                      "decode_kv_gbs_pipelined_lower_bound": kv_bytes / t_pipe / 1e9},
@@ -368,6 +391,9 @@ def main():
                     "engine; -1 = auto: 16 CTAs in the pipelined-serving mode (long decode launches that saturate HBM starve "
                     "the copy engine), copy engine in the single-batch end-to-end leg (short launches: a co-resident copy "
                     "CTA makes its SM the straggler of every launch)")
+    ap.add_argument("--kv-store", default="bf16", choices=["bf16", "fp8"],
+                    help="pipelined serving: keep the host / file chunk pool as plain bf16 blobs or compressed (e4m3 codes with a "
+                    "power-of-two scale per 64-token block, expanded to bf16 while staged; a lossy store, so a separate workload)")
     ap.add_argument("--decode-impl", type=int, default=0, choices=[0, 1, 2],
                     help="decode kernel: 0 auto (chunk-major when the batch's requests share chunks), 1 request-major, 2 chunk-major")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")

@@ -78,13 +78,13 @@ __global__ void __launch_bounds__(128) k_stage_expand_fp8(const uint4 *__restric
     for (int i = threadIdx.x; i < (n_exps + 15) / 16; i += blockDim.x) ((uint4 *)s_exps)[i] = __ldcs((const uint4 *)exps + i);
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n_vec; i0 += 4 * stride) {
-        uint4 v[4];
+    for (int64_t i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n_vec; i0 += 8 * stride) {
+        uint4 v[8];   // eight 16-byte loads in flight per thread: the link's latency is microseconds
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < 8; ++k)
             if (i0 + k * stride < n_vec) v[k] = __ldcs(codes + i0 + k * stride);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < 8; ++k) {
             const int64_t i = i0 + k * stride;   // 16 codes: never across a block, a block is a multiple of 16 codes
             if (i >= n_vec) break;
             const int64_t slab = i / vec_per_slab;
