@@ -230,12 +230,15 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
         if (tid == 0) atomicCAS(p.status, 0, MATKV_E_CAPACITY);
         t0 = max(0, min(t0, p.max_tail - p.S));
     }
-    const int tail_tiles = cdiv(t0, kTile), new_tiles = cdiv(p.S, kTile);
+    const int R = p.S * G;                       // query rows of the (request, KV head)
+    const int row0 = rb * NBLK * kRowsPerCta;
+    // new-token tiles past this CTA's last suffix token are invisible to all of its rows (causal): not visited at all,
+    // which halves the work of a long causal sub-prefill (a chunk materialised alone: S = its length, no chunks)
+    const int tok_last = min(p.S - 1, (row0 + NBLK * kRowsPerCta - 1) / G);
+    const int tail_tiles = cdiv(t0, kTile), new_tiles = tok_last / kTile + 1;
     const int T = rq.chunk_tiles + tail_tiles + new_tiles;
     const int t_begin = (int)((int64_t)sp * T / p.n_split), t_end = (int)((int64_t)(sp + 1) * T / p.n_split);
     const int n_tiles = t_end - t_begin;
-    const int R = p.S * G;                       // query rows of the (request, KV head)
-    const int row0 = rb * NBLK * kRowsPerCta;
 
     const uint32_t bar0 = smem_u32(bars);
     const uint32_t full_kv = bar0 + kBarFull * 8, empty_kv = bar0 + kBarEmpty * 8, s_full = bar0 + kBarSFull * 8,
@@ -292,6 +295,23 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
 
     if (warp == 0) {
         // ===================== producer =====================
+        // appends this split's share of the new tokens to the tail for later calls (the splits of row group 0
+        // divide the S tokens among themselves)
+        auto append_share = [&]() {
+            constexpr int CPR = D / 8;
+            const int a0 = (int)((int64_t)sp * p.S / p.n_split), a1 = (int)((int64_t)(sp + 1) * p.S / p.n_split);
+#pragma unroll 4
+            for (int idx = a0 * CPR + lane; idx < a1 * CPR; idx += 32) {
+                const int tok = idx / CPR, ch = idx % CPR;
+                if (t0 + tok < p.max_tail) {
+                    const int64_t src = (int64_t)l_rel * p.kn_sl + (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
+                    const int64_t dsto = ((((int64_t)b * p.n_layers_total + layer) * p.Hkv + g) * p.max_tail + t0 + tok) * D + ch * 8;
+                    *(uint4 *)(p.tail_k + dsto) = *(const uint4 *)(p.k_new + src);
+                    *(uint4 *)(p.tail_v + dsto) = *(const uint4 *)(p.v_new + src);
+                }
+            }
+        };
+        if (rb == 0 && n_tiles == 0) append_share();  // a split without tiles of its own still owes its share
         int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
@@ -329,22 +349,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     }
                 }
             }
-            // append this split's share of the new tokens to the tail for later calls (the splits of row
-            // group 0 divide the S tokens among themselves), once the CTA's first loads are in flight
-            if (j == 0 && rb == 0) {
-                constexpr int CPR = D / 8;
-                const int a0 = (int)((int64_t)sp * p.S / p.n_split), a1 = (int)((int64_t)(sp + 1) * p.S / p.n_split);
-#pragma unroll 4
-                for (int idx = a0 * CPR + lane; idx < a1 * CPR; idx += 32) {
-                    const int tok = idx / CPR, ch = idx % CPR;
-                    if (t0 + tok < p.max_tail) {
-                        const int64_t src = (int64_t)l_rel * p.kn_sl + (int64_t)b * p.kn_sb + (int64_t)tok * p.kn_ss + (int64_t)g * D + ch * 8;
-                        const int64_t dsto = ((((int64_t)b * p.n_layers_total + layer) * p.Hkv + g) * p.max_tail + t0 + tok) * D + ch * 8;
-                        *(uint4 *)(p.tail_k + dsto) = *(const uint4 *)(p.k_new + src);
-                        *(uint4 *)(p.tail_v + dsto) = *(const uint4 *)(p.v_new + src);
-                    }
-                }
-            }
+            if (j == 0 && rb == 0) append_share();  // once the CTA's first loads are in flight
         }
     } else if (warp == 1) {
         // ===================== MMA issuer (one thread) =====================
