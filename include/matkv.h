@@ -93,6 +93,11 @@ typedef struct {
                                       workspace has room for its partials), 1 = request-major always, 2 = chunk-major
                                       always (MATKV_E_CAPACITY when the workspace is too small) */
 #define MATKV_OPT_SHARE_TILES   7  /* chunk-major decode: 64-token tiles per work item (default 16); read when a table is built */
+#define MATKV_OPT_FP8_RESIDENT  8  /* staging of compressed chunks (matkv_register_chunk_fp8 / _file_fp8): 0 (default) = expand
+                                      to the bf16 blob in HBM; 1 = keep them compressed in HBM too (head_dim 128 only): the
+                                      streaming kernel then reads the codes and converts in registers, halving the HBM bytes of
+                                      decode; sub-prefill over such chunks also runs on the streaming kernel, and the chunk-major
+                                      decode, the allocation-free decode and matkv_gather_debug refuse tables that hold them */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
 
 /* ---- context -------------------------------------------------------------------------- */

@@ -25,6 +25,7 @@ namespace matkv {
 struct StreamParams {
     const DevReq *reqs;
     const CUtensorMap *tmaps;   // [n_seg_total] chunk maps, then tail K, tail V
+    const CUtensorMap *tmaps8;  // [n_seg_total][2] maps of compressed-resident chunks (K codes, transposed V codes), or null
     const DevSeg *segs;         // [n_seg_total]
     int32_t n_seg_total;
     const int32_t *tail_len;
@@ -136,7 +137,7 @@ __global__ void k_lse_combine(int n_rows, int P, int D, const float *__restrict_
 }
 
 // ---- K1 -------------------------------------------------------------------------------------------
-template <int D, int G>
+template <int D, int G, bool F8 = false>
 struct StreamCfg {
     static constexpr int TPU = kUnitRows / G;              // suffix tokens per unit
     static constexpr int NBOX = D / 64;                    // 64-column TMA boxes per row
@@ -150,7 +151,8 @@ struct StreamCfg {
     // that fills shared memory.  Config 2, all-layers launch: 107.7 us with 4 stages of 32 KB, 107.9 with 5,
     // 111.1 with 6; config 4: 11.63 / 11.84 / 12.50 ms.  More copies in flight than the memory latency needs
     // only lengthen the queues in front of DRAM.
-    static constexpr int NSTAGE_CAP = 128 * 1024 / STAGE_BYTES;
+    // (a tile of codes fills only half of its 32 KB stage: the compressed variant keeps six stages in flight)
+    static constexpr int NSTAGE_CAP = (F8 ? 192 : 128) * 1024 / STAGE_BYTES;
     static constexpr int NSTAGE = NSTAGE_MAX > NSTAGE_CAP ? NSTAGE_CAP : NSTAGE_MAX;
     static constexpr int SMEM_BYTES = NSTAGE * STAGE_BYTES + FIXED_BYTES;
     static_assert(G >= 1 && G <= kUnitRows && kUnitRows % G == 0, "unsupported group size");
@@ -158,10 +160,11 @@ struct StreamCfg {
 };
 
 
-template <int D, int G>
+template <int D, int G, bool F8>
 __global__ void __launch_bounds__(kThreads, 1)
 k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ CUtensorMap kn_map, const __grid_constant__ CUtensorMap vn_map) {
-    using C = StreamCfg<D, G>;
+    using C = StreamCfg<D, G, F8>;
+    static_assert(!F8 || D == 128, "compressed-resident chunks: head_dim 128 only");
     extern __shared__ unsigned char smem_raw[];
     // the swizzle pattern repeats every 1024 bytes: align the ring to it
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -221,7 +224,8 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
         // chunk rows are read once per launch unless requests share chunks: keep them out of L2's way then
         const uint64_t pol = p.stream_hint ? l2_policy_evict_first() : l2_policy_evict_normal();
         UnitPos u = range->first;
-        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;  // cursor over the request's segments
+        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0, seg_fmt = 0;  // cursor over the request's segments
+        const unsigned char *seg_base = nullptr;
         int64_t f = f_begin;
         uint32_t seq = 0;
         bool ok = true;
@@ -253,10 +257,27 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                     while (seg < 0 || t >= tiles_before + seg_tiles) {
                         tiles_before += seg_tiles;
                         ++seg;
-                        seg_len = p.segs[u.seg_begin + seg].len;
+                        const DevSeg sg = p.segs[u.seg_begin + seg];
+                        seg_len = sg.len;
+                        seg_fmt = sg.fmt;
+                        seg_base = (const unsigned char *)sg.base;
                         seg_tiles = ceil_div(seg_len, kTile);
                     }
                     const int r0 = (t - tiles_before) * kTile;
+                    if constexpr (F8) {
+                        if (seg_fmt == 1) {
+                            // codes of one 64-token block: K rows (8 KB), V transposed (8 KB), the block's exponent record (16 bytes)
+                            const int64_t blk = ((int64_t)layer * p.Hkv + u.g) * seg_tiles + (t - tiles_before);
+                            const int64_t region = ((int64_t)p.n_layers_total * p.Hkv * seg_tiles * kTile * D + 255) / 256 * 256;
+                            const CUtensorMap *m8 = p.tmaps8 + 2 * (u.seg_begin + seg);
+                            tags[stage] = (uint32_t)min(kTile, seg_len - r0) | kTagF8 | (use << 16);
+                            mbar_expect_tx(bar, 2 * kTile * D + 16);
+                            tma_load_2d_hint(dst, m8, 0, (int32_t)(blk * kTile), bar, pol);
+                            tma_load_2d_hint(dst + kTile * D, m8 + 1, 0, (int32_t)(blk * D), bar, pol);
+                            bulk_load(dst + 2 * kTile * D, seg_base + 2 * region + blk * 16, 16, bar);
+                            continue;
+                        }
+                    }
                     mk = mv = p.tmaps + u.seg_begin + seg;
                     yk = ((layer * 2) * p.Hkv + u.g) * seg_len + r0;
                     yv = ((layer * 2 + 1) * p.Hkv + u.g) * seg_len + r0;
@@ -301,6 +322,13 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
     const int mi = lane >> 3, ri = lane & 7;
 
     uint32_t qa[C::KS][2];   // A fragments of Q for the real rows: [k-step][cols 0-7 | cols 8-15]
+    // compressed tiles: the same rows as fp16 (scaled by 2^-eq so that any bf16 row fits), with the 16 dimensions of a
+    // k-step assigned to the fragment's k slots the way four consecutive codes fall out of ldmatrix (slots 2qc, 2qc+1
+    // <- dimensions 4qc, 4qc+1; slots 2qc+8, 2qc+9 <- 4qc+2, 4qc+3); q_scale = softmax scale * 2^eq undoes the scaling
+    uint32_t qh[F8 ? C::KS : 1][2];
+    float q_scale = 0.f;
+    int ev_cur = 0;          // compressed V: exponent the O accumulators are currently expressed in
+    bool ev_set = false;
     float o[2 * C::KS][4];   // O accumulators: [8-column block of d][c0, c1 real row; c2, c3 padding rows]
     // running max (scaled, log2 units), this thread's share of the sum of the numerators (for the log-sum-exp)
     // and of the sum of their bf16 roundings (what the tensor core multiplies with V: O is normalised by it,
@@ -326,6 +354,26 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
             for (int ks = 0; ks < C::KS; ++ks) {
                 qa[ks][0] = real ? *(const uint32_t *)(qrow + ks * 16 + 2 * qc) : 0u;
                 qa[ks][1] = real ? *(const uint32_t *)(qrow + ks * 16 + 8 + 2 * qc) : 0u;
+            }
+            if constexpr (F8) {
+                uint2 raw[C::KS];
+                uint32_t amax = 0;   // largest |q| of the row, as bf16 bits (they order like the values)
+#pragma unroll
+                for (int ks = 0; ks < C::KS; ++ks) {
+                    raw[ks] = real ? *(const uint2 *)(qrow + ks * 16 + 4 * qc) : make_uint2(0u, 0u);
+                    amax = max(amax, max(max(raw[ks].x & 0x7fffu, (raw[ks].x >> 16) & 0x7fffu), max(raw[ks].y & 0x7fffu, (raw[ks].y >> 16) & 0x7fffu)));
+                }
+                amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+                amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+                const int eq = amax >= 0x80u ? min((int)(amax >> 7) - 127, 126) : -126;  // |q| * 2^-eq < 2 (< 4 for the largest binade)
+                const float down = __uint_as_float((uint32_t)(127 - eq) << 23);        // 2^-eq (eq in [-126, 127])
+                q_scale = p.scale_log2 * __uint_as_float((uint32_t)(127 + max(eq, -126)) << 23);
+#pragma unroll
+                for (int ks = 0; ks < C::KS; ++ks) {
+                    qh[ks][0] = pack_f16(bf_lo(raw[ks].x) * down, bf_hi(raw[ks].x) * down);
+                    qh[ks][1] = pack_f16(bf_lo(raw[ks].y) * down, bf_hi(raw[ks].y) * down);
+                }
+                ev_set = false;
             }
 #pragma unroll
             for (int nb = 0; nb < 2 * C::KS; ++nb) o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f;
@@ -359,20 +407,49 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
             if (rows > 0) {
                 // ---------- S = Q K^T for 16 tokens (two 8-token blocks) ----------
                 float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+                const bool is_f8 = F8 && (tag & kTagF8) != 0;
+                // token of the piece behind each of this thread's four score columns (s0[0], s0[1], s1[0], s1[1])
+                int c0 = 2 * qc, c1 = 2 * qc + 1, c2 = 8 + 2 * qc, c3 = 9 + 2 * qc;
+                float xs = p.scale_log2;
+                if (is_f8) {
+                    if constexpr (F8) {
+                        // A K row is 128 codes: one 16-byte chunk per k-step.  The two 8-token MMA blocks take tokens
+                        // {0,1,4,5,8,9,12,13} and {2,3,6,7,10,11,14,15} of the piece, so that a thread's score columns are
+                        // tokens 4qc .. 4qc+3: the four consecutive codes it later gets from a row of transposed V.
+                        const int set = mi >> 1, tr = r0 + (ri >> 1) * 4 + (ri & 1) + 2 * set;
 #pragma unroll
-                for (int ks = 0; ks < C::KS; ++ks) {
-                    // matrices: (tokens 0-7, d-chunk 2ks), (tokens 0-7, 2ks+1), (tokens 8-15, 2ks), (tokens 8-15, 2ks+1)
-                    const int c = (ks * 2 + (mi & 1)) & 7;
-                    uint32_t kb[4];
-                    ldsm_x4(stage_u32 + (ks / 4) * C::BOX_BYTES + swz(r0 + (mi >> 1) * 8 + ri, c), kb);
-                    mma_bf16(s0, qa[ks][0], 0u, qa[ks][1], 0u, kb[0], kb[1]);
-                    mma_bf16(s1, qa[ks][0], 0u, qa[ks][1], 0u, kb[2], kb[3]);
+                        for (int kp = 0; kp < C::KS / 2; ++kp) {
+                            uint32_t kb[4], b0, b1;
+                            ldsm_x4(stage_u32 + tr * 128 + (((2 * kp + (mi & 1)) ^ (tr & 7)) << 4), kb);
+                            cvt_e4m3x4_f16(kb[0], b0, b1);
+                            mma_f16(s0, qh[2 * kp][0], 0u, qh[2 * kp][1], 0u, b0, b1);
+                            cvt_e4m3x4_f16(kb[1], b0, b1);
+                            mma_f16(s0, qh[2 * kp + 1][0], 0u, qh[2 * kp + 1][1], 0u, b0, b1);
+                            cvt_e4m3x4_f16(kb[2], b0, b1);
+                            mma_f16(s1, qh[2 * kp][0], 0u, qh[2 * kp][1], 0u, b0, b1);
+                            cvt_e4m3x4_f16(kb[3], b0, b1);
+                            mma_f16(s1, qh[2 * kp + 1][0], 0u, qh[2 * kp + 1][1], 0u, b0, b1);
+                        }
+                        c0 = 4 * qc; c1 = 4 * qc + 1; c2 = 4 * qc + 2; c3 = 4 * qc + 3;
+                        const int ek = (int)*(const signed char *)(ring + stage * C::STAGE_BYTES + 2 * kTile * D);
+                        xs = q_scale * __uint_as_float((uint32_t)(127 + max(ek, -126)) << 23);
+                    }
+                } else {
+#pragma unroll
+                    for (int ks = 0; ks < C::KS; ++ks) {
+                        // matrices: (tokens 0-7, d-chunk 2ks), (tokens 0-7, 2ks+1), (tokens 8-15, 2ks), (tokens 8-15, 2ks+1)
+                        const int c = (ks * 2 + (mi & 1)) & 7;
+                        uint32_t kb[4];
+                        ldsm_x4(stage_u32 + (ks / 4) * C::BOX_BYTES + swz(r0 + (mi >> 1) * 8 + ri, c), kb);
+                        mma_bf16(s0, qa[ks][0], 0u, qa[ks][1], 0u, kb[0], kb[1]);
+                        mma_bf16(s1, qa[ks][0], 0u, qa[ks][1], 0u, kb[2], kb[3]);
+                    }
                 }
                 // ---------- online softmax (this thread: row qr, tokens 2qc, 2qc+1, 8+2qc, 9+2qc) ----------
-                const float x0 = 2 * qc < vis ? s0[0] * p.scale_log2 : -CUDART_INF_F;
-                const float x1 = 2 * qc + 1 < vis ? s0[1] * p.scale_log2 : -CUDART_INF_F;
-                const float x2 = 8 + 2 * qc < vis ? s1[0] * p.scale_log2 : -CUDART_INF_F;
-                const float x3 = 9 + 2 * qc < vis ? s1[1] * p.scale_log2 : -CUDART_INF_F;
+                const float x0 = c0 < vis ? s0[0] * xs : -CUDART_INF_F;
+                const float x1 = c1 < vis ? s0[1] * xs : -CUDART_INF_F;
+                const float x2 = c2 < vis ? s1[0] * xs : -CUDART_INF_F;
+                const float x3 = c3 < vis ? s1[1] * xs : -CUDART_INF_F;
                 float tmax = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
                 tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
                 tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
@@ -382,9 +459,11 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                 const float alpha = m_new == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);
                 const float p0 = fast_exp2(x0 - m_use), p1 = fast_exp2(x1 - m_use);
                 const float p2 = fast_exp2(x2 - m_use), p3 = fast_exp2(x3 - m_use);
-                const uint32_t pa0 = pack_bf16(p0, p1), pa2 = pack_bf16(p2, p3);
+                // P as the second MMA's operand: bf16, or fp16 against a tile of codes
+                const uint32_t pa0 = is_f8 ? pack_f16(p0, p1) : pack_bf16(p0, p1), pa2 = is_f8 ? pack_f16(p2, p3) : pack_bf16(p2, p3);
                 l_run = l_run * alpha + ((p0 + p1) + (p2 + p3));
-                l_rnd = l_rnd * alpha + ((bf_lo(pa0) + bf_hi(pa0)) + (bf_lo(pa2) + bf_hi(pa2)));
+                l_rnd = l_rnd * alpha + (is_f8 ? ((f16_lo(pa0) + f16_hi(pa0)) + (f16_lo(pa2) + f16_hi(pa2)))
+                                               : ((bf_lo(pa0) + bf_hi(pa0)) + (bf_lo(pa2) + bf_hi(pa2))));
                 m_run = m_new;
                 if (__any_sync(0xffffffffu, alpha != 1.0f)) {
 #pragma unroll
@@ -394,6 +473,40 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                     }
                 }
                 // ---------- O += P V ----------
+                if constexpr (F8) {
+                    // the accumulators are kept in units of 2^ev of the V block last seen (0 for bf16 tiles); a change of
+                    // exponent rescales them (a power of two: exact), like a change of the running maximum does
+                    const int ev = is_f8 ? (int)*(const signed char *)(ring + stage * C::STAGE_BYTES + 2 * kTile * D + 1) : 0;
+                    if (!ev_set) {
+                        ev_cur = ev;
+                        ev_set = true;
+                    } else if (ev != ev_cur) {
+                        const float f = exp2f((float)max(-126, min(126, ev_cur - ev)));
+#pragma unroll
+                        for (int nb = 0; nb < 2 * C::KS; ++nb) {
+                            o[nb][0] *= f;
+                            o[nb][1] *= f;
+                        }
+                        ev_cur = ev;
+                    }
+                }
+                if (is_f8) {
+                    if constexpr (F8) {
+                        // V codes of the block, transposed: row d holds its 64 tokens; this piece is 16-byte chunk r0 / 16 of it
+                        const uint32_t v8 = stage_u32 + kTile * D;
+#pragma unroll
+                        for (int q4 = 0; q4 < D / 32; ++q4) {
+                            const int d = 32 * q4 + 8 * mi + ri;
+                            uint32_t vb[4], b0, b1;
+                            ldsm_x4(v8 + d * 64 + (((r0 >> 4) ^ ((d >> 1) & 3)) << 4), vb);
+#pragma unroll
+                            for (int m2 = 0; m2 < 4; ++m2) {
+                                cvt_e4m3x4_f16(vb[m2], b0, b1);
+                                mma_f16(o[4 * q4 + m2], pa0, 0u, pa2, 0u, b0, b1);
+                            }
+                        }
+                    }
+                } else {
                 const uint32_t v_u32 = stage_u32 + C::NBOX * C::BOX_BYTES;
 #pragma unroll
                 for (int dp = 0; dp < C::KS; ++dp) {
@@ -403,6 +516,7 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                     ldsm_x4_trans(v_u32 + (dp / 4) * C::BOX_BYTES + swz(r0 + (mi & 1) * 8 + ri, c), vb);
                     mma_bf16(o[2 * dp], pa0, 0u, pa2, 0u, vb[0], vb[1]);
                     mma_bf16(o[2 * dp + 1], pa0, 0u, pa2, 0u, vb[2], vb[3]);
+                }
                 }
                 // ---------- the unit's own new tokens go to the tail for later calls ----------
                 if (is_new) {
@@ -432,9 +546,11 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
             l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
             r_tot += __shfl_xor_sync(0xffffffffu, r_tot, 1);
             r_tot += __shfl_xor_sync(0xffffffffu, r_tot, 2);
+            float ev_f = 1.f;
+            if constexpr (F8) ev_f = ev_set ? exp2f((float)max(-126, min(126, ev_cur))) : 1.f;   // back to plain units
 #pragma unroll
             for (int nb = 0; nb < 2 * C::KS; ++nb)
-                *(float2 *)(merge_o + (warp * kUnitRows + qr) * D + nb * 8 + 2 * qc) = make_float2(o[nb][0], o[nb][1]);
+                *(float2 *)(merge_o + (warp * kUnitRows + qr) * D + nb * 8 + 2 * qc) = make_float2(o[nb][0] * ev_f, o[nb][1] * ev_f);
             if (qc == 0) {
                 merge_m[warp * kUnitRows + qr] = m_run;
                 merge_l[warp * kUnitRows + qr] = l_tot;
@@ -505,15 +621,15 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
 }
 
 // ---- launchers --------------------------------------------------------------------------------------
-template <int D, int G>
+template <int D, int G, bool F8 = false>
 static int launch_stream_t(const StreamParams &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
-    using C = StreamCfg<D, G>;
+    using C = StreamCfg<D, G, F8>;
     static bool configured = false;
     if (!configured) {
-        MATKV_CUDA(cudaFuncSetAttribute(k_attend_stream<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        MATKV_CUDA(cudaFuncSetAttribute(k_attend_stream<D, G, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
         configured = true;
     }
-    k_attend_stream<D, G><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
+    k_attend_stream<D, G, F8><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());
     return MATKV_OK;
 }
@@ -527,6 +643,7 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     StreamParams p;
     p.reqs = t->d_reqs;
     p.tmaps = t->d_tmaps;
+    p.tmaps8 = t->d_tmaps8;
     p.segs = t->d_segs;
     p.n_seg_total = t->n_seg_total;
     p.tail_len = t->d_tail_len;
@@ -566,6 +683,13 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     // bound by HBM with ~130 CTAs already; a copy CTA sharing an SM with a decode CTA makes that SM the straggler)
     int64_t grid = ctx->opt_decode_ctas > 0 ? ctx->opt_decode_ctas : std::max<int64_t>(ctx->n_sm - ctx->opt_stage_ctas, ctx->n_sm / 2);
     grid = std::max<int64_t>(1, std::min<int64_t>(grid, W));
+    if (t->has_fp8) {   // tables with compressed-resident chunks: the variant that also reads tiles of codes
+#define MATKV_CASE8(GG) \
+        if (c.head_dim == 128 && G == GG) return launch_stream_t<128, GG, true>(p, kn_map, vn_map, (int)grid, stream);
+        MATKV_CASE8(1) MATKV_CASE8(2) MATKV_CASE8(4) MATKV_CASE8(8)
+#undef MATKV_CASE8
+        return fail(MATKV_E_INVALID_ARG, "compressed-resident chunks: unsupported head_dim %d / group %d", c.head_dim, G);
+    }
 #define MATKV_CASE(DD, GG) \
     if (c.head_dim == DD && G == GG) return launch_stream_t<DD, GG>(p, kn_map, vn_map, (int)grid, stream);
     MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)
@@ -604,6 +728,7 @@ extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_
     if (((uintptr_t)q | (uintptr_t)k_new | (uintptr_t)v_new | (uintptr_t)out) % 16)
         return fail(MATKV_E_ALIGNMENT, "matkv_attend_decode_static: q, k_new, v_new and out must be 16-byte aligned");
     if (c.rope_theta != 0.f) return fail(MATKV_E_INVALID_ARG, "matkv_attend_decode_static: rotary mode is not available");
+    if (t->has_fp8) return fail(MATKV_E_INVALID_ARG, "matkv_attend_decode_static: the table holds compressed-resident chunks");
     if (t->tail_len_host + 1 > c.max_tail_tokens)
         return fail(MATKV_E_CAPACITY, "matkv_attend_decode_static: tail holds %d tokens, one more exceeds max_tail_tokens %d",
                     t->tail_len_host, c.max_tail_tokens);
@@ -639,6 +764,7 @@ extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_
         StreamParams p;
         p.reqs = t->d_reqs;
         p.tmaps = t->d_tmaps;
+        p.tmaps8 = nullptr;
         p.segs = t->d_segs;
         p.n_seg_total = t->n_seg_total;
         p.tail_len = t->d_tail_len;

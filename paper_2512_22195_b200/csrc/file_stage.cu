@@ -145,7 +145,7 @@ int io_engine_errors(matkv_ctx *ctx, const char **msg) {
 }
 
 // Enqueues: read (worker threads) -> [copy stream] wait for the read, copy slab -> dst, release the slab.
-int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream, int32_t fp8_tokens) {
+int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream, int32_t fp8_tokens, bool fp8_resident) {
     IoEngine *e = ctx->io;
     if (!e) return fail(MATKV_E_INVALID_ARG, "file-backed chunk: no bounce buffer set (matkv_set_bounce_buffer)");
     if (bytes > e->slab_bytes)
@@ -164,8 +164,9 @@ int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void 
     e->cv.notify_all();
     MATKV_CUDA(cudaLaunchHostFunc(copy_stream, cb_wait_read, new IoCallback{e, job.slab, job.use}));
     if (fp8_tokens > 0) {  // compressed chunk: the expanding copy reads the slab over the link (it must be device-accessible pinned memory)
-        int rc = launch_stage_expand_fp8(ctx, e->base + (size_t)job.slab * e->slab_bytes, dst, fp8_tokens,
-                                         ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, copy_stream);
+        int rc = fp8_resident ? launch_stage_relayout_fp8(ctx, e->base + (size_t)job.slab * e->slab_bytes, dst, fp8_tokens, copy_stream)
+                              : launch_stage_expand_fp8(ctx, e->base + (size_t)job.slab * e->slab_bytes, dst, fp8_tokens,
+                                                        ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, copy_stream);
         if (rc) return rc;
     } else {
         MATKV_CUDA(cudaMemcpyAsync(dst, e->base + (size_t)job.slab * e->slab_bytes, bytes, cudaMemcpyHostToDevice, copy_stream));

@@ -112,6 +112,74 @@ __global__ void __launch_bounds__(128) k_stage_expand_fp8(const uint4 *__restric
     }
 }
 
+
+// ---- the HBM-resident compressed form (read by the streaming attention kernel without expansion) -----------
+// nb = ceil(n_tokens / 64) blocks per (layer, KV head); three regions, each starting at a multiple of 256 bytes:
+//   K codes   [L][Hkv][nb * 64][D]      token rows of D bytes (rows past n_tokens are zero)
+//   V codes   [L][Hkv][nb][D][64]       per block transposed: row d holds the block's 64 tokens (the P V product wants
+//                                       consecutive tokens of one dimension side by side)
+//   exponents [L][Hkv][nb] x 16 bytes   byte 0 = K block exponent, byte 1 = V block exponent (a 16-byte record so that
+//                                       one bulk copy brings it in beside the tile)
+size_t fp8_resident_bytes(const matkv_config &c, int32_t n_tokens) {
+    const size_t nb = (size_t)(n_tokens + 63) / 64, slabs = (size_t)c.n_layers * c.n_kv_heads;
+    return 2 * up256(slabs * nb * 64 * c.head_dim) + up256(slabs * nb * 16);
+}
+
+// one CTA per (layer, KV head, block): store form -> resident form
+__global__ void __launch_bounds__(256) k_relayout_fp8(const uint8_t *__restrict__ codes, const int8_t *__restrict__ exps,
+                                                      uint8_t *__restrict__ k_out, uint8_t *__restrict__ v_out, uint8_t *__restrict__ e_out,
+                                                      int32_t n_tokens, int32_t D, int32_t Hkv, int32_t nb) {
+    __shared__ __align__(16) uint8_t tile[64 * 129];   // V block, rows padded to 129 bytes for the transposed read
+    const int b = blockIdx.x, lh = blockIdx.y;          // block, layer * Hkv + head
+    const int l = lh / Hkv, h = lh % Hkv;
+    const int t0 = b * 64, nt = min(64, n_tokens - t0);
+    const int64_t k_slab = ((int64_t)(l * 2) * Hkv + h), v_slab = ((int64_t)(l * 2 + 1) * Hkv + h);
+    // K rows: straight copy, 16 bytes at a time (D is a multiple of 16), zero rows past the end
+    const uint4 *ksrc = (const uint4 *)(codes + (k_slab * n_tokens + t0) * D);
+    uint4 *kdst = (uint4 *)(k_out + (((int64_t)lh * nb + b) * 64) * D);
+    const int vec_row = D / 16;
+    for (int i = threadIdx.x; i < 64 * vec_row; i += blockDim.x)
+        kdst[i] = i / vec_row < nt ? __ldcs(ksrc + i) : make_uint4(0u, 0u, 0u, 0u);
+    // V block through shared memory, transposed on the way out
+    const uint4 *vsrc = (const uint4 *)(codes + (v_slab * n_tokens + t0) * D);
+    for (int i = threadIdx.x; i < 64 * vec_row; i += blockDim.x) {
+        const int t = i / vec_row, c = i % vec_row;
+        const uint4 v = t < nt ? __ldcs(vsrc + i) : make_uint4(0u, 0u, 0u, 0u);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 16; ++j) tile[t * 129 + c * 16 + j] = (uint8_t)(w[j >> 2] >> (8 * (j & 3)));
+    }
+    __syncthreads();
+    uint8_t *vdst = v_out + (((int64_t)lh * nb + b) * D) * 64;
+    for (int i = threadIdx.x; i < D * 16; i += blockDim.x) {   // 4 tokens (one 32-bit word) of one dimension per step
+        const int d = i / 16, tq = (i % 16) * 4;
+        const uint32_t w = (uint32_t)tile[tq * 129 + d] | ((uint32_t)tile[(tq + 1) * 129 + d] << 8) |
+                           ((uint32_t)tile[(tq + 2) * 129 + d] << 16) | ((uint32_t)tile[(tq + 3) * 129 + d] << 24);
+        *(uint32_t *)(vdst + d * 64 + tq) = w;
+    }
+    if (threadIdx.x < 4) {
+        uint32_t w = 0;
+        if (threadIdx.x == 0)
+            w = (uint32_t)(uint8_t)exps[k_slab * nb + b] | ((uint32_t)(uint8_t)exps[v_slab * nb + b] << 8);
+        ((uint32_t *)(e_out + ((int64_t)lh * nb + b) * 16))[threadIdx.x] = w;
+    }
+}
+
+int launch_stage_relayout_fp8(matkv_ctx *ctx, const void *src_fp8, void *dev_dst, int32_t n_tokens, cudaStream_t stream) {
+    const matkv_config &c = ctx->cfg;
+    if (c.head_dim != 128) return fail(MATKV_E_INVALID_ARG, "compressed-resident chunks need head_dim 128");
+    const int nb = (n_tokens + 63) / 64;
+    const int64_t lh = (int64_t)c.n_layers * c.n_kv_heads;
+    if (lh > 65535) return fail(MATKV_E_CAPACITY, "too many (layer, head) slabs for one re-layout launch");
+    const uint8_t *codes = (const uint8_t *)src_fp8;
+    const int8_t *exps = (const int8_t *)(codes + up256(fp8_codes_bytes(c, n_tokens)));
+    const size_t region = up256((size_t)lh * nb * 64 * c.head_dim);
+    uint8_t *k_out = (uint8_t *)dev_dst, *v_out = k_out + region, *e_out = v_out + region;
+    k_relayout_fp8<<<dim3(nb, (unsigned)lh), 256, 0, stream>>>(codes, exps, k_out, v_out, e_out, n_tokens, c.head_dim, c.n_kv_heads, nb);
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
+}
+
 int launch_quantize_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_fp8, cudaStream_t stream) {
     const matkv_config &c = ctx->cfg;
     const int nb = (n_tokens + 63) / 64;

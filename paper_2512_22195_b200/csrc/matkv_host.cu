@@ -66,6 +66,35 @@ int encode_rows_map(CUtensorMap *out, const void *base, int D, uint64_t rows) {
     return MATKV_OK;
 }
 
+// Tensor maps of a compressed-resident chunk (head_dim 128): [0] K codes as rows of 128 bytes, box 64 rows, 128-byte
+// swizzle; [1] V codes, per block transposed, as rows of 64 bytes (one dimension's 64 tokens), box 128 rows, 64-byte swizzle.
+int encode_fp8_maps(CUtensorMap *out2, const void *dev_resident, const matkv_config &c, int32_t n_tokens) {
+    EncodeFn fn = tensor_map_encoder();
+    if (!fn) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    const uint64_t nb = (uint64_t)(n_tokens + 63) / 64, lh = (uint64_t)c.n_layers * c.n_kv_heads;
+    const size_t region = align_up((size_t)(lh * nb * 64 * c.head_dim), 256);
+    const cuuint32_t estride[2] = {1, 1};
+    {
+        const cuuint64_t gdim[2] = {(cuuint64_t)c.head_dim, (cuuint64_t)(lh * nb * 64)};
+        const cuuint64_t gstride[1] = {(cuuint64_t)c.head_dim};
+        const cuuint32_t box[2] = {128, 64};
+        CUresult r = fn(&out2[0], CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(dev_resident), gdim, gstride, box, estride,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled (K codes) failed with %d", (int)r);
+    }
+    {
+        const cuuint64_t gdim[2] = {64, (cuuint64_t)(lh * nb * c.head_dim)};
+        const cuuint64_t gstride[1] = {64};
+        const cuuint32_t box[2] = {64, 128};
+        CUresult r = fn(&out2[1], CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (char *)const_cast<void *>(dev_resident) + region, gdim, gstride, box,
+                        estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled (V codes) failed with %d", (int)r);
+    }
+    return MATKV_OK;
+}
+
 int encode_new_rows_map(CUtensorMap *out, const void *base, int D, int Hkv, uint64_t n_tok) {
     EncodeFn fn = tensor_map_encoder();
     if (!fn) return fail(MATKV_E_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
@@ -264,6 +293,10 @@ int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
             if (value < 0 || value > 2) return fail(MATKV_E_INVALID_ARG, "decode impl must be 0..2");
             ctx->opt_decode_impl = value;
             return MATKV_OK;
+        case MATKV_OPT_FP8_RESIDENT:
+            if (value < 0 || value > 1) return fail(MATKV_E_INVALID_ARG, "fp8-resident must be 0 or 1");
+            ctx->opt_fp8_resident = value;
+            return MATKV_OK;
         case MATKV_OPT_SHARE_TILES:
             if (value < 1 || value > 1024) return fail(MATKV_E_INVALID_ARG, "tiles per chunk-major item must be 1..1024");
             ctx->opt_share_tiles = value;
@@ -456,9 +489,13 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
             return fail(ctx->io ? MATKV_E_CAPACITY : MATKV_E_INVALID_ARG,
                         "chunk %llu lives in a file: set a bounce buffer with slabs of at least %zu bytes first",
                         (unsigned long long)ids[i], stored);
-        if (blob_bytes(ctx->cfg, c.n_tokens) > slot_bytes)
+        const bool keep8 = c.fp8 && ctx->opt_fp8_resident;   // stays compressed in HBM
+        if (keep8 && ctx->cfg.head_dim != 128)
+            return fail(MATKV_E_INVALID_ARG, "compressed-resident chunks need head_dim 128");
+        const size_t in_slot = keep8 ? fp8_resident_bytes(ctx->cfg, c.n_tokens) : blob_bytes(ctx->cfg, c.n_tokens);
+        if (in_slot > slot_bytes)
             return fail(MATKV_E_CAPACITY, "chunk %llu (%zu bytes) does not fit a slot of %zu bytes",
-                        (unsigned long long)ids[i], blob_bytes(ctx->cfg, c.n_tokens), slot_bytes);
+                        (unsigned long long)ids[i], in_slot, slot_bytes);
         if (std::find(want.begin(), want.end(), ids[i]) == want.end()) want.push_back(ids[i]);
     }
     if ((int64_t)want.size() > n_slots)
@@ -516,10 +553,12 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
         }
         if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;  // moves from another region
         void *dst = (char *)dev_slots + (size_t)next_free * slot_bytes;
+        const bool keep8 = c.fp8 && ctx->opt_fp8_resident;
         if (c.host_blob && c.fp8) {
-            // compressed chunk: expanded to bf16 on its way in (always by the SM copy kernel; the host blob must be
-            // device-accessible pinned memory)
-            int rc = launch_stage_expand_fp8(ctx, c.host_blob, dst, c.n_tokens, ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, cs);
+            // compressed chunk: expanded to bf16 on its way in, or re-laid out into the resident compressed form (always
+            // by an SM kernel that reads the host blob over the link: it must be device-accessible pinned memory)
+            int rc = keep8 ? launch_stage_relayout_fp8(ctx, c.host_blob, dst, c.n_tokens, cs)
+                           : launch_stage_expand_fp8(ctx, c.host_blob, dst, c.n_tokens, ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, cs);
             if (rc) {
                 cudaEventDestroy(tk.done);
                 return rc;
@@ -539,18 +578,20 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
             }
         } else {  // storage tier: read into the bounce ring, then copy, all in the copy stream's order
             int rc = io_engine_stage(ctx, c.file_fd, c.file_offset, c.fp8 ? fp8_blob_bytes(ctx->cfg, c.n_tokens) : blob_bytes(ctx->cfg, c.n_tokens),
-                                     dst, cs, c.fp8 ? c.n_tokens : 0);
+                                     dst, cs, c.fp8 ? c.n_tokens : 0, keep8);
             if (rc) {
                 cudaEventDestroy(tk.done);
                 return rc;
             }
         }
         {
-            int rc = encode_rows_map(&c.tmap, dst, ctx->cfg.head_dim, (uint64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * c.n_tokens);
+            int rc = keep8 ? encode_fp8_maps(c.tmap8, dst, ctx->cfg, c.n_tokens)
+                           : encode_rows_map(&c.tmap, dst, ctx->cfg.head_dim, (uint64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * c.n_tokens);
             if (rc) {
                 cudaEventDestroy(tk.done);
                 return rc;
             }
+            c.resident_fp8 = keep8;
         }
         r->used[next_free] = 1;
         r->occupant[next_free] = id;
@@ -613,7 +654,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     t->tail_k = (__nv_bfloat16 *)tail_k;
     t->tail_v = (__nv_bfloat16 *)tail_v;
     std::vector<cudaEvent_t> waits;
-    std::vector<const CUtensorMap *> seg_maps;
+    std::vector<const CUtensorMap *> seg_maps, seg_maps8;
     int64_t k = 0;
     for (int32_t r = 0; r < batch; ++r) {
         DevReq rq;
@@ -643,8 +684,12 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
             sg.base = (const __nv_bfloat16 *)dev;
             sg.len = c.n_tokens;
             sg.start = rq.n_chunk_tokens;
+            sg.fmt = (!c.dev_blob && c.resident_fp8) ? 1 : 0;
+            sg.pad = 0;
+            if (sg.fmt) t->has_fp8 = true;
             t->h_segs.push_back(sg);
             seg_maps.push_back(&c.tmap);
+            seg_maps8.push_back(c.tmap8);
             rq.n_chunk_tokens += c.n_tokens;
             rq.chunk_tiles += (c.n_tokens + kTile - 1) / kTile;
             longest = std::max(longest, c.n_tokens);
@@ -685,7 +730,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
         for (auto &kv : members) t->distinct_chunk_tiles += (kv.first.second + kTile - 1) / kTile;
         bool fits = true;  // the kernel's item queue keeps request indices and part counts in 16 bits
         for (int32_t r = 0; r < batch; ++r) fits = fits && t->h_reqs[r].n_parts <= 32767;
-        if (R > 0 && fits) {
+        if (R > 0 && fits && !t->has_fp8) {   // the chunk-major kernel reads bf16 chunks only
             for (auto &kv : members) {
                 const int32_t len = kv.first.second, tiles = (len + kTile - 1) / kTile;
                 const auto &m = kv.second;
@@ -718,8 +763,9 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     const size_t reqs_bytes = align_up(sizeof(DevReq) * (size_t)batch, 256);
     const size_t tl_bytes = align_up(sizeof(int32_t) * (size_t)batch, 256);
     const size_t maps_bytes = align_up(sizeof(CUtensorMap) * (seg_maps.size() + 2), 256);
-    const size_t items_bytes = sizeof(DevItem) * std::max<size_t>(items.size(), 1);
-    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes + maps_bytes + items_bytes;
+    const size_t items_bytes = align_up(sizeof(DevItem) * std::max<size_t>(items.size(), 1), 256);
+    const size_t maps8_bytes = t->has_fp8 ? sizeof(CUtensorMap) * 2 * seg_maps8.size() : 0;
+    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes + maps_bytes + items_bytes + maps8_bytes;
     CUtensorMap tail_maps[2];
     {
         const uint64_t tail_rows = (uint64_t)batch * ctx->cfg.n_layers * ctx->cfg.n_kv_heads * ctx->cfg.max_tail_tokens;
@@ -763,6 +809,12 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     t->d_items = (DevItem *)((char *)t->d_image + segs_bytes + reqs_bytes + tl_bytes + maps_bytes);
     if (!items.empty())
         memcpy((char *)t->h_pinned + segs_bytes + reqs_bytes + tl_bytes + maps_bytes, items.data(), sizeof(DevItem) * items.size());
+    if (t->has_fp8) {
+        const size_t off8 = segs_bytes + reqs_bytes + tl_bytes + maps_bytes + items_bytes;
+        t->d_tmaps8 = (CUtensorMap *)((char *)t->d_image + off8);
+        CUtensorMap *h8 = (CUtensorMap *)((char *)t->h_pinned + off8);
+        for (size_t i = 0; i < seg_maps8.size(); ++i) memcpy(h8 + 2 * i, seg_maps8[i], 2 * sizeof(CUtensorMap));
+    }
     {
         CUtensorMap *hm = (CUtensorMap *)((char *)t->h_pinned + segs_bytes + reqs_bytes + tl_bytes);
         for (size_t i = 0; i < seg_maps.size(); ++i) memcpy(hm + i, seg_maps[i], sizeof(CUtensorMap));
@@ -870,7 +922,8 @@ static bool shared_region(matkv_ctx *ctx, const matkv_table *t, int n_layers_lau
 static int launch_decode(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream) {
     const int64_t impl = ctx->opt_decode_impl;
     // automatic choice: chunk-major when stacking saves at least a fifth of the chunk reads
-    bool shared = impl == 2 || (impl == 0 && t->share_ok && t->n_items > 0 && t->total_chunk_tiles * 4 >= t->item_tiles * 5);
+    if (t->has_fp8 && impl == 2) return fail(MATKV_E_INVALID_ARG, "the chunk-major decode does not read compressed-resident chunks");
+    bool shared = !t->has_fp8 && (impl == 2 || (impl == 0 && t->share_ok && t->n_items > 0 && t->total_chunk_tiles * 4 >= t->item_tiles * 5));
     void *region = nullptr;
     size_t region_bytes = 0;
     if (shared) {
@@ -984,7 +1037,8 @@ int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t 
     }
     // long suffixes go to the tcgen05 tile kernel, short ones stay on the streaming kernel
     const int G = c.n_q_heads / c.n_kv_heads;
-    const bool tensor_core = ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
+    // (compressed-resident chunks are read by the streaming kernel only)
+    const bool tensor_core = !t->has_fp8 && (ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64));
     if (tensor_core) return launch_prefill_tc(ctx, t, a, (cudaStream_t)stream);
     return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
 }
@@ -1013,7 +1067,8 @@ int matkv_attend_prefill_all_layers(matkv_ctx *ctx, matkv_table *t, int32_t S, c
         if (rc) return rc;
     }
     const int G = c.n_q_heads / c.n_kv_heads;
-    const bool tensor_core = ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
+    // (compressed-resident chunks are read by the streaming kernel only)
+    const bool tensor_core = !t->has_fp8 && (ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64));
     if (tensor_core) return launch_prefill_tc(ctx, t, a, (cudaStream_t)stream);
     // short suffixes run on the streaming kernel; when its units do not fit the workspace's counters in one
     // launch, the layers are launched one by one (same result)
@@ -1087,6 +1142,7 @@ int matkv_gather_debug(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t re
                                           (long long)capacity_rows);
     if (((uintptr_t)k_out | (uintptr_t)v_out) % 16) return fail(MATKV_E_ALIGNMENT, "gather outputs must be 16-byte aligned");
     if (rows == 0) return MATKV_OK;
+    if (t && t->has_fp8) return fail(MATKV_E_INVALID_ARG, "matkv_gather_debug: the table holds compressed-resident chunks");
     DeviceGuard guard(ctx->device);
     return launch_gather(ctx, t, layer, req, k_out, v_out, rows, (cudaStream_t)stream);
 }

@@ -23,6 +23,8 @@ struct DevSeg {
     const __nv_bfloat16 *base;  // blob [L][2][Hkv][len][D]
     int32_t len;                // tokens
     int32_t start;              // tokens before this segment in the request's logical order
+    int32_t fmt;                // 0: bf16 blob; 1: compressed, HBM-resident form (see fp8_store.cu)
+    int32_t pad;
 };
 struct DevReq {
     int32_t seg_begin;       // index of the request's first segment in the segment array
@@ -61,6 +63,8 @@ struct Chunk {
     uint64_t file_offset = 0;
     void *dev_blob = nullptr;      // caller-resident device copy
     bool fp8 = false;              // host_blob / the file holds the compressed form (e4m3 codes + block exponents)
+    bool resident_fp8 = false;     // the staged device copy is the compressed, HBM-resident form
+    alignas(64) CUtensorMap tmap8[2];  // resident form: K codes [rows][D] (128-byte swizzle), V codes transposed per block [rows][64] (64-byte swizzle)
     void *staged = nullptr;        // device copy inside a slot region (or nullptr)
     Region *region = nullptr;
     int32_t slot = -1;
@@ -94,7 +98,7 @@ struct matkv_ctx {
     void *workspace = nullptr;
     size_t workspace_bytes = 0;
     int64_t opt_decode_ctas = 0, opt_prefill_impl = 0, opt_prefill_ctas = 0, opt_stage_ctas = 0, opt_fused_advance = 0;
-    int64_t opt_decode_impl = 0, opt_share_tiles = 16;
+    int64_t opt_decode_impl = 0, opt_share_tiles = 16, opt_fp8_resident = 0;
     std::unordered_map<uint64_t, matkv::Chunk> chunks;
     std::map<void *, matkv::Region *> regions;
     std::unordered_map<uint64_t, matkv::Ticket> tickets;
@@ -120,6 +124,8 @@ struct matkv_table {
     matkv::DevReq *d_reqs = nullptr;
     int32_t *d_tail_len = nullptr;
     CUtensorMap *d_tmaps = nullptr;  // one per segment, then the K tail and the V tail
+    CUtensorMap *d_tmaps8 = nullptr; // two per segment (K codes, transposed V codes) when the table has compressed-resident chunks
+    bool has_fp8 = false;            // some segment is compressed-resident: only the streaming kernel reads those
     matkv::DevItem *d_items = nullptr;  // chunk-major decode: the chunk items of one (layer, KV head)
     bool share_ok = false;              // the head grouping fits the chunk-major kernel
     int32_t n_items = 0;                // chunk items (the requests' tail items follow implicitly)
@@ -183,11 +189,16 @@ int io_engine_create(matkv_ctx *ctx, void *pinned, size_t bytes, size_t slab_byt
 void io_engine_destroy(matkv_ctx *ctx);
 size_t io_engine_slab_bytes(const matkv_ctx *ctx);
 int io_engine_errors(matkv_ctx *ctx, const char **msg);
-// fp8_tokens > 0: the file holds a compressed chunk of that many tokens, expanded on its way from the slab to dst
-int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream, int32_t fp8_tokens = 0);
+// fp8_tokens > 0: the file holds a compressed chunk of that many tokens; on its way from the slab to dst it is expanded to
+// bf16 (fp8_resident false) or re-laid out into the HBM-resident compressed form (true)
+int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream, int32_t fp8_tokens = 0,
+                    bool fp8_resident = false);
 size_t fp8_codes_bytes(const matkv_config &c, int32_t n_tokens);
 size_t fp8_blob_bytes(const matkv_config &c, int32_t n_tokens);
 int launch_quantize_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_fp8, cudaStream_t stream);
+size_t fp8_resident_bytes(const matkv_config &c, int32_t n_tokens);
+int launch_stage_relayout_fp8(matkv_ctx *ctx, const void *src_fp8, void *dev_dst, int32_t n_tokens, cudaStream_t stream);
+int encode_fp8_maps(CUtensorMap *out2, const void *dev_resident, const matkv_config &c, int32_t n_tokens);
 int launch_stage_expand_fp8(matkv_ctx *ctx, const void *src_fp8, void *dev_dst, int32_t n_tokens, int n_ctas, cudaStream_t stream);
 int open_chunk_file(const char *path, uint64_t offset, size_t bytes, int *fd_out);
 void close_chunk_file(int fd);

@@ -17,6 +17,7 @@ constexpr int kMaxDynSmem = 232448;             // 227 KB opt-in limit per CTA o
 constexpr long long kWaitCycles = 2000000000LL; // bounded waits give up after about a second
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr uint32_t kTagF8 = 0x0080u;            // tile tag: a tile of e4m3 codes (compressed-resident chunk)
 constexpr uint32_t kTagNew = 0x8000u;           // tile tag: a tile of the call's new tokens (bits 8..14: its index)
 
 // ---- PTX helpers ---------------------------------------------------------------------------------
@@ -127,6 +128,38 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// the same with fp16 operands (the compressed-chunk path: e4m3 codes convert to fp16 with one instruction per pair)
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// four e4m3 codes (one 32-bit word) -> two fp16 pairs: codes 0,1 and codes 2,3 (exact)
+__device__ __forceinline__ void cvt_e4m3x4_f16(uint32_t w, uint32_t &lo, uint32_t &hi) {
+    asm("{\n .reg .b16 a, b;\n mov.b32 {a, b}, %2;\n cvt.rn.f16x2.e4m3x2 %0, a;\n cvt.rn.f16x2.e4m3x2 %1, b;\n}" : "=r"(lo), "=r"(hi) : "r"(w));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %2, %1;" : "=r"(r) : "f"(lo), "f"(hi));   // the first source lands in the upper half
+    return r;
+}
+__device__ __forceinline__ float f16_lo(uint32_t w) {
+    float f;
+    asm("{\n .reg .b16 a, b;\n mov.b32 {a, b}, %1;\n cvt.f32.f16 %0, a;\n}" : "=f"(f) : "r"(w));
+    return f;
+}
+__device__ __forceinline__ float f16_hi(uint32_t w) {
+    float f;
+    asm("{\n .reg .b16 a, b;\n mov.b32 {a, b}, %1;\n cvt.f32.f16 %0, b;\n}" : "=f"(f) : "r"(w));
+    return f;
+}
+// untiled bulk copy global -> shared with mbarrier completion (both addresses 16-byte aligned, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src), "r"(bytes),
+                 "r"(bar)
+                 : "memory");
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);

@@ -131,3 +131,73 @@ def test_compressed_chunk_files_through_the_bounce_ring(tmp_path):
     assert np.array_equal(dev_to_bits(v), np.concatenate([deq[1][0, 1], deq[0][0, 1]], axis=1))
     sess.close()
     del ring
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (32, 8), (16, 2), (4, 4), (4, 2)])
+def test_compressed_resident_chunks_attend_like_the_oracle(Hq, Hkv):
+    """Compressed chunks kept compressed in HBM (MATKV_OPT_FP8_RESIDENT): the streaming kernel reads the codes and
+    converts in registers.  Ragged lengths, different block exponents, one ordinary bf16 chunk in the same table,
+    sub-prefill (several token blocks) and decode with a tail that crosses a tile; against the oracle on the values
+    the codes stand for."""
+    import paper_2512_22195_b200 as mk
+    from paper_2512_22195_b200.harness import Session, bits_to_dev, dev_to_bits
+    L, D = 2, 128
+    lens = [200, 64, 33, 1, 130]
+    S, T = 5, 4
+    sess = Session(L, Hq, Hkv, D, 3, 4, 70 + S + T)
+    mk.matkv_set_option(sess.ctx, mk.OPT_FP8_RESIDENT, 1)
+    sh = oracle.Shape(L, Hq, Hkv, D)
+    vals, keep = {}, []
+    for cid, n in enumerate(lens[:4]):
+        blob = rand_bits(74, cid, (L, 2, Hkv, n, D), cid - 3)       # scales 1/8 .. 1: different block exponents
+        codes, exps = oracle.fp8_quantize_blob(sh, blob)
+        vals[cid] = oracle.fp8_dequantize_blob(sh, codes, exps)
+        host = torch.from_numpy(_fp8_blob_np(sess, mk, codes, exps)).pin_memory()
+        keep.append(host)
+        mk.matkv_register_chunk_fp8(sess.ctx, cid, n, host.data_ptr())
+    vals[4] = rand_bits(74, 4, (L, 2, Hkv, lens[4], D))               # a plain bf16 chunk, device-resident
+    sess.register_device_chunk(4, vals[4])
+    slot_bytes = (L * 2 * Hkv * max(lens) * D * 2 + 255) // 256 * 256
+    slots = torch.zeros(4 * slot_bytes, dtype=torch.uint8, device="cuda")
+    sess.stage([0, 1, 2, 3], slots, slot_bytes, torch.cuda.Stream())
+    ids = [[0, 4, 2], [3, 1, 0, 2], [4]]
+    sess.build_table(ids)
+    B = len(ids)
+    reqs = [oracle.Request(sh, [vals[c] for c in row], 70 + S + T) for row in ids]
+    # a tail of 62 tokens first (plain appends), so that the decode steps cross the 64-token tile boundary
+    pre = 62
+    for layer in range(L):
+        q, k, v = (rand_bits(74, 50 + 3 * layer + i, (B, pre, Hq if i == 0 else Hkv, D)) for i in range(3))
+        sess.prefill(layer, bits_to_dev(q), bits_to_dev(k), bits_to_dev(v))
+        for r in range(B):
+            reqs[r].append_only(layer, k[r], v[r])
+    sess.advance(pre)
+    for rq in reqs:
+        rq.advance(pre)
+    for layer in range(L):
+        q, k, v = (rand_bits(74, 100 + 3 * layer + i, (B, S, Hq if i == 0 else Hkv, D)) for i in range(3))
+        out, lse = sess.prefill(layer, bits_to_dev(q), bits_to_dev(k), bits_to_dev(v))
+        for r in range(B):
+            o_ref, l_ref = reqs[r].attend_new(layer, q[r], k[r], v[r])
+            check(dev_to_bits(out)[r], o_ref, lse.cpu().numpy()[r], l_ref, f"prefill over resident codes, layer {layer} request {r}")
+    sess.advance(S)
+    for rq in reqs:
+        rq.advance(S)
+    for t in range(T):
+        q, k, v = (rand_bits(74, 200 + 3 * t + i, (L, B, Hq if i == 0 else Hkv, D)) for i in range(3))
+        if t % 2:
+            out, lse = sess.decode_all_layers(bits_to_dev(q), bits_to_dev(k), bits_to_dev(v))
+            ob, lb = dev_to_bits(out), lse.cpu().numpy()
+        else:
+            outs = [sess.decode(layer, bits_to_dev(q[layer]), bits_to_dev(k[layer]), bits_to_dev(v[layer])) for layer in range(L)]
+            ob = np.stack([dev_to_bits(o) for o, _ in outs])
+            lb = np.stack([l.cpu().numpy() for _, l in outs])
+        for layer in range(L):
+            for r in range(B):
+                o_ref, l_ref = reqs[r].attend_new(layer, q[layer, r][None], k[layer, r][None], v[layer, r][None])
+                check(ob[layer, r], o_ref[0], lb[layer, r], l_ref[0], f"decode over resident codes, step {t} layer {layer} request {r}")
+        sess.advance(1)
+        for rq in reqs:
+            rq.advance(1)
+    assert sess.status() == 0
+    sess.close()
