@@ -394,6 +394,9 @@ def main():
     ap.add_argument("--kv-store", default="bf16", choices=["bf16", "fp8"],
                     help="pipelined serving: keep the host / file chunk pool as plain bf16 blobs or compressed (e4m3 codes with a "
                     "power-of-two scale per 64-token block, expanded to bf16 while staged; a lossy store, so a separate workload)")
+    ap.add_argument("--kv-hbm", default="bf16", choices=["bf16", "fp8"],
+                    help="fp8: the chunks sit in HBM as e4m3 codes (MATKV_OPT_FP8_RESIDENT) and the streaming kernel converts them "
+                    "in registers; a lossy KV format, so a workload of its own (forces --no-e2e)")
     ap.add_argument("--decode-impl", type=int, default=0, choices=[0, 1, 2],
                     help="decode kernel: 0 auto (chunk-major when the batch's requests share chunks), 1 request-major, 2 chunk-major")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
@@ -445,10 +448,31 @@ def main():
     # every rank works on its own replica of the batch (independent requests: no data-path collective)
     chunks = {}
     pool = torch.empty((len(needed), L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device=dev)
-    for i, c in enumerate(needed):
-        gen.fill_bf16(pool[i], w.seed, mi.STREAM_CHUNK + c)
-        chunks[c] = pool[i]
-        sess.register_device_chunk(c, pool[i])
+    fp8_hbm = args.kv_hbm == "fp8"
+    if fp8_hbm:
+        # compress every chunk (device quantiser), park the codes in pinned host memory, stage them ONCE into device slots
+        # in the compressed-resident form; the timed steps then only build tables over the staged chunks
+        args.no_e2e = True
+        w.name += "-fp8hbm"
+        mk.matkv_set_option(sess.ctx, mk.OPT_FP8_RESIDENT, 1)
+        stored = mk.matkv_fp8_blob_bytes(sess.ctx, w.chunk_tokens)
+        host8 = torch.empty((len(needed), stored), dtype=torch.uint8, pin_memory=True)
+        tmp8 = torch.empty(stored, dtype=torch.uint8, device=dev)
+        for i, c in enumerate(needed):
+            gen.fill_bf16(pool[i], w.seed, mi.STREAM_CHUNK + c)
+            chunks[c] = pool[i]
+            mk.matkv_quantize_chunk_fp8(sess.ctx, pool[i].data_ptr(), w.chunk_tokens, tmp8.data_ptr())
+            host8[i].copy_(tmp8)
+            mk.matkv_register_chunk_fp8(sess.ctx, c, w.chunk_tokens, host8[i].data_ptr())
+        slot8 = mk.matkv_fp8_resident_bytes(sess.ctx, w.chunk_tokens)   # the resident form: codes plus 16-byte exponent records
+        slots8 = torch.empty(len(needed) * slot8, dtype=torch.uint8, device=dev)
+        cs8 = torch.cuda.Stream(device=dev)
+        mk.matkv_stage_wait(sess.ctx, sess.stage(needed, slots8, slot8, cs8))
+    else:
+        for i, c in enumerate(needed):
+            gen.fill_bf16(pool[i], w.seed, mi.STREAM_CHUNK + c)
+            chunks[c] = pool[i]
+            sess.register_device_chunk(c, pool[i])
     q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device=dev)
     k_pf = torch.empty((L, B, S, Hkv, D), dtype=torch.bfloat16, device=dev)
     v_pf = torch.empty_like(k_pf)
@@ -589,6 +613,10 @@ def main():
     n_req = [sum(chunks[c].shape[3] for c in row) for row in ids]
     kv_bytes_decode = sum((n + S + t + 1) * w.beta for n in n_req for t in range(T)) * L
     kv_bytes_prefill = sum((n + S) * w.beta for n in n_req) * L
+    if fp8_hbm:   # chunk tokens cost half the bytes plus a 16-byte exponent record per 64-token block and KV head; the tail stays bf16
+        beta8 = w.beta // 2 + Hkv * 16 / 64.0
+        kv_bytes_decode = sum(n * beta8 + (S + t + 1) * w.beta for n in n_req for t in range(T)) * L
+        kv_bytes_prefill = sum(n * beta8 + S * w.beta for n in n_req) * L
     tokens = B * T * world
     value = tokens * args.steps / (ms * 1e-3)
     decode_launches = T * (1 if args.decode_launch == "all_layers" else L)
@@ -609,7 +637,7 @@ def main():
     result = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16 in, fp32 softmax/accumulate", "data": "synthetic",
+        "vs_baseline": None, "dtype": "bf16 in, fp32 softmax/accumulate" + (", chunk KV as e4m3 codes in HBM (fp16 MMAs)" if fp8_hbm else ""), "data": "synthetic",
         "config": {"workload": w.name, "layers": L, "q_heads": Hq, "kv_heads": Hkv, "head_dim": D, "batch": B,
                    "chunks_per_request": w.chunks_per_req, "chunk_tokens": w.chunk_tokens, "suffix": S, "decode_steps": T,
                    "decode_launch": args.decode_launch, "prefill_launch": "all_layers" if args.decode_launch == "all_layers" else "per_layer", "l2": "inputs larger than L2 (KV per decode step = "

@@ -155,6 +155,8 @@ int matkv_set_bounce_buffer(matkv_ctx *ctx, void *pinned_host, size_t bytes, siz
  *   matkv_register_chunk_file_fp8  the same for a compressed blob stored in a file (see
  *                            matkv_register_chunk_file); it passes through the pinned bounce ring.             */
 size_t matkv_fp8_blob_bytes(const matkv_ctx *ctx, int32_t n_tokens);
+/* device slot bytes a compressed chunk needs when it stays compressed in HBM (MATKV_OPT_FP8_RESIDENT = 1) */
+size_t matkv_fp8_resident_bytes(const matkv_ctx *ctx, int32_t n_tokens);
 int matkv_quantize_chunk_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_blob_fp8, void *stream);
 int matkv_register_chunk_fp8(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const void *host_blob_fp8);
 int matkv_register_chunk_file_fp8(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const char *path, uint64_t file_offset);

@@ -28,7 +28,7 @@ EXPORTS = [
     "matkv_probe_read", "matkv_attend_decode_static", "matkv_selftest_wait_timeout",
     "matkv_register_chunk_file", "matkv_set_bounce_buffer", "matkv_export_tail_as_chunk",
     "matkv_attend_prefill_all_layers", "matkv_table_sharing", "matkv_table_workspace_bytes",
-    "matkv_fp8_blob_bytes", "matkv_quantize_chunk_fp8", "matkv_register_chunk_fp8", "matkv_register_chunk_file_fp8",
+    "matkv_fp8_blob_bytes", "matkv_fp8_resident_bytes", "matkv_quantize_chunk_fp8", "matkv_register_chunk_fp8", "matkv_register_chunk_file_fp8",
 ]
 
 
@@ -89,6 +89,7 @@ def lib() -> C.CDLL:
             "matkv_table_sharing": (C.c_int, [vp, C.POINTER(i64), C.POINTER(i64)]),
             "matkv_table_workspace_bytes": (C.c_size_t, [vp, i32]),
             "matkv_fp8_blob_bytes": (C.c_size_t, [vp, i32]),
+            "matkv_fp8_resident_bytes": (C.c_size_t, [vp, i32]),
             "matkv_quantize_chunk_fp8": (C.c_int, [vp, vp, i32, vp, vp]),
             "matkv_register_chunk_fp8": (C.c_int, [vp, u64, i32, vp]),
             "matkv_register_chunk_file_fp8": (C.c_int, [vp, u64, i32, C.c_char_p, u64]),
@@ -268,6 +269,10 @@ def matkv_table_workspace_bytes(table: int, n_layers_launch: int) -> int:
 
 def matkv_fp8_blob_bytes(ctx: int, n_tokens: int) -> int:
     return int(lib().matkv_fp8_blob_bytes(ctx, n_tokens))
+
+
+def matkv_fp8_resident_bytes(ctx: int, n_tokens: int) -> int:
+    return int(lib().matkv_fp8_resident_bytes(ctx, n_tokens))
 
 
 def matkv_quantize_chunk_fp8(ctx: int, dev_blob: int, n_tokens: int, dev_blob_fp8: int, stream: int = 0) -> None:

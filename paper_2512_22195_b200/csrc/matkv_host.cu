@@ -384,6 +384,11 @@ size_t matkv_fp8_blob_bytes(const matkv_ctx *ctx, int32_t n_tokens) {
     return fp8_blob_bytes(ctx->cfg, n_tokens);
 }
 
+size_t matkv_fp8_resident_bytes(const matkv_ctx *ctx, int32_t n_tokens) {
+    if (!ctx || n_tokens < 1) return 0;
+    return fp8_resident_bytes(ctx->cfg, n_tokens);
+}
+
 int matkv_quantize_chunk_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_blob_fp8, void *stream) {
     if (!ctx || !dev_blob || !dev_blob_fp8) return fail(MATKV_E_INVALID_ARG, "matkv_quantize_chunk_fp8: null argument");
     if (n_tokens < 1) return fail(MATKV_E_INVALID_ARG, "matkv_quantize_chunk_fp8: n_tokens must be >= 1");
