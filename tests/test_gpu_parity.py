@@ -417,3 +417,12 @@ def test_auto_choice_matches_sharing():
     assert mk.matkv_table_sharing(t) == (5, 5)
     assert mk.matkv_table_workspace_bytes(t, 1) >= mk.matkv_workspace_bytes(sess.ctx)
     sess.close()
+
+
+def test_chunk_major_decode_many_parts_and_rotary_mode():
+    """More than 32 partials per request (one-tile items of a 2,200-token chunk: the general merge path), and the
+    chunk-major kernel behind the rotary pre-rotation (q and k_new rotated at each request's own position)."""
+    pool = [2200, 130]
+    run_requests(1, 8, 2, 128, [[0, 1], [0], [1, 0]], 2, 2, seed=64, pool=pool, decode_impl=2, share_tiles=1)
+    run_requests(2, 8, 2, 64, [[0, 1], [1], [1, 0]], 3, 3, seed=65, pool=[70, 33], decode_impl=2, rope_theta=10000.0)
+    run_requests(2, 8, 2, 64, [[0, 1], [1], [1, 0]], 3, 3, seed=66, pool=[70, 33], decode_impl=2, rope_theta=500000.0, pos_mode=1)
