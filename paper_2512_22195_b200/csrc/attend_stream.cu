@@ -192,8 +192,10 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
         flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        locate_range(p, *range, n_blk);
     }
+    // short launches are chains of latencies: the range lookup (dependent loads of the table) runs in another warp beside
+    // the barrier set-up
+    if (tid == 32) locate_range(p, *range, n_blk);
     __syncthreads();
     const int64_t f_begin = range->begin, f_end = range->end, W = range->W;
     // the fused tail advance: the last CTA of the launch to get here moves every request's tail length

@@ -177,8 +177,12 @@ static __device__ void combine_warp(const float *o_parts, int64_t o_stride, cons
     const int lane = threadIdx.x & 31;
     const int dpl = D >> 5;  // every lane owns D/32 consecutive dims
     if (P <= 32 && dpl == 4) {
-        // common case (at most 32 parts, D = 128): one part's lse per lane, a single round trip for them,
-        // then the parts' rows 16 loads at a time; weights travel by shuffle
+        // common case (at most 32 parts, D = 128): the first 16 parts' rows and one part's lse per lane are requested
+        // together (one round trip to L2 for up to 16 parts, two beyond); the weights travel by shuffle
+        float4 v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            v[i] = i < P ? __ldcg((const float4 *)(o_parts + i * o_stride + lane * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
         const float lse_l = lane < P ? __ldcg(lse_parts + lane * lse_stride) : -CUDART_INF_F;
         float m = lse_l;
 #pragma unroll
@@ -195,10 +199,11 @@ static __device__ void combine_warp(const float *o_parts, int64_t o_stride, cons
         w_l /= z;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int p0 = 0; p0 < P; p0 += 16) {
-            float4 v[16];
+            if (p0) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i)
-                v[i] = p0 + i < P ? __ldcg((const float4 *)(o_parts + (p0 + i) * o_stride + lane * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int i = 0; i < 16; ++i)
+                    v[i] = p0 + i < P ? __ldcg((const float4 *)(o_parts + (p0 + i) * o_stride + lane * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const float w = __shfl_sync(0xffffffffu, w_l, (p0 + i) & 31);
