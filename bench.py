@@ -500,11 +500,14 @@ def main():
     ev_d0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ev_d1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     ev_p0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    table_us = []   # host time of matkv_build_chunk_table per timed step
 
     def one_step(q_pf_p, k_pf_p, v_pf_p, q_dc_p, k_dc_p, v_dc_p, timed_index=None, mode=args.decode_launch):
         """All pointers are device addresses; nothing here but C-ABI calls."""
+        t_h = time.perf_counter()
         table = sess.build_table(ids, sp)
         if timed_index is not None:
+            table_us.append((time.perf_counter() - t_h) * 1e6)
             ev_p0[timed_index].record(stream)
         if mode == "all_layers":
             mk.matkv_attend_prefill_all_layers(ctx, table, S, q_pf_p, k_pf_p, v_pf_p, o_pf.data_ptr(), None, sp)
@@ -587,6 +590,9 @@ def main():
             raise RuntimeError(f"device status {st} after the timed region")
         dec_ms = sum(a.elapsed_time(b) for a, b in zip(ev_d0, ev_d1))
         pre_ms = sum(a.elapsed_time(b) for a, b in zip(ev_p0, ev_d0))
+        step_ms = sorted(a.elapsed_time(b) for a, b in zip(ev_p0, ev_d1))      # every timed step on its own (table upload excluded)
+        dec_step_ms = sorted(a.elapsed_time(b) for a, b in zip(ev_d0, ev_d1))
+        table_us_main = sorted(table_us)
         # the other launch mode, for the record (same work, different launch granularity)
         other = "per_layer_graph" if args.decode_launch == "all_layers" else "all_layers"
         dec_ms_o = None
@@ -617,6 +623,8 @@ def main():
         beta8 = w.beta // 2 + Hkv * 16 / 64.0
         kv_bytes_decode = sum(n * beta8 + (S + t + 1) * w.beta for n in n_req for t in range(T)) * L
         kv_bytes_prefill = sum(n * beta8 + S * w.beta for n in n_req) * L
+    # algorithmic flops of the sub-prefill: 4 * Hq * D per (query token, visible key), the causal part of the suffix block once
+    prefill_flops = 4.0 * Hq * D * L * sum(S * n + S * (S + 1) / 2 for n in n_req)
     tokens = B * T * world
     value = tokens * args.steps / (ms * 1e-3)
     decode_launches = T * (1 if args.decode_launch == "all_layers" else L)
@@ -654,7 +662,12 @@ def main():
                      "algorithmic_bytes_per_launch": (read_bytes_decode if chunk_major else kv_bytes_decode) / decode_launches,
                      "logical_kv_gbs": logical_gbs,
                      "avg_launch_us": avg_launch_ms * 1e3},
+        "repeats": {"steps": args.steps, "step_ms_min": step_ms[0], "step_ms_median": step_ms[len(step_ms) // 2],
+                    "decode_ms_min": dec_step_ms[0], "decode_ms_median": dec_step_ms[len(dec_step_ms) // 2],
+                    "tokens_per_s_best_step": B * T * world / (step_ms[0] * 1e-3),
+                    "table_build_host_us_median": table_us_main[len(table_us_main) // 2]},
         "phases": {"prefill_ms_per_step": pre_ms / args.steps, "decode_ms_per_step": dec_ms / args.steps,
+                   "prefill_tflops": prefill_flops * args.steps / (pre_ms * 1e-3) / 1e12,
                    "decode_only_tokens_per_s": B * T * args.steps / (dec_ms * 1e-3),
                    "decode_kv_gbs": kv_bytes_decode * args.steps / (dec_ms * 1e-3) / 1e9,
                    "prefill_kv_gbs": kv_bytes_prefill * args.steps / (pre_ms * 1e-3) / 1e9,
