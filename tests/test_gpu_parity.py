@@ -426,3 +426,32 @@ def test_chunk_major_decode_many_parts_and_rotary_mode():
     run_requests(1, 8, 2, 128, [[0, 1], [0], [1, 0]], 2, 2, seed=64, pool=pool, decode_impl=2, share_tiles=1)
     run_requests(2, 8, 2, 64, [[0, 1], [1], [1, 0]], 3, 3, seed=65, pool=[70, 33], decode_impl=2, rope_theta=10000.0)
     run_requests(2, 8, 2, 64, [[0, 1], [1], [1, 0]], 3, 3, seed=66, pool=[70, 33], decode_impl=2, rope_theta=500000.0, pos_mode=1)
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_tables_against_the_oracle(case):
+    """Seeded random workloads: head shapes, ragged chunk lengths, shared and repeated chunks, empty lists, suffix
+    and decode lengths, launch granularity, grid size and kernel choice are all drawn; every output is compared."""
+    rng = np.random.default_rng(1000 + case)
+    Hkv = int(rng.choice([1, 2, 4, 8]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    D = int(rng.choice([64, 128]))
+    L = int(rng.integers(1, 4))
+    n_pool = int(rng.integers(1, 6))
+    pool = [int(rng.choice([1, 7, 33, 64, 65, 127, 128, 200, 300, 513])) for _ in range(n_pool)]
+    B = int(rng.integers(1, 6))
+    ids = []
+    for _ in range(B):
+        k = int(rng.integers(0, 4))
+        ids.append([int(rng.integers(0, n_pool)) for _ in range(k)])       # repeats inside a request are allowed
+    S = int(rng.choice([1, 3, 9, 17, 40]))
+    T = int(rng.integers(1, 5))
+    kw = dict(
+        ctas=int(rng.choice([0, 0, 1, 5, 37])),
+        all_layers=bool(rng.integers(0, 2)),
+        decode_impl=int(rng.choice([0, 1, 2])),
+        share_tiles=int(rng.choice([0, 1, 3])),
+        prefill_impl=int(rng.choice([0, 1, 2, 3])),
+    )
+    kw["fused_advance"] = kw["all_layers"] and bool(rng.integers(0, 2))
+    run_requests(L, Hkv * G, Hkv, D, ids, S, T, seed=500 + case, pool=pool, **kw)
