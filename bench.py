@@ -394,6 +394,7 @@ def main():
     ap.add_argument("--kv-store", default="bf16", choices=["bf16", "fp8"],
                     help="pipelined serving: keep the host / file chunk pool as plain bf16 blobs or compressed (e4m3 codes with a "
                     "power-of-two scale per 64-token block, expanded to bf16 while staged; a lossy store, so a separate workload)")
+    ap.add_argument("--copy-streams", type=int, default=2, help="end-to-end leg: copy streams the chunk staging of a step is split over")
     ap.add_argument("--kv-hbm", default="bf16", choices=["bf16", "fp8"],
                     help="fp8: the chunks sit in HBM as e4m3 codes (MATKV_OPT_FP8_RESIDENT) and the streaming kernel converts them "
                     "in registers; a lossy KV format, so a workload of its own (forces --no-e2e)")
@@ -694,7 +695,12 @@ def main():
         for c in needed:
             mk.matkv_register_chunk(sess2.ctx, c, w.chunk_tokens, host[c].data_ptr(), None)
         slot_bytes = w.chunk_bytes
-        slots = [torch.empty(len(needed) * slot_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+        # the chunks of a step are split over N_COPY copy streams, each with slot regions of its own: several copies in
+        # flight keep the link busier while the decode saturates HBM
+        n_copy = max(1, min(args.copy_streams, len(needed)))
+        parts = [needed[k::n_copy] for k in range(n_copy)]
+        copies = [copy] + [torch.cuda.Stream(device=dev) for _ in range(n_copy - 1)]
+        slots = [[torch.empty(len(parts[k]) * slot_bytes, dtype=torch.uint8, device=dev) for k in range(n_copy)] for _ in range(2)]
         # query-side inputs and outputs are double-buffered on the device: step i+1's inputs arrive (copy stream)
         # and step i-1's outputs leave (output stream) while step i computes
         d_in = [tuple(torch.empty_like(x) for x in (q_pf, k_pf, v_pf, q_dc, k_dc, v_dc)) for _ in range(2)]
@@ -718,7 +724,8 @@ def main():
                 for dst, src in zip(d_in[i % 2], h_in):
                     dst.copy_(src, non_blocking=True)
                 in_ready[i % 2].record(copy)
-            sess2.stage(needed, slots[i % 2], slot_bytes, copy)
+            for k in range(n_copy):
+                sess2.stage(parts[k], slots[i % 2][k], slot_bytes, copies[k])
             state["loaded"] = i
 
         def e2e_step(i, last=False):
@@ -773,7 +780,7 @@ def main():
                          "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e,
                          "overlap": "next step's chunks and query-side inputs copied in, and the previous step's outputs copied out, "
                                     "on side streams under this step's prefill and decode",
-                         "staging": f"copy kernel, {args.stage_ctas} CTAs" if args.stage_ctas > 0 else "copy engine",
+                         "staging": (f"copy kernel, {args.stage_ctas} CTAs" if args.stage_ctas > 0 else "copy engine") + f", {n_copy} copy streams",
                          "h2d_gbs_if_copy_bound": h2d * k_e2e / (ms_e * 1e-3) / 1e9}
         sess2.close()
         del host, slots
