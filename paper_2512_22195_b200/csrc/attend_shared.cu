@@ -534,10 +534,9 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
 template <int D, int G>
 static int launch_shared_t(const SharedParams &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
     using C = SharedCfg<D, G>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (configured.need()) {
         MATKV_CUDA(cudaFuncSetAttribute(k_attend_shared<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-        configured = true;
     }
     k_attend_shared<D, G><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());

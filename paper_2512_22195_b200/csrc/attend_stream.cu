@@ -626,10 +626,9 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
 template <int D, int G, bool F8 = false>
 static int launch_stream_t(const StreamParams &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
     using C = StreamCfg<D, G, F8>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (configured.need()) {
         MATKV_CUDA(cudaFuncSetAttribute(k_attend_stream<D, G, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-        configured = true;
     }
     k_attend_stream<D, G, F8><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());

@@ -148,26 +148,10 @@ static void reap_graveyard(matkv_ctx *ctx, bool force);
 using namespace matkv;
 
 // table images (pinned upload buffer + device copy) are recycled: allocating them per batch costs
-// milliseconds (cudaMallocHost and cudaMalloc synchronise).  A freed table's image waits in the
-// graveyard until the stream work that may still read it has finished, then moves to the pool.
-struct Grave {
-    cudaEvent_t ev;
-    void *h_pinned;
-    void *d_image;
-    size_t bytes;
-};
-struct PooledImage {
-    void *h_pinned;
-    void *d_image;
-    size_t bytes;
-};
-static std::map<matkv_ctx *, std::vector<PooledImage>> g_pool;
-static std::map<matkv_ctx *, std::vector<Grave>> g_graves;
-
+// milliseconds (cudaMallocHost and cudaMalloc synchronise).  A freed table's image waits in the context's
+// graveyard until the stream work that may still read it has finished, then moves to the context's pool.
 static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
-    auto it = g_graves.find(ctx);
-    if (it == g_graves.end()) return;
-    auto &v = it->second;
+    auto &v = ctx->image_graves;
     for (size_t i = 0; i < v.size();) {
         bool done = force;
         if (force) cudaEventSynchronize(v[i].ev);
@@ -177,7 +161,7 @@ static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
                 cudaFreeHost(v[i].h_pinned);
                 cudaFree(v[i].d_image);
             } else {
-                g_pool[ctx].push_back(PooledImage{v[i].h_pinned, v[i].d_image, v[i].bytes});
+                ctx->image_pool.push_back(PooledImage{v[i].h_pinned, v[i].d_image, v[i].bytes});
             }
             cudaEventDestroy(v[i].ev);
             v[i] = v.back();
@@ -187,15 +171,11 @@ static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
         }
     }
     if (force) {
-        g_graves.erase(it);
-        auto pit = g_pool.find(ctx);
-        if (pit != g_pool.end()) {
-            for (auto &im : pit->second) {
-                cudaFreeHost(im.h_pinned);
-                cudaFree(im.d_image);
-            }
-            g_pool.erase(pit);
+        for (auto &im : ctx->image_pool) {
+            cudaFreeHost(im.h_pinned);
+            cudaFree(im.d_image);
         }
+        ctx->image_pool.clear();
     }
 }
 
@@ -783,7 +763,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     }
     cudaError_t e = cudaSuccess;
     {
-        auto &pool = g_pool[ctx];
+        auto &pool = ctx->image_pool;
         for (size_t i = 0; i < pool.size(); ++i)
             if (pool[i].bytes >= t->image_bytes) {
                 t->h_pinned = pool[i].h_pinned;
@@ -857,7 +837,7 @@ int matkv_table_free(matkv_table *t, void *stream) {
     g.h_pinned = t->h_pinned;
     g.d_image = t->d_image;
     g.bytes = t->image_alloc;
-    g_graves[ctx].push_back(g);
+    ctx->image_graves.push_back(g);
     ctx->tables.erase(std::remove(ctx->tables.begin(), ctx->tables.end(), t), ctx->tables.end());
     delete t;
     reap_graveyard(ctx, false);

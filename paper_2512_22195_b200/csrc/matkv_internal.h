@@ -83,6 +83,18 @@ struct Region {
     bool has_last_use = false;
 };
 
+struct Grave {        // a freed table's image, until the stream work that may still read it is done
+    cudaEvent_t ev;
+    void *h_pinned;
+    void *d_image;
+    size_t bytes;
+};
+struct PooledImage {  // a table image (pinned upload buffer + device copy) ready for reuse
+    void *h_pinned;
+    void *d_image;
+    size_t bytes;
+};
+
 struct Ticket {
     cudaEvent_t done = nullptr;
 };
@@ -105,6 +117,8 @@ struct matkv_ctx {
     uint64_t next_ticket = 1;
     std::vector<matkv_table *> tables;
     matkv::IoEngine *io = nullptr;
+    std::vector<matkv::PooledImage> image_pool;
+    std::vector<matkv::Grave> image_graves;
 };
 
 struct matkv_table {
@@ -144,6 +158,18 @@ int cuda_fail(cudaError_t e, const char *what);
         cudaError_t e__ = (x);                                     \
         if (e__ != cudaSuccess) return ::matkv::cuda_fail(e__, #x); \
     } while (0)
+
+// The opt-in shared-memory size of a kernel is a per-device attribute: launchers keep one flag per device ordinal.
+struct PerDeviceOnce {
+    bool done[64] = {};
+    bool need() {   // true the first time on the current device
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+        if (done[dev]) return false;
+        done[dev] = true;
+        return true;
+    }
+};
 
 constexpr int kUnitRows = 8;  // query rows (suffix tokens x heads of one KV group) one streaming unit carries
 

@@ -555,10 +555,9 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
 template <int D, int G, int NBLK>
 static int launch_k3(const k3::Params &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
     using C = k3::Cfg<D, NBLK>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    if (configured.need()) {
         MATKV_CUDA(cudaFuncSetAttribute(k3::k_prefill_tc<D, G, NBLK>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-        configured = true;
     }
     k3::k_prefill_tc<D, G, NBLK><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());
