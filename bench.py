@@ -369,6 +369,85 @@ def run_pipeline(args):
     sess.close()
 
 
+# ---- materialisation side (store_KV): chunks prefilled alone and written out ----------------------------
+def run_materialise(args):
+    """The paper's store_KV on this path's terms: every chunk is attended alone, causally, from position 0 (synthetic
+    q/k/v stand in for the model's projections), its K,V are laid out as a chunk blob, optionally compressed, and copied
+    to pinned host memory on a side stream while the next chunk is computed."""
+    import torch
+    import paper_2512_22195_b200 as mk
+    import matkv_inputs.device as gen
+    from paper_2512_22195_b200.harness import Session
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    w = mi.workload("cfg2")
+    if args.layers:
+        w.n_layers = args.layers
+    L, Hq, Hkv, D, n = w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.chunk_tokens
+    n_chunks = args.batches or 16
+    fp8 = args.kv_store == "fp8"
+    sess = Session(L, Hq, Hkv, D, 1, 1, n, device=dev.index)
+    q = torch.empty((L, 1, n, Hq, D), dtype=torch.bfloat16, device=dev)
+    k = torch.empty((L, 1, n, Hkv, D), dtype=torch.bfloat16, device=dev)
+    v = torch.empty_like(k)
+    for t_, st in ((q, mi.STREAM_Q_PREFILL), (k, mi.STREAM_K_PREFILL), (v, mi.STREAM_V_PREFILL)):
+        gen.fill_bf16(t_, w.seed, st)
+    out = torch.empty_like(q)
+    stored = mk.matkv_fp8_blob_bytes(sess.ctx, n) if fp8 else w.chunk_bytes
+    blobs = [torch.empty(w.chunk_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+    blobs8 = [torch.empty(stored, dtype=torch.uint8, device=dev) for _ in range(2)] if fp8 else None
+    host = torch.empty((n_chunks, stored), dtype=torch.uint8, pin_memory=True)
+    stream, side = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    sp = stream.cuda_stream
+    done = [torch.cuda.Event() for _ in range(2)]
+    copied = [torch.cuda.Event() for _ in range(2)]
+
+    def one(c):
+        i = c % 2
+        table = sess.build_table([[]], sp)
+        mk.matkv_attend_prefill_all_layers(sess.ctx, table, n, q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), None, sp)
+        mk.matkv_table_advance(table, n, sp)
+        if c >= 2:
+            stream.wait_event(copied[i])                  # the blob buffer's previous contents have left
+        mk.matkv_export_tail_as_chunk(sess.ctx, table, 0, n, blobs[i].data_ptr(), None, sp)
+        src = blobs[i]
+        if fp8:
+            mk.matkv_quantize_chunk_fp8(sess.ctx, blobs[i].data_ptr(), n, blobs8[i].data_ptr(), sp)
+            src = blobs8[i]
+        done[i].record(stream)
+        side.wait_event(done[i])
+        with torch.cuda.stream(side):
+            host[c].copy_(src, non_blocking=True)
+            copied[i].record(side)
+
+    with torch.cuda.stream(stream):
+        for c in range(2):
+            one(c)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for c in range(n_chunks):
+            one(c)
+        stream.wait_stream(side)
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if sess.status() != 0:
+        raise RuntimeError("device status non-zero")
+    flops = 4.0 * Hq * D * L * (n * (n + 1) / 2) * n_chunks
+    print(json.dumps({
+        "metric": "materialised_tokens_per_s", "value": n_chunks * n / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1, "steps": n_chunks,
+        "warmup": 2, "ms_per_step": ms / n_chunks, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 in, fp32 softmax/accumulate", "data": "synthetic",
+        "config": {"workload": "materialise", "layers": L, "q_heads": Hq, "kv_heads": Hkv, "head_dim": D, "chunk_tokens": n,
+                   "chunks": n_chunks, "stored_as": "e4m3 codes + block exponents" if fp8 else "bf16 blob",
+                   "note": "attention and write-out only: the model's projections and MLPs are outside this path"},
+        "phases": {"causal_attention_tflops": flops / (ms * 1e-3) / 1e12, "bytes_to_host_per_chunk": stored,
+                   "d2h_gbs": stored * n_chunks / (ms * 1e-3) / 1e9, "chunks_per_s": n_chunks / (ms * 1e-3)},
+    }), flush=True)
+    sess.close()
+
+
 # ---- the CUDA arm ----------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -407,6 +486,8 @@ def main():
         return run_reference(args)
     import __graft_entry__ as ge
     ge.build()                      # no-op when the in-tree libraries are up to date
+    if args.workload == "materialise":
+        return run_materialise(args)
     if args.workload == "cfg5":
         return run_pipeline(args)
     args.warmup = max(args.warmup, 3)

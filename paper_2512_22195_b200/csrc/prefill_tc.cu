@@ -295,11 +295,13 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
 
     if (warp == 0) {
         // ===================== producer =====================
-        // appends this split's share of the new tokens to the tail for later calls (the splits of row group 0
-        // divide the S tokens among themselves)
+        // appends this CTA's share of the new tokens to the tail for later calls: the suffix tokens of its own query rows,
+        // divided among the KV splits (a long suffix copied by the CTAs of row group 0 alone kept their SMs for hundreds
+        // of microseconds)
         auto append_share = [&]() {
             constexpr int CPR = D / 8;
-            const int a0 = (int)((int64_t)sp * p.S / p.n_split), a1 = (int)((int64_t)(sp + 1) * p.S / p.n_split);
+            const int tok_a = row0 / G, tok_b = min(p.S, (row0 + NBLK * kRowsPerCta) / G), n_own = max(0, tok_b - tok_a);
+            const int a0 = tok_a + (int)((int64_t)sp * n_own / p.n_split), a1 = tok_a + (int)((int64_t)(sp + 1) * n_own / p.n_split);
 #pragma unroll 4
             for (int idx = a0 * CPR + lane; idx < a1 * CPR; idx += 32) {
                 const int tok = idx / CPR, ch = idx % CPR;
@@ -311,7 +313,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 }
             }
         };
-        if (rb == 0 && n_tiles == 0) append_share();  // a split without tiles of its own still owes its share
+        if (n_tiles == 0) append_share();  // a split without tiles of its own still owes its share
         int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
@@ -349,7 +351,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     }
                 }
             }
-            if (j == 0 && rb == 0) append_share();  // once the CTA's first loads are in flight
+            if (j == 0) append_share();  // once the CTA's first loads are in flight
         }
     } else if (warp == 1) {
         // ===================== MMA issuer (one thread) =====================
