@@ -302,7 +302,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             constexpr int CPR = D / 8;
             const int tok_a = row0 / G, tok_b = min(p.S, (row0 + NBLK * kRowsPerCta) / G), n_own = max(0, tok_b - tok_a);
             const int a0 = tok_a + (int)((int64_t)sp * n_own / p.n_split), a1 = tok_a + (int)((int64_t)(sp + 1) * n_own / p.n_split);
-#pragma unroll 4
+#pragma unroll 8
             for (int idx = a0 * CPR + lane; idx < a1 * CPR; idx += 32) {
                 const int tok = idx / CPR, ch = idx % CPR;
                 if (t0 + tok < p.max_tail) {
@@ -313,7 +313,6 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 }
             }
         };
-        if (n_tiles == 0) append_share();  // a split without tiles of its own still owes its share
         int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
@@ -351,8 +350,11 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     }
                 }
             }
-            if (j == 0) append_share();  // once the CTA's first loads are in flight
         }
+        // Only later calls read the tail (this one takes the new tokens from k_new / v_new): the copy waits until every
+        // tile load of the CTA has been issued.  Issued between two tile loads it held the second one back by its whole
+        // duration (measured: 30 us per CTA on a 1,024-token suffix).
+        append_share();
     } else if (warp == 1) {
         // ===================== MMA issuer (one thread) =====================
         if (lane == 0) {
