@@ -51,8 +51,8 @@ struct SharedCfg {
     static constexpr int BOX_BYTES = kTile * 128;
     static constexpr int STAGE_BYTES = 2 * NBOX * BOX_BYTES;
     static constexpr int KS = D / 16;
-    // merge area: one 64-column half of O per warp and row, then m, l, rounded l per warp and row
-    static constexpr int MERGE_BYTES = (kCW * kShareRows * (64 + 3) * 4 + 15) / 16 * 16;
+    // merge area: one 64-column half of O per warp and row, then m, l, rounded l per warp and row, the rows' maxima
+    static constexpr int MERGE_BYTES = ((kCW * kShareRows * (64 + 3) + kShareRows) * 4 + 15) / 16 * 16;
     static constexpr int MISC_BYTES = 3840;                // barriers, tags, flags, the item queue
     static constexpr int FIXED_BYTES = MERGE_BYTES + MISC_BYTES + 1024;  // + slack for the 1024-byte alignment of the ring
     static constexpr int NSTAGE_MAX = (kMaxDynSmem - FIXED_BYTES) / STAGE_BYTES;
@@ -146,6 +146,7 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
     float *merge_m = merge_o + kCW * kShareRows * 64;               // [warp][row]  (log2 units, scaled)
     float *merge_l = merge_m + kCW * kShareRows;
     float *merge_r = merge_l + kCW * kShareRows;
+    float *row_max = merge_r + kCW * kShareRows;                    // [row] overall running maximum of the item
     unsigned char *misc = smem + C::NSTAGE * C::STAGE_BYTES + C::MERGE_BYTES;
     uint64_t *bars = (uint64_t *)misc;                                   // full[NSTAGE], empty[NSTAGE]
     volatile uint32_t *tags = (volatile uint32_t *)(misc + 2 * 12 * 8);  // per stage: rows | kTagNew | fill << 16
@@ -442,15 +443,29 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
         // prepared by the producer, its query rows are fetched while this item's partials are being reduced, and
         // the arrival tickets wait for the next batched flush.
         if (tid == 0) await_entry(k + 1);
+        // The seven warps' states are merged through shared memory.  First the running maxima: once every thread
+        // knows its rows' overall maximum it scales its own accumulators while it writes them, so that the reduction
+        // itself is a plain sum (no exponentials, no per-warp weights).
+        if (qc == 0) {
+            merge_m[warp * kShareRows + qr] = m_run[0];
+            merge_m[warp * kShareRows + qr + 8] = m_run[1];
+        }
+        consumer_bar();
+        float sw[2];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
+            const int r = qr + 8 * hh;
+            float M = merge_m[r];
+#pragma unroll
+            for (int w = 1; w < kCW; ++w) M = fmaxf(M, merge_m[w * kShareRows + r]);
+            sw[hh] = m_run[hh] == -CUDART_INF_F ? 0.f : fast_exp2(m_run[hh] - M);   // a warp without pieces of this item: weight 0
             float l_tot = l_run[hh];
             l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
             l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
             if (qc == 0) {
-                merge_m[warp * kShareRows + qr + 8 * hh] = m_run[hh];
-                merge_l[warp * kShareRows + qr + 8 * hh] = l_tot;
-                merge_r[warp * kShareRows + qr + 8 * hh] = lr[2 * hh];
+                merge_l[warp * kShareRows + r] = l_tot * sw[hh];
+                merge_r[warp * kShareRows + r] = lr[2 * hh] * sw[hh];
+                if (warp == 0) row_max[r] = M;
             }
         }
         bool have_next = false;
@@ -459,8 +474,10 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
             if (half) consumer_bar();  // the previous half has been read
 #pragma unroll
             for (int nb = 0; nb < 8; ++nb) {
-                *(float2 *)(merge_o + (warp * kShareRows + qr) * 64 + nb * 8 + 2 * qc) = make_float2(o[half * 8 + nb][0], o[half * 8 + nb][1]);
-                *(float2 *)(merge_o + (warp * kShareRows + qr + 8) * 64 + nb * 8 + 2 * qc) = make_float2(o[half * 8 + nb][2], o[half * 8 + nb][3]);
+                *(float2 *)(merge_o + (warp * kShareRows + qr) * 64 + nb * 8 + 2 * qc) =
+                    make_float2(o[half * 8 + nb][0] * sw[0], o[half * 8 + nb][1] * sw[0]);
+                *(float2 *)(merge_o + (warp * kShareRows + qr + 8) * 64 + nb * 8 + 2 * qc) =
+                    make_float2(o[half * 8 + nb][2] * sw[1], o[half * 8 + nb][3] * sw[1]);
             }
             consumer_bar();
             if (half == 0) {
@@ -471,36 +488,36 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
                 have_next = flags[1] == 0;
                 if (have_next) load_q(item_q + (k + 1) % kItemQ);
             }
-            // one (row, four columns) unit per thread and pass
+            // one (row, four columns) unit per thread and pass: plain sums over the warps
             for (int idx = tid; idx < n_rows * 16; idx += kCW * 32) {
                 const int r = idx >> 4, c4 = idx & 15;
-                float M = -CUDART_INF_F;
+                float4 acc = *(const float4 *)(merge_o + r * 64 + 4 * c4);
+                float Lr = merge_r[r];
 #pragma unroll
-                for (int w = 0; w < kCW; ++w) M = fmaxf(M, merge_m[w * kShareRows + r]);
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                float L = 0.f, Lr = 0.f;
-#pragma unroll
-                for (int w = 0; w < kCW; ++w) {
-                    const float mw = merge_m[w * kShareRows + r];
-                    const float sw = mw == -CUDART_INF_F ? 0.f : fast_exp2(mw - M);
+                for (int w = 1; w < kCW; ++w) {
                     const float4 v = *(const float4 *)(merge_o + (w * kShareRows + r) * 64 + 4 * c4);
-                    acc.x = fmaf(sw, v.x, acc.x); acc.y = fmaf(sw, v.y, acc.y);
-                    acc.z = fmaf(sw, v.z, acc.z); acc.w = fmaf(sw, v.w, acc.w);
-                    L = fmaf(sw, merge_l[w * kShareRows + r], L);
-                    Lr = fmaf(sw, merge_r[w * kShareRows + r], Lr);
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                    Lr += merge_r[w * kShareRows + r];
                 }
                 const float inv = 1.f / Lr;
                 acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
                 const int j = r / G, h = r % G, d = half * 64 + 4 * c4;
                 const int b = e->req[j];
+                float lse = 0.f;
+                if (d == 0) {
+                    float L = merge_l[r];
+#pragma unroll
+                    for (int w = 1; w < kCW; ++w) L += merge_l[w * kShareRows + r];
+                    lse = (row_max[r] + log2f(L)) * kLn2;
+                }
                 if (e->np[j] == 1) {  // a request without chunks: its tail item is the whole answer
                     *(uint2 *)(p.out + (int64_t)l_rel * p.q_sl + (int64_t)b * p.q_sb + (int64_t)(g * G + h) * D + d) =
                         make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-                    if (p.lse_out && d == 0) p.lse_out[(int64_t)l_rel * p.lse_sl + (int64_t)b * p.lse_sb + g * G + h] = (M + log2f(L)) * kLn2;
+                    if (p.lse_out && d == 0) p.lse_out[(int64_t)l_rel * p.lse_sl + (int64_t)b * p.lse_sb + g * G + h] = lse;
                 } else {
                     const int64_t row = ((int64_t)lg * p.parts_total + e->part[j]) * G + h;
                     *(float4 *)(p.part_o + row * D + d) = acc;
-                    if (d == 0) p.part_lse[row] = (M + log2f(L)) * kLn2;
+                    if (d == 0) p.part_lse[row] = lse;
                 }
             }
         }
