@@ -127,6 +127,23 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t 
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same with the descriptors given as (low word, high word): the high word (SBO, version, swizzle) is a constant
+// of the operand kind and the low word (address and LBO) advances by a plain 32-bit add, so the single issuing
+// thread spends a handful of instructions per MMA instead of rebuilding two 64-bit descriptors.
+__device__ __forceinline__ void umma2(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t b_hi_sel, uint32_t idesc, uint32_t accumulate) {
+    // both operand kinds used here share the high word except for nothing: SBO 1024, version 1, 128-byte swizzle
+    (void)b_hi_sel;
+    constexpr uint32_t kHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // bits 32.. of the descriptor
+    asm volatile(
+        "{\n .reg .pred p;\n .reg .b64 da, db;\n setp.ne.b32 p, %4, 0;\n mov.b64 da, {%1, %5};\n mov.b64 db, {%2, %5};\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kHi)
+        : "memory");
+}
+// low word of a descriptor: address >> 4 in bits [0,14), LBO >> 4 in bits [16,30)
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+    return ((addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -369,10 +386,11 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 for (int blk = 0; blk < NBLK; ++blk) {
                     if (!mbar_wait(p_ready + (blk * 2 + bf) * 8, (t >> 1) & 1, abort_flag)) return false;
                     tc_fence_after();
+                    const uint32_t p_lo = desc_lo(p_u32 + (blk * 2 + bf) * C::P_BYTES, 0), v_lo = desc_lo(v_u32, C::BOX_BYTES);
 #pragma unroll
-                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA
-                        umma(tmem + blk * C::COL_BLK + C::COL_O, smem_desc(p_u32 + (blk * 2 + bf) * C::P_BYTES + ks * 32, 0, 1024),
-                             smem_desc(v_u32 + ks * 2048, C::BOX_BYTES, 1024), idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 32 bytes, V 16 rows of 128 bytes
+                        umma2(tmem + blk * C::COL_BLK + C::COL_O, p_lo + ks * (32 >> 4), v_lo + ks * (2048 >> 4), 0, idesc_pv,
+                              (t > 0 || ks > 0) ? 1u : 0u);
                     umma_commit(o_done + blk * 8);
                 }
                 umma_commit(empty_kv + st * 8);  // K and V of the tile are free once these MMAs have run
@@ -386,11 +404,11 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 const uint32_t k_u32 = kv_u32 + st * C::STAGE_BYTES;
 #pragma unroll
                 for (int blk = 0; blk < NBLK; ++blk) {
+                    const uint32_t q_lo = desc_lo(q_u32 + blk * C::QBLK_BYTES, 0), k_lo = desc_lo(k_u32, 0);
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
-                        umma(tmem + blk * C::COL_BLK + (j & 1) * kTile,
-                             smem_desc(q_u32 + blk * C::QBLK_BYTES + (ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32, 0, 1024),
-                             smem_desc(k_u32 + (ks / 4) * C::BOX_BYTES + (ks % 4) * 32, 0, 1024), idesc_qk, ks > 0);
+                        umma2(tmem + blk * C::COL_BLK + (j & 1) * kTile, q_lo + (((ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32) >> 4),
+                              k_lo + (((ks / 4) * C::BOX_BYTES + (ks % 4) * 32) >> 4), 0, idesc_qk, ks > 0);
                     umma_commit(s_full + (blk * 2 + (j & 1)) * 8);
                 }
                 if (j >= 1) ok = do_pv(j - 1);
