@@ -140,6 +140,29 @@ __device__ __forceinline__ void umma2(uint32_t d_tmem, uint32_t a_lo, uint32_t b
         "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kHi)
         : "memory");
 }
+// A operand taken from tensor memory (lane = row, 32-bit columns hold consecutive pairs of bf16 along K): the softmax
+// threads leave P where S was, so the second MMA reads only V from shared memory.  Shared-memory bandwidth is what
+// bounds this kernel: an M 128 x N 64 x K 16 MMA reads 6 KB of operands in the 32 cycles it computes.
+__device__ __forceinline__ void umma_ta(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+    constexpr uint32_t kHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    asm volatile(
+        "{\n .reg .pred p;\n .reg .b64 db;\n setp.ne.b32 p, %4, 0;\n mov.b64 db, {%2, %5};\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n}" ::"r"(d_tmem),
+        "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kHi)
+        : "memory");
+}
+// 32 consecutive 32-bit columns of this thread's TMEM lane (warp-collective), then wait for the store
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+        "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+        "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
+        "r"(r[31])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 // low word of a descriptor: address >> 4 in bits [0,14), LBO >> 4 in bits [16,30)
 __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
     return ((addr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
@@ -386,11 +409,11 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 for (int blk = 0; blk < NBLK; ++blk) {
                     if (!mbar_wait(p_ready + (blk * 2 + bf) * 8, (t >> 1) & 1, abort_flag)) return false;
                     tc_fence_after();
-                    const uint32_t p_lo = desc_lo(p_u32 + (blk * 2 + bf) * C::P_BYTES, 0), v_lo = desc_lo(v_u32, C::BOX_BYTES);
+                    const uint32_t v_lo = desc_lo(v_u32, C::BOX_BYTES);
 #pragma unroll
-                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 32 bytes, V 16 rows of 128 bytes
-                        umma2(tmem + blk * C::COL_BLK + C::COL_O, p_lo + ks * (32 >> 4), v_lo + ks * (2048 >> 4), 0, idesc_pv,
-                              (t > 0 || ks > 0) ? 1u : 0u);
+                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 8 TMEM columns (in S's place), V 16 rows of 128 bytes
+                        umma_ta(tmem + blk * C::COL_BLK + C::COL_O, tmem + blk * C::COL_BLK + bf * kTile + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv,
+                                (t > 0 || ks > 0) ? 1u : 0u);
                     umma_commit(o_done + blk * 8);
                 }
                 umma_commit(empty_kv + st * 8);  // K and V of the tile are free once these MMAs have run
@@ -497,7 +520,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             }
             const float m_neg = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
             float2 psum2 = make_float2(0.f, 0.f), prnd2 = make_float2(0.f, 0.f);  // packed fp32 pairs: half the adds
-            unsigned char *prow = p_s + (blk * 2 + bf) * C::P_BYTES + r * 128;
+            uint32_t pw[kTile / 2];   // the row's P as bf16 pairs: goes where S was (first 32 columns of the buffer)
 #pragma unroll
             for (int ch = 0; ch < kTile / 8; ++ch) {
                 float e[8];
@@ -509,8 +532,9 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     psum2 = fadd2(psum2, make_float2(e[2 * i], e[2 * i + 1]));
                     prnd2 = fadd2(prnd2, make_float2(__uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u)));
                 }
-                *(uint4 *)(prow + ((ch ^ (r & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                pw[ch * 4] = pk[0]; pw[ch * 4 + 1] = pk[1]; pw[ch * 4 + 2] = pk[2]; pw[ch * 4 + 3] = pk[3];
             }
+            tmem_st32(lane_base + bf * kTile, pw);
             const float psum = psum2.x + psum2.y, prnd = prnd2.x + prnd2.y;
             l_run += psum;
             l_rnd += prnd;
@@ -519,7 +543,6 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
             }
-            fence_async_smem();
             tc_fence_before();
             mbar_arrive(p_ready + (blk * 2 + bf) * 8);
         }
