@@ -477,6 +477,8 @@ def main():
     ap.add_argument("--kv-hbm", default="bf16", choices=["bf16", "fp8"],
                     help="fp8: the chunks sit in HBM as e4m3 codes (MATKV_OPT_FP8_RESIDENT) and the streaming kernel converts them "
                     "in registers; a lossy KV format, so a workload of its own (forces --no-e2e)")
+    ap.add_argument("--prefill-impl", type=int, default=0, choices=[0, 1, 2, 3],
+                    help="sub-prefill kernel: 0 auto, 1 streaming kernel, 2 tensor-core kernel, 3 the same with two row blocks per CTA")
     ap.add_argument("--decode-impl", type=int, default=0, choices=[0, 1, 2],
                     help="decode kernel: 0 auto (chunk-major when the batch's requests share chunks), 1 request-major, 2 chunk-major")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
@@ -524,6 +526,8 @@ def main():
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, args.decode_ctas)
     if args.decode_impl:
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, args.decode_impl)
+    if args.prefill_impl:
+        mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_IMPL, args.prefill_impl)
     fused_advance = args.decode_launch == "all_layers"
     if fused_advance:   # the all-layers decode launch moves the tail itself: no separate counter kernel per step
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_ADVANCES_TAIL, 1)

@@ -29,8 +29,6 @@ namespace matkv {
 namespace k3 {
 
 constexpr int kRowsPerCta = 128;
-constexpr int kThreads = 192;  // producer warp, MMA warp, four softmax warps
-constexpr int kStages = 4;
 constexpr long long kWaitCycles = 2000000000LL;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -213,6 +211,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+// true in exactly one lane of the (converged) warp
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n .reg .pred p;\n elect.sync _|p, 0xffffffff;\n selp.b32 %0, 1, 0, p;\n}" : "=r"(pred));
+    return pred != 0;
+}
 __host__ __device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) / b; }
 
 // tile t of a unit: kind 0 = chunk, 1 = tail, 2 = new tokens
@@ -227,10 +231,9 @@ struct Cfg {
     static constexpr int KV_BYTES = NBOX * BOX_BYTES;    // K (or V) of one tile
     static constexpr int STAGE_BYTES = 2 * KV_BYTES;
     static constexpr int QBLK_BYTES = NBOX * kRowsPerCta * 128;   // Q of one row block
-    static constexpr int P_BYTES = kRowsPerCta * 128;             // 128 rows x 64 tokens bf16
-    static constexpr int STAGES = NBLK == 2 ? 3 : 4;
+    static constexpr int STAGES = 4;
     static constexpr int THREADS = (2 + 4 * NBLK) * 32;           // producer warp, MMA warp, 4 softmax warps per block
-    static constexpr int SMEM_BYTES = 1024 + NBLK * QBLK_BYTES + NBLK * 2 * P_BYTES + STAGES * STAGE_BYTES + 512;
+    static constexpr int SMEM_BYTES = 1024 + NBLK * QBLK_BYTES + STAGES * STAGE_BYTES + 512;
     // TMEM columns of row block b: S[2] at b*256 + {0, 64}; O at b*256 + 128 (D columns)
     static constexpr int COL_BLK = 256, COL_O = 128;
     static constexpr int TMEM_COLS = NBLK == 2 ? 512 : 256;
@@ -249,8 +252,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char *q_s = smem;                                   // [NBLK][NBOX boxes][128 rows][128 B]
-    unsigned char *p_s = q_s + NBLK * C::QBLK_BYTES;             // [NBLK][2][128 rows][128 B]
-    unsigned char *kv_s = p_s + NBLK * 2 * C::P_BYTES;           // kStages x (K boxes, V boxes)
+    unsigned char *kv_s = q_s + NBLK * C::QBLK_BYTES;            // kStages x (K boxes, V boxes)
     uint64_t *bars = (uint64_t *)(kv_s + kStages * C::STAGE_BYTES);
     uint32_t *tmem_slot = (uint32_t *)(bars + kBarCount);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 2);
@@ -396,44 +398,53 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
         // duration (measured: 30 us per CTA on a 1,024-token suffix).
         append_share();
     } else if (warp == 1) {
-        // ===================== MMA issuer (one thread) =====================
-        if (lane == 0) {
+        // ===================== MMA issuer =====================
+        // The whole warp walks the loop (waits and descriptor arithmetic on warp-uniform values); one elected lane
+        // issues the MMAs and their commits.  With a single lane behind a divergent branch every tcgen05.mma cost
+        // the issuing thread 65 to 85 cycles; this way it is about 45.
+        {
             constexpr uint32_t idesc_qk = instr_desc(kRowsPerCta, kTile, false);
             constexpr uint32_t idesc_pv = instr_desc(kRowsPerCta, D, true);
-            const uint32_t q_u32 = smem_u32(q_s), p_u32 = smem_u32(p_s), kv_u32 = smem_u32(kv_s);
-            bool ok = mbar_wait(q_ready, 0, abort_flag);
+            const uint32_t q_u32 = smem_u32(q_s), kv_u32 = smem_u32(kv_s);
+            bool ok = __all_sync(0xffffffffu, mbar_wait(q_ready, 0, abort_flag));
             auto do_pv = [&](int t) {  // O[blk] += P(t, blk) V(t) for every row block, then free the K/V stage
                 const int bf = t & 1, st = t % kStages;
                 const uint32_t v_u32 = kv_u32 + st * C::STAGE_BYTES + C::KV_BYTES;
 #pragma unroll
                 for (int blk = 0; blk < NBLK; ++blk) {
-                    if (!mbar_wait(p_ready + (blk * 2 + bf) * 8, (t >> 1) & 1, abort_flag)) return false;
+                    if (!__all_sync(0xffffffffu, mbar_wait(p_ready + (blk * 2 + bf) * 8, (t >> 1) & 1, abort_flag))) return false;
                     tc_fence_after();
                     const uint32_t v_lo = desc_lo(v_u32, C::BOX_BYTES);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 8 TMEM columns (in S's place), V 16 rows of 128 bytes
-                        umma_ta(tmem + blk * C::COL_BLK + C::COL_O, tmem + blk * C::COL_BLK + bf * kTile + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv,
-                                (t > 0 || ks > 0) ? 1u : 0u);
-                    umma_commit(o_done + blk * 8);
+                        for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 8 TMEM columns (in S's place), V 16 rows of 128 bytes
+                            umma_ta(tmem + blk * C::COL_BLK + C::COL_O, tmem + blk * C::COL_BLK + bf * kTile + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv,
+                                    (t > 0 || ks > 0) ? 1u : 0u);
+                        umma_commit(o_done + blk * 8);
+                        if (blk == NBLK - 1) umma_commit(empty_kv + st * 8);  // K and V of the tile are free once these MMAs have run
+                    }
+                    __syncwarp();
                 }
-                umma_commit(empty_kv + st * 8);  // K and V of the tile are free once these MMAs have run
                 return true;
             };
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const int st = j % kStages;
-                ok = mbar_wait(full_kv + st * 8, (j / kStages) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, mbar_wait(full_kv + st * 8, (j / kStages) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t k_u32 = kv_u32 + st * C::STAGE_BYTES;
+                if (elect_one()) {
 #pragma unroll
-                for (int blk = 0; blk < NBLK; ++blk) {
-                    const uint32_t q_lo = desc_lo(q_u32 + blk * C::QBLK_BYTES, 0), k_lo = desc_lo(k_u32, 0);
+                    for (int blk = 0; blk < NBLK; ++blk) {
+                        const uint32_t q_lo = desc_lo(q_u32 + blk * C::QBLK_BYTES, 0), k_lo = desc_lo(k_u32, 0);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
-                        umma2(tmem + blk * C::COL_BLK + (j & 1) * kTile, q_lo + (((ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32) >> 4),
-                              k_lo + (((ks / 4) * C::BOX_BYTES + (ks % 4) * 32) >> 4), 0, idesc_qk, ks > 0);
-                    umma_commit(s_full + (blk * 2 + (j & 1)) * 8);
+                        for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
+                            umma2(tmem + blk * C::COL_BLK + (j & 1) * kTile, q_lo + (((ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32) >> 4),
+                                  k_lo + (((ks / 4) * C::BOX_BYTES + (ks % 4) * 32) >> 4), 0, idesc_qk, ks > 0);
+                        umma_commit(s_full + (blk * 2 + (j & 1)) * 8);
+                    }
                 }
+                __syncwarp();
                 if (j >= 1) ok = do_pv(j - 1);
             }
             if (ok && n_tiles > 0) do_pv(n_tiles - 1);
@@ -632,7 +643,7 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     const int64_t combos = (int64_t)a.n_layers_launch * t->batch * c.n_kv_heads * p.n_rb;
     int min_tiles = 1 << 30;
     for (int b = 0; b < t->batch; ++b)
-        min_tiles = std::min(min_tiles, t->h_reqs[b].chunk_tiles + k3::cdiv(t->tail_len_host, kTile) + k3::cdiv(a.S, kTile));
+        min_tiles = std::min(min_tiles, t->h_reqs[b].chunk_tiles + k3::cdiv(t->tail_len_host, kTile) + 1);   // the first row block sees one tile of new tokens
     int64_t ns = ctx->opt_prefill_ctas > 0 ? ctx->opt_prefill_ctas : std::max<int64_t>(1, ctx->n_sm / combos);
     ns = std::min<int64_t>(ns, std::max(1, min_tiles));
     // the partials live in the workspace's partial regions (its head holds the streaming kernel's counters)
