@@ -110,27 +110,16 @@ __device__ __forceinline__ float fast_exp2(float x) {
 //   MN-major operand (rows = K index, the 128 bytes run along M or N): SBO = 1024 (next 8 K rows),
 //                     LBO = distance to the next 64-wide block along N.
 // bits: [0,14) address >> 4, [16,30) LBO >> 4, [32,46) SBO >> 4, [46,48) version 1, [61,64) layout 2 = SWIZZLE_128B.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
-           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
-}
+// (desc_lo below builds bits 0..31; the MMA helpers append the constant bits 32..63.)
 // Instruction descriptor, kind::f16: fp32 accumulate, bf16 x bf16, A K-major, B K- or MN-major, M x N.
 __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) |
            ((uint32_t)(M >> 4) << 24);
 }
-__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// The same with the descriptors given as (low word, high word): the high word (SBO, version, swizzle) is a constant
-// of the operand kind and the low word (address and LBO) advances by a plain 32-bit add, so the single issuing
-// thread spends a handful of instructions per MMA instead of rebuilding two 64-bit descriptors.
-__device__ __forceinline__ void umma2(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t b_hi_sel, uint32_t idesc, uint32_t accumulate) {
-    // both operand kinds used here share the high word except for nothing: SBO 1024, version 1, 128-byte swizzle
-    (void)b_hi_sel;
+// D (TMEM) = or += A (smem) B (smem).  The descriptors are given as low words (address and LBO, see desc_lo): the high
+// word (SBO 1024, version 1, 128-byte swizzle) is the same for every operand here, so the low word advances by a plain
+// 32-bit add and the issuing thread spends a handful of instructions per MMA instead of rebuilding 64-bit descriptors.
+__device__ __forceinline__ void umma2(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
     constexpr uint32_t kHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // bits 32.. of the descriptor
     asm volatile(
         "{\n .reg .pred p;\n .reg .b64 da, db;\n setp.ne.b32 p, %4, 0;\n mov.b64 da, {%1, %5};\n mov.b64 db, {%2, %5};\n"
@@ -168,9 +157,8 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// 32 consecutive fp32 columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-    uint32_t r[32];
+// 32 consecutive 32-bit columns of this thread's TMEM lane: the load is only issued; tmem_ld_wait() completes it
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
         "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
@@ -179,7 +167,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    tmem_ld32_issue(taddr, r);
+    tmem_ld_wait();
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
@@ -188,6 +182,14 @@ __device__ __forceinline__ float2 fadd2(float2 a, float2 b) {  // two fp32 adds 
     asm("add.rn.f32x2 %0, %1, %2;"
         : "=l"(d)
         : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)));
+    return *reinterpret_cast<float2 *>(&d);
+}
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {  // two fp32 FMAs in one instruction (sm_100)
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;"
+        : "=l"(d)
+        : "l"(*reinterpret_cast<unsigned long long *>(&a)), "l"(*reinterpret_cast<unsigned long long *>(&b)),
+          "l"(*reinterpret_cast<unsigned long long *>(&c)));
     return *reinterpret_cast<float2 *>(&d);
 }
 // multiply 32 consecutive fp32 columns of this thread's TMEM lane by `f` (load, scale, store back)
@@ -440,7 +442,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
 #pragma unroll
                         for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
                             umma2(tmem + blk * C::COL_BLK + (j & 1) * kTile, q_lo + (((ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32) >> 4),
-                                  k_lo + (((ks / 4) * C::BOX_BYTES + (ks % 4) * 32) >> 4), 0, idesc_qk, ks > 0);
+                                  k_lo + (((ks / 4) * C::BOX_BYTES + (ks % 4) * 32) >> 4), idesc_qk, ks > 0);
                         umma_commit(s_full + (blk * 2 + (j & 1)) * 8);
                     }
                 }
@@ -484,14 +486,16 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             if (!ok) break;
             tc_fence_after();
             float s[kTile];
-            {
-                float v[32];
-                tmem_ld32(lane_base + bf * kTile, v);
+            {   // both halves in flight before the one wait
+                uint32_t r0[32], r1[32];
+                tmem_ld32_issue(lane_base + bf * kTile, r0);
+                tmem_ld32_issue(lane_base + bf * kTile + 32, r1);
+                tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) s[i] = v[i];
-                tmem_ld32(lane_base + bf * kTile + 32, v);
-#pragma unroll
-                for (int i = 0; i < 32; ++i) s[32 + i] = v[i];
+                for (int i = 0; i < 32; ++i) {
+                    s[i] = __uint_as_float(r0[i]);
+                    s[32 + i] = __uint_as_float(r1[i]);
+                }
             }
             // visible columns: all valid rows of a chunk / tail tile; causal inside the new tokens.
             // Scores stay raw (unscaled) here: the scale is folded into the exponent's FMA below.
@@ -501,9 +505,15 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
 #pragma unroll
                 for (int i = 0; i < kTile; ++i) s[i] = i < n_vis ? s[i] : -CUDART_INF_F;
             }
-            float tmax = -CUDART_INF_F;
+            float tmax;
+            {   // eight independent chains, then a tree: a single chain of 64 dependent maxima costs 250 cycles of latency
+                float mx[8];
 #pragma unroll
-            for (int i = 0; i < kTile; ++i) tmax = fmaxf(tmax, s[i]);
+                for (int i = 0; i < 8; ++i) mx[i] = s[i];
+#pragma unroll
+                for (int i = 8; i < kTile; ++i) mx[i & 7] = fmaxf(mx[i & 7], s[i]);
+                tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+            }
             tmax *= p.scale_log2;   // the scale is positive: the maximum commutes with it
             // lazy rescale: move the reference only when the maximum has grown by more than 2^8
             const bool grow_ref = tmax > m_ref + 8.0f;   // also true for the first visible column (m_ref = -inf)
@@ -530,13 +540,18 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 }
             }
             const float m_neg = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), mn2 = make_float2(m_neg, m_neg);
             float2 psum2 = make_float2(0.f, 0.f), prnd2 = make_float2(0.f, 0.f);  // packed fp32 pairs: half the adds
             uint32_t pw[kTile / 2];   // the row's P as bf16 pairs: goes where S was (first 32 columns of the buffer)
 #pragma unroll
             for (int ch = 0; ch < kTile / 8; ++ch) {
                 float e[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) e[i] = fast_exp2(fmaf(s[ch * 8 + i], p.scale_log2, m_neg));
+                for (int i = 0; i < 4; ++i) {   // scale and offset as packed pairs: half the FMAs
+                    const float2 x = ffma2(make_float2(s[ch * 8 + 2 * i], s[ch * 8 + 2 * i + 1]), sc2, mn2);
+                    e[2 * i] = fast_exp2(x.x);
+                    e[2 * i + 1] = fast_exp2(x.y);
+                }
                 const uint32_t pk[4] = {pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7])};
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
