@@ -467,13 +467,14 @@ def main():
                     "(storage tier: reader threads -> pinned bounce ring -> device) instead of in pinned host memory")
     ap.add_argument("--io-threads", type=int, default=8)
     ap.add_argument("--stage-ctas", type=int, default=-1, help="stage host chunks with a copy kernel of this many CTAs; 0 = copy "
-                    "engine; -1 = auto: 16 CTAs in the pipelined-serving mode (long decode launches that saturate HBM starve "
-                    "the copy engine), copy engine in the single-batch end-to-end leg (short launches: a co-resident copy "
-                    "CTA makes its SM the straggler of every launch)")
+                    "engine; -1 = auto: 16 CTAs in the pipelined-serving mode, 8 in the single-batch end-to-end leg (a decode that "
+                    "saturates HBM starves the copy engine: 38 GB/s against 45 with the copy kernel; more than 10 copy CTAs "
+                    "slow the short decode launches of that leg down more than they add)")
     ap.add_argument("--kv-store", default="bf16", choices=["bf16", "fp8"],
                     help="pipelined serving: keep the host / file chunk pool as plain bf16 blobs or compressed (e4m3 codes with a "
                     "power-of-two scale per 64-token block, expanded to bf16 while staged; a lossy store, so a separate workload)")
-    ap.add_argument("--copy-streams", type=int, default=2, help="end-to-end leg: copy streams the chunk staging of a step is split over")
+    ap.add_argument("--copy-streams", type=int, default=0, help="end-to-end leg: copy streams the chunk staging of a step is split over "
+                    "(0 = auto: one with the copy kernel, two with the copy engine)")
     ap.add_argument("--kv-hbm", default="bf16", choices=["bf16", "fp8"],
                     help="fp8: the chunks sit in HBM as e4m3 codes (MATKV_OPT_FP8_RESIDENT) and the streaming kernel converts them "
                     "in registers; a lossy KV format, so a workload of its own (forces --no-e2e)")
@@ -775,54 +776,69 @@ def main():
         ho_dc = torch.empty(o_dc.shape, dtype=torch.bfloat16, pin_memory=True)
         torch.cuda.synchronize()
         sess2 = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
-        if args.stage_ctas > 0:
-            mk.matkv_set_option(sess2.ctx, mk.OPT_STAGE_CTAS, args.stage_ctas)
+        e2e_stage_ctas = args.stage_ctas if args.stage_ctas >= 0 else 8
+        if e2e_stage_ctas > 0:
+            mk.matkv_set_option(sess2.ctx, mk.OPT_STAGE_CTAS, e2e_stage_ctas)
         for c in needed:
             mk.matkv_register_chunk(sess2.ctx, c, w.chunk_tokens, host[c].data_ptr(), None)
         slot_bytes = w.chunk_bytes
         # the chunks of a step are split over N_COPY copy streams, each with slot regions of its own: several copies in
         # flight keep the link busier while the decode saturates HBM
-        n_copy = max(1, min(args.copy_streams, len(needed)))
+        n_copy = max(1, min(args.copy_streams if args.copy_streams > 0 else (1 if e2e_stage_ctas > 0 else 2), len(needed)))
         parts = [needed[k::n_copy] for k in range(n_copy)]
         copies = [copy] + [torch.cuda.Stream(device=dev) for _ in range(n_copy - 1)]
-        slots = [[torch.empty(len(parts[k]) * slot_bytes, dtype=torch.uint8, device=dev) for k in range(n_copy)] for _ in range(2)]
-        # query-side inputs and outputs are double-buffered on the device: step i+1's inputs arrive (copy stream)
-        # and step i-1's outputs leave (output stream) while step i computes
-        d_in = [tuple(torch.empty_like(x) for x in (q_pf, k_pf, v_pf, q_dc, k_dc, v_dc)) for _ in range(2)]
-        d_out = [(torch.empty_like(o_pf), torch.empty_like(o_dc)) for _ in range(2)]
+        # Three regions of chunk slots and of query-side buffers: the copies of step i+2 start as soon as step i-1 has
+        # finished with its region, so the link never waits for the compute (with two regions the copies of step i+1
+        # could only start when step i's compute did, and a step took as long as its copies plus the hand-over).
+        NB = 3
+        slots = [[torch.empty(len(parts[k]) * slot_bytes, dtype=torch.uint8, device=dev) for k in range(n_copy)] for _ in range(NB)]
+        d_in = [tuple(torch.empty_like(x) for x in (q_pf, k_pf, v_pf, q_dc, k_dc, v_dc)) for _ in range(NB)]
+        d_out = [(torch.empty_like(o_pf), torch.empty_like(o_dc)) for _ in range(NB)]
         h_in = (hq_pf, hk_pf, hv_pf, hq_dc, hk_dc, hv_dc)
         h2d = len(needed) * slot_bytes + sum(x.numel() * 2 for x in h_in)
         d2h = (ho_pf.numel() + ho_dc.numel()) * 2
         ctx2 = sess2.ctx
         out_stream = torch.cuda.Stream(device=dev)
-        in_ready = [torch.cuda.Event() for _ in range(2)]
-        comp_done = [torch.cuda.Event() for _ in range(2)]
-        out_done = [torch.cuda.Event() for _ in range(2)]
-        state = {"loaded": -1}
+        in_ready = [torch.cuda.Event() for _ in range(NB)]
+        comp_done = [torch.cuda.Event() for _ in range(NB)]
+        out_done = [torch.cuda.Event() for _ in range(NB)]
+        load_done = [torch.cuda.Event() for _ in range(n_copy)]
+        state = {"loaded": -1, "table": None}
 
         def load(i):
-            """Everything step i needs from the host, on the copy stream: its query-side inputs (small, first),
-            then its chunks into slot region i % 2."""
-            if i >= 2:
-                copy.wait_event(comp_done[i % 2])          # step i-2 has finished with these input buffers
+            """Everything step i needs from the host: its query-side inputs (small, first) on the first copy stream, its
+            chunks into slot region i % NB over all copy streams.  No copy starts before step i - NB, the last user of
+            the region, has finished."""
+            r = i % NB
+            if i >= NB:
+                for cs in copies:
+                    cs.wait_event(comp_done[r])
             with torch.cuda.stream(copy):
-                for dst, src in zip(d_in[i % 2], h_in):
+                for dst, src in zip(d_in[r], h_in):
                     dst.copy_(src, non_blocking=True)
-                in_ready[i % 2].record(copy)
+                in_ready[r].record(copy)
             for k in range(n_copy):
-                sess2.stage(parts[k], slots[i % 2][k], slot_bytes, copies[k])
+                sess2.stage(parts[k], slots[r][k], slot_bytes, copies[k])
+                load_done[k].record(copies[k])
             state["loaded"] = i
 
+        def drain_copies():
+            """The compute stream waits for every copy issued so far.  Called right before the timed region and at its
+            end: the region then holds exactly as many whole loads as steps (the loads it starts with in flight are
+            finished first, the ones it issues ahead for later steps are finished inside it)."""
+            for k in range(n_copy):
+                stream.wait_event(load_done[k])
+
         def e2e_step(i, last=False):
-            if state["loaded"] < i:
-                load(i)
-            dq_pf, dk_pf, dv_pf, dq_dc, dk_dc, dv_dc = d_in[i % 2]
-            eo_pf, eo_dc = d_out[i % 2]
-            table = sess2.build_table(ids, sp)             # makes the compute stream wait for this step's chunk copies
-            stream.wait_event(in_ready[i % 2])
-            if i >= 2:
-                stream.wait_event(out_done[i % 2])         # step i-2's outputs have left these buffers
-            load(i + 1)                                    # the next step's copies run under this step's compute
+            # step i's table was built at the end of step i-1 (or before the first step), AFTER load(i) and BEFORE
+            # load(i+1): a table points at the places its chunks were staged to most recently
+            table = state["table"]
+            r = i % NB
+            dq_pf, dk_pf, dv_pf, dq_dc, dk_dc, dv_dc = d_in[r]
+            eo_pf, eo_dc = d_out[r]
+            stream.wait_event(in_ready[r])
+            if i >= NB:
+                stream.wait_event(out_done[r])             # step i-NB's outputs have left these buffers
             if args.decode_launch == "all_layers":
                 mk.matkv_attend_prefill_all_layers(ctx2, table, S, dq_pf.data_ptr(), dk_pf.data_ptr(), dv_pf.data_ptr(), eo_pf.data_ptr(), None, sp)
             else:
@@ -842,30 +858,39 @@ def main():
                                                dk_dc.data_ptr() + t * kd_t + layer * kd_l, dv_dc.data_ptr() + t * kd_t + layer * kd_l,
                                                eo_dc.data_ptr() + t * qd_t + layer * qd_l, None, sp)
                 mk.matkv_table_advance(table, 1, sp)
-            comp_done[i % 2].record(stream)
-            out_stream.wait_event(comp_done[i % 2])
+            comp_done[r].record(stream)
+            out_stream.wait_event(comp_done[r])
             with torch.cuda.stream(out_stream):            # the step's results go back to the host
                 ho_pf.copy_(eo_pf, non_blocking=True)
                 ho_dc.copy_(eo_dc, non_blocking=True)
-                out_done[i % 2].record(out_stream)
+                out_done[r].record(out_stream)
+            # the next step's table (its build makes the compute stream wait for that step's chunk copies, issued one
+            # step ago), then the copies of the step after it
+            state["table"] = sess2.build_table(ids, sp)
+            load(i + 2)
             if last:
-                stream.wait_event(out_done[i % 2])         # the timed region ends when the last result is on the host
+                stream.wait_event(out_done[r])             # the timed region ends when the last result is on the host
+                drain_copies()                             # and when every copy it issued has landed
             return 0
 
         if fused_advance:
             mk.matkv_set_option(ctx2, mk.OPT_DECODE_ADVANCES_TAIL, 1)
         with torch.cuda.stream(stream):
+            load(0)
+            state["table"] = sess2.build_table(ids, sp)
+            load(1)
             for i in range(2):
                 e2e_step(i)
+            drain_copies()
             k_e2e = min(args.steps, 5)
             ms_e, _, _, _ = timed_region(lambda i: e2e_step(i + 2, last=(i == k_e2e - 1)), k_e2e)
         if sess2.status() != 0:
             raise RuntimeError("device status non-zero after the end-to-end region")
         result["e2e"] = {"value": tokens * k_e2e / (ms_e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
                          "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e,
-                         "overlap": "next step's chunks and query-side inputs copied in, and the previous step's outputs copied out, "
-                                    "on side streams under this step's prefill and decode",
-                         "staging": (f"copy kernel, {args.stage_ctas} CTAs" if args.stage_ctas > 0 else "copy engine") + f", {n_copy} copy streams",
+                         "overlap": "the chunks and query-side inputs of the next two steps copied in (three slot regions), and the previous "
+                                    "step's outputs copied out, on side streams under this step's prefill and decode",
+                         "staging": (f"copy kernel, {e2e_stage_ctas} CTAs" if e2e_stage_ctas > 0 else "copy engine") + f", {n_copy} copy streams",
                          "h2d_gbs_if_copy_bound": h2d * k_e2e / (ms_e * 1e-3) / 1e9}
         sess2.close()
         del host, slots
