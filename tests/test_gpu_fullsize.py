@@ -1,6 +1,7 @@
 """Parity at the benchmark's full size and launch configuration (config 2: 32 layers, Llama-3-8B head
 shape, 5 x 1,024-token chunks, 64-token suffix through the tile kernel, 128 decode steps with all layers
-in one launch; config 3: batch 16, 10 of 256 chunks per request by Zipf rank, chunk-major decode), on
+in one launch; config 3: batch 16, 10 of 256 chunks per request by Zipf rank, chunk-major decode; config 4: the 70B head
+shape with 64K tokens of context per request), on
 sampled outputs the oracle computes one by one."""
 import numpy as np
 import pytest
@@ -133,4 +134,75 @@ def test_cfg3_full_size_chunk_major_sampled_units():
             o_ref, l_ref = rq.attend_new(0, q[layer, r][None], k[layer, r][None], v[layer, r][None])
             check(got[step][0][layer, r], o_ref[0], got[step][1][layer, r], l_ref[0],
                   f"full-size chunk-major decode step {step} layer {layer} request {r}")
+    sess.close()
+
+
+def test_cfg4_full_size_sampled_units():
+    """Config 4 at full size (Llama-3-70B head shape: 64 query heads on 8 KV heads, 80 layers, 4 requests x 32 chunks of
+    2,048 tokens = 86 GB of chunks in HBM, 128-token suffix: 1,024 query rows per KV head through the tile kernel with
+    two row blocks per CTA, all 80 layers in one launch of 10,240 CTAs; 64 decode steps, all layers per launch);
+    sampled outputs against the oracle."""
+    import matkv_inputs.device as gen
+    from paper_2512_22195_b200.harness import Session, dev_to_bits
+    w = mi.workload("cfg4")
+    L, B, S, T, Hq, Hkv, D = w.n_layers, w.batch, w.suffix, w.decode_steps, w.n_q_heads, w.n_kv_heads, w.head_dim
+    free, _ = torch.cuda.mem_get_info()
+    if free < 100e9:
+        pytest.skip("needs 100 GB of free device memory")
+    ids = w.chunk_ids(0)
+    needed = sorted({c for row in ids for c in row})
+    sess = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T)
+    pool = torch.empty((len(needed), L, 2, Hkv, w.chunk_tokens, D), dtype=torch.bfloat16, device="cuda")
+    for i, c in enumerate(needed):
+        gen.fill_bf16(pool[i], w.seed, mi.STREAM_CHUNK + c)
+        sess.register_device_chunk(c, pool[i])
+    q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device="cuda")
+    k_pf = torch.empty((L, B, S, Hkv, D), dtype=torch.bfloat16, device="cuda")
+    v_pf = torch.empty_like(k_pf)
+    q_dc = torch.empty((T, L, B, Hq, D), dtype=torch.bfloat16, device="cuda")
+    k_dc = torch.empty((T, L, B, Hkv, D), dtype=torch.bfloat16, device="cuda")
+    v_dc = torch.empty_like(k_dc)
+    for t_, st in ((q_pf, mi.STREAM_Q_PREFILL), (k_pf, mi.STREAM_K_PREFILL), (v_pf, mi.STREAM_V_PREFILL),
+                   (q_dc, mi.STREAM_Q_DECODE), (k_dc, mi.STREAM_K_DECODE), (v_dc, mi.STREAM_V_DECODE)):
+        gen.fill_bf16(t_, w.seed, st)
+    sess.build_table(ids)
+    pf_out, pf_lse = sess.prefill_all_layers(q_pf, k_pf, v_pf)
+    sess.advance(S)
+    samples = {0: [(0, 0)], 31: [(40, 2)], T - 1: [(L - 1, 3)]}          # decode step -> (layer, request)
+    got = {}
+    for t in range(T):
+        out, lse = sess.decode_all_layers(q_dc[t], k_dc[t], v_dc[t])
+        if t in samples:
+            got[t] = (dev_to_bits(out), lse.cpu().numpy())
+        sess.advance(1)
+    assert sess.status() == 0
+    sh1 = oracle.Shape(1, Hq, Hkv, D)
+
+    def layer_request(layer, r, n_decode):
+        blobs = [dev_to_bits(pool[needed.index(c)][layer:layer + 1]) for c in ids[r]]
+        rq = oracle.Request(sh1, blobs, S + T)
+        _, k, v = mi.prefill_inputs(w, layer)
+        rq.append_only(0, k[r], v[r])
+        rq.advance(S)
+        for s_ in range(n_decode):
+            _, k, v = mi.decode_inputs(w, s_)
+            rq.append_only(0, k[layer, r][None], v[layer, r][None])
+            rq.advance(1)
+        return rq
+
+    # sub-prefill: first, middle and last suffix token of a request in the first and the last layer (every head)
+    for layer, r in ((0, 0), (L - 1, B - 1)):
+        rq = layer_request(layer, r, 0)
+        q, _, _ = mi.prefill_inputs(w, layer)
+        rows = [0, S // 2 - 1, S - 1]
+        o_ref, l_ref = oracle.attend(sh1, 0, rq.chunks, rq.tail_k[0], rq.tail_v[0], q[r][rows], [x + 1 for x in rows])
+        check(dev_to_bits(pf_out[layer])[r][rows], o_ref, pf_lse[layer].cpu().numpy()[r][rows], l_ref,
+              f"config 4 full-size prefill layer {layer} request {r}")
+    for step, pairs in samples.items():
+        q, k, v = mi.decode_inputs(w, step)
+        for layer, r in pairs:
+            rq = layer_request(layer, r, step)
+            o_ref, l_ref = rq.attend_new(0, q[layer, r][None], k[layer, r][None], v[layer, r][None])
+            check(got[step][0][layer, r], o_ref[0], got[step][1][layer, r], l_ref[0],
+                  f"config 4 full-size decode step {step} layer {layer} request {r}")
     sess.close()
