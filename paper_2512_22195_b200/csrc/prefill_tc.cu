@@ -244,7 +244,7 @@ struct Cfg {
 
 // barrier slots (8 bytes each)
 constexpr int kBarFull = 0, kBarEmpty = 4, kBarSFull = 8 /* [blk][2] */, kBarPReady = 12 /* [blk][2] */,
-              kBarODone = 16 /* [blk] */, kBarQReady = 18, kBarCount = 20;
+              kBarODone = 16 /* [blk][2] */, kBarQReady = 20, kBarCount = 21;
 
 template <int D, int G, int NBLK>
 __global__ void __launch_bounds__((2 + 4 * NBLK) * 32, 1)
@@ -294,8 +294,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             mbar_init(s_full + s * 8, 1);
             mbar_init(p_ready + s * 8, 128);
         }
-        mbar_init(o_done, 1);
-        mbar_init(o_done + 8, 1);
+        for (int s = 0; s < 4; ++s) mbar_init(o_done + s * 8, 1);
         mbar_init(q_ready, 128 * NBLK);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -422,7 +421,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                         for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 8 TMEM columns (in S's place), V 16 rows of 128 bytes
                             umma_ta(tmem + blk * C::COL_BLK + C::COL_O, tmem + blk * C::COL_BLK + bf * kTile + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv,
                                     (t > 0 || ks > 0) ? 1u : 0u);
-                        umma_commit(o_done + blk * 8);
+                        umma_commit(o_done + (blk * 2 + bf) * 8);
                         if (blk == NBLK - 1) umma_commit(empty_kv + st * 8);  // K and V of the tile are free once these MMAs have run
                     }
                     __syncwarp();
@@ -478,8 +477,16 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
         float m_ref = -CUDART_INF_F, l_run = 0.f, l_rnd = 0.f;
         int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
         bool ok = true;
+        int plain_end = 0;   // tiles before it (of the unit) are full chunk tiles: every column visible, nothing to look up
         for (int j = 0; j < n_tiles && ok; ++j) {
-            const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len);
+            // visible columns: all valid rows of a chunk / tail tile; causal inside the new tokens
+            int n_vis = kTile;
+            if (t_begin + j >= plain_end) {
+                const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len);
+                n_vis = ti.rows;
+                if (ti.kind == 2) n_vis = min(ti.rows, tok - ti.r0 + 1);
+                if (ti.kind == 0) plain_end = tiles_before + seg_len / kTile;
+            }
             const int bf = j & 1;
             ok = mbar_wait(s_full + (blk * 2 + bf) * 8, (j >> 1) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);   // the TMEM loads below are warp-collective
@@ -497,10 +504,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     s[32 + i] = __uint_as_float(r1[i]);
                 }
             }
-            // visible columns: all valid rows of a chunk / tail tile; causal inside the new tokens.
             // Scores stay raw (unscaled) here: the scale is folded into the exponent's FMA below.
-            int n_vis = ti.rows;
-            if (ti.kind == 2) n_vis = min(ti.rows, tok - ti.r0 + 1);
             if (n_vis < kTile) {  // ragged or causal tile: mask (a full tile skips this)
 #pragma unroll
                 for (int i = 0; i < kTile; ++i) s[i] = i < n_vis ? s[i] : -CUDART_INF_F;
@@ -517,17 +521,16 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             tmax *= p.scale_log2;   // the scale is positive: the maximum commutes with it
             // lazy rescale: move the reference only when the maximum has grown by more than 2^8
             const bool grow_ref = tmax > m_ref + 8.0f;   // also true for the first visible column (m_ref = -inf)
-            // Every thread consumes every phase of o_done in order (P V of tile j-1 during tile j): a one-bit
-            // phase can only be told apart from its neighbours, never from a phase two steps away.
-            bool pv_prev_done = j == 0;
+            // o_done has one barrier per parity of the tile index, like S: a waiter is never more than one use of a
+            // barrier behind (the P V of tile j+1 cannot be issued before this thread has delivered P of tile j+1), so
+            // tiles whose completion nobody needs to see are simply not waited for.
             if (__any_sync(0xffffffffu, grow_ref)) {     // tcgen05.ld / st are warp-collective: decide per warp
                 const float alpha = grow_ref ? (m_ref == -CUDART_INF_F ? 0.f : fast_exp2(m_ref - tmax)) : 1.f;
                 if (j > 0) {
                     // O of tiles 0..j-1 must be complete before it is scaled
-                    ok = mbar_wait(o_done + blk * 8, (j - 1) & 1, abort_flag);
+                    ok = mbar_wait(o_done + (blk * 2 + ((j - 1) & 1)) * 8, ((j - 1) >> 1) & 1, abort_flag);
                     ok = __all_sync(0xffffffffu, ok);
                     if (!ok) break;
-                    pv_prev_done = true;
                     tc_fence_after();
 #pragma unroll
                     for (int c0 = 0; c0 < D; c0 += 32) tmem_scale32(lane_base + C::COL_O + c0, alpha);
@@ -564,17 +567,12 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             const float psum = psum2.x + psum2.y, prnd = prnd2.x + prnd2.y;
             l_run += psum;
             l_rnd += prnd;
-            if (!pv_prev_done) {  // normally long since complete: the wait only keeps the phase count in step
-                ok = mbar_wait(o_done + blk * 8, (j - 1) & 1, abort_flag);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-            }
             tc_fence_before();
             mbar_arrive(p_ready + (blk * 2 + bf) * 8);
         }
         // epilogue: O is complete once the last P V has run
         if (ok && n_tiles > 0) {
-            ok = mbar_wait(o_done + blk * 8, (n_tiles - 1) & 1, abort_flag);
+            ok = mbar_wait(o_done + (blk * 2 + ((n_tiles - 1) & 1)) * 8, ((n_tiles - 1) >> 1) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
         }
         if (ok) {
