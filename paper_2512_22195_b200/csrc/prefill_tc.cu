@@ -234,7 +234,8 @@ struct Cfg {
     static constexpr int STAGE_BYTES = 2 * KV_BYTES;
     static constexpr int QBLK_BYTES = NBOX * kRowsPerCta * 128;   // Q of one row block
     static constexpr int STAGES = 4;
-    static constexpr int THREADS = (2 + 4 * NBLK) * 32;           // producer warp, MMA warp, 4 softmax warps per block
+    // producer warp, MMA warp of row block 0, 4 softmax warps per block, and (last) the MMA warp of row block 1
+    static constexpr int THREADS = (2 + 4 * NBLK + (NBLK - 1)) * 32;
     static constexpr int SMEM_BYTES = 1024 + NBLK * QBLK_BYTES + STAGES * STAGE_BYTES + 512;
     // TMEM columns of row block b: S[2] at b*256 + {0, 64}; O at b*256 + 128 (D columns)
     static constexpr int COL_BLK = 256, COL_O = 128;
@@ -247,7 +248,7 @@ constexpr int kBarFull = 0, kBarEmpty = 4, kBarSFull = 8 /* [blk][2] */, kBarPRe
               kBarODone = 16 /* [blk][2] */, kBarQReady = 20, kBarCount = 21;
 
 template <int D, int G, int NBLK>
-__global__ void __launch_bounds__((2 + 4 * NBLK) * 32, 1)
+__global__ void __launch_bounds__((2 + 4 * NBLK + (NBLK - 1)) * 32, 1)
 k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap kn_map, const __grid_constant__ CUtensorMap vn_map) {
     using C = Cfg<D, NBLK>;
     constexpr int kStages = C::STAGES;
@@ -290,7 +291,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
     if (tid == 0) {
         for (int s = 0; s < 4; ++s) {
             mbar_init(full_kv + s * 8, 1);
-            mbar_init(empty_kv + s * 8, 1);
+            mbar_init(empty_kv + s * 8, NBLK);   // one commit per row block's MMA warp
             mbar_init(s_full + s * 8, 1);
             mbar_init(p_ready + s * 8, 128);
         }
@@ -398,34 +399,34 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
         // tile load of the CTA has been issued.  Issued between two tile loads it held the second one back by its whole
         // duration (measured: 30 us per CTA on a 1,024-token suffix).
         append_share();
-    } else if (warp == 1) {
-        // ===================== MMA issuer =====================
+    } else if (warp == 1 || warp == 2 + 4 * NBLK) {
+        // ===================== MMA issuers: one warp per row block =====================
         // The whole warp walks the loop (waits and descriptor arithmetic on warp-uniform values); one elected lane
         // issues the MMAs and their commits.  With a single lane behind a divergent branch every tcgen05.mma cost
         // the issuing thread 65 to 85 cycles; this way it is about 45.
+        // Each row block has an issuing warp of its own, so the blocks are independent pipelines that share only the
+        // K/V ring (a stage is free when both warps' P V of its tile have run) and the tensor pipe itself: with one
+        // warp issuing for both in a fixed order, each block's S = Q K^T waited for the other block's softmax.
         {
+            const int blk = warp == 1 ? 0 : 1;
             constexpr uint32_t idesc_qk = instr_desc(kRowsPerCta, kTile, false);
             constexpr uint32_t idesc_pv = instr_desc(kRowsPerCta, D, true);
-            const uint32_t q_u32 = smem_u32(q_s), kv_u32 = smem_u32(kv_s);
+            const uint32_t q_lo = desc_lo(smem_u32(q_s) + blk * C::QBLK_BYTES, 0), kv_u32 = smem_u32(kv_s);
+            const uint32_t tm = tmem + blk * C::COL_BLK;
             bool ok = __all_sync(0xffffffffu, mbar_wait(q_ready, 0, abort_flag));
-            auto do_pv = [&](int t) {  // O[blk] += P(t, blk) V(t) for every row block, then free the K/V stage
+            auto do_pv = [&](int t) {  // O += P(t) V(t), then this block's share of freeing the K/V stage
                 const int bf = t & 1, st = t % kStages;
-                const uint32_t v_u32 = kv_u32 + st * C::STAGE_BYTES + C::KV_BYTES;
+                if (!__all_sync(0xffffffffu, mbar_wait(p_ready + (blk * 2 + bf) * 8, (t >> 1) & 1, abort_flag))) return false;
+                tc_fence_after();
+                const uint32_t v_lo = desc_lo(kv_u32 + st * C::STAGE_BYTES + C::KV_BYTES, C::BOX_BYTES);
+                if (elect_one()) {
 #pragma unroll
-                for (int blk = 0; blk < NBLK; ++blk) {
-                    if (!__all_sync(0xffffffffu, mbar_wait(p_ready + (blk * 2 + bf) * 8, (t >> 1) & 1, abort_flag))) return false;
-                    tc_fence_after();
-                    const uint32_t v_lo = desc_lo(v_u32, C::BOX_BYTES);
-                    if (elect_one()) {
-#pragma unroll
-                        for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 8 TMEM columns (in S's place), V 16 rows of 128 bytes
-                            umma_ta(tmem + blk * C::COL_BLK + C::COL_O, tmem + blk * C::COL_BLK + bf * kTile + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv,
-                                    (t > 0 || ks > 0) ? 1u : 0u);
-                        umma_commit(o_done + (blk * 2 + bf) * 8);
-                        if (blk == NBLK - 1) umma_commit(empty_kv + st * 8);  // K and V of the tile are free once these MMAs have run
-                    }
-                    __syncwarp();
+                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 8 TMEM columns (in S's place), V 16 rows of 128 bytes
+                        umma_ta(tm + C::COL_O, tm + bf * kTile + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+                    umma_commit(o_done + (blk * 2 + bf) * 8);
+                    umma_commit(empty_kv + st * 8);
                 }
+                __syncwarp();
                 return true;
             };
             for (int j = 0; j < n_tiles && ok; ++j) {
@@ -433,17 +434,13 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 ok = __all_sync(0xffffffffu, mbar_wait(full_kv + st * 8, (j / kStages) & 1, abort_flag));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t k_u32 = kv_u32 + st * C::STAGE_BYTES;
+                const uint32_t k_lo = desc_lo(kv_u32 + st * C::STAGE_BYTES, 0);
                 if (elect_one()) {
 #pragma unroll
-                    for (int blk = 0; blk < NBLK; ++blk) {
-                        const uint32_t q_lo = desc_lo(q_u32 + blk * C::QBLK_BYTES, 0), k_lo = desc_lo(k_u32, 0);
-#pragma unroll
-                        for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
-                            umma2(tmem + blk * C::COL_BLK + (j & 1) * kTile, q_lo + (((ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32) >> 4),
-                                  k_lo + (((ks / 4) * C::BOX_BYTES + (ks % 4) * 32) >> 4), idesc_qk, ks > 0);
-                        umma_commit(s_full + (blk * 2 + (j & 1)) * 8);
-                    }
+                    for (int ks = 0; ks < D / 16; ++ks)  // 16 dims per MMA; 4 such slices per 64-wide box
+                        umma2(tm + (j & 1) * kTile, q_lo + (((ks / 4) * (kRowsPerCta * 128) + (ks % 4) * 32) >> 4),
+                              k_lo + (((ks / 4) * C::BOX_BYTES + (ks % 4) * 32) >> 4), idesc_qk, ks > 0);
+                    umma_commit(s_full + (blk * 2 + (j & 1)) * 8);
                 }
                 __syncwarp();
                 if (j >= 1) ok = do_pv(j - 1);
