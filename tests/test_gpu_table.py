@@ -277,3 +277,44 @@ def test_materialise_then_reuse_round_trip():
     check(to_bits(out)[0], o_ref[0], lse.cpu().numpy()[0], l_ref[0], "decode over the re-used chunk")
     assert sess.status() == 0 and sess2.status() == 0
     sess.close(); sess2.close()
+
+
+def test_context_and_table_churn_leaves_no_device_memory_behind():
+    """A serving process creates and frees tables for every batch and contexts now and then: 150 contexts, ten tables
+    each (both decode kernels' tables), a sub-prefill and two decode steps per table; the device's free memory at
+    the end is what it was after the first cycle (torch's caching allocator keeps the harness's own tensors, so what
+    would show here is memory the library itself allocated and lost)."""
+    mk, Session, bits_to_dev, dev_to_bits = _mk()
+    L, Hq, Hkv, D, B = 2, 8, 2, 128, 3
+    blobs = [bits_to_dev(rand_bits(91, i, (L, 2, Hkv, n, D))) for i, n in enumerate([130, 64, 200])]
+    q = bits_to_dev(rand_bits(91, 10, (B, 5, Hq, D)))
+    k = bits_to_dev(rand_bits(91, 11, (B, 5, Hkv, D)))
+    q1, k1 = q[:, :1].contiguous(), k[:, :1].contiguous()
+
+    def cycle(i):
+        sess = Session(L, Hq, Hkv, D, B, 3, 16)
+        if i % 2:
+            mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, 2)
+        for c, b in enumerate(blobs):
+            sess.register_device_chunk(c, b)
+        for t in range(10):
+            sess.build_table([[0, 1, 2], [t % 3], [2, 0]])
+            for layer in range(L):
+                sess.prefill(layer, q, k, k, want_lse=False)
+            sess.advance(5)
+            for _ in range(2):
+                for layer in range(L):
+                    sess.decode(layer, q1[:, 0], k1[:, 0], k1[:, 0])
+                sess.advance(1)
+        assert sess.status() == 0
+        sess.close()
+
+    cycle(0)
+    cycle(1)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for i in range(150):
+        cycle(i)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free0 - free1 < 8 << 20, f"{(free0 - free1) / 2**20:.1f} MiB of device memory did not come back"
