@@ -552,8 +552,10 @@ template <int D, int G>
 static int launch_shared_t(const SharedParams &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
     using C = SharedCfg<D, G>;
     static PerDeviceOnce configured;
-    if (configured.need()) {
+    int once_dev;
+    if (configured.need(&once_dev)) {
         MATKV_CUDA(cudaFuncSetAttribute(k_attend_shared<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        configured.mark(once_dev);
     }
     k_attend_shared<D, G><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());

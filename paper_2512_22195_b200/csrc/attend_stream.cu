@@ -627,8 +627,10 @@ template <int D, int G, bool F8 = false>
 static int launch_stream_t(const StreamParams &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
     using C = StreamCfg<D, G, F8>;
     static PerDeviceOnce configured;
-    if (configured.need()) {
+    int once_dev;
+    if (configured.need(&once_dev)) {
         MATKV_CUDA(cudaFuncSetAttribute(k_attend_stream<D, G, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        configured.mark(once_dev);
     }
     k_attend_stream<D, G, F8><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());

@@ -204,8 +204,10 @@ int launch_stage_expand_fp8(matkv_ctx *ctx, const void *src_fp8, void *dev_dst, 
     const int32_t vec_per_slab = (int32_t)((int64_t)n_tokens * c.head_dim / 16);
     const int32_t vec_per_block = 64 * c.head_dim / 16;
     static PerDeviceOnce configured;
-    if (configured.need()) {
+    int once_dev;
+    if (configured.need(&once_dev)) {
         MATKV_CUDA(cudaFuncSetAttribute(k_stage_expand_fp8, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        configured.mark(once_dev);
     }
     k_stage_expand_fp8<<<n_ctas, 128, (size_t)((n_exps + 15) / 16 * 16), stream>>>((const uint4 *)codes, exps, (uint4 *)dev_dst, n_vec, vec_per_slab,
                                                                                  vec_per_block, nb, (int32_t)n_exps);

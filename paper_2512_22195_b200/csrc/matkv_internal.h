@@ -1,5 +1,6 @@
 // Internal declarations shared by the host-side C ABI and the kernels' launchers.
 #pragma once
+#include <atomic>
 #include <cuda.h>  // CUtensorMap (types only; the encoder is fetched through the runtime, libcuda is not linked)
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
@@ -161,13 +162,18 @@ int cuda_fail(cudaError_t e, const char *what);
 
 // The opt-in shared-memory size of a kernel is a per-device attribute: launchers keep one flag per device ordinal.
 struct PerDeviceOnce {
-    bool done[64] = {};
-    bool need() {   // true the first time on the current device
+    std::atomic<bool> done[64] = {};
+    // true until done() has been called on the current device.  Two host threads (two contexts) may both see true
+    // and both run the one-time step, which is harmless for what it guards (setting a kernel attribute); neither
+    // launches before the step has been done.
+    bool need(int *dev_out) {
         int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
-        if (done[dev]) return false;
-        done[dev] = true;
-        return true;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = -1;
+        *dev_out = dev;
+        return dev < 0 || !done[dev].load(std::memory_order_acquire);
+    }
+    void mark(int dev) {
+        if (dev >= 0) done[dev].store(true, std::memory_order_release);
     }
 };
 

@@ -622,8 +622,10 @@ template <int D, int G, int NBLK>
 static int launch_k3(const k3::Params &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
     using C = k3::Cfg<D, NBLK>;
     static PerDeviceOnce configured;
-    if (configured.need()) {
+    int once_dev;
+    if (configured.need(&once_dev)) {
         MATKV_CUDA(cudaFuncSetAttribute(k3::k_prefill_tc<D, G, NBLK>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        configured.mark(once_dev);
     }
     k3::k_prefill_tc<D, G, NBLK><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());

@@ -318,3 +318,27 @@ def test_context_and_table_churn_leaves_no_device_memory_behind():
     torch.cuda.synchronize()
     free1, _ = torch.cuda.mem_get_info()
     assert free0 - free1 < 8 << 20, f"{(free0 - free1) / 2**20:.1f} MiB of device memory did not come back"
+
+
+def test_two_host_threads_with_a_context_each():
+    """Contexts are independent: two host threads, each with a context, tables and launches of its own, run at the
+    same time (the binding releases the interpreter lock inside the library); every output of both is compared with
+    the oracle.  (Calls on ONE context from several threads must be serialised by the caller.)"""
+    import threading
+    from test_gpu_parity import run_requests
+    errors = []
+
+    def worker(seed, impl):
+        try:
+            for rep in range(3):
+                run_requests(2, 8, 2, 128, [[130, 64], [200]], 40, 3, seed=seed + rep, prefill_impl=impl, all_layers=bool(rep & 1))
+                run_requests(1, 8, 4, 64, [[0, 1], [1]], 3, 2, seed=seed + 10 + rep, pool=[70, 33], decode_impl=2)
+        except BaseException as e:   # noqa: BLE001 - reported by the main thread
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(700, 2)), threading.Thread(target=worker, args=(800, 0))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
