@@ -182,6 +182,7 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_blk = ceil_div(p.S, C::TPU);
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next launch may be set up under this one
     if (tid == 0) {
         for (int s = 0; s < C::NSTAGE; ++s) {
             mbar_init(smem_u32(bars + s), 1);
@@ -194,8 +195,11 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     // short launches are chains of latencies: the range lookup (dependent loads of the table) runs in another warp beside
-    // the barrier set-up
+    // the barrier set-up.  Everything from here on may read what the previous kernel on the stream wrote (tail lengths,
+    // tail rows, the call's q / k / v, the workspace): wait for it to have completed.
+    if (tid != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 32) locate_range(p, *range, n_blk);
+    if (tid == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
     const int64_t f_begin = range->begin, f_end = range->end, W = range->W;
     // the fused tail advance: the last CTA of the launch to get here moves every request's tail length
@@ -632,8 +636,21 @@ static int launch_stream_t(const StreamParams &p, const CUtensorMap &kn_map, con
         MATKV_CUDA(cudaFuncSetAttribute(k_attend_stream<D, G, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
         configured.mark(once_dev);
     }
-    k_attend_stream<D, G, F8><<<grid, kThreads, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
-    MATKV_CUDA(cudaGetLastError());
+    // Programmatic dependent launch: when the kernel before this one on the stream lets its dependents go early (this
+    // kernel does, first thing), the launch itself and this kernel's barrier set-up run under that kernel's tail; the
+    // kernel waits for the predecessor's completion (griddepcontrol.wait) before it reads anything a predecessor may
+    // have written.  With any other predecessor the attribute changes nothing.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)kThreads);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    MATKV_CUDA(cudaLaunchKernelEx(&cfg, k_attend_stream<D, G, F8>, p, kn_map, vn_map));
     return MATKV_OK;
 }
 
