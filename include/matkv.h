@@ -195,7 +195,14 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
  * matkv_stage_chunks_async into them waits for it) and frees the table stream-ordered.        */
 int matkv_table_free(matkv_table *table, void *stream);
 /* Adds n_tokens to every request's tail length (device-side counter, so a captured decode
- * loop can replay it).  Attend calls never move it: all layers of one step see one length.    */
+ * loop can replay it).  Attend calls never move it: all layers of one step see one length.
+ * The library also keeps a host-side copy of the length, moved by these two calls (and by a
+ * decode launch that advances the tail itself) when they are made, not when a captured graph
+ * is replayed.  Attend calls outside stream capture split their work by the host-side copy
+ * (they can then start before the previous kernel on the stream has finished) and compare it
+ * with the device counter: after replaying a captured loop, call matkv_table_set_tail_len
+ * before the next attend call outside a capture, or that launch reports MATKV_E_BOUNDS in
+ * the device status and its output is void.                                                 */
 int matkv_table_advance(matkv_table *table, int32_t n_tokens, void *stream);
 int matkv_table_set_tail_len(matkv_table *table, int32_t tail_len, void *stream);
 

@@ -43,6 +43,11 @@ struct StreamParams {
     int32_t advance;      // > 0: the last CTA to finish adds this to every request's tail length
     int32_t *done_count;  // CTAs of the launch that have finished (reset by the last one)
     int32_t stream_hint;  // 1: no chunk of the table is listed twice, load chunk tiles with the evict-first L2 policy
+    // >= 0: every request's tail length as the host knows it.  The work split is then computed from it, BEFORE the
+    // kernel waits for its predecessor on the stream, and the producer pulls its first chunk tiles (immutable data)
+    // into the ring under the predecessor's tail; the device counter is compared with it after the wait
+    // (MATKV_E_BOUNDS in the status word if they differ).  -1: read the device counter (after the wait).
+    int32_t tail_hint;
 };
 
 // ---- the flat work list ----------------------------------------------------------------------------
@@ -61,7 +66,7 @@ struct CtaRange {
 };
 
 __device__ __forceinline__ int32_t clamp_t0(const StreamParams &p, int b) {
-    int32_t t0 = p.tail_len[b];
+    int32_t t0 = p.tail_hint >= 0 ? p.tail_hint : p.tail_len[b];
     if (t0 < 0 || t0 + p.S > p.max_tail) {
         atomicCAS(p.status, 0, MATKV_E_CAPACITY);
         t0 = max(0, min(t0, p.max_tail - p.S));
@@ -197,10 +202,19 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
     // short launches are chains of latencies: the range lookup (dependent loads of the table) runs in another warp beside
     // the barrier set-up.  Everything from here on may read what the previous kernel on the stream wrote (tail lengths,
     // tail rows, the call's q / k / v, the workspace): wait for it to have completed.
-    if (tid != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+    // With the host's tail length at hand the split is located first and only the threads that touch such data wait
+    // (the producer thread goes ahead with chunk tiles, see there).
+    const bool early = p.tail_hint >= 0;
+    if (!early && tid != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 32) locate_range(p, *range, n_blk);
-    if (tid == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!early && tid == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
+    if (early && !(warp == kCW && lane == 0)) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (blockIdx.x == 0)   // the host's tail length must be the device's: a launch split by a stale value is void
+            for (int b = tid; b < p.B; b += kThreads)
+                if (p.tail_len[b] != p.tail_hint) atomicCAS(p.status, 0, MATKV_E_BOUNDS);
+    }
     const int64_t f_begin = range->begin, f_end = range->end, W = range->W;
     // the fused tail advance: the last CTA of the launch to get here moves every request's tail length
     auto finish_cta = [&]() {
@@ -235,10 +249,15 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
         int64_t f = f_begin;
         uint32_t seq = 0;
         bool ok = true;
+        bool waited = !early;   // chunk tiles are immutable: they may be fetched before the predecessor kernel is done
         while (f < f_end && ok) {
             const int t_end = (int)min((int64_t)u.rt, f_end - u.flat_begin);
             const int layer = p.layer0 + u.l_rel;
             for (int t = u.tile; t < t_end; ++t, ++f, ++seq) {
+                if (!waited && t >= u.chunk_tiles) {   // tail rows and the call's new tokens: written by earlier kernels
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                    waited = true;
+                }
                 const uint32_t stage = seq % C::NSTAGE, use = seq / C::NSTAGE;
                 if (use > 0 && !mbar_wait(empty_u32 + stage * 8, (use - 1) & 1, flags)) {
                     ok = false;
@@ -525,7 +544,8 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                 }
                 }
                 // ---------- the unit's own new tokens go to the tail for later calls ----------
-                if (is_new) {
+                // (not when the launch was split by a stale tail length: it is void and must leave the tail alone)
+                if (is_new && !(early && p.tail_len[u.b] != p.tail_hint)) {
                     constexpr int CPR = D / 8;  // 16-byte chunks per row; lanes 0..CPR-1 move K, the next CPR lanes move V
                     const unsigned char *ring_stage = ring + stage * C::STAGE_BYTES;
                     for (int r = max(0, tok0 - new0); r < rows; ++r) {
@@ -682,6 +702,10 @@ int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
     p.advance = a.advance;
     p.done_count = ctx->d_status + 2;
     p.stream_hint = t->distinct_chunk_tiles == t->total_chunk_tiles && n_blk == 1;  // several token blocks re-read the tiles
+    {   // the host's mirror of the tail length is exact unless the stream is being captured (replays do not move it)
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        p.tail_hint = (cudaStreamIsCapturing(stream, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) ? t->tail_len_host : -1;
+    }
     const int64_t n_units = (int64_t)a.n_layers_launch * t->batch * n_blk * c.n_kv_heads;
     if (n_units > ws.n_counter_slots)
         return fail(MATKV_E_CAPACITY, "launch of %lld units exceeds the workspace's %lld", (long long)n_units,
@@ -806,6 +830,7 @@ extern "C" int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *t, int32_
         p.advance = 0;
         p.done_count = ctx->d_status + 2;
         p.stream_hint = t->distinct_chunk_tiles == t->total_chunk_tiles;
+        p.tail_hint = -1;
         CUtensorMap kn_map, vn_map;
         rc = encode_new_rows_map(&kn_map, k_new, c.head_dim, c.n_kv_heads, (uint64_t)t->batch);
         if (!rc) rc = encode_new_rows_map(&vn_map, v_new, c.head_dim, c.n_kv_heads, (uint64_t)t->batch);

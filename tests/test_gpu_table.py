@@ -342,3 +342,50 @@ def test_two_host_threads_with_a_context_each():
     for t in threads:
         t.join()
     assert not errors, errors
+
+
+def test_attend_after_graph_replays_needs_the_tail_length_set_again():
+    """A captured decode step advances the device-side tail counter every time it is replayed, but the host-side copy
+    only when it was captured.  An attend call outside a capture splits its work by the host-side copy and checks it
+    against the device counter: after replays it reports MATKV_E_BOUNDS in the device status unless the tail length
+    has been set again; after matkv_table_set_tail_len the same call is right (compared with the oracle)."""
+    import oracle
+    from _util import check
+    mk, Session, bits_to_dev, dev_to_bits = _mk()
+    L, Hq, Hkv, D, B = 1, 8, 2, 128, 1
+    blob = rand_bits(95, 0, (L, 2, Hkv, 150, D))
+    sess = Session(L, Hq, Hkv, D, B, 1, 16)
+    sess.register_device_chunk(0, bits_to_dev(blob))
+    sess.build_table([[0]])
+    qs = [rand_bits(95, 10 + i, (B, Hq, D)) for i in range(4)]
+    ks = [rand_bits(95, 20 + i, (B, Hkv, D)) for i in range(4)]
+    g_q, g_k = bits_to_dev(qs[0]).clone(), bits_to_dev(ks[0]).clone()
+    g_o = torch.empty_like(g_q)
+    stream = torch.cuda.Stream()
+    sp = stream.cuda_stream
+    with torch.cuda.stream(stream):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            mk.matkv_attend_decode(sess.ctx, sess.table, 0, g_q.data_ptr(), g_k.data_ptr(), g_k.data_ptr(), g_o.data_ptr(), None, sp)
+            mk.matkv_table_advance(sess.table, 1, sp)
+        mk.matkv_table_set_tail_len(sess.table, 0, sp)          # the capture moved the host-side copy only
+        for i in range(3):                                      # three replayed steps: the device counter is at 3
+            g_q.copy_(bits_to_dev(qs[i])); g_k.copy_(bits_to_dev(ks[i]))
+            graph.replay()
+        q3, k3 = bits_to_dev(qs[3]), bits_to_dev(ks[3])
+        out = torch.empty_like(q3)
+        mk.matkv_attend_decode(sess.ctx, sess.table, 0, q3.data_ptr(), k3.data_ptr(), k3.data_ptr(), out.data_ptr(), None, sp)
+        stream.synchronize()
+        assert sess.status(clear=True) == mk.E_BOUNDS
+        mk.matkv_table_set_tail_len(sess.table, 3, sp)
+        lse = torch.empty((B, Hq), dtype=torch.float32, device="cuda")
+        mk.matkv_attend_decode(sess.ctx, sess.table, 0, q3.data_ptr(), k3.data_ptr(), k3.data_ptr(), out.data_ptr(), lse.data_ptr(), sp)
+        stream.synchronize()
+    assert sess.status() == 0
+    req = oracle.Request(oracle.Shape(L, Hq, Hkv, D), [blob], 16)
+    for i in range(3):
+        req.append_only(0, ks[i][0][None], ks[i][0][None])
+        req.advance(1)
+    o_ref, l_ref = req.attend_new(0, qs[3][0][None], ks[3][0][None], ks[3][0][None])
+    check(dev_to_bits(out)[0], o_ref[0], lse.cpu().numpy()[0], l_ref[0], "decode after replays, tail length set again")
+    sess.close()
