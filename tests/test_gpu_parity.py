@@ -160,6 +160,64 @@ def test_decode_launch_that_advances_the_tail_itself(ctas):
     run_requests(2, 8, 2, 128, [[200, 31], [97], []], 3, 5, seed=28, all_layers=True, fused_advance=True, ctas=ctas)
 
 
+@pytest.mark.parametrize("decode_impl,L,lens", [(1, 2, [[130, 64], [200], [64]]), (1, 32, [[1024, 1024, 512]]), (2, 2, [[130, 64], [200], [64]])])
+def test_back_to_back_decode_launches_across_a_tail_tile_boundary(decode_impl, L, lens):
+    """Twelve decode steps issued back to back WITHOUT a host synchronisation in between, every launch advancing the
+    tail itself, while the tail grows from 58 to 70 tokens (a second tail tile appears at 64): each launch is split
+    by the host's copy of the tail length and starts under its predecessor's tail (its producer already fetching
+    chunk tiles), and each step's appended row must be there for the next.  All outputs are compared afterwards."""
+    import paper_2512_22195_b200 as mk
+    Hq, Hkv, D, S, T, seed = 8, 2, 128, 58, 12, 29
+    B = len(lens)
+    sess = _session(L, Hq, Hkv, D, B, max(len(x) for x in lens), S + T)
+    mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, decode_impl)
+    mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_ADVANCES_TAIL, 1)
+    sh = oracle.Shape(L, Hq, Hkv, D)
+    reqs, ids, cid = [], [], 0
+    for row in lens:
+        blobs, mine = [], []
+        for n in row:
+            bl = rand_bits(seed, 100 + cid, (L, 2, Hkv, n, D))
+            sess.register_device_chunk(cid, _dev(bl))
+            blobs.append(bl); mine.append(cid); cid += 1
+        reqs.append(oracle.Request(sh, blobs, S + T)); ids.append(mine)
+    sess.build_table(ids)
+    q = rand_bits(seed, 1, (L, B, S, Hq, D)); k = rand_bits(seed, 2, (L, B, S, Hkv, D)); v = rand_bits(seed, 3, (L, B, S, Hkv, D))
+    sess.prefill_all_layers(_dev(q), _dev(k), _dev(v), want_lse=False)
+    for layer in range(L):
+        for r in range(B):
+            reqs[r].append_only(layer, k[layer, r], v[layer, r])
+    sess.advance(S)
+    for r in reqs:
+        r.advance(S)
+    qs = [rand_bits(seed, 2000 + t, (L, B, Hq, D)) for t in range(T)]
+    ks = [rand_bits(seed, 3000 + t, (L, B, Hkv, D)) for t in range(T)]
+    vs = [rand_bits(seed, 4000 + t, (L, B, Hkv, D)) for t in range(T)]
+    dq, dk, dv = [_dev(x) for x in qs], [_dev(x) for x in ks], [_dev(x) for x in vs]
+    torch.cuda.synchronize()
+    outs = [sess.decode_all_layers(dq[t], dk[t], dv[t]) for t in range(T)]      # nothing in between: the launches queue up
+    torch.cuda.synchronize()
+    assert sess.status() == 0
+    sample_layers = sorted({0, L // 2, L - 1})
+    for t in range(T):
+        ob, lb = _bits(outs[t][0]), outs[t][1].cpu().numpy()
+        for layer in range(L):
+            for r in range(B):
+                if layer in sample_layers:
+                    o_ref, l_ref = reqs[r].attend_new(layer, qs[t][layer, r][None], ks[t][layer, r][None], vs[t][layer, r][None])
+                    check(ob[layer, r], o_ref[0], lb[layer, r], l_ref[0], f"step {t} layer {layer} request {r}")
+                else:
+                    reqs[r].append_only(layer, ks[t][layer, r][None], vs[t][layer, r][None])
+        for r in reqs:
+            r.advance(1)
+    tk, tv = _bits(sess.tail_k), _bits(sess.tail_v)
+    for r in range(B):
+        n = reqs[r].tail_len
+        assert n == S + T
+        assert np.array_equal(tk[r, :, :, :n], reqs[r].tail_k[:, :, :n]) and np.array_equal(tv[r, :, :, :n], reqs[r].tail_v[:, :, :n])
+    sess.close()
+
+
 def test_peaky_queries():
     run_requests(1, 8, 2, 128, [[300, 300]], 8, 4, seed=25, q_shift=3)   # q scaled by 8: sharp softmax
 
