@@ -122,7 +122,10 @@ int matkv_status(matkv_ctx *ctx, int32_t *dev_status_out, int32_t clear);
 /* ---- a1: chunk registry (the paper's "file named chunk_id"; Section IV, store_KV) ------- */
 /* Records where the materialised K,V of `chunk_id` live.  host_blob: pinned (or pageable)
  * host memory or NULL; dev_blob: device memory or NULL; at least one non-NULL.  Both are
- * borrowed until matkv_unregister_chunk / matkv_destroy.  Re-registering an id is an error. */
+ * borrowed until matkv_unregister_chunk / matkv_destroy.  Re-registering an id is an error.
+ * A chunk is immutable (the method's premise): the device copy a table points at must not be
+ * written while the table is in use, not even by earlier work on the same stream, because an
+ * attend launch may fetch chunk rows before the kernel queued before it has finished.        */
 int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, const void *host_blob,
                          void *dev_blob);
 /* The same for a chunk whose blob is stored in a file, `blob bytes` long at file_offset: the paper's
