@@ -887,15 +887,16 @@ def main():
             load(0)
             state["table"] = sess2.build_table(ids, sp)
             load(1)
-            for i in range(2):
+            w_e2e = max(3, min(args.warmup, 5))
+            for i in range(w_e2e):
                 e2e_step(i)
             drain_copies()
             k_e2e = min(args.steps, 5)
-            ms_e, _, _, _ = timed_region(lambda i: e2e_step(i + 2, last=(i == k_e2e - 1)), k_e2e)
+            ms_e, _, _, _ = timed_region(lambda i: e2e_step(i + w_e2e, last=(i == k_e2e - 1)), k_e2e)
         if sess2.status() != 0:
             raise RuntimeError("device status non-zero after the end-to-end region")
         result["e2e"] = {"value": tokens * k_e2e / (ms_e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e,
+                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e, "warmup": w_e2e,
                          "overlap": "the chunks and query-side inputs of the next two steps copied in (three slot regions), and the previous "
                                     "step's outputs copied out, on side streams under this step's prefill and decode",
                          "staging": (f"copy kernel, {e2e_stage_ctas} CTAs" if e2e_stage_ctas > 0 else "copy engine") + f", {n_copy} copy streams",
