@@ -253,7 +253,6 @@ def run_pipeline(args):
     torch.cuda.synchronize()
     del tmp8
     del tmp
-    slots = [torch.empty(n_slots * slot_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
     q_pf = torch.empty((L, B, S, Hq, D), dtype=torch.bfloat16, device=dev)
     k_pf = torch.empty((L, B, S, Hkv, D), dtype=torch.bfloat16, device=dev)
     v_pf = torch.empty_like(k_pf)
@@ -266,21 +265,16 @@ def run_pipeline(args):
     o_pf, o_dc = torch.empty_like(q_pf), torch.empty_like(q_dc)
     ho_dc = torch.empty(o_dc.shape, dtype=torch.bfloat16, pin_memory=True)
     stream, copy = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-    sp, ctx = stream.cuda_stream, sess.ctx
-    qs_l, ks_l, qd_t, kd_t = q_pf[0].numel() * 2, k_pf[0].numel() * 2, q_dc[0].numel() * 2, k_dc[0].numel() * 2
+    ctx = sess.ctx
+    from paper_2512_22195_b200.pipeline import PipelinedBatches
+    pipe = PipelinedBatches(sess, n_slots, slot_bytes, stream, copy)     # two slot regions; the tests run this same class
     torch.cuda.synchronize()
 
     def stage(n):
-        return sess.stage(needed[n], slots[n % 2], slot_bytes, copy)
+        return pipe.stage(n, needed[n])
 
-    def compute(n):
-        table = sess.build_table(batches[n], sp)
-        mk.matkv_attend_prefill_all_layers(ctx, table, S, q_pf.data_ptr(), k_pf.data_ptr(), v_pf.data_ptr(), o_pf.data_ptr(), None, sp)
-        mk.matkv_table_advance(table, S, sp)
-        for t in range(T):
-            mk.matkv_attend_decode_all_layers(ctx, table, q_dc.data_ptr() + t * qd_t, k_dc.data_ptr() + t * kd_t,
-                                              v_dc.data_ptr() + t * kd_t, o_dc.data_ptr() + t * qd_t, None, sp)
-            mk.matkv_table_advance(table, 1, sp)
+    def compute(n, stage_next=None):
+        pipe.compute(n, batches[n], S, T, q_pf, k_pf, v_pf, o_pf, q_dc, k_dc, v_dc, o_dc, stage_next=stage_next)
         with torch.cuda.stream(stream):
             ho_dc.copy_(o_dc, non_blocking=True)
 
@@ -304,21 +298,8 @@ def run_pipeline(args):
 
     def pipelined():
         stage(0)
-        for n in range(n_batches):
-            compute_with_stage(n)   # builds table n (resolves its slots), then sends batch n+1 to the other region
-
-    def compute_with_stage(n):
-        table = sess.build_table(batches[n], sp)
-        if n + 1 < n_batches:
-            stage(n + 1)
-        mk.matkv_attend_prefill_all_layers(ctx, table, S, q_pf.data_ptr(), k_pf.data_ptr(), v_pf.data_ptr(), o_pf.data_ptr(), None, sp)
-        mk.matkv_table_advance(table, S, sp)
-        for t in range(T):
-            mk.matkv_attend_decode_all_layers(ctx, table, q_dc.data_ptr() + t * qd_t, k_dc.data_ptr() + t * kd_t,
-                                              v_dc.data_ptr() + t * kd_t, o_dc.data_ptr() + t * qd_t, None, sp)
-            mk.matkv_table_advance(table, 1, sp)
-        with torch.cuda.stream(stream):
-            ho_dc.copy_(o_dc, non_blocking=True)
+        for n in range(n_batches):   # table n is built (its slots resolved), then batch n+1 goes to the other region
+            compute(n, stage_next=needed[n + 1] if n + 1 < n_batches else None)
 
     # warm-up: two batches through the whole path
     stage(0); compute(0); stage(1); compute(1)

@@ -2,7 +2,7 @@
  * matkv.h -- C ABI of the B200 (sm_100a) attention path that remains on the GPU
  * in MatKV-style retrieval-augmented inference.
  *
- * Method (paper, Section III-A and Section IV): the K,V tensors of every
+ * Method (paper, Section III-B and Section IV): the K,V tensors of every
  * document chunk are computed once, each chunk alone with its tokens at
  * positions 0..len-1, stored under a chunk id, and at request time loaded
  * instead of recomputed and placed BEFORE the query.  Only the query suffix
@@ -72,7 +72,11 @@ typedef struct {
     int32_t pos_mode;            /* rotary mode only: position of the first tail token.
                                     0 = sum of the request's chunk lengths (the query continues
                                     after the documents, each of which starts at position 0);
-                                    1 = longest chunk length.  Inert when rope_theta == 0.     */
+                                    1 = longest chunk length; 2 = given per request with
+                                    matkv_table_set_pos_base (until then as mode 0).  The paper
+                                    fixes the documents' positions (each starts at the first input
+                                    position, Section III-B) and is silent on the query's, hence a
+                                    parameter.  Inert when rope_theta == 0.                      */
     int32_t device;              /* CUDA device ordinal, -1 = current device                */
 } matkv_config;
 
@@ -99,6 +103,10 @@ typedef struct {
                                       decode; sub-prefill over such chunks also runs on the streaming kernel, and the chunk-major
                                       decode, the allocation-free decode and matkv_gather_debug refuse tables that hold them */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
+#define MATKV_OPT_IO_TIMEOUT_MS 9  /* storage tier: how long the copy stream waits for one chunk's read before the staging call
+                                      is marked failed (MATKV_E_IO) and the stream moves on; default 30,000 ms */
+#define MATKV_OPT_IO_TEST_DELAY_MS 10 /* failure injection on the host, for tests: every storage read sleeps this long first
+                                         (0 = off); with a time limit below it the reads "hang" without any GPU fault */
 
 /* ---- context -------------------------------------------------------------------------- */
 /* Creates a context on cfg->device.  Allocates the device status word and nothing large.   */
@@ -121,7 +129,8 @@ int matkv_status(matkv_ctx *ctx, int32_t *dev_status_out, int32_t clear);
 
 /* ---- a1: chunk registry (the paper's "file named chunk_id"; Section IV, store_KV) ------- */
 /* Records where the materialised K,V of `chunk_id` live.  host_blob: pinned (or pageable)
- * host memory or NULL; dev_blob: device memory or NULL; at least one non-NULL.  Both are
+ * host memory or NULL (a pageable blob is always staged by the copy engine, whatever
+ * MATKV_OPT_STAGE_CTAS says: only page-locked memory can be read by the copy kernel); dev_blob: device memory or NULL; at least one non-NULL.  Both are
  * borrowed until matkv_unregister_chunk / matkv_destroy.  Re-registering an id is an error.
  * A chunk is immutable (the method's premise): the device copy a table points at must not be
  * written while the table is in use, not even by earlier work on the same stream, because an
@@ -169,7 +178,7 @@ int matkv_register_chunk_file_fp8(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_t
 int matkv_unregister_chunk(matkv_ctx *ctx, uint64_t chunk_id);
 
 /* ---- a2: staging (the paper's load_KV, CPU bounce buffer -> GPU; Section IV, and the
- *      overlap of the next batch's load with the current decode, Section III-B) ------------ */
+ *      overlap of the next batch's load with the current decode, Section III-C) ------------ */
 /* Copies the listed chunks' host blobs into `dev_slots` (n_slots slots of slot_bytes each,
  * device memory, 256-byte aligned, borrowed) with one asynchronous copy per chunk on
  * `copy_stream`, and records an event per call.  Duplicates in the list, chunks registered
@@ -183,10 +192,19 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *chunk_ids, int32_t 
 int matkv_stage_query(matkv_ctx *ctx, uint64_t ticket);
 /* Blocks the calling host thread until the ticket's copies have finished.                     */
 int matkv_stage_wait(matkv_ctx *ctx, uint64_t ticket);
+/* Both return MATKV_E_IO when a storage read of that call failed or did not return within the
+ * time limit (the slots of its chunks then hold garbage): a later matkv_build_chunk_table over
+ * such a chunk is refused with MATKV_E_IO once the failure is known, and the device status
+ * word reads MATKV_E_IO as soon as the copy stream has passed the call, so that attention
+ * launched behind it without any host wait is flagged too.  A ticket that has been seen
+ * complete (by these calls, or by a later staging call) is retired: its event is destroyed
+ * and it keeps answering MATKV_OK / MATKV_E_IO.
+ * matkv_stage_pending: number of staging calls not yet seen complete.                         */
+int matkv_stage_pending(matkv_ctx *ctx, int32_t *n_out);
 
 /* ---- a3: chunk table (replaces the concatenation of put_KV, Section IV) ------------------ */
 /* chunk_ids_flat is the concatenation of each request's ORDERED id list (documents before
- * the query, Section III-A); n_chunks_per_req[r] may be 0 and ids may repeat.  tail_k / tail_v:
+ * the query, Section III-B); n_chunks_per_req[r] may be 0 and ids may repeat.  tail_k / tail_v:
  * device tails (layout above, batch = `batch`), borrowed, written by the attend calls.
  * Resolves every id to its device copy (MATKV_E_NOT_STAGED if it has none), makes `stream`
  * wait for the staging copies it depends on (never the host), uploads the table on `stream`
@@ -208,6 +226,11 @@ int matkv_table_free(matkv_table *table, void *stream);
  * the device status and its output is void.                                                 */
 int matkv_table_advance(matkv_table *table, int32_t n_tokens, void *stream);
 int matkv_table_set_tail_len(matkv_table *table, int32_t tail_len, void *stream);
+/* pos_mode 2 only: sets, on `stream`, the position of the first tail token of every request
+ * (pos_base: host array of `batch` non-negative values, read before the call returns).  Tail
+ * token i of request r is then rotated at pos_base[r] + i.  Call it before the first attend
+ * call of the table.                                                                          */
+int matkv_table_set_pos_base(matkv_table *table, const int32_t *pos_base, void *stream);
 
 /* ---- a4: query sub-prefill (Section V-A "Prefill time": from the end of loading to the
  *      first token; the query is prefilled on top of the loaded KVs) ----------------------- */
@@ -245,7 +268,9 @@ int matkv_attend_decode_all_layers(matkv_ctx *ctx, matkv_table *table, const voi
  *   - The split-KV partials and arrival counters live in an array built into the library
  *     (2,114,560 bytes of device memory per GPU that loads it, held until the process exits) instead
  *     of the workspace given to matkv_set_workspace, which this call neither needs nor touches.
- *   - Limit: batch x n_kv_heads <= 256 and head_dim <= 128; larger calls return MATKV_E_CAPACITY.
+ *   - Limits: batch x n_kv_heads <= 256 and head_dim <= 128; larger calls return MATKV_E_CAPACITY.  Two kinds of
+ *     call are refused with MATKV_E_INVALID_ARG: a context in rotary mode (rope_theta != 0: the rotated q / k_new
+ *     would need scratch of their own) and a table that holds compressed-resident chunks.
  *   - Nothing is allocated or freed: no cudaMalloc / cudaFree and no allocating library routine.  The
  *     first call on a device looks up the array's device address (cudaGetSymbolAddress); make that
  *     first call outside any stream capture.
@@ -256,7 +281,7 @@ int matkv_attend_decode_static(matkv_ctx *ctx, matkv_table *table, int32_t layer
                                const void *v_new, void *out, float *lse_out, void *stream);
 
 /* Chunk-major decode for batches whose requests share chunks (the paper's skewed retrieval: a few
- * materialised chunks take most of the hits, Section V).  matkv_attend_decode and
+ * materialised chunks take most of the hits, Section II-C).  matkv_attend_decode and
  * matkv_attend_decode_all_layers then read a chunk listed by several requests of the table ONCE per
  * layer and KV head: the requests' query heads are stacked into one tensor-core tile (16 / G requests;
  * more requests repeat the read right away, where it hits L2), every (chunk, request) pair leaves a

@@ -6,7 +6,7 @@ smoke check and the benchmark's CPU-baseline / reference legs may import this
 package; the CUDA library and its Python binding never do, and nothing here
 imports them.
 
-Semantics (paper, Section III-A and Section IV): the materialised chunks sit
+Semantics (paper, Section III-B and Section IV): the materialised chunks sit
 before the query, all of their tokens are visible, their K is used verbatim
 (each chunk was computed with its tokens at positions 0..len-1), and the query
 suffix and generated tokens form an ordinary causal continuation.

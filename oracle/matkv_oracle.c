@@ -6,7 +6,7 @@
  * called only from the tests, the smoke check and the benchmark's CPU-baseline
  * leg.
  *
- * What is computed (paper, Section III-A "Materializing and Retrieving KV
+ * What is computed (paper, Section III-B "Materializing and Retrieving KV
  * Caches" and Section IV "Avoiding Prefill Using KV in SSD"): the precomputed
  * K,V of the retrieved document chunks are placed BEFORE the query, each chunk
  * having been materialised alone with its tokens at positions 0..len-1, and

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(HERE, "libmatkv.so")
 OK, E_INVALID_ARG, E_UNKNOWN_CHUNK, E_NOT_STAGED, E_NOT_READY = 0, -1, -2, -3, -4
 E_CAPACITY, E_ALIGNMENT, E_CUDA, E_TIMEOUT, E_BOUNDS, E_IO = -5, -6, -7, -8, -9, -10
 OPT_DECODE_CTAS, OPT_PREFILL_IMPL, OPT_PREFILL_CTAS, OPT_STAGE_CTAS, OPT_DECODE_ADVANCES_TAIL = 1, 2, 3, 4, 5
-OPT_DECODE_IMPL, OPT_SHARE_TILES, OPT_FP8_RESIDENT = 6, 7, 8
+OPT_DECODE_IMPL, OPT_SHARE_TILES, OPT_FP8_RESIDENT, OPT_IO_TIMEOUT_MS, OPT_IO_TEST_DELAY_MS = 6, 7, 8, 9, 10
 
 EXPORTS = [
     "matkv_create", "matkv_destroy", "matkv_last_error", "matkv_set_option", "matkv_workspace_bytes",
@@ -29,6 +29,7 @@ EXPORTS = [
     "matkv_register_chunk_file", "matkv_set_bounce_buffer", "matkv_export_tail_as_chunk",
     "matkv_attend_prefill_all_layers", "matkv_table_sharing", "matkv_table_workspace_bytes",
     "matkv_fp8_blob_bytes", "matkv_fp8_resident_bytes", "matkv_quantize_chunk_fp8", "matkv_register_chunk_fp8", "matkv_register_chunk_file_fp8",
+    "matkv_table_set_pos_base", "matkv_stage_pending",
 ]
 
 
@@ -74,6 +75,8 @@ def lib() -> C.CDLL:
             "matkv_table_free": (C.c_int, [vp, vp]),
             "matkv_table_advance": (C.c_int, [vp, i32, vp]),
             "matkv_table_set_tail_len": (C.c_int, [vp, i32, vp]),
+            "matkv_table_set_pos_base": (C.c_int, [vp, C.POINTER(i32), vp]),
+            "matkv_stage_pending": (C.c_int, [vp, C.POINTER(i32)]),
             "matkv_attend_prefill": (C.c_int, [vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]),
             "matkv_attend_decode": (C.c_int, [vp, vp, i32, vp, vp, vp, vp, vp, vp]),
             "matkv_attend_decode_all_layers": (C.c_int, [vp, vp, vp, vp, vp, vp, vp, vp]),
@@ -285,3 +288,16 @@ def matkv_register_chunk_fp8(ctx: int, chunk_id: int, n_tokens: int, host_blob_f
 
 def matkv_register_chunk_file_fp8(ctx: int, chunk_id: int, n_tokens: int, path: str, file_offset: int = 0) -> None:
     _check(lib().matkv_register_chunk_file_fp8(ctx, chunk_id, n_tokens, path.encode(), file_offset))
+
+
+def matkv_table_set_pos_base(table: int, pos_base: Sequence[int], stream: int = 0) -> None:
+    """pos_mode 2: position of the first tail token of every request (one value per request of the table)."""
+    arr = (C.c_int32 * max(len(pos_base), 1))(*pos_base)
+    _check(lib().matkv_table_set_pos_base(table, arr, stream or None))
+
+
+def matkv_stage_pending(ctx: int) -> int:
+    """Staging calls not yet seen complete."""
+    n = C.c_int32(0)
+    _check(lib().matkv_stage_pending(ctx, C.byref(n)))
+    return n.value

@@ -1,6 +1,6 @@
 // Chunk-major decode: the decode step (one new token per request) for batches whose requests list the
 // same chunks.  The paper observes that retrieval is skewed: a small share of the chunks takes most of
-// the hits (Section III-B / V: re-use of materialised KVs across requests).  A request-major kernel
+// the hits (Section II-C, the access-skew figure: most chunks are retrieved by several queries).  A request-major kernel
 // reads a chunk once per request that lists it; here the work item is a CHUNK (up to `n_tiles` tiles of
 // it, one KV head, one layer) and the query rows of every request that lists it are stacked into the 16
 // rows of the MMA tile (16 / G requests), so the chunk's K and V rows cross HBM once for all of them.

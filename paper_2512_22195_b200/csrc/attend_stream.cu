@@ -606,8 +606,10 @@ k_attend_stream(const __grid_constant__ StreamParams p, const __grid_constant__ 
                 L = fmaf(sw, merge_l[w * kUnitRows + r], L);
                 Lr = fmaf(sw, merge_r[w * kUnitRows + r], Lr);
             }
-            const float ov = acc / Lr;
-            const float lse = (M + log2f(L)) * kLn2;
+            // a share that holds only tiles no row can see (new-token tiles past the block's last token) is an empty
+            // part: zero output, lse = -inf, never 0 / 0
+            const float ov = Lr > 0.f ? acc / Lr : 0.f;
+            const float lse = L > 0.f ? (M + log2f(L)) * kLn2 : -CUDART_INF_F;
             if (n_parts == 1) {
                 p.out[q_base + (int64_t)(r / G) * p.q_ss + (r % G) * D + d] = __float2bfloat16(ov);
                 if (p.lse_out && d == 0) p.lse_out[lse_base + (int64_t)(r / G) * p.lse_ss + (r % G)] = lse;

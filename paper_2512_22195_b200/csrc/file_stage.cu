@@ -5,11 +5,16 @@
 // for the chunk's read, the host-to-device copy out of the ring slab, and a callback that hands the
 // slab back to the readers.  So storage reads, PCIe copies and the GPU's attention kernels overlap
 // (three stages), and the staging call itself never blocks its caller.
+// Failures stay on the host side of the link and are reported, never waited on for ever: a read that fails
+// (or a file that turned out short) marks its staging call as failed; the callback's wait for a read has a
+// limit, after which the call is marked failed too and the stream moves on; either way the status word
+// reads MATKV_E_IO once the stream has passed the call, and table builds over such chunks are refused.
 #include <errno.h>
 #include <fcntl.h>
 #include <string.h>
 #include <unistd.h>
 
+#include <chrono>
 #include <condition_variable>
 #include <deque>
 #include <mutex>
@@ -25,6 +30,7 @@ struct IoJob {
     size_t bytes;
     int slab;
     uint64_t use;  // how many times the slab was used before this job
+    std::shared_ptr<std::atomic<int>> failed;  // the staging call's failure flag
 };
 
 struct IoEngine {
@@ -40,7 +46,21 @@ struct IoEngine {
     bool stop = false;
     int errors = 0;
     char last_error[256] = "";
+    int *h_flag = nullptr;   // page-locked word the device can read: non-zero once any read has failed
+    std::atomic<int64_t> timeout_ms{30000}, test_delay_ms{0};
 };
+
+// raises the device status word when the host has seen a read fail (launched behind a staging call's copies)
+__global__ void k_io_flag(const volatile int *host_flag, int32_t *status) {
+    if (*host_flag) atomicCAS(status, 0, MATKV_E_IO);
+}
+
+static void note_failure(IoEngine *e, const std::shared_ptr<std::atomic<int>> &failed, const char *msg) {  // e->m held
+    ++e->errors;
+    snprintf(e->last_error, sizeof e->last_error, "%s", msg);
+    if (failed) failed->store(1, std::memory_order_release);
+    if (e->h_flag) *(volatile int *)e->h_flag = 1;
+}
 
 static void io_worker(IoEngine *e) {
     for (;;) {
@@ -51,10 +71,13 @@ static void io_worker(IoEngine *e) {
             if (e->queue.empty()) return;  // stop requested and nothing left
             job = e->queue.front();
             e->queue.pop_front();
-            // the slab must have been handed back by the copy that used it last
-            e->cv.wait(lk, [&] { return e->stop || e->releases_done[job.slab] == job.use; });
-            if (e->stop && e->releases_done[job.slab] != job.use) return;
+            // the slab must have been handed back by the copy that used it last, and the read that filled it last must
+            // have returned (a read the stream gave up waiting for may still be writing into the slab)
+            auto slab_free = [&] { return e->releases_done[job.slab] == job.use && e->reads_done[job.slab] == job.use; };
+            e->cv.wait(lk, [&] { return e->stop || slab_free(); });
+            if (e->stop && !slab_free()) return;
         }
+        if (const int64_t d = e->test_delay_ms.load()) std::this_thread::sleep_for(std::chrono::milliseconds(d));  // failure injection
         char *dst = e->base + (size_t)job.slab * e->slab_bytes;
         size_t done = 0;
         int err = 0;
@@ -75,9 +98,10 @@ static void io_worker(IoEngine *e) {
         {
             std::lock_guard<std::mutex> lk(e->m);
             if (err) {
-                ++e->errors;
-                snprintf(e->last_error, sizeof e->last_error, "read of %zu bytes at offset %llu failed: %s", job.bytes,
-                         (unsigned long long)job.offset, strerror(err));
+                char msg[256];
+                snprintf(msg, sizeof msg, "read of %zu bytes at offset %llu failed: %s", job.bytes, (unsigned long long)job.offset,
+                         strerror(err));
+                note_failure(e, job.failed, msg);
             }
             e->reads_done[job.slab] = job.use + 1;
         }
@@ -89,13 +113,20 @@ struct IoCallback {
     IoEngine *e;
     int slab;
     uint64_t use;
+    std::shared_ptr<std::atomic<int>> failed;
 };
 
-static void CUDART_CB cb_wait_read(void *p) {  // runs in stream order before the copy out of the slab
+// Runs in stream order before the copy out of the slab.  The wait has a limit: a read that does not return
+// (a hung network file system) must not stall every later operation of the copy stream for ever.  When the
+// limit runs out the staging call is marked failed and the stream moves on (the copy then moves whatever the
+// slab holds; the failure flag is what tells the caller not to use it).
+static void CUDART_CB cb_wait_read(void *p) {
     IoCallback *c = (IoCallback *)p;
     {
         std::unique_lock<std::mutex> lk(c->e->m);
-        c->e->cv.wait(lk, [&] { return c->e->reads_done[c->slab] >= c->use + 1; });
+        const bool done = c->e->cv.wait_for(lk, std::chrono::milliseconds(std::max<int64_t>(1, c->e->timeout_ms.load())),
+                                            [&] { return c->e->reads_done[c->slab] >= c->use + 1; });
+        if (!done) note_failure(c->e, c->failed, "a storage read did not return within the time limit");
     }
     delete c;
 }
@@ -117,6 +148,17 @@ int io_engine_create(matkv_ctx *ctx, void *pinned, size_t bytes, size_t slab_byt
     e->n_slabs = (int)(bytes / slab_bytes);
     e->reads_done.assign(e->n_slabs, 0);
     e->releases_done.assign(e->n_slabs, 0);
+    e->timeout_ms = ctx->opt_io_timeout_ms;
+    e->test_delay_ms = ctx->opt_io_test_delay_ms;
+    {
+        DeviceGuard guard(ctx->device);
+        cudaError_t err = cudaHostAlloc((void **)&e->h_flag, 64, cudaHostAllocMapped | cudaHostAllocPortable);
+        if (err != cudaSuccess) {
+            delete e;
+            return cuda_fail(err, "cudaHostAlloc(read-failure flag)");
+        }
+        *e->h_flag = 0;
+    }
     for (int i = 0; i < n_threads; ++i) e->threads.emplace_back(io_worker, e);
     ctx->io = e;
     return MATKV_OK;
@@ -131,8 +173,22 @@ void io_engine_destroy(matkv_ctx *ctx) {
     }
     e->cv.notify_all();
     for (auto &t : e->threads) t.join();
+    if (e->h_flag) cudaFreeHost(e->h_flag);
     delete e;
     ctx->io = nullptr;
+}
+
+void io_engine_configure(matkv_ctx *ctx) {
+    if (!ctx->io) return;
+    ctx->io->timeout_ms = ctx->opt_io_timeout_ms;
+    ctx->io->test_delay_ms = ctx->opt_io_test_delay_ms;
+}
+
+int io_engine_flag_status(matkv_ctx *ctx, cudaStream_t copy_stream) {
+    if (!ctx->io || !ctx->io->h_flag) return MATKV_OK;
+    k_io_flag<<<1, 1, 0, copy_stream>>>(ctx->io->h_flag, ctx->d_status);
+    MATKV_CUDA(cudaGetLastError());
+    return MATKV_OK;
 }
 
 size_t io_engine_slab_bytes(const matkv_ctx *ctx) { return ctx->io ? ctx->io->slab_bytes : 0; }
@@ -144,8 +200,20 @@ int io_engine_errors(matkv_ctx *ctx, const char **msg) {
     return ctx->io->errors;
 }
 
+// Hands a slab back on the host after an enqueue failed half-way: waits (with the read limit) for the slab's read to
+// return, so that the next read into the slab cannot overlap it, then marks the slab released.
+static void release_on_host(IoEngine *e, int slab, uint64_t use) {
+    {
+        std::unique_lock<std::mutex> lk(e->m);
+        e->cv.wait_for(lk, std::chrono::milliseconds(std::max<int64_t>(1, e->timeout_ms.load())), [&] { return e->reads_done[slab] >= use + 1; });
+        e->releases_done[slab] = use + 1;
+    }
+    e->cv.notify_all();
+}
+
 // Enqueues: read (worker threads) -> [copy stream] wait for the read, copy slab -> dst, release the slab.
-int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream, int32_t fp8_tokens, bool fp8_resident) {
+int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream,
+                    const std::shared_ptr<std::atomic<int>> &failed, int32_t fp8_tokens, bool fp8_resident) {
     IoEngine *e = ctx->io;
     if (!e) return fail(MATKV_E_INVALID_ARG, "file-backed chunk: no bounce buffer set (matkv_set_bounce_buffer)");
     if (bytes > e->slab_bytes)
@@ -159,20 +227,35 @@ int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void 
         job.fd = fd;
         job.offset = offset;
         job.bytes = bytes;
+        job.failed = failed;
         e->queue.push_back(job);
     }
     e->cv.notify_all();
-    MATKV_CUDA(cudaLaunchHostFunc(copy_stream, cb_wait_read, new IoCallback{e, job.slab, job.use}));
-    if (fp8_tokens > 0) {  // compressed chunk: the expanding copy reads the slab over the link (it must be device-accessible pinned memory)
-        int rc = fp8_resident ? launch_stage_relayout_fp8(ctx, e->base + (size_t)job.slab * e->slab_bytes, dst, fp8_tokens, copy_stream)
-                              : launch_stage_expand_fp8(ctx, e->base + (size_t)job.slab * e->slab_bytes, dst, fp8_tokens,
-                                                        ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, copy_stream);
-        if (rc) return rc;
-    } else {
-        MATKV_CUDA(cudaMemcpyAsync(dst, e->base + (size_t)job.slab * e->slab_bytes, bytes, cudaMemcpyHostToDevice, copy_stream));
+    // from here on the slab is owed a release: by the stream's second callback, or on the host when enqueueing fails
+    IoCallback *cb = new IoCallback{e, job.slab, job.use, failed};
+    cudaError_t err = cudaLaunchHostFunc(copy_stream, cb_wait_read, cb);
+    if (err != cudaSuccess) {
+        delete cb;
+        release_on_host(e, job.slab, job.use);
+        return cuda_fail(err, "cudaLaunchHostFunc(wait for the read)");
     }
-    MATKV_CUDA(cudaLaunchHostFunc(copy_stream, cb_release_slab, new IoCallback{e, job.slab, job.use}));
-    return MATKV_OK;
+    int rc = MATKV_OK;
+    if (fp8_tokens > 0) {  // compressed chunk: the expanding copy reads the slab over the link (it must be device-accessible pinned memory)
+        rc = fp8_resident ? launch_stage_relayout_fp8(ctx, e->base + (size_t)job.slab * e->slab_bytes, dst, fp8_tokens, copy_stream)
+                          : launch_stage_expand_fp8(ctx, e->base + (size_t)job.slab * e->slab_bytes, dst, fp8_tokens,
+                                                    ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, copy_stream);
+    } else {
+        err = cudaMemcpyAsync(dst, e->base + (size_t)job.slab * e->slab_bytes, bytes, cudaMemcpyHostToDevice, copy_stream);
+        if (err != cudaSuccess) rc = cuda_fail(err, "copy out of the bounce slab");
+    }
+    cb = new IoCallback{e, job.slab, job.use, failed};
+    err = cudaLaunchHostFunc(copy_stream, cb_release_slab, cb);
+    if (err != cudaSuccess) {
+        delete cb;
+        release_on_host(e, job.slab, job.use);
+        if (rc == MATKV_OK) rc = cuda_fail(err, "cudaLaunchHostFunc(release of the slab)");
+    }
+    return rc;
 }
 
 int open_chunk_file(const char *path, uint64_t offset, size_t bytes, int *fd_out) {

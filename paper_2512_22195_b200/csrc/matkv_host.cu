@@ -25,17 +25,6 @@ int cuda_fail(cudaError_t e, const char *what) {
     return fail(MATKV_E_CUDA, "CUDA error %d (%s) in %s", (int)e, cudaGetErrorString(e), what);
 }
 
-struct DeviceGuard {
-    int prev = -1;
-    bool switched = false;
-    explicit DeviceGuard(int dev) {
-        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
-    }
-    ~DeviceGuard() {
-        if (switched) cudaSetDevice(prev);
-    }
-};
-
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 typedef CUresult (*EncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
@@ -179,6 +168,31 @@ static void matkv::reap_graveyard(matkv_ctx *ctx, bool force) {
     }
 }
 
+// A staging call that has been seen complete gives its event back: the chunks it staged no longer need to wait for
+// it, so they drop their reference, the event is destroyed and the ticket leaves the map (a failed one leaves its
+// number behind).  Called from the query / wait functions and, for every finished ticket, from the next staging call.
+static void retire_ticket(matkv_ctx *ctx, std::unordered_map<uint64_t, Ticket>::iterator it) {
+    Ticket &tk = it->second;
+    for (uint64_t id : tk.chunk_ids) {
+        auto c = ctx->chunks.find(id);
+        if (c != ctx->chunks.end() && c->second.ticket == it->first) c->second.ready = nullptr;
+    }
+    if (tk.io_failed && tk.io_failed->load(std::memory_order_acquire)) {
+        if (ctx->failed_tickets.size() >= 1024) ctx->failed_tickets.erase(ctx->failed_tickets.begin());
+        ctx->failed_tickets.push_back(it->first);
+    }
+    cudaEventDestroy(tk.done);
+    ctx->tickets.erase(it);
+}
+
+static void retire_finished_tickets(matkv_ctx *ctx) {
+    for (auto it = ctx->tickets.begin(); it != ctx->tickets.end();) {
+        auto cur = it++;
+        if (cudaEventQuery(cur->second.done) == cudaSuccess) retire_ticket(ctx, cur);
+        else cudaGetLastError();
+    }
+}
+
 static size_t blob_bytes(const matkv_config &c, int32_t n_tokens) {
     return (size_t)c.n_layers * 2 * c.n_kv_heads * (size_t)n_tokens * c.head_dim * sizeof(__nv_bfloat16);
 }
@@ -201,7 +215,7 @@ int matkv_create(const matkv_config *cfg, matkv_ctx **out) {
         return fail(MATKV_E_INVALID_ARG, "matkv_create: bad capacity");
     if ((int64_t)cfg->max_batch * cfg->n_layers * cfg->n_kv_heads * cfg->max_tail_tokens >= (int64_t)1 << 31)
         return fail(MATKV_E_CAPACITY, "matkv_create: max_batch x layers x KV heads x max_tail_tokens must stay below 2^31 rows");
-    if (cfg->softmax_scale < 0.f || cfg->rope_theta < 0.f || cfg->pos_mode < 0 || cfg->pos_mode > 1)
+    if (cfg->softmax_scale < 0.f || cfg->rope_theta < 0.f || cfg->pos_mode < 0 || cfg->pos_mode > 2)
         return fail(MATKV_E_INVALID_ARG, "matkv_create: bad scale / rotary settings");
     int dev = cfg->device;
     if (dev < 0) MATKV_CUDA(cudaGetDevice(&dev));
@@ -281,6 +295,16 @@ int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
             if (value < 1 || value > 1024) return fail(MATKV_E_INVALID_ARG, "tiles per chunk-major item must be 1..1024");
             ctx->opt_share_tiles = value;
             return MATKV_OK;
+        case MATKV_OPT_IO_TIMEOUT_MS:
+            if (value < 1 || value > 3600000) return fail(MATKV_E_INVALID_ARG, "storage read time limit must be 1..3600000 ms");
+            ctx->opt_io_timeout_ms = value;
+            io_engine_configure(ctx);
+            return MATKV_OK;
+        case MATKV_OPT_IO_TEST_DELAY_MS:
+            if (value < 0 || value > 60000) return fail(MATKV_E_INVALID_ARG, "injected read delay must be 0..60000 ms");
+            ctx->opt_io_test_delay_ms = value;
+            io_engine_configure(ctx);
+            return MATKV_OK;
         case MATKV_OPT_PREFILL_CTAS:
             if (value < 0 || value > 64) return fail(MATKV_E_INVALID_ARG, "prefill CTAs per head must be 0..64");
             ctx->opt_prefill_ctas = value;
@@ -334,6 +358,16 @@ int matkv_register_chunk(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens, co
     c.n_tokens = n_tokens;
     c.host_blob = host_blob;
     c.dev_blob = dev_blob;
+    if (host_blob) {
+        // the staging copy kernel reads a host blob over the link: only page-locked (or managed) memory allows that;
+        // a pageable blob is staged by the copy engine whatever MATKV_OPT_STAGE_CTAS says
+        DeviceGuard guard(ctx->device);
+        cudaPointerAttributes at;
+        if (cudaPointerGetAttributes(&at, host_blob) == cudaSuccess)
+            c.host_device_readable = at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeManaged || at.type == cudaMemoryTypeDevice;
+        else
+            cudaGetLastError();
+    }
     if (dev_blob) {
         int rc = encode_rows_map(&c.tmap, dev_blob, ctx->cfg.head_dim, (uint64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * n_tokens);
         if (rc) return rc;
@@ -399,6 +433,7 @@ int matkv_register_chunk_fp8(matkv_ctx *ctx, uint64_t chunk_id, int32_t n_tokens
     Chunk c;
     c.n_tokens = n_tokens;
     c.host_blob = host_blob_fp8;
+    c.host_device_readable = true;
     c.fp8 = true;
     ctx->chunks.emplace(chunk_id, c);
     return MATKV_OK;
@@ -524,60 +559,56 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
     // the region's previous readers must be done before anything is overwritten
     if (r->has_last_use) MATKV_CUDA(cudaStreamWaitEvent(cs, r->last_use, 0));
 
+    retire_finished_tickets(ctx);   // staging calls already seen complete give their events back: the map stays bounded
     Ticket tk;
     MATKV_CUDA(cudaEventCreateWithFlags(&tk.done, cudaEventDisableTiming));
+    tk.io_failed = std::make_shared<std::atomic<int>>(0);
     const uint64_t ticket = ctx->next_ticket++;
     int32_t next_free = 0;
+    int rc_fail = MATKV_OK;   // a failure part-way: the chunks already touched keep a valid event, then the error is returned
+    bool any_file = false;
     for (uint64_t id : want) {
         Chunk &c = ctx->chunks[id];
         if (c.region == r && c.slot >= 0 && r->used[c.slot] && r->occupant[c.slot] == id) continue;  // already here
         while (next_free < n_slots && r->used[next_free]) ++next_free;
         if (next_free >= n_slots) {
-            cudaEventDestroy(tk.done);
-            return fail(MATKV_E_CAPACITY, "no free slot left in the region");
+            rc_fail = fail(MATKV_E_CAPACITY, "no free slot left in the region");
+            break;
         }
-        if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;  // moves from another region
         void *dst = (char *)dev_slots + (size_t)next_free * slot_bytes;
         const bool keep8 = c.fp8 && ctx->opt_fp8_resident;
+        int rc = MATKV_OK;
         if (c.host_blob && c.fp8) {
             // compressed chunk: expanded to bf16 on its way in, or re-laid out into the resident compressed form (always
             // by an SM kernel that reads the host blob over the link: it must be device-accessible pinned memory)
-            int rc = keep8 ? launch_stage_relayout_fp8(ctx, c.host_blob, dst, c.n_tokens, cs)
-                           : launch_stage_expand_fp8(ctx, c.host_blob, dst, c.n_tokens, ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, cs);
-            if (rc) {
-                cudaEventDestroy(tk.done);
-                return rc;
-            }
-        } else if (c.host_blob && ctx->opt_stage_ctas > 0) {
-            // SM-driven copy (the host blob must be device-accessible: pinned memory under unified addressing)
-            int rc = launch_stage_copy(ctx, c.host_blob, dst, blob_bytes(ctx->cfg, c.n_tokens), (int)ctx->opt_stage_ctas, cs);
-            if (rc) {
-                cudaEventDestroy(tk.done);
-                return rc;
-            }
+            rc = keep8 ? launch_stage_relayout_fp8(ctx, c.host_blob, dst, c.n_tokens, cs)
+                       : launch_stage_expand_fp8(ctx, c.host_blob, dst, c.n_tokens, ctx->opt_stage_ctas > 0 ? (int)ctx->opt_stage_ctas : 16, cs);
+        } else if (c.host_blob && ctx->opt_stage_ctas > 0 && c.host_device_readable) {
+            // SM-driven copy (checked at registration: the blob is page-locked memory the device can read)
+            rc = launch_stage_copy(ctx, c.host_blob, dst, blob_bytes(ctx->cfg, c.n_tokens), (int)ctx->opt_stage_ctas, cs);
         } else if (c.host_blob) {
             cudaError_t e = cudaMemcpyAsync(dst, c.host_blob, blob_bytes(ctx->cfg, c.n_tokens), cudaMemcpyHostToDevice, cs);
-            if (e != cudaSuccess) {
-                cudaEventDestroy(tk.done);
-                return cuda_fail(e, "staging copy");
-            }
+            if (e != cudaSuccess) rc = cuda_fail(e, "staging copy");
         } else {  // storage tier: read into the bounce ring, then copy, all in the copy stream's order
-            int rc = io_engine_stage(ctx, c.file_fd, c.file_offset, c.fp8 ? fp8_blob_bytes(ctx->cfg, c.n_tokens) : blob_bytes(ctx->cfg, c.n_tokens),
-                                     dst, cs, c.fp8 ? c.n_tokens : 0, keep8);
-            if (rc) {
-                cudaEventDestroy(tk.done);
-                return rc;
-            }
+            any_file = true;
+            rc = io_engine_stage(ctx, c.file_fd, c.file_offset, c.fp8 ? fp8_blob_bytes(ctx->cfg, c.n_tokens) : blob_bytes(ctx->cfg, c.n_tokens),
+                                 dst, cs, tk.io_failed, c.fp8 ? c.n_tokens : 0, keep8);
         }
-        {
-            int rc = keep8 ? encode_fp8_maps(c.tmap8, dst, ctx->cfg, c.n_tokens)
-                           : encode_rows_map(&c.tmap, dst, ctx->cfg.head_dim, (uint64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * c.n_tokens);
-            if (rc) {
-                cudaEventDestroy(tk.done);
-                return rc;
-            }
-            c.resident_fp8 = keep8;
+        if (rc == MATKV_OK)
+            rc = keep8 ? encode_fp8_maps(c.tmap8, dst, ctx->cfg, c.n_tokens)
+                       : encode_rows_map(&c.tmap, dst, ctx->cfg.head_dim, (uint64_t)ctx->cfg.n_layers * 2 * ctx->cfg.n_kv_heads * c.n_tokens);
+        if (rc) {
+            // this chunk has no usable device copy (whatever was enqueued for it lands in a slot nobody points at)
+            if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;
+            c.staged = nullptr;
+            c.region = nullptr;
+            c.slot = -1;
+            c.ready = nullptr;
+            rc_fail = rc;
+            break;
         }
+        if (c.region && c.slot >= 0) c.region->used[c.slot] = 0;  // moves from another region (or another slot)
+        c.resident_fp8 = keep8;
         r->used[next_free] = 1;
         r->occupant[next_free] = id;
         c.staged = dst;
@@ -585,31 +616,50 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
         c.slot = next_free;
         c.ready = tk.done;
         c.ticket = ticket;
+        c.io_failed = tk.io_failed;
+        tk.chunk_ids.push_back(id);
     }
-    MATKV_CUDA(cudaEventRecord(tk.done, cs));
+    if (any_file) io_engine_flag_status(ctx, cs);   // a read failure of this call shows in the status word once the stream gets here
+    cudaError_t e_rec = cudaEventRecord(tk.done, cs);
     ctx->tickets.emplace(ticket, tk);
     *ticket_out = ticket;
+    if (rc_fail) return rc_fail;
+    if (e_rec != cudaSuccess) return cuda_fail(e_rec, "cudaEventRecord(staging ticket)");
+    return MATKV_OK;
+}
+
+// A ticket is live until its copies have been seen complete; retired tickets answer MATKV_OK (or MATKV_E_IO when a
+// storage read of theirs failed).
+static int retired_ticket_result(matkv_ctx *ctx, uint64_t ticket) {
+    if (ticket == 0 || ticket >= ctx->next_ticket) return fail(MATKV_E_INVALID_ARG, "unknown staging ticket %llu", (unsigned long long)ticket);
+    if (std::find(ctx->failed_tickets.begin(), ctx->failed_tickets.end(), ticket) != ctx->failed_tickets.end()) {
+        const char *msg = "";
+        io_engine_errors(ctx, &msg);
+        return fail(MATKV_E_IO, "staging ticket %llu: reading from storage failed: %s", (unsigned long long)ticket, msg);
+    }
     return MATKV_OK;
 }
 
 int matkv_stage_query(matkv_ctx *ctx, uint64_t ticket) {
     if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_stage_query: null context");
     auto it = ctx->tickets.find(ticket);
-    if (it == ctx->tickets.end()) return fail(MATKV_E_INVALID_ARG, "unknown staging ticket %llu", (unsigned long long)ticket);
+    if (it == ctx->tickets.end()) return retired_ticket_result(ctx, ticket);
+    DeviceGuard guard(ctx->device);
     cudaError_t e = cudaEventQuery(it->second.done);
-    if (e == cudaSuccess) return MATKV_OK;
     if (e == cudaErrorNotReady) return fail(MATKV_E_NOT_READY, "staging ticket %llu still copying", (unsigned long long)ticket);
-    return cuda_fail(e, "cudaEventQuery");
+    if (e != cudaSuccess) return cuda_fail(e, "cudaEventQuery");
+    retire_ticket(ctx, it);
+    return retired_ticket_result(ctx, ticket);
 }
 
 int matkv_stage_wait(matkv_ctx *ctx, uint64_t ticket) {
     if (!ctx) return fail(MATKV_E_INVALID_ARG, "matkv_stage_wait: null context");
     auto it = ctx->tickets.find(ticket);
-    if (it == ctx->tickets.end()) return fail(MATKV_E_INVALID_ARG, "unknown staging ticket %llu", (unsigned long long)ticket);
+    if (it == ctx->tickets.end()) return retired_ticket_result(ctx, ticket);
+    DeviceGuard guard(ctx->device);
     MATKV_CUDA(cudaEventSynchronize(it->second.done));
-    const char *msg = "";
-    if (io_engine_errors(ctx, &msg) > 0) return fail(MATKV_E_IO, "staging from storage failed: %s", msg);
-    return MATKV_OK;
+    retire_ticket(ctx, it);
+    return retired_ticket_result(ctx, ticket);
 }
 
 // ---- a3 --------------------------------------------------------------------------------------
@@ -660,8 +710,15 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
                 return fail(MATKV_E_NOT_STAGED, "request %d: chunk %llu has no device copy (stage it first)", r,
                             (unsigned long long)ids[k]);
             }
+            if (!c.dev_blob && c.io_failed && c.io_failed->load(std::memory_order_acquire)) {
+                delete t;
+                const char *msg = "";
+                io_engine_errors(ctx, &msg);
+                return fail(MATKV_E_IO, "request %d: chunk %llu was staged by a call whose storage reads failed: %s", r,
+                            (unsigned long long)ids[k], msg);
+            }
             if (!c.dev_blob) {
-                if (std::find(waits.begin(), waits.end(), c.ready) == waits.end()) waits.push_back(c.ready);
+                if (c.ready && std::find(waits.begin(), waits.end(), c.ready) == waits.end()) waits.push_back(c.ready);
                 if (std::find(t->regions.begin(), t->regions.end(), c.region) == t->regions.end())
                     t->regions.push_back(c.region);
             }
@@ -679,7 +736,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
             rq.chunk_tiles += (c.n_tokens + kTile - 1) / kTile;
             longest = std::max(longest, c.n_tokens);
         }
-        rq.pos_base = ctx->cfg.pos_mode == 0 ? rq.n_chunk_tokens : longest;
+        rq.pos_base = ctx->cfg.pos_mode == 1 ? longest : rq.n_chunk_tokens;   // mode 2: the caller may replace it (matkv_table_set_pos_base)
         t->max_chunk_tiles = std::max(t->max_chunk_tiles, rq.chunk_tiles);
         t->total_chunk_tiles += rq.chunk_tiles;
         t->h_reqs.push_back(rq);
@@ -864,6 +921,33 @@ int matkv_table_set_tail_len(matkv_table *t, int32_t tail_len, void *stream) {
     int rc = launch_add_tail_len(t, 0, tail_len, true, (cudaStream_t)stream);
     if (rc == MATKV_OK) t->tail_len_host = tail_len;
     return rc;
+}
+
+int matkv_table_set_pos_base(matkv_table *t, const int32_t *pos_base, void *stream) {
+    if (!t || !pos_base) return fail(MATKV_E_INVALID_ARG, "matkv_table_set_pos_base: null argument");
+    matkv_ctx *ctx = t->ctx;
+    if (ctx->cfg.pos_mode != 2) return fail(MATKV_E_INVALID_ARG, "matkv_table_set_pos_base: the context was not created with pos_mode 2");
+    for (int32_t r = 0; r < t->batch; ++r)
+        if (pos_base[r] < 0 || (int64_t)pos_base[r] + ctx->cfg.max_tail_tokens >= (int64_t)1 << 30)
+            return fail(MATKV_E_INVALID_ARG, "matkv_table_set_pos_base: base %d of request %d out of range", pos_base[r], r);
+    DeviceGuard guard(ctx->device);
+    // the request records sit in the table's pinned upload image right behind the segments; the copy is ordered
+    // behind the table's own upload on the same stream
+    DevReq *h_reqs = (DevReq *)((char *)t->h_pinned + ((char *)t->d_reqs - (char *)t->d_image));
+    for (int32_t r = 0; r < t->batch; ++r) {
+        t->h_reqs[r].pos_base = pos_base[r];
+        h_reqs[r].pos_base = pos_base[r];
+    }
+    MATKV_CUDA(cudaMemcpyAsync(t->d_reqs, h_reqs, sizeof(DevReq) * (size_t)t->batch, cudaMemcpyHostToDevice, (cudaStream_t)stream));
+    return MATKV_OK;
+}
+
+int matkv_stage_pending(matkv_ctx *ctx, int32_t *n_out) {
+    if (!ctx || !n_out) return fail(MATKV_E_INVALID_ARG, "matkv_stage_pending: null argument");
+    DeviceGuard guard(ctx->device);
+    retire_finished_tickets(ctx);
+    *n_out = (int32_t)ctx->tickets.size();
+    return MATKV_OK;
 }
 
 // ---- a4 / a5 / a6 argument checks, then the launchers -----------------------------------------

@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include <map>
+#include <memory>
 #include <string>
 #include <unordered_map>
 #include <vector>
@@ -60,6 +61,7 @@ struct IoEngine;  // reader threads + pinned bounce ring for file-backed chunks
 struct Chunk {
     int32_t n_tokens = 0;
     const void *host_blob = nullptr;
+    bool host_device_readable = false;  // host_blob is page-locked (or managed) memory a kernel may read over the link
     int file_fd = -1;              // >= 0: the blob lives in a file, at file_offset
     uint64_t file_offset = 0;
     void *dev_blob = nullptr;      // caller-resident device copy
@@ -69,8 +71,10 @@ struct Chunk {
     void *staged = nullptr;        // device copy inside a slot region (or nullptr)
     Region *region = nullptr;
     int32_t slot = -1;
-    cudaEvent_t ready = nullptr;   // event of the staging call that (last) copied it; borrowed from the ticket
+    cudaEvent_t ready = nullptr;   // event of the staging call that (last) copied it; borrowed from the ticket, null once
+                                   // that call has been seen complete (the ticket is retired then and its event destroyed)
     uint64_t ticket = 0;
+    std::shared_ptr<std::atomic<int>> io_failed;  // set by the storage tier when a read of that staging call failed
     alignas(64) CUtensorMap tmap;  // 2-D view [rows][D] of the current device copy, 64 x kTile boxes, 128-byte swizzle
 };
 
@@ -98,6 +102,8 @@ struct PooledImage {  // a table image (pinned upload buffer + device copy) read
 
 struct Ticket {
     cudaEvent_t done = nullptr;
+    std::vector<uint64_t> chunk_ids;              // chunks whose `ready` borrows the event
+    std::shared_ptr<std::atomic<int>> io_failed;  // shared with the storage tier's read jobs of this call
 };
 
 }  // namespace matkv
@@ -114,8 +120,10 @@ struct matkv_ctx {
     int64_t opt_decode_impl = 0, opt_share_tiles = 16, opt_fp8_resident = 0;
     std::unordered_map<uint64_t, matkv::Chunk> chunks;
     std::map<void *, matkv::Region *> regions;
-    std::unordered_map<uint64_t, matkv::Ticket> tickets;
+    std::unordered_map<uint64_t, matkv::Ticket> tickets;   // staging calls not yet seen complete
+    std::vector<uint64_t> failed_tickets;                  // retired tickets whose storage reads failed
     uint64_t next_ticket = 1;
+    int64_t opt_io_timeout_ms = 30000, opt_io_test_delay_ms = 0;
     std::vector<matkv_table *> tables;
     matkv::IoEngine *io = nullptr;
     std::vector<matkv::PooledImage> image_pool;
@@ -151,6 +159,18 @@ struct matkv_table {
 };
 
 namespace matkv {
+
+// makes `dev` the current device for the scope (and restores the previous one)
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
 
 int fail(int code, const char *fmt, ...);   // records the thread-local message, returns code
 int cuda_fail(cudaError_t e, const char *what);
@@ -219,12 +239,15 @@ int launch_gather(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t req, vo
                   int64_t rows, cudaStream_t stream);
 int io_engine_create(matkv_ctx *ctx, void *pinned, size_t bytes, size_t slab_bytes, int n_threads);
 void io_engine_destroy(matkv_ctx *ctx);
+void io_engine_configure(matkv_ctx *ctx);   // takes the read time limit (and the injected read delay) over from the context's options
 size_t io_engine_slab_bytes(const matkv_ctx *ctx);
 int io_engine_errors(matkv_ctx *ctx, const char **msg);
 // fp8_tokens > 0: the file holds a compressed chunk of that many tokens; on its way from the slab to dst it is expanded to
 // bf16 (fp8_resident false) or re-laid out into the HBM-resident compressed form (true)
-int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream, int32_t fp8_tokens = 0,
-                    bool fp8_resident = false);
+int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream,
+                    const std::shared_ptr<std::atomic<int>> &failed, int32_t fp8_tokens = 0, bool fp8_resident = false);
+// one tiny launch on the copy stream that turns a failed read of the calls so far into MATKV_E_IO in the status word
+int io_engine_flag_status(matkv_ctx *ctx, cudaStream_t copy_stream);
 size_t fp8_codes_bytes(const matkv_config &c, int32_t n_tokens);
 size_t fp8_blob_bytes(const matkv_config &c, int32_t n_tokens);
 int launch_quantize_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_fp8, cudaStream_t stream);

@@ -4,7 +4,8 @@
 // head of the KV group), row = token * G + head, so the G heads that share a KV head and up to
 // NBLK*128/G suffix tokens share every K/V tile that is fetched.  Per 64-token KV tile and row block:
 //     S  = Q K^T      tcgen05.mma  M=128, N=64,  K=D   (both operands K-major, 128-byte swizzle)  -> TMEM
-//     P  = softmax numerators of S (one thread per row: tcgen05.ld, fp32, exp2-based) -> bf16 in smem
+//     P  = softmax numerators of S (one thread per row: tcgen05.ld, fp32, exp2-based) -> bf16 pairs written back
+//          into S's own TMEM columns (tcgen05.st): the second MMA takes P as its A operand from tensor memory
 //     O += P V        tcgen05.mma  M=128, N=D,   K=64  (V is MN-major straight from its [token][d] tile),
 //                     accumulated in TMEM across the tiles
 // The exponent's reference maximum of a row only moves when the running maximum has grown by more than

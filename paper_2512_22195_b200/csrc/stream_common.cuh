@@ -207,6 +207,7 @@ static __device__ void combine_warp(const float *o_parts, int64_t o_stride, cons
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
                 const float w = __shfl_sync(0xffffffffu, w_l, (p0 + i) & 31);
+                if (w == 0.f) continue;   // an empty part carries no weight, whatever its row holds
                 acc.x = fmaf(w, v[i].x, acc.x); acc.y = fmaf(w, v[i].y, acc.y);
                 acc.z = fmaf(w, v[i].z, acc.z); acc.w = fmaf(w, v[i].w, acc.w);
             }
@@ -239,6 +240,7 @@ static __device__ void combine_warp(const float *o_parts, int64_t o_stride, cons
 #pragma unroll 4
         for (int pp = 0; pp < np; ++pp) {
             const float w = __shfl_sync(0xffffffffu, w_mine, pp);
+            if (w == 0.f) continue;   // an empty part carries no weight, whatever its row holds
             const float *row = o_parts + (p0 + pp) * o_stride + lane * dpl;
             if (dpl == 4) {
                 const float4 v = __ldcg((const float4 *)row);

@@ -363,6 +363,15 @@ def test_prefill_streaming_kernel_long_suffix():
     run_requests(1, 8, 2, 128, [[100, 30]], 37, 2, seed=43, prefill_impl=1)   # forced onto the streaming kernel
 
 
+@pytest.mark.parametrize("Hq,Hkv,S,ctas,all_layers", [(8, 2, 70, 1000, False), (8, 2, 130, 1000, True), (8, 1, 70, 37, False),
+                                                       (4, 4, 200, 1000, False), (8, 2, 70, 0, False)])
+def test_prefill_streaming_kernel_suffix_of_several_new_token_tiles(Hq, Hkv, S, ctas, all_layers):
+    """A suffix longer than one tile on the streaming kernel: every token block lists all ceil(S / 64) new-token tiles,
+    and a block of early tokens sees nothing in the later ones.  With one CTA per tile such a tile is a CTA's whole
+    share of the unit: an empty part (zero weight, lse = -inf) that the merge must ignore, never 0 / 0."""
+    run_requests(2, Hq, Hkv, 128, [[100, 30], []], S, 2, seed=48, prefill_impl=1, ctas=ctas, all_layers=all_layers)
+
+
 def test_prefill_appends_after_existing_tail():
     """Two prefill calls in a row (chunked sub-prefill): the second sees the first's tokens in the tail."""
     import paper_2512_22195_b200 as mk

@@ -389,3 +389,173 @@ def test_attend_after_graph_replays_needs_the_tail_length_set_again():
     o_ref, l_ref = req.attend_new(0, qs[3][0][None], ks[3][0][None], ks[3][0][None])
     check(dev_to_bits(out)[0], o_ref[0], lse.cpu().numpy()[0], l_ref[0], "decode after replays, tail length set again")
     sess.close()
+
+
+def test_pageable_host_blob_is_staged_by_the_copy_engine_even_with_the_copy_kernel_on():
+    """The copy kernel reads host blobs over the link, which only page-locked memory allows.  A pageable blob
+    (an ordinary numpy array) must therefore never reach it: it is staged by the copy engine instead."""
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D, n = 1, 4, 2, 64, 200
+    sess = Session(L, Hq, Hkv, D, 1, 2, 4)
+    mk.matkv_set_option(sess.ctx, mk.OPT_STAGE_CTAS, 4)
+    pageable = np.ascontiguousarray(rand_bits(46, 0, (L, 2, Hkv, n, D)))       # ordinary host memory
+    assert pageable.ctypes.data % 16 == 0
+    mk.matkv_register_chunk(sess.ctx, 0, n, pageable.ctypes.data, None)
+    pinned = sess.register_host_chunk(1, rand_bits(46, 1, (L, 2, Hkv, n, D)))  # this one goes through the copy kernel
+    slot_bytes = pageable.nbytes
+    slots = torch.zeros(2 * slot_bytes, dtype=torch.uint8, device="cuda")
+    tk = sess.stage([0, 1], slots, slot_bytes, torch.cuda.Stream())
+    mk.matkv_stage_wait(sess.ctx, tk)
+    sess.build_table([[0, 1]])
+    k, v = sess.gather(0, 0, 2 * n)
+    assert np.array_equal(to_bits(k)[:, :n], pageable[0, 0]) and np.array_equal(to_bits(v)[:, :n], pageable[0, 1])
+    assert np.array_equal(to_bits(k)[:, n:], to_bits(pinned)[0, 0])
+    assert sess.status() == 0
+    sess.close()
+
+
+def test_staging_tickets_are_retired_so_a_long_serving_loop_stays_bounded():
+    """Every staging call creates an event; a server stages a batch per step for ever.  Finished calls must give
+    their events back (seen complete by a query, a wait or simply by the next staging call), and a retired ticket
+    keeps answering."""
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D, n = 1, 4, 2, 64, 64
+    sess = Session(L, Hq, Hkv, D, 1, 2, 4)
+    blobs = [rand_bits(47, i, (L, 2, Hkv, n, D)) for i in range(4)]
+    for i, b in enumerate(blobs):
+        sess.register_host_chunk(i, b)
+    slot_bytes = blobs[0].nbytes
+    regions = [torch.empty(2 * slot_bytes, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    copy = torch.cuda.Stream()
+    tickets = []
+    for step in range(300):
+        pair = [(2 * step) % 4, (2 * step + 1) % 4]
+        tickets.append(sess.stage(pair, regions[step % 2], slot_bytes, copy))
+        sess.build_table([pair])                               # never queries or waits for a ticket
+        if step % 50 == 49:
+            torch.cuda.synchronize()
+            assert mk.matkv_stage_pending(sess.ctx) == 0       # everything finished has been retired
+    assert mk.matkv_stage_pending(sess.ctx) <= 2
+    k, v = sess.gather(0, 0, 2 * n)                            # the last table still reads the right bytes
+    assert np.array_equal(to_bits(k), np.concatenate([blobs[2][0, 0], blobs[3][0, 0]], axis=1))
+    for tk in (tickets[0], tickets[150], tickets[-1]):
+        mk.matkv_stage_wait(sess.ctx, tk)                      # retired tickets answer as finished
+        assert mk.matkv_stage_query(sess.ctx, tk)
+    with pytest.raises(mk.MatkvError):
+        mk.matkv_stage_query(sess.ctx, tickets[-1] + 1000)     # a number never handed out
+    assert sess.status() == 0
+    sess.close()
+
+
+def test_storage_read_failures_reach_the_attention_path(tmp_path):
+    """Failures injected on the host, no GPU fault anywhere: (1) a chunk file truncated after registration makes the
+    read come back short; (2) reads delayed beyond the time limit make the copy stream give up on them.  Either way
+    the wait reports MATKV_E_IO, a table over such a chunk is refused, and the device status word reads MATKV_E_IO
+    for work queued behind the staging call without any host wait; the context stays usable afterwards."""
+    import os
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D, n = 1, 4, 2, 64, 64
+    blobs = [rand_bits(48, i, (L, 2, Hkv, n, D)) for i in range(3)]
+    slot_bytes = (blobs[0].nbytes + 4095) // 4096 * 4096
+
+    def fresh():
+        sess = Session(L, Hq, Hkv, D, 1, 3, 4)
+        for i, b in enumerate(blobs):
+            with open(tmp_path / f"{i}.kv", "wb") as f:
+                f.write(b.tobytes())
+            mk.matkv_register_chunk_file(sess.ctx, i, n, str(tmp_path / f"{i}.kv"))
+        ring = torch.empty(2 * slot_bytes + 4096, dtype=torch.uint8, pin_memory=True)
+        base = (ring.data_ptr() + 4095) // 4096 * 4096
+        mk.matkv_set_bounce_buffer(sess.ctx, base, 2 * slot_bytes, slot_bytes, 2)
+        slots = torch.zeros(3 * slot_bytes, dtype=torch.uint8, device="cuda")
+        return sess, ring, slots
+
+    # (1) short file
+    sess, ring, slots = fresh()
+    os.truncate(tmp_path / "1.kv", blobs[1].nbytes // 2)
+    copy = torch.cuda.Stream()
+    tk = sess.stage([0, 1, 2], slots, slot_bytes, copy)
+    try:                                                        # usually too early for the host to know of the failure
+        table = mk.matkv_build_chunk_table(sess.ctx, [[0, 1, 2]], sess.tail_k.data_ptr(), sess.tail_v.data_ptr())
+    except mk.MatkvError as e:
+        assert e.code == mk.E_IO
+        table = None
+    torch.cuda.synchronize()
+    assert sess.status(clear=True) == mk.E_IO                   # flagged behind the copies, no host wait needed
+    if table:
+        mk.matkv_table_free(table)
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_stage_wait(sess.ctx, tk)
+    assert e.value.code == mk.E_IO
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_stage_query(sess.ctx, tk)                      # the retired ticket remembers
+    assert e.value.code == mk.E_IO
+    with pytest.raises(mk.MatkvError) as e:
+        sess.build_table([[0, 1, 2]])                           # now the failure is known: refused
+    assert e.value.code == mk.E_IO
+    sess.close()
+    del ring
+
+    # (2) reads that take longer than the stream is willing to wait
+    sess, ring, slots = fresh()
+    mk.matkv_set_option(sess.ctx, mk.OPT_IO_TIMEOUT_MS, 50)
+    mk.matkv_set_option(sess.ctx, mk.OPT_IO_TEST_DELAY_MS, 400)
+    tk = sess.stage([0], slots, slot_bytes, copy)
+    with pytest.raises(mk.MatkvError) as e:
+        mk.matkv_stage_wait(sess.ctx, tk)
+    assert e.value.code == mk.E_IO
+    assert sess.status(clear=True) == mk.E_IO
+    # the late read returns, the slab is free again, and the same context stages the chunk properly
+    mk.matkv_set_option(sess.ctx, mk.OPT_IO_TEST_DELAY_MS, 0)
+    mk.matkv_set_option(sess.ctx, mk.OPT_IO_TIMEOUT_MS, 30000)
+    slots2 = torch.zeros(3 * slot_bytes, dtype=torch.uint8, device="cuda")
+    tk = sess.stage([0, 2], slots2, slot_bytes, copy)
+    mk.matkv_stage_wait(sess.ctx, tk)
+    sess.build_table([[2, 0]])
+    k, v = sess.gather(0, 0, 2 * n)
+    assert np.array_equal(to_bits(k), np.concatenate([blobs[2][0, 0], blobs[0][0, 0]], axis=1))
+    sess.close()
+    del ring
+
+
+def test_p9_rotary_position_base_given_by_the_caller():
+    """pos_mode 2: the position of every request's first tail token is whatever the caller says."""
+    import oracle
+    from _util import check
+    mk, Session, to_dev, to_bits = _mk()
+    L, Hq, Hkv, D, S = 1, 8, 2, 128, 6
+    theta = 500000.0
+    sess = Session(L, Hq, Hkv, D, 2, 2, S + 2, rope_theta=theta, pos_mode=2)
+    blobs = [rand_bits(54, i, (L, 2, Hkv, n, D)) for i, n in enumerate([100, 30])]
+    for i, b in enumerate(blobs):
+        sess.register_device_chunk(i, b)
+    ids = [[0, 1], [1]]
+    bases = [7, 4096]
+    sess.build_table(ids)
+    mk.matkv_table_set_pos_base(sess.table, bases)
+    sh = oracle.Shape(L, Hq, Hkv, D)
+    reqs = [oracle.Request(sh, [blobs[c] for c in row], S + 2, rope_theta=theta, pos_base=bases[r]) for r, row in enumerate(ids)]
+    q, k, v = rand_bits(54, 10, (2, S, Hq, D)), rand_bits(54, 11, (2, S, Hkv, D)), rand_bits(54, 12, (2, S, Hkv, D))
+    out, lse = sess.prefill(0, to_dev(q), to_dev(k), to_dev(v))
+    for r in range(2):
+        o_ref, l_ref = reqs[r].attend_new(0, q[r], k[r], v[r])
+        check(to_bits(out)[r], o_ref, lse.cpu().numpy()[r], l_ref, f"caller-given base, prefill request {r}")
+        reqs[r].advance(S)
+    sess.advance(S)
+    q, k, v = rand_bits(54, 20, (2, Hq, D)), rand_bits(54, 21, (2, Hkv, D)), rand_bits(54, 22, (2, Hkv, D))
+    out, lse = sess.decode(0, to_dev(q), to_dev(k), to_dev(v))
+    for r in range(2):
+        o_ref, l_ref = reqs[r].attend_new(0, q[r][None], k[r][None], v[r][None])
+        check(to_bits(out)[r], o_ref[0], lse.cpu().numpy()[r], l_ref[0], f"caller-given base, decode request {r}")
+    tk = to_bits(sess.tail_k)
+    for r in range(2):                                          # the rotated keys in the tail match bit for bit
+        assert np.array_equal(tk[r, :, :, :S + 1], reqs[r].tail_k[:, :, :S + 1])
+    # a context in another mode refuses the call
+    other = Session(L, Hq, Hkv, D, 1, 1, 4, rope_theta=theta)
+    other.register_device_chunk(0, blobs[0])
+    other.build_table([[0]])
+    with pytest.raises(mk.MatkvError):
+        mk.matkv_table_set_pos_base(other.table, [5])
+    other.close()
+    assert sess.status() == 0
+    sess.close()

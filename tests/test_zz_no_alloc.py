@@ -1,17 +1,18 @@
-"""The allocation-free decode entry point against the ordinary one (collected last on purpose).
+"""The allocation-free decode entry point against the CPU oracle and the ordinary entry point (collected last on purpose).
 
 `matkv_attend_decode_static` serves callers that may neither allocate device memory nor lend a
 workspace (a server whose KV pool owns all of HBM, a plug-in under a host that forbids allocation
 after start-up): its split-KV scratch is an array built into the library.  It must give what
-`matkv_attend_decode` gives, on consecutive calls that reuse that one array, and must refuse calls
-larger than the array with a clear error.
+the oracle computes and what `matkv_attend_decode` gives, on consecutive calls that reuse that one array,
+and must refuse calls larger than the array with a clear error.
 """
 import numpy as np
 import pytest
 import torch
 
 import matkv_inputs as mi
-from _util import MAX_ABS, MEAN_ABS, rand_bits
+import oracle
+from _util import MAX_ABS, MEAN_ABS, check, rand_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -22,25 +23,32 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
     L, Hq, Hkv, D, B = 2, 32, 8, 128, 2
     sess = Session(L, Hq, Hkv, D, B, 3, 8)
     lens = [700, 130, 64]
-    for i, n in enumerate(lens):
-        sess.register_device_chunk(i, rand_bits(77, i, (L, 2, Hkv, n, D)))
-    sess.build_table([[0, 1, 2], [2, 0]])
+    blobs = [rand_bits(77, i, (L, 2, Hkv, n, D)) for i, n in enumerate(lens)]
+    for i, b in enumerate(blobs):
+        sess.register_device_chunk(i, b)
+    ids = [[0, 1, 2], [2, 0]]
+    sess.build_table(ids)
+    reqs = [oracle.Request(oracle.Shape(L, Hq, Hkv, D), [blobs[c] for c in row], 8) for row in ids]
     for step in range(2):                                   # two calls in a row share the built-in array
         for layer in range(L):
-            q = bits_to_dev(rand_bits(77, 100 + 10 * step + layer, (B, Hq, D)))
-            k = bits_to_dev(rand_bits(77, 200 + 10 * step + layer, (B, Hkv, D)))
-            v = bits_to_dev(rand_bits(77, 300 + 10 * step + layer, (B, Hkv, D)))
+            qb, kb, vb = (rand_bits(77, s0 + 10 * step + layer, (B, Hq if s0 == 100 else Hkv, D)) for s0 in (100, 200, 300))
+            q, k, v = bits_to_dev(qb), bits_to_dev(kb), bits_to_dev(vb)
             ref, ref_lse = sess.decode(layer, q, k, v)
             out = torch.zeros_like(q)
             lse = torch.zeros((B, Hq), dtype=torch.float32, device="cuda")
             mk.matkv_attend_decode_static(sess.ctx, sess.table, layer, q.data_ptr(), k.data_ptr(), v.data_ptr(),
                                           out.data_ptr(), lse.data_ptr())
+            for r in range(B):                              # first against the oracle, like every other kernel
+                o_ref, l_ref = reqs[r].attend_new(layer, qb[r][None], kb[r][None], vb[r][None])
+                check(dev_to_bits(out)[r], o_ref[0], lse.cpu().numpy()[r], l_ref[0], f"static decode step {step} layer {layer} request {r}")
             a, b = mi.bf16_bits_to_f64(dev_to_bits(out)), mi.bf16_bits_to_f64(dev_to_bits(ref))
             assert np.all(np.isfinite(a))
             assert np.max(np.abs(a - b)) <= MAX_ABS and np.mean(np.abs(a - b)) <= MEAN_ABS
             assert np.max(np.abs(lse.cpu().numpy() - ref_lse.cpu().numpy())) <= 1e-3
             assert np.linalg.norm(b) > 0
         sess.advance(1)
+        for rq in reqs:
+            rq.advance(1)
     assert sess.status() == 0
     sess.close()
 
