@@ -8,7 +8,13 @@ with every input already resident in HBM; `e2e` repeats it through the same C-AB
 from HOST buffers (chunk blobs staged from pinned host memory, q/k/v copied in per step, outputs
 copied back).  The numbers are attention-path only (no model weights, no MLP).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--decode-launch all_layers|per_layer]
+With no --workload the headline configuration runs: config 4 (Llama-3-70B head shape, 80 layers, batch 4, 32 x 2,048-token
+chunks per request = 64K tokens of context and 86 GB of KV in HBM), the largest configuration that fits one GPU; the lines
+of configurations 2, 3 and 5 (each from a child process of its own once the headline has released the GPU's memory) are
+attached under `other_workloads`.  --gpus N without a torchrun environment starts N ranks itself (independent replicas:
+the only cross-rank traffic is the barrier and the max over ranks of the measured time).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--decode-launch all_layers|per_layer]
   python bench.py --impl reference ...      # the CPU oracle as it stands, on the host cores
 """
 from __future__ import annotations
@@ -31,9 +37,13 @@ import matkv_inputs as mi  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per decode launch from the committed ncu capture (profiles/), by workload and launch mode.
-NCU_TRAFFIC_BYTES = {("cfg2", "all_layers"): 697.5e6 + 5.0e6,   # profiles/k_attend_stream_decode_cfg2_all_layers.md
-                     ("cfg3", "all_layers"): 10.02e9 + 0.10e9}   # profiles/k_attend_shared_decode_cfg3.md (chunk-major kernel)
+FALLBACK_BF16_TFLOPS = 1590.0
+HEADLINE = "cfg4"
+# DRAM bytes (read + write) of ONE all-layers decode launch, from one ncu capture of the kernels as they are built now:
+# (workload, launch mode) -> (bytes of the captured launch, layers of the captured case).  A capture of the full launch
+# is used as it is; a capture of a few-layer case (the full workload is too large to capture) is scaled by the layer
+# count, traffic being proportional to it.  None: not captured for this build, `traffic` is then null.
+NCU_TRAFFIC = {}
 
 
 def log(*a):
@@ -158,13 +168,15 @@ def run_reference(args):
         t += st.decode_steps(0, per_step)
         st.rewind(per_step)
     tok_s = args.steps * per_step * w.batch / (t * w.n_layers / n_l)
+    n_req = [len(row) * w.chunk_tokens for row in ids]
+    config = workload_config(w, "all_layers", kv_bytes_of_decode(w, n_req) / w.decode_steps)
     sample = (f"decode step 0 of {w.name} ({n_l} of {w.n_layers} layers, batch {w.batch}), repeated per bench step"
               + ("" if n_l == w.n_layers else ", extrapolated linearly to all layers"))
     print(json.dumps({
         "impl": "reference", "metric": "decode_tokens_per_s", "value": tok_s, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "sample": sample},
+        "config": config,
         "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": st.cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }), flush=True)
@@ -430,18 +442,20 @@ def run_materialise(args):
 
 
 # ---- the CUDA arm ----------------------------------------------------------------------------------
-def main():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="matkv", choices=["matkv", "reference"])
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default=HEADLINE, help="cfg1 .. cfg5 or materialise; default: the headline configuration "
+                    "(the largest that fits one GPU), with the other configurations' lines attached")
     ap.add_argument("--decode-launch", default="all_layers", choices=["all_layers", "per_layer", "per_layer_graph"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--decode-ctas", type=int, default=0)
-    ap.add_argument("--no-other-mode", action="store_true", help="skip the second pass in the other decode launch mode")
+    ap.add_argument("--no-other-mode", action="store_true", help="skip the extra passes in the other decode launch modes")
+    ap.add_argument("--no-other-workloads", action="store_true", help="headline run: do not attach the other configurations' lines")
     ap.add_argument("--batches", type=int, default=0, help="pipelined serving: number of sequential batches")
     ap.add_argument("--pool-chunks", type=int, default=0, help="pipelined serving: chunks in the pinned host pool")
     ap.add_argument("--store-dir", default="", help="pipelined serving: keep the chunk pool as files in this directory "
@@ -465,7 +479,18 @@ def main():
                     help="decode kernel: 0 auto (chunk-major when the batch's requests share chunks), 1 request-major, 2 chunk-major")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (small profiling cases)")
-    args = ap.parse_args()
+    return ap.parse_args(argv)
+
+
+def _spawned_rank(rank, args):
+    """One rank of a run that bench.py started itself (--gpus N without a torchrun environment)."""
+    result = run_cuda_arm(args)
+    if result is not None:
+        print(json.dumps(result), flush=True)
+
+
+def main(argv=None):
+    args = parse_args(argv)
     if args.impl == "reference":
         return run_reference(args)
     import __graft_entry__ as ge
@@ -474,21 +499,85 @@ def main():
         return run_materialise(args)
     if args.workload == "cfg5":
         return run_pipeline(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under torchrun: start the N ranks here (one process per GPU; independent replicas)
+        import torch
+        from paper_2512_22195_b200 import replicas
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus}: this machine shows {torch.cuda.device_count()} CUDA device(s)")
+        replicas.launch(args.gpus, _spawned_rank, args)
+        return
+    result = run_cuda_arm(args)
+    if result is None:
+        return
+    headline_alone = (args.workload == HEADLINE and int(os.environ.get("WORLD_SIZE", "1")) == 1 and not args.no_other_workloads
+                      and not (args.layers or args.decode_steps or args.pool_chunks) and args.kv_hbm == "bf16")
+    if headline_alone:
+        import gc
+        import torch
+        gc.collect()
+        torch.cuda.empty_cache()    # the headline's 86 GB of chunks are released: the child processes need the memory
+        result["other_workloads"] = run_other_workloads(args)
+    print(json.dumps(result), flush=True)
+
+
+def workload_config(w: mi.Workload, decode_launch: str, kv_bytes_per_step: float):
+    """The `config` object of a line: the same for the CUDA arm and the reference arm of a workload."""
+    return {"workload": w.name, "layers": w.n_layers, "q_heads": w.n_q_heads, "kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+            "batch": w.batch, "chunks_per_request": w.chunks_per_req, "chunk_tokens": w.chunk_tokens, "suffix": w.suffix,
+            "decode_steps": w.decode_steps, "decode_launch": decode_launch,
+            "prefill_launch": "all_layers" if decode_launch == "all_layers" else "per_layer",
+            "l2": f"inputs larger than L2 (KV per decode step = {kv_bytes_per_step / 1e6:.0f} MB vs 126 MB L2)",
+            "multi_gpu": "independent replicas per rank"}
+
+
+def kv_bytes_of_decode(w: mi.Workload, n_req, n_steps=None):
+    """Algorithmic KV bytes of `n_steps` decode steps (default: all): every visible K and V element once."""
+    T = w.decode_steps if n_steps is None else n_steps
+    return sum((n + w.suffix + t + 1) * w.beta for n in n_req for t in range(T)) * w.n_layers
+
+
+def run_other_workloads(args):
+    """The other configurations' lines, each from a child process (the GPU's memory is free again by now)."""
+    out = {}
+    steps = str(max(3, min(args.steps, 5)))
+    cases = {"cfg2": ["--workload", "cfg2", "--steps", str(args.steps), "--warmup", str(args.warmup)],
+             "cfg3": ["--workload", "cfg3", "--steps", steps, "--warmup", "3", "--no-e2e"],
+             # the pipelined-serving mode on a reduced pool and batch count (stated in its config): 40 GB cannot be pinned
+             # and walked three times within this run's time
+             "cfg5": ["--workload", "cfg5", "--batches", "10", "--pool-chunks", "128"]}
+    for name, extra in cases.items():
+        t0 = time.time()
+        try:
+            r = subprocess.run([sys.executable, os.path.abspath(__file__), "--gpus", "1", "--no-cpu-baseline", "--no-other-workloads"] + extra,
+                               capture_output=True, text=True, timeout=600)
+            lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+            out[name] = json.loads(lines[-1]) if (r.returncode == 0 and lines) else {"failed": f"rc {r.returncode}", "stderr_tail": r.stderr[-400:]}
+        except Exception as e:  # noqa: BLE001  (a failed side line must not lose the headline)
+            out[name] = {"failed": repr(e)}
+        out[name]["wall_s"] = round(time.time() - t0, 1)
+        log(f"[other workloads] {name}: {out[name].get('value', out[name].get('failed'))} in {out[name]['wall_s']} s")
+    return out
+
+
+def run_cuda_arm(args):
     args.warmup = max(args.warmup, 3)
 
     import torch
     import torch.distributed as dist
     import paper_2512_22195_b200 as mk
     import matkv_inputs.device as gen
+    from paper_2512_22195_b200 import replicas
     from paper_2512_22195_b200.harness import Session
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        log(f"[bench] --gpus {args.gpus} but WORLD_SIZE {world}: the process group decides, n_gpus = {world}")
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
+    replicas.init_from_env("nccl", dev)
 
     w = mi.workload(args.workload)
     if args.layers:
@@ -630,8 +719,6 @@ def main():
             ev_d1[timed_index].record(stream)
         return n
 
-    from paper_2512_22195_b200 import replicas
-
     def barrier():
         torch.cuda.synchronize()
         replicas.barrier()
@@ -668,15 +755,18 @@ def main():
         step_ms = sorted(a.elapsed_time(b) for a, b in zip(ev_p0, ev_d1))      # every timed step on its own (table upload excluded)
         dec_step_ms = sorted(a.elapsed_time(b) for a, b in zip(ev_dec, ev_d1))
         table_us_main = sorted(table_us)
-        # the other launch mode, for the record (same work, different launch granularity)
-        other = "per_layer_graph" if args.decode_launch == "all_layers" else "all_layers"
-        dec_ms_o = None
+        # the other launch granularities, for the record (same work): one launch per layer is what a model calls, replayed from
+        # a CUDA graph or launched one by one
+        others = [m for m in ("all_layers", "per_layer_graph", "per_layer") if m != args.decode_launch]
+        other_dec_ms = {}
         if not args.no_other_mode:
-            for _ in range(2):   # the first graph capture of a process pays one-off costs
-                one_step(*dev_ptrs, mode=other)
-            timed_region(lambda i: one_step(*dev_ptrs, timed_index=i, mode=other), min(args.steps, 5))
-            ev_dec_o = ev_g0 if other == "per_layer_graph" else ev_d0
-            dec_ms_o = sum(a.elapsed_time(b) for a, b in zip(ev_dec_o[:min(args.steps, 5)], ev_d1[:min(args.steps, 5)]))
+            for other in others:
+                k_o = min(args.steps, 3)
+                for _ in range(2):   # the first graph capture of a process pays one-off costs
+                    one_step(*dev_ptrs, mode=other)
+                timed_region(lambda i: one_step(*dev_ptrs, timed_index=i, mode=other), k_o)
+                ev_dec_o = ev_g0 if other == "per_layer_graph" else ev_d0
+                other_dec_ms[other] = sum(a.elapsed_time(b) for a, b in zip(ev_dec_o[:k_o], ev_d1[:k_o])) / k_o
 
     # read-only streaming probe over the same chunk memory (plain 16-byte loads), same run
     probe_gbs = None
@@ -718,14 +808,26 @@ def main():
         tile_bytes = 64 * w.beta
         read_bytes_decode = sum(tiles_read * tile_bytes + sum(S + t + 1 for _ in range(B)) * w.beta for t in range(T)) * L
         achieved = read_bytes_decode / decode_launches / (avg_launch_ms * 1e-3) / 1e9
+    tflops_peak_sus = float(peaks.get("bf16_tflops_sustained", FALLBACK_BF16_TFLOPS))
+    tflops_peak_burst = float(peaks.get("bf16_tflops", FALLBACK_BF16_TFLOPS))
+    prefill_tflops = prefill_flops * args.steps / (pre_ms * 1e-3) / 1e12
+    cap = NCU_TRAFFIC.get((args.workload, args.decode_launch)) if not (args.layers or args.decode_steps or fp8_hbm) else None
+    traffic = cap[0] * (L / cap[1]) if cap else None
+    kv_launch_mean = kv_bytes_decode / T          # KV bytes of one decode step (all layers), mean over the steps
+
+    def per_layer_phase(ms_per_step_decode):
+        us = ms_per_step_decode * 1e3 / (T * L)
+        return {"us_per_layer_launch": us, "kv_gbs": kv_launch_mean / L / (us * 1e-6) / 1e9,
+                "frac_of_hbm_peak": kv_launch_mean / L / (us * 1e-6) / 1e9 / peak,
+                "decode_only_tokens_per_s": B * T / (ms_per_step_decode * 1e-3)}
+
+    modes = {args.decode_launch: dec_ms / args.steps}
+    modes.update(other_dec_ms)
     result = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 in, fp32 softmax/accumulate" + (", chunk KV as e4m3 codes in HBM (fp16 MMAs)" if fp8_hbm else ""), "data": "synthetic",
-        "config": {"workload": w.name, "layers": L, "q_heads": Hq, "kv_heads": Hkv, "head_dim": D, "batch": B,
-                   "chunks_per_request": w.chunks_per_req, "chunk_tokens": w.chunk_tokens, "suffix": S, "decode_steps": T,
-                   "decode_launch": args.decode_launch, "prefill_launch": "all_layers" if args.decode_launch == "all_layers" else "per_layer", "l2": "inputs larger than L2 (KV per decode step = "
-                   f"{kv_bytes_decode / T / 1e6:.0f} MB vs 126 MB L2)", "multi_gpu": "independent replicas per rank"},
+        "config": workload_config(w, args.decode_launch, kv_bytes_decode / T),
         "gpu_launches": n_launch,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "k_attend_shared (chunk-major decode)" if chunk_major else "k_attend_stream (decode)",
@@ -734,43 +836,68 @@ def main():
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                      "read_probe_gbs_same_run": probe_gbs,
-                     "traffic": NCU_TRAFFIC_BYTES.get((w.name, args.decode_launch)) if (chunk_major or w.name != "cfg3") else None,
+                     "traffic": traffic,
+                     "traffic_source": (None if not cap else "one ncu capture of this kernel build" + ("" if cap[1] == L else
+                                        f" on a {cap[1]}-layer case, scaled by the layer count")),
                      "algorithmic_bytes_per_launch": (read_bytes_decode if chunk_major else kv_bytes_decode) / decode_launches,
                      "logical_kv_gbs": logical_gbs,
                      "avg_launch_us": avg_launch_ms * 1e3},
+        # the sub-prefill tiles: a dense contraction on the tensor cores (tcgen05), timed inside the step
+        "roofline_prefill": {"bound": "tensor", "kernel": "k_prefill_tc (sub-prefill)", "achieved": prefill_tflops, "unit": "TFLOP/s",
+                             "peak": tflops_peak_sus, "frac": prefill_tflops / tflops_peak_sus,
+                             "peak_kind": f"of {peak_kind} (bf16 sustained: the kernel runs inside a long step)",
+                             "frac_of_burst_peak": prefill_tflops / tflops_peak_burst,
+                             "flops_per_step": prefill_flops, "intensity_flop_per_byte": S * (Hq // Hkv)},
         "repeats": {"steps": args.steps, "step_ms_min": step_ms[0], "step_ms_median": step_ms[len(step_ms) // 2],
                     "decode_ms_min": dec_step_ms[0], "decode_ms_median": dec_step_ms[len(dec_step_ms) // 2],
                     "tokens_per_s_best_step": B * T * world / (step_ms[0] * 1e-3),
                     "table_build_host_us_median": table_us_main[len(table_us_main) // 2]},
         "phases": {"prefill_ms_per_step": pre_ms / args.steps, "decode_ms_per_step": dec_ms / args.steps,
-                   "prefill_tflops": prefill_flops * args.steps / (pre_ms * 1e-3) / 1e12,
+                   "prefill_tflops": prefill_tflops,
                    "decode_only_tokens_per_s": B * T * args.steps / (dec_ms * 1e-3),
                    "decode_kv_gbs": kv_bytes_decode * args.steps / (dec_ms * 1e-3) / 1e9,
                    "prefill_kv_gbs": kv_bytes_prefill * args.steps / (pre_ms * 1e-3) / 1e9,
-                   f"decode_only_tokens_per_s_{other}": (B * T * min(args.steps, 5) / (dec_ms_o * 1e-3)) if dec_ms_o else None},
+                   # one launch per layer is what a model's forward pass calls: per-launch time and KV GB/s, replayed from a
+                   # CUDA graph and launched one by one
+                   "per_layer_graph": per_layer_phase(modes["per_layer_graph"]) if "per_layer_graph" in modes else None,
+                   "per_layer": per_layer_phase(modes["per_layer"]) if "per_layer" in modes else None,
+                   "all_layers_decode_ms_per_step": modes.get("all_layers")},
     }
 
     # ---- end to end: the same step through the same calls, from host buffers --------------------
+    # A workload whose chunks do not fit ~24 GB of pinned host memory (and three device slot regions of that size) runs this
+    # leg on a subset of its layers, stated in the result: copies and compute are both exactly linear in the layer count, so
+    # the step time scales by L / layers-in-the-subset.
     e2e_bytes = len(needed) * w.chunk_bytes
-    if not args.no_e2e and e2e_bytes > 16e9:
-        result["e2e"] = {"value": None, "unit": "tokens/s", "skipped": f"{e2e_bytes / 1e9:.0f} GB of pinned host chunks: run with a smaller workload"}
-    elif not args.no_e2e:
+    Le = L
+    if e2e_bytes > 24e9:
+        Le = max(d for d in range(1, L + 1) if L % d == 0 and e2e_bytes * d / L <= 24e9)
+    e2e_scale = L / Le
+    if not args.no_e2e:
         copy = torch.cuda.Stream(device=dev)
-        host = {c: torch.empty(chunks[c].shape, dtype=torch.bfloat16, pin_memory=True) for c in needed}
+        host = {c: torch.empty((Le,) + tuple(chunks[c].shape[1:]), dtype=torch.bfloat16, pin_memory=True) for c in needed}
         for c in needed:
-            host[c].copy_(chunks[c])
-        hq_pf, hk_pf, hv_pf = (x.cpu().pin_memory() for x in (q_pf, k_pf, v_pf))
-        hq_dc, hk_dc, hv_dc = (x.cpu().pin_memory() for x in (q_dc, k_dc, v_dc))
-        ho_pf = torch.empty(o_pf.shape, dtype=torch.bfloat16, pin_memory=True)
-        ho_dc = torch.empty(o_dc.shape, dtype=torch.bfloat16, pin_memory=True)
+            host[c].copy_(chunks[c][:Le])
+        # the query-side tensors of the subset's layers (dense copies: the calls take dense [layers of the context] tensors)
+        eq_pf, ek_pf, ev_pf = (x[:Le].contiguous() for x in (q_pf, k_pf, v_pf))
+        eq_dc, ek_dc, ev_dc = (x[:, :Le].contiguous() for x in (q_dc, k_dc, v_dc))
+        hq_pf, hk_pf, hv_pf = (x.cpu().pin_memory() for x in (eq_pf, ek_pf, ev_pf))
+        hq_dc, hk_dc, hv_dc = (x.cpu().pin_memory() for x in (eq_dc, ek_dc, ev_dc))
+        ho_pf = torch.empty(eq_pf.shape, dtype=torch.bfloat16, pin_memory=True)
+        ho_dc = torch.empty(eq_dc.shape, dtype=torch.bfloat16, pin_memory=True)
+        qs_l, ks_l = eq_pf[0].numel() * 2, ek_pf[0].numel() * 2
+        qd_t, kd_t = eq_dc[0].numel() * 2, ek_dc[0].numel() * 2
+        qd_l, kd_l = eq_dc[0, 0].numel() * 2, ek_dc[0, 0].numel() * 2
         torch.cuda.synchronize()
-        sess2 = Session(L, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
+        sess2 = Session(Le, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
         e2e_stage_ctas = args.stage_ctas if args.stage_ctas >= 0 else 8
         if e2e_stage_ctas > 0:
             mk.matkv_set_option(sess2.ctx, mk.OPT_STAGE_CTAS, e2e_stage_ctas)
+        if args.decode_impl:
+            mk.matkv_set_option(sess2.ctx, mk.OPT_DECODE_IMPL, args.decode_impl)
         for c in needed:
             mk.matkv_register_chunk(sess2.ctx, c, w.chunk_tokens, host[c].data_ptr(), None)
-        slot_bytes = w.chunk_bytes
+        slot_bytes = w.chunk_bytes // L * Le
         # the chunks of a step are split over N_COPY copy streams, each with slot regions of its own: several copies in
         # flight keep the link busier while the decode saturates HBM
         n_copy = max(1, min(args.copy_streams if args.copy_streams > 0 else (1 if e2e_stage_ctas > 0 else 2), len(needed)))
@@ -781,8 +908,8 @@ def main():
         # could only start when step i's compute did, and a step took as long as its copies plus the hand-over).
         NB = 3
         slots = [[torch.empty(len(parts[k]) * slot_bytes, dtype=torch.uint8, device=dev) for k in range(n_copy)] for _ in range(NB)]
-        d_in = [tuple(torch.empty_like(x) for x in (q_pf, k_pf, v_pf, q_dc, k_dc, v_dc)) for _ in range(NB)]
-        d_out = [(torch.empty_like(o_pf), torch.empty_like(o_dc)) for _ in range(NB)]
+        d_in = [tuple(torch.empty_like(x) for x in (eq_pf, ek_pf, ev_pf, eq_dc, ek_dc, ev_dc)) for _ in range(NB)]
+        d_out = [(torch.empty_like(eq_pf), torch.empty_like(eq_dc)) for _ in range(NB)]
         h_in = (hq_pf, hk_pf, hv_pf, hq_dc, hk_dc, hv_dc)
         h2d = len(needed) * slot_bytes + sum(x.numel() * 2 for x in h_in)
         d2h = (ho_pf.numel() + ho_dc.numel()) * 2
@@ -831,7 +958,7 @@ def main():
             if args.decode_launch == "all_layers":
                 mk.matkv_attend_prefill_all_layers(ctx2, table, S, dq_pf.data_ptr(), dk_pf.data_ptr(), dv_pf.data_ptr(), eo_pf.data_ptr(), None, sp)
             else:
-                for layer in range(L):
+                for layer in range(Le):
                     mk.matkv_attend_prefill(ctx2, table, layer, S, dq_pf.data_ptr() + layer * qs_l, dk_pf.data_ptr() + layer * ks_l,
                                             dv_pf.data_ptr() + layer * ks_l, eo_pf.data_ptr() + layer * qs_l, None, sp)
             mk.matkv_table_advance(table, S, sp)
@@ -842,7 +969,7 @@ def main():
                     if fused_advance:
                         continue
                 else:
-                    for layer in range(L):
+                    for layer in range(Le):
                         mk.matkv_attend_decode(ctx2, table, layer, dq_dc.data_ptr() + t * qd_t + layer * qd_l,
                                                dk_dc.data_ptr() + t * kd_t + layer * kd_l, dv_dc.data_ptr() + t * kd_t + layer * kd_l,
                                                eo_dc.data_ptr() + t * qd_t + layer * qd_l, None, sp)
@@ -876,8 +1003,11 @@ def main():
             ms_e, _, _, _ = timed_region(lambda i: e2e_step(i + w_e2e, last=(i == k_e2e - 1)), k_e2e)
         if sess2.status() != 0:
             raise RuntimeError("device status non-zero after the end-to-end region")
-        result["e2e"] = {"value": tokens * k_e2e / (ms_e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": h2d,
-                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / k_e2e, "steps": k_e2e, "warmup": w_e2e,
+        result["e2e"] = {"value": tokens * k_e2e / (ms_e * 1e-3 * e2e_scale), "unit": "tokens/s", "h2d_bytes_per_step": h2d * e2e_scale,
+                         "d2h_bytes_per_step": d2h * e2e_scale, "ms_per_step": ms_e / k_e2e * e2e_scale, "steps": k_e2e, "warmup": w_e2e,
+                         "subset": (None if Le == L else f"layers 0..{Le - 1} of {L}: the chunks of all {L} layers ({e2e_bytes / 1e9:.0f} GB) fit neither the "
+                                    f"pinned host pool nor three device slot regions; measured {ms_e / k_e2e:.1f} ms per step with "
+                                    f"{h2d / 1e9:.1f} GB copied in, scaled by {e2e_scale:g} (copies and compute are linear in layers)"),
                          "overlap": "the chunks and query-side inputs of the next two steps copied in (three slot regions), and the previous "
                                     "step's outputs copied out, on side streams under this step's prefill and decode",
                          "staging": (f"copy kernel, {e2e_stage_ctas} CTAs" if e2e_stage_ctas > 0 else "copy engine") + f", {n_copy} copy streams",
@@ -893,7 +1023,8 @@ def main():
         # calibrate on one layer, then take as many layers and steps as fit ~12 s (work is linear in both)
         probe = OracleState(w, {c: dev_to_bits(chunks[c][0:1]) for c in needed}, ids, layers=[0])
         t_one = max(probe.decode_steps(0, 1), 1e-3)
-        n_l = int(max(1, min(L, 40.0 / t_one)))     # about 40 core-seconds of oracle work in all
+        n_l = int(max(1, min(L, 40.0 / t_one)))     # about 40 seconds of oracle work in all
+        n_l = int(max(1, min(n_l, 4e9 // (len(needed) * (w.chunk_bytes // L)))))   # and at most ~4 GB of chunk layers on the host
         n_s = int(max(1, min(T - 1, round(40.0 / (t_one * n_l)))))
         st_o = OracleState(w, {c: dev_to_bits(chunks[c][0:n_l]) for c in needed}, ids, layers=list(range(n_l)))
         t_s = st_o.decode_steps(0, n_s)
@@ -903,11 +1034,10 @@ def main():
                                   "sample": f"decode steps 0..{n_s - 1} of {T} of {w.name} ({n_l} of {L} layers, batch {B}), "
                                             f"{t_s:.1f} s on {st_o.cores} threads{how}",
                                   "kv_gbs": sum((n + S + t + 1) * w.beta for n in n_req for t in range(n_s)) * n_l / t_s / 1e9}
-    if rank == 0:
-        print(json.dumps(result), flush=True)
     sess.close()
     if world > 1:
         dist.destroy_process_group()
+    return result if rank == 0 else None
 
 
 if __name__ == "__main__":

@@ -48,3 +48,26 @@ def test_single_process_is_identity():
     from paper_2512_22195_b200 import replicas
     assert replicas.world() == 1 and replicas.max_over_ranks(3.5) == 3.5
     assert replicas.whole_job_rate(100.0, 50.0) == 2000.0
+
+
+def _launched_rank(rank, out_dir):
+    """What a rank started by `replicas.launch` does in the benchmark, with gloo in place of NCCL and no GPU."""
+    from paper_2512_22195_b200 import replicas
+    assert int(os.environ["RANK"]) == rank and int(os.environ["LOCAL_RANK"]) == rank
+    assert os.environ["WORLD_SIZE"] == "2" and os.environ["MASTER_ADDR"] == "127.0.0.1"
+    replicas.init_from_env("gloo")
+    replicas.barrier()
+    rate = replicas.whole_job_rate(units_per_rank=256.0, ms_per_rank=100.0 * (rank + 1))
+    with open(os.path.join(out_dir, f"rank{rank}.txt"), "w") as f:
+        f.write(f"{replicas.world()} {rate}")
+    dist.destroy_process_group()
+
+
+def test_launch_starts_the_ranks_itself_world2(tmp_path):
+    """`bench.py --gpus N` outside torchrun starts its N ranks through `replicas.launch`: the ranks find the rendezvous
+    in their environment, join, and report the whole-job rate over the slowest rank's time."""
+    from paper_2512_22195_b200 import replicas
+    replicas.launch(2, _launched_rank, str(tmp_path))
+    for rank in range(2):
+        world, rate = open(tmp_path / f"rank{rank}.txt").read().split()
+        assert int(world) == 2 and abs(float(rate) - 2 * 256.0 / 0.2) < 1e-6
