@@ -103,6 +103,12 @@ typedef struct {
                                       decode; sub-prefill over such chunks also runs on the streaming kernel, and the chunk-major
                                       decode, the allocation-free decode and matkv_gather_debug refuse tables that hold them */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
+#define MATKV_OPT_CLUSTER_DECODE 11 /* matkv_attend_decode of a small batch (a launch of a few tiles per SM: a chain of latencies, not a
+                                      stream): 1 (default) = served by thread-block clusters, one cluster per (request, KV head), whose
+                                      CTAs merge their partials through distributed shared memory (no workspace traffic) and fetch
+                                      their first chunk tiles under the previous kernel's tail; 0 = always the streaming kernel;
+                                      2 = clusters even when MATKV_OPT_DECODE_IMPL is 1.  Larger launches use the streaming kernel
+                                      either way */
 #define MATKV_OPT_IO_TIMEOUT_MS 9  /* storage tier: how long the copy stream waits for one chunk's read before the staging call
                                       is marked failed (MATKV_E_IO) and the stream moves on; default 30,000 ms */
 #define MATKV_OPT_IO_TEST_DELAY_MS 10 /* failure injection on the host, for tests: every storage read sleeps this long first
@@ -223,7 +229,8 @@ int matkv_table_free(matkv_table *table, void *stream);
  * (they can then start before the previous kernel on the stream has finished) and compare it
  * with the device counter: after replaying a captured loop, call matkv_table_set_tail_len
  * before the next attend call outside a capture, or that launch reports MATKV_E_BOUNDS in
- * the device status and its output is void.                                                 */
+ * the device status and its output is void (a launch served by the cluster kernel, see
+ * MATKV_OPT_CLUSTER_DECODE, uses the host-side copy for balance only and is right anyway). */
 int matkv_table_advance(matkv_table *table, int32_t n_tokens, void *stream);
 int matkv_table_set_tail_len(matkv_table *table, int32_t tail_len, void *stream);
 /* pos_mode 2 only: sets, on `stream`, the position of the first tail token of every request

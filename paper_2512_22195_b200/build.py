@@ -9,7 +9,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmatkv.so")
-SOURCES = ["matkv_host.cu", "gather.cu", "attend_stream.cu", "attend_shared.cu", "prefill_tc.cu", "rope.cu", "file_stage.cu", "fp8_store.cu"]
+SOURCES = ["matkv_host.cu", "gather.cu", "attend_stream.cu", "attend_cluster.cu", "attend_shared.cu", "prefill_tc.cu", "rope.cu", "file_stage.cu", "fp8_store.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -305,6 +305,10 @@ int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
             ctx->opt_io_test_delay_ms = value;
             io_engine_configure(ctx);
             return MATKV_OK;
+        case MATKV_OPT_CLUSTER_DECODE:
+            if (value < 0 || value > 2) return fail(MATKV_E_INVALID_ARG, "cluster decode must be 0, 1 or 2");
+            ctx->opt_cluster_decode = value;
+            return MATKV_OK;
         case MATKV_OPT_PREFILL_CTAS:
             if (value < 0 || value > 64) return fail(MATKV_E_INVALID_ARG, "prefill CTAs per head must be 0..64");
             ctx->opt_prefill_ctas = value;
@@ -806,8 +810,21 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
     const size_t tl_bytes = align_up(sizeof(int32_t) * (size_t)batch, 256);
     const size_t maps_bytes = align_up(sizeof(CUtensorMap) * (seg_maps.size() + 2), 256);
     const size_t items_bytes = align_up(sizeof(DevItem) * std::max<size_t>(items.size(), 1), 256);
-    const size_t maps8_bytes = t->has_fp8 ? sizeof(CUtensorMap) * 2 * seg_maps8.size() : 0;
-    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes + maps_bytes + items_bytes + maps8_bytes;
+    const size_t maps8_bytes = t->has_fp8 ? align_up(sizeof(CUtensorMap) * 2 * seg_maps8.size(), 256) : 0;
+    // tile directory for the cluster decode kernel: a CTA finds any chunk tile of a request with one load
+    std::vector<int4> tile_dir;
+    if (!t->has_fp8 && t->total_chunk_tiles <= (int64_t)1 << 20) {
+        for (int32_t r = 0; r < batch; ++r) {
+            const DevReq &rq = t->h_reqs[r];
+            t->h_dir_begin.push_back((int32_t)tile_dir.size());
+            for (int32_t i = 0; i < rq.n_seg; ++i) {
+                const int32_t len = t->h_segs[rq.seg_begin + i].len;
+                for (int32_t r0 = 0; r0 < len; r0 += kTile) tile_dir.push_back(make_int4(rq.seg_begin + i, r0, len, std::min(kTile, len - r0)));
+            }
+        }
+    }
+    const size_t dir_bytes = align_up(sizeof(int4) * std::max<size_t>(tile_dir.size(), 1), 256);
+    t->image_bytes = segs_bytes + reqs_bytes + tl_bytes + maps_bytes + items_bytes + maps8_bytes + dir_bytes;
     CUtensorMap tail_maps[2];
     {
         const uint64_t tail_rows = (uint64_t)batch * ctx->cfg.n_layers * ctx->cfg.n_kv_heads * ctx->cfg.max_tail_tokens;
@@ -856,6 +873,11 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
         t->d_tmaps8 = (CUtensorMap *)((char *)t->d_image + off8);
         CUtensorMap *h8 = (CUtensorMap *)((char *)t->h_pinned + off8);
         for (size_t i = 0; i < seg_maps8.size(); ++i) memcpy(h8 + 2 * i, seg_maps8[i], 2 * sizeof(CUtensorMap));
+    }
+    if (!t->h_dir_begin.empty()) {
+        const size_t offd = segs_bytes + reqs_bytes + tl_bytes + maps_bytes + items_bytes + maps8_bytes;
+        t->d_tile_dir = (int4 *)((char *)t->d_image + offd);
+        if (!tile_dir.empty()) memcpy((char *)t->h_pinned + offd, tile_dir.data(), sizeof(int4) * tile_dir.size());
     }
     {
         CUtensorMap *hm = (CUtensorMap *)((char *)t->h_pinned + segs_bytes + reqs_bytes + tl_bytes);
@@ -1005,6 +1027,13 @@ static int launch_decode(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cu
         }
     }
     if (shared) return launch_attend_shared(ctx, t, a, region, region_bytes, stream);
+    if (impl != 1 || ctx->opt_cluster_decode == 2) {   // (an explicit request for the request-major kernel means the streaming kernel)
+        if (ctx->opt_cluster_decode != 0) {
+            bool taken = false;
+            int rc = launch_decode_cluster(ctx, t, a, stream, &taken);
+            if (rc || taken) return rc;
+        }
+    }
     return launch_attend_stream(ctx, t, a, stream);
 }
 

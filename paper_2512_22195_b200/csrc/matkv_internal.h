@@ -124,6 +124,7 @@ struct matkv_ctx {
     std::vector<uint64_t> failed_tickets;                  // retired tickets whose storage reads failed
     uint64_t next_ticket = 1;
     int64_t opt_io_timeout_ms = 30000, opt_io_test_delay_ms = 0;
+    int64_t opt_cluster_decode = 1;
     std::vector<matkv_table *> tables;
     matkv::IoEngine *io = nullptr;
     std::vector<matkv::PooledImage> image_pool;
@@ -149,6 +150,9 @@ struct matkv_table {
     CUtensorMap *d_tmaps = nullptr;  // one per segment, then the K tail and the V tail
     CUtensorMap *d_tmaps8 = nullptr; // two per segment (K codes, transposed V codes) when the table has compressed-resident chunks
     bool has_fp8 = false;            // some segment is compressed-resident: only the streaming kernel reads those
+    int4 *d_tile_dir = nullptr;      // one record per chunk tile of every request, in the request's order:
+                                     // {descriptor index, first row inside the chunk, chunk tokens, valid rows}
+    std::vector<int32_t> h_dir_begin;  // first record of each request
     matkv::DevItem *d_items = nullptr;  // chunk-major decode: the chunk items of one (layer, KV head)
     bool share_ok = false;              // the head grouping fits the chunk-major kernel
     int32_t n_items = 0;                // chunk items (the requests' tail items follow implicitly)
@@ -228,6 +232,8 @@ struct AttendArgs {
     int32_t advance = 0;          // streaming kernel only: tokens the launch adds to the tail lengths when it is done
 };
 int launch_attend_stream(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream);
+// decode step of one layer of a small batch as thread-block clusters; *taken = false when the launch does not fit it
+int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaStream_t stream, bool *taken);
 // chunk-major decode (S = 1): region = scratch for the partials, region_bytes its size
 int launch_attend_shared(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, void *region, size_t region_bytes, cudaStream_t stream);
 size_t shared_region_bytes(const matkv_config &c, const matkv_table *t, int n_layers_launch);

@@ -4,7 +4,7 @@ every tile, every KV-split boundary and every item cut is crossed), the tail's f
 own new token -- and a key one past the causal edge must not be seen at all.  Random-data parity alone leaves a
 dropped tile at long context close to the tolerance; a needle makes it exact.  Run through the tensor-core
 sub-prefill (one and two row blocks per CTA, one and several KV splits), the chunk-major decode (items of one
-and three tiles) and the request-major decode with one CTA per tile."""
+and three tiles), the request-major decode with one CTA per tile and the cluster decode."""
 import numpy as np
 import pytest
 import torch
@@ -103,8 +103,9 @@ def test_needles_through_the_tensor_core_prefill(impl, splits):
     sess.close()
 
 
-@pytest.mark.parametrize("decode_impl,share_tiles,ctas", [(2, 1, 0), (2, 3, 0), (2, 3, 5), (1, 0, 1000), (1, 0, 0)])
-def test_needles_through_the_decode_kernels(decode_impl, share_tiles, ctas):
+@pytest.mark.parametrize("decode_impl,share_tiles,ctas,cluster", [(2, 1, 0, 0), (2, 3, 0, 0), (2, 3, 5, 0), (1, 0, 1000, 0), (1, 0, 0, 0),
+                                                                  (1, 0, 0, 2)])
+def test_needles_through_the_decode_kernels(decode_impl, share_tiles, ctas, cluster):
     mk, Session, to_dev, to_bits = _mk()
     pool = [200, 64, 33, 129]
     ids = [[0, 1], [0, 2, 3], [1, 0], [0], [3, 0]]       # chunk 0 is listed by five requests: two stacked groups at G = 4
@@ -112,6 +113,7 @@ def test_needles_through_the_decode_kernels(decode_impl, share_tiles, ctas):
     seed = 92
     sess = Session(L, HQ, HKV, D, B, 3, PRE + 3)
     mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, decode_impl)
+    mk.matkv_set_option(sess.ctx, mk.OPT_CLUSTER_DECODE, cluster)     # 2: the cluster kernel (clusters of 8 CTAs per request and KV head)
     if share_tiles:
         mk.matkv_set_option(sess.ctx, mk.OPT_SHARE_TILES, share_tiles)
     if ctas:

@@ -29,7 +29,7 @@ def _bits(t):
 
 def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=False, q_shift=0, cap=None,
                  prefill_impl=0, prefill_ctas=0, rope_theta=0.0, pos_mode=0, fused_advance=False, pool=None,
-                 decode_impl=0, share_tiles=0):
+                 decode_impl=0, share_tiles=0, cluster=None):
     """Prefill S tokens then T decode steps for a batch; compare every output with the oracle.
     lens_per_req: chunk lengths per request (every chunk its own), or, with `pool` (a list of chunk lengths),
     indices into the pool per request, so that requests can list the same chunk."""
@@ -39,6 +39,8 @@ def run_requests(L, Hq, Hkv, D, lens_per_req, S, T, seed, ctas=0, all_layers=Fal
     sess = _session(L, Hq, Hkv, D, B, max(1, max(len(x) for x in lens_per_req)), cap, rope_theta=rope_theta, pos_mode=pos_mode)
     if decode_impl:
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, decode_impl)
+    if cluster is not None:
+        mk.matkv_set_option(sess.ctx, mk.OPT_CLUSTER_DECODE, cluster)
     if share_tiles:
         mk.matkv_set_option(sess.ctx, mk.OPT_SHARE_TILES, share_tiles)
     if ctas:
@@ -215,6 +217,135 @@ def test_back_to_back_decode_launches_across_a_tail_tile_boundary(decode_impl, L
         n = reqs[r].tail_len
         assert n == S + T
         assert np.array_equal(tk[r, :, :, :n], reqs[r].tail_k[:, :, :n]) and np.array_equal(tv[r, :, :, :n], reqs[r].tail_v[:, :, :n])
+    sess.close()
+
+
+# ---- per-layer decode of small batches as thread-block clusters ----------------------------------------
+@pytest.mark.parametrize("Hq,Hkv,D,lens", [
+    (32, 8, 128, [[1024, 1024, 512]]),                 # 8 units: clusters of 16 CTAs (42 tiles per unit)
+    (8, 2, 128, [[300, 77], [129]]),                   # 4 units, unequal requests
+    (64, 8, 128, [[200, 64]]),                         # G = 8: clusters of 8 at most (landing zone rows)
+    (8, 2, 64, [[128, 128]]),                          # D = 64
+    (4, 4, 128, [[65, 1, 64], [], [7]]),               # G = 1; a request without chunks; shares without any tile
+    (16, 2, 128, [[33]]),                              # fewer tiles than a full cluster
+    (8, 8, 64, [[500], [40, 40], [64], [1]]),          # 32 units: clusters of 4
+])
+def test_cluster_decode_matches_the_oracle(Hq, Hkv, D, lens):
+    """decode_impl 1 + cluster 2 forces the cluster kernel wherever the launch fits it; the tail grows through a tile
+    boundary (suffix of 60 tokens, 8 steps); sharper queries (scaled by 2) in a second pass."""
+    run_requests(2, Hq, Hkv, D, lens, 60, 8, seed=81, decode_impl=1, cluster=2)
+    run_requests(1, Hq, Hkv, D, lens, 3, 2, seed=82, decode_impl=1, cluster=2, q_shift=1)
+
+
+def test_cluster_decode_replayed_from_a_graph_while_the_tail_grows():
+    """One decode step (a launch per layer, then the tail counter) captured when the tail holds 60 tokens and replayed
+    twelve times: the shares were balanced for one tail tile, the tail grows into a second one, and every replayed
+    launch must still see exactly its tail (the kernel places tail tiles by the device's counter) and start its chunk
+    loads under its predecessor's tail.  Every step against the oracle; the tails bit for bit."""
+    import paper_2512_22195_b200 as mk
+    L, Hq, Hkv, D, S, T, seed = 3, 32, 8, 128, 60, 12, 83
+    lens = [1024, 300]
+    sess = _session(L, Hq, Hkv, D, 1, 2, S + T)
+    blobs = [rand_bits(seed, 100 + i, (L, 2, Hkv, n, D)) for i, n in enumerate(lens)]
+    for i, b in enumerate(blobs):
+        sess.register_device_chunk(i, b)
+    sess.build_table([[0, 1]])
+    req = oracle.Request(oracle.Shape(L, Hq, Hkv, D), blobs, S + T)
+    q, k, v = rand_bits(seed, 1, (L, 1, S, Hq, D)), rand_bits(seed, 2, (L, 1, S, Hkv, D)), rand_bits(seed, 3, (L, 1, S, Hkv, D))
+    sess.prefill_all_layers(_dev(q), _dev(k), _dev(v), want_lse=False)
+    for layer in range(L):
+        req.append_only(layer, k[layer, 0], v[layer, 0])
+    sess.advance(S)
+    req.advance(S)
+    qs = [rand_bits(seed, 2000 + t, (L, 1, Hq, D)) for t in range(T)]
+    ks = [rand_bits(seed, 3000 + t, (L, 1, Hkv, D)) for t in range(T)]
+    vs = [rand_bits(seed, 4000 + t, (L, 1, Hkv, D)) for t in range(T)]
+    g_q, g_k, g_v = _dev(qs[0]).clone(), _dev(ks[0]).clone(), _dev(vs[0]).clone()
+    g_o = torch.empty_like(g_q)
+    g_l = torch.empty((L, 1, Hq), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.Stream()
+    sp = stream.cuda_stream
+    outs = []
+    with torch.cuda.stream(stream):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for layer in range(L):
+                mk.matkv_attend_decode(sess.ctx, sess.table, layer, g_q[layer].data_ptr(), g_k[layer].data_ptr(), g_v[layer].data_ptr(),
+                                       g_o[layer].data_ptr(), g_l[layer].data_ptr(), sp)
+            mk.matkv_table_advance(sess.table, 1, sp)
+        mk.matkv_table_set_tail_len(sess.table, S, sp)          # the capture ran nothing but moved the host-side mirror
+        for t in range(T):
+            g_q.copy_(_dev(qs[t])); g_k.copy_(_dev(ks[t])); g_v.copy_(_dev(vs[t]))
+            graph.replay()
+            outs.append((g_o.clone(), g_l.clone()))
+        stream.synchronize()
+    assert sess.status() == 0
+    for t in range(T):
+        ob, lb = _bits(outs[t][0]), outs[t][1].cpu().numpy()
+        for layer in range(L):
+            o_ref, l_ref = req.attend_new(layer, qs[t][layer, 0][None], ks[t][layer, 0][None], vs[t][layer, 0][None])
+            check(ob[layer, 0], o_ref[0], lb[layer, 0], l_ref[0], f"replayed step {t} layer {layer}")
+        req.advance(1)
+    tk, tv = _bits(sess.tail_k), _bits(sess.tail_v)
+    assert np.array_equal(tk[0, :, :, :S + T], req.tail_k[:, :, :S + T]) and np.array_equal(tv[0, :, :, :S + T], req.tail_v[:, :, :S + T])
+    sess.close()
+
+
+def test_cluster_decode_long_replay_never_reads_a_tile_before_it_has_landed():
+    """The benchmark's per-layer mode at the Llama-3-8B head shape: 5 x 1,024-token chunks, a decode step of 8
+    per-layer launches captured once and replayed 128 times while the tail grows from 64 to 192 tokens (one, two, then
+    three tail tiles against shares balanced for one).  The two groups of consumer warps of a CTA reach a ring stage at
+    different times, so a stage's fill number has to be checked before its barrier phase: thousands of back-to-back
+    launches must leave the status word clean (a consumer that ran ahead would end in a bounded wait running out), and
+    sampled steps must match the oracle."""
+    import paper_2512_22195_b200 as mk
+    L, Hq, Hkv, D, S, T, seed = 8, 32, 8, 128, 64, 128, 84
+    sess = _session(L, Hq, Hkv, D, 1, 5, S + T)
+    blobs = [rand_bits(seed, 100 + i, (L, 2, Hkv, 1024, D)) for i in range(5)]
+    for i, b in enumerate(blobs):
+        sess.register_device_chunk(i, b)
+    sess.build_table([list(range(5))])
+    req = oracle.Request(oracle.Shape(L, Hq, Hkv, D), blobs, S + T)
+    q, k, v = rand_bits(seed, 1, (L, 1, S, Hq, D)), rand_bits(seed, 2, (L, 1, S, Hkv, D)), rand_bits(seed, 3, (L, 1, S, Hkv, D))
+    sess.prefill_all_layers(_dev(q), _dev(k), _dev(v), want_lse=False)
+    for layer in range(L):
+        req.append_only(layer, k[layer, 0], v[layer, 0])
+    sess.advance(S)
+    req.advance(S)
+    qs = rand_bits(seed, 2000, (T, L, 1, Hq, D))
+    ks = rand_bits(seed, 3000, (T, L, 1, Hkv, D))
+    vs = rand_bits(seed, 4000, (T, L, 1, Hkv, D))
+    dq, dk, dv = _dev(qs), _dev(ks), _dev(vs)
+    g_q, g_k, g_v = dq[0].clone(), dk[0].clone(), dv[0].clone()
+    g_o = torch.empty_like(g_q)
+    outs = torch.empty_like(dq)
+    stream = torch.cuda.Stream()
+    sp = stream.cuda_stream
+    with torch.cuda.stream(stream):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            for layer in range(L):
+                mk.matkv_attend_decode(sess.ctx, sess.table, layer, g_q[layer].data_ptr(), g_k[layer].data_ptr(), g_v[layer].data_ptr(),
+                                       g_o[layer].data_ptr(), None, sp)
+            mk.matkv_table_advance(sess.table, 1, sp)
+        mk.matkv_table_set_tail_len(sess.table, S, sp)
+        for t in range(T):
+            g_q.copy_(dq[t], non_blocking=True); g_k.copy_(dk[t], non_blocking=True); g_v.copy_(dv[t], non_blocking=True)
+            graph.replay()
+            outs[t].copy_(g_o, non_blocking=True)
+        stream.synchronize()
+    assert sess.status() == 0
+    ob = _bits(outs)
+    for t in range(T):
+        for layer in range(L):
+            if t in (0, 1, 63, 64, 127) and layer in (0, L - 1):
+                o_ref, _ = req.attend_new(layer, qs[t, layer, 0][None], ks[t, layer, 0][None], vs[t, layer, 0][None])
+                check(ob[t, layer, 0], o_ref[0], None, None, f"replayed step {t} layer {layer}")
+            else:
+                req.append_only(layer, ks[t, layer, 0][None], vs[t, layer, 0][None])
+        req.advance(1)
+    tk = _bits(sess.tail_k)
+    assert np.array_equal(tk[0, :, :, :S + T], req.tail_k[:, :, :S + T])
     sess.close()
 
 

@@ -355,6 +355,7 @@ def test_attend_after_graph_replays_needs_the_tail_length_set_again():
     L, Hq, Hkv, D, B = 1, 8, 2, 128, 1
     blob = rand_bits(95, 0, (L, 2, Hkv, 150, D))
     sess = Session(L, Hq, Hkv, D, B, 1, 16)
+    mk.matkv_set_option(sess.ctx, mk.OPT_CLUSTER_DECODE, 0)     # the streaming kernel (the cluster kernel never splits by the host's copy)
     sess.register_device_chunk(0, bits_to_dev(blob))
     sess.build_table([[0]])
     qs = [rand_bits(95, 10 + i, (B, Hq, D)) for i in range(4)]
