@@ -156,8 +156,11 @@ def run_reference(args):
     ids = w.chunk_ids(0)
     needed = sorted({c for row in ids for c in row})
     log(f"[reference] generating {len(needed)} chunks on the host ...")
-    n_l = w.n_layers if w.name in ("cfg1", "cfg2") else 1   # larger workloads: one layer per step (stated in `sample`)
-    blobs = {c: mi.chunk_blob_layers(w, c, n_l) for c in needed}
+    # larger workloads: a few layers per step, enough (layer, request) units to keep every host thread busy (stated in `sample`)
+    cores = os.cpu_count() or 1
+    n_l = w.n_layers if w.name in ("cfg1", "cfg2") else max(1, min(w.n_layers, 4, -(-cores // w.batch)))
+    with ThreadPoolExecutor(max_workers=cores) as ex:       # the generator is numpy: it releases the interpreter lock
+        blobs = dict(zip(needed, ex.map(lambda c: mi.chunk_blob_layers(w, c, n_l), needed)))
     st = OracleState(w, blobs, ids, layers=list(range(n_l)))
     per_step = 1  # each bench step = one decode step of the workload over the sampled layers and all requests
     for _ in range(args.warmup):
@@ -177,7 +180,7 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": config,
-        "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": st.cores, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": min(st.cores, n_l * w.batch), "kind": "oracle", "sample": sample},
         "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }), flush=True)
 
@@ -890,7 +893,9 @@ def run_cuda_arm(args):
         qd_l, kd_l = eq_dc[0, 0].numel() * 2, ek_dc[0, 0].numel() * 2
         torch.cuda.synchronize()
         sess2 = Session(Le, Hq, Hkv, D, B, w.chunks_per_req, S + T, device=local)
-        e2e_stage_ctas = args.stage_ctas if args.stage_ctas >= 0 else 8
+        # staging: 8 copy CTAs beside short decode launches (config 2: 45 GB/s against 38 with the copy engine); the copy engine
+        # on two streams when a step moves tens of gigabytes under long launches (config 4: 54.7 GB/s against 41 with 16 - 32 copy CTAs)
+        e2e_stage_ctas = args.stage_ctas if args.stage_ctas >= 0 else (8 if e2e_bytes < 4e9 else 0)
         if e2e_stage_ctas > 0:
             mk.matkv_set_option(sess2.ctx, mk.OPT_STAGE_CTAS, e2e_stage_ctas)
         if args.decode_impl:
@@ -1030,7 +1035,7 @@ def run_cuda_arm(args):
         t_s = st_o.decode_steps(0, n_s)
         per_step_full = t_s / n_s * (L / n_l)
         how = "" if n_l == L else f", extrapolated linearly from layers 0..{n_l - 1} to all {L}"
-        result["cpu_baseline"] = {"value": B / per_step_full, "unit": "tokens/s", "cores": st_o.cores, "kind": "oracle",
+        result["cpu_baseline"] = {"value": B / per_step_full, "unit": "tokens/s", "cores": min(st_o.cores, n_l * B), "kind": "oracle",
                                   "sample": f"decode steps 0..{n_s - 1} of {T} of {w.name} ({n_l} of {L} layers, batch {B}), "
                                             f"{t_s:.1f} s on {st_o.cores} threads{how}",
                                   "kv_gbs": sum((n + S + t + 1) * w.beta for n in n_req for t in range(n_s)) * n_l / t_s / 1e9}
