@@ -43,7 +43,8 @@ HEADLINE = "cfg4"
 # (workload, launch mode) -> (bytes of the captured launch, layers of the captured case).  A capture of the full launch
 # is used as it is; a capture of a few-layer case (the full workload is too large to capture) is scaled by the layer
 # count, traffic being proportional to it.  None: not captured for this build, `traffic` is then null.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {("cfg2", "all_layers"): (688_347_008 + 1_927_168, 32),      # k_attend_stream<128,4>: all 32 layers captured
+               ("cfg4", "all_layers"): (2_153_027_840 + 2_343_680, 2)}       # k_attend_stream<128,8>: a 2-layer case (2.15 GB), scaled x 40
 
 
 def log(*a):
