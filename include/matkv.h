@@ -100,8 +100,9 @@ typedef struct {
 #define MATKV_OPT_FP8_RESIDENT  8  /* staging of compressed chunks (matkv_register_chunk_fp8 / _file_fp8): 0 (default) = expand
                                       to the bf16 blob in HBM; 1 = keep them compressed in HBM too (head_dim 128 only): the
                                       streaming kernel then reads the codes and converts in registers, halving the HBM bytes of
-                                      decode; sub-prefill over such chunks also runs on the streaming kernel, and the chunk-major
-                                      decode, the allocation-free decode and matkv_gather_debug refuse tables that hold them */
+                                      decode; the tensor-core sub-prefill expands their code tiles to bf16 in shared memory (one row
+                                      block per CTA); the chunk-major decode, the cluster decode (such launches take the streaming
+                                      kernel), the allocation-free decode and matkv_gather_debug do not read tables that hold them */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
 #define MATKV_OPT_CLUSTER_DECODE 11 /* matkv_attend_decode of a small batch (a launch of a few tiles per SM: a chain of latencies, not a
                                       stream): 1 (default) = served by thread-block clusters, one cluster per (request, KV head), whose

@@ -1135,8 +1135,8 @@ int matkv_attend_prefill(matkv_ctx *ctx, matkv_table *t, int32_t layer, int32_t 
     }
     // long suffixes go to the tcgen05 tile kernel, short ones stay on the streaming kernel
     const int G = c.n_q_heads / c.n_kv_heads;
-    // (compressed-resident chunks are read by the streaming kernel only)
-    const bool tensor_core = !t->has_fp8 && (ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64));
+    // (compressed-resident chunks exist for head_dim 128 only; the tile kernel expands their codes in shared memory)
+    const bool tensor_core = ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
     if (tensor_core) return launch_prefill_tc(ctx, t, a, (cudaStream_t)stream);
     return launch_attend_stream(ctx, t, a, (cudaStream_t)stream);
 }
@@ -1165,8 +1165,8 @@ int matkv_attend_prefill_all_layers(matkv_ctx *ctx, matkv_table *t, int32_t S, c
         if (rc) return rc;
     }
     const int G = c.n_q_heads / c.n_kv_heads;
-    // (compressed-resident chunks are read by the streaming kernel only)
-    const bool tensor_core = !t->has_fp8 && (ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64));
+    // (compressed-resident chunks exist for head_dim 128 only; the tile kernel expands their codes in shared memory)
+    const bool tensor_core = ctx->opt_prefill_impl >= 2 || (ctx->opt_prefill_impl == 0 && S * G >= 64);
     if (tensor_core) return launch_prefill_tc(ctx, t, a, (cudaStream_t)stream);
     // short suffixes run on the streaming kernel; when its units do not fit the workspace's counters in one
     // launch, the layers are launched one by one (same result)

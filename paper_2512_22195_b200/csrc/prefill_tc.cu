@@ -17,8 +17,15 @@
 // double-buffered in TMEM so that the tensor core works on tile j+1 while the softmax threads work on
 // tile j; with two row blocks two softmax warps share each SM sub-partition.  Every wait is bounded and
 // reports through the status word; TMEM is always released.
+//
+// Compressed-resident chunks (template parameter F8; head_dim 128, one row block per CTA): the producer brings a tile's
+// e4m3 codes (K rows, V transposed per 64-token block, the block's two exponents) into a staging ring, and four
+// converter warps expand them to bf16 in the operand ring: K as before, V^T [d][token] as a K-major B operand of
+// O += P V (so the transposed store needs no transposing).  Every code stands for a bf16 number, so the expansion is
+// exact and the tiles the tensor core sees are the ones the expanding staging copy would have written to HBM.
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <math_constants.h>
 
 #include <algorithm>
@@ -38,6 +45,7 @@ struct Params {
     const DevReq *reqs;
     const DevSeg *segs;
     const CUtensorMap *tmaps;
+    const CUtensorMap *tmaps8;  // [n_seg_total][2] maps of compressed-resident chunks (K codes, transposed V codes), or null
     int32_t n_seg_total;
     const int32_t *tail_len;
     __nv_bfloat16 *tail_k, *tail_v;
@@ -95,6 +103,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
         "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
+}
+// untiled bulk copy global -> shared with mbarrier completion (both addresses 16-byte aligned, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst), "l"(src), "r"(bytes),
+                 "r"(bar)
+                 : "memory");
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -214,6 +228,21 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+// 16 e4m3 codes (one 16-byte chunk) times a power of two -> 16 bf16 (two chunks); exact: every code x 2^e is a bf16 number
+__device__ __forceinline__ void expand16(const uint4 w, const float scale, uint4 &lo, uint4 &hi) {
+    const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+    uint32_t out[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t h0, h1;   // codes 0,1 and 2,3 of the word as fp16 pairs (exact)
+        asm("{\n .reg .b16 a, b;\n mov.b32 {a, b}, %2;\n cvt.rn.f16x2.e4m3x2 %0, a;\n cvt.rn.f16x2.e4m3x2 %1, b;\n}" : "=r"(h0), "=r"(h1) : "r"(in[i]));
+        const float2 f0 = __half22float2(*reinterpret_cast<const __half2 *>(&h0)), f1 = __half22float2(*reinterpret_cast<const __half2 *>(&h1));
+        out[2 * i] = pack_bf16(f0.x * scale, f0.y * scale);
+        out[2 * i + 1] = pack_bf16(f1.x * scale, f1.y * scale);
+    }
+    lo = make_uint4(out[0], out[1], out[2], out[3]);
+    hi = make_uint4(out[4], out[5], out[6], out[7]);
+}
 // true in exactly one lane of the (converged) warp
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
@@ -225,41 +254,50 @@ __host__ __device__ __forceinline__ int cdiv(int a, int b) { return (a + b - 1) 
 // tile t of a unit: kind 0 = chunk, 1 = tail, 2 = new tokens
 struct Tile {
     int kind, seg, r0, rows, seg_len;
+    int fmt;   // chunk tiles: 0 = bf16 blob, 1 = compressed-resident codes
 };
 
-template <int D, int NBLK>
+template <int D, int NBLK, bool F8 = false>
 struct Cfg {
     static constexpr int NBOX = D / 64;
     static constexpr int BOX_BYTES = kTile * 128;        // 64 rows x 128 bytes
     static constexpr int KV_BYTES = NBOX * BOX_BYTES;    // K (or V) of one tile
     static constexpr int STAGE_BYTES = 2 * KV_BYTES;
     static constexpr int QBLK_BYTES = NBOX * kRowsPerCta * 128;   // Q of one row block
-    static constexpr int STAGES = 4;
-    // producer warp, MMA warp of row block 0, 4 softmax warps per block, and (last) the MMA warp of row block 1
-    static constexpr int THREADS = (2 + 4 * NBLK + (NBLK - 1)) * 32;
-    static constexpr int SMEM_BYTES = 1024 + NBLK * QBLK_BYTES + STAGES * STAGE_BYTES + 512;
+    static constexpr int STAGES = F8 ? 3 : 4;
+    // staging ring of code tiles (compressed-resident chunks): K codes, V codes, then the block's exponent record
+    static constexpr int CODE_STAGES = F8 ? 3 : 0;
+    static constexpr int CODE_BYTES = kTile * D;                  // codes of K (or of V) of one tile
+    static constexpr int CODE_STAGE_BYTES = 2 * CODE_BYTES + 1024;   // (+ the 16-byte record; keeps the 1024-byte alignment)
+    static constexpr int CONV_WARPS = F8 ? 4 : 0;
+    // producer warp, MMA warp of row block 0, 4 softmax warps per block, (last) the MMA warp of row block 1; then the converter warps
+    static constexpr int THREADS = (2 + 4 * NBLK + (NBLK - 1) + CONV_WARPS) * 32;
+    static constexpr int SMEM_BYTES = 1024 + NBLK * QBLK_BYTES + STAGES * STAGE_BYTES + CODE_STAGES * CODE_STAGE_BYTES + 512;
     // TMEM columns of row block b: S[2] at b*256 + {0, 64}; O at b*256 + 128 (D columns)
     static constexpr int COL_BLK = 256, COL_O = 128;
     static constexpr int TMEM_COLS = NBLK == 2 ? 512 : 256;
     static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+    static_assert(!F8 || (NBLK == 1 && D == 128), "compressed-resident chunks: head_dim 128, one row block per CTA");
 };
 
 // barrier slots (8 bytes each)
 constexpr int kBarFull = 0, kBarEmpty = 4, kBarSFull = 8 /* [blk][2] */, kBarPReady = 12 /* [blk][2] */,
-              kBarODone = 16 /* [blk][2] */, kBarQReady = 20, kBarCount = 21;
+              kBarODone = 16 /* [blk][2] */, kBarQReady = 20, kBarCodeFull = 21 /* [3] */, kBarCodeEmpty = 24 /* [3] */, kBarCount = 27;
 
-template <int D, int G, int NBLK>
-__global__ void __launch_bounds__((2 + 4 * NBLK + (NBLK - 1)) * 32, 1)
+template <int D, int G, int NBLK, bool F8 = false>
+__global__ void __launch_bounds__(Cfg<D, NBLK, F8>::THREADS, 1)
 k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap kn_map, const __grid_constant__ CUtensorMap vn_map) {
-    using C = Cfg<D, NBLK>;
+    using C = Cfg<D, NBLK, F8>;
     constexpr int kStages = C::STAGES;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char *q_s = smem;                                   // [NBLK][NBOX boxes][128 rows][128 B]
     unsigned char *kv_s = q_s + NBLK * C::QBLK_BYTES;            // kStages x (K boxes, V boxes)
-    uint64_t *bars = (uint64_t *)(kv_s + kStages * C::STAGE_BYTES);
+    unsigned char *code_s = kv_s + kStages * C::STAGE_BYTES;     // CODE_STAGES x (K codes, V codes, exponent record)
+    uint64_t *bars = (uint64_t *)(code_s + C::CODE_STAGES * C::CODE_STAGE_BYTES);
     uint32_t *tmem_slot = (uint32_t *)(bars + kBarCount);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 2);
+    volatile int *v_kmajor = abort_flag + 1;                     // [kStages] 1: the stage's V is stored [d][token] (expanded codes)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // which unit
@@ -297,6 +335,11 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             mbar_init(p_ready + s * 8, 128);
         }
         for (int s = 0; s < 4; ++s) mbar_init(o_done + s * 8, 1);
+        for (int s = 0; s < 3; ++s) {
+            mbar_init(bar0 + (kBarCodeFull + s) * 8, 1);
+            mbar_init(bar0 + (kBarCodeEmpty + s) * 8, 1);
+        }
+        for (int s = 0; s < kStages; ++s) v_kmajor[s] = 0;
         mbar_init(q_ready, 128 * NBLK);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -314,16 +357,19 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
     const uint32_t tmem = *tmem_slot;
 
     // tile lookup shared by the producer and the softmax threads
-    auto tile_at = [&](int t, int &seg, int &tiles_before, int &seg_tiles, int &seg_len) {
+    auto tile_at = [&](int t, int &seg, int &tiles_before, int &seg_tiles, int &seg_len, int &seg_fmt) {
         Tile ti;
+        ti.fmt = 0;
         if (t < rq.chunk_tiles) {
             while (seg < 0 || t >= tiles_before + seg_tiles) {
                 tiles_before += seg_tiles;
                 ++seg;
-                seg_len = p.segs[rq.seg_begin + seg].len;
+                const DevSeg sg = p.segs[rq.seg_begin + seg];
+                seg_len = sg.len;
+                seg_fmt = F8 ? sg.fmt : 0;
                 seg_tiles = cdiv(seg_len, kTile);
             }
-            ti.kind = 0; ti.seg = seg; ti.seg_len = seg_len;
+            ti.kind = 0; ti.seg = seg; ti.seg_len = seg_len; ti.fmt = seg_fmt;
             ti.r0 = (t - tiles_before) * kTile;
             ti.rows = min(kTile, seg_len - ti.r0);
         } else if (t < rq.chunk_tiles + tail_tiles) {
@@ -358,16 +404,42 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 }
             }
         };
-        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
+        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0, seg_fmt = 0;
+        int n_code = 0;   // code tiles issued so far (their staging ring has a sequence of its own)
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
             const int st = j % kStages, use = j / kStages;
+            const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len, seg_fmt);
+            if constexpr (F8) {
+                if (ti.kind == 0 && ti.fmt == 1) {
+                    // a tile of codes goes to the staging ring; the converter warps expand it into operand stage `st`
+                    // (they wait for that stage to be free themselves)
+                    const int cst = n_code % C::CODE_STAGES, cuse = n_code / C::CODE_STAGES;
+                    ++n_code;
+                    if (cuse > 0) ok = mbar_wait(bar0 + (kBarCodeEmpty + cst) * 8, (cuse - 1) & 1, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        const DevSeg sg = p.segs[rq.seg_begin + ti.seg];
+                        const int st_tiles = cdiv(ti.seg_len, kTile);
+                        const int64_t blk = ((int64_t)layer * p.Hkv + g) * st_tiles + ti.r0 / kTile;
+                        const int64_t region = ((int64_t)p.n_layers_total * p.Hkv * st_tiles * kTile * D + 255) / 256 * 256;
+                        const CUtensorMap *m8 = p.tmaps8 + 2 * (rq.seg_begin + ti.seg);
+                        const uint32_t cdst = smem_u32(code_s + cst * C::CODE_STAGE_BYTES), cbar = bar0 + (kBarCodeFull + cst) * 8;
+                        mbar_expect_tx(cbar, 2 * C::CODE_BYTES + 16);
+                        tma_load_2d(cdst, m8, 0, (int32_t)(blk * kTile), cbar);
+                        tma_load_2d(cdst + C::CODE_BYTES, m8 + 1, 0, (int32_t)(blk * D), cbar);
+                        bulk_load(cdst + 2 * C::CODE_BYTES, (const unsigned char *)sg.base + 2 * region + blk * 16, 16, cbar);
+                    }
+                    continue;
+                }
+            }
             if (use > 0) ok = mbar_wait(empty_kv + st * 8, (use - 1) & 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len);
             const uint32_t dst = smem_u32(kv_s + st * C::STAGE_BYTES), bar = full_kv + st * 8;
             if (lane == 0) {
+                if constexpr (F8) v_kmajor[st] = 0;   // (ordered before the consumers' look by the barrier's release / acquire)
                 mbar_expect_tx(bar, C::STAGE_BYTES);
                 if (ti.kind < 2) {
                     const CUtensorMap *mk, *mv;
@@ -400,7 +472,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
         // tile load of the CTA has been issued.  Issued between two tile loads it held the second one back by its whole
         // duration (measured: 30 us per CTA on a 1,024-token suffix).
         append_share();
-    } else if (warp == 1 || warp == 2 + 4 * NBLK) {
+    } else if (warp == 1 || (NBLK == 2 && warp == 2 + 4 * NBLK)) {
         // ===================== MMA issuers: one warp per row block =====================
         // The whole warp walks the loop (waits and descriptor arithmetic on warp-uniform values); one elected lane
         // issues the MMAs and their commits.  With a single lane behind a divergent branch every tcgen05.mma cost
@@ -411,7 +483,7 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
         {
             const int blk = warp == 1 ? 0 : 1;
             constexpr uint32_t idesc_qk = instr_desc(kRowsPerCta, kTile, false);
-            constexpr uint32_t idesc_pv = instr_desc(kRowsPerCta, D, true);
+            constexpr uint32_t idesc_pv = instr_desc(kRowsPerCta, D, true), idesc_pv_k = instr_desc(kRowsPerCta, D, false);
             const uint32_t q_lo = desc_lo(smem_u32(q_s) + blk * C::QBLK_BYTES, 0), kv_u32 = smem_u32(kv_s);
             const uint32_t tm = tmem + blk * C::COL_BLK;
             bool ok = __all_sync(0xffffffffu, mbar_wait(q_ready, 0, abort_flag));
@@ -419,11 +491,15 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 const int bf = t & 1, st = t % kStages;
                 if (!__all_sync(0xffffffffu, mbar_wait(p_ready + (blk * 2 + bf) * 8, (t >> 1) & 1, abort_flag))) return false;
                 tc_fence_after();
-                const uint32_t v_lo = desc_lo(kv_u32 + st * C::STAGE_BYTES + C::KV_BYTES, C::BOX_BYTES);
+                // V as stored, [token][d] (MN-major: 16 tokens = 16 rows of 128 bytes per step), or, expanded from codes,
+                // V^T [d][token] (K-major like K: 16 tokens = 32 bytes per step)
+                const bool vk = F8 && v_kmajor[st] != 0;
+                const uint32_t v_lo = desc_lo(kv_u32 + st * C::STAGE_BYTES + C::KV_BYTES, vk ? 0 : C::BOX_BYTES);
+                const uint32_t v_step = vk ? (32 >> 4) : (2048 >> 4), idesc_v = vk ? idesc_pv_k : idesc_pv;
                 if (elect_one()) {
 #pragma unroll
-                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 8 TMEM columns (in S's place), V 16 rows of 128 bytes
-                        umma_ta(tm + C::COL_O, tm + bf * kTile + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+                    for (int ks = 0; ks < kTile / 16; ++ks)  // 16 tokens per MMA: P advances 8 TMEM columns (in S's place)
+                        umma_ta(tm + C::COL_O, tm + bf * kTile + ks * 8, v_lo + ks * v_step, idesc_v, (t > 0 || ks > 0) ? 1u : 0u);
                     umma_commit(o_done + (blk * 2 + bf) * 8);
                     umma_commit(empty_kv + st * 8);
                 }
@@ -447,6 +523,58 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                 if (j >= 1) ok = do_pv(j - 1);
             }
             if (ok && n_tiles > 0) do_pv(n_tiles - 1);
+        }
+    } else if (F8 && warp >= 2 + 4 * NBLK + (NBLK - 1)) {
+        // ===================== converter warps: tiles of codes -> bf16 operand tiles =====================
+        if constexpr (F8) {
+            const int ct = tid - (2 + 4 * NBLK + (NBLK - 1)) * 32;   // 0..127
+            int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0, seg_fmt = 0, n_code = 0;
+            bool ok = true;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len, seg_fmt);
+                if (!(ti.kind == 0 && ti.fmt == 1)) continue;
+                const int st = j % kStages, use = j / kStages;
+                const int cst = n_code % C::CODE_STAGES, cuse = n_code / C::CODE_STAGES;
+                ++n_code;
+                ok = mbar_wait(bar0 + (kBarCodeFull + cst) * 8, cuse & 1, abort_flag);
+                if (ok && use > 0) ok = mbar_wait(empty_kv + st * 8, (use - 1) & 1, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const unsigned char *cs_ = code_s + cst * C::CODE_STAGE_BYTES;
+                unsigned char *ks_ = kv_s + st * C::STAGE_BYTES;
+                const int ek = (int)*(const signed char *)(cs_ + 2 * C::CODE_BYTES), ev = (int)*(const signed char *)(cs_ + 2 * C::CODE_BYTES + 1);
+                const float sk = __uint_as_float(ek > -127 ? (uint32_t)(ek + 127) << 23 : 0x00400000u);   // 2^e (2^-127 is a subnormal float)
+                const float sv = __uint_as_float(ev > -127 ? (uint32_t)(ev + 127) << 23 : 0x00400000u);
+#pragma unroll
+                for (int i = 0; i < kTile * D / 16 / 128; ++i) {
+                    // K: row t of 128 codes (128-byte swizzle); 16 codes = dimensions 16c .. 16c+15 -> two 16-byte chunks of bf16
+                    const int q = ct + 128 * i, t = q >> 3, c = q & 7;
+                    const uint4 w = *(const uint4 *)(cs_ + t * 128 + ((c ^ (t & 7)) << 4));
+                    uint4 lo, hi;
+                    expand16(w, sk, lo, hi);
+                    unsigned char *row = ks_ + (c >> 2) * C::BOX_BYTES + t * 128;
+                    *(uint4 *)(row + ((((2 * c) & 7) ^ (t & 7)) << 4)) = lo;
+                    *(uint4 *)(row + ((((2 * c + 1) & 7) ^ (t & 7)) << 4)) = hi;
+                }
+#pragma unroll
+                for (int i = 0; i < kTile * D / 16 / 128; ++i) {
+                    // V^T: row d of 64 codes (64-byte swizzle); 16 codes = tokens 16c .. 16c+15 -> two chunks of the [d][token] tile
+                    const int q = ct + 128 * i, d = q >> 2, c = q & 3;
+                    const uint4 w = *(const uint4 *)(cs_ + C::CODE_BYTES + d * 64 + ((c ^ ((d >> 1) & 3)) << 4));
+                    uint4 lo, hi;
+                    expand16(w, sv, lo, hi);
+                    unsigned char *row = ks_ + C::KV_BYTES + d * 128;
+                    *(uint4 *)(row + (((2 * c) ^ (d & 7)) << 4)) = lo;
+                    *(uint4 *)(row + (((2 * c + 1) ^ (d & 7)) << 4)) = hi;
+                }
+                fence_async_smem();                                   // the tensor core reads these tiles through the async proxy
+                asm volatile("bar.sync 2, 128;" ::: "memory");        // the four converter warps
+                if (ct == 0) {
+                    v_kmajor[st] = 1;
+                    mbar_arrive(full_kv + st * 8);                    // the operand stage holds tile j
+                    mbar_arrive(bar0 + (kBarCodeEmpty + cst) * 8);    // the code stage may be refilled
+                }
+            }
         }
     } else {
         // ===================== softmax threads: one query row each =====================
@@ -473,14 +601,14 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
         // l_rnd: the same sum over the bf16-rounded numerators the tensor core really multiplies with V; O is
         // normalised by it (a dominant token's rounding error then cancels), the log-sum-exp uses l_run.
         float m_ref = -CUDART_INF_F, l_run = 0.f, l_rnd = 0.f;
-        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0;
+        int seg = -1, tiles_before = 0, seg_tiles = 0, seg_len = 0, seg_fmt = 0;
         bool ok = true;
         int plain_end = 0;   // tiles before it (of the unit) are full chunk tiles: every column visible, nothing to look up
         for (int j = 0; j < n_tiles && ok; ++j) {
             // visible columns: all valid rows of a chunk / tail tile; causal inside the new tokens
             int n_vis = kTile;
             if (t_begin + j >= plain_end) {
-                const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len);
+                const Tile ti = tile_at(t_begin + j, seg, tiles_before, seg_tiles, seg_len, seg_fmt);
                 n_vis = ti.rows;
                 if (ti.kind == 2) n_vis = min(ti.rows, tok - ti.r0 + 1);
                 if (ti.kind == 0) plain_end = tiles_before + seg_len / kTile;
@@ -619,16 +747,16 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
 
 }  // namespace k3
 
-template <int D, int G, int NBLK>
+template <int D, int G, int NBLK, bool F8 = false>
 static int launch_k3(const k3::Params &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int grid, cudaStream_t stream) {
-    using C = k3::Cfg<D, NBLK>;
+    using C = k3::Cfg<D, NBLK, F8>;
     static PerDeviceOnce configured;
     int once_dev;
     if (configured.need(&once_dev)) {
-        MATKV_CUDA(cudaFuncSetAttribute(k3::k_prefill_tc<D, G, NBLK>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        MATKV_CUDA(cudaFuncSetAttribute(k3::k_prefill_tc<D, G, NBLK, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
         configured.mark(once_dev);
     }
-    k3::k_prefill_tc<D, G, NBLK><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
+    k3::k_prefill_tc<D, G, NBLK, F8><<<grid, C::THREADS, C::SMEM_BYTES, stream>>>(p, kn_map, vn_map);
     MATKV_CUDA(cudaGetLastError());
     return MATKV_OK;
 }
@@ -637,7 +765,7 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     const matkv_config &c = ctx->cfg;
     const int G = c.n_q_heads / c.n_kv_heads, D = c.head_dim;
     k3::Params p;
-    p.reqs = t->d_reqs; p.segs = t->d_segs; p.tmaps = t->d_tmaps; p.n_seg_total = t->n_seg_total;
+    p.reqs = t->d_reqs; p.segs = t->d_segs; p.tmaps = t->d_tmaps; p.tmaps8 = t->d_tmaps8; p.n_seg_total = t->n_seg_total;
     p.tail_len = t->d_tail_len; p.tail_k = t->tail_k; p.tail_v = t->tail_v;
     p.q = a.q; p.k_new = a.k_new; p.v_new = a.v_new; p.out = a.out; p.lse_out = a.lse_out;
     p.q_sl = a.q_sl; p.q_sb = a.q_sb; p.q_ss = a.q_ss; p.kn_sl = a.kn_sl; p.kn_sb = a.kn_sb; p.kn_ss = a.kn_ss;
@@ -647,7 +775,8 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
     // enough CTAs to fill most of the SMs (otherwise one block per CTA and more KV splits)
     const int R = a.S * G;
     const bool fill = (int64_t)a.n_layers_launch * t->batch * c.n_kv_heads * ((R + 255) / 256) * 10 >= 6 * (int64_t)ctx->n_sm;
-    const int nblk = (R > k3::kRowsPerCta && (fill || ctx->opt_prefill_impl == 3)) ? 2 : 1;
+    // (tables with compressed-resident chunks: one row block per CTA, the converter warps take the other block's place)
+    const int nblk = (!t->has_fp8 && R > k3::kRowsPerCta && (fill || ctx->opt_prefill_impl == 3)) ? 2 : 1;
     p.n_rb = (a.S * G + nblk * k3::kRowsPerCta - 1) / (nblk * k3::kRowsPerCta);
     p.scale_log2 = ctx->scale * k3::kLog2e;
     p.status = ctx->d_status;
@@ -677,6 +806,16 @@ int launch_prefill_tc(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, cudaS
         if (rc2) return rc2;
     }
     int rc = fail(MATKV_E_INVALID_ARG, "tensor-core prefill: unsupported head_dim %d / group %d", D, G);
+    if (t->has_fp8) {
+#define MATKV_CASE8(GG) \
+        if (D == 128 && G == GG) rc = launch_k3<128, GG, 1, true>(p, kn_map, vn_map, (int)grid, stream);
+        MATKV_CASE8(1) MATKV_CASE8(2) MATKV_CASE8(4) MATKV_CASE8(8)
+#undef MATKV_CASE8
+        if (rc) return rc;
+        if (p.n_split > 1)
+            return launch_lse_combine(ctx, (int32_t)rows, p.n_split, D, p.part_o, p.part_lse, a.out, a.lse_out, stream);
+        return MATKV_OK;
+    }
 #define MATKV_CASE(DD, GG) \
     if (D == DD && G == GG) rc = nblk == 2 ? launch_k3<DD, GG, 2>(p, kn_map, vn_map, (int)grid, stream) : launch_k3<DD, GG, 1>(p, kn_map, vn_map, (int)grid, stream);
     MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)

@@ -203,30 +203,35 @@ def test_compressed_resident_chunks_attend_like_the_oracle(Hq, Hkv):
     sess.close()
 
 
-@pytest.mark.parametrize("ctas", [0, 1000])
-def test_compressed_resident_chunks_suffix_of_two_new_token_tiles(ctas):
-    """A 70-token suffix over compressed-resident chunks (two tiles of new tokens per token block; with one CTA per
-    tile the second tile is an empty part for the blocks of early tokens)."""
+@pytest.mark.parametrize("impl,ctas,splits", [(1, 0, 0), (1, 1000, 0), (2, 0, 0), (2, 0, 1), (2, 0, 3)])
+def test_compressed_resident_chunks_suffix_of_two_new_token_tiles(impl, ctas, splits):
+    """A 70-token suffix over compressed-resident chunks, on the streaming kernel (two tiles of new tokens per token
+    block; with one CTA per tile the second tile is an empty part for the blocks of early tokens) and on the tensor-core
+    tile kernel, whose converter warps expand the code tiles to bf16 operand tiles in shared memory (one and several KV
+    splits: 280 query rows per KV head in three row blocks)."""
     import paper_2512_22195_b200 as mk
     from paper_2512_22195_b200.harness import Session, bits_to_dev, dev_to_bits
     L, Hq, Hkv, D, S = 1, 8, 2, 128, 70
-    lens = [130, 64]
-    sess = Session(L, Hq, Hkv, D, 1, 2, S + 2)
+    lens = [130, 64, 33, 500]
+    sess = Session(L, Hq, Hkv, D, 1, 4, S + 2)
     mk.matkv_set_option(sess.ctx, mk.OPT_FP8_RESIDENT, 1)
+    mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_IMPL, impl)
     if ctas:
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_CTAS, ctas)
+    if splits:
+        mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_CTAS, splits)
     sh = oracle.Shape(L, Hq, Hkv, D)
     vals, keep = [], []
     for cid, n in enumerate(lens):
-        codes, exps = oracle.fp8_quantize_blob(sh, rand_bits(75, cid, (L, 2, Hkv, n, D)))
+        codes, exps = oracle.fp8_quantize_blob(sh, rand_bits(75, cid, (L, 2, Hkv, n, D), cid - 3))   # scales 1/8 .. 1: different block exponents
         vals.append(oracle.fp8_dequantize_blob(sh, codes, exps))
         host = torch.from_numpy(_fp8_blob_np(sess, mk, codes, exps)).pin_memory()
         keep.append(host)
         mk.matkv_register_chunk_fp8(sess.ctx, cid, n, host.data_ptr())
     slot_bytes = (L * 2 * Hkv * max(lens) * D * 2 + 255) // 256 * 256
-    slots = torch.zeros(2 * slot_bytes, dtype=torch.uint8, device="cuda")
-    sess.stage([0, 1], slots, slot_bytes, torch.cuda.Stream())
-    sess.build_table([[0, 1]])
+    slots = torch.zeros(4 * slot_bytes, dtype=torch.uint8, device="cuda")
+    sess.stage([0, 1, 2, 3], slots, slot_bytes, torch.cuda.Stream())
+    sess.build_table([[0, 1, 2, 3]])
     rq = oracle.Request(sh, vals, S + 2)
     q, k, v = (rand_bits(75, 10 + i, (1, S, Hq if i == 0 else Hkv, D)) for i in range(3))
     out, lse = sess.prefill(0, bits_to_dev(q), bits_to_dev(k), bits_to_dev(v))
