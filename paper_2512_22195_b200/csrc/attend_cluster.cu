@@ -78,8 +78,17 @@ __device__ __forceinline__ void cl_stamp(int layer, int point) {
     if (layer < 64 && blockIdx.x < 160) g_cl_stamps[layer][blockIdx.x][point] = t;
 }
 #define CL_STAMP(point) cl_stamp(p.layer, point)
+// per-tile stamps: [layer][CTA][kind: 0 issued, 1 seen landed, 2 consumed][tile]
+__device__ unsigned long long g_cl_tiles[64][160][3][8];
+__device__ __forceinline__ void cl_tile_stamp(int layer, int kind, int tile) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (layer < 64 && blockIdx.x < 160 && tile < 8) g_cl_tiles[layer][blockIdx.x][kind][tile] = t;
+}
+#define CL_TILE(kind, tile) cl_tile_stamp(p.layer, kind, tile)
 #else
 #define CL_STAMP(point)
+#define CL_TILE(kind, tile)
 #endif
 
 // ---- cluster / distributed shared memory helpers ---------------------------------------------------
@@ -241,6 +250,7 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
                     tma_load_2d_hint(dst + (C::NBOX + bx) * C::BOX_BYTES, m, bx * 64, yv, bar, pol);
                 }
                 if (j == 0) CL_STAMP(1);
+                CL_TILE(0, j);
             }
             // tail rows and the step's new token were written by earlier kernels on the stream
             CL_GDC_WAIT();
@@ -263,6 +273,7 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
                         tma_load_2d_hint(dst + bx * C::BOX_BYTES, mk, bx * 64, y, bar, pol_n);
                         tma_load_2d_hint(dst + (C::NBOX + bx) * C::BOX_BYTES, mv, bx * 64, y, bar, pol_n);
                     }
+                    CL_TILE(0, (int)seq);
                 }
                 if (s.has_new && ok) {
                     uint32_t stage, bar, dst;
@@ -274,6 +285,7 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
                             tma_load_3d(dst + bx * C::BOX_BYTES, &kn_map, bx * 64, g, b, bar);
                             tma_load_3d(dst + (C::NBOX + bx) * C::BOX_BYTES, &vn_map, bx * 64, g, b, bar);
                         }
+                        CL_TILE(0, (int)seq);
                         ++seq;
                     }
                 }
@@ -300,13 +312,13 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
     const int mi = lane >> 3, ri = lane & 7;   // ldmatrix addressing
     CL_GDC_WAIT();   // q, the tail length and the tail rows come from earlier kernels
     if (tid == 0) CL_STAMP(3);
-    int32_t t0 = p.tail_len[b];
-    if (t0 < 0 || t0 + 1 > p.max_tail) {
-        if (tid == 0) atomicCAS(p.status, 0, MATKV_E_CAPACITY);
-        t0 = max(0, min(t0, p.max_tail - 1));
-    }
-    const ClShare sh = cl_share(ct, p.tt_nom, cs, rank, ceil_div(t0, kTile));
-    const int n_mine = sh.n_chunk + sh.n_tail + sh.has_new;
+    // The chunk part of the share is known from the launch parameters; how many tail tiles follow depends on the device's
+    // tail length, which is requested now and first looked at when the chunk tiles are done (a dependent load less in
+    // front of the first tile).
+    const int32_t t0_dev = p.tail_len[b];
+    int32_t t0 = 0;
+    int n_mine = cl_share(ct, p.tt_nom, cs, rank, 0).n_chunk;
+    bool tail_known = false;
 
     // Q^T as the B operand of S^T = K Q^T: column n = tq is query row tq, k = the 16 dimensions of a k-step
     uint32_t qb[C::KS][2];
@@ -328,11 +340,24 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
     float m_run[2] = {-CUDART_INF_F, -CUDART_INF_F}, l_run[2] = {0.f, 0.f}, l_rnd[2] = {0.f, 0.f};
     const int r0 = (warp & 3) * kItemRows;   // this warp's 16 tokens of its tiles
 
-    for (int j = warp >> 2; j < n_mine; j += 2) {
+    for (int j = warp >> 2;; j += 2) {
+        if (j >= n_mine) {
+            if (tail_known) break;
+            tail_known = true;
+            t0 = t0_dev;
+            if (t0 < 0 || t0 + 1 > p.max_tail) {
+                if (tid == 0) atomicCAS(p.status, 0, MATKV_E_CAPACITY);
+                t0 = max(0, min(t0, p.max_tail - 1));
+            }
+            const ClShare sh = cl_share(ct, p.tt_nom, cs, rank, ceil_div(t0, kTile));
+            n_mine = sh.n_chunk + sh.n_tail + sh.has_new;
+            if (j >= n_mine) break;
+        }
         const uint32_t stage = j % kClStages, use = j / kClStages;
         // (after a bounded wait ran out the loop goes on without computing: every lane of the warp takes the same path)
         const uint32_t tag = __shfl_sync(0xffffffffu, stage_wait(tags + stage, use, full_u32 + stage * 8, use & 1, flags), 0);   // 0: gave up
         if (tid == 0 && j == 0) CL_STAMP(4);
+        if (lane == 0 && (warp & 3) == 0) CL_TILE(1, j);
         const uint32_t stage_u32 = ring_u32 + stage * C::STAGE_BYTES;
         const int rows = (int)(tag & 0x7f) - r0;   // valid tokens of this warp's piece (may be <= 0)
         if (rows > 0) {
@@ -400,6 +425,7 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_u32 + stage * 8);
+        if (lane == 0 && (warp & 3) == 0) CL_TILE(2, j);
     }
 
     // ---- the warps' states are merged through shared memory (the ring is free: every tile has been consumed) ----
@@ -649,5 +675,8 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
 #ifdef MATKV_STAMPS
 extern "C" int matkv_debug_cluster_stamps(unsigned long long *host_out) {
     return (int)cudaMemcpyFromSymbol(host_out, matkv::g_cl_stamps, sizeof(matkv::g_cl_stamps));
+}
+extern "C" int matkv_debug_cluster_tiles(unsigned long long *host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, matkv::g_cl_tiles, sizeof(matkv::g_cl_tiles));
 }
 #endif
