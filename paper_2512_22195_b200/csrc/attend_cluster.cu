@@ -638,6 +638,10 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
     if (W >= 32 * grid_max) return MATKV_OK;   // long launches stream best through the persistent kernel
     int cs = 1;
     while (cs * 2 <= kClMaxCs && (int64_t)n_units * cs * 2 <= grid_max && c.head_dim / (cs * 2) >= 4 && cs * 2 <= min_tiles) cs *= 2;
+    // Measured (8B and 70B head shapes, 5 x 1,024-token chunks per request, launches replayed from a graph): with up to
+    // ~20 tiles per CTA the clusters win (B = 1: 9.4 against 11.9 us, B = 2: 12.5 / 15.3, B = 4: 19.2 / 21.5); with 41 tiles
+    // per CTA (B = 6: clusters of 2) the streaming kernel's deeper ring does (30.1 / 27.9).
+    if (W > 24 * (int64_t)n_units * cs) return MATKV_OK;
     ClusterParams p;
     p.tile_dir = t->d_tile_dir;
     p.tmaps = t->d_tmaps;
