@@ -24,13 +24,15 @@
 
 namespace matkv {
 
+constexpr int kFailWords = 256;   // staging calls whose failure words are live at once
+
 struct IoJob {
     int fd;
     uint64_t offset;
     size_t bytes;
     int slab;
     uint64_t use;  // how many times the slab was used before this job
-    std::shared_ptr<std::atomic<int>> failed;  // the staging call's failure flag
+    std::shared_ptr<FailFlag> failed;  // the staging call's failure flag
 };
 
 struct IoEngine {
@@ -46,7 +48,7 @@ struct IoEngine {
     bool stop = false;
     int errors = 0;
     char last_error[256] = "";
-    int *h_flag = nullptr;   // page-locked word the device can read: non-zero once any read has failed
+    int *h_flag = nullptr;   // kFailWords page-locked words the device can read, one per staging call in flight (ticket mod kFailWords)
     std::atomic<int64_t> timeout_ms{30000}, test_delay_ms{0};
 };
 
@@ -55,11 +57,13 @@ __global__ void k_io_flag(const volatile int *host_flag, int32_t *status) {
     if (*host_flag) atomicCAS(status, 0, MATKV_E_IO);
 }
 
-static void note_failure(IoEngine *e, const std::shared_ptr<std::atomic<int>> &failed, const char *msg) {  // e->m held
+static void note_failure(IoEngine *e, const std::shared_ptr<FailFlag> &failed, const char *msg) {  // e->m held
     ++e->errors;
     snprintf(e->last_error, sizeof e->last_error, "%s", msg);
-    if (failed) failed->store(1, std::memory_order_release);
-    if (e->h_flag) *(volatile int *)e->h_flag = 1;
+    if (failed) {
+        failed->host.store(1, std::memory_order_release);
+        if (failed->word) *failed->word = 1;
+    }
 }
 
 static void io_worker(IoEngine *e) {
@@ -113,7 +117,7 @@ struct IoCallback {
     IoEngine *e;
     int slab;
     uint64_t use;
-    std::shared_ptr<std::atomic<int>> failed;
+    std::shared_ptr<FailFlag> failed;
 };
 
 // Runs in stream order before the copy out of the slab.  The wait has a limit: a read that does not return
@@ -152,12 +156,12 @@ int io_engine_create(matkv_ctx *ctx, void *pinned, size_t bytes, size_t slab_byt
     e->test_delay_ms = ctx->opt_io_test_delay_ms;
     {
         DeviceGuard guard(ctx->device);
-        cudaError_t err = cudaHostAlloc((void **)&e->h_flag, 64, cudaHostAllocMapped | cudaHostAllocPortable);
+        cudaError_t err = cudaHostAlloc((void **)&e->h_flag, kFailWords * sizeof(int), cudaHostAllocMapped | cudaHostAllocPortable);
         if (err != cudaSuccess) {
             delete e;
             return cuda_fail(err, "cudaHostAlloc(read-failure flag)");
         }
-        *e->h_flag = 0;
+        memset(e->h_flag, 0, kFailWords * sizeof(int));
     }
     for (int i = 0; i < n_threads; ++i) e->threads.emplace_back(io_worker, e);
     ctx->io = e;
@@ -184,9 +188,15 @@ void io_engine_configure(matkv_ctx *ctx) {
     ctx->io->test_delay_ms = ctx->opt_io_test_delay_ms;
 }
 
-int io_engine_flag_status(matkv_ctx *ctx, cudaStream_t copy_stream) {
-    if (!ctx->io || !ctx->io->h_flag) return MATKV_OK;
-    k_io_flag<<<1, 1, 0, copy_stream>>>(ctx->io->h_flag, ctx->d_status);
+void io_engine_bind_fail_word(matkv_ctx *ctx, uint64_t ticket, FailFlag *flag) {
+    if (!ctx->io || !ctx->io->h_flag) return;
+    flag->word = ctx->io->h_flag + ticket % kFailWords;
+    *flag->word = 0;
+}
+
+int io_engine_flag_status(matkv_ctx *ctx, const std::shared_ptr<FailFlag> &failed, cudaStream_t copy_stream) {
+    if (!ctx->io || !failed || !failed->word) return MATKV_OK;
+    k_io_flag<<<1, 1, 0, copy_stream>>>(failed->word, ctx->d_status);
     MATKV_CUDA(cudaGetLastError());
     return MATKV_OK;
 }
@@ -213,7 +223,7 @@ static void release_on_host(IoEngine *e, int slab, uint64_t use) {
 
 // Enqueues: read (worker threads) -> [copy stream] wait for the read, copy slab -> dst, release the slab.
 int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream,
-                    const std::shared_ptr<std::atomic<int>> &failed, int32_t fp8_tokens, bool fp8_resident) {
+                    const std::shared_ptr<FailFlag> &failed, int32_t fp8_tokens, bool fp8_resident) {
     IoEngine *e = ctx->io;
     if (!e) return fail(MATKV_E_INVALID_ARG, "file-backed chunk: no bounce buffer set (matkv_set_bounce_buffer)");
     if (bytes > e->slab_bytes)

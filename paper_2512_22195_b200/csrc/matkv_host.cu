@@ -177,7 +177,7 @@ static void retire_ticket(matkv_ctx *ctx, std::unordered_map<uint64_t, Ticket>::
         auto c = ctx->chunks.find(id);
         if (c != ctx->chunks.end() && c->second.ticket == it->first) c->second.ready = nullptr;
     }
-    if (tk.io_failed && tk.io_failed->load(std::memory_order_acquire)) {
+    if (tk.io_failed && tk.io_failed->host.load(std::memory_order_acquire)) {
         if (ctx->failed_tickets.size() >= 1024) ctx->failed_tickets.erase(ctx->failed_tickets.begin());
         ctx->failed_tickets.push_back(it->first);
     }
@@ -566,8 +566,9 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
     retire_finished_tickets(ctx);   // staging calls already seen complete give their events back: the map stays bounded
     Ticket tk;
     MATKV_CUDA(cudaEventCreateWithFlags(&tk.done, cudaEventDisableTiming));
-    tk.io_failed = std::make_shared<std::atomic<int>>(0);
+    tk.io_failed = std::make_shared<FailFlag>();
     const uint64_t ticket = ctx->next_ticket++;
+    io_engine_bind_fail_word(ctx, ticket, tk.io_failed.get());
     int32_t next_free = 0;
     int rc_fail = MATKV_OK;   // a failure part-way: the chunks already touched keep a valid event, then the error is returned
     bool any_file = false;
@@ -623,7 +624,7 @@ int matkv_stage_chunks_async(matkv_ctx *ctx, const uint64_t *ids, int32_t n, voi
         c.io_failed = tk.io_failed;
         tk.chunk_ids.push_back(id);
     }
-    if (any_file) io_engine_flag_status(ctx, cs);   // a read failure of this call shows in the status word once the stream gets here
+    if (any_file) io_engine_flag_status(ctx, tk.io_failed, cs);   // a read failure of this call shows in the status word once the stream gets here
     cudaError_t e_rec = cudaEventRecord(tk.done, cs);
     ctx->tickets.emplace(ticket, tk);
     *ticket_out = ticket;
@@ -714,7 +715,7 @@ int matkv_build_chunk_table(matkv_ctx *ctx, int32_t batch, const int32_t *n_chun
                 return fail(MATKV_E_NOT_STAGED, "request %d: chunk %llu has no device copy (stage it first)", r,
                             (unsigned long long)ids[k]);
             }
-            if (!c.dev_blob && c.io_failed && c.io_failed->load(std::memory_order_acquire)) {
+            if (!c.dev_blob && c.io_failed && c.io_failed->host.load(std::memory_order_acquire)) {
                 delete t;
                 const char *msg = "";
                 io_engine_errors(ctx, &msg);

@@ -58,6 +58,14 @@ struct DevItem {
 struct Region;    // staged slot region
 struct IoEngine;  // reader threads + pinned bounce ring for file-backed chunks
 
+// Failure of a staging call's storage reads: the host's flag, and a page-locked word of the reader engine that a
+// one-thread kernel behind the call's copies looks at (one word per call in flight, so that a later call that went
+// well does not inherit an earlier call's failure).
+struct FailFlag {
+    std::atomic<int> host{0};
+    volatile int *word = nullptr;
+};
+
 struct Chunk {
     int32_t n_tokens = 0;
     const void *host_blob = nullptr;
@@ -74,7 +82,7 @@ struct Chunk {
     cudaEvent_t ready = nullptr;   // event of the staging call that (last) copied it; borrowed from the ticket, null once
                                    // that call has been seen complete (the ticket is retired then and its event destroyed)
     uint64_t ticket = 0;
-    std::shared_ptr<std::atomic<int>> io_failed;  // set by the storage tier when a read of that staging call failed
+    std::shared_ptr<FailFlag> io_failed;  // set by the storage tier when a read of that staging call failed
     alignas(64) CUtensorMap tmap;  // 2-D view [rows][D] of the current device copy, 64 x kTile boxes, 128-byte swizzle
 };
 
@@ -103,7 +111,7 @@ struct PooledImage {  // a table image (pinned upload buffer + device copy) read
 struct Ticket {
     cudaEvent_t done = nullptr;
     std::vector<uint64_t> chunk_ids;              // chunks whose `ready` borrows the event
-    std::shared_ptr<std::atomic<int>> io_failed;  // shared with the storage tier's read jobs of this call
+    std::shared_ptr<FailFlag> io_failed;  // shared with the storage tier's read jobs of this call
 };
 
 }  // namespace matkv
@@ -251,9 +259,11 @@ int io_engine_errors(matkv_ctx *ctx, const char **msg);
 // fp8_tokens > 0: the file holds a compressed chunk of that many tokens; on its way from the slab to dst it is expanded to
 // bf16 (fp8_resident false) or re-laid out into the HBM-resident compressed form (true)
 int io_engine_stage(matkv_ctx *ctx, int fd, uint64_t offset, size_t bytes, void *dst, cudaStream_t copy_stream,
-                    const std::shared_ptr<std::atomic<int>> &failed, int32_t fp8_tokens = 0, bool fp8_resident = false);
+                    const std::shared_ptr<FailFlag> &failed, int32_t fp8_tokens = 0, bool fp8_resident = false);
 // one tiny launch on the copy stream that turns a failed read of the calls so far into MATKV_E_IO in the status word
-int io_engine_flag_status(matkv_ctx *ctx, cudaStream_t copy_stream);
+int io_engine_flag_status(matkv_ctx *ctx, const std::shared_ptr<FailFlag> &failed, cudaStream_t copy_stream);
+// gives a staging call its page-locked failure word (cleared); no-op without a reader engine
+void io_engine_bind_fail_word(matkv_ctx *ctx, uint64_t ticket, FailFlag *flag);
 size_t fp8_codes_bytes(const matkv_config &c, int32_t n_tokens);
 size_t fp8_blob_bytes(const matkv_config &c, int32_t n_tokens);
 int launch_quantize_fp8(matkv_ctx *ctx, const void *dev_blob, int32_t n_tokens, void *dev_fp8, cudaStream_t stream);

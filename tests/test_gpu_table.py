@@ -515,6 +515,7 @@ def test_storage_read_failures_reach_the_attention_path(tmp_path):
     sess.build_table([[2, 0]])
     k, v = sess.gather(0, 0, 2 * n)
     assert np.array_equal(to_bits(k), np.concatenate([blobs[2][0, 0], blobs[0][0, 0]], axis=1))
+    assert sess.status() == 0                                   # a staging call that went well does not inherit the earlier failure
     sess.close()
     del ring
 
