@@ -624,7 +624,8 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
     *taken = false;
     const matkv_config &c = ctx->cfg;
     const int G = c.n_q_heads / c.n_kv_heads;
-    if (a.S != 1 || a.n_layers_launch != 1 || t->has_fp8 || t->batch > kClMaxReq || !t->d_tile_dir || ctx->opt_decode_ctas > 0) return MATKV_OK;
+    // (a launch that is to advance the tail itself stays with the streaming kernel, whose last CTA does that)
+    if (a.S != 1 || a.n_layers_launch != 1 || a.advance != 0 || t->has_fp8 || t->batch > kClMaxReq || !t->d_tile_dir || ctx->opt_decode_ctas > 0) return MATKV_OK;
     const int n_units = t->batch * c.n_kv_heads;
     const int64_t grid_max = std::max<int64_t>(ctx->n_sm - ctx->opt_stage_ctas, ctx->n_sm / 2);
     if (n_units > grid_max) return MATKV_OK;

@@ -162,6 +162,12 @@ def test_decode_launch_that_advances_the_tail_itself(ctas):
     run_requests(2, 8, 2, 128, [[200, 31], [97], []], 3, 5, seed=28, all_layers=True, fused_advance=True, ctas=ctas)
 
 
+def test_decode_launch_that_advances_the_tail_itself_single_layer_model():
+    """With one layer the all-layers launch is a one-layer launch: it must still advance the tail (such a launch stays
+    with the streaming kernel, whose last CTA moves the counter)."""
+    run_requests(1, 8, 2, 128, [[200, 31], [97]], 3, 5, seed=30, all_layers=True, fused_advance=True)
+
+
 @pytest.mark.parametrize("decode_impl,L,lens", [(1, 2, [[130, 64], [200], [64]]), (1, 32, [[1024, 1024, 512]]), (2, 2, [[130, 64], [200], [64]])])
 def test_back_to_back_decode_launches_across_a_tail_tile_boundary(decode_impl, L, lens):
     """Twelve decode steps issued back to back WITHOUT a host synchronisation in between, every launch advancing the
