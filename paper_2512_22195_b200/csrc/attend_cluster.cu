@@ -19,7 +19,7 @@
 //     through movmatrix (an 8 x 8 transpose across the warp); fp32 online softmax per query row; the warps' states
 //     are merged through shared memory at the end;
 //   - the CTAs' partials (o, lse) are exchanged through distributed shared memory as a reduce-scatter: CTA i of the
-//     cluster owns D / CS output columns, every CTA stores that column slice of its partial straight into CTA i's
+//     cluster owns the output column groups (of four) i, i + CS, ..., every CTA stores those groups of its partial straight into CTA i's
 //     shared memory (st.shared::cluster) and announces it on an mbarrier there (remote arrive, release at cluster
 //     scope); every CTA then merges its own slice over the CS parts by log-sum-exp and writes those columns of the
 //     output.  No global partials, no device-wide fence, no atomic ticket, no workspace, and the landing zone of a
@@ -155,9 +155,10 @@ struct ClusterCfg {
     // the warps' states at the end of the CTA's share sit in the ring (all of its tiles have been consumed by then)
     static constexpr int MROW = D + 4;                            // padded row of the merge area (bank spread)
     static constexpr int MERGE_BYTES = kClWarps * kUnitRows * (MROW + 3) * 4;
-    // landing zone: this CTA's column slice of every CTA's partial ([part][row][D / CS] = rows x D floats whatever CS is),
-    // then every CTA's lse per row
-    static constexpr int LAND_BYTES = (kUnitRows * D + kClMaxCs * kUnitRows) * 4;
+    // landing zone: this CTA's column groups of every CTA's partial ([part][row][ceil(D / 4 / CS)] groups of four floats: at
+    // most rows x (D / 4 + CS) groups whatever CS is), then every CTA's lse per row
+    static constexpr int LAND_O_FLOATS = kUnitRows * (D / 4 + kClMaxCs) * 4;
+    static constexpr int LAND_BYTES = (LAND_O_FLOATS + kClMaxCs * kUnitRows) * 4;
     static constexpr int MISC_BYTES = 256;
     static constexpr int SMEM_BYTES = 1024 + RING_BYTES + LAND_BYTES + MISC_BYTES;
     static_assert(MERGE_BYTES <= RING_BYTES, "merge area must fit the ring");
@@ -171,8 +172,8 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // the same offset in every CTA of the cluster
     unsigned char *ring = smem;
-    float *land_o = (float *)(smem + C::RING_BYTES);                // [part][row][D / cs]: this CTA's columns of every partial
-    float *land_lse = land_o + kUnitRows * D;                       // [part][row]
+    float *land_o = (float *)(smem + C::RING_BYTES);                // [part][row][ceil(D / 4 / cs)][4]: this CTA's column groups of every partial
+    float *land_lse = land_o + C::LAND_O_FLOATS;                    // [part][row]
     unsigned char *misc = smem + C::RING_BYTES + C::LAND_BYTES;
     uint64_t *bars = (uint64_t *)misc;                              // full[stages], empty[stages], landing
     volatile uint32_t *tags = (volatile uint32_t *)(misc + 64);     // per stage: valid rows | kTagNew | (number of the stage's current fill) << 16
@@ -465,8 +466,9 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
     if (tid == 0) CL_STAMP(10);
     if (cs > 1) cluster_wait_acquire();   // the start-up barrier: every neighbour's landing zone and barrier exist from here on
     if (tid == 0) CL_STAMP(11);
-    // one (row, four columns) unit per thread and pass; CTA i of the cluster owns columns [i * sw, (i + 1) * sw)
-    const int sw = D / cs;
+    // one (row, group of four columns) unit per thread and pass; column group q belongs to CTA q mod cs of the cluster (any
+    // cluster size works), which keeps it as group q / cs of its landing zone
+    const int ngm = ceil_div(D / 4, cs);   // groups a CTA owns at most
     const uint32_t land_o_u32 = smem_u32(land_o), land_lse_u32 = smem_u32(land_lse);
     for (int idx = tid; idx < n_rows * (D / 4); idx += kClWarps * 32) {
         const int r = idx / (D / 4), d = (idx % (D / 4)) * 4;
@@ -492,9 +494,9 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
             if (p.lse_out && d == 0) p.lse_out[(int64_t)b * p.lse_sb + g * G + r] = lse;
             continue;
         }
-        // these four columns belong to CTA `dst`: into part `rank` of its landing zone (its own slice stays local)
-        const int dst = d / sw;
-        const uint32_t off = (uint32_t)(((rank * n_rows + r) * sw + (d - dst * sw)) * 4);
+        // these four columns belong to CTA `dst`: into part `rank` of its landing zone (its own groups stay local)
+        const int dst = (d / 4) % cs;
+        const uint32_t off = (uint32_t)(((rank * n_rows + r) * ngm + (d / 4) / cs) * 16);
         if (dst == rank) *(float4 *)((unsigned char *)land_o + off) = acc;
         else if (!aborted) st_cluster_f4(map_to_rank(land_o_u32, dst) + off, acc);
         if (d == 0) land_lse[rank * n_rows + r] = lse;   // (sent to the neighbours below)
@@ -514,7 +516,8 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
     }
     // ---- this CTA's columns: merge over the CS parts by log-sum-exp ----
     // every thread that takes part in the merge waits for the neighbours' parts itself (bounded)
-    const int n_items = n_rows * (sw / 2);   // one (row, pair of columns) unit per thread
+    const int ng = (D / 4 - rank + cs - 1) / cs;   // column groups this CTA owns: rank, rank + cs, ...
+    const int n_items = n_rows * ng;               // one (row, group of four columns) unit per thread
     if (tid < n_items || tid == 0) {
         bool got = mbar_try_wait_acquire_cluster(land_u32, 0);
         const long long tw = clock64();
@@ -526,7 +529,7 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
         if (!got) {
             if (tid == 0) atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
         } else if (tid < n_items) {
-            const int r = tid / (sw / 2), d = (tid % (sw / 2)) * 2;
+            const int r = tid / ng, li = tid % ng;
             // the parts' weights w = exp(lse_part - lse_row), formed by every thread for its row (independent loads)
             float lc[kClMaxCs];
             float M = -CUDART_INF_F;
@@ -535,25 +538,24 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
                 lc[c] = c < cs ? land_lse[c * n_rows + r] : -CUDART_INF_F;
                 M = fmaxf(M, lc[c]);
             }
-            float2 acc = make_float2(0.f, 0.f);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             float Z = 0.f;
             if (M != -CUDART_INF_F) {
 #pragma unroll
                 for (int c = 0; c < kClMaxCs; ++c) {
                     if (c < cs && lc[c] != -CUDART_INF_F) {   // an empty part carries no weight, whatever its row holds
                         const float wgt = fast_exp2((lc[c] - M) * kLog2e);
-                        const float2 v = *(const float2 *)(land_o + (c * n_rows + r) * sw + d);
-                        acc.x = fmaf(wgt, v.x, acc.x);
-                        acc.y = fmaf(wgt, v.y, acc.y);
+                        const float4 v = *(const float4 *)(land_o + ((c * n_rows + r) * ngm + li) * 4);
+                        acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y); acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
                         Z += wgt;
                     }
                 }
                 const float inv = 1.f / Z;
-                acc.x *= inv;
-                acc.y *= inv;
+                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
             }
-            *(uint32_t *)(p.out + (int64_t)b * p.q_sb + (int64_t)(g * G + r) * D + rank * sw + d) = pack_bf16(acc.x, acc.y);
-            if (d == 0 && rank == 0 && p.lse_out) p.lse_out[(int64_t)b * p.lse_sb + g * G + r] = Z > 0.f ? M + logf(Z) : -CUDART_INF_F;
+            const int d = (li * cs + rank) * 4;
+            *(uint2 *)(p.out + (int64_t)b * p.q_sb + (int64_t)(g * G + r) * D + d) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+            if (li == 0 && rank == 0 && p.lse_out) p.lse_out[(int64_t)b * p.lse_sb + g * G + r] = Z > 0.f ? M + logf(Z) : -CUDART_INF_F;
         }
     }
     if (tid == 0) CL_STAMP(9);
@@ -586,10 +588,10 @@ static int launch_cluster_t(const ClusterParams &p, const CUtensorMap &kn_map, c
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     // every cluster of the launch must be able to run at once (one wave): asked once per cluster size and device
-    static std::atomic<int> max_clusters[64][5] = {};
-    int dev = 0, slot = 0;
+    static std::atomic<int> max_clusters[64][kClMaxCs + 1] = {};
+    int dev = 0;
+    const int slot = p.cs;
     cudaGetDevice(&dev);
-    for (int c = p.cs; c > 1; c >>= 1) ++slot;
     if (dev >= 0 && dev < 64) {
         int known = max_clusters[dev][slot].load(std::memory_order_acquire);
         if (known == 0) {
@@ -636,13 +638,19 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
         W += (int64_t)c.n_kv_heads * tiles;
         min_tiles = std::min(min_tiles, tiles);
     }
-    if (W >= 32 * grid_max) return MATKV_OK;   // long launches stream best through the persistent kernel
-    int cs = 1;
-    while (cs * 2 <= kClMaxCs && (int64_t)n_units * cs * 2 <= grid_max && c.head_dim / (cs * 2) >= 4 && cs * 2 <= min_tiles) cs *= 2;
-    // Measured (8B and 70B head shapes, 5 x 1,024-token chunks per request, launches replayed from a graph): with up to
-    // ~20 tiles per CTA the clusters win (B = 1: 9.4 against 11.9 us, B = 2: 12.5 / 15.3, B = 4: 19.2 / 21.5); with 41 tiles
-    // per CTA (B = 6: clusters of 2) the streaming kernel's deeper ring does (30.1 / 27.9).
-    if (W > 24 * (int64_t)n_units * cs) return MATKV_OK;
+    if (W >= 96 * grid_max) return MATKV_OK;   // long launches stream best through the persistent kernel
+    // cluster size: as many CTAs per unit as the SMs allow (any size up to 16, not only powers of two)
+    int cs = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kClMaxCs, grid_max / n_units), std::min<int64_t>(min_tiles, c.head_dim / 4)));
+    // Which kernel is faster was measured (8B and 70B head shapes, 5 x 1,024-token chunks per request, B = 1 .. 18,
+    // launches replayed from a graph) and follows a simple model: the streaming kernel takes about 8 us plus 4.95 ns
+    // per tile of the launch (all SMs stream, but a launch cannot start beside its predecessor), this kernel about
+    // 6 us plus 0.65 us per tile of a CTA's share.  Examples (us, this kernel / streaming): B = 1: 9.4 / 12.0,
+    // B = 3 (clusters of 6): 15.4 / 18.4, B = 6 (clusters of 3): 25.6 / 27.8, B = 9 (clusters of 2, 144 CTAs):
+    // 33.6 / 39.0, B = 10 (80 CTAs of one unit each): 53.1 / 41.5, B = 18 (144 CTAs): 61.2 / 65.0.
+    {
+        const double ctas = (double)n_units * cs;
+        if ((double)W * (0.65 / ctas - 0.00495) >= 2.0) return MATKV_OK;
+    }
     ClusterParams p;
     p.tile_dir = t->d_tile_dir;
     p.tmaps = t->d_tmaps;
