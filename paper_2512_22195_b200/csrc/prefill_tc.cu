@@ -619,8 +619,10 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
             if (!ok) break;
             tc_fence_after();
             float s[kTile];
-            {   // both halves in flight before the one wait
-                uint32_t r0[32], r1[32];
+            // the row's 64 scores from tensor memory (warp-collective), masked: ragged or causal tiles (a full tile skips that).
+            // Scores stay raw (unscaled): the scale is folded into the exponent's FMA below.
+            auto load_scores = [&]() {
+                uint32_t r0[32], r1[32];   // both halves in flight before the one wait
                 tmem_ld32_issue(lane_base + bf * kTile, r0);
                 tmem_ld32_issue(lane_base + bf * kTile + 32, r1);
                 tmem_ld_wait();
@@ -629,68 +631,87 @@ k_prefill_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorM
                     s[i] = __uint_as_float(r0[i]);
                     s[32 + i] = __uint_as_float(r1[i]);
                 }
-            }
-            // Scores stay raw (unscaled) here: the scale is folded into the exponent's FMA below.
-            if (n_vis < kTile) {  // ragged or causal tile: mask (a full tile skips this)
+                if (n_vis < kTile) {
 #pragma unroll
-                for (int i = 0; i < kTile; ++i) s[i] = i < n_vis ? s[i] : -CUDART_INF_F;
-            }
-            float tmax;
-            {   // eight independent chains, then a tree: a single chain of 64 dependent maxima costs 250 cycles of latency
-                float mx[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) mx[i] = s[i];
-#pragma unroll
-                for (int i = 8; i < kTile; ++i) mx[i & 7] = fmaxf(mx[i & 7], s[i]);
-                tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
-            }
-            tmax *= p.scale_log2;   // the scale is positive: the maximum commutes with it
-            // lazy rescale: move the reference only when the maximum has grown by more than 2^8
-            const bool grow_ref = tmax > m_ref + 8.0f;   // also true for the first visible column (m_ref = -inf)
-            // o_done has one barrier per parity of the tile index, like S: a waiter is never more than one use of a
-            // barrier behind (the P V of tile j+1 cannot be issued before this thread has delivered P of tile j+1), so
-            // tiles whose completion nobody needs to see are simply not waited for.
-            if (__any_sync(0xffffffffu, grow_ref)) {     // tcgen05.ld / st are warp-collective: decide per warp
-                const float alpha = grow_ref ? (m_ref == -CUDART_INF_F ? 0.f : fast_exp2(m_ref - tmax)) : 1.f;
-                if (j > 0) {
-                    // O of tiles 0..j-1 must be complete before it is scaled
-                    ok = mbar_wait(o_done + (blk * 2 + ((j - 1) & 1)) * 8, ((j - 1) >> 1) & 1, abort_flag);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int c0 = 0; c0 < D; c0 += 32) tmem_scale32(lane_base + C::COL_O + c0, alpha);
-                    tc_fence_before();
+                    for (int i = 0; i < kTile; ++i) s[i] = i < n_vis ? s[i] : -CUDART_INF_F;
                 }
-                if (grow_ref) {
-                    l_run *= alpha;
-                    l_rnd *= alpha;
-                    m_ref = tmax;
-                }
-            }
-            const float m_neg = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
-            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), mn2 = make_float2(m_neg, m_neg);
-            float2 psum2 = make_float2(0.f, 0.f), prnd2 = make_float2(0.f, 0.f);  // packed fp32 pairs: half the adds
-            uint32_t pw[kTile / 2];   // the row's P as bf16 pairs: goes where S was (first 32 columns of the buffer)
+            };
+            load_scores();
+            // The row's numerators against the CURRENT reference maximum: P as bf16 pairs (they go where S was: the first 32
+            // columns of the buffer), their sum and the sum of their roundings.
+            uint32_t pw[kTile / 2];
+            float psum, prnd;
+            auto numerators = [&]() {
+                const float m_neg = m_ref == -CUDART_INF_F ? 0.f : -m_ref;
+                const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), mn2 = make_float2(m_neg, m_neg);
+                float2 psum2 = make_float2(0.f, 0.f), prnd2 = make_float2(0.f, 0.f);  // packed fp32 pairs: half the adds
 #pragma unroll
-            for (int ch = 0; ch < kTile / 8; ++ch) {
-                float e[8];
+                for (int ch = 0; ch < kTile / 8; ++ch) {
+                    float e[8];
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {   // scale and offset as packed pairs: half the FMAs
-                    const float2 x = ffma2(make_float2(s[ch * 8 + 2 * i], s[ch * 8 + 2 * i + 1]), sc2, mn2);
-                    e[2 * i] = fast_exp2(x.x);
-                    e[2 * i + 1] = fast_exp2(x.y);
-                }
-                const uint32_t pk[4] = {pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7])};
+                    for (int i = 0; i < 4; ++i) {   // scale and offset as packed pairs: half the FMAs
+                        const float2 x = ffma2(make_float2(s[ch * 8 + 2 * i], s[ch * 8 + 2 * i + 1]), sc2, mn2);
+                        e[2 * i] = fast_exp2(x.x);
+                        e[2 * i + 1] = fast_exp2(x.y);
+                    }
+                    const uint32_t pk[4] = {pack_bf16(e[0], e[1]), pack_bf16(e[2], e[3]), pack_bf16(e[4], e[5]), pack_bf16(e[6], e[7])};
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    psum2 = fadd2(psum2, make_float2(e[2 * i], e[2 * i + 1]));
-                    prnd2 = fadd2(prnd2, make_float2(__uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u)));
+                    for (int i = 0; i < 4; ++i) {
+                        psum2 = fadd2(psum2, make_float2(e[2 * i], e[2 * i + 1]));
+                        prnd2 = fadd2(prnd2, make_float2(__uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u)));
+                    }
+                    pw[ch * 4] = pk[0]; pw[ch * 4 + 1] = pk[1]; pw[ch * 4 + 2] = pk[2]; pw[ch * 4 + 3] = pk[3];
                 }
-                pw[ch * 4] = pk[0]; pw[ch * 4 + 1] = pk[1]; pw[ch * 4 + 2] = pk[2]; pw[ch * 4 + 3] = pk[3];
+                psum = psum2.x + psum2.y;
+                prnd = prnd2.x + prnd2.y;
+            };
+            // Lazy rescale, decided optimistically.  The reference only has to move when some numerator would exceed 2^8,
+            // and after the first tiles that is rare: the numerators are formed against the reference as it stands, and
+            // only a row sum of 2^8 or more (no numerator can be that large otherwise; an overflow to infinity lands here
+            // too), or a row that has no reference yet, makes the warp look for the row maximum at all.  The 64-way
+            // maximum, which cost a quarter of the row pass, is off the common path.
+            numerators();
+            const bool look = m_ref == -CUDART_INF_F ? n_vis > 0 : !(psum < 256.0f);
+            if (__any_sync(0xffffffffu, look)) {     // tcgen05.ld / st are warp-collective: decide per warp
+                load_scores();   // again (P has not been stored over them yet): the common path need not keep 64 scores alive
+                float tmax = -CUDART_INF_F;
+                if (look) {   // eight independent chains, then a tree: a single chain of 64 dependent maxima costs 250 cycles of latency
+                    float mx[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) mx[i] = s[i];
+#pragma unroll
+                    for (int i = 8; i < kTile; ++i) mx[i & 7] = fmaxf(mx[i & 7], s[i]);
+                    tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])), fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+                    tmax *= p.scale_log2;   // the scale is positive: the maximum commutes with it
+                }
+                // move the reference only when the maximum has grown by more than 2^8
+                const bool grow_ref = look && tmax > m_ref + 8.0f;   // also true for the first visible column (m_ref = -inf)
+                // o_done has one barrier per parity of the tile index, like S: a waiter is never more than one use of a
+                // barrier behind (the P V of tile j+1 cannot be issued before this thread has delivered P of tile j+1), so
+                // tiles whose completion nobody needs to see are simply not waited for.
+                if (__any_sync(0xffffffffu, grow_ref)) {
+                    const float alpha = grow_ref ? (m_ref == -CUDART_INF_F ? 0.f : fast_exp2(m_ref - tmax)) : 1.f;
+                    if (j > 0) {
+                        // O of tiles 0..j-1 must be complete before it is scaled
+                        ok = mbar_wait(o_done + (blk * 2 + ((j - 1) & 1)) * 8, ((j - 1) >> 1) & 1, abort_flag);
+                        ok = __all_sync(0xffffffffu, ok);
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c0 = 0; c0 < D; c0 += 32) tmem_scale32(lane_base + C::COL_O + c0, alpha);
+                        tc_fence_before();
+                    }
+                    if (grow_ref) {
+                        l_run *= alpha;
+                        l_rnd *= alpha;
+                        m_ref = tmax;
+                    }
+                }
+                // again, against the reference as it is now (every lane: the lanes whose reference stayed get the same values,
+                // and nothing of the first pass has to be kept alive across this rare path)
+                numerators();
             }
             tmem_st32(lane_base + bf * kTile, pw);
-            const float psum = psum2.x + psum2.y, prnd = prnd2.x + prnd2.y;
             l_run += psum;
             l_rnd += prnd;
             tc_fence_before();
