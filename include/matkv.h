@@ -113,6 +113,7 @@ typedef struct {
                                       use the streaming kernel either way.  A captured (graph) launch balances its shares for the tail
                                       length at capture time and stays exact as the tail grows; re-capture now and then in a long
                                       generation to keep the balance */
+#define MATKV_OPT_CLUSTER_MAX 12   /* largest cluster (CTAs per request and KV head) the cluster decode may use; 0 (default) = automatic */
 #define MATKV_OPT_IO_TIMEOUT_MS 9  /* storage tier: how long the copy stream waits for one chunk's read before the staging call
                                       is marked failed (MATKV_E_IO) and the stream moves on; default 30,000 ms */
 #define MATKV_OPT_IO_TEST_DELAY_MS 10 /* failure injection on the host, for tests: every storage read sleeps this long first

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(HERE, "libmatkv.so")
 OK, E_INVALID_ARG, E_UNKNOWN_CHUNK, E_NOT_STAGED, E_NOT_READY = 0, -1, -2, -3, -4
 E_CAPACITY, E_ALIGNMENT, E_CUDA, E_TIMEOUT, E_BOUNDS, E_IO = -5, -6, -7, -8, -9, -10
 OPT_DECODE_CTAS, OPT_PREFILL_IMPL, OPT_PREFILL_CTAS, OPT_STAGE_CTAS, OPT_DECODE_ADVANCES_TAIL = 1, 2, 3, 4, 5
-OPT_DECODE_IMPL, OPT_SHARE_TILES, OPT_FP8_RESIDENT, OPT_IO_TIMEOUT_MS, OPT_IO_TEST_DELAY_MS, OPT_CLUSTER_DECODE = 6, 7, 8, 9, 10, 11
+OPT_DECODE_IMPL, OPT_SHARE_TILES, OPT_FP8_RESIDENT, OPT_IO_TIMEOUT_MS, OPT_IO_TEST_DELAY_MS, OPT_CLUSTER_DECODE, OPT_CLUSTER_MAX = 6, 7, 8, 9, 10, 11, 12
 
 EXPORTS = [
     "matkv_create", "matkv_destroy", "matkv_last_error", "matkv_set_option", "matkv_workspace_bytes",

@@ -71,16 +71,27 @@ struct ClusterParams {
 
 #ifdef MATKV_STAMPS
 // Timeline stamps of a profiling build (never compiled into the library proper): [layer][CTA][point], nanoseconds.
-__device__ unsigned long long g_cl_stamps[64][160][12];
+__device__ unsigned long long g_cl_stamps[64][160][16];
+__device__ long long g_cl_clk[64][160][16];   // the same points in SM clock cycles (finer than the global timer)
 __device__ __forceinline__ void cl_stamp(int layer, int point) {
+#ifdef MATKV_STAMPS_CLOCK_ONLY   // reading the global timer costs hundreds of cycles: leave it out when phases are measured in cycles
+    if (layer < 64 && blockIdx.x < 160) g_cl_clk[layer][blockIdx.x][point] = clock64();
+#else
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    if (layer < 64 && blockIdx.x < 160) g_cl_stamps[layer][blockIdx.x][point] = t;
+    if (layer < 64 && blockIdx.x < 160) {
+        g_cl_stamps[layer][blockIdx.x][point] = t;
+        g_cl_clk[layer][blockIdx.x][point] = clock64();
+    }
+#endif
 }
 #define CL_STAMP(point) cl_stamp(p.layer, point)
 // per-tile stamps: [layer][CTA][kind: 0 issued, 1 seen landed, 2 consumed][tile]
 __device__ unsigned long long g_cl_tiles[64][160][3][8];
 __device__ __forceinline__ void cl_tile_stamp(int layer, int kind, int tile) {
+#ifdef MATKV_STAMPS_CLOCK_ONLY
+    return;
+#endif
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     if (layer < 64 && blockIdx.x < 160 && tile < 8) g_cl_tiles[layer][blockIdx.x][kind][tile] = t;
@@ -132,7 +143,7 @@ struct ClShare {
 };
 __device__ __forceinline__ ClShare cl_share(int32_t ct, int32_t tt_nom, int32_t cs, int32_t rank, int32_t tt_real) {
     const int32_t total = ct + tt_nom + 1;
-    const int32_t lo = (int32_t)((int64_t)rank * total / cs), hi = (int32_t)((int64_t)(rank + 1) * total / cs);
+    const int32_t lo = rank * total / cs, hi = (rank + 1) * total / cs;   // (a request lists at most 2^20 chunk tiles here)
     ClShare s;
     s.c0 = min(lo, ct);
     s.n_chunk = min(hi, ct) - s.c0;
@@ -311,25 +322,27 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
     // 2 qc + 1 (accumulator) or tq (B operand of S^T); as accumulator rows it has tokens (or dimensions) tq and tq + 8.
     const int tq = lane >> 2, qc = lane & 3;
     const int mi = lane >> 3, ri = lane & 7;   // ldmatrix addressing
-    CL_GDC_WAIT();   // q, the tail length and the tail rows come from earlier kernels
-    if (tid == 0) CL_STAMP(3);
-    // The chunk part of the share is known from the launch parameters; how many tail tiles follow depends on the device's
-    // tail length, which is requested now and first looked at when the chunk tiles are done (a dependent load less in
-    // front of the first tile).
-    const int32_t t0_dev = p.tail_len[b];
-    int32_t t0 = 0;
+    // Everything that does not depend on the predecessor kernel comes before the wait for it: what follows the wait is
+    // the launch's critical path.  The chunk part of the share is known from the launch parameters; how many tail tiles
+    // follow depends on the device's tail length, which is requested right after the wait and first looked at when the
+    // chunk tiles are done (a dependent load less in front of the first tile).
     int n_mine = cl_share(ct, p.tt_nom, cs, rank, 0).n_chunk;
     bool tail_known = false;
+    int32_t t0 = 0;
+    const bool real = tq < n_rows;
+    const __nv_bfloat16 *qrow = p.q + (int64_t)b * p.q_sb + (int64_t)(g * G + (real ? tq : 0)) * D + 2 * qc;
+    const int32_t *tail_len_b = p.tail_len + b;
+    CL_GDC_WAIT();   // q, the tail length and the tail rows come from earlier kernels
+    if (tid == 0) CL_STAMP(3);
+    const int32_t t0_dev = *tail_len_b;
 
     // Q^T as the B operand of S^T = K Q^T: column n = tq is query row tq, k = the 16 dimensions of a k-step
     uint32_t qb[C::KS][2];
     {
-        const bool real = tq < n_rows;
-        const __nv_bfloat16 *qrow = p.q + (int64_t)b * p.q_sb + (int64_t)(g * G + (real ? tq : 0)) * D;
 #pragma unroll
         for (int ks = 0; ks < C::KS; ++ks) {
-            qb[ks][0] = real ? *(const uint32_t *)(qrow + ks * 16 + 2 * qc) : 0u;
-            qb[ks][1] = real ? *(const uint32_t *)(qrow + ks * 16 + 8 + 2 * qc) : 0u;
+            qb[ks][0] = real ? *(const uint32_t *)(qrow + ks * 16) : 0u;
+            qb[ks][1] = real ? *(const uint32_t *)(qrow + ks * 16 + 8) : 0u;
         }
     }
     // O^T accumulators: [16-dimension block][c0: (d = tq, row 2 qc), c1: (tq, 2 qc + 1), c2: (tq + 8, 2 qc), c3: (tq + 8, 2 qc + 1)]
@@ -517,8 +530,9 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
     // ---- this CTA's columns: merge over the CS parts by log-sum-exp ----
     // every thread that takes part in the merge waits for the neighbours' parts itself (bounded)
     const int ng = (D / 4 - rank + cs - 1) / cs;   // column groups this CTA owns: rank, rank + cs, ...
-    const int n_items = n_rows * ng;               // one (row, group of four columns) unit per thread
-    if (tid < n_items || tid == 0) {
+    const int n_items = n_rows * ng;               // (row, group of four columns) units; TP threads share one: each takes every
+    const int tp = cs >= 4 ? 4 : 2;                // TP-th part, then the TP partial sums meet by shuffle (few threads, short chains)
+    if (tid < 32 * ceil_div(n_items * tp, 32)) {   // whole warps, for the shuffles
         bool got = mbar_try_wait_acquire_cluster(land_u32, 0);
         const long long tw = clock64();
         while (!got) {
@@ -526,36 +540,47 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
             if (!got && clock64() - tw > 2 * kWaitCycles) break;
         }
         if (tid == 0) CL_STAMP(8);
+        got = __all_sync(0xffffffffu, got);
         if (!got) {
             if (tid == 0) atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
-        } else if (tid < n_items) {
-            const int r = tid / ng, li = tid % ng;
-            // the parts' weights w = exp(lse_part - lse_row), formed by every thread for its row (independent loads)
-            float lc[kClMaxCs];
+        } else {
+            const int item = tid / tp, sub = tid % tp;
+            const bool valid = item < n_items;
+            const int r = valid ? item / ng : 0, li = valid ? item % ng : 0;
+            // the row's maximum over all parts (independent loads), then this thread's parts with their weights exp(lse_part - max)
             float M = -CUDART_INF_F;
 #pragma unroll
-            for (int c = 0; c < kClMaxCs; ++c) {
-                lc[c] = c < cs ? land_lse[c * n_rows + r] : -CUDART_INF_F;
-                M = fmaxf(M, lc[c]);
-            }
+            for (int c = 0; c < kClMaxCs; ++c)
+                if (c < cs) M = fmaxf(M, land_lse[c * n_rows + r]);
+            if (tid == 0) CL_STAMP(12);
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             float Z = 0.f;
-            if (M != -CUDART_INF_F) {
 #pragma unroll
-                for (int c = 0; c < kClMaxCs; ++c) {
-                    if (c < cs && lc[c] != -CUDART_INF_F) {   // an empty part carries no weight, whatever its row holds
-                        const float wgt = fast_exp2((lc[c] - M) * kLog2e);
+            for (int k = 0; k < kClMaxCs / 2; ++k) {
+                const int c = sub + k * tp;
+                if (c < cs) {
+                    const float lc = land_lse[c * n_rows + r];
+                    if (lc != -CUDART_INF_F) {   // an empty part carries no weight, whatever its row holds
+                        const float wgt = fast_exp2((lc - M) * kLog2e);
                         const float4 v = *(const float4 *)(land_o + ((c * n_rows + r) * ngm + li) * 4);
                         acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y); acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
                         Z += wgt;
                     }
                 }
-                const float inv = 1.f / Z;
-                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
             }
-            const int d = (li * cs + rank) * 4;
-            *(uint2 *)(p.out + (int64_t)b * p.q_sb + (int64_t)(g * G + r) * D + d) = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-            if (li == 0 && rank == 0 && p.lse_out) p.lse_out[(int64_t)b * p.lse_sb + g * G + r] = Z > 0.f ? M + logf(Z) : -CUDART_INF_F;
+            for (int off = 1; off < tp; off <<= 1) {
+                acc.x += __shfl_xor_sync(0xffffffffu, acc.x, off); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, off);
+                acc.z += __shfl_xor_sync(0xffffffffu, acc.z, off); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, off);
+                Z += __shfl_xor_sync(0xffffffffu, Z, off);
+            }
+            if (tid == 0) CL_STAMP(13);
+            if (valid && sub == 0) {
+                const float inv = Z > 0.f ? __frcp_rn(Z) : 0.f;
+                const int d = (li * cs + rank) * 4;
+                *(uint2 *)(p.out + (int64_t)b * p.q_sb + (int64_t)(g * G + r) * D + d) =
+                    make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+                if (li == 0 && rank == 0 && p.lse_out) p.lse_out[(int64_t)b * p.lse_sb + g * G + r] = Z > 0.f ? M + logf(Z) : -CUDART_INF_F;
+            }
         }
     }
     if (tid == 0) CL_STAMP(9);
@@ -641,6 +666,7 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
     if (W >= 96 * grid_max) return MATKV_OK;   // long launches stream best through the persistent kernel
     // cluster size: as many CTAs per unit as the SMs allow (any size up to 16, not only powers of two)
     int cs = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kClMaxCs, grid_max / n_units), std::min<int64_t>(min_tiles, c.head_dim / 4)));
+    if (ctx->opt_cluster_max > 0) cs = std::min<int>(cs, (int)ctx->opt_cluster_max);
     // Which kernel is faster was measured (8B and 70B head shapes, 5 x 1,024-token chunks per request, B = 1 .. 18,
     // launches replayed from a graph) and follows a simple model: the streaming kernel takes about 8 us plus 4.95 ns
     // per tile of the launch (all SMs stream, but a launch cannot start beside its predecessor), this kernel about
@@ -688,6 +714,9 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
 #ifdef MATKV_STAMPS
 extern "C" int matkv_debug_cluster_stamps(unsigned long long *host_out) {
     return (int)cudaMemcpyFromSymbol(host_out, matkv::g_cl_stamps, sizeof(matkv::g_cl_stamps));
+}
+extern "C" int matkv_debug_cluster_clk(long long *host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, matkv::g_cl_clk, sizeof(matkv::g_cl_clk));
 }
 extern "C" int matkv_debug_cluster_tiles(unsigned long long *host_out) {
     return (int)cudaMemcpyFromSymbol(host_out, matkv::g_cl_tiles, sizeof(matkv::g_cl_tiles));

@@ -309,6 +309,10 @@ int matkv_set_option(matkv_ctx *ctx, int32_t option, int64_t value) {
             if (value < 0 || value > 2) return fail(MATKV_E_INVALID_ARG, "cluster decode must be 0, 1 or 2");
             ctx->opt_cluster_decode = value;
             return MATKV_OK;
+        case MATKV_OPT_CLUSTER_MAX:
+            if (value < 0 || value > 16) return fail(MATKV_E_INVALID_ARG, "largest cluster must be 0 (automatic) .. 16");
+            ctx->opt_cluster_max = value;
+            return MATKV_OK;
         case MATKV_OPT_PREFILL_CTAS:
             if (value < 0 || value > 64) return fail(MATKV_E_INVALID_ARG, "prefill CTAs per head must be 0..64");
             ctx->opt_prefill_ctas = value;

@@ -132,7 +132,7 @@ struct matkv_ctx {
     std::vector<uint64_t> failed_tickets;                  // retired tickets whose storage reads failed
     uint64_t next_ticket = 1;
     int64_t opt_io_timeout_ms = 30000, opt_io_test_delay_ms = 0;
-    int64_t opt_cluster_decode = 1;
+    int64_t opt_cluster_decode = 1, opt_cluster_max = 0;
     std::vector<matkv_table *> tables;
     matkv::IoEngine *io = nullptr;
     std::vector<matkv::PooledImage> image_pool;
