@@ -263,6 +263,7 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
 
     // ================= consumers =================
     const int qr = lane >> 2, qc = lane & 3;   // mma rows qr and qr + 8, column pair qc
+    const int tq = qr;                         // transposed items: accumulator rows (tokens, then dimensions) tq and tq + 8
     const int mi = lane >> 3, ri = lane & 7;   // ldmatrix addressing
 
     uint32_t qa[C::KS][4];   // A fragments of Q: rows qr / qr+8, k columns 0-7 / 8-15 of every k-step
@@ -291,6 +292,17 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
     auto load_q = [&](const volatile QEntry *e) {
         const int n_rows = e->n_req * G;
         const int64_t base = (int64_t)e->l_rel * p.q_sl + (int64_t)e->g * G * D;
+        if (n_rows <= 8) {
+            // transposed item (see the piece loop): Q^T as the B operand, column tq = query row tq
+            const bool real = tq < n_rows;
+            const __nv_bfloat16 *qrow = p.q + base + (int64_t)(real ? e->req[tq / G] : 0) * p.q_sb + (tq % G) * D;
+#pragma unroll
+            for (int ks = 0; ks < C::KS; ++ks) {
+                qa[ks][0] = real ? *(const uint32_t *)(qrow + ks * 16 + 2 * qc) : 0u;
+                qa[ks][1] = real ? *(const uint32_t *)(qrow + ks * 16 + 8 + 2 * qc) : 0u;
+            }
+            return;
+        }
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             const int r = qr + 8 * hh;
@@ -349,6 +361,7 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
         const int layer = p.layer0 + l_rel;
         const int lg = l_rel * p.Hkv + g;
         const int n_rows = n_req * G;
+        const bool tr = n_rows <= 8;   // the transposed form (see the piece loop)
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             m_run[hh] = -CUDART_INF_F;
@@ -368,7 +381,58 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
             const uint32_t tag = stage_wait(tags + stage, use, full_u32 + stage * 8, use & 1, flags);
             const uint32_t stage_u32 = ring_u32 + stage * C::STAGE_BYTES;
             const int vis = (int)(tag & 0x7f) - r0;   // valid tokens of this piece (may be <= 0)
-            if (vis > 0) {
+            if (vis > 0 && tr) {
+                // ---------- an item of at most 8 query rows: the products transposed, S^T = K Q^T and O^T += V^T P^T (tokens,
+                // then head dimensions, on the 16-row axis of the MMA, the query rows on its 8-column axis): half the MMAs of
+                // the stacked form, whose rows 8..15 would be padding here.  o[0 .. KS-1], m_run, l_run, lr[0 .. 1] hold the state. ----------
+                float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int ks = 0; ks < C::KS; ++ks) {
+                    // A = K rows, fragments a0..a3: (tokens 0-7, d-chunk 2ks), (tokens 8-15, 2ks), (tokens 0-7, 2ks+1), (tokens 8-15, 2ks+1)
+                    uint32_t ka[4];
+                    ldsm_x4(stage_u32 + (ks / 4) * C::BOX_BYTES + swz(r0 + (mi & 1) * 8 + ri, (ks * 2 + (mi >> 1)) & 7), ka);
+                    if (ks & 1) mma_bf16(sb, ka[0], ka[1], ka[2], ka[3], qa[ks][0], qa[ks][1]);
+                    else mma_bf16(sa, ka[0], ka[1], ka[2], ka[3], qa[ks][0], qa[ks][1]);
+                }
+                // this thread: tokens tq (x0, x1) and tq + 8 (x2, x3) against query rows 2 qc (x0, x2) and 2 qc + 1 (x1, x3)
+                const float x0 = tq < vis ? (sa[0] + sb[0]) * p.scale_log2 : -CUDART_INF_F;
+                const float x1 = tq < vis ? (sa[1] + sb[1]) * p.scale_log2 : -CUDART_INF_F;
+                const float x2 = tq + 8 < vis ? (sa[2] + sb[2]) * p.scale_log2 : -CUDART_INF_F;
+                const float x3 = tq + 8 < vis ? (sa[3] + sb[3]) * p.scale_log2 : -CUDART_INF_F;
+                float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {   // over the eight token pairs of the piece (lanes with the same qc)
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+                }
+                const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);   // finite: token 0 of the piece is valid
+                const float al0 = fast_exp2(m_run[0] - mn0), al1 = fast_exp2(m_run[1] - mn1);
+                const float p0 = fast_exp2(x0 - mn0), p1 = fast_exp2(x1 - mn1), p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
+                const uint32_t w0 = pack_bf16(p0, p1), w1 = pack_bf16(p2, p3);   // (token tq | tq + 8; rows 2 qc, 2 qc + 1)
+                l_run[0] = l_run[0] * al0 + (p0 + p2);
+                l_run[1] = l_run[1] * al1 + (p1 + p3);
+                lr[0] = lr[0] * al0 + (bf_lo(w0) + bf_lo(w1));   // this thread's share of the rounded numerators' sums
+                lr[1] = lr[1] * al1 + (bf_hi(w0) + bf_hi(w1));
+                m_run[0] = mn0;
+                m_run[1] = mn1;
+                if (__any_sync(0xffffffffu, al0 != 1.0f || al1 != 1.0f)) {
+#pragma unroll
+                    for (int mt = 0; mt < C::KS; ++mt) {
+                        o[mt][0] *= al0; o[mt][1] *= al1; o[mt][2] *= al0; o[mt][3] *= al1;
+                    }
+                }
+                uint32_t pb0, pb1;   // P^T as the B operand: the 8 x 8 blocks (tokens x rows) transposed across the warp
+                asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pb0) : "r"(w0));
+                asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(pb1) : "r"(w1));
+                const uint32_t v_u32 = stage_u32 + C::NBOX * C::BOX_BYTES;
+#pragma unroll
+                for (int mt = 0; mt < C::KS; ++mt) {
+                    // A = V^T: (d-chunk 2mt, tokens 0-7), (2mt+1, tokens 0-7), (2mt, tokens 8-15), (2mt+1, tokens 8-15), transposed on the way
+                    uint32_t va[4];
+                    ldsm_x4_trans(v_u32 + (mt / 4) * C::BOX_BYTES + swz(r0 + (mi >> 1) * 8 + ri, (mt * 2 + (mi & 1)) & 7), va);
+                    mma_bf16(o[mt], va[0], va[1], va[2], va[3], pb0, pb1);
+                }
+            } else if (vis > 0) {
                 // ---------- S = Q K^T for 16 tokens ----------
                 float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -422,6 +486,8 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
                     mma_bf16(o[2 * dp], pa[0], pa[1], pa[2], pa[3], vb[0], vb[1]);
                     mma_bf16(o[2 * dp + 1], pa[0], pa[1], pa[2], pa[3], vb[2], vb[3]);
                 }
+            }
+            if (vis > 0) {
                 // ---------- the new token goes to the request's tail for later steps ----------
                 if ((tag & kTagNew) && r0 == 0 && t0 < p.max_tail) {
                     constexpr int CPR = D / 8;  // 16-byte chunks per row; lanes 0..CPR-1 move K, the next CPR lanes move V
@@ -446,25 +512,35 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
         // The seven warps' states are merged through shared memory.  First the running maxima: once every thread
         // knows its rows' overall maximum it scales its own accumulators while it writes them, so that the reduction
         // itself is a plain sum (no exponentials, no per-warp weights).
-        if (qc == 0) {
-            merge_m[warp * kShareRows + qr] = m_run[0];
-            merge_m[warp * kShareRows + qr + 8] = m_run[1];
+        // (stacked items: this thread's rows are qr and qr + 8, a row's tokens sit in the four lanes of a quad; transposed
+        // items: rows 2 qc and 2 qc + 1, a row's tokens sit in the eight lanes that share qc)
+        if (tr ? tq == 0 : qc == 0) {
+            merge_m[warp * kShareRows + (tr ? 2 * qc : qr)] = m_run[0];
+            merge_m[warp * kShareRows + (tr ? 2 * qc + 1 : qr + 8)] = m_run[1];
         }
         consumer_bar();
         float sw[2];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
-            const int r = qr + 8 * hh;
+            const int r = tr ? 2 * qc + hh : qr + 8 * hh;
             float M = merge_m[r];
 #pragma unroll
             for (int w = 1; w < kCW; ++w) M = fmaxf(M, merge_m[w * kShareRows + r]);
             sw[hh] = m_run[hh] == -CUDART_INF_F ? 0.f : fast_exp2(m_run[hh] - M);   // a warp without pieces of this item: weight 0
-            float l_tot = l_run[hh];
-            l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
-            l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
-            if (qc == 0) {
+            float l_tot = l_run[hh], r_tot = tr ? lr[hh] : lr[2 * hh];
+            if (tr) {
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {
+                    l_tot += __shfl_xor_sync(0xffffffffu, l_tot, off);
+                    r_tot += __shfl_xor_sync(0xffffffffu, r_tot, off);
+                }
+            } else {
+                l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 1);
+                l_tot += __shfl_xor_sync(0xffffffffu, l_tot, 2);
+            }
+            if (tr ? tq == 0 : qc == 0) {
                 merge_l[warp * kShareRows + r] = l_tot * sw[hh];
-                merge_r[warp * kShareRows + r] = lr[2 * hh] * sw[hh];
+                merge_r[warp * kShareRows + r] = r_tot * sw[hh];
                 if (warp == 0) row_max[r] = M;
             }
         }
@@ -472,12 +548,24 @@ k_attend_shared(const __grid_constant__ SharedParams p, const __grid_constant__ 
 #pragma unroll
         for (int half = 0; half < D / 64; ++half) {
             if (half) consumer_bar();  // the previous half has been read
+            if (tr) {   // O^T accumulators: [16-dimension block][(d = tq, row 2 qc), (tq, 2 qc + 1), (tq + 8, 2 qc), (tq + 8, 2 qc + 1)]
 #pragma unroll
-            for (int nb = 0; nb < 8; ++nb) {
-                *(float2 *)(merge_o + (warp * kShareRows + qr) * 64 + nb * 8 + 2 * qc) =
-                    make_float2(o[half * 8 + nb][0] * sw[0], o[half * 8 + nb][1] * sw[0]);
-                *(float2 *)(merge_o + (warp * kShareRows + qr + 8) * 64 + nb * 8 + 2 * qc) =
-                    make_float2(o[half * 8 + nb][2] * sw[1], o[half * 8 + nb][3] * sw[1]);
+                for (int m4 = 0; m4 < 4; ++m4) {
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        float *row = merge_o + (warp * kShareRows + 2 * qc + hh) * 64 + m4 * 16 + tq;
+                        row[0] = o[half * 4 + m4][hh] * sw[hh];
+                        row[8] = o[half * 4 + m4][2 + hh] * sw[hh];
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int nb = 0; nb < 8; ++nb) {
+                    *(float2 *)(merge_o + (warp * kShareRows + qr) * 64 + nb * 8 + 2 * qc) =
+                        make_float2(o[half * 8 + nb][0] * sw[0], o[half * 8 + nb][1] * sw[0]);
+                    *(float2 *)(merge_o + (warp * kShareRows + qr + 8) * 64 + nb * 8 + 2 * qc) =
+                        make_float2(o[half * 8 + nb][2] * sw[1], o[half * 8 + nb][3] * sw[1]);
+                }
             }
             consumer_bar();
             if (half == 0) {
