@@ -20,8 +20,8 @@
 //     are merged through shared memory at the end;
 //   - the CTAs' partials (o, lse) are exchanged through distributed shared memory as a reduce-scatter: CTA i of the
 //     cluster owns the output column groups (of four) i, i + CS, ..., every CTA stores those groups of its partial straight into CTA i's
-//     shared memory (st.shared::cluster) and announces it on an mbarrier there (remote arrive, release at cluster
-//     scope); every CTA then merges its own slice over the CS parts by log-sum-exp and writes those columns of the
+//     shared memory (st.shared::cluster) and each storing thread announces its unit on an mbarrier there (remote arrive,
+//     release at cluster scope); every CTA then merges its own slice over the CS parts by log-sum-exp and writes those columns of the
 //     output.  No global partials, no device-wide fence, no atomic ticket, no workspace, and the landing zone of a
 //     CTA is a few kilobytes.
 // A CTA needs ~100 KB of shared memory (a ring of three 32 KB tiles) and few registers, so two launches' CTAs fit an SM
@@ -209,7 +209,9 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
             mbar_init(empty_u32 + s * 8, 4);   // the four warps that share a tile
             tags[s] = 0xffff0000u;
         }
-        mbar_init(land_u32, cs > 1 ? cs - 1 : 1);
+        // the landing barrier counts one arrival per (row, column group) unit this CTA owns from every CTA of the cluster
+        // (its own included): every thread that stores a unit announces it itself, no CTA-wide step in between
+        mbar_init(land_u32, cs > 1 ? cs * G * ((D / 4 - rank + cs - 1) / cs) : 1);
         flags[0] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -477,7 +479,8 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
     const bool aborted = flags[0] != 0;
     if (aborted && tid == 0) atomicCAS(p.status, 0, MATKV_E_TIMEOUT);
     if (tid == 0) CL_STAMP(10);
-    if (cs > 1) cluster_wait_acquire();   // the start-up barrier: every neighbour's landing zone and barrier exist from here on
+    if (cs > 1) cluster_wait_acquire();
+   // the start-up barrier: every neighbour's landing zone and barrier exist from here on
     if (tid == 0) CL_STAMP(11);
     // one (row, group of four columns) unit per thread and pass; column group q belongs to CTA q mod cs of the cluster (any
     // cluster size works), which keeps it as group q / cs of its landing zone
@@ -510,25 +513,19 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
         // these four columns belong to CTA `dst`: into part `rank` of its landing zone (its own groups stay local)
         const int dst = (d / 4) % cs;
         const uint32_t off = (uint32_t)(((rank * n_rows + r) * ngm + (d / 4) / cs) * 16);
-        if (dst == rank) *(float4 *)((unsigned char *)land_o + off) = acc;
-        else if (!aborted) st_cluster_f4(map_to_rank(land_o_u32, dst) + off, acc);
-        if (d == 0) land_lse[rank * n_rows + r] = lse;   // (sent to the neighbours below)
+        // (the unit's row lse travels with it: the owner gets it once per unit of that row, always the same value).  Then the
+        // unit is announced on the owner's landing barrier, after a timeout too (nobody must wait for this CTA): the release
+        // orders this thread's stores before the arrival, which is all the owner's acquire needs.
+        if (!aborted) {
+            st_cluster_f4(map_to_rank(land_o_u32, dst) + off, acc);   // (the own rank maps to this CTA's own memory)
+            st_cluster_f1(map_to_rank(land_lse_u32, dst) + (uint32_t)((rank * n_rows + r) * 4), lse);
+        }
+        mbar_arrive_remote_release(map_to_rank(land_u32, dst));
     }
     if (cs == 1) return;
-    asm volatile("bar.sync 1, %0;" ::"n"(kClWarps * 32) : "memory");   // every thread's stores have been issued
     if (tid == 0) CL_STAMP(7);
-    // Announce this CTA's part to every neighbour (after a timeout too: nobody must wait for it).  The release makes the
-    // stores of the whole CTA, ordered before it by the barrier above, visible to the neighbour's acquire.
-    // Thread c sends the rows' lse to CTA c first.
-    if (tid < cs && tid != rank) {
-        if (!aborted) {
-            const uint32_t dst_lse = map_to_rank(land_lse_u32, tid) + (uint32_t)(rank * n_rows * 4);
-            for (int r = 0; r < n_rows; ++r) st_cluster_f1(dst_lse + r * 4, land_lse[rank * n_rows + r]);
-        }
-        mbar_arrive_remote_release(map_to_rank(land_u32, tid));
-    }
     // ---- this CTA's columns: merge over the CS parts by log-sum-exp ----
-    // every thread that takes part in the merge waits for the neighbours' parts itself (bounded)
+    // every thread that takes part in the merge waits for all parts itself (bounded)
     const int ng = (D / 4 - rank + cs - 1) / cs;   // column groups this CTA owns: rank, rank + cs, ...
     const int n_items = n_rows * ng;               // (row, group of four columns) units; TP threads share one: each takes every
     const int tp = cs >= 4 ? 4 : 2;                // TP-th part, then the TP partial sums meet by shuffle (few threads, short chains)
