@@ -104,15 +104,15 @@ typedef struct {
                                       block per CTA); the chunk-major decode, the cluster decode (such launches take the streaming
                                       kernel), the allocation-free decode and matkv_gather_debug do not read tables that hold them */
 #define MATKV_OPT_PREFILL_CTAS  3  /* CTAs per (request, KV head) the tensor-core prefill splits the KV over; 0 = auto */
-#define MATKV_OPT_CLUSTER_DECODE 11 /* matkv_attend_decode (one layer per launch) of small and medium batches, where a launch is short
-                                      enough for its fixed latencies to matter: 1 (default) = served by thread-block clusters, one
-                                      cluster of up to 16 CTAs per (request, KV head), whose CTAs merge their partials through
-                                      distributed shared memory (no workspace traffic) and fetch their first chunk tiles under the
-                                      previous kernel's tail, whenever a measured cost model says this is the faster kernel; 0 =
-                                      always the streaming kernel; 2 = clusters even when MATKV_OPT_DECODE_IMPL is 1.  Long launches
-                                      use the streaming kernel either way.  A captured (graph) launch balances its shares for the tail
-                                      length at capture time and stays exact as the tail grows; re-capture now and then in a long
-                                      generation to keep the balance */
+#define MATKV_OPT_CLUSTER_DECODE 11 /* matkv_attend_decode (one layer per launch): 1 (default) = served by thread-block clusters, one
+                                      cluster of up to 16 CTAs per (request, KV head), two CTAs per SM, whose CTAs merge their partials
+                                      through distributed shared memory (no workspace traffic) and fetch their first chunk tiles under
+                                      the previous kernel's tail; measured 5 - 25 % faster than the streaming kernel for launches of
+                                      1 to 64 requests; 0 = always the streaming kernel; 2 = clusters even when MATKV_OPT_DECODE_IMPL
+                                      is 1.  Launches it cannot spread over enough CTAs, tables with compressed-resident chunks and
+                                      all-layers launches use the streaming kernel.  A captured (graph) launch balances its shares for
+                                      the tail length at capture time and stays exact as the tail grows; re-capture now and then in a
+                                      long generation to keep the balance */
 #define MATKV_OPT_CLUSTER_MAX 12   /* largest cluster (CTAs per request and KV head) the cluster decode may use; 0 (default) = automatic */
 #define MATKV_OPT_IO_TIMEOUT_MS 9  /* storage tier: how long the copy stream waits for one chunk's read before the staging call
                                       is marked failed (MATKV_E_IO) and the stream moves on; default 30,000 ms */

@@ -36,7 +36,7 @@
 
 namespace matkv {
 
-constexpr int kClMaxReq = 32;      // requests per launch the parameter block has room for
+constexpr int kClMaxReq = 64;      // requests per launch the parameter block has room for
 constexpr int kClWarps = 8;        // consumer warps: warp w takes tokens [16 (w & 3), 16 (w & 3) + 16) of the tiles of parity w >> 2
 constexpr int kClThreads = (kClWarps + 1) * 32;
 constexpr int kClStages = 3;
@@ -584,9 +584,45 @@ k_decode_cluster(const __grid_constant__ ClusterParams p, const __grid_constant_
 }
 
 // ---- launcher ---------------------------------------------------------------------------------------
+// How many clusters of `cs` CTAs of this kernel the device can hold at once (asked once per size and device; -1: cannot say).
 template <int D, int G>
-static int launch_cluster_t(const ClusterParams &p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int n_units, cudaStream_t stream,
-                            bool *fits) {
+static int max_active_clusters(int cs) {
+    using C = ClusterCfg<D, G>;
+    static std::atomic<int> cache[64][kClMaxCs + 1] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    int known = cache[dev][cs].load(std::memory_order_acquire);
+    if (known == 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)cs);
+        cfg.blockDim = dim3((unsigned)kClThreads);
+        cfg.dynamicSmemBytes = C::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, k_decode_cluster<D, G>, &cfg) != cudaSuccess) {
+            cudaGetLastError();
+            n = -1;
+        }
+        known = n > 0 ? n : -1;
+        cache[dev][cs].store(known, std::memory_order_release);
+#ifdef MATKV_STAMPS
+        fprintf(stderr, "[cluster decode] cluster size %d: %d clusters can be active at once, %d bytes of shared memory per CTA\n", cs, n, C::SMEM_BYTES);
+#endif
+    }
+    return known;
+}
+
+// Picks the cluster size (the largest up to cs_max whose clusters can all be resident at once and whose CTAs stay within
+// `cta_limit`), and launches; *fits = false when no size will do.
+template <int D, int G>
+static int launch_cluster_t(ClusterParams p, const CUtensorMap &kn_map, const CUtensorMap &vn_map, int n_units, int cs_max, int64_t cta_limit,
+                            int64_t cta_limit_pairs, cudaStream_t stream, bool *fits) {
     using C = ClusterCfg<D, G>;
     static PerDeviceOnce configured;
     int once_dev;
@@ -595,8 +631,19 @@ static int launch_cluster_t(const ClusterParams &p, const CUtensorMap &kn_map, c
         MATKV_CUDA(cudaFuncSetAttribute(k_decode_cluster<D, G>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1));
         configured.mark(once_dev);
     }
+    int cs = 0;
+    for (int c = cs_max; c >= 1; --c) {
+        if ((int64_t)n_units * c > (c <= 2 ? cta_limit_pairs : cta_limit)) continue;
+        if (max_active_clusters<D, G>(c) >= n_units) {
+            cs = c;
+            break;
+        }
+    }
+    *fits = cs > 0;
+    if (!cs) return MATKV_OK;
+    p.cs = cs;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(n_units * p.cs));
+    cfg.gridDim = dim3((unsigned)(n_units * cs));
     cfg.blockDim = dim3((unsigned)kClThreads);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = stream;
@@ -604,40 +651,11 @@ static int launch_cluster_t(const ClusterParams &p, const CUtensorMap &kn_map, c
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = (unsigned)p.cs;
+    attr[1].val.clusterDim.x = (unsigned)cs;
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    // every cluster of the launch must be able to run at once (one wave): asked once per cluster size and device
-    static std::atomic<int> max_clusters[64][kClMaxCs + 1] = {};
-    int dev = 0;
-    const int slot = p.cs;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64) {
-        int known = max_clusters[dev][slot].load(std::memory_order_acquire);
-        if (known == 0) {
-            int n = 0;
-            cudaError_t e = cudaOccupancyMaxActiveClusters(&n, k_decode_cluster<D, G>, &cfg);
-            if (e != cudaSuccess) {
-                cudaGetLastError();
-                n = -1;
-            }
-            known = n > 0 ? n : -1;
-            max_clusters[dev][slot].store(known, std::memory_order_release);
-#ifdef MATKV_STAMPS
-            int per_sm = 0;
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_decode_cluster<D, G>, kClThreads, C::SMEM_BYTES);
-            fprintf(stderr, "[cluster decode] cluster size %d: %d clusters can be active at once, %d CTAs per SM, %d bytes of shared memory per CTA\n",
-                    p.cs, n, per_sm, C::SMEM_BYTES);
-#endif
-        }
-        if (known < n_units) {
-            *fits = false;
-            return MATKV_OK;
-        }
-    }
-    *fits = true;
     MATKV_CUDA(cudaLaunchKernelEx(&cfg, k_decode_cluster<D, G>, p, kn_map, vn_map));
     return MATKV_OK;
 }
@@ -652,7 +670,12 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
     if (a.S != 1 || a.n_layers_launch != 1 || a.advance != 0 || t->has_fp8 || t->batch > kClMaxReq || !t->d_tile_dir || ctx->opt_decode_ctas > 0) return MATKV_OK;
     const int n_units = t->batch * c.n_kv_heads;
     const int64_t grid_max = std::max<int64_t>(ctx->n_sm - ctx->opt_stage_ctas, ctx->n_sm / 2);
-    if (n_units > grid_max) return MATKV_OK;
+    // Two CTAs of this kernel fit an SM.  A launch may take both places of every SM (it then cannot start beside its
+    // predecessor, but all the SMs' shared memory is prefetching for it); measured, launches of more than 0.9 x 2 x SMs CTAs in
+    // clusters of three or more do not become resident in one wave (B = 7 in clusters of 5, 280 CTAs: 36 us against 25.6 in
+    // clusters of 4), pairs and single CTAs do up to the full 2 x SMs.
+    const int64_t cta_limit = 2 * grid_max * 9 / 10, cta_limit_pairs = 2 * grid_max;
+    if (n_units > cta_limit_pairs) return MATKV_OK;
     const int tt_nom = ceil_div(t->tail_len_host, kTile);
     int64_t W = 0, min_tiles = 1 << 30;
     for (int b = 0; b < t->batch; ++b) {
@@ -660,20 +683,16 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
         W += (int64_t)c.n_kv_heads * tiles;
         min_tiles = std::min(min_tiles, tiles);
     }
-    if (W >= 96 * grid_max) return MATKV_OK;   // long launches stream best through the persistent kernel
     // cluster size: as many CTAs per unit as the SMs allow (any size up to 16, not only powers of two)
-    int cs = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kClMaxCs, grid_max / n_units), std::min<int64_t>(min_tiles, c.head_dim / 4)));
-    if (ctx->opt_cluster_max > 0) cs = std::min<int>(cs, (int)ctx->opt_cluster_max);
-    // Which kernel is faster was measured (8B and 70B head shapes, 5 x 1,024-token chunks per request, B = 1 .. 18,
-    // launches replayed from a graph) and follows a simple model: the streaming kernel takes about 8 us plus 4.95 ns
-    // per tile of the launch (all SMs stream, but a launch cannot start beside its predecessor), this kernel about
-    // 6 us plus 0.65 us per tile of a CTA's share.  Examples (us, this kernel / streaming): B = 1: 9.4 / 12.0,
-    // B = 3 (clusters of 6): 15.4 / 18.4, B = 6 (clusters of 3): 25.6 / 27.8, B = 9 (clusters of 2, 144 CTAs):
-    // 33.6 / 39.0, B = 10 (80 CTAs of one unit each): 53.1 / 41.5, B = 18 (144 CTAs): 61.2 / 65.0.
-    {
-        const double ctas = (double)n_units * cs;
-        if ((double)W * (0.65 / ctas - 0.00495) >= 2.0) return MATKV_OK;
-    }
+    int cs_max = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kClMaxCs, cta_limit_pairs / n_units), std::min<int64_t>(min_tiles, c.head_dim / 4)));
+    if (ctx->opt_cluster_max > 0) cs_max = std::min<int>(cs_max, (int)ctx->opt_cluster_max);
+    // Measured against the streaming kernel (8B and 70B head shapes, 5 / 10 / 40 chunks of 1,024 tokens per request, B = 1 .. 32,
+    // launches replayed from a graph; us per layer, this kernel / streaming): 5 chunks: B = 1 9.4 / 12.0, B = 2 12.3 / 15.6,
+    // B = 4 17.1 / 21.6, B = 8 28.4 / 35.6, B = 12 43.2 / 49.1, B = 16 52.9 / 59.6, B = 24 82 / 87, B = 32 102 / 110;
+    // 10 chunks: B = 4 28.6 / 35.4, B = 16 101 / 107, B = 32 198 / 202; 40 chunks, G = 8: B = 2 59 / 65, B = 8 194 / 202.
+    // It loses only where it cannot put enough CTAs to work: a launch with much work on few CTAs stays with the streaming
+    // kernel, whose flat split uses every SM (B = 1 over 40 chunks in clusters of 8: 49.7 against 43.7).
+    if ((int64_t)n_units * cs_max * 10 < grid_max * 6 && W >= 32 * grid_max) return MATKV_OK;
     ClusterParams p;
     p.tile_dir = t->d_tile_dir;
     p.tmaps = t->d_tmaps;
@@ -684,7 +703,7 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
     p.q = a.q; p.out = a.out; p.lse_out = a.lse_out;
     p.q_sb = a.q_sb; p.lse_sb = a.lse_sb;
     p.layer = a.layer0; p.n_layers_total = c.n_layers; p.B = t->batch; p.Hkv = c.n_kv_heads; p.max_tail = c.max_tail_tokens;
-    p.cs = cs;
+    p.cs = 0;   // (chosen by the launcher)
     p.tt_nom = tt_nom;
     p.scale_log2 = ctx->scale * kLog2e;
     p.status = ctx->d_status;
@@ -699,7 +718,7 @@ int launch_decode_cluster(matkv_ctx *ctx, matkv_table *t, const AttendArgs &a, c
     if (rc) return rc;
     rc = fail(MATKV_E_INVALID_ARG, "unsupported head_dim %d / group %d", c.head_dim, G);
 #define MATKV_CASE(DD, GG) \
-    if (c.head_dim == DD && G == GG) rc = launch_cluster_t<DD, GG>(p, kn_map, vn_map, n_units, stream, taken);
+    if (c.head_dim == DD && G == GG) rc = launch_cluster_t<DD, GG>(p, kn_map, vn_map, n_units, cs_max, cta_limit, cta_limit_pairs, stream, taken);
     MATKV_CASE(128, 1) MATKV_CASE(128, 2) MATKV_CASE(128, 4) MATKV_CASE(128, 8)
     MATKV_CASE(64, 1) MATKV_CASE(64, 2) MATKV_CASE(64, 4) MATKV_CASE(64, 8)
 #undef MATKV_CASE
