@@ -234,7 +234,9 @@ def test_back_to_back_decode_launches_across_a_tail_tile_boundary(decode_impl, L
     (8, 2, 64, [[128, 128]]),                          # D = 64
     (4, 4, 128, [[65, 1, 64], [], [7]]),               # G = 1; a request without chunks; shares without any tile
     (16, 2, 128, [[33]]),                              # fewer tiles than a full cluster
-    (8, 8, 64, [[500], [40, 40], [64], [1]]),          # 32 units: clusters of 4
+    (8, 8, 64, [[500], [40, 40], [64], [1]]),          # 32 units: clusters of up to 9
+    (8, 8, 64, [[70, 3]] * 33),                        # 264 units: one CTA each, both CTA places of every SM taken
+    (16, 4, 128, [[130], [64, 64], []] * 7),           # 84 units in clusters of 3, ragged requests, some without chunks
 ])
 def test_cluster_decode_matches_the_oracle(Hq, Hkv, D, lens):
     """decode_impl 1 + cluster 2 forces the cluster kernel wherever the launch fits it; the tail grows through a tile
