@@ -482,6 +482,7 @@ def parse_args(argv=None):
                     help="sub-prefill kernel: 0 auto, 1 streaming kernel, 2 tensor-core kernel, 3 the same with two row blocks per CTA")
     ap.add_argument("--decode-impl", type=int, default=0, choices=[0, 1, 2],
                     help="decode kernel: 0 auto (chunk-major when the batch's requests share chunks), 1 request-major, 2 chunk-major")
+    ap.add_argument("--share-tiles", type=int, default=0, help="chunk-major decode: 64-token tiles per work item (0 = the library's default)")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (small profiling cases)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (small profiling cases)")
     return ap.parse_args(argv)
@@ -604,6 +605,8 @@ def run_cuda_arm(args):
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_IMPL, args.decode_impl)
     if args.prefill_impl:
         mk.matkv_set_option(sess.ctx, mk.OPT_PREFILL_IMPL, args.prefill_impl)
+    if args.share_tiles:
+        mk.matkv_set_option(sess.ctx, mk.OPT_SHARE_TILES, args.share_tiles)
     fused_advance = args.decode_launch == "all_layers"
     if fused_advance:   # the all-layers decode launch moves the tail itself: no separate counter kernel per step
         mk.matkv_set_option(sess.ctx, mk.OPT_DECODE_ADVANCES_TAIL, 1)
